@@ -1,0 +1,207 @@
+/*
+ * taskkv.h -- C ABI of the Task-KV hot path for NVIDIA B200 (sm_100a).
+ *
+ * Task-KV (arXiv 2501.15113) compresses a transformer's KV cache per attention
+ * head after prefill and then decodes over the compacted, ragged cache:
+ *
+ *   prefill side (Sec. IV-A, IV-B)
+ *     window scores      C  = mean over the observation window's softmax rows   (Eq. 12, 13)
+ *     semantic vector    v' = sum over the top-t positions of C[j] V[j,:]       (Eq. 14, 15)
+ *     semantic separator center = mean of the layer's v' (Eq. 8), distance =
+ *                        L2 norm of the offset (Eq. 7), the f(r) farthest heads
+ *                        are heterogeneous (Eq. 16), the closest remaining head
+ *                        joins them                                             (Sec. IV-A)
+ *     allocation         heterogeneous heads keep every position; the others keep
+ *                        sinks + recent + the k middle positions of highest
+ *                        pooled score                                           (Sec. IV-B, V-D, Eq. 17)
+ *     gather             retained K/V rows copied into one segment per KV head
+ *   decode side
+ *     append             the new token's k, v join every head's segment
+ *     attention          softmax(q K^T / sqrt(d)) V over each head's segment    (Eq. 1)
+ *
+ * Every step runs in CUDA kernels; the library has no CPU fallback.  All calls
+ * return a status code and never throw or abort.  Unless stated otherwise a
+ * pointer is a DEVICE pointer, 16-byte aligned, and work is enqueued on the
+ * caller's stream without synchronising.  "Host" arrays are read before the
+ * call returns and may be freed afterwards.
+ *
+ * A "unit" is one (sequence b, layer r, KV head h); units are numbered
+ * u = (b * n_layers + r) * n_kv_heads + h.  With grouped-query attention the
+ * G = n_heads / n_kv_heads query heads a = h*G .. h*G+G-1 share unit h, and
+ * heads are classified per KV head (one semantic vector per KV head, from the
+ * mean of the group's G*L window rows).
+ */
+#ifndef TASKKV_H_
+#define TASKKV_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef int32_t taskkv_status;
+#define TASKKV_OK        0
+#define TASKKV_EINVAL   (-1)  /* bad argument; nothing was launched */
+#define TASKKV_EALLOC   (-2)  /* device or host allocation failed, or a caller buffer is too small */
+#define TASKKV_ECUDA    (-3)  /* a CUDA runtime call failed */
+#define TASKKV_ETIMEOUT (-4)  /* a bounded device-side wait ran out */
+#define TASKKV_ESTATE   (-5)  /* cache in a wrong state (e.g. append beyond capacity) */
+
+#define TASKKV_F32  0
+#define TASKKV_BF16 1
+
+#define TASKKV_CLASS_NON_HETERO 0
+#define TASKKV_CLASS_HETERO     1
+#define TASKKV_CLASS_CENTER     2   /* the head closest to the center, promoted to a full cache */
+
+#define TASKKV_MAX_TOP_T       1024
+#define TASKKV_MAX_KV_HEADS    64
+#define TASKKV_MAX_WINDOW_ROWS 128  /* G * window */
+
+typedef struct taskkv_cache taskkv_cache;   /* opaque; owns pools, lengths, indices, statistics */
+typedef void* taskkv_stream;                /* a cudaStream_t */
+
+/* Problem statement of Sec. IV.  Pointers inside are HOST arrays. */
+typedef struct taskkv_params {
+  int32_t n_layers;      /* R */
+  int32_t n_heads;       /* query heads n */
+  int32_t n_kv_heads;    /* n_kv; n_heads % n_kv_heads == 0, <= TASKKV_MAX_KV_HEADS */
+  int32_t head_dim;      /* d: 64 or 128 */
+  int32_t batch;         /* number of sequences */
+  int32_t sink;          /* s1: leading positions every head keeps (Sec. IV-B) */
+  int32_t recent;        /* s2: trailing positions every head keeps */
+  int32_t mid_budget;    /* k: middle activations per non-heterogeneous head (Eq. 17) */
+  int32_t window;        /* L: observation window (Eq. 12); G*L <= TASKKV_MAX_WINDOW_ROWS, L <= min N_b */
+  int32_t top_t;         /* t of Eq. 14 (256 in Sec. V-D); <= TASKKV_MAX_TOP_T */
+  int32_t pool_kernel;   /* average-pooling kernel of Sec. V-D (7), odd, <= 31; 1 = off */
+  int32_t m_top;         /* m of Eq. 16 */
+  float   beta;          /* beta of Eq. 16 */
+  int32_t promote_center;    /* 1: the closest remaining head also keeps a full cache (Sec. IV-A) */
+  int32_t force_class;       /* -1: run the separator; 1: every head heterogeneous; 0: none */
+  int32_t dtype;             /* TASKKV_F32 or TASKKV_BF16: element type of q, k, v, out and the pools */
+  int32_t max_new_tokens;    /* rows reserved per unit for taskkv_append */
+  int32_t reserved_;
+  const int32_t* seq_lens;   /* host [batch]: N_b (ragged batches allowed) */
+  const int32_t* mid_budget_per_layer;  /* host [n_layers] or NULL; overrides mid_budget */
+  const int32_t* n_hetero;   /* host [batch][n_layers] or NULL; overrides Eq. 16 */
+} taskkv_params;
+
+typedef struct taskkv_plan_info {
+  int64_t n_units;
+  int64_t pool_rows;         /* rows of K (and of V) in the compacted pools, reserve included */
+  int64_t retained_rows;     /* rows kept right after compression */
+  int64_t cache_bytes;       /* persistent device memory of one cache */
+  int64_t workspace_bytes;   /* device memory needed only while taskkv_compress_ex runs on the stream */
+  int64_t max_decode_items;  /* split-K work items of one decode call at full capacity */
+  int64_t gather_items;      /* row blocks the gather step copies */
+  int64_t index_stride;      /* ints per unit of the retained-index table */
+} taskkv_plan_info;
+
+/* Fills the defaults of Sec. V-D: top_t 256, pool_kernel 7, sink 16, recent 256,
+ * window 32, beta 0.25 / m 4, promote_center 1, force_class -1, dtype bf16. */
+void taskkv_params_default(taskkv_params* p);
+
+/* Host only.  Validates p and sizes every buffer.  The number of full-cache
+ * heads per layer is fixed by Eq. 16 (only WHICH heads is data dependent), so
+ * pool sizes are exact before any kernel runs. */
+taskkv_status taskkv_plan(const taskkv_params* p, taskkv_plan_info* out);
+
+/*
+ * Prefill-side compression of every layer of every sequence (Sec. IV-A, IV-B).
+ *   q_win[b]  device [n_layers][n_heads][L][d]      the last L query rows, Q[-L:,:] of Eq. 12
+ *   k[b],v[b] device [n_layers][n_kv_heads][N_b][d] post-RoPE keys / values as a model caches them
+ *   q_win, k, v themselves are host arrays of `batch` device pointers.
+ *   cache_mem / workspace_mem: device buffers of at least the planned sizes, 256-byte
+ *   aligned, owned by the caller; NULL lets the library allocate (cudaMalloc) and
+ *   own them.  The workspace may be released once the stream has passed this
+ *   call; the cache memory must outlive the cache.  K and V are copied, never
+ *   aliased: the caller may free them once the stream has passed this call.
+ * On success *out_cache holds the compacted cache: per unit a segment of
+ * retained rows in ascending position, its length, class, distance and
+ * semantic vector.  Errors: EINVAL (arguments), EALLOC, ECUDA.
+ */
+taskkv_status taskkv_compress_ex(const taskkv_params* p, const void* const* q_win,
+                                 const void* const* k, const void* const* v,
+                                 void* cache_mem, size_t cache_bytes,
+                                 void* workspace_mem, size_t workspace_bytes,
+                                 taskkv_stream stream, taskkv_cache** out_cache);
+
+/* The flat form of the same call: one bf16 sequence, Sec. V-D defaults for
+ * everything not listed, library-owned memory, max_new_tokens = 4096. */
+taskkv_status taskkv_compress(const void* q_win, const void* k, const void* v,
+                              int32_t n_layers, int32_t n_heads, int32_t n_kv_heads, int32_t head_dim,
+                              int32_t seq_len, int32_t sink, int32_t recent, int32_t mid_budget,
+                              int32_t window, taskkv_stream stream, taskkv_cache** out_cache);
+
+/* As taskkv_compress_ex, but q_win[b], k[b], v[b] are HOST buffers (pinned
+ * memory gives asynchronous copies).  Layers are staged through device
+ * buffers the library allocates, so the host-to-device copies are part of the
+ * call.  Cache memory is library-owned. */
+taskkv_status taskkv_compress_host(const taskkv_params* p, const void* const* q_win,
+                                   const void* const* k, const void* const* v,
+                                   taskkv_stream stream, taskkv_cache** out_cache);
+
+/* Decode-time growth: writes k_new, v_new [batch][n_layers][n_kv_heads][d] at
+ * row len_u of every unit and increments len_u.  A unit already at capacity is
+ * left unchanged and the cache's sticky status becomes ESTATE. */
+taskkv_status taskkv_append(taskkv_cache* c, const void* k_new, const void* v_new, taskkv_stream stream);
+
+/* Decode attention (Eq. 1, one query row per head, no mask) over the ragged
+ * cache: q, out [batch][n_layers][n_heads][d] in the cache's dtype, fp32
+ * accumulation.  lengths: device int32 [n_units] to attend over a prefix of
+ * each segment, or NULL for the cache's own lengths. */
+taskkv_status taskkv_decode(const void* q, taskkv_cache* c, const int32_t* lengths, void* out,
+                            taskkv_stream stream);
+
+/* One decode step with HOST buffers: copies q, k_new, v_new in, appends,
+ * attends and copies out back (k_new and v_new may both be NULL to skip the
+ * append).  Synchronises the stream before returning. */
+taskkv_status taskkv_decode_host(const void* q, const void* k_new, const void* v_new, taskkv_cache* c,
+                                 void* out, taskkv_stream stream);
+
+/* Synchronising device-to-host reads for tests and reports. */
+#define TASKKV_Q_LENGTHS   0   /* int32 [n_units] */
+#define TASKKV_Q_CLASSES   1   /* int32 [n_units] */
+#define TASKKV_Q_DIST      2   /* float [n_units]: distance to the layer's center */
+#define TASKKV_Q_SEMVEC    3   /* float [n_units][d]: semantic vectors v' */
+#define TASKKV_Q_OFFSETS   4   /* int64 [n_units+1]: first pool row of each segment */
+#define TASKKV_Q_INDICES   5   /* int32 [n_units][index_stride]: retained positions of class-0 units */
+#define TASKKV_Q_SCORES    6   /* float, units concatenated: C (valid while the workspace is intact) */
+#define TASKKV_Q_TOPT      7   /* int32 [n_units][top_t]: I of Eq. 14, ascending, -1 padded (workspace) */
+#define TASKKV_Q_STATUS    8   /* int32 [1]: sticky device status word */
+#define TASKKV_Q_KPOOL     9   /* raw K pool bytes */
+#define TASKKV_Q_VPOOL    10   /* raw V pool bytes */
+#define TASKKV_Q_CAPACITY 11   /* int32 [n_units] */
+int64_t       taskkv_cache_query_bytes(const taskkv_cache* c, int32_t what);
+taskkv_status taskkv_cache_query(const taskkv_cache* c, int32_t what, void* host_dst, size_t bytes);
+taskkv_status taskkv_cache_plan(const taskkv_cache* c, taskkv_plan_info* out);
+void          taskkv_cache_destroy(taskkv_cache* c);
+
+const char*   taskkv_status_str(taskkv_status s);
+
+/* Eq. 16, f(r) = n*beta - (n*beta - m)/(R-1)*r, rounded half up and clamped to
+ * [0, n]; a single layer gives n*beta.  Host only. */
+int32_t taskkv_hetero_count(int32_t n, float beta, int32_t m, int32_t R, int32_t r);
+
+/* Eq. 17, k = (B - N*h)/(n - h) - s1 - s2 with h the number of full-cache heads
+ * of the layer, the quotient floored, clamped to [0, N - s1 - s2].  Host only. */
+int32_t taskkv_mid_budget(double budget_tokens, int32_t N, int32_t h_full, int32_t n,
+                          int32_t sink, int32_t recent);
+
+/* Kernel launches issued by this library in this process so far. */
+int64_t taskkv_launch_count(void);
+
+/* Optional per-kernel timing: when enabled every launch is bracketed by CUDA
+ * events on its stream.  taskkv_timing_collect synchronises the device, then
+ * writes up to `max` records as (kernel id, milliseconds) pairs and clears the
+ * log; returns the number written.  Names: taskkv_timing_name(id). */
+void        taskkv_timing_enable(int32_t on);
+int32_t     taskkv_timing_collect(int32_t* ids, float* ms, int32_t max);
+const char* taskkv_timing_name(int32_t id);
+
+#ifdef __cplusplus
+}
+#endif
+#endif  /* TASKKV_H_ */

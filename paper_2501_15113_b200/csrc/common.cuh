@@ -1,0 +1,167 @@
+// Shared declarations of the Task-KV CUDA library (internal; the public
+// boundary is include/taskkv.h).
+#pragma once
+
+#include <cuda_bf16.h>
+#include <cuda_runtime.h>
+#include <stdint.h>
+
+#include "taskkv.h"
+
+namespace taskkv {
+
+constexpr int kDecodeChunk = 256;                 // rows of one split-K decode item
+constexpr int kGatherRows = 64;                   // rows of one gather item
+constexpr int kScoreChunk = 1024;                 // keys of one window-score work item
+constexpr float kLog2e = 1.4426950408889634f;
+
+// kernel ids for launch counting / timing
+enum KernelId : int32_t {
+  K_WINDOW_STATS = 0,
+  K_WINDOW_REDUCE,
+  K_WINDOW_SCORES,
+  K_SELECT,
+  K_SEPARATOR,
+  K_PLAN,
+  K_GATHER,
+  K_APPEND,
+  K_DECODE_PLAN,
+  K_DECODE_ATTN,
+  K_DECODE_COMBINE,
+  K_WINDOW_TC,
+  K_COUNT
+};
+
+// Device-side description of one compression / decode problem.  All pointers
+// are device pointers into the cache memory or the workspace.
+struct DeviceProblem {
+  int32_t U;            // units
+  int32_t R, n_heads, n_kv, G, d;
+  int32_t L;            // window
+  int32_t rows;         // G * L
+  int32_t rows_pad;     // rows rounded up to 16
+  int32_t top_t, pool_w;
+  int32_t sink, recent;
+  int32_t promote_center, force_class;
+  int32_t max_new;
+  int32_t idx_stride;   // ints per unit in idx
+  int32_t chunks_max;   // score chunks of the longest sequence
+  int64_t pool_rows;
+  int64_t max_items;    // decode work items the scratch can hold
+  // per unit tables
+  const int32_t* unit_N;      // [U] sequence length
+  const int32_t* unit_mid;    // [U] middle budget k of the unit's layer
+  const int32_t* nhet;        // [B*R] far heads per (sequence, layer)
+  const int64_t* c_off;       // [U+1] offset of the unit's scores in C
+  const void* const* q_ptr;   // [U] -> [rows][d]
+  const void* const* k_ptr;   // [U] -> [N][d]
+  const void* const* v_ptr;   // [U] -> [N][d]
+  // results
+  int32_t* status;            // sticky status word
+  int32_t* len;               // [U]
+  int32_t* cap;               // [U]
+  int64_t* seg_off;           // [U+1] first pool row
+  int32_t* cls;               // [U]
+  float* dist;                // [U]
+  float* sem;                 // [U][d]
+  int32_t* idx;               // [U][idx_stride]
+  int32_t* gather_off;        // [U+1] gather work items
+  int32_t* dec_off;           // [U+1] decode work items
+  void* k_pool;
+  void* v_pool;
+  // decode scratch
+  float* part_acc;            // [items][G][d]
+  float* part_ml;             // [items][G][2]
+  // workspace
+  float* C;                   // scores, units concatenated
+  float* stat_part;           // [U][chunks_max][rows_pad][2]
+  float* stat;                // [U][rows_pad][2]  (row max in log2 units, 1/Z)
+  int32_t* topt;              // [U][top_t]
+};
+
+// launch bookkeeping (api.cu)
+void note_launch_begin(int32_t id, cudaStream_t s);
+void note_launch_end(int32_t id, cudaStream_t s);
+
+struct LaunchScope {
+  int32_t id;
+  cudaStream_t s;
+  LaunchScope(int32_t id_, cudaStream_t s_) : id(id_), s(s_) { note_launch_begin(id, s); }
+  ~LaunchScope() { note_launch_end(id, s); }
+};
+
+// kernel launchers (one per translation unit)
+cudaError_t launch_window_scores(const DeviceProblem& p, int dtype, int max_N, cudaStream_t s);
+cudaError_t launch_select(const DeviceProblem& p, int dtype, cudaStream_t s);
+cudaError_t launch_separator_plan(const DeviceProblem& p, int n_br, cudaStream_t s);
+cudaError_t launch_decode_plan(const DeviceProblem& p, const int32_t* lengths, cudaStream_t s);
+cudaError_t launch_gather(const DeviceProblem& p, int dtype, int64_t gather_items, cudaStream_t s);
+cudaError_t launch_append(const DeviceProblem& p, int dtype, const void* k_new, const void* v_new,
+                          cudaStream_t s);
+cudaError_t launch_decode(const DeviceProblem& p, int dtype, const void* q, void* out, cudaStream_t s);
+
+// ---------------------------------------------------------------- device helpers
+#ifdef __CUDACC__
+
+__device__ __forceinline__ float to_float(float x) { return x; }
+__device__ __forceinline__ float to_float(__nv_bfloat16 x) { return __bfloat162float(x); }
+
+__device__ __forceinline__ void store_out(float* p, float x) { *p = x; }
+__device__ __forceinline__ void store_out(__nv_bfloat16* p, float x) { *p = __float2bfloat16_rn(x); }
+
+// Unpack a 16-byte vector of elements into floats: 4 for fp32, 8 for bf16.
+template <typename T>
+struct Vec16;
+template <>
+struct Vec16<float> {
+  static constexpr int N = 4;
+  __device__ __forceinline__ static void unpack(const uint4& r, float* f) {
+    f[0] = __uint_as_float(r.x);
+    f[1] = __uint_as_float(r.y);
+    f[2] = __uint_as_float(r.z);
+    f[3] = __uint_as_float(r.w);
+  }
+};
+template <>
+struct Vec16<__nv_bfloat16> {
+  static constexpr int N = 8;
+  __device__ __forceinline__ static void unpack(const uint4& r, float* f) {
+    // a bf16 is the high half of an fp32; the low half of a word is the earlier element
+    f[0] = __uint_as_float(r.x << 16);
+    f[1] = __uint_as_float(r.x & 0xffff0000u);
+    f[2] = __uint_as_float(r.y << 16);
+    f[3] = __uint_as_float(r.y & 0xffff0000u);
+    f[4] = __uint_as_float(r.z << 16);
+    f[5] = __uint_as_float(r.z & 0xffff0000u);
+    f[6] = __uint_as_float(r.w << 16);
+    f[7] = __uint_as_float(r.w & 0xffff0000u);
+  }
+};
+
+__device__ __forceinline__ float warp_max(float v) {
+#pragma unroll
+  for (int o = 16; o > 0; o >>= 1) v = fmaxf(v, __shfl_xor_sync(0xffffffffu, v, o));
+  return v;
+}
+__device__ __forceinline__ float warp_sum(float v) {
+#pragma unroll
+  for (int o = 16; o > 0; o >>= 1) v += __shfl_xor_sync(0xffffffffu, v, o);
+  return v;
+}
+
+// Largest index i in [0, n) with off[i] <= x, for a non-decreasing off[0..n]
+// with off[0] <= x < off[n].
+__device__ __forceinline__ int upper_unit(const int32_t* off, int n, int x) {
+  int lo = 0, hi = n;
+  while (hi - lo > 1) {
+    const int mid = (lo + hi) >> 1;
+    if (off[mid] <= x) lo = mid; else hi = mid;
+  }
+  return lo;
+}
+
+__device__ __forceinline__ void set_status(int32_t* status, int32_t code) { atomicCAS(status, 0, code); }
+
+#endif  // __CUDACC__
+
+}  // namespace taskkv

@@ -1,0 +1,118 @@
+// Data movement of the compacted cache (Sec. IV-B): the retained K and V rows of
+// every unit are copied into the unit's pool segment in ascending position
+// (full-cache units copy all N rows), and decode-time appends add one row per
+// unit.  Rows move as 16-byte vectors.
+#include "common.cuh"
+
+namespace taskkv {
+
+namespace {
+
+constexpr int kGatherThreads = 256;
+
+// One block copies kGatherRows consecutive segment rows of one unit, K and V.
+template <int ROW_BYTES>
+__global__ void __launch_bounds__(kGatherThreads) gather_kernel(DeviceProblem p) {
+  constexpr int VPR = ROW_BYTES / 16;                 // vectors (threads) per row
+  constexpr int RPP = kGatherThreads / VPR;           // rows per pass
+  constexpr int PASSES = kGatherRows / RPP;
+  __shared__ int s_unit;
+  const int item = blockIdx.x;
+  if (threadIdx.x == 0) s_unit = (item < p.gather_off[p.U]) ? upper_unit(p.gather_off, p.U, item) : -1;
+  __syncthreads();
+  const int u = s_unit;
+  if (u < 0) return;
+  const int len = p.len[u];
+  const int N = p.unit_N[u];
+  const int r0 = (item - p.gather_off[u]) * kGatherRows;
+  const int64_t seg = p.seg_off[u];
+  if (seg + len > p.pool_rows) return;                // planning overflow, already flagged
+  const bool identity = (len == N);
+  const int32_t* idx = p.idx + (size_t)u * p.idx_stride;
+  const unsigned char* ksrc = static_cast<const unsigned char*>(p.k_ptr[u]);
+  const unsigned char* vsrc = static_cast<const unsigned char*>(p.v_ptr[u]);
+  unsigned char* kdst = static_cast<unsigned char*>(p.k_pool) + (size_t)seg * ROW_BYTES;
+  unsigned char* vdst = static_cast<unsigned char*>(p.v_pool) + (size_t)seg * ROW_BYTES;
+  const int rr = threadIdx.x / VPR, vc = threadIdx.x % VPR;
+
+  uint4 kreg[PASSES], vreg[PASSES];
+#pragma unroll
+  for (int ps = 0; ps < PASSES; ++ps) {
+    const int r = r0 + ps * RPP + rr;
+    if (r < len) {
+      int src = identity ? r : idx[r];
+      src = min(max(src, 0), N - 1);
+      kreg[ps] = *reinterpret_cast<const uint4*>(ksrc + (size_t)src * ROW_BYTES + vc * 16);
+      vreg[ps] = *reinterpret_cast<const uint4*>(vsrc + (size_t)src * ROW_BYTES + vc * 16);
+    }
+  }
+#pragma unroll
+  for (int ps = 0; ps < PASSES; ++ps) {
+    const int r = r0 + ps * RPP + rr;
+    if (r < len) {
+      *reinterpret_cast<uint4*>(kdst + (size_t)r * ROW_BYTES + vc * 16) = kreg[ps];
+      *reinterpret_cast<uint4*>(vdst + (size_t)r * ROW_BYTES + vc * 16) = vreg[ps];
+    }
+  }
+}
+
+// One warp per unit: the new token's k, v rows go to row len_u of the segment.
+template <int ROW_BYTES>
+__global__ void __launch_bounds__(256) append_kernel(DeviceProblem p, const unsigned char* k_new,
+                                                     const unsigned char* v_new) {
+  constexpr int VPR = ROW_BYTES / 16;
+  const int u = blockIdx.x * 8 + (threadIdx.x >> 5);
+  const int lane = threadIdx.x & 31;
+  if (u >= p.U) return;
+  const int len = p.len[u];
+  const int64_t seg = p.seg_off[u];
+  const bool ok = len < p.cap[u] && seg + len < p.pool_rows;
+  __syncwarp();
+  if (ok && lane < VPR) {
+    const size_t dst = ((size_t)seg + len) * ROW_BYTES + lane * 16;
+    const size_t src = (size_t)u * ROW_BYTES + lane * 16;
+    *reinterpret_cast<uint4*>(static_cast<unsigned char*>(p.k_pool) + dst) =
+        *reinterpret_cast<const uint4*>(k_new + src);
+    *reinterpret_cast<uint4*>(static_cast<unsigned char*>(p.v_pool) + dst) =
+        *reinterpret_cast<const uint4*>(v_new + src);
+  }
+  __syncwarp();
+  if (lane == 0) {
+    if (ok) p.len[u] = len + 1;
+    else set_status(p.status, TASKKV_ESTATE);
+  }
+}
+
+}  // namespace
+
+cudaError_t launch_gather(const DeviceProblem& p, int dtype, int64_t gather_items, cudaStream_t s) {
+  if (gather_items <= 0) return cudaSuccess;
+  LaunchScope ls(K_GATHER, s);
+  const int row_bytes = p.d * (dtype == TASKKV_F32 ? 4 : 2);
+  const unsigned grid = (unsigned)gather_items;
+  switch (row_bytes) {
+    case 128: gather_kernel<128><<<grid, kGatherThreads, 0, s>>>(p); break;
+    case 256: gather_kernel<256><<<grid, kGatherThreads, 0, s>>>(p); break;
+    case 512: gather_kernel<512><<<grid, kGatherThreads, 0, s>>>(p); break;
+    default: return cudaErrorInvalidValue;
+  }
+  return cudaGetLastError();
+}
+
+cudaError_t launch_append(const DeviceProblem& p, int dtype, const void* k_new, const void* v_new,
+                          cudaStream_t s) {
+  LaunchScope ls(K_APPEND, s);
+  const int row_bytes = p.d * (dtype == TASKKV_F32 ? 4 : 2);
+  const unsigned grid = (unsigned)((p.U + 7) / 8);
+  const unsigned char* kn = static_cast<const unsigned char*>(k_new);
+  const unsigned char* vn = static_cast<const unsigned char*>(v_new);
+  switch (row_bytes) {
+    case 128: append_kernel<128><<<grid, 256, 0, s>>>(p, kn, vn); break;
+    case 256: append_kernel<256><<<grid, 256, 0, s>>>(p, kn, vn); break;
+    case 512: append_kernel<512><<<grid, 256, 0, s>>>(p, kn, vn); break;
+    default: return cudaErrorInvalidValue;
+  }
+  return cudaGetLastError();
+}
+
+}  // namespace taskkv
