@@ -1,0 +1,623 @@
+// Host side of the Task-KV library: argument validation, exact buffer planning,
+// the cache handle, and the kernel sequences behind the exported calls.
+#include <atomic>
+#include <cmath>
+#include <cstdio>
+#include <cstring>
+#include <mutex>
+#include <new>
+#include <vector>
+
+#include "common.cuh"
+
+using namespace taskkv;
+
+namespace {
+
+constexpr size_t kAlign = 256;
+inline size_t align_up(size_t x) { return (x + kAlign - 1) / kAlign * kAlign; }
+
+struct HostPlan {
+  taskkv_plan_info info;
+  int64_t c_total = 0;
+  int32_t max_N = 0, min_N = 0;
+  int32_t chunks_max = 0, rows = 0, rows_pad = 0, idx_stride = 0;
+  std::vector<int32_t> seq_lens, mid, nhet;     // [B], [R], [B*R]
+  std::vector<int32_t> full;                    // [B*R] full-cache heads
+  // byte offsets inside the cache memory
+  size_t o_unit_N, o_unit_mid, o_nhet, o_c_off, o_qp, o_kp, o_vp, meta_bytes;
+  size_t o_status, o_len, o_cap, o_seg, o_cls, o_dist, o_sem, o_idx, o_goff, o_doff, o_pacc, o_pml, o_kpool,
+      o_vpool;
+  // inside the workspace
+  size_t w_C, w_spart, w_stat, w_topt;
+};
+
+int32_t hetero_count_impl(int32_t n, float beta, int32_t m, int32_t R, int32_t r) {
+  const double top = (double)n * (double)beta;
+  const double val = (R <= 1) ? top : top - (top - (double)m) / (double)(R - 1) * (double)r;
+  long f = (long)std::floor(val + 0.5);
+  if (f < 0) f = 0;
+  if (f > n) f = n;
+  return (int32_t)f;
+}
+
+taskkv_status make_plan(const taskkv_params* p, HostPlan& hp) {
+  if (!p || !p->seq_lens) return TASKKV_EINVAL;
+  if (p->n_layers < 1 || p->batch < 1 || p->n_heads < 1 || p->n_kv_heads < 1) return TASKKV_EINVAL;
+  if (p->n_kv_heads > TASKKV_MAX_KV_HEADS || p->n_heads % p->n_kv_heads != 0) return TASKKV_EINVAL;
+  if (p->head_dim != 64 && p->head_dim != 128) return TASKKV_EINVAL;
+  if (p->dtype != TASKKV_F32 && p->dtype != TASKKV_BF16) return TASKKV_EINVAL;
+  const int G = p->n_heads / p->n_kv_heads;
+  if (G != 1 && G != 2 && G != 4 && G != 8) return TASKKV_EINVAL;
+  if (p->window < 1 || (int64_t)G * p->window > TASKKV_MAX_WINDOW_ROWS) return TASKKV_EINVAL;
+  if (p->sink < 0 || p->recent < 0 || p->mid_budget < 0 || p->max_new_tokens < 0) return TASKKV_EINVAL;
+  if (p->top_t < 1 || p->top_t > TASKKV_MAX_TOP_T) return TASKKV_EINVAL;
+  if (p->pool_kernel < 1 || p->pool_kernel > 31 || p->pool_kernel % 2 == 0) return TASKKV_EINVAL;
+  if (p->force_class < -1 || p->force_class > 1) return TASKKV_EINVAL;
+  const int B = p->batch, R = p->n_layers, nkv = p->n_kv_heads;
+  if ((int64_t)B * R * nkv > (1 << 20)) return TASKKV_EINVAL;
+
+  hp.seq_lens.assign(p->seq_lens, p->seq_lens + B);
+  hp.max_N = 0;
+  hp.min_N = INT32_MAX;
+  for (int b = 0; b < B; ++b) {
+    const int N = hp.seq_lens[b];
+    if (N < 1 || N > (1 << 24)) return TASKKV_EINVAL;
+    hp.max_N = std::max(hp.max_N, N);
+    hp.min_N = std::min(hp.min_N, N);
+  }
+  if (p->window > hp.min_N) return TASKKV_EINVAL;
+  hp.mid.resize(R);
+  for (int r = 0; r < R; ++r) {
+    hp.mid[r] = p->mid_budget_per_layer ? p->mid_budget_per_layer[r] : p->mid_budget;
+    if (hp.mid[r] < 0) return TASKKV_EINVAL;
+  }
+  hp.nhet.resize((size_t)B * R);
+  hp.full.resize((size_t)B * R);
+  for (int b = 0; b < B; ++b)
+    for (int r = 0; r < R; ++r) {
+      int f = p->n_hetero ? p->n_hetero[(size_t)b * R + r] : hetero_count_impl(nkv, p->beta, p->m_top, R, r);
+      if (f < 0) return TASKKV_EINVAL;
+      f = std::min(f, nkv);
+      hp.nhet[(size_t)b * R + r] = f;
+      int h = std::min(nkv, f + ((p->promote_center && f < nkv) ? 1 : 0));
+      if (p->force_class == 1) h = nkv;
+      if (p->force_class == 0) h = 0;
+      hp.full[(size_t)b * R + r] = h;
+    }
+
+  const int64_t U = (int64_t)B * R * nkv;
+  const int s1 = p->sink, s2 = p->recent, mn = p->max_new_tokens;
+  int64_t pool = 0, kept_rows = 0, gitems = 0, ditems = 0, c_total = 0;
+  int32_t stride = 1;
+  for (int b = 0; b < B; ++b) {
+    const int64_t N = hp.seq_lens[b];
+    for (int r = 0; r < R; ++r) {
+      const int64_t h = hp.full[(size_t)b * R + r];
+      int64_t kept = N;
+      if (N > (int64_t)s1 + s2) kept = s1 + s2 + std::min<int64_t>(hp.mid[r], N - s1 - s2);
+      if (kept < N) stride = std::max<int32_t>(stride, (int32_t)kept);
+      pool += h * (N + mn) + (nkv - h) * (kept + mn);
+      kept_rows += h * N + (nkv - h) * kept;
+      gitems += h * ((N + kGatherRows - 1) / kGatherRows) + (nkv - h) * ((kept + kGatherRows - 1) / kGatherRows);
+      ditems += h * ((N + mn + kDecodeChunk - 1) / kDecodeChunk) +
+                (nkv - h) * ((kept + mn + kDecodeChunk - 1) / kDecodeChunk);
+      c_total += (int64_t)nkv * N;
+    }
+  }
+  if (gitems > 0x7fffffff || ditems > 0x7fffffff) return TASKKV_EINVAL;
+  hp.idx_stride = (stride + 3) / 4 * 4;
+  hp.c_total = c_total;
+  hp.rows = G * p->window;
+  hp.rows_pad = (hp.rows + 15) / 16 * 16;
+  hp.chunks_max = (hp.max_N + kScoreChunk - 1) / kScoreChunk;
+
+  const size_t es = p->dtype == TASKKV_F32 ? 4 : 2;
+  const size_t d = p->head_dim;
+  size_t o = 0;
+  auto take = [&](size_t bytes) { size_t at = o; o = align_up(o + bytes); return at; };
+  hp.o_unit_N = take(U * 4);
+  hp.o_unit_mid = take(U * 4);
+  hp.o_nhet = take((size_t)B * R * 4);
+  hp.o_c_off = take((U + 1) * 8);
+  hp.o_qp = take(U * 8);
+  hp.o_kp = take(U * 8);
+  hp.o_vp = take(U * 8);
+  hp.meta_bytes = o;
+  hp.o_status = take(64);
+  hp.o_len = take(U * 4);
+  hp.o_cap = take(U * 4);
+  hp.o_seg = take((U + 1) * 8);
+  hp.o_cls = take(U * 4);
+  hp.o_dist = take(U * 4);
+  hp.o_sem = take(U * d * 4);
+  hp.o_idx = take((size_t)U * hp.idx_stride * 4);
+  hp.o_goff = take((U + 1) * 4);
+  hp.o_doff = take((U + 1) * 4);
+  hp.o_pacc = take((size_t)ditems * G * d * 4);
+  hp.o_pml = take((size_t)ditems * G * 2 * 4);
+  hp.o_kpool = take((size_t)pool * d * es);
+  hp.o_vpool = take((size_t)pool * d * es);
+  const size_t cache_bytes = o;
+  o = 0;
+  hp.w_C = take((size_t)c_total * 4);
+  hp.w_spart = take((size_t)U * hp.chunks_max * hp.rows_pad * 8);
+  hp.w_stat = take((size_t)U * hp.rows_pad * 8);
+  hp.w_topt = take((size_t)U * p->top_t * 4);
+  const size_t work_bytes = o;
+
+  hp.info.n_units = U;
+  hp.info.pool_rows = pool;
+  hp.info.retained_rows = kept_rows;
+  hp.info.cache_bytes = (int64_t)cache_bytes;
+  hp.info.workspace_bytes = (int64_t)work_bytes;
+  hp.info.max_decode_items = ditems;
+  hp.info.gather_items = gitems;
+  hp.info.index_stride = hp.idx_stride;
+  return TASKKV_OK;
+}
+
+// ---------------------------------------------------------------- launch log
+std::atomic<int64_t> g_launches{0};
+std::atomic<int> g_timing{0};
+struct TimingRec { int32_t id; cudaEvent_t a, b; };
+std::mutex g_tmu;
+std::vector<TimingRec> g_trecs;
+thread_local cudaEvent_t tl_start = nullptr;
+
+const char* kKernelNames[K_COUNT] = {
+    "window_stats", "window_reduce", "window_scores", "select", "separator", "plan",
+    "gather", "append", "decode_plan", "decode_attn", "decode_combine", "window_tc"};
+
+}  // namespace
+
+namespace taskkv {
+void note_launch_begin(int32_t, cudaStream_t s) {
+  g_launches.fetch_add(1, std::memory_order_relaxed);
+  if (g_timing.load(std::memory_order_relaxed)) {
+    cudaEventCreate(&tl_start);
+    cudaEventRecord(tl_start, s);
+  }
+}
+void note_launch_end(int32_t id, cudaStream_t s) {
+  if (g_timing.load(std::memory_order_relaxed) && tl_start) {
+    TimingRec r;
+    r.id = id;
+    r.a = tl_start;
+    tl_start = nullptr;
+    cudaEventCreate(&r.b);
+    cudaEventRecord(r.b, s);
+    std::lock_guard<std::mutex> lk(g_tmu);
+    g_trecs.push_back(r);
+  }
+}
+}  // namespace taskkv
+
+struct taskkv_cache {
+  taskkv_params prm;
+  HostPlan hp;
+  DeviceProblem dp;
+  std::vector<unsigned char> meta;
+  void* cache_mem = nullptr;
+  void* work_mem = nullptr;
+  bool own_cache = false, own_work = false;
+  // staging for the host-buffer decode path
+  void* stage = nullptr;
+  size_t stage_bytes = 0;
+};
+
+namespace {
+
+void fill_device_problem(taskkv_cache* c) {
+  const taskkv_params& p = c->prm;
+  const HostPlan& hp = c->hp;
+  DeviceProblem& d = c->dp;
+  unsigned char* cm = static_cast<unsigned char*>(c->cache_mem);
+  unsigned char* wm = static_cast<unsigned char*>(c->work_mem);
+  std::memset(&d, 0, sizeof(d));
+  d.U = (int32_t)hp.info.n_units;
+  d.R = p.n_layers;
+  d.n_heads = p.n_heads;
+  d.n_kv = p.n_kv_heads;
+  d.G = p.n_heads / p.n_kv_heads;
+  d.d = p.head_dim;
+  d.L = p.window;
+  d.rows = hp.rows;
+  d.rows_pad = hp.rows_pad;
+  d.top_t = p.top_t;
+  d.pool_w = p.pool_kernel;
+  d.sink = p.sink;
+  d.recent = p.recent;
+  d.promote_center = p.promote_center;
+  d.force_class = p.force_class;
+  d.max_new = p.max_new_tokens;
+  d.idx_stride = hp.idx_stride;
+  d.chunks_max = hp.chunks_max;
+  d.pool_rows = hp.info.pool_rows;
+  d.max_items = hp.info.max_decode_items;
+  d.unit_N = reinterpret_cast<const int32_t*>(cm + hp.o_unit_N);
+  d.unit_mid = reinterpret_cast<const int32_t*>(cm + hp.o_unit_mid);
+  d.nhet = reinterpret_cast<const int32_t*>(cm + hp.o_nhet);
+  d.c_off = reinterpret_cast<const int64_t*>(cm + hp.o_c_off);
+  d.q_ptr = reinterpret_cast<const void* const*>(cm + hp.o_qp);
+  d.k_ptr = reinterpret_cast<const void* const*>(cm + hp.o_kp);
+  d.v_ptr = reinterpret_cast<const void* const*>(cm + hp.o_vp);
+  d.status = reinterpret_cast<int32_t*>(cm + hp.o_status);
+  d.len = reinterpret_cast<int32_t*>(cm + hp.o_len);
+  d.cap = reinterpret_cast<int32_t*>(cm + hp.o_cap);
+  d.seg_off = reinterpret_cast<int64_t*>(cm + hp.o_seg);
+  d.cls = reinterpret_cast<int32_t*>(cm + hp.o_cls);
+  d.dist = reinterpret_cast<float*>(cm + hp.o_dist);
+  d.sem = reinterpret_cast<float*>(cm + hp.o_sem);
+  d.idx = reinterpret_cast<int32_t*>(cm + hp.o_idx);
+  d.gather_off = reinterpret_cast<int32_t*>(cm + hp.o_goff);
+  d.dec_off = reinterpret_cast<int32_t*>(cm + hp.o_doff);
+  d.part_acc = reinterpret_cast<float*>(cm + hp.o_pacc);
+  d.part_ml = reinterpret_cast<float*>(cm + hp.o_pml);
+  d.k_pool = cm + hp.o_kpool;
+  d.v_pool = cm + hp.o_vpool;
+  if (wm) {
+    d.C = reinterpret_cast<float*>(wm + hp.w_C);
+    d.stat_part = reinterpret_cast<float*>(wm + hp.w_spart);
+    d.stat = reinterpret_cast<float*>(wm + hp.w_stat);
+    d.topt = reinterpret_cast<int32_t*>(wm + hp.w_topt);
+  }
+}
+
+void build_meta(taskkv_cache* c, const void* const* q_win, const void* const* k, const void* const* v) {
+  const taskkv_params& p = c->prm;
+  const HostPlan& hp = c->hp;
+  const int B = p.batch, R = p.n_layers, nkv = p.n_kv_heads;
+  const int G = p.n_heads / nkv;
+  const size_t es = p.dtype == TASKKV_F32 ? 4 : 2;
+  const size_t d = p.head_dim;
+  c->meta.assign(hp.meta_bytes, 0);
+  unsigned char* m = c->meta.data();
+  int32_t* unit_N = reinterpret_cast<int32_t*>(m + hp.o_unit_N);
+  int32_t* unit_mid = reinterpret_cast<int32_t*>(m + hp.o_unit_mid);
+  int32_t* nhet = reinterpret_cast<int32_t*>(m + hp.o_nhet);
+  int64_t* c_off = reinterpret_cast<int64_t*>(m + hp.o_c_off);
+  const void** qp = reinterpret_cast<const void**>(m + hp.o_qp);
+  const void** kp = reinterpret_cast<const void**>(m + hp.o_kp);
+  const void** vp = reinterpret_cast<const void**>(m + hp.o_vp);
+  std::memcpy(nhet, hp.nhet.data(), hp.nhet.size() * 4);
+  int64_t coff = 0;
+  size_t u = 0;
+  for (int b = 0; b < B; ++b) {
+    const size_t N = hp.seq_lens[b];
+    for (int r = 0; r < R; ++r)
+      for (int h = 0; h < nkv; ++h, ++u) {
+        unit_N[u] = (int32_t)N;
+        unit_mid[u] = hp.mid[r];
+        c_off[u] = coff;
+        coff += (int64_t)N;
+        qp[u] = static_cast<const unsigned char*>(q_win[b]) +
+                (((size_t)r * p.n_heads + (size_t)h * G) * p.window) * d * es;
+        kp[u] = static_cast<const unsigned char*>(k[b]) + (((size_t)r * nkv + h) * N) * d * es;
+        vp[u] = static_cast<const unsigned char*>(v[b]) + (((size_t)r * nkv + h) * N) * d * es;
+      }
+  }
+  c_off[u] = coff;
+}
+
+taskkv_status cuda_status(cudaError_t e) { return e == cudaSuccess ? TASKKV_OK : TASKKV_ECUDA; }
+
+}  // namespace
+
+// ================================================================ exported calls
+extern "C" {
+
+void taskkv_params_default(taskkv_params* p) {
+  if (!p) return;
+  std::memset(p, 0, sizeof(*p));
+  p->n_layers = 1;
+  p->batch = 1;
+  p->sink = 16;
+  p->recent = 256;
+  p->mid_budget = 0;
+  p->window = 32;
+  p->top_t = 256;
+  p->pool_kernel = 7;
+  p->beta = 0.25f;
+  p->m_top = 4;
+  p->promote_center = 1;
+  p->force_class = -1;
+  p->dtype = TASKKV_BF16;
+  p->max_new_tokens = 0;
+}
+
+taskkv_status taskkv_plan(const taskkv_params* p, taskkv_plan_info* out) {
+  if (!out) return TASKKV_EINVAL;
+  HostPlan hp;
+  const taskkv_status st = make_plan(p, hp);
+  if (st != TASKKV_OK) return st;
+  *out = hp.info;
+  return TASKKV_OK;
+}
+
+taskkv_status taskkv_compress_ex(const taskkv_params* p, const void* const* q_win, const void* const* k,
+                                 const void* const* v, void* cache_mem, size_t cache_bytes,
+                                 void* workspace_mem, size_t workspace_bytes, taskkv_stream stream,
+                                 taskkv_cache** out_cache) {
+  if (!p || !q_win || !k || !v || !out_cache) return TASKKV_EINVAL;
+  *out_cache = nullptr;
+  taskkv_cache* c = new (std::nothrow) taskkv_cache();
+  if (!c) return TASKKV_EALLOC;
+  taskkv_status st = make_plan(p, c->hp);
+  if (st != TASKKV_OK) { delete c; return st; }
+  for (int b = 0; b < p->batch; ++b) {
+    if (!q_win[b] || !k[b] || !v[b] || ((uintptr_t)q_win[b] | (uintptr_t)k[b] | (uintptr_t)v[b]) & 15) {
+      delete c;
+      return TASKKV_EINVAL;
+    }
+  }
+  c->prm = *p;
+  c->prm.seq_lens = c->hp.seq_lens.data();
+  c->prm.mid_budget_per_layer = c->hp.mid.data();
+  c->prm.n_hetero = c->hp.nhet.data();
+  cudaStream_t s = static_cast<cudaStream_t>(stream);
+
+  if (cache_mem) {
+    if (cache_bytes < (size_t)c->hp.info.cache_bytes || ((uintptr_t)cache_mem & (kAlign - 1))) {
+      const bool small = cache_bytes < (size_t)c->hp.info.cache_bytes;
+      delete c;
+      return small ? TASKKV_EALLOC : TASKKV_EINVAL;
+    }
+    c->cache_mem = cache_mem;
+  } else {
+    if (cudaMalloc(&c->cache_mem, (size_t)c->hp.info.cache_bytes) != cudaSuccess) {
+      cudaGetLastError();
+      delete c;
+      return TASKKV_EALLOC;
+    }
+    c->own_cache = true;
+  }
+  if (workspace_mem) {
+    if (workspace_bytes < (size_t)c->hp.info.workspace_bytes || ((uintptr_t)workspace_mem & (kAlign - 1))) {
+      const bool small = workspace_bytes < (size_t)c->hp.info.workspace_bytes;
+      taskkv_cache_destroy(c);
+      return small ? TASKKV_EALLOC : TASKKV_EINVAL;
+    }
+    c->work_mem = workspace_mem;
+  } else {
+    if (cudaMalloc(&c->work_mem, (size_t)c->hp.info.workspace_bytes) != cudaSuccess) {
+      cudaGetLastError();
+      taskkv_cache_destroy(c);
+      return TASKKV_EALLOC;
+    }
+    c->own_work = true;
+  }
+  fill_device_problem(c);
+  build_meta(c, q_win, k, v);
+
+  cudaError_t e = cudaMemcpyAsync(c->cache_mem, c->meta.data(), c->hp.meta_bytes, cudaMemcpyHostToDevice, s);
+  if (e == cudaSuccess) e = cudaMemsetAsync(c->dp.status, 0, 64, s);
+  if (e == cudaSuccess) e = launch_window_scores(c->dp, p->dtype, c->hp.max_N, s);
+  if (e == cudaSuccess) e = launch_select(c->dp, p->dtype, s);
+  if (e == cudaSuccess) e = launch_separator_plan(c->dp, p->batch * p->n_layers, s);
+  if (e == cudaSuccess) e = launch_gather(c->dp, p->dtype, c->hp.info.gather_items, s);
+  if (e != cudaSuccess) {
+    std::fprintf(stderr, "taskkv_compress_ex: CUDA error: %s\n", cudaGetErrorString(e));
+    taskkv_cache_destroy(c);
+    return TASKKV_ECUDA;
+  }
+  *out_cache = c;
+  return TASKKV_OK;
+}
+
+taskkv_status taskkv_compress(const void* q_win, const void* k, const void* v, int32_t n_layers,
+                              int32_t n_heads, int32_t n_kv_heads, int32_t head_dim, int32_t seq_len,
+                              int32_t sink, int32_t recent, int32_t mid_budget, int32_t window,
+                              taskkv_stream stream, taskkv_cache** out_cache) {
+  taskkv_params p;
+  taskkv_params_default(&p);
+  p.n_layers = n_layers;
+  p.n_heads = n_heads;
+  p.n_kv_heads = n_kv_heads;
+  p.head_dim = head_dim;
+  p.batch = 1;
+  p.seq_lens = &seq_len;
+  p.sink = sink;
+  p.recent = recent;
+  p.mid_budget = mid_budget;
+  p.window = window;
+  if (n_kv_heads != n_heads) { p.beta = 0.3f; p.m_top = 1; }   // the grouped-query setting of Sec. V-D
+  p.max_new_tokens = 4096;
+  const void* qa[1] = {q_win};
+  const void* ka[1] = {k};
+  const void* va[1] = {v};
+  return taskkv_compress_ex(&p, qa, ka, va, nullptr, 0, nullptr, 0, stream, out_cache);
+}
+
+taskkv_status taskkv_compress_host(const taskkv_params* p, const void* const* q_win, const void* const* k,
+                                   const void* const* v, taskkv_stream stream, taskkv_cache** out_cache) {
+  if (!p || !q_win || !k || !v || !out_cache) return TASKKV_EINVAL;
+  *out_cache = nullptr;
+  HostPlan hp;
+  taskkv_status st = make_plan(p, hp);
+  if (st != TASKKV_OK) return st;
+  cudaStream_t s = static_cast<cudaStream_t>(stream);
+  const size_t es = p->dtype == TASKKV_F32 ? 4 : 2;
+  const size_t d = p->head_dim;
+  const int B = p->batch;
+  std::vector<void*> dq(B, nullptr), dk(B, nullptr), dv(B, nullptr);
+  auto release = [&]() {
+    for (int b = 0; b < B; ++b) { cudaFree(dq[b]); cudaFree(dk[b]); cudaFree(dv[b]); }
+  };
+  cudaError_t e = cudaSuccess;
+  for (int b = 0; b < B && e == cudaSuccess; ++b) {
+    if (!q_win[b] || !k[b] || !v[b]) { release(); return TASKKV_EINVAL; }
+    const size_t qb = (size_t)p->n_layers * p->n_heads * p->window * d * es;
+    const size_t kb = (size_t)p->n_layers * p->n_kv_heads * (size_t)hp.seq_lens[b] * d * es;
+    e = cudaMalloc(&dq[b], qb);
+    if (e == cudaSuccess) e = cudaMalloc(&dk[b], kb);
+    if (e == cudaSuccess) e = cudaMalloc(&dv[b], kb);
+    if (e != cudaSuccess) { cudaGetLastError(); release(); return TASKKV_EALLOC; }
+    e = cudaMemcpyAsync(dq[b], q_win[b], qb, cudaMemcpyHostToDevice, s);
+    if (e == cudaSuccess) e = cudaMemcpyAsync(dk[b], k[b], kb, cudaMemcpyHostToDevice, s);
+    if (e == cudaSuccess) e = cudaMemcpyAsync(dv[b], v[b], kb, cudaMemcpyHostToDevice, s);
+  }
+  if (e != cudaSuccess) { release(); return TASKKV_ECUDA; }
+  st = taskkv_compress_ex(p, dq.data(), dk.data(), dv.data(), nullptr, 0, nullptr, 0, stream, out_cache);
+  e = cudaStreamSynchronize(s);
+  release();
+  if (st == TASKKV_OK && e != cudaSuccess) {
+    taskkv_cache_destroy(*out_cache);
+    *out_cache = nullptr;
+    return TASKKV_ECUDA;
+  }
+  return st;
+}
+
+taskkv_status taskkv_append(taskkv_cache* c, const void* k_new, const void* v_new, taskkv_stream stream) {
+  if (!c || !k_new || !v_new || (((uintptr_t)k_new | (uintptr_t)v_new) & 15)) return TASKKV_EINVAL;
+  return cuda_status(launch_append(c->dp, c->prm.dtype, k_new, v_new, static_cast<cudaStream_t>(stream)));
+}
+
+taskkv_status taskkv_decode(const void* q, taskkv_cache* c, const int32_t* lengths, void* out,
+                            taskkv_stream stream) {
+  if (!c || !q || !out || (((uintptr_t)q | (uintptr_t)out) & 15)) return TASKKV_EINVAL;
+  return cuda_status(launch_decode(c->dp, c->prm.dtype, q, lengths, out, static_cast<cudaStream_t>(stream)));
+}
+
+taskkv_status taskkv_decode_host(const void* q, const void* k_new, const void* v_new, taskkv_cache* c,
+                                 void* out, taskkv_stream stream) {
+  if (!c || !q || !out || ((k_new == nullptr) != (v_new == nullptr))) return TASKKV_EINVAL;
+  cudaStream_t s = static_cast<cudaStream_t>(stream);
+  const size_t es = c->prm.dtype == TASKKV_F32 ? 4 : 2;
+  const size_t qb = align_up((size_t)c->dp.U * c->dp.G * c->dp.d * es);
+  const size_t kb = align_up((size_t)c->dp.U * c->dp.d * es);
+  const size_t need = 2 * qb + 2 * kb;
+  if (c->stage_bytes < need) {
+    cudaFree(c->stage);
+    c->stage = nullptr;
+    c->stage_bytes = 0;
+    if (cudaMalloc(&c->stage, need) != cudaSuccess) { cudaGetLastError(); return TASKKV_EALLOC; }
+    c->stage_bytes = need;
+  }
+  unsigned char* st = static_cast<unsigned char*>(c->stage);
+  void* dq = st;
+  void* dout = st + qb;
+  void* dkn = st + 2 * qb;
+  void* dvn = st + 2 * qb + kb;
+  const size_t q_bytes = (size_t)c->dp.U * c->dp.G * c->dp.d * es;
+  const size_t k_bytes = (size_t)c->dp.U * c->dp.d * es;
+  cudaError_t e = cudaMemcpyAsync(dq, q, q_bytes, cudaMemcpyHostToDevice, s);
+  if (k_new && e == cudaSuccess) {
+    e = cudaMemcpyAsync(dkn, k_new, k_bytes, cudaMemcpyHostToDevice, s);
+    if (e == cudaSuccess) e = cudaMemcpyAsync(dvn, v_new, k_bytes, cudaMemcpyHostToDevice, s);
+    if (e == cudaSuccess) e = launch_append(c->dp, c->prm.dtype, dkn, dvn, s);
+  }
+  if (e == cudaSuccess) e = launch_decode(c->dp, c->prm.dtype, dq, nullptr, dout, s);
+  if (e == cudaSuccess) e = cudaMemcpyAsync(out, dout, q_bytes, cudaMemcpyDeviceToHost, s);
+  if (e == cudaSuccess) e = cudaStreamSynchronize(s);
+  return cuda_status(e);
+}
+
+int64_t taskkv_cache_query_bytes(const taskkv_cache* c, int32_t what) {
+  if (!c) return -1;
+  const int64_t U = c->dp.U;
+  const int64_t es = c->prm.dtype == TASKKV_F32 ? 4 : 2;
+  switch (what) {
+    case TASKKV_Q_LENGTHS: case TASKKV_Q_CLASSES: case TASKKV_Q_DIST: case TASKKV_Q_CAPACITY: return U * 4;
+    case TASKKV_Q_SEMVEC: return U * c->dp.d * 4;
+    case TASKKV_Q_OFFSETS: return (U + 1) * 8;
+    case TASKKV_Q_INDICES: return U * c->dp.idx_stride * 4;
+    case TASKKV_Q_SCORES: return c->work_mem ? c->hp.c_total * 4 : -1;
+    case TASKKV_Q_TOPT: return c->work_mem ? U * c->dp.top_t * 4 : -1;
+    case TASKKV_Q_STATUS: return 4;
+    case TASKKV_Q_KPOOL: case TASKKV_Q_VPOOL: return c->dp.pool_rows * c->dp.d * es;
+    default: return -1;
+  }
+}
+
+taskkv_status taskkv_cache_query(const taskkv_cache* c, int32_t what, void* host_dst, size_t bytes) {
+  if (!c || !host_dst) return TASKKV_EINVAL;
+  const int64_t need = taskkv_cache_query_bytes(c, what);
+  if (need < 0 || bytes < (size_t)need) return TASKKV_EINVAL;
+  const void* src = nullptr;
+  switch (what) {
+    case TASKKV_Q_LENGTHS: src = c->dp.len; break;
+    case TASKKV_Q_CLASSES: src = c->dp.cls; break;
+    case TASKKV_Q_DIST: src = c->dp.dist; break;
+    case TASKKV_Q_CAPACITY: src = c->dp.cap; break;
+    case TASKKV_Q_SEMVEC: src = c->dp.sem; break;
+    case TASKKV_Q_OFFSETS: src = c->dp.seg_off; break;
+    case TASKKV_Q_INDICES: src = c->dp.idx; break;
+    case TASKKV_Q_SCORES: src = c->dp.C; break;
+    case TASKKV_Q_TOPT: src = c->dp.topt; break;
+    case TASKKV_Q_STATUS: src = c->dp.status; break;
+    case TASKKV_Q_KPOOL: src = c->dp.k_pool; break;
+    case TASKKV_Q_VPOOL: src = c->dp.v_pool; break;
+    default: return TASKKV_EINVAL;
+  }
+  if (cudaDeviceSynchronize() != cudaSuccess) return TASKKV_ECUDA;
+  if (need == 0) return TASKKV_OK;
+  return cuda_status(cudaMemcpy(host_dst, src, (size_t)need, cudaMemcpyDeviceToHost));
+}
+
+taskkv_status taskkv_cache_plan(const taskkv_cache* c, taskkv_plan_info* out) {
+  if (!c || !out) return TASKKV_EINVAL;
+  *out = c->hp.info;
+  return TASKKV_OK;
+}
+
+void taskkv_cache_destroy(taskkv_cache* c) {
+  if (!c) return;
+  if (c->own_cache || c->own_work || c->stage) cudaDeviceSynchronize();
+  if (c->own_cache) cudaFree(c->cache_mem);
+  if (c->own_work) cudaFree(c->work_mem);
+  if (c->stage) cudaFree(c->stage);
+  delete c;
+}
+
+const char* taskkv_status_str(taskkv_status s) {
+  switch (s) {
+    case TASKKV_OK: return "ok";
+    case TASKKV_EINVAL: return "invalid argument";
+    case TASKKV_EALLOC: return "allocation failed or buffer too small";
+    case TASKKV_ECUDA: return "CUDA runtime error";
+    case TASKKV_ETIMEOUT: return "device-side wait timed out";
+    case TASKKV_ESTATE: return "cache in wrong state";
+    default: return "unknown status";
+  }
+}
+
+int32_t taskkv_hetero_count(int32_t n, float beta, int32_t m, int32_t R, int32_t r) {
+  if (n < 0) return 0;
+  return hetero_count_impl(n, beta, m, R, r);
+}
+
+int32_t taskkv_mid_budget(double budget_tokens, int32_t N, int32_t h_full, int32_t n, int32_t sink,
+                          int32_t recent) {
+  if (n <= h_full) return 0;
+  const double per_head = std::floor((budget_tokens - (double)N * (double)h_full) / (double)(n - h_full));
+  double k = per_head - (double)sink - (double)recent;
+  const double room = std::max(0, N - sink - recent);
+  if (k < 0) k = 0;
+  if (k > room) k = room;
+  return (int32_t)k;
+}
+
+int64_t taskkv_launch_count(void) { return g_launches.load(); }
+
+void taskkv_timing_enable(int32_t on) { g_timing.store(on ? 1 : 0); }
+
+int32_t taskkv_timing_collect(int32_t* ids, float* ms, int32_t max) {
+  cudaDeviceSynchronize();
+  std::lock_guard<std::mutex> lk(g_tmu);
+  int32_t n = 0;
+  for (auto& r : g_trecs) {
+    float t = 0.f;
+    cudaEventElapsedTime(&t, r.a, r.b);
+    if (ids && ms && n < max) { ids[n] = r.id; ms[n] = t; ++n; }
+    cudaEventDestroy(r.a);
+    cudaEventDestroy(r.b);
+  }
+  g_trecs.clear();
+  return n;
+}
+
+const char* taskkv_timing_name(int32_t id) { return (id >= 0 && id < K_COUNT) ? kKernelNames[id] : "?"; }
+
+}  // extern "C"

@@ -98,7 +98,8 @@ cudaError_t launch_decode_plan(const DeviceProblem& p, const int32_t* lengths, c
 cudaError_t launch_gather(const DeviceProblem& p, int dtype, int64_t gather_items, cudaStream_t s);
 cudaError_t launch_append(const DeviceProblem& p, int dtype, const void* k_new, const void* v_new,
                           cudaStream_t s);
-cudaError_t launch_decode(const DeviceProblem& p, int dtype, const void* q, void* out, cudaStream_t s);
+cudaError_t launch_decode(const DeviceProblem& p, int dtype, const void* q, const int32_t* lengths, void* out,
+                          cudaStream_t s);
 
 // ---------------------------------------------------------------- device helpers
 #ifdef __CUDACC__
