@@ -1,0 +1,338 @@
+"""ctypes binding of libtaskkv.so: argument marshalling only.
+
+Every step of the Task-KV hot path runs inside the CUDA library; this module
+turns torch tensors into pointers, keeps buffers alive, and reads results
+back.  There is no fallback: if the library is missing, importing this module
+raises.
+"""
+from __future__ import annotations
+
+import ctypes as C
+import os
+from typing import List, Optional, Sequence
+
+import numpy as np
+import torch
+
+_HERE = os.path.dirname(os.path.abspath(__file__))
+LIB_PATH = os.path.join(_HERE, "libtaskkv.so")
+
+if not os.path.exists(LIB_PATH):
+    raise ImportError(
+        f"{LIB_PATH} is missing: build it with `python -m paper_2501_15113_b200.build` "
+        "(the Task-KV path has no non-CUDA implementation)")
+
+lib = C.CDLL(LIB_PATH)
+
+OK, EINVAL, EALLOC, ECUDA, ETIMEOUT, ESTATE = 0, -1, -2, -3, -4, -5
+F32, BF16 = 0, 1
+(Q_LENGTHS, Q_CLASSES, Q_DIST, Q_SEMVEC, Q_OFFSETS, Q_INDICES, Q_SCORES, Q_TOPT, Q_STATUS, Q_KPOOL,
+ Q_VPOOL, Q_CAPACITY) = range(12)
+
+
+class taskkv_params(C.Structure):
+    _fields_ = [
+        ("n_layers", C.c_int32), ("n_heads", C.c_int32), ("n_kv_heads", C.c_int32), ("head_dim", C.c_int32),
+        ("batch", C.c_int32), ("sink", C.c_int32), ("recent", C.c_int32), ("mid_budget", C.c_int32),
+        ("window", C.c_int32), ("top_t", C.c_int32), ("pool_kernel", C.c_int32), ("m_top", C.c_int32),
+        ("beta", C.c_float), ("promote_center", C.c_int32), ("force_class", C.c_int32), ("dtype", C.c_int32),
+        ("max_new_tokens", C.c_int32), ("reserved_", C.c_int32),
+        ("seq_lens", C.POINTER(C.c_int32)), ("mid_budget_per_layer", C.POINTER(C.c_int32)),
+        ("n_hetero", C.POINTER(C.c_int32)),
+    ]
+
+
+class taskkv_plan_info(C.Structure):
+    _fields_ = [(n, C.c_int64) for n in (
+        "n_units", "pool_rows", "retained_rows", "cache_bytes", "workspace_bytes", "max_decode_items",
+        "gather_items", "index_stride")]
+
+
+_vp = C.c_void_p
+_pp = C.POINTER(C.c_void_p)
+lib.taskkv_params_default.argtypes = [C.POINTER(taskkv_params)]
+lib.taskkv_params_default.restype = None
+lib.taskkv_plan.argtypes = [C.POINTER(taskkv_params), C.POINTER(taskkv_plan_info)]
+lib.taskkv_plan.restype = C.c_int32
+lib.taskkv_compress_ex.argtypes = [C.POINTER(taskkv_params), _pp, _pp, _pp, _vp, C.c_size_t, _vp, C.c_size_t,
+                                   _vp, C.POINTER(_vp)]
+lib.taskkv_compress_ex.restype = C.c_int32
+lib.taskkv_compress.argtypes = [_vp, _vp, _vp] + [C.c_int32] * 9 + [_vp, C.POINTER(_vp)]
+lib.taskkv_compress.restype = C.c_int32
+lib.taskkv_compress_host.argtypes = [C.POINTER(taskkv_params), _pp, _pp, _pp, _vp, C.POINTER(_vp)]
+lib.taskkv_compress_host.restype = C.c_int32
+lib.taskkv_append.argtypes = [_vp, _vp, _vp, _vp]
+lib.taskkv_append.restype = C.c_int32
+lib.taskkv_decode.argtypes = [_vp, _vp, _vp, _vp, _vp]
+lib.taskkv_decode.restype = C.c_int32
+lib.taskkv_decode_host.argtypes = [_vp, _vp, _vp, _vp, _vp, _vp]
+lib.taskkv_decode_host.restype = C.c_int32
+lib.taskkv_cache_query_bytes.argtypes = [_vp, C.c_int32]
+lib.taskkv_cache_query_bytes.restype = C.c_int64
+lib.taskkv_cache_query.argtypes = [_vp, C.c_int32, _vp, C.c_size_t]
+lib.taskkv_cache_query.restype = C.c_int32
+lib.taskkv_cache_plan.argtypes = [_vp, C.POINTER(taskkv_plan_info)]
+lib.taskkv_cache_plan.restype = C.c_int32
+lib.taskkv_cache_destroy.argtypes = [_vp]
+lib.taskkv_cache_destroy.restype = None
+lib.taskkv_status_str.argtypes = [C.c_int32]
+lib.taskkv_status_str.restype = C.c_char_p
+lib.taskkv_hetero_count.argtypes = [C.c_int32, C.c_float, C.c_int32, C.c_int32, C.c_int32]
+lib.taskkv_hetero_count.restype = C.c_int32
+lib.taskkv_mid_budget.argtypes = [C.c_double] + [C.c_int32] * 5
+lib.taskkv_mid_budget.restype = C.c_int32
+lib.taskkv_launch_count.argtypes = []
+lib.taskkv_launch_count.restype = C.c_int64
+lib.taskkv_timing_enable.argtypes = [C.c_int32]
+lib.taskkv_timing_enable.restype = None
+lib.taskkv_timing_collect.argtypes = [C.POINTER(C.c_int32), C.POINTER(C.c_float), C.c_int32]
+lib.taskkv_timing_collect.restype = C.c_int32
+lib.taskkv_timing_name.argtypes = [C.c_int32]
+lib.taskkv_timing_name.restype = C.c_char_p
+
+
+class TaskKVError(RuntimeError):
+    def __init__(self, status: int, where: str):
+        self.status = status
+        super().__init__(f"{where}: {lib.taskkv_status_str(status).decode()} ({status})")
+
+
+def _check(status: int, where: str) -> None:
+    if status != OK:
+        raise TaskKVError(status, where)
+
+
+def taskkv_hetero_count(n: int, beta: float, m: int, R: int, r: int) -> int:
+    return int(lib.taskkv_hetero_count(n, beta, m, R, r))
+
+
+def taskkv_mid_budget(budget_tokens: float, N: int, h_full: int, n: int, sink: int, recent: int) -> int:
+    return int(lib.taskkv_mid_budget(budget_tokens, N, h_full, n, sink, recent))
+
+
+def taskkv_launch_count() -> int:
+    return int(lib.taskkv_launch_count())
+
+
+def taskkv_timing_enable(on: bool) -> None:
+    lib.taskkv_timing_enable(1 if on else 0)
+
+
+def taskkv_timing_collect(max_records: int = 1 << 16) -> List[tuple]:
+    ids = (C.c_int32 * max_records)()
+    ms = (C.c_float * max_records)()
+    n = lib.taskkv_timing_collect(ids, ms, max_records)
+    return [(lib.taskkv_timing_name(ids[i]).decode(), float(ms[i])) for i in range(n)]
+
+
+def _stream_handle(stream) -> int:
+    if stream is None:
+        stream = torch.cuda.current_stream()
+    return int(stream.cuda_stream)
+
+
+class Params:
+    """Owns a taskkv_params struct and the host arrays it points to."""
+
+    def __init__(self, *, n_layers, n_heads, n_kv_heads, head_dim, seq_lens: Sequence[int], sink, recent,
+                 mid_budget, window, dtype, top_t=256, pool_kernel=7, beta=0.25, m_top=4,
+                 n_hetero: Optional[Sequence[Sequence[int]]] = None, promote_center=True, force_class=-1,
+                 max_new_tokens=0):
+        p = taskkv_params()
+        lib.taskkv_params_default(C.byref(p))
+        p.n_layers, p.n_heads, p.n_kv_heads, p.head_dim = n_layers, n_heads, n_kv_heads, head_dim
+        p.batch = len(seq_lens)
+        self._seq = (C.c_int32 * len(seq_lens))(*[int(x) for x in seq_lens])
+        p.seq_lens = C.cast(self._seq, C.POINTER(C.c_int32))
+        p.sink, p.recent, p.window = sink, recent, window
+        if isinstance(mid_budget, (list, tuple)):
+            self._mid = (C.c_int32 * len(mid_budget))(*[int(x) for x in mid_budget])
+            p.mid_budget_per_layer = C.cast(self._mid, C.POINTER(C.c_int32))
+            p.mid_budget = int(mid_budget[0])
+        else:
+            self._mid = None
+            p.mid_budget = int(mid_budget)
+        p.top_t, p.pool_kernel, p.beta, p.m_top = top_t, pool_kernel, beta, m_top
+        if n_hetero is not None:
+            flat = [int(x) for row in n_hetero for x in row]
+            self._nh = (C.c_int32 * len(flat))(*flat)
+            p.n_hetero = C.cast(self._nh, C.POINTER(C.c_int32))
+        else:
+            self._nh = None
+        p.promote_center = 1 if promote_center else 0
+        p.force_class = force_class
+        p.dtype = BF16 if dtype in (BF16, "bf16", torch.bfloat16) else F32
+        p.max_new_tokens = max_new_tokens
+        self.c = p
+
+    @property
+    def torch_dtype(self):
+        return torch.bfloat16 if self.c.dtype == BF16 else torch.float32
+
+
+def taskkv_plan(params: Params) -> taskkv_plan_info:
+    info = taskkv_plan_info()
+    _check(lib.taskkv_plan(C.byref(params.c), C.byref(info)), "taskkv_plan")
+    return info
+
+
+def _ptr_array(tensors: Sequence[torch.Tensor]):
+    arr = (C.c_void_p * len(tensors))(*[t.data_ptr() for t in tensors])
+    return arr
+
+
+class Cache:
+    """Handle of a compacted cache (taskkv_cache*) plus the torch buffers backing it."""
+
+    def __init__(self, handle: int, params: Params, keep):
+        self._h = C.c_void_p(handle)
+        self.params = params
+        self._keep = keep
+        info = taskkv_plan_info()
+        _check(lib.taskkv_cache_plan(self._h, C.byref(info)), "taskkv_cache_plan")
+        self.info = info
+
+    def release_workspace(self):
+        """Drops the compress-time workspace (scores and top-t queries stop working)."""
+        self._keep.pop("workspace", None)
+
+    def close(self):
+        if self._h:
+            lib.taskkv_cache_destroy(self._h)
+            self._h = None
+            self._keep = None
+
+    def __del__(self):
+        try:
+            self.close()
+        except Exception:
+            pass
+
+    # -- the decode-side calls
+    def taskkv_append(self, k_new: torch.Tensor, v_new: torch.Tensor, stream=None) -> None:
+        _check(lib.taskkv_append(self._h, k_new.data_ptr(), v_new.data_ptr(), _stream_handle(stream)),
+               "taskkv_append")
+
+    def taskkv_decode(self, q: torch.Tensor, out: Optional[torch.Tensor] = None,
+                      lengths: Optional[torch.Tensor] = None, stream=None) -> torch.Tensor:
+        if out is None:
+            out = torch.empty_like(q)
+        lp = lengths.data_ptr() if lengths is not None else None
+        _check(lib.taskkv_decode(q.data_ptr(), self._h, lp, out.data_ptr(), _stream_handle(stream)),
+               "taskkv_decode")
+        return out
+
+    def taskkv_decode_host(self, q: torch.Tensor, k_new: Optional[torch.Tensor], v_new: Optional[torch.Tensor],
+                           out: torch.Tensor, stream=None) -> torch.Tensor:
+        kp = k_new.data_ptr() if k_new is not None else None
+        vp = v_new.data_ptr() if v_new is not None else None
+        _check(lib.taskkv_decode_host(q.data_ptr(), kp, vp, self._h, out.data_ptr(), _stream_handle(stream)),
+               "taskkv_decode_host")
+        return out
+
+    # -- synchronising reads
+    def query(self, what: int) -> np.ndarray:
+        nbytes = lib.taskkv_cache_query_bytes(self._h, what)
+        if nbytes < 0:
+            raise TaskKVError(EINVAL, "taskkv_cache_query_bytes")
+        buf = np.empty(max(int(nbytes), 1), dtype=np.uint8)
+        _check(lib.taskkv_cache_query(self._h, what, buf.ctypes.data, int(nbytes)), "taskkv_cache_query")
+        buf = buf[:nbytes]
+        U = int(self.info.n_units)
+        if what in (Q_LENGTHS, Q_CLASSES, Q_CAPACITY, Q_STATUS):
+            return buf.view(np.int32)
+        if what == Q_DIST:
+            return buf.view(np.float32)
+        if what == Q_SEMVEC:
+            return buf.view(np.float32).reshape(U, -1)
+        if what == Q_OFFSETS:
+            return buf.view(np.int64)
+        if what == Q_INDICES:
+            return buf.view(np.int32).reshape(U, -1)
+        if what == Q_SCORES:
+            return buf.view(np.float32)
+        if what == Q_TOPT:
+            return buf.view(np.int32).reshape(U, -1)
+        return buf
+
+    def lengths(self):
+        return self.query(Q_LENGTHS)
+
+    def classes(self):
+        return self.query(Q_CLASSES)
+
+    def status(self) -> int:
+        return int(self.query(Q_STATUS)[0])
+
+    def pool_rows(self, which: str, u: int) -> torch.Tensor:
+        """Rows of unit u's K ('k') or V ('v') segment as a CPU tensor [len_u, d]."""
+        off = self.query(Q_OFFSETS)
+        ln = self.query(Q_LENGTHS)
+        raw = self.query(Q_KPOOL if which == "k" else Q_VPOOL)
+        d = self.params.c.head_dim
+        es = 2 if self.params.c.dtype == BF16 else 4
+        seg = raw[int(off[u]) * d * es:(int(off[u]) + int(ln[u])) * d * es]
+        t = torch.from_numpy(seg.copy())
+        return t.view(self.params.torch_dtype).reshape(int(ln[u]), d)
+
+    def retained_indices(self, u: int, N: int) -> np.ndarray:
+        ln = int(self.query(Q_LENGTHS)[u])
+        if ln >= N:
+            return np.arange(N, dtype=np.int64)
+        return self.query(Q_INDICES)[u, :ln].astype(np.int64)
+
+
+def taskkv_compress_ex(params: Params, q_win: Sequence[torch.Tensor], k: Sequence[torch.Tensor],
+                       v: Sequence[torch.Tensor], stream=None, cache_mem: Optional[torch.Tensor] = None,
+                       workspace_mem: Optional[torch.Tensor] = None) -> Cache:
+    """q_win[b]: [R, n, L, d]; k[b], v[b]: [R, n_kv, N_b, d] contiguous CUDA tensors.
+    Cache and workspace memory are torch allocations unless supplied."""
+    info = taskkv_plan(params)
+    dev = k[0].device
+    if cache_mem is None:
+        cache_mem = torch.empty(int(info.cache_bytes), dtype=torch.uint8, device=dev)
+    if workspace_mem is None:
+        workspace_mem = torch.empty(int(info.workspace_bytes), dtype=torch.uint8, device=dev)
+    for t in list(q_win) + list(k) + list(v):
+        if not t.is_contiguous() or not t.is_cuda:
+            raise ValueError("inputs must be contiguous CUDA tensors")
+    qa, ka, va = _ptr_array(q_win), _ptr_array(k), _ptr_array(v)
+    h = C.c_void_p()
+    _check(lib.taskkv_compress_ex(C.byref(params.c), qa, ka, va, cache_mem.data_ptr(), cache_mem.numel(),
+                                  workspace_mem.data_ptr(), workspace_mem.numel(), _stream_handle(stream),
+                                  C.byref(h)), "taskkv_compress_ex")
+    return Cache(h.value, params, {"cache": cache_mem, "workspace": workspace_mem})
+
+
+def taskkv_compress_host(params: Params, q_win: Sequence[torch.Tensor], k: Sequence[torch.Tensor],
+                         v: Sequence[torch.Tensor], stream=None) -> Cache:
+    """Same call with HOST tensors (pinned for asynchronous copies)."""
+    qa, ka, va = _ptr_array(q_win), _ptr_array(k), _ptr_array(v)
+    h = C.c_void_p()
+    _check(lib.taskkv_compress_host(C.byref(params.c), qa, ka, va, _stream_handle(stream), C.byref(h)),
+           "taskkv_compress_host")
+    return Cache(h.value, params, {})
+
+
+def taskkv_compress(q_win: torch.Tensor, k: torch.Tensor, v: torch.Tensor, *, sink: int, recent: int,
+                    mid_budget: int, window: int, stream=None) -> Cache:
+    """The flat form: one bf16 sequence, Sec. V-D defaults, library-owned memory."""
+    R, n, L, d = q_win.shape
+    _, n_kv, N, _ = k.shape
+    h = C.c_void_p()
+    _check(lib.taskkv_compress(q_win.data_ptr(), k.data_ptr(), v.data_ptr(), R, n, n_kv, d, N, sink, recent,
+                               mid_budget, window, _stream_handle(stream), C.byref(h)), "taskkv_compress")
+    beta, m = (0.25, 4) if n == n_kv else (0.3, 1)
+    params = Params(n_layers=R, n_heads=n, n_kv_heads=n_kv, head_dim=d, seq_lens=[N], sink=sink, recent=recent,
+                    mid_budget=mid_budget, window=window, dtype=BF16, beta=beta, m_top=m, max_new_tokens=4096)
+    return Cache(h.value, params, {})
+
+
+def params_from_workload(wl, max_new_tokens: Optional[int] = None, **overrides) -> Params:
+    kw = dict(n_layers=wl.n_layers, n_heads=wl.n_heads, n_kv_heads=wl.n_kv_heads, head_dim=wl.head_dim,
+              seq_lens=wl.seq_lens, sink=wl.sink, recent=wl.recent, mid_budget=list(wl.mid_budget),
+              window=wl.window, dtype=wl.dtype, top_t=wl.top_t, pool_kernel=wl.pool_kernel,
+              n_hetero=wl.n_hetero, promote_center=wl.promote_center,
+              max_new_tokens=wl.decode_steps if max_new_tokens is None else max_new_tokens)
+    kw.update(overrides)
+    return Params(**kw)

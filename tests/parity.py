@@ -1,0 +1,164 @@
+"""Shared machinery of the GPU parity tests: runs the CPU oracle on the same
+seeded inputs as the CUDA library and compares stage by stage.
+
+Index rule: retained positions must be identical, except at a selection
+boundary where the oracle's own scores are tied to within 1e-5 relative (the
+GPU ranks fp32 scores, the oracle fp64 ones); such differences are counted and
+returned so that tests can report and bound them.
+"""
+from __future__ import annotations
+
+import dataclasses
+from typing import Dict, List
+
+import numpy as np
+import torch
+
+from oracle import taskkv_oracle as O
+from paper_2501_15113_b200 import binding as tk
+from paper_2501_15113_b200 import workloads as W
+
+TIE_REL = 1e-5
+TOL_OUT = {"f32": 1e-5, "bf16": 2e-2}
+# C is computed in fp32 from exact products; the design doc derives the bound
+TOL_SCORE_REL = 2e-5
+
+
+@dataclasses.dataclass
+class Report:
+    units: int = 0
+    topt_ties: int = 0
+    mid_ties: int = 0
+    class_near_ties: int = 0
+    max_score_rel: float = 0.0
+    max_sem_rel: float = 0.0
+    max_out_abs: float = 0.0
+    notes: List[str] = dataclasses.field(default_factory=list)
+
+
+def to64(t: torch.Tensor) -> np.ndarray:
+    return t.detach().to("cpu").double().numpy()
+
+
+def check_selection(got: np.ndarray, want: np.ndarray, score: np.ndarray, what: str) -> int:
+    """Sets must agree except for swaps among boundary ties of the oracle's scores.
+    Returns the number of tied swaps."""
+    got_s, want_s = set(got.tolist()), set(want.tolist())
+    assert len(got) == len(got_s), f"{what}: duplicate positions"
+    assert len(got_s) == len(want_s), f"{what}: {len(got_s)} positions, oracle keeps {len(want_s)}"
+    diff = got_s ^ want_s
+    if not diff:
+        return 0
+    thr = min(score[j] for j in want_s)
+    for j in diff:
+        rel = abs(score[j] - thr) / abs(thr)
+        assert rel < TIE_REL, f"{what}: position {j} differs and is not a boundary tie (rel gap {rel:.3e})"
+    return len(diff) // 2
+
+
+def oracle_layer(wl: W.Workload, b: int, r: int, q, k, v, force_class: int = -1) -> Dict:
+    return O.compress_layer(to64(q), to64(k), to64(v), n_hetero=wl.n_hetero[b][r], sink=wl.sink,
+                            recent=wl.recent, mid=wl.mid_budget[r], top_t=wl.top_t,
+                            pool_kernel=wl.pool_kernel, promote_center=wl.promote_center,
+                            force_class=force_class)
+
+
+def unit_index(wl: W.Workload, b: int, r: int, h: int) -> int:
+    return (b * wl.n_layers + r) * wl.n_kv_heads + h
+
+
+def score_offsets(wl: W.Workload) -> np.ndarray:
+    off = [0]
+    for b in range(wl.batch):
+        for _ in range(wl.n_layers * wl.n_kv_heads):
+            off.append(off[-1] + wl.seq_lens[b])
+    return np.array(off, dtype=np.int64)
+
+
+def compare_layer(cache: tk.Cache, wl: W.Workload, b: int, r: int, ref: Dict, rep: Report,
+                  scores: np.ndarray = None, topt: np.ndarray = None) -> None:
+    """Stage-by-stage comparison of one (sequence, layer) against the oracle result `ref`."""
+    N = wl.seq_lens[b]
+    nkv = wl.n_kv_heads
+    lens = cache.lengths()
+    cls = cache.classes()
+    sem = cache.query(tk.Q_SEMVEC)
+    dist = cache.query(tk.Q_DIST)
+    idx_tab = cache.query(tk.Q_INDICES)
+    coff = score_offsets(wl)
+    u0 = unit_index(wl, b, r, 0)
+    flips_in_layer = 0
+    for h in range(nkv):
+        u = u0 + h
+        rep.units += 1
+        # Eq. 12-13: scores
+        if scores is not None:
+            c_gpu = scores[coff[u]:coff[u + 1]].astype(np.float64)
+            rel = np.abs(c_gpu - ref["C"][h]) / ref["C"][h]
+            rep.max_score_rel = max(rep.max_score_rel, float(rel.max()))
+            assert rel.max() < TOL_SCORE_REL, f"unit {u}: scores off by {rel.max():.3e} relative"
+            assert abs(c_gpu.sum() - 1.0) < 1e-4
+        # Eq. 14: top-t set
+        flips = 0
+        if topt is not None:
+            got = topt[u]
+            got = got[got >= 0]
+            flips = check_selection(got, ref["top"][h], ref["C"][h], f"unit {u} top-t")
+            assert np.all(np.diff(got) > 0), f"unit {u}: top-t list not ascending"
+            rep.topt_ties += flips
+            flips_in_layer += flips
+        # Eq. 15: semantic vector (comparable only when the same positions were summed)
+        if flips == 0:
+            scale = max(np.abs(ref["sem"][h]).max(), 1e-30)
+            rel = float(np.abs(sem[u].astype(np.float64) - ref["sem"][h]).max() / scale)
+            rep.max_sem_rel = max(rep.max_sem_rel, rel)
+            assert rel < 1e-4, f"unit {u}: semantic vector off by {rel:.3e} of its largest component"
+    # Eq. 7-8 / Sec. IV-A: distances and classes
+    ref_cls = ref["cls"]
+    got_cls = cls[u0:u0 + nkv]
+    if flips_in_layer == 0:
+        np.testing.assert_allclose(dist[u0:u0 + nkv], ref["dist"], rtol=1e-4, atol=1e-30)
+    if got_cls.tolist() != ref_cls.tolist():
+        # legitimate only if the oracle's own ranking margin is below what the fp32 scores can resolve
+        d = np.sort(ref["dist"])
+        gaps = np.diff(d) / d[1:]
+        assert flips_in_layer > 0 or gaps.min() < 1e-4, \
+            f"(b={b}, r={r}): classes {got_cls.tolist()} differ from the oracle's {ref_cls.tolist()}"
+        rep.class_near_ties += 1
+        rep.notes.append(f"class near-tie at b={b} r={r}")
+        return
+    # Sec. IV-B: lengths and retained positions
+    assert lens[u0:u0 + nkv].tolist() == ref["len"].tolist(), f"(b={b}, r={r}): lengths differ"
+    for h in range(nkv):
+        u = u0 + h
+        want = ref["idx"][h]
+        if len(want) == N:
+            continue
+        got = idx_tab[u, :lens[u]].astype(np.int64)
+        assert np.all(np.diff(got) > 0), f"unit {u}: retained positions not ascending"
+        s1, s2 = wl.sink, wl.recent
+        assert got[:s1].tolist() == list(range(s1)) and got[len(got) - s2:].tolist() == list(range(N - s2, N))
+        pooled = O.average_pool(ref["C"][h], wl.pool_kernel)
+        rep.mid_ties += check_selection(got[s1:len(got) - s2], want[s1:len(want) - s2], pooled, f"unit {u} middle")
+
+
+def compare_pool_rows(cache: tk.Cache, wl: W.Workload, b: int, r: int, k, v) -> None:
+    """The gathered segments hold exactly the source rows at the GPU's own retained positions (bit-exact copy)."""
+    N = wl.seq_lens[b]
+    for h in range(wl.n_kv_heads):
+        u = unit_index(wl, b, r, h)
+        idx = torch.from_numpy(cache.retained_indices(u, N))
+        kk = cache.pool_rows("k", u)
+        vv = cache.pool_rows("v", u)
+        assert torch.equal(kk.view(torch.uint8), k[h].cpu()[idx].contiguous().view(torch.uint8)), f"unit {u}: K rows"
+        assert torch.equal(vv.view(torch.uint8), v[h].cpu()[idx].contiguous().view(torch.uint8)), f"unit {u}: V rows"
+
+
+def oracle_decode_steps(wl: W.Workload, b: int, r: int, k, v, idx: list, steps_qkv: list) -> List[np.ndarray]:
+    """Decode outputs of one (sequence, layer): append then attend, step by step."""
+    kc, vc = O.gather_cache(to64(k), to64(v), idx)
+    outs = []
+    for (q, kn, vn) in steps_qkv:
+        O.append_layer(kc, vc, to64(kn[b, r]), to64(vn[b, r]))
+        outs.append(O.decode_layer(to64(q[b, r]), kc, vc))
+    return outs

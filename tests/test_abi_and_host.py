@@ -1,0 +1,101 @@
+"""CPU-side checks: the C-ABI library loads and exports every declared symbol,
+and its host-only logic (argument validation, planning, Eq. 16 / Eq. 17 helpers)
+agrees with the oracle and with closed forms.  No kernel is launched here."""
+import ctypes as C
+import os
+import re
+
+import pytest
+
+from oracle import taskkv_oracle as O
+from paper_2501_15113_b200 import workloads as W
+
+ROOT = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
+
+
+@pytest.fixture(scope="module")
+def tk():
+    import __graft_entry__ as g
+    g.build()
+    from paper_2501_15113_b200 import binding
+    return binding
+
+
+def declared_functions():
+    text = open(os.path.join(ROOT, "include", "taskkv.h")).read()
+    text = re.sub(r"/\*.*?\*/", "", text, flags=re.S)
+    return sorted(set(re.findall(r"\b(taskkv_[a-z_0-9]+)\s*\(", text)))
+
+
+def test_every_declared_symbol_is_exported(tk):
+    names = declared_functions()
+    assert len(names) >= 18
+    for n in names:
+        assert hasattr(tk.lib, n), f"{n} is declared in taskkv.h but not exported"
+
+
+def test_params_struct_layout_matches_header(tk):
+    p = tk.taskkv_params()
+    tk.lib.taskkv_params_default(C.byref(p))
+    assert (p.top_t, p.pool_kernel, p.sink, p.recent, p.window) == (256, 7, 16, 256, 32)
+    assert abs(p.beta - 0.25) < 1e-7 and p.m_top == 4 and p.promote_center == 1 and p.force_class == -1
+    assert p.dtype == tk.BF16
+
+
+def test_hetero_count_matches_oracle(tk):
+    for n in (8, 32, 40):
+        for beta in (0.2, 0.25, 0.3, 0.35, 0.4):
+            for m in (0, 1, 4, 6):
+                for R in (1, 2, 5, 32):
+                    for r in range(R):
+                        assert tk.taskkv_hetero_count(n, beta, m, R, r) == \
+                            O.hetero_count(n, float(C.c_float(beta).value), m, R, r)
+
+
+def test_mid_budget_matches_oracle(tk):
+    for N in (512, 30000, 131072):
+        for n, h in ((8, 0), (8, 2), (8, 3), (32, 5), (8, 8)):
+            for frac in (0.1, 0.4, 0.6, 1.0):
+                B = frac * n * N
+                assert tk.taskkv_mid_budget(B, N, h, n, 4, 256) == O.mid_budget(B, N, h, n, 4, 256)
+
+
+def test_plan_matches_closed_forms(tk):
+    from paper_2501_15113_b200 import configs
+    for wl in (configs.config1_toy(), configs.config2_llama2(), configs.config3_llama3(),
+               configs.config4_mistral(), configs.config5_sweep(2, 256)):
+        info = tk.taskkv_plan(tk.params_from_workload(wl))
+        U = wl.batch * wl.n_layers * wl.n_kv_heads
+        assert info.n_units == U
+        assert info.retained_rows == wl.retained_rows()
+        assert info.pool_rows == wl.retained_rows() + U * wl.decode_steps
+        es = wl.elem_size
+        assert info.cache_bytes >= 2 * info.pool_rows * wl.head_dim * es
+    # config 3 keeps 40 % of the full cache (Sec. V-E budget), never more
+    wl = configs.config3_llama3()
+    full = wl.n_layers * wl.n_kv_heads * wl.seq_lens[0]
+    assert 0.399 < wl.retained_rows() / full <= 0.4
+
+
+def test_invalid_arguments_are_rejected_before_any_launch(tk):
+    wl = W.toy()
+    good = dict(n_layers=1, n_heads=8, n_kv_heads=8, head_dim=64, seq_lens=[512], sink=4, recent=32,
+                mid_budget=32, window=16, dtype="f32")
+    tk.taskkv_plan(tk.Params(**good))
+    bad = [dict(head_dim=96), dict(n_kv_heads=3), dict(window=0), dict(window=1024), dict(seq_lens=[8]),
+           dict(top_t=5000), dict(pool_kernel=4), dict(sink=-1), dict(n_heads=8 * 16, n_kv_heads=8),
+           dict(mid_budget=-2), dict(force_class=7), dict(seq_lens=[0])]
+    for override in bad:
+        kw = dict(good)
+        kw.update(override)
+        with pytest.raises(tk.TaskKVError) as ei:
+            tk.taskkv_plan(tk.Params(**kw))
+        assert ei.value.status == tk.EINVAL, override
+    # null pointers never reach the device
+    h = C.c_void_p()
+    assert tk.lib.taskkv_compress_ex(None, None, None, None, None, 0, None, 0, None, C.byref(h)) == tk.EINVAL
+    assert tk.lib.taskkv_decode(None, None, None, None, None) == tk.EINVAL
+    assert tk.lib.taskkv_append(None, None, None, None) == tk.EINVAL
+    assert tk.lib.taskkv_cache_query(None, 0, None, 0) == tk.EINVAL
+    assert tk.lib.taskkv_status_str(tk.ESTATE) == b"cache in wrong state"
+    assert wl.retained_rows() == 3 * 512 + 5 * 68

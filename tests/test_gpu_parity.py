@@ -1,0 +1,216 @@
+"""GPU parity: the CUDA library (through its C ABI) against the CPU oracle on
+the same seeded inputs, element by element."""
+import numpy as np
+import pytest
+import torch
+
+from oracle import taskkv_oracle as O
+from paper_2501_15113_b200 import workloads as W
+
+pytestmark = pytest.mark.gpu
+
+DEV = "cuda:0"
+
+
+def _tk():
+    from paper_2501_15113_b200 import binding
+    return binding
+
+
+def _parity():
+    from tests import parity
+    return parity
+
+
+def run_workload(wl: W.Workload, layers=None, decode_steps=None, check_pool=True, force_class=-1,
+                 check_scores=True):
+    """Compress + decode on the GPU, oracle on the chosen (b, r) pairs, compare everything."""
+    tk, P = _tk(), _parity()
+    qs, ks, vs = W.materialize(wl, DEV)
+    steps = wl.decode_steps if decode_steps is None else decode_steps
+    params = tk.params_from_workload(wl, max_new_tokens=steps, force_class=force_class)
+    cache = tk.taskkv_compress_ex(params, qs, ks, vs)
+    assert cache.status() == 0
+    rep = P.Report()
+    scores = cache.query(tk.Q_SCORES) if check_scores else None
+    topt = cache.query(tk.Q_TOPT)
+    pairs = layers if layers is not None else [(b, r) for b in range(wl.batch) for r in range(wl.n_layers)]
+    refs = {}
+    for (b, r) in pairs:
+        ref = P.oracle_layer(wl, b, r, qs[b][r], ks[b][r], vs[b][r], force_class=force_class)
+        refs[(b, r)] = ref
+        P.compare_layer(cache, wl, b, r, ref, rep, scores=scores, topt=topt)
+        if check_pool:
+            P.compare_pool_rows(cache, wl, b, r, ks[b][r], vs[b][r])
+    # totals the host planned must match what the device produced
+    off = cache.query(tk.Q_OFFSETS)
+    cap = cache.query(tk.Q_CAPACITY)
+    assert off[-1] == cache.info.pool_rows == int(cap.sum())
+    assert int(cache.lengths().sum()) == cache.info.retained_rows == wl.retained_rows() or force_class != -1
+
+    # decode: append + attend, every step compared on the chosen layers
+    step_inputs = [W.gen_decode_step(wl, s, DEV) for s in range(steps)]
+    outs = []
+    for (q, kn, vn) in step_inputs:
+        cache.taskkv_append(kn, vn)
+        outs.append(cache.taskkv_decode(q))
+    assert cache.status() == 0
+    tol = P.TOL_OUT[wl.dtype]
+    for (b, r) in pairs:
+        if rep.class_near_ties and any(f"b={b} r={r}" in n for n in rep.notes):
+            continue
+        want = P.oracle_decode_steps(wl, b, r, ks[b][r], vs[b][r], refs[(b, r)]["idx"], step_inputs)
+        for s in range(steps):
+            err = float(np.abs(P.to64(outs[s][b, r]) - want[s]).max())
+            rep.max_out_abs = max(rep.max_out_abs, err)
+            assert err < tol, f"decode step {s} (b={b}, r={r}): max abs err {err:.3e} >= {tol}"
+    lens = cache.lengths()
+    assert int(lens.sum()) == int(cache.info.retained_rows) + steps * int(cache.info.n_units) or force_class != -1
+    print(f"\n[{wl.name}] units={rep.units} topt_ties={rep.topt_ties} mid_ties={rep.mid_ties} "
+          f"class_near_ties={rep.class_near_ties} max_score_rel={rep.max_score_rel:.2e} "
+          f"max_sem_rel={rep.max_sem_rel:.2e} max_out_abs={rep.max_out_abs:.2e}")
+    cache.close()
+    return rep
+
+
+def small(name, *, n, n_kv, d, N, L, s1, s2, k, dtype, R=1, B=1, t=256, pool=7, nh=1, steps=3, seed=11,
+          variance=None, seq_lens=None, promote=True):
+    lens = seq_lens if seq_lens is not None else [N] * B
+    wl = W.Workload(name=name, batch=len(lens), n_layers=R, n_heads=n, n_kv_heads=n_kv, head_dim=d, seq_lens=lens,
+                    dtype=dtype, sink=s1, recent=s2, window=L, mid_budget=[k] * R,
+                    n_hetero=[[nh] * R for _ in lens], decode_steps=steps, top_t=t, pool_kernel=pool,
+                    promote_center=promote, seed=seed,
+                    variance=variance if variance is not None else (1.0 if dtype == "f32" else 1.0 / np.sqrt(d)),
+                    plant_offset=1.0)
+    wl.planted = W._choose_planted(wl)
+    return wl
+
+
+def test_toy_config_exact():
+    """Config 1: MHA 8 x 64, 512 tokens, fp32, planted heads 2 and 5, 16 decode steps."""
+    wl = W.toy()
+    rep = run_workload(wl)
+    assert rep.topt_ties == 0 and rep.mid_ties == 0 and rep.class_near_ties == 0
+
+
+def test_toy_config_without_pooling():
+    wl = W.toy()
+    wl.pool_kernel = 1
+    run_workload(wl)
+
+
+CASES = [
+    # tiles and ragged tails, both dtypes and head dims
+    dict(n=4, n_kv=4, d=128, N=2341, L=32, s1=4, s2=64, k=100, dtype="bf16"),
+    dict(n=4, n_kv=4, d=64, N=1500, L=16, s1=4, s2=32, k=77, dtype="bf16"),
+    dict(n=4, n_kv=4, d=128, N=1283, L=16, s1=3, s2=50, k=64, dtype="f32"),
+    dict(n=4, n_kv=4, d=64, N=3000, L=32, s1=0, s2=17, k=129, dtype="f32"),
+    # grouped queries: G = 2, 4, 8 and a single KV head
+    dict(n=8, n_kv=4, d=128, N=1100, L=32, s1=4, s2=64, k=50, dtype="bf16"),
+    dict(n=16, n_kv=4, d=128, N=2100, L=32, s1=4, s2=64, k=50, dtype="bf16"),
+    dict(n=16, n_kv=2, d=64, N=900, L=16, s1=4, s2=64, k=50, dtype="f32", nh=0),
+    dict(n=4, n_kv=1, d=128, N=700, L=32, s1=4, s2=64, k=50, dtype="bf16", nh=0),
+    # degenerate budgets and windows
+    dict(n=4, n_kv=4, d=64, N=90, L=8, s1=40, s2=60, k=10, dtype="f32"),          # N <= sink + recent
+    dict(n=4, n_kv=4, d=64, N=600, L=8, s1=4, s2=32, k=0, dtype="f32"),           # no middle activations
+    dict(n=4, n_kv=4, d=64, N=600, L=8, s1=4, s2=32, k=10 ** 6, dtype="bf16"),    # budget covers the middle
+    dict(n=4, n_kv=4, d=64, N=200, L=8, s1=4, s2=32, k=20, dtype="f32", t=1000),  # t >= N
+    dict(n=4, n_kv=4, d=64, N=300, L=1, s1=4, s2=32, k=20, dtype="f32"),          # one-row window
+    dict(n=2, n_kv=2, d=64, N=128, L=128, s1=4, s2=32, k=20, dtype="f32", nh=0),  # window = whole sequence
+    dict(n=4, n_kv=4, d=64, N=1000, L=8, s1=4, s2=32, k=20, dtype="bf16", nh=4),  # every head heterogeneous
+    dict(n=4, n_kv=4, d=64, N=1000, L=8, s1=4, s2=32, k=20, dtype="bf16", nh=0, promote=False),
+    # several layers and a ragged batch
+    dict(n=8, n_kv=2, d=128, N=0, L=32, s1=4, s2=128, k=256, dtype="bf16", R=3, seq_lens=[1500, 2049, 1024], nh=1),
+]
+
+
+@pytest.mark.parametrize("case", CASES, ids=[f"case{i}" for i in range(len(CASES))])
+def test_shapes_and_edge_cases(case):
+    wl = small("case", **case)
+    run_workload(wl)
+
+
+def test_every_head_heterogeneous_is_full_attention():
+    """force_class = 1: the cache is the whole K/V and decode is textbook attention."""
+    wl = small("full", n=8, n_kv=4, d=128, N=1111, L=32, s1=4, s2=64, k=50, dtype="bf16")
+    tk = _tk()
+    qs, ks, vs = W.materialize(wl, DEV)
+    params = tk.params_from_workload(wl, max_new_tokens=0, force_class=1)
+    cache = tk.taskkv_compress_ex(params, qs, ks, vs)
+    assert cache.lengths().tolist() == [1111] * 4 and cache.classes().tolist() == [1] * 4
+    q, _, _ = W.gen_decode_step(wl, 0, DEV)
+    out = cache.taskkv_decode(q)
+    ref = torch.nn.functional.scaled_dot_product_attention(
+        q[0, 0].double().cpu().reshape(4, 2, 128), ks[0][0].double().cpu(), vs[0][0].double().cpu())
+    err = (out[0, 0].double().cpu() - ref.reshape(8, 128)).abs().max().item()
+    assert err < 2e-2
+
+
+def test_decode_prefix_lengths():
+    """A caller-supplied lengths array attends over a prefix of every segment."""
+    tk, P = _tk(), _parity()
+    wl = small("prefix", n=4, n_kv=4, d=64, N=700, L=8, s1=4, s2=32, k=20, dtype="f32")
+    qs, ks, vs = W.materialize(wl, DEV)
+    cache = tk.taskkv_compress_ex(tk.params_from_workload(wl, max_new_tokens=0), qs, ks, vs)
+    lens = cache.lengths()
+    pre = np.maximum(1, lens // 3).astype(np.int32)
+    q, _, _ = W.gen_decode_step(wl, 0, DEV)
+    out = cache.taskkv_decode(q, lengths=torch.from_numpy(pre).to(DEV))
+    ref = P.oracle_layer(wl, 0, 0, qs[0][0], ks[0][0], vs[0][0])
+    kc, vc = O.gather_cache(P.to64(ks[0][0]), P.to64(vs[0][0]), ref["idx"])
+    kc = [kc[u][:pre[u]] for u in range(4)]
+    vc = [vc[u][:pre[u]] for u in range(4)]
+    want = O.decode_layer(P.to64(q[0, 0]), kc, vc)
+    assert np.abs(P.to64(out[0, 0]) - want).max() < 1e-5
+
+
+def test_append_beyond_capacity_sets_status():
+    tk = _tk()
+    wl = small("cap", n=4, n_kv=4, d=64, N=300, L=8, s1=4, s2=32, k=20, dtype="f32")
+    qs, ks, vs = W.materialize(wl, DEV)
+    cache = tk.taskkv_compress_ex(tk.params_from_workload(wl, max_new_tokens=1), qs, ks, vs)
+    _, kn, vn = W.gen_decode_step(wl, 0, DEV)
+    cache.taskkv_append(kn, vn)
+    assert cache.status() == 0
+    before = cache.lengths().copy()
+    cache.taskkv_append(kn, vn)
+    assert cache.status() == tk.ESTATE
+    assert cache.lengths().tolist() == before.tolist()
+
+
+def test_compress_is_deterministic():
+    tk = _tk()
+    wl = small("det", n=8, n_kv=4, d=128, N=3333, L=32, s1=4, s2=64, k=200, dtype="bf16", R=2)
+    qs, ks, vs = W.materialize(wl, DEV)
+    res = []
+    for _ in range(2):
+        cache = tk.taskkv_compress_ex(tk.params_from_workload(wl, max_new_tokens=0), qs, ks, vs)
+        res.append((cache.query(tk.Q_SCORES).copy(), cache.query(tk.Q_SEMVEC).copy(),
+                    cache.query(tk.Q_INDICES).copy(), cache.lengths().copy()))
+        cache.close()
+    for a, b in zip(res[0], res[1]):
+        assert np.array_equal(a, b)
+
+
+def test_flat_entry_point_and_host_buffers():
+    """taskkv_compress (flat form) and the host-buffer calls give the same cache as the _ex call."""
+    tk = _tk()
+    wl = small("flat", n=8, n_kv=8, d=128, N=2000, L=32, s1=16, s2=256, k=100, dtype="bf16", R=2, nh=2)
+    # the flat call applies Eq. 16 itself: beta .25, m 4 over 8 heads and 2 layers -> 2 then 4
+    wl.n_hetero = [[tk.taskkv_hetero_count(8, 0.25, 4, 2, r) for r in range(2)]]
+    qs, ks, vs = W.materialize(wl, DEV)
+    ref = tk.taskkv_compress_ex(tk.params_from_workload(wl, max_new_tokens=4096), qs, ks, vs)
+    flat = tk.taskkv_compress(qs[0], ks[0], vs[0], sink=16, recent=256, mid_budget=100, window=32)
+    params = tk.params_from_workload(wl, max_new_tokens=4096)
+    host = tk.taskkv_compress_host(params, [t.cpu().pin_memory() for t in qs], [t.cpu().pin_memory() for t in ks],
+                                   [t.cpu().pin_memory() for t in vs])
+    for other in (flat, host):
+        assert other.lengths().tolist() == ref.lengths().tolist()
+        assert other.classes().tolist() == ref.classes().tolist()
+        assert np.array_equal(other.query(tk.Q_SEMVEC), ref.query(tk.Q_SEMVEC))
+    q, kn, vn = W.gen_decode_step(wl, 0, DEV)
+    ref.taskkv_append(kn, vn)
+    want = ref.taskkv_decode(q)
+    out_h = torch.empty(q.shape, dtype=q.dtype).pin_memory()
+    host.taskkv_decode_host(q.cpu().pin_memory(), kn.cpu().pin_memory(), vn.cpu().pin_memory(), out_h)
+    assert torch.equal(out_h, want.cpu())
