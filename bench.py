@@ -1,0 +1,406 @@
+#!/usr/bin/env python
+"""Benchmark of the Task-KV hot path on B200.
+
+One "step" is one pass of the whole path over one batch of synthetic input:
+prefill-side compression of every layer (window scores, top-t + semantic
+vectors, separator, middle top-k, gather) followed by the workload's decode
+steps (append + ragged attention each).  Default workload: the Llama-2-7B-shaped
+stack (32 layers, MHA 32 x 128, 32768 tokens, bf16, 256 decode steps).
+
+Prints ONE JSON line.  `value` is decode attention steps per second (all layers
+per step), measured on the device with inputs resident in HBM; compression
+tokens per second is reported beside it, and `e2e` repeats the measurement
+through the host-buffer entry points with the copies inside the timed region.
+`--impl reference` times the CPU oracle on a bounded sample instead.
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import statistics
+import subprocess
+import sys
+import time
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+if ROOT not in sys.path:
+    sys.path.insert(0, ROOT)
+
+import torch  # noqa: E402
+
+NOMINAL_HBM_GBS = 8000.0
+FALLBACK_HBM_GBS = 6650.0
+
+
+def load_peaks():
+    path = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    try:
+        with open(path) as fh:
+            d = json.load(fh)
+        return float(d["hbm_gbs"]), "measured"
+    except Exception:
+        return FALLBACK_HBM_GBS, "fallback"
+
+
+def get_workload(name: str, args):
+    from paper_2501_15113_b200 import configs
+    if name == "llama2":
+        return configs.config2_llama2(seq_len=args.seq_len or 32768, n_layers=args.layers or 32,
+                                      decode_steps=args.decode_steps or 256)
+    if name == "llama3":
+        return configs.config3_llama3(seq_len=args.seq_len or 131072, n_layers=args.layers or 32,
+                                      decode_steps=args.decode_steps or 128)
+    if name == "mistral":
+        return configs.config4_mistral(n_layers=args.layers or 32, decode_steps=args.decode_steps or 512)
+    if name == "toy":
+        return configs.config1_toy()
+    if name.startswith("sweep"):
+        _, h, k = name.split(":")
+        return configs.config5_sweep(int(h), int(k), decode_steps=args.decode_steps or 64)
+    raise SystemExit(f"unknown workload {name}")
+
+
+class ClockSampler:
+    QUERY = ("index,clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.active,"
+             "clocks_event_reasons.hw_slowdown,clocks_event_reasons.hw_thermal_slowdown,"
+             "clocks_event_reasons.sw_thermal_slowdown,clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, gpu_index: int):
+        self.gpu = gpu_index
+        self.proc = None
+
+    def start(self):
+        try:
+            self.proc = subprocess.Popen(
+                ["nvidia-smi", f"--query-gpu={self.QUERY}", "--format=csv,noheader,nounits", "-lms", "100",
+                 "-i", str(self.gpu)], stdout=subprocess.PIPE, stderr=subprocess.DEVNULL, text=True)
+        except Exception:
+            self.proc = None
+
+    def stop(self):
+        if self.proc is None:
+            return {"sm_mhz": None, "sm_max_mhz": None, "reasons": ["nvidia-smi unavailable"]}
+        self.proc.terminate()
+        try:
+            out, _ = self.proc.communicate(timeout=5)
+        except Exception:
+            self.proc.kill()
+            out = ""
+        sm, mx, reasons = [], [], set()
+        names = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
+        for ln in out.splitlines():
+            f = [x.strip() for x in ln.split(",")]
+            if len(f) < 9:
+                continue
+            try:
+                sm.append(float(f[1]))
+                mx.append(float(f[2]))
+            except ValueError:
+                continue
+            for nm, val in zip(names, f[5:9]):
+                if val.lower().startswith("active"):
+                    reasons.add(nm)
+        return {"sm_mhz": statistics.median(sm) if sm else None, "sm_max_mhz": max(mx) if mx else None,
+                "samples": len(sm), "reasons": sorted(reasons)}
+
+
+def algorithmic_bytes(wl, info):
+    """Bytes the method itself must move: compress and one decode step."""
+    es, d = wl.elem_size, wl.head_dim
+    G = wl.group
+    comp = 0
+    for b in range(wl.batch):
+        N = wl.seq_lens[b]
+        for r in range(wl.n_layers):
+            h = wl.full_heads(b, r)
+            kept = wl.kept_len(b, r)
+            per_unit = N * d * es + G * wl.window * d * es + 12 * N + min(wl.top_t, N) * d * es
+            comp += wl.n_kv_heads * per_unit + 4 * d * es * (h * N + (wl.n_kv_heads - h) * kept)
+    return comp
+
+
+def run_ours(args):
+    import __graft_entry__ as ge
+    ge.build()
+    from paper_2501_15113_b200 import binding as tk
+    from paper_2501_15113_b200 import workloads as W
+
+    rank = int(os.environ.get("RANK", "0"))
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    local = int(os.environ.get("LOCAL_RANK", "0"))
+    if world > 1:
+        import torch.distributed as dist
+        dist.init_process_group("nccl", device_id=torch.device(f"cuda:{local}"))
+    torch.cuda.set_device(local)
+    dev = f"cuda:{local}"
+    peak, peak_kind = load_peaks()
+
+    wl = get_workload(args.workload, args)
+    wl.seed += 1000 * rank            # weak scaling: every rank owns an independent replica of the batch
+    wl.planted = W._choose_planted(wl)
+    S = wl.decode_steps
+    qs, ks, vs = W.materialize(wl, dev)
+    steps_in = [W.gen_decode_step(wl, s, dev) for s in range(S)]
+    params = tk.params_from_workload(wl, max_new_tokens=S)
+    info = tk.taskkv_plan(params)
+    cache_mem = torch.empty(int(info.cache_bytes), dtype=torch.uint8, device=dev)
+    work_mem = torch.empty(int(info.workspace_bytes), dtype=torch.uint8, device=dev)
+    out = torch.empty_like(steps_in[0][0])
+    stream = torch.cuda.current_stream()
+
+    def one_pass(ev=None):
+        if ev:
+            ev[0].record(stream)
+        cache = tk.taskkv_compress_ex(params, qs, ks, vs, cache_mem=cache_mem, workspace_mem=work_mem)
+        if ev:
+            ev[1].record(stream)
+        for (q, kn, vn) in steps_in:
+            cache.taskkv_append(kn, vn)
+            cache.taskkv_decode(q, out=out)
+        if ev:
+            ev[2].record(stream)
+        return cache
+
+    for _ in range(args.warmup):
+        one_pass().close()
+    torch.cuda.synchronize()
+
+    def barrier():
+        if world > 1:
+            import torch.distributed as dist
+            dist.barrier()
+        torch.cuda.synchronize()
+
+    sampler = ClockSampler(local)
+    launches0 = tk.taskkv_launch_count()
+    evs = [[torch.cuda.Event(enable_timing=True) for _ in range(3)] for _ in range(args.steps)]
+    barrier()
+    sampler.start()
+    t0 = torch.cuda.Event(enable_timing=True)
+    t1 = torch.cuda.Event(enable_timing=True)
+    t0.record(stream)
+    caches = []
+    for i in range(args.steps):
+        caches.append(one_pass(evs[i]))
+    t1.record(stream)
+    barrier()
+    clocks = sampler.stop()
+    launches = tk.taskkv_launch_count() - launches0
+    status = caches[-1].status()
+    for c in caches:
+        c.close()
+    total_ms = t0.elapsed_time(t1)
+    comp_ms = sum(e[0].elapsed_time(e[1]) for e in evs)
+    dec_ms = sum(e[1].elapsed_time(e[2]) for e in evs)
+    if world > 1:
+        import torch.distributed as dist
+        t = torch.tensor([total_ms, comp_ms, dec_ms], device=dev, dtype=torch.float64)
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+        total_ms, comp_ms, dec_ms = t.tolist()
+
+    # per-kernel durations: one more identical pass with every launch bracketed by events on its stream
+    tk.taskkv_timing_enable(True)
+    one_pass().close()
+    recs = tk.taskkv_timing_collect()
+    tk.taskkv_timing_enable(False)
+    per = {}
+    for name, ms in recs:
+        a = per.setdefault(name, [0, 0.0])
+        a[0] += 1
+        a[1] += ms
+
+    K = args.steps
+    tokens = sum(wl.seq_lens)
+    es, d = wl.elem_size, wl.head_dim
+    comp_bytes = algorithmic_bytes(wl, info)
+    U = int(info.n_units)
+    # decode step s (1-based) reads K and V rows of every segment once: retained rows + s appended per unit
+    dec_bytes_avg = 2 * d * es * (int(info.retained_rows) + U * (S + 1) / 2.0)
+    dec_step_ms = dec_ms / (K * S)
+    comp_pass_ms = comp_ms / K
+    value = world * 1e3 / dec_step_ms
+    comp_tps = world * tokens * 1e3 / comp_pass_ms
+
+    kern = {}
+    for name, (n, ms) in per.items():
+        kern[name] = {"launches": n, "avg_ms": ms / n, "total_ms": ms}
+    attn = kern.get("decode_attn", {"avg_ms": float("nan")})
+    attn_gbs = dec_bytes_avg / (attn["avg_ms"] * 1e-3) / 1e9
+    comp_kernel_ms = sum(v["total_ms"] for k, v in kern.items() if not k.startswith(("decode", "append")))
+
+    line = {
+        "metric": "decode attn steps/s (compress tokens/s beside it)",
+        "value": value, "unit": "steps/s", "n_gpus": world, "steps": K, "warmup": args.warmup,
+        "ms_per_step": total_ms / K, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
+        "dtype": wl.dtype, "data": "synthetic",
+        "config": dict(wl.describe(), l2="inputs (>=8 GB of K, >=3 GB retained cache) exceed the 126 MB L2",
+                       step="compress all layers + decode_steps x (append + attention)"),
+        "decode_ms_per_step": dec_step_ms, "compress_ms": comp_pass_ms, "compress_tokens_per_s": comp_tps,
+        "hbm": {
+            "peak_gbs": peak, "peak_kind": peak_kind, "nominal_gbs": NOMINAL_HBM_GBS,
+            "decode_gbs": dec_bytes_avg / (dec_step_ms * 1e-3) / 1e9,
+            "decode_frac": dec_bytes_avg / (dec_step_ms * 1e-3) / 1e9 / peak,
+            "compress_gbs": comp_bytes / (comp_pass_ms * 1e-3) / 1e9,
+            "compress_frac": comp_bytes / (comp_pass_ms * 1e-3) / 1e9 / peak,
+            "decode_bytes_per_step": dec_bytes_avg, "compress_bytes": comp_bytes,
+        },
+        "roofline": {"bound": "hbm", "kernel": "decode_attn", "achieved": attn_gbs, "peak": peak, "unit": "GB/s",
+                     "frac": attn_gbs / peak, "peak_kind": peak_kind, "traffic": None,
+                     "avg_launch_ms": attn["avg_ms"]},
+        "kernels": kern, "compress_kernel_ms": comp_kernel_ms,
+        "gpu_launches": launches, "device_status": status, "clocks": clocks,
+    }
+
+    if rank == 0 and not args.no_e2e:
+        line["e2e"] = run_e2e(tk, wl, params, qs, ks, vs, steps_in, world)
+    if rank == 0 and world == 1 and not args.no_cpu:
+        line["cpu_baseline"] = cpu_baseline(wl, qs, ks, vs, steps_in)
+    if rank == 0:
+        print(json.dumps(line))
+    if world > 1:
+        import torch.distributed as dist
+        dist.barrier()
+        dist.destroy_process_group()
+
+
+def run_e2e(tk, wl, params, qs, ks, vs, steps_in, world):
+    """Same metric through the host-buffer entry points: pinned host inputs, copies inside the timed region."""
+    hq = [t.cpu().pin_memory() for t in qs]
+    hk = [t.cpu().pin_memory() for t in ks]
+    hv = [t.cpu().pin_memory() for t in vs]
+    hsteps = [tuple(t.cpu().pin_memory() for t in s) for s in steps_in]
+    hout = torch.empty(steps_in[0][0].shape, dtype=steps_in[0][0].dtype).pin_memory()
+    torch.cuda.synchronize()
+    cache = tk.taskkv_compress_host(params, hq, hk, hv)      # warm-up (allocations, page mapping)
+    for s in range(min(3, len(hsteps))):
+        cache.taskkv_decode_host(hsteps[s][0], None, None, hout)
+    cache.close()
+    torch.cuda.synchronize()
+    t0 = time.perf_counter()
+    cache = tk.taskkv_compress_host(params, hq, hk, hv)
+    t1 = time.perf_counter()
+    for (q, kn, vn) in hsteps:
+        cache.taskkv_decode_host(q, kn, vn, hout)
+    t2 = time.perf_counter()
+    cache.close()
+    S = len(hsteps)
+    h2d = sum(t.numel() * t.element_size() for t in hq + hk + hv) + \
+        sum(t.numel() * t.element_size() for s in hsteps for t in s)
+    d2h = S * hout.numel() * hout.element_size()
+    return {"value": world * S / (t2 - t1), "unit": "steps/s", "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h,
+            "compress_tokens_per_s": sum(wl.seq_lens) / (t1 - t0), "compress_s": t1 - t0,
+            "decode_ms_per_step": (t2 - t1) * 1e3 / S, "timing": "host wall clock around synchronous calls"}
+
+
+def oracle_sample(wl, qs, ks, vs, steps_in, n_units: int, n_steps: int):
+    """Times the oracle on the first n_units KV heads of layer 0 of sequence 0 and
+    n_steps decode steps of those units; returns seconds (compress, decode) and the scale factors."""
+    import numpy as np
+    from oracle import taskkv_oracle as O
+    G = wl.group
+    n_units = min(n_units, wl.n_kv_heads)
+    q = qs[0][0][:n_units * G].double().cpu().numpy()
+    k = ks[0][0][:n_units].double().cpu().numpy()
+    v = vs[0][0][:n_units].double().cpu().numpy()
+    t0 = time.perf_counter()
+    ref = O.compress_layer(q, k, v, n_hetero=min(wl.n_hetero[0][0], n_units), sink=wl.sink, recent=wl.recent,
+                           mid=wl.mid_budget[0], top_t=wl.top_t, pool_kernel=wl.pool_kernel,
+                           promote_center=wl.promote_center)
+    kc, vc = O.gather_cache(k, v, ref["idx"])
+    t1 = time.perf_counter()
+    for s in range(n_steps):
+        qd, kn, vn = steps_in[s]
+        O.append_layer(kc, vc, kn[0, 0, :n_units].double().cpu().numpy(), vn[0, 0, :n_units].double().cpu().numpy())
+        O.decode_layer(qd[0, 0, :n_units * G].double().cpu().numpy(), kc, vc)
+    t2 = time.perf_counter()
+    rows_sample = int(sum(len(i) for i in ref["idx"]))
+    return (t1 - t0), (t2 - t1), n_units, rows_sample
+
+
+def cpu_threads():
+    try:
+        from threadpoolctl import threadpool_info
+        n = [p.get("num_threads", 1) for p in threadpool_info()]
+        return max(n) if n else 1
+    except Exception:
+        return os.cpu_count() or 1
+
+
+def cpu_baseline(wl, qs, ks, vs, steps_in):
+    n_steps = min(4, len(steps_in))
+    comp_s, dec_s, n_units, rows_sample = oracle_sample(wl, qs, ks, vs, steps_in, 8, n_steps)
+    U = wl.batch * wl.n_layers * wl.n_kv_heads
+    tokens_units = sum(wl.seq_lens[b] * wl.n_layers * wl.n_kv_heads for b in range(wl.batch))
+    # compress cost scales with keys scanned; decode cost with rows read
+    comp_full = comp_s * tokens_units / (n_units * wl.seq_lens[0])
+    dec_full = (dec_s / n_steps) * wl.retained_rows() / rows_sample
+    return {"value": 1.0 / dec_full, "unit": "steps/s", "cores": cpu_threads(), "kind": "oracle",
+            "compress_tokens_per_s": sum(wl.seq_lens) / comp_full,
+            "sample": f"{n_units} KV heads of layer 0 (sequence 0): compress {comp_s:.2f} s, {n_steps} decode steps "
+                      f"{dec_s:.2f} s; scaled by keys scanned ({U} units) and by rows read ({wl.retained_rows()} rows)"}
+
+
+def run_reference(args):
+    """The oracle, as it stands, on the host cores: each step is a bounded sample of the workload."""
+    rank = int(os.environ.get("RANK", "0"))
+    if rank != 0:
+        return
+    from paper_2501_15113_b200 import workloads as W
+    wl = get_workload(args.workload, args)
+    n_units = 4
+    sub = W.Workload(**{**wl.__dict__})
+    qs, ks, vs = [], [], []
+    q, k, v = W.gen_layer(wl, 0, 0, "cpu")
+    qs.append(q[None])
+    ks.append(k[None])
+    vs.append(v[None])
+    steps_in = [W.gen_decode_step(wl, s, "cpu") for s in range(2)]
+    times = []
+    for i in range(args.warmup + args.steps):
+        c, d, nu, rows = oracle_sample(sub, qs, ks, vs, steps_in, n_units, 2)
+        if i >= args.warmup:
+            times.append((c, d, nu, rows))
+    comp_s = statistics.mean(t[0] for t in times)
+    dec_s = statistics.mean(t[1] for t in times) / 2
+    nu, rows = times[0][2], times[0][3]
+    tokens_units = sum(wl.seq_lens[b] * wl.n_layers * wl.n_kv_heads for b in range(wl.batch))
+    comp_full = comp_s * tokens_units / (nu * wl.seq_lens[0])
+    dec_full = dec_s * wl.retained_rows() / rows
+    value = 1.0 / dec_full
+    sample = (f"{nu} KV heads of layer 0 per step: oracle compress {comp_s:.2f} s + 2 decode steps; scaled to the "
+              f"whole workload by keys scanned and rows read")
+    line = {"impl": "reference", "metric": "decode attn steps/s (compress tokens/s beside it)", "value": value,
+            "unit": "steps/s", "n_gpus": args.gpus, "steps": args.steps, "warmup": args.warmup,
+            "ms_per_step": (comp_s + 2 * dec_s) * 1e3, "higher_is_better": True, "scaling": "weak",
+            "vs_baseline": None, "dtype": "f64", "data": "synthetic", "config": wl.describe(),
+            "compress_tokens_per_s": sum(wl.seq_lens) / comp_full,
+            "cpu_baseline": {"value": value, "unit": "steps/s", "cores": cpu_threads(), "kind": "oracle",
+                             "sample": sample},
+            "e2e": {"value": value, "unit": "steps/s", "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0}}
+    print(json.dumps(line))
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=5)
+    ap.add_argument("--warmup", type=int, default=3)
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--workload", default="llama2")
+    ap.add_argument("--seq-len", type=int, default=0)
+    ap.add_argument("--layers", type=int, default=0)
+    ap.add_argument("--decode-steps", type=int, default=0)
+    ap.add_argument("--no-e2e", action="store_true")
+    ap.add_argument("--no-cpu", action="store_true")
+    args = ap.parse_args()
+    import __graft_entry__ as ge
+    ge.build()          # the workload tables use the library's host-only schedule / budget helpers
+    if args.impl == "reference":
+        run_reference(args)
+    else:
+        run_ours(args)
+
+
+if __name__ == "__main__":
+    main()
