@@ -120,7 +120,7 @@ CASES = [
     dict(n=4, n_kv=4, d=64, N=1000, L=8, s1=4, s2=32, k=20, dtype="bf16", nh=4),  # every head heterogeneous
     dict(n=4, n_kv=4, d=64, N=1000, L=8, s1=4, s2=32, k=20, dtype="bf16", nh=0, promote=False),
     # several layers and a ragged batch
-    dict(n=8, n_kv=2, d=128, N=0, L=32, s1=4, s2=128, k=256, dtype="bf16", R=3, seq_lens=[1500, 2049, 1024], nh=1),
+    dict(n=16, n_kv=4, d=128, N=0, L=32, s1=4, s2=128, k=256, dtype="bf16", R=3, seq_lens=[1500, 2049, 1024], nh=1),
 ]
 
 
