@@ -161,6 +161,34 @@ taskkv_status taskkv_decode(const void* q, taskkv_cache* c, const int32_t* lengt
 taskkv_status taskkv_decode_host(const void* q, const void* k_new, const void* v_new, taskkv_cache* c,
                                  void* out, taskkv_stream stream);
 
+/* Decode attention without any allocation.  (The paper has no counterpart to
+ * this call; it exists for deployment.)  Some callers may not allocate device
+ * memory: code running inside a serving engine that has already given all
+ * device memory to its own pool, or a latency-critical decode loop in which
+ * the device-wide synchronisation of cudaMalloc / cudaFree is unacceptable.
+ * This call computes the same result as taskkv_decode over caller-held pools,
+ * with its split-K scratch in a fixed 32 MiB device array that is part of the
+ * library image (every GPU that loads the library holds it until the process
+ * exits).  It calls no cudaMalloc, cudaFree or other allocating routine.
+ *   q, out    [n_units * group][head_dim] in `dtype`; unit u serves query heads u*group .. u*group+group-1
+ *   k_pool, v_pool   rows of head_dim elements; unit u owns rows seg_off[u] .. seg_off[u] + lengths[u] - 1
+ *   seg_off   device int64 [n_units];  lengths  device int32 [n_units]
+ *   max_len   host-side upper bound of every lengths[u] (sets the work split)
+ * Limits: group in {1,2,4,8}, head_dim in {64,128}, and
+ * n_units * group * (head_dim + 2) * 4 bytes must fit the 32 MiB scratch;
+ * beyond that the call returns TASKKV_EINVAL (with a line on stderr) and
+ * launches nothing.
+ * The first call on each device looks up the array's device address (with that
+ * device current); make that first call before starting any stream capture.
+ * All calls share the one array and it keeps the previous call's contents
+ * (every slot a call reads is first rewritten by that call): calls whose
+ * kernels may overlap on the GPU - different streams or host threads - race
+ * and must be serialised by the caller. */
+taskkv_status taskkv_decode_noalloc(const void* q, const void* k_pool, const void* v_pool,
+                                    const int64_t* seg_off, const int32_t* lengths, int32_t n_units,
+                                    int32_t group, int32_t head_dim, int32_t dtype, int32_t max_len,
+                                    void* out, taskkv_stream stream);
+
 /* Synchronising device-to-host reads for tests and reports. */
 #define TASKKV_Q_LENGTHS   0   /* int32 [n_units] */
 #define TASKKV_Q_CLASSES   1   /* int32 [n_units] */

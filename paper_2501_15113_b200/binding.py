@@ -67,6 +67,8 @@ lib.taskkv_decode.argtypes = [_vp, _vp, _vp, _vp, _vp]
 lib.taskkv_decode.restype = C.c_int32
 lib.taskkv_decode_host.argtypes = [_vp, _vp, _vp, _vp, _vp, _vp]
 lib.taskkv_decode_host.restype = C.c_int32
+lib.taskkv_decode_noalloc.argtypes = [_vp, _vp, _vp, _vp, _vp] + [C.c_int32] * 5 + [_vp, _vp]
+lib.taskkv_decode_noalloc.restype = C.c_int32
 lib.taskkv_cache_query_bytes.argtypes = [_vp, C.c_int32]
 lib.taskkv_cache_query_bytes.restype = C.c_int64
 lib.taskkv_cache_query.argtypes = [_vp, C.c_int32, _vp, C.c_size_t]
@@ -326,6 +328,24 @@ def taskkv_compress(q_win: torch.Tensor, k: torch.Tensor, v: torch.Tensor, *, si
     params = Params(n_layers=R, n_heads=n, n_kv_heads=n_kv, head_dim=d, seq_lens=[N], sink=sink, recent=recent,
                     mid_budget=mid_budget, window=window, dtype=BF16, beta=beta, m_top=m, max_new_tokens=4096)
     return Cache(h.value, params, {})
+
+
+def taskkv_decode_noalloc(q: torch.Tensor, k_pool: torch.Tensor, v_pool: torch.Tensor, seg_off: torch.Tensor,
+                          lengths: torch.Tensor, *, group: int, max_len: int,
+                          out: Optional[torch.Tensor] = None, stream=None) -> torch.Tensor:
+    """Decode attention over caller-held pools with the library's fixed scratch: no
+    allocation happens inside the call (`out` is allocated here, by torch, only if
+    the caller passes none).  q: [n_units * group, d]; pools: [rows, d];
+    seg_off int64 [n_units]; lengths int32 [n_units]; max_len >= lengths.max()."""
+    if out is None:
+        out = torch.empty_like(q)
+    d = q.shape[-1]
+    n_units = lengths.numel()
+    dtype = BF16 if q.dtype == torch.bfloat16 else F32
+    _check(lib.taskkv_decode_noalloc(q.data_ptr(), k_pool.data_ptr(), v_pool.data_ptr(), seg_off.data_ptr(),
+                                     lengths.data_ptr(), n_units, group, d, dtype, max_len, out.data_ptr(),
+                                     _stream_handle(stream)), "taskkv_decode_noalloc")
+    return out
 
 
 def params_from_workload(wl, max_new_tokens: Optional[int] = None, **overrides) -> Params:
