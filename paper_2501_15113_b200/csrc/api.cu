@@ -110,7 +110,7 @@ taskkv_status make_plan(const taskkv_params* p, HostPlan& hp) {
   hp.c_total = c_total;
   hp.rows = G * p->window;
   hp.rows_pad = (hp.rows + 15) / 16 * 16;
-  hp.chunks_max = (hp.max_N + kScoreChunk - 1) / kScoreChunk;
+  hp.chunks_max = ((hp.max_N + 2047) / 2048) * 4;   // partial-statistic slots per unit (covers both window paths)
 
   const size_t es = p->dtype == TASKKV_F32 ? 4 : 2;
   const size_t d = p->head_dim;
@@ -392,7 +392,12 @@ taskkv_status taskkv_compress_ex(const taskkv_params* p, const void* const* q_wi
 
   cudaError_t e = cudaMemcpyAsync(c->cache_mem, c->meta.data(), c->hp.meta_bytes, cudaMemcpyHostToDevice, s);
   if (e == cudaSuccess) e = cudaMemsetAsync(c->dp.status, 0, 64, s);
-  if (e == cudaSuccess) e = launch_window_scores(c->dp, p->dtype, c->hp.max_N, s);
+  WindowHostInfo wh;
+  wh.batch = p->batch;
+  wh.seq_lens = c->hp.seq_lens.data();
+  wh.q = q_win;
+  wh.k = k;
+  if (e == cudaSuccess) e = launch_window_scores(c->dp, p->dtype, c->hp.max_N, wh, s);
   if (e == cudaSuccess) e = launch_select(c->dp, p->dtype, s);
   if (e == cudaSuccess) e = launch_separator_plan(c->dp, p->batch * p->n_layers, s);
   if (e == cudaSuccess) e = launch_gather(c->dp, p->dtype, c->hp.info.gather_items, s);

@@ -90,8 +90,19 @@ struct LaunchScope {
   ~LaunchScope() { note_launch_end(id, s); }
 };
 
+// Host-side view of the inputs, for launchers that build per-sequence descriptors.
+struct WindowHostInfo {
+  int batch;
+  const int32_t* seq_lens;      // host [batch]
+  const void* const* q;         // host [batch] device pointers: [R][n][L][d]
+  const void* const* k;         // host [batch] device pointers: [R][n_kv][N_b][d]
+};
+
 // kernel launchers (one per translation unit)
-cudaError_t launch_window_scores(const DeviceProblem& p, int dtype, int max_N, cudaStream_t s);
+cudaError_t launch_window_scores(const DeviceProblem& p, int dtype, int max_N, const WindowHostInfo& h,
+                                 cudaStream_t s);
+bool window_tc_supported(const DeviceProblem& p, int dtype);
+cudaError_t launch_window_scores_tc(const DeviceProblem& p, const WindowHostInfo& h, cudaStream_t s);
 cudaError_t launch_select(const DeviceProblem& p, int dtype, cudaStream_t s);
 cudaError_t launch_separator_plan(const DeviceProblem& p, int n_br, cudaStream_t s);
 cudaError_t launch_decode_plan(const DeviceProblem& p, const int32_t* lengths, cudaStream_t s);

@@ -182,7 +182,10 @@ cudaError_t launch_generic(const DeviceProblem& p, int max_N, cudaStream_t s) {
 
 }  // namespace
 
-cudaError_t launch_window_scores(const DeviceProblem& p, int dtype, int max_N, cudaStream_t s) {
+cudaError_t launch_window_scores(const DeviceProblem& p, int dtype, int max_N, const WindowHostInfo& h,
+                                 cudaStream_t s) {
+  // bf16 with 32 / 64 / 128 window rows runs on the tensor cores; everything else here
+  if (window_tc_supported(p, dtype)) return launch_window_scores_tc(p, h, s);
   if (dtype == TASKKV_F32) {
     return p.d == 64 ? launch_generic<float, 64>(p, max_N, s) : launch_generic<float, 128>(p, max_N, s);
   }

@@ -1,0 +1,494 @@
+// Observation-window scores (Eq. 12, Eq. 13) on the 5th-generation tensor cores,
+// for bf16 inputs with G*L in {32, 64, 128} window rows.
+//
+// The contraction S = Q_win K^T is 2*G*L*d flop per key (32-128 flop per byte of
+// K): too much for the CUDA cores next to an HBM-rate K stream, little for
+// tcgen05.  Each CTA is a persistent, warp-specialised pipeline:
+//   warp 0   TMA producer: K tiles of 128 keys (and the unit's Q rows) into
+//            128-byte-swizzled shared memory, completion on mbarriers
+//   warp 1   tcgen05.mma issuer (one elected thread), accumulators in TMEM,
+//            double buffered; tcgen05.commit frees the smem stage and hands the
+//            accumulator to the epilogue
+//   warps 2-5  epilogue: tcgen05.ld, softmax arithmetic in fp32 registers
+// Two passes, as Eq. 13 needs every row's normaliser before rows can be summed:
+//   pass 1 (row statistics)  D[row, key] = Q K^T: a TMEM lane is a window row, so
+//     the running max / exp-sum over keys stays inside one thread.  With fewer
+//     than 128 rows the Q block is replicated over the lane quadrants, each
+//     against its own sub-tile of keys, so all four epilogue warps share the work.
+//   pass 2 (scores)  D[key, row] = K Q^T: a TMEM lane is a key, so
+//     C[key] = sum_rows exp2(s - max_row) / Z_row is a sum inside one thread.
+// Scores are kept in log2 units (scale log2(e)/sqrt(d)); exp is one ex2.approx.
+// Every wait is bounded: on time-out the CTA records TASKKV_ETIMEOUT, stops
+// issuing work, releases its TMEM and returns.
+#include <cuda.h>
+
+#include "common.cuh"
+
+namespace taskkv {
+
+namespace {
+
+constexpr int kTile = 128;          // keys per tile (UMMA M in pass 2, key sub-tiles in pass 1)
+constexpr int kChunk = 2048;        // keys per work item
+constexpr int kStages = 4;          // K tiles in flight per CTA
+constexpr int kThreads = 192;
+constexpr uint32_t kTmemCols = 256; // two accumulator stages of up to 128 columns
+constexpr uint32_t kSpinLimit = 1u << 22;
+
+struct TcArgs {
+  int pass;          // 1: row statistics, 2: scores
+  int u0;            // first unit of this sequence
+  int n_local;       // units in this launch (layers * kv heads)
+  int N;             // sequence length
+  int chunks;        // work items per unit
+};
+
+// ---------------------------------------------------------------- PTX wrappers
+__device__ __forceinline__ uint32_t smem_u32(const void* p) {
+  return (uint32_t)__cvta_generic_to_shared(p);
+}
+__device__ __forceinline__ void mbar_init(uint32_t bar, uint32_t count) {
+  asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(bar), "r"(count));
+}
+__device__ __forceinline__ void mbar_expect_tx(uint32_t bar, uint32_t bytes) {
+  asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar), "r"(bytes) : "memory");
+}
+__device__ __forceinline__ void mbar_arrive(uint32_t bar) {
+  asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(bar) : "memory");
+}
+__device__ __forceinline__ uint32_t mbar_try_wait(uint32_t bar, uint32_t parity) {
+  uint32_t ok;
+  asm volatile(
+      "{\n\t.reg .pred p;\n\t"
+      "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
+      "selp.u32 %0, 1, 0, p;\n\t}"
+      : "=r"(ok)
+      : "r"(bar), "r"(parity)
+      : "memory");
+  return ok;
+}
+// Bounded wait: false if the CTA is aborting or the limit ran out (which raises the abort flag).
+__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile int* abort_flag) {
+  for (uint32_t spin = 0;; ++spin) {
+    if (mbar_try_wait(bar, parity)) return true;
+    if (*abort_flag) return false;
+    if (spin > kSpinLimit) {
+      *abort_flag = 1;
+      return false;
+    }
+    if (spin > 32) __nanosleep(128);
+  }
+}
+__device__ __forceinline__ void tma_load_2d(uint32_t dst, const CUtensorMap* map, int x, int y, uint32_t bar) {
+  asm volatile(
+      "cp.async.bulk.tensor.2d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3}], [%4];"
+      ::"r"(dst), "l"(map), "r"(x), "r"(y), "r"(bar)
+      : "memory");
+}
+__device__ __forceinline__ void tc_alloc(uint32_t smem_dst, uint32_t cols) {
+  asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_dst), "r"(cols)
+               : "memory");
+}
+__device__ __forceinline__ void tc_relinquish() {
+  asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+}
+__device__ __forceinline__ void tc_dealloc(uint32_t taddr, uint32_t cols) {
+  asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(taddr), "r"(cols) : "memory");
+}
+__device__ __forceinline__ void tc_fence_before() { asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory"); }
+__device__ __forceinline__ void tc_fence_after() { asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory"); }
+__device__ __forceinline__ void tc_mma(uint32_t d_tmem, uint64_t adesc, uint64_t bdesc, uint32_t idesc,
+                                       uint32_t accumulate) {
+  asm volatile(
+      "{\n\t.reg .pred p;\n\t"
+      "setp.ne.b32 p, %4, 0;\n\t"
+      "tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, p;\n\t}"
+      ::"r"(d_tmem), "l"(adesc), "l"(bdesc), "r"(idesc), "r"(accumulate)
+      : "memory");
+}
+__device__ __forceinline__ void tc_commit(uint32_t bar) {
+  asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(bar) : "memory");
+}
+__device__ __forceinline__ void tc_ld32(uint32_t taddr, uint32_t* r) {
+  asm volatile(
+      "tcgen05.ld.sync.aligned.32x32b.x32.b32 "
+      "{%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15, "
+      "%16, %17, %18, %19, %20, %21, %22, %23, %24, %25, %26, %27, %28, %29, %30, %31}, [%32];"
+      : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7]),
+        "=r"(r[8]), "=r"(r[9]), "=r"(r[10]), "=r"(r[11]), "=r"(r[12]), "=r"(r[13]), "=r"(r[14]), "=r"(r[15]),
+        "=r"(r[16]), "=r"(r[17]), "=r"(r[18]), "=r"(r[19]), "=r"(r[20]), "=r"(r[21]), "=r"(r[22]), "=r"(r[23]),
+        "=r"(r[24]), "=r"(r[25]), "=r"(r[26]), "=r"(r[27]), "=r"(r[28]), "=r"(r[29]), "=r"(r[30]), "=r"(r[31])
+      : "r"(taddr)
+      : "memory");
+}
+__device__ __forceinline__ void tc_wait_ld() { asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory"); }
+__device__ __forceinline__ float ex2(float x) {
+  float y;
+  asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
+  return y;
+}
+
+// Shared-memory matrix descriptor: K-major operand, rows of 128 bytes, 128-byte
+// swizzle, 8-row groups 1024 bytes apart.
+__device__ __forceinline__ uint64_t smem_desc(uint32_t saddr) {
+  uint64_t d = 0;
+  d |= (uint64_t)((saddr & 0x3FFFFu) >> 4);       // start address
+  d |= (uint64_t)(1024u >> 4) << 32;              // stride between 8-row groups
+  d |= (uint64_t)1 << 46;                         // descriptor version of this architecture
+  d |= (uint64_t)2 << 61;                         // 128-byte swizzle
+  return d;
+}
+// Instruction descriptor: bf16 x bf16 -> fp32, both operands K-major, M x N tile.
+__device__ __forceinline__ uint32_t instr_desc(int M, int N) {
+  return (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(N >> 3) << 17) | ((uint32_t)(M >> 4) << 24);
+}
+
+template <int D>
+struct TcSmem {
+  static constexpr int KB = D / 64;                       // 128-byte k-blocks per row
+  static constexpr int kTileBytes = KB * kTile * 128;     // one K tile
+  static constexpr int kQRowsMax = 224;                   // 256 - rows at rows = 32
+  static constexpr int kQBytes = KB * kQRowsMax * 128;
+  static constexpr int kBytes = kStages * kTileBytes + kQBytes + 4 * 128 * (int)sizeof(float2) + 256 + 1024;
+};
+
+template <int D, int PASS>
+__global__ void __launch_bounds__(kThreads, 1)
+window_tc_kernel(const __grid_constant__ CUtensorMap tmap_k, const __grid_constant__ CUtensorMap tmap_q,
+                 DeviceProblem p, TcArgs a) {
+  constexpr int KB = TcSmem<D>::KB;
+  extern __shared__ unsigned char smem_raw[];
+  // 1024-byte alignment: the swizzle pattern is a function of the address bits
+  unsigned char* smem = reinterpret_cast<unsigned char*>(((uintptr_t)smem_raw + 1023) & ~(uintptr_t)1023);
+  unsigned char* sK = smem;                                         // [kStages][KB][128 rows][128 B]
+  unsigned char* sQ = sK + kStages * TcSmem<D>::kTileBytes;         // [KB][q_rows][128 B]
+  float2* sStat = reinterpret_cast<float2*>(sQ + TcSmem<D>::kQBytes);  // [4 warps][128]
+  uint64_t* bars = reinterpret_cast<uint64_t*>(reinterpret_cast<unsigned char*>(sStat) + 4 * 128 * sizeof(float2));
+  // barrier slots: full[0..3], empty[4..7], q_full 8, q_empty 9, tmem_full 10..11, tmem_empty 12..13
+  uint32_t* s_tmem = reinterpret_cast<uint32_t*>(bars + 14);
+  volatile int* s_abort = reinterpret_cast<volatile int*>(s_tmem + 1);
+
+  const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+  const int rows = p.rows;                  // 32, 64 or 128
+  const int rep = 128 / rows;               // lane quadrant groups in pass 1
+  const int zero_before = 128 - rows;       // zero rows ahead of Q in its buffer
+  const int q_rows = 256 - rows;            // rows of the Q buffer per k-block
+  const int N = a.N, L = p.L;
+  const uint32_t bar0 = smem_u32(bars);
+  auto BAR = [&](int i) { return bar0 + 8u * (uint32_t)i; };
+
+  if (tid == 0) {
+    for (int i = 0; i < kStages; ++i) { mbar_init(BAR(i), 1); mbar_init(BAR(4 + i), 1); }
+    mbar_init(BAR(8), 1);
+    mbar_init(BAR(9), 1);
+    mbar_init(BAR(10), 1);
+    mbar_init(BAR(11), 1);
+    mbar_init(BAR(12), 4);
+    mbar_init(BAR(13), 4);
+    *s_abort = 0;
+    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+  }
+  // zero the Q buffer once: its padding rows are never written again
+  for (int i = tid; i < TcSmem<D>::kQBytes / 16; i += kThreads) reinterpret_cast<uint4*>(sQ)[i] = make_uint4(0, 0, 0, 0);
+  asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+  if (warp == 1) {
+    tc_alloc(smem_u32(s_tmem), kTmemCols);
+    tc_relinquish();
+  }
+  tc_fence_before();
+  __syncthreads();
+  tc_fence_after();
+  const uint32_t tmem_base = *s_tmem;
+
+  const int n_items = a.n_local * a.chunks;
+  const float scale2 = kLog2e * rsqrtf((float)D);
+
+  if (warp == 0) {
+    // ------------------------------------------------------------ TMA producer
+    if (lane == 0) {
+      int stage = 0;
+      uint32_t phase = 0, qphase = 0;
+      bool ok = true;
+      for (int it = blockIdx.x; it < n_items && ok; it += gridDim.x) {
+        const int lu = it / a.chunks, ch = it % a.chunks;
+        const int key0 = ch * kChunk;
+        const int ntiles = (min(N, key0 + kChunk) - key0 + kTile - 1) / kTile;
+        ok = mbar_wait(BAR(9), qphase ^ 1, s_abort);
+        if (!ok) break;
+        mbar_expect_tx(BAR(8), (uint32_t)(KB * rows * 128));
+        for (int kb = 0; kb < KB; ++kb)
+          tma_load_2d(smem_u32(sQ + (size_t)kb * q_rows * 128 + (size_t)zero_before * 128), &tmap_q, kb * 64,
+                      lu * rows, BAR(8));
+        qphase ^= 1;
+        for (int t = 0; t < ntiles; ++t) {
+          ok = mbar_wait(BAR(4 + stage), phase ^ 1, s_abort);
+          if (!ok) break;
+          mbar_expect_tx(BAR(stage), (uint32_t)TcSmem<D>::kTileBytes);
+          for (int kb = 0; kb < KB; ++kb)
+            tma_load_2d(smem_u32(sK + (size_t)stage * TcSmem<D>::kTileBytes + (size_t)kb * kTile * 128), &tmap_k,
+                        kb * 64, lu * N + key0 + t * kTile, BAR(stage));
+          if (++stage == kStages) { stage = 0; phase ^= 1; }
+        }
+      }
+    }
+  } else if (warp == 1) {
+    // ------------------------------------------------------------ MMA issuer
+    if (lane == 0) {
+      int stage = 0, acc = 0;
+      uint32_t phase = 0, qphase = 0, accphase = 0;
+      const uint32_t idesc = instr_desc(128, rows);
+      bool ok = true;
+      for (int it = blockIdx.x; it < n_items && ok; it += gridDim.x) {
+        const int ch = it % a.chunks;
+        const int key0 = ch * kChunk;
+        const int ntiles = (min(N, key0 + kChunk) - key0 + kTile - 1) / kTile;
+        ok = mbar_wait(BAR(8), qphase, s_abort);
+        if (!ok) break;
+        qphase ^= 1;
+        for (int t = 0; t < ntiles; ++t) {
+          ok = mbar_wait(BAR(stage), phase, s_abort);
+          if (!ok) break;
+          ok = mbar_wait(BAR(12 + acc), accphase ^ 1, s_abort);
+          if (!ok) break;
+          tc_fence_after();
+          const uint32_t d_tmem = tmem_base + (uint32_t)acc * 128u;
+          const uint32_t kt = smem_u32(sK + (size_t)stage * TcSmem<D>::kTileBytes);
+          const uint32_t qb = smem_u32(sQ);
+          if (PASS == 1) {
+            // quadrant w: Q rows on lanes [w*rows, (w+1)*rows), keys [w*rows, (w+1)*rows) of the tile
+            uint32_t first = 1;
+            for (int w = 0; w < rep; ++w)
+              for (int kb = 0; kb < KB; ++kb)
+#pragma unroll
+                for (int k = 0; k < 4; ++k) {
+                  const uint64_t ad = smem_desc(qb + (uint32_t)(kb * q_rows * 128 + (zero_before - w * rows) * 128 + k * 32));
+                  const uint64_t bd = smem_desc(kt + (uint32_t)(kb * kTile * 128 + w * rows * 128 + k * 32));
+                  tc_mma(d_tmem, ad, bd, idesc, first ? 0u : 1u);
+                  first = 0;
+                }
+          } else {
+            for (int kb = 0; kb < KB; ++kb)
+#pragma unroll
+              for (int k = 0; k < 4; ++k) {
+                const uint64_t ad = smem_desc(kt + (uint32_t)(kb * kTile * 128 + k * 32));
+                const uint64_t bd = smem_desc(qb + (uint32_t)(kb * q_rows * 128 + zero_before * 128 + k * 32));
+                tc_mma(d_tmem, ad, bd, idesc, (kb | k) ? 1u : 0u);
+              }
+          }
+          tc_commit(BAR(4 + stage));     // smem stage free once these MMAs have read it
+          tc_commit(BAR(10 + acc));      // accumulator ready for the epilogue
+          if (++stage == kStages) { stage = 0; phase ^= 1; }
+          if (++acc == 2) { acc = 0; accphase ^= 1; }
+        }
+        tc_commit(BAR(9));               // Q buffer free once the item's MMAs are done
+      }
+    }
+  } else {
+    // ------------------------------------------------------------ epilogue (4 warps = 128 TMEM lanes)
+    const int quad = warp & 3;                      // TMEM lane quadrant this warp may read
+    const int tl = quad * 32 + lane;                // TMEM lane of this thread
+    float2* myStat = sStat + (warp - 2) * 128;
+    int acc = 0;
+    uint32_t accphase = 0;
+    bool ok = true;
+    for (int it = blockIdx.x; it < n_items && ok; it += gridDim.x) {
+      const int lu = it / a.chunks, ch = it % a.chunks;
+      const int u = a.u0 + lu;
+      const int key0 = ch * kChunk;
+      const int ntiles = (min(N, key0 + kChunk) - key0 + kTile - 1) / kTile;
+      float m_run = -INFINITY, z_run = 0.f;         // pass 1 state of this thread's (row, key quadrant)
+      const int row1 = tl % rows, kq = tl / rows;   // pass 1: window row and key sub-tile
+      if (PASS == 2) {
+        __syncwarp();
+        for (int i = lane; i < rows; i += 32)
+          myStat[i] = reinterpret_cast<const float2*>(p.stat)[(size_t)u * p.rows_pad + i];
+        __syncwarp();
+      }
+      for (int t = 0; t < ntiles; ++t) {
+        ok = mbar_wait(BAR(10 + acc), accphase, s_abort);
+        if (!ok) break;
+        tc_fence_after();
+        const uint32_t taddr = tmem_base + ((uint32_t)(quad * 32) << 16) + (uint32_t)acc * 128u;
+        const int tbase = key0 + t * kTile;
+        if (PASS == 1) {
+          const int pos = N - L + (row1 % L);       // last key this window row may see
+          const int jb = tbase + kq * rows;
+          for (int c0 = 0; c0 < rows; c0 += 32) {
+            uint32_t r[32];
+            tc_ld32(taddr + (uint32_t)c0, r);
+            tc_wait_ld();
+            float x[32];
+            float cm = -INFINITY;
+#pragma unroll
+            for (int c = 0; c < 32; ++c) {
+              const int j = jb + c0 + c;
+              x[c] = (j <= pos && j < N) ? __uint_as_float(r[c]) * scale2 : -INFINITY;
+              cm = fmaxf(cm, x[c]);
+            }
+            if (cm > m_run) {
+              z_run *= ex2(m_run - cm);
+              m_run = cm;
+            }
+            if (m_run > -INFINITY) {
+              float zs = 0.f;
+#pragma unroll
+              for (int c = 0; c < 32; ++c) zs += ex2(x[c] - m_run);
+              z_run += zs;
+            }
+          }
+        } else {
+          const int j = tbase + tl;                 // this thread's key
+          const bool tail = (tbase + kTile - 1 > N - L);
+          float csum = 0.f;
+          for (int c0 = 0; c0 < rows; c0 += 32) {
+            uint32_t r[32];
+            tc_ld32(taddr + (uint32_t)c0, r);
+            tc_wait_ld();
+            if (!tail) {
+#pragma unroll
+              for (int c = 0; c < 32; ++c) {
+                const float2 ms = myStat[c0 + c];
+                csum = fmaf(ex2(fmaf(__uint_as_float(r[c]), scale2, -ms.x)), ms.y, csum);
+              }
+            } else {
+#pragma unroll
+              for (int c = 0; c < 32; ++c) {
+                const float2 ms = myStat[c0 + c];
+                const bool vis = (j < N) && (j <= N - L + ((c0 + c) % L));
+                if (vis) csum = fmaf(ex2(fmaf(__uint_as_float(r[c]), scale2, -ms.x)), ms.y, csum);
+              }
+            }
+          }
+          if (j < N) p.C[p.c_off[u] + j] = csum * (1.0f / (float)rows);
+        }
+        tc_fence_before();
+        __syncwarp();
+        if (lane == 0) mbar_arrive(BAR(12 + acc));
+        if (++acc == 2) { acc = 0; accphase ^= 1; }
+      }
+      if (PASS == 1 && ok) {
+        // slot = chunk * rep + key quadrant
+        reinterpret_cast<float2*>(p.stat_part)[((size_t)u * p.chunks_max + (size_t)ch * rep + kq) * p.rows_pad + row1] =
+            make_float2(m_run, z_run);
+      }
+    }
+  }
+
+  // ---------------------------------------------------------------- teardown
+  tc_fence_before();
+  __syncthreads();
+  if (warp == 1) {
+    tc_fence_after();
+    tc_dealloc(tmem_base, kTmemCols);
+  }
+  if (tid == 0 && *s_abort) set_status(p.status, TASKKV_ETIMEOUT);
+}
+
+// Combine the partial statistics of one unit: slots = chunks * rep per row.
+__global__ void window_tc_reduce_kernel(DeviceProblem p, int u0, int slots) {
+  const int u = u0 + blockIdx.x;
+  const int row = threadIdx.x;
+  if (row >= p.rows) return;
+  const float2* part = reinterpret_cast<const float2*>(p.stat_part) + (size_t)u * p.chunks_max * p.rows_pad;
+  float M = -INFINITY;
+  for (int c = 0; c < slots; ++c) M = fmaxf(M, part[(size_t)c * p.rows_pad + row].x);
+  float z = 0.f;
+  for (int c = 0; c < slots; ++c) {
+    const float2 o = part[(size_t)c * p.rows_pad + row];
+    if (o.x > -INFINITY) z += o.y * exp2f(o.x - M);
+  }
+  reinterpret_cast<float2*>(p.stat)[(size_t)u * p.rows_pad + row] =
+      z > 0.f ? make_float2(M, 1.0f / z) : make_float2(0.f, 0.f);
+}
+
+typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
+                                  const cuuint64_t*, const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave,
+                                  CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+
+EncodeTiledFn encode_fn() {
+  static EncodeTiledFn fn = nullptr;
+  static bool tried = false;
+  if (!tried) {
+    tried = true;
+    void* ptr = nullptr;
+    cudaDriverEntryPointQueryResult qres;
+    if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &ptr, cudaEnableDefault, &qres) == cudaSuccess &&
+        qres == cudaDriverEntryPointSuccess)
+      fn = reinterpret_cast<EncodeTiledFn>(ptr);
+  }
+  return fn;
+}
+
+// 2-D bf16 tensor [rows_total][d], box of 64 elements x box_rows rows, 128-byte swizzle.
+bool make_map(CUtensorMap* map, const void* base, int d, uint64_t rows_total, int box_rows) {
+  EncodeTiledFn fn = encode_fn();
+  if (!fn) return false;
+  const cuuint64_t dims[2] = {(cuuint64_t)d, (cuuint64_t)rows_total};
+  const cuuint64_t strides[1] = {(cuuint64_t)d * 2};
+  const cuuint32_t box[2] = {64u, (cuuint32_t)box_rows};
+  const cuuint32_t estr[2] = {1u, 1u};
+  return fn(map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<void*>(base), dims, strides, box, estr,
+            CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_128B,
+            CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+}
+
+template <int D>
+cudaError_t launch_tc_d(const DeviceProblem& p, const WindowHostInfo& h, cudaStream_t s) {
+  static int n_sm = 0;
+  if (n_sm == 0) {
+    int dev = 0;
+    cudaGetDevice(&dev);
+    cudaDeviceGetAttribute(&n_sm, cudaDevAttrMultiProcessorCount, dev);
+    if (n_sm <= 0) n_sm = 148;
+  }
+  const int smem = TcSmem<D>::kBytes;
+  cudaError_t e = cudaFuncSetAttribute(window_tc_kernel<D, 1>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem);
+  if (e != cudaSuccess) return e;
+  e = cudaFuncSetAttribute(window_tc_kernel<D, 2>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem);
+  if (e != cudaSuccess) return e;
+  const int per_seq = p.R * p.n_kv;
+  const int rep = 128 / p.rows;
+  for (int b = 0; b < h.batch; ++b) {
+    const int N = h.seq_lens[b];
+    CUtensorMap mk, mq;
+    if (!make_map(&mk, h.k[b], D, (uint64_t)per_seq * (uint64_t)N, kTile)) return cudaErrorUnknown;
+    if (!make_map(&mq, h.q[b], D, (uint64_t)per_seq * (uint64_t)p.rows, p.rows)) return cudaErrorUnknown;
+    TcArgs a;
+    a.u0 = b * per_seq;
+    a.n_local = per_seq;
+    a.N = N;
+    a.chunks = (N + kChunk - 1) / kChunk;
+    const int items = a.n_local * a.chunks;
+    const int grid = items < n_sm ? items : n_sm;
+    a.pass = 1;
+    {
+      LaunchScope ls(K_WINDOW_TC, s);
+      window_tc_kernel<D, 1><<<grid, kThreads, smem, s>>>(mk, mq, p, a);
+    }
+    {
+      LaunchScope ls(K_WINDOW_REDUCE, s);
+      window_tc_reduce_kernel<<<per_seq, 128, 0, s>>>(p, a.u0, a.chunks * rep);
+    }
+    a.pass = 2;
+    {
+      LaunchScope ls(K_WINDOW_TC, s);
+      window_tc_kernel<D, 2><<<grid, kThreads, smem, s>>>(mk, mq, p, a);
+    }
+    e = cudaGetLastError();
+    if (e != cudaSuccess) return e;
+  }
+  return cudaSuccess;
+}
+
+}  // namespace
+
+bool window_tc_supported(const DeviceProblem& p, int dtype) {
+  return dtype == TASKKV_BF16 && (p.rows == 32 || p.rows == 64 || p.rows == 128) && p.L <= p.rows &&
+         encode_fn() != nullptr;
+}
+
+cudaError_t launch_window_scores_tc(const DeviceProblem& p, const WindowHostInfo& h, cudaStream_t s) {
+  return p.d == 64 ? launch_tc_d<64>(p, h, s) : launch_tc_d<128>(p, h, s);
+}
+
+}  // namespace taskkv

@@ -105,6 +105,9 @@ CASES = [
     dict(n=4, n_kv=4, d=64, N=1500, L=16, s1=4, s2=32, k=77, dtype="bf16"),
     dict(n=4, n_kv=4, d=128, N=1283, L=16, s1=3, s2=50, k=64, dtype="f32"),
     dict(n=4, n_kv=4, d=64, N=3000, L=32, s1=0, s2=17, k=129, dtype="f32"),
+    dict(n=4, n_kv=4, d=64, N=5000, L=32, s1=4, s2=64, k=300, dtype="bf16"),       # tensor-core path, d = 64
+    dict(n=8, n_kv=2, d=128, N=6500, L=32, s1=4, s2=64, k=300, dtype="bf16", nh=0),  # 128 window rows, 4 chunks
+    dict(n=4, n_kv=2, d=128, N=4097, L=32, s1=4, s2=64, k=300, dtype="bf16", nh=0),  # 64 window rows
     # grouped queries: G = 2, 4, 8 and a single KV head
     dict(n=8, n_kv=4, d=128, N=1100, L=32, s1=4, s2=64, k=50, dtype="bf16"),
     dict(n=16, n_kv=4, d=128, N=2100, L=32, s1=4, s2=64, k=50, dtype="bf16"),
