@@ -29,7 +29,7 @@ struct HostPlan {
   size_t o_status, o_len, o_cap, o_seg, o_cls, o_dist, o_sem, o_idx, o_goff, o_doff, o_pacc, o_pml, o_kpool,
       o_vpool;
   // inside the workspace
-  size_t w_C, w_spart, w_stat, w_topt;
+  size_t w_C, w_spart, w_stat, w_topt, w_sync;
 };
 
 int32_t hetero_count_impl(int32_t n, float beta, int32_t m, int32_t R, int32_t r) {
@@ -110,7 +110,7 @@ taskkv_status make_plan(const taskkv_params* p, HostPlan& hp) {
   hp.c_total = c_total;
   hp.rows = G * p->window;
   hp.rows_pad = (hp.rows + 15) / 16 * 16;
-  hp.chunks_max = ((hp.max_N + 2047) / 2048) * 4;   // partial-statistic slots per unit (covers both window paths)
+  hp.chunks_max = ((hp.max_N + kTcChunk - 1) / kTcChunk) * 4;   // partial-statistic slots per unit (covers both window paths)
 
   const size_t es = p->dtype == TASKKV_F32 ? 4 : 2;
   const size_t d = p->head_dim;
@@ -144,6 +144,7 @@ taskkv_status make_plan(const taskkv_params* p, HostPlan& hp) {
   hp.w_spart = take((size_t)U * hp.chunks_max * hp.rows_pad * 8);
   hp.w_stat = take((size_t)U * hp.rows_pad * 8);
   hp.w_topt = take((size_t)U * p->top_t * 4);
+  hp.w_sync = take((size_t)U * 2 * 4);
   const size_t work_bytes = o;
 
   hp.info.n_units = U;
@@ -261,6 +262,7 @@ void fill_device_problem(taskkv_cache* c) {
     d.stat_part = reinterpret_cast<float*>(wm + hp.w_spart);
     d.stat = reinterpret_cast<float*>(wm + hp.w_stat);
     d.topt = reinterpret_cast<int32_t*>(wm + hp.w_topt);
+    d.tc_sync = reinterpret_cast<int32_t*>(wm + hp.w_sync);
   }
 }
 
@@ -626,3 +628,7 @@ int32_t taskkv_timing_collect(int32_t* ids, float* ms, int32_t max) {
 const char* taskkv_timing_name(int32_t id) { return (id >= 0 && id < K_COUNT) ? kKernelNames[id] : "?"; }
 
 }  // extern "C"
+
+extern "C" void taskkv_debug_window_mode(int32_t mode, int32_t chunk, int32_t delay) {
+  taskkv::window_tc_set_mode(mode, chunk, delay);
+}

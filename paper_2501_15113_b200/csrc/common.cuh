@@ -12,7 +12,8 @@ namespace taskkv {
 
 constexpr int kDecodeChunk = 256;                 // rows of one split-K decode item
 constexpr int kGatherRows = 64;                   // rows of one gather item
-constexpr int kScoreChunk = 1024;                 // keys of one window-score work item
+constexpr int kScoreChunk = 1024;                 // keys of one window-score work item (CUDA-core path)
+constexpr int kTcChunk = 1024;                    // keys of one window-score work item (tensor-core path)
 constexpr float kLog2e = 1.4426950408889634f;
 
 // kernel ids for launch counting / timing
@@ -77,6 +78,7 @@ struct DeviceProblem {
   float* stat_part;           // [U][chunks_max][rows_pad][2]
   float* stat;                // [U][rows_pad][2]  (row max in log2 units, 1/Z)
   int32_t* topt;              // [U][top_t]
+  int32_t* tc_sync;           // [2][U] per-unit counters / flags of the tensor-core window path
 };
 
 // launch bookkeeping (api.cu)
@@ -103,6 +105,7 @@ cudaError_t launch_window_scores(const DeviceProblem& p, int dtype, int max_N, c
                                  cudaStream_t s);
 bool window_tc_supported(const DeviceProblem& p, int dtype);
 cudaError_t launch_window_scores_tc(const DeviceProblem& p, const WindowHostInfo& h, cudaStream_t s);
+void window_tc_set_mode(int mode, int chunk, int delay);
 cudaError_t launch_select(const DeviceProblem& p, int dtype, cudaStream_t s);
 cudaError_t launch_separator_plan(const DeviceProblem& p, int n_br, cudaStream_t s);
 cudaError_t launch_decode_plan(const DeviceProblem& p, const int32_t* lengths, cudaStream_t s);

@@ -29,19 +29,35 @@ namespace taskkv {
 namespace {
 
 constexpr int kTile = 128;          // keys per tile (UMMA M in pass 2, key sub-tiles in pass 1)
-constexpr int kChunk = 2048;        // keys per work item
 constexpr int kStages = 4;          // K tiles in flight per CTA
 constexpr int kThreads = 192;
 constexpr uint32_t kTmemCols = 256; // two accumulator stages of up to 128 columns
 constexpr uint32_t kSpinLimit = 1u << 22;
 
+// Work items of one launch (one sequence and one pass): (unit, chunk of chunk_keys keys), unit-major,
+// taken round-robin by the resident CTAs.
 struct TcArgs {
   int pass;          // 1: row statistics, 2: scores
   int u0;            // first unit of this sequence
   int n_local;       // units in this launch (layers * kv heads)
   int N;             // sequence length
   int chunks;        // work items per unit
+  int chunk_keys;    // keys per work item (multiple of 128, >= kTcChunk)
+  int total;         // work items
 };
+
+struct Item {
+  int pass, lu, ch;
+  bool valid;
+};
+__device__ __forceinline__ Item decode_item(const TcArgs& a, int s) {
+  Item it;
+  it.pass = a.pass;
+  it.lu = s / a.chunks;
+  it.ch = s % a.chunks;
+  it.valid = true;
+  return it;
+}
 
 // ---------------------------------------------------------------- PTX wrappers
 __device__ __forceinline__ uint32_t smem_u32(const void* p) {
@@ -147,12 +163,20 @@ template <int D>
 struct TcSmem {
   static constexpr int KB = D / 64;                       // 128-byte k-blocks per row
   static constexpr int kTileBytes = KB * kTile * 128;     // one K tile
-  static constexpr int kQRowsMax = 224;                   // 256 - rows at rows = 32
-  static constexpr int kQBytes = KB * kQRowsMax * 128;
-  static constexpr int kBytes = kStages * kTileBytes + kQBytes + 4 * 128 * (int)sizeof(float2) + 256 + 1024;
+  static constexpr int kQBlockBytes = KB * 128 * 128;     // one Q block (up to 128 rows), double buffered
+  static constexpr int kStatBytes = 4 * 128 * (int)sizeof(float2);
+  static constexpr int kTransBytes = 4 * 32 * 33 * (int)sizeof(float);   // per-warp 32x32 transposition tiles
+  static constexpr int kMergeBytes = 2 * 4 * 128 * (int)sizeof(float2);  // [item parity][warp][row]
+  static constexpr int kBytes =
+      kStages * kTileBytes + 2 * kQBlockBytes + kStatBytes + kTransBytes + kMergeBytes + 256 + 1024;
 };
 
-template <int D, int PASS>
+// barrier slots
+enum : int {
+  B_FULL = 0, B_EMPTY = 4, B_QFULL = 8, B_QEMPTY = 10, B_TFULL = 12, B_TEMPTY = 14, B_EPI = 16, B_COUNT = 17
+};
+
+template <int D>
 __global__ void __launch_bounds__(kThreads, 1)
 window_tc_kernel(const __grid_constant__ CUtensorMap tmap_k, const __grid_constant__ CUtensorMap tmap_q,
                  DeviceProblem p, TcArgs a) {
@@ -160,37 +184,33 @@ window_tc_kernel(const __grid_constant__ CUtensorMap tmap_k, const __grid_consta
   extern __shared__ unsigned char smem_raw[];
   // 1024-byte alignment: the swizzle pattern is a function of the address bits
   unsigned char* smem = reinterpret_cast<unsigned char*>(((uintptr_t)smem_raw + 1023) & ~(uintptr_t)1023);
-  unsigned char* sK = smem;                                         // [kStages][KB][128 rows][128 B]
-  unsigned char* sQ = sK + kStages * TcSmem<D>::kTileBytes;         // [KB][q_rows][128 B]
-  float2* sStat = reinterpret_cast<float2*>(sQ + TcSmem<D>::kQBytes);  // [4 warps][128]
-  uint64_t* bars = reinterpret_cast<uint64_t*>(reinterpret_cast<unsigned char*>(sStat) + 4 * 128 * sizeof(float2));
-  // barrier slots: full[0..3], empty[4..7], q_full 8, q_empty 9, tmem_full 10..11, tmem_empty 12..13
-  uint32_t* s_tmem = reinterpret_cast<uint32_t*>(bars + 14);
+  unsigned char* sK = smem;                                         // [kStages][KB][128 keys][128 B]
+  unsigned char* sQ = sK + kStages * TcSmem<D>::kTileBytes;         // [2][KB][rows][128 B]
+  float2* sStat = reinterpret_cast<float2*>(sQ + 2 * TcSmem<D>::kQBlockBytes);   // [4 warps][128]
+  float* sTrans = reinterpret_cast<float*>(reinterpret_cast<unsigned char*>(sStat) + TcSmem<D>::kStatBytes);
+  float2* sMerge = reinterpret_cast<float2*>(reinterpret_cast<unsigned char*>(sTrans) + TcSmem<D>::kTransBytes);
+  uint64_t* bars = reinterpret_cast<uint64_t*>(reinterpret_cast<unsigned char*>(sMerge) + TcSmem<D>::kMergeBytes);
+  uint32_t* s_tmem = reinterpret_cast<uint32_t*>(bars + B_COUNT);
   volatile int* s_abort = reinterpret_cast<volatile int*>(s_tmem + 1);
 
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
   const int rows = p.rows;                  // 32, 64 or 128
-  const int rep = 128 / rows;               // lane quadrant groups in pass 1
-  const int zero_before = 128 - rows;       // zero rows ahead of Q in its buffer
-  const int q_rows = 256 - rows;            // rows of the Q buffer per k-block
   const int N = a.N, L = p.L;
   const uint32_t bar0 = smem_u32(bars);
   auto BAR = [&](int i) { return bar0 + 8u * (uint32_t)i; };
 
   if (tid == 0) {
-    for (int i = 0; i < kStages; ++i) { mbar_init(BAR(i), 1); mbar_init(BAR(4 + i), 1); }
-    mbar_init(BAR(8), 1);
-    mbar_init(BAR(9), 1);
-    mbar_init(BAR(10), 1);
-    mbar_init(BAR(11), 1);
-    mbar_init(BAR(12), 4);
-    mbar_init(BAR(13), 4);
+    for (int i = 0; i < kStages; ++i) { mbar_init(BAR(B_FULL + i), 1); mbar_init(BAR(B_EMPTY + i), 1); }
+    for (int i = 0; i < 2; ++i) {
+      mbar_init(BAR(B_QFULL + i), 1);
+      mbar_init(BAR(B_QEMPTY + i), 1);
+      mbar_init(BAR(B_TFULL + i), 1);
+      mbar_init(BAR(B_TEMPTY + i), 4);
+    }
+    mbar_init(BAR(B_EPI), 128);
     *s_abort = 0;
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
   }
-  // zero the Q buffer once: its padding rows are never written again
-  for (int i = tid; i < TcSmem<D>::kQBytes / 16; i += kThreads) reinterpret_cast<uint4*>(sQ)[i] = make_uint4(0, 0, 0, 0);
-  asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
   if (warp == 1) {
     tc_alloc(smem_u32(s_tmem), kTmemCols);
     tc_relinquish();
@@ -199,146 +219,153 @@ window_tc_kernel(const __grid_constant__ CUtensorMap tmap_k, const __grid_consta
   __syncthreads();
   tc_fence_after();
   const uint32_t tmem_base = *s_tmem;
-
-  const int n_items = a.n_local * a.chunks;
   const float scale2 = kLog2e * rsqrtf((float)D);
 
   if (warp == 0) {
     // ------------------------------------------------------------ TMA producer
     if (lane == 0) {
-      int stage = 0;
-      uint32_t phase = 0, qphase = 0;
+      int stage = 0, qb = 0;
+      uint32_t phase = 0, qphase[2] = {0, 0};
       bool ok = true;
-      for (int it = blockIdx.x; it < n_items && ok; it += gridDim.x) {
-        const int lu = it / a.chunks, ch = it % a.chunks;
-        const int key0 = ch * kChunk;
-        const int ntiles = (min(N, key0 + kChunk) - key0 + kTile - 1) / kTile;
-        ok = mbar_wait(BAR(9), qphase ^ 1, s_abort);
+      for (int s = blockIdx.x; s < a.total && ok; s += gridDim.x) {
+        const Item it = decode_item(a, s);
+        if (!it.valid) continue;
+        const int key0 = it.ch * a.chunk_keys;
+        const int ntiles = (min(N, key0 + a.chunk_keys) - key0 + kTile - 1) / kTile;
+        ok = mbar_wait(BAR(B_QEMPTY + qb), qphase[qb] ^ 1, s_abort);
         if (!ok) break;
-        mbar_expect_tx(BAR(8), (uint32_t)(KB * rows * 128));
+        mbar_expect_tx(BAR(B_QFULL + qb), (uint32_t)(KB * rows * 128));
         for (int kb = 0; kb < KB; ++kb)
-          tma_load_2d(smem_u32(sQ + (size_t)kb * q_rows * 128 + (size_t)zero_before * 128), &tmap_q, kb * 64,
-                      lu * rows, BAR(8));
-        qphase ^= 1;
+          tma_load_2d(smem_u32(sQ + (size_t)qb * TcSmem<D>::kQBlockBytes + (size_t)kb * rows * 128), &tmap_q, kb * 64,
+                      it.lu * rows, BAR(B_QFULL + qb));
+        qphase[qb] ^= 1;
+        qb ^= 1;
         for (int t = 0; t < ntiles; ++t) {
-          ok = mbar_wait(BAR(4 + stage), phase ^ 1, s_abort);
+          ok = mbar_wait(BAR(B_EMPTY + stage), phase ^ 1, s_abort);
           if (!ok) break;
-          mbar_expect_tx(BAR(stage), (uint32_t)TcSmem<D>::kTileBytes);
+          mbar_expect_tx(BAR(B_FULL + stage), (uint32_t)TcSmem<D>::kTileBytes);
           for (int kb = 0; kb < KB; ++kb)
             tma_load_2d(smem_u32(sK + (size_t)stage * TcSmem<D>::kTileBytes + (size_t)kb * kTile * 128), &tmap_k,
-                        kb * 64, lu * N + key0 + t * kTile, BAR(stage));
+                        kb * 64, it.lu * N + key0 + t * kTile, BAR(B_FULL + stage));
           if (++stage == kStages) { stage = 0; phase ^= 1; }
         }
       }
     }
   } else if (warp == 1) {
-    // ------------------------------------------------------------ MMA issuer
+    // ------------------------------------------------------------ MMA issuer: D[key, row] = K Q^T, both passes
     if (lane == 0) {
-      int stage = 0, acc = 0;
-      uint32_t phase = 0, qphase = 0, accphase = 0;
+      int stage = 0, acc = 0, qb = 0;
+      uint32_t phase = 0, accphase = 0, qphase[2] = {0, 0};
       const uint32_t idesc = instr_desc(128, rows);
       bool ok = true;
-      for (int it = blockIdx.x; it < n_items && ok; it += gridDim.x) {
-        const int ch = it % a.chunks;
-        const int key0 = ch * kChunk;
-        const int ntiles = (min(N, key0 + kChunk) - key0 + kTile - 1) / kTile;
-        ok = mbar_wait(BAR(8), qphase, s_abort);
+      for (int s = blockIdx.x; s < a.total && ok; s += gridDim.x) {
+        const Item it = decode_item(a, s);
+        if (!it.valid) continue;
+        const int key0 = it.ch * a.chunk_keys;
+        const int ntiles = (min(N, key0 + a.chunk_keys) - key0 + kTile - 1) / kTile;
+        ok = mbar_wait(BAR(B_QFULL + qb), qphase[qb], s_abort);
         if (!ok) break;
-        qphase ^= 1;
+        qphase[qb] ^= 1;
+        const uint32_t qbase = smem_u32(sQ + (size_t)qb * TcSmem<D>::kQBlockBytes);
         for (int t = 0; t < ntiles; ++t) {
-          ok = mbar_wait(BAR(stage), phase, s_abort);
+          ok = mbar_wait(BAR(B_FULL + stage), phase, s_abort);
           if (!ok) break;
-          ok = mbar_wait(BAR(12 + acc), accphase ^ 1, s_abort);
+          ok = mbar_wait(BAR(B_TEMPTY + acc), accphase ^ 1, s_abort);
           if (!ok) break;
           tc_fence_after();
           const uint32_t d_tmem = tmem_base + (uint32_t)acc * 128u;
           const uint32_t kt = smem_u32(sK + (size_t)stage * TcSmem<D>::kTileBytes);
-          const uint32_t qb = smem_u32(sQ);
-          if (PASS == 1) {
-            // quadrant w: Q rows on lanes [w*rows, (w+1)*rows), keys [w*rows, (w+1)*rows) of the tile
-            uint32_t first = 1;
-            for (int w = 0; w < rep; ++w)
-              for (int kb = 0; kb < KB; ++kb)
 #pragma unroll
-                for (int k = 0; k < 4; ++k) {
-                  const uint64_t ad = smem_desc(qb + (uint32_t)(kb * q_rows * 128 + (zero_before - w * rows) * 128 + k * 32));
-                  const uint64_t bd = smem_desc(kt + (uint32_t)(kb * kTile * 128 + w * rows * 128 + k * 32));
-                  tc_mma(d_tmem, ad, bd, idesc, first ? 0u : 1u);
-                  first = 0;
-                }
-          } else {
-            for (int kb = 0; kb < KB; ++kb)
+          for (int kb = 0; kb < KB; ++kb)
 #pragma unroll
-              for (int k = 0; k < 4; ++k) {
-                const uint64_t ad = smem_desc(kt + (uint32_t)(kb * kTile * 128 + k * 32));
-                const uint64_t bd = smem_desc(qb + (uint32_t)(kb * q_rows * 128 + zero_before * 128 + k * 32));
-                tc_mma(d_tmem, ad, bd, idesc, (kb | k) ? 1u : 0u);
-              }
-          }
-          tc_commit(BAR(4 + stage));     // smem stage free once these MMAs have read it
-          tc_commit(BAR(10 + acc));      // accumulator ready for the epilogue
+            for (int k = 0; k < 4; ++k) {
+              const uint64_t ad = smem_desc(kt + (uint32_t)(kb * kTile * 128 + k * 32));
+              const uint64_t bd = smem_desc(qbase + (uint32_t)(kb * rows * 128 + k * 32));
+              tc_mma(d_tmem, ad, bd, idesc, (kb | k) ? 1u : 0u);
+            }
+          tc_commit(BAR(B_EMPTY + stage));   // smem stage free once these MMAs have read it
+          tc_commit(BAR(B_TFULL + acc));     // accumulator ready for the epilogue
           if (++stage == kStages) { stage = 0; phase ^= 1; }
           if (++acc == 2) { acc = 0; accphase ^= 1; }
         }
-        tc_commit(BAR(9));               // Q buffer free once the item's MMAs are done
+        tc_commit(BAR(B_QEMPTY + qb));       // Q block free once the item's MMAs are done
+        qb ^= 1;
       }
     }
   } else {
-    // ------------------------------------------------------------ epilogue (4 warps = 128 TMEM lanes)
+    // ------------------------------------------------------------ epilogue: 4 warps, a TMEM lane is a key
     const int quad = warp & 3;                      // TMEM lane quadrant this warp may read
-    const int tl = quad * 32 + lane;                // TMEM lane of this thread
     float2* myStat = sStat + (warp - 2) * 128;
+    float* myT = sTrans + (warp - 2) * (32 * 33);
     int acc = 0;
-    uint32_t accphase = 0;
+    uint32_t accphase = 0, epiphase = 0;
+    int n_done = 0;
     bool ok = true;
-    for (int it = blockIdx.x; it < n_items && ok; it += gridDim.x) {
-      const int lu = it / a.chunks, ch = it % a.chunks;
-      const int u = a.u0 + lu;
-      const int key0 = ch * kChunk;
-      const int ntiles = (min(N, key0 + kChunk) - key0 + kTile - 1) / kTile;
-      float m_run = -INFINITY, z_run = 0.f;         // pass 1 state of this thread's (row, key quadrant)
-      const int row1 = tl % rows, kq = tl / rows;   // pass 1: window row and key sub-tile
-      if (PASS == 2) {
+    for (int s = blockIdx.x; s < a.total && ok; s += gridDim.x) {
+      const Item it = decode_item(a, s);
+      if (!it.valid) continue;
+      const int u = a.u0 + it.lu;
+      const int key0 = it.ch * a.chunk_keys;
+      const int ntiles = (min(N, key0 + a.chunk_keys) - key0 + kTile - 1) / kTile;
+      // pass 1 state: after the transposition lane = window row (rg * 32 + lane); raw (unscaled) maxima
+      float m_run[4], z_run[4];
+#pragma unroll
+      for (int rg = 0; rg < 4; ++rg) { m_run[rg] = -INFINITY; z_run[rg] = 0.f; }
+      if (it.pass == 2) {
         __syncwarp();
         for (int i = lane; i < rows; i += 32)
           myStat[i] = reinterpret_cast<const float2*>(p.stat)[(size_t)u * p.rows_pad + i];
         __syncwarp();
       }
       for (int t = 0; t < ntiles; ++t) {
-        ok = mbar_wait(BAR(10 + acc), accphase, s_abort);
+        ok = mbar_wait(BAR(B_TFULL + acc), accphase, s_abort);
         if (!ok) break;
         tc_fence_after();
         const uint32_t taddr = tmem_base + ((uint32_t)(quad * 32) << 16) + (uint32_t)acc * 128u;
         const int tbase = key0 + t * kTile;
-        if (PASS == 1) {
-          const int pos = N - L + (row1 % L);       // last key this window row may see
-          const int jb = tbase + kq * rows;
-          for (int c0 = 0; c0 < rows; c0 += 32) {
-            uint32_t r[32];
-            tc_ld32(taddr + (uint32_t)c0, r);
-            tc_wait_ld();
-            float x[32];
-            float cm = -INFINITY;
+        const bool tail = (tbase + kTile - 1 > N - L);   // some key of the tile is masked for some row
+        if (it.pass == 1) {
+          const int jw = tbase + quad * 32;              // first key of this warp's 32 lanes
 #pragma unroll
-            for (int c = 0; c < 32; ++c) {
-              const int j = jb + c0 + c;
-              x[c] = (j <= pos && j < N) ? __uint_as_float(r[c]) * scale2 : -INFINITY;
-              cm = fmaxf(cm, x[c]);
-            }
-            if (cm > m_run) {
-              z_run *= ex2(m_run - cm);
-              m_run = cm;
-            }
-            if (m_run > -INFINITY) {
-              float zs = 0.f;
+          for (int rg = 0; rg < 4; ++rg) {
+            if (rg * 32 < rows) {
+              uint32_t r[32];
+              tc_ld32(taddr + (uint32_t)(rg * 32), r);
+              tc_wait_ld();
+              // transpose the warp's [32 keys][32 rows] block through shared memory
 #pragma unroll
-              for (int c = 0; c < 32; ++c) zs += ex2(x[c] - m_run);
-              z_run += zs;
+              for (int c = 0; c < 32; ++c) myT[lane * 33 + c] = __uint_as_float(r[c]);
+              __syncwarp();
+              float x[32];
+              float cm = -INFINITY;
+              if (!tail) {
+#pragma unroll
+                for (int k = 0; k < 32; ++k) { x[k] = myT[k * 33 + lane]; cm = fmaxf(cm, x[k]); }
+              } else {
+                const int pos = N - L + ((rg * 32 + lane) % L);   // last key this window row may see
+#pragma unroll
+                for (int k = 0; k < 32; ++k) {
+                  const int j = jw + k;
+                  x[k] = (j <= pos && j < N) ? myT[k * 33 + lane] : -INFINITY;
+                  cm = fmaxf(cm, x[k]);
+                }
+              }
+              __syncwarp();
+              if (cm > m_run[rg]) {
+                z_run[rg] *= ex2((m_run[rg] - cm) * scale2);
+                m_run[rg] = cm;
+              }
+              if (m_run[rg] > -INFINITY) {
+                const float ms = -m_run[rg] * scale2;
+                float zs = 0.f;
+#pragma unroll
+                for (int k = 0; k < 32; ++k) zs += ex2(fmaf(x[k], scale2, ms));
+                z_run[rg] += zs;
+              }
             }
           }
         } else {
-          const int j = tbase + tl;                 // this thread's key
-          const bool tail = (tbase + kTile - 1 > N - L);
+          const int j = tbase + quad * 32 + lane;   // this thread's key
           float csum = 0.f;
           for (int c0 = 0; c0 < rows; c0 += 32) {
             uint32_t r[32];
@@ -363,13 +390,35 @@ window_tc_kernel(const __grid_constant__ CUtensorMap tmap_k, const __grid_consta
         }
         tc_fence_before();
         __syncwarp();
-        if (lane == 0) mbar_arrive(BAR(12 + acc));
+        if (lane == 0) mbar_arrive(BAR(B_TEMPTY + acc));
         if (++acc == 2) { acc = 0; accphase ^= 1; }
       }
-      if (PASS == 1 && ok) {
-        // slot = chunk * rep + key quadrant
-        reinterpret_cast<float2*>(p.stat_part)[((size_t)u * p.chunks_max + (size_t)ch * rep + kq) * p.rows_pad + row1] =
-            make_float2(m_run, z_run);
+      if (!ok) break;
+      if (it.pass == 1) {
+        // merge the four warps' (max, sum) per row in a fixed order; one slot per work item
+        float2* mg = sMerge + (n_done & 1) * (4 * 128);
+#pragma unroll
+        for (int rg = 0; rg < 4; ++rg)
+          if (rg * 32 < rows) mg[(warp - 2) * 128 + rg * 32 + lane] = make_float2(m_run[rg] * scale2, z_run[rg]);
+        mbar_arrive(BAR(B_EPI));
+        ok = mbar_wait(BAR(B_EPI), epiphase, s_abort);
+        epiphase ^= 1;
+        if (!ok) break;
+        const int tl = (warp - 2) * 32 + lane;
+        if (tl < rows) {
+          float M = -INFINITY;
+#pragma unroll
+          for (int w = 0; w < 4; ++w) M = fmaxf(M, mg[w * 128 + tl].x);
+          float z = 0.f;
+#pragma unroll
+          for (int w = 0; w < 4; ++w) {
+            const float2 o = mg[w * 128 + tl];
+            if (o.x > -INFINITY) z = fmaf(o.y, ex2(o.x - M), z);
+          }
+          reinterpret_cast<float2*>(p.stat_part)[((size_t)u * p.chunks_max + it.ch) * p.rows_pad + tl] =
+              make_float2(M, z);
+        }
+        ++n_done;
       }
     }
   }
@@ -384,7 +433,7 @@ window_tc_kernel(const __grid_constant__ CUtensorMap tmap_k, const __grid_consta
   if (tid == 0 && *s_abort) set_status(p.status, TASKKV_ETIMEOUT);
 }
 
-// Combine the partial statistics of one unit: slots = chunks * rep per row.
+// Combine the per-item statistics of one unit, in item order: (row max, 1 / row sum).
 __global__ void window_tc_reduce_kernel(DeviceProblem p, int u0, int slots) {
   const int u = u0 + blockIdx.x;
   const int row = threadIdx.x;
@@ -395,7 +444,7 @@ __global__ void window_tc_reduce_kernel(DeviceProblem p, int u0, int slots) {
   float z = 0.f;
   for (int c = 0; c < slots; ++c) {
     const float2 o = part[(size_t)c * p.rows_pad + row];
-    if (o.x > -INFINITY) z += o.y * exp2f(o.x - M);
+    if (o.x > -INFINITY) z = fmaf(o.y, exp2f(o.x - M), z);
   }
   reinterpret_cast<float2*>(p.stat)[(size_t)u * p.rows_pad + row] =
       z > 0.f ? make_float2(M, 1.0f / z) : make_float2(0.f, 0.f);
@@ -415,6 +464,8 @@ EncodeTiledFn encode_fn() {
     if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &ptr, cudaEnableDefault, &qres) == cudaSuccess &&
         qres == cudaDriverEntryPointSuccess)
       fn = reinterpret_cast<EncodeTiledFn>(ptr);
+    else
+      cudaGetLastError();
   }
   return fn;
 }
@@ -432,6 +483,8 @@ bool make_map(CUtensorMap* map, const void* base, int d, uint64_t rows_total, in
             CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
 }
 
+int g_tc_chunk = 2048;   // keys per work item
+
 template <int D>
 cudaError_t launch_tc_d(const DeviceProblem& p, const WindowHostInfo& h, cudaStream_t s) {
   static int n_sm = 0;
@@ -442,12 +495,9 @@ cudaError_t launch_tc_d(const DeviceProblem& p, const WindowHostInfo& h, cudaStr
     if (n_sm <= 0) n_sm = 148;
   }
   const int smem = TcSmem<D>::kBytes;
-  cudaError_t e = cudaFuncSetAttribute(window_tc_kernel<D, 1>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem);
-  if (e != cudaSuccess) return e;
-  e = cudaFuncSetAttribute(window_tc_kernel<D, 2>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem);
+  cudaError_t e = cudaFuncSetAttribute(window_tc_kernel<D>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem);
   if (e != cudaSuccess) return e;
   const int per_seq = p.R * p.n_kv;
-  const int rep = 128 / p.rows;
   for (int b = 0; b < h.batch; ++b) {
     const int N = h.seq_lens[b];
     CUtensorMap mk, mq;
@@ -457,22 +507,23 @@ cudaError_t launch_tc_d(const DeviceProblem& p, const WindowHostInfo& h, cudaStr
     a.u0 = b * per_seq;
     a.n_local = per_seq;
     a.N = N;
-    a.chunks = (N + kChunk - 1) / kChunk;
-    const int items = a.n_local * a.chunks;
-    const int grid = items < n_sm ? items : n_sm;
+    a.chunk_keys = g_tc_chunk < kTcChunk ? kTcChunk : g_tc_chunk / 128 * 128;
+    a.chunks = (N + a.chunk_keys - 1) / a.chunk_keys;
+    a.total = a.n_local * a.chunks;
+    const int grid = a.total < n_sm ? a.total : n_sm;
     a.pass = 1;
     {
       LaunchScope ls(K_WINDOW_TC, s);
-      window_tc_kernel<D, 1><<<grid, kThreads, smem, s>>>(mk, mq, p, a);
+      window_tc_kernel<D><<<grid, kThreads, smem, s>>>(mk, mq, p, a);
     }
     {
       LaunchScope ls(K_WINDOW_REDUCE, s);
-      window_tc_reduce_kernel<<<per_seq, 128, 0, s>>>(p, a.u0, a.chunks * rep);
+      window_tc_reduce_kernel<<<per_seq, 128, 0, s>>>(p, a.u0, a.chunks);
     }
     a.pass = 2;
     {
       LaunchScope ls(K_WINDOW_TC, s);
-      window_tc_kernel<D, 2><<<grid, kThreads, smem, s>>>(mk, mq, p, a);
+      window_tc_kernel<D><<<grid, kThreads, smem, s>>>(mk, mq, p, a);
     }
     e = cudaGetLastError();
     if (e != cudaSuccess) return e;
@@ -489,6 +540,10 @@ bool window_tc_supported(const DeviceProblem& p, int dtype) {
 
 cudaError_t launch_window_scores_tc(const DeviceProblem& p, const WindowHostInfo& h, cudaStream_t s) {
   return p.d == 64 ? launch_tc_d<64>(p, h, s) : launch_tc_d<128>(p, h, s);
+}
+
+void window_tc_set_mode(int, int chunk, int) {
+  if (chunk > 0) g_tc_chunk = chunk;
 }
 
 }  // namespace taskkv
