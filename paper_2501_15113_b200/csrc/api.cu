@@ -102,7 +102,7 @@ taskkv_status make_plan(const taskkv_params* p, HostPlan& hp) {
       gitems += h * ((N + kGatherRows - 1) / kGatherRows) + (nkv - h) * ((kept + kGatherRows - 1) / kGatherRows);
       ditems += h * ((N + mn + kDecodeChunk - 1) / kDecodeChunk) +
                 (nkv - h) * ((kept + mn + kDecodeChunk - 1) / kDecodeChunk);
-      c_total += (int64_t)nkv * N;
+      c_total += (int64_t)nkv * ((N + 3) / 4 * 4);
     }
   }
   if (gitems > 0x7fffffff || ditems > 0x7fffffff) return TASKKV_EINVAL;
@@ -292,7 +292,7 @@ void build_meta(taskkv_cache* c, const void* const* q_win, const void* const* k,
         unit_N[u] = (int32_t)N;
         unit_mid[u] = hp.mid[r];
         c_off[u] = coff;
-        coff += (int64_t)N;
+        coff += (int64_t)((N + 3) / 4 * 4);
         qp[u] = static_cast<const unsigned char*>(q_win[b]) +
                 (((size_t)r * p.n_heads + (size_t)h * G) * p.window) * d * es;
         kp[u] = static_cast<const unsigned char*>(k[b]) + (((size_t)r * nkv + h) * N) * d * es;
@@ -400,7 +400,7 @@ taskkv_status taskkv_compress_ex(const taskkv_params* p, const void* const* q_wi
   wh.q = q_win;
   wh.k = k;
   if (e == cudaSuccess) e = launch_window_scores(c->dp, p->dtype, c->hp.max_N, wh, s);
-  if (e == cudaSuccess) e = launch_select(c->dp, p->dtype, s);
+  if (e == cudaSuccess) e = launch_select(c->dp, p->dtype, c->hp.max_N, s);
   if (e == cudaSuccess) e = launch_separator_plan(c->dp, p->batch * p->n_layers, s);
   if (e == cudaSuccess) e = launch_gather(c->dp, p->dtype, c->hp.info.gather_items, s);
   if (e != cudaSuccess) {

@@ -19,6 +19,9 @@ __device__ __forceinline__ uint32_t ordered_key(float x) {
   const uint32_t b = __float_as_uint(x);
   return (b & 0x80000000u) ? ~b : (b | 0x80000000u);
 }
+__device__ __forceinline__ float key_score(uint32_t k) {   // inverse of ordered_key
+  return __uint_as_float((k & 0x80000000u) ? (k & 0x7fffffffu) : ~k);
+}
 
 struct ScoreKey {          // key of C[j]
   const float* C;
@@ -220,10 +223,221 @@ __global__ void __launch_bounds__(kThreads) select_kernel(DeviceProblem p) {
   }
 }
 
+
+// ---------------------------------------------------------------------------
+// Register-resident variant for N <= 32768 (and pooling kernel 1 or 7): every
+// thread keeps 32 consecutive scores in registers, so a selection is a bisection
+// over the 32 key bits -- each step is 32 compares per thread plus one block-wide
+// count -- and the ordered compaction is a single block scan.  Same results as
+// the radix path: exact k-th key, lower position first among equal keys, pooled
+// sums added in ascending position.
+constexpr int kEpt = 32;
+
+struct FastSmem {
+  int cnt[2][kWarps];
+  uint32_t mn[kWarps], mx[kWarps];
+  int scan[kWarps];
+  int scan_tot;
+};
+
+__device__ __forceinline__ int block_count_ge(const uint32_t (&key)[kEpt], uint32_t cand, int* slot) {
+  int c = 0;
+#pragma unroll
+  for (int e = 0; e < kEpt; ++e) c += (key[e] >= cand) ? 1 : 0;
+  c = __reduce_add_sync(0xffffffffu, c);
+  const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+  if (lane == 0) slot[warp] = c;
+  __syncthreads();
+  return __reduce_add_sync(0xffffffffu, slot[lane]);
+}
+
+// k-th largest key (1 <= want <= number of non-zero keys) and how many keys equal to it belong to the top `want`.
+__device__ void block_bisect(FastSmem& fs, const uint32_t (&key)[kEpt], int want, uint32_t& thr, int& need_eq) {
+  const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+  // bits above the highest bit in which the non-zero keys differ are common to the answer
+  uint32_t lo = 0xffffffffu, hi = 0u;
+#pragma unroll
+  for (int e = 0; e < kEpt; ++e)
+    if (key[e]) { lo = min(lo, key[e]); hi = max(hi, key[e]); }
+  lo = __reduce_min_sync(0xffffffffu, lo);
+  hi = __reduce_max_sync(0xffffffffu, hi);
+  if (lane == 0) { fs.mn[warp] = lo; fs.mx[warp] = hi; }
+  __syncthreads();
+  lo = __reduce_min_sync(0xffffffffu, fs.mn[lane]);
+  hi = __reduce_max_sync(0xffffffffu, fs.mx[lane]);
+  const uint32_t diff = lo ^ hi;
+  int bit = diff ? 31 - __clz(diff) : -1;
+  uint32_t t = diff ? (hi & ~((2u << bit) - 1u)) : hi;
+  int par = 0;
+  for (; bit >= 0; --bit) {
+    const uint32_t cand = t | (1u << bit);
+    if (block_count_ge(key, cand, fs.cnt[par]) >= want) t = cand;
+    par ^= 1;
+  }
+  const int n_gt = (t == 0xffffffffu) ? 0 : block_count_ge(key, t + 1u, fs.cnt[par]);
+  thr = t;
+  need_eq = want - n_gt;
+  __syncthreads();
+}
+
+// Ordered compaction of this thread's 32 consecutive positions [base, base + 32).
+template <class Emit>
+__device__ void block_compact_regs(FastSmem& fs, const uint32_t (&key)[kEpt], int base, uint32_t thr, int need_eq,
+                                   const Emit& emit) {
+  const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+  int gt = 0, eq = 0;
+#pragma unroll
+  for (int e = 0; e < kEpt; ++e) { gt += key[e] > thr; eq += key[e] == thr; }
+  const int packed = gt | (eq << 16);
+  int incl = packed;
+#pragma unroll
+  for (int o = 1; o < 32; o <<= 1) {
+    const int y = __shfl_up_sync(0xffffffffu, incl, o);
+    if (lane >= o) incl += y;
+  }
+  if (lane == 31) fs.scan[warp] = incl;
+  __syncthreads();
+  int wp = fs.scan[lane];
+  int wi = wp;
+#pragma unroll
+  for (int o = 1; o < 32; o <<= 1) {
+    const int y = __shfl_up_sync(0xffffffffu, wi, o);
+    if (lane >= o) wi += y;
+  }
+  const int wexcl = __shfl_sync(0xffffffffu, wi - wp, warp);
+  const int excl = incl - packed + wexcl;
+  int gt_before = excl & 0xffff, eq_before = excl >> 16;
+#pragma unroll
+  for (int e = 0; e < kEpt; ++e) {
+    const bool g = key[e] > thr, q = key[e] == thr;
+    if (g || (q && eq_before < need_eq)) emit(gt_before + min(eq_before, need_eq), base + e, e);
+    gt_before += g;
+    eq_before += q;
+  }
+  __syncthreads();
+}
+
+template <typename T, int D, int POOL_HALF>
+__global__ void __launch_bounds__(kThreads, 1) select_fast_kernel(DeviceProblem p) {
+  __shared__ FastSmem fs;
+  __shared__ int sel[TASKKV_MAX_TOP_T];
+  __shared__ float selw[TASKKV_MAX_TOP_T];
+  __shared__ float red[kWarps][D];
+
+  const int u = blockIdx.x;
+  const int N = p.unit_N[u];
+  const float* C = p.C + p.c_off[u];
+  const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+  const int base = tid * kEpt;
+
+  // only the keys are kept (a key maps back to its score exactly); key 0 marks "no element"
+  uint32_t key[kEpt];
+  if (base + kEpt <= N && ((reinterpret_cast<uintptr_t>(C + base) & 15) == 0)) {
+#pragma unroll
+    for (int e = 0; e < kEpt; e += 4) {
+      const float4 v = *reinterpret_cast<const float4*>(C + base + e);
+      key[e] = ordered_key(v.x); key[e + 1] = ordered_key(v.y);
+      key[e + 2] = ordered_key(v.z); key[e + 3] = ordered_key(v.w);
+    }
+  } else {
+#pragma unroll
+    for (int e = 0; e < kEpt; ++e) key[e] = (base + e < N) ? ordered_key(C[base + e]) : 0u;
+  }
+
+  // ---- Eq. 14: I = top-min(t, N) of C
+  const int t = min(p.top_t, N);
+  uint32_t thr;
+  int need_eq;
+  block_bisect(fs, key, t, thr, need_eq);
+  int* topt = p.topt + (size_t)u * p.top_t;
+  block_compact_regs(fs, key, base, thr, need_eq, [&](int pos, int j, int e) {
+    sel[pos] = j;
+    selw[pos] = key_score(key[e]);
+    topt[pos] = j;
+  });
+  for (int i = t + tid; i < p.top_t; i += kThreads) topt[i] = -1;
+
+  // ---- Eq. 15: v' = sum_{j in I} C[j] V[j,:], fixed summation order
+  constexpr int EPL = D / 32;
+  float acc[EPL];
+#pragma unroll
+  for (int e = 0; e < EPL; ++e) acc[e] = 0.f;
+  const T* V = static_cast<const T*>(p.v_ptr[u]);
+  for (int i = warp; i < t; i += kWarps) {
+    const float w = selw[i];
+    const T* row = V + (size_t)sel[i] * D + lane * EPL;
+#pragma unroll
+    for (int e = 0; e < EPL; ++e) acc[e] = fmaf(w, to_float(row[e]), acc[e]);
+  }
+#pragma unroll
+  for (int e = 0; e < EPL; ++e) red[warp][lane * EPL + e] = acc[e];
+  __syncthreads();
+  if (tid < D) {
+    float s = 0.f;
+    for (int w = 0; w < kWarps; ++w) s += red[w][tid];
+    p.sem[(size_t)u * D + tid] = s;
+  }
+
+  // ---- Sec. IV-B: sinks, middle activations (top-k of the pooled scores), recent window
+  const int s1 = p.sink, s2 = p.recent;
+  if (N <= s1 + s2) return;
+  const int lo = s1, hi = N - s2;
+  const int kmid = min(p.unit_mid[u], hi - lo);
+  if (kmid >= hi - lo) return;
+  int* idx = p.idx + (size_t)u * p.idx_stride;
+  for (int i = tid; i < s1; i += kThreads) idx[i] = i;
+  for (int i = tid; i < s2; i += kThreads) idx[s1 + kmid + i] = N - s2 + i;
+  if (kmid == 0) return;
+
+  // pooled window sums in ascending position: ext = [3 left neighbours][32 own][3 right neighbours]
+  if (POOL_HALF > 0) {
+    float ext[kEpt + 2 * POOL_HALF];
+#pragma unroll
+    for (int h = 0; h < POOL_HALF; ++h) {
+      const int jl = base - POOL_HALF + h, jr = base + kEpt + h;
+      ext[h] = (jl >= 0 && jl < N) ? C[jl] : 0.f;
+      ext[POOL_HALF + kEpt + h] = (jr < N) ? C[jr] : 0.f;
+    }
+#pragma unroll
+    for (int e = 0; e < kEpt; ++e) ext[POOL_HALF + e] = (base + e < N) ? key_score(key[e]) : 0.f;
+#pragma unroll
+    for (int e = 0; e < kEpt; ++e) {
+      float sum = 0.f;
+#pragma unroll
+      for (int o = 0; o <= 2 * POOL_HALF; ++o) sum += ext[e + o];
+      const int j = base + e;
+      key[e] = (j >= lo && j < hi) ? ordered_key(sum) : 0u;
+    }
+  } else {
+#pragma unroll
+    for (int e = 0; e < kEpt; ++e) {
+      const int j = base + e;
+      if (!(j >= lo && j < hi)) key[e] = 0u;
+    }
+  }
+  __syncthreads();
+  block_bisect(fs, key, kmid, thr, need_eq);
+  block_compact_regs(fs, key, base, thr, need_eq, [&](int pos, int j, int) { idx[s1 + pos] = j; });
+}
+
+template <typename T, int D>
+void launch_fast(const DeviceProblem& p, cudaStream_t s) {
+  if (p.pool_w == 7) select_fast_kernel<T, D, 3><<<p.U, kThreads, 0, s>>>(p);
+  else select_fast_kernel<T, D, 0><<<p.U, kThreads, 0, s>>>(p);
+}
+
 }  // namespace
 
-cudaError_t launch_select(const DeviceProblem& p, int dtype, cudaStream_t s) {
+cudaError_t launch_select(const DeviceProblem& p, int dtype, int max_N, cudaStream_t s) {
   LaunchScope ls(K_SELECT, s);
+  if (max_N <= kThreads * kEpt && (p.pool_w == 7 || p.pool_w == 1)) {
+    if (dtype == TASKKV_F32) {
+      if (p.d == 64) launch_fast<float, 64>(p, s); else launch_fast<float, 128>(p, s);
+    } else {
+      if (p.d == 64) launch_fast<__nv_bfloat16, 64>(p, s); else launch_fast<__nv_bfloat16, 128>(p, s);
+    }
+    return cudaGetLastError();
+  }
   if (dtype == TASKKV_F32) {
     if (p.d == 64) select_kernel<float, 64><<<p.U, kThreads, 0, s>>>(p);
     else select_kernel<float, 128><<<p.U, kThreads, 0, s>>>(p);

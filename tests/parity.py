@@ -71,7 +71,7 @@ def score_offsets(wl: W.Workload) -> np.ndarray:
     off = [0]
     for b in range(wl.batch):
         for _ in range(wl.n_layers * wl.n_kv_heads):
-            off.append(off[-1] + wl.seq_lens[b])
+            off.append(off[-1] + (wl.seq_lens[b] + 3) // 4 * 4)     # units are padded to 4 floats
     return np.array(off, dtype=np.int64)
 
 
@@ -93,7 +93,7 @@ def compare_layer(cache: tk.Cache, wl: W.Workload, b: int, r: int, ref: Dict, re
         rep.units += 1
         # Eq. 12-13: scores
         if scores is not None:
-            c_gpu = scores[coff[u]:coff[u + 1]].astype(np.float64)
+            c_gpu = scores[coff[u]:coff[u] + N].astype(np.float64)
             rel = np.abs(c_gpu - ref["C"][h]) / ref["C"][h]
             rep.max_score_rel = max(rep.max_score_rel, float(rel.max()))
             assert rel.max() < TOL_SCORE_REL, f"unit {u}: scores off by {rel.max():.3e} relative"
