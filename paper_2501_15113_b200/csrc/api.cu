@@ -110,7 +110,7 @@ taskkv_status make_plan(const taskkv_params* p, HostPlan& hp) {
   hp.c_total = c_total;
   hp.rows = G * p->window;
   hp.rows_pad = (hp.rows + 15) / 16 * 16;
-  hp.chunks_max = ((hp.max_N + kTcChunk - 1) / kTcChunk) * 4;   // partial-statistic slots per unit (covers both window paths)
+  hp.chunks_max = (hp.max_N + kTcChunk - 1) / kTcChunk;   // partial-statistic slots per unit (kTcChunk == kScoreChunk)
 
   const size_t es = p->dtype == TASKKV_F32 ? 4 : 2;
   const size_t d = p->head_dim;

@@ -34,28 +34,53 @@ constexpr int kThreads = 192;
 constexpr uint32_t kTmemCols = 256; // two accumulator stages of up to 128 columns
 constexpr uint32_t kSpinLimit = 1u << 22;
 
-// Work items of one launch (one sequence and one pass): (unit, chunk of chunk_keys keys), unit-major,
-// taken round-robin by the resident CTAs.
+// Work items of one launch (one sequence): (pass, unit, chunk of chunk_keys keys).
+// mode 1 / 2: one pass per launch, unit-major (statistics combined by a kernel in between).
+// mode 0: both passes in one launch so that the second read of the keys is served by L2.  Positions
+//   alternate between the pass-1 stream (item i at position 2i) and the pass-2 stream, which lags by
+//   `lag2` items; the statistics of unit u are combined ("finalised") by the epilogue warps of the CTA
+//   that takes pass-1 position u*C + C-1 + lag_r, i.e. lag_r items after the unit's last pass-1 item.
+//   lag_r and lag2 - C - lag_r exceed the number of positions in flight, so the data a step needs is
+//   normally there; if not, it polls (bounded): every partial and every statistic is one 8-byte word
+//   that is NaN until written, so no fence or counter is involved.  A step only ever depends on
+//   earlier positions, which resident CTAs taking positions in order have already started.
 struct TcArgs {
-  int pass;          // 1: row statistics, 2: scores
+  int mode;
   int u0;            // first unit of this sequence
   int n_local;       // units in this launch (layers * kv heads)
   int N;             // sequence length
-  int chunks;        // work items per unit
-  int chunk_keys;    // keys per work item (multiple of 128, >= kTcChunk)
-  int total;         // work items
+  int chunks;        // C: work items per unit and pass
+  int chunk_keys;    // keys per work item (multiple of 128)
+  int lag_r, lag2;   // mode 0
+  int total;         // positions
 };
 
 struct Item {
   int pass, lu, ch;
-  bool valid;
+  bool valid;        // has tiles to process
+  int fin_unit;      // >= 0: first finalise this (local) unit's statistics
 };
 __device__ __forceinline__ Item decode_item(const TcArgs& a, int s) {
   Item it;
-  it.pass = a.pass;
-  it.lu = s / a.chunks;
-  it.ch = s % a.chunks;
-  it.valid = true;
+  it.fin_unit = -1;
+  int i;
+  if (a.mode != 0) {
+    it.pass = a.mode;
+    i = s;
+    it.valid = true;
+  } else if ((s & 1) == 0) {
+    it.pass = 1;
+    i = s >> 1;
+    it.valid = i < a.n_local * a.chunks;
+    const int r = i - a.lag_r - (a.chunks - 1);
+    if (r >= 0 && r % a.chunks == 0 && r / a.chunks < a.n_local) it.fin_unit = r / a.chunks;
+  } else {
+    it.pass = 2;
+    i = (s >> 1) - a.lag2;
+    it.valid = i >= 0 && i < a.n_local * a.chunks;
+  }
+  it.lu = it.valid ? i / a.chunks : 0;
+  it.ch = it.valid ? i % a.chunks : 0;
   return it;
 }
 
@@ -142,6 +167,30 @@ __device__ __forceinline__ float ex2(float x) {
   float y;
   asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
   return y;
+}
+
+// (a, b) pairs that double as their own "written" flag: the buffers are filled with 0xFF bytes (NaN)
+// before the launch, a pair is published with one 8-byte store and read with one 8-byte load.
+__device__ __forceinline__ void publish_pair(float2* addr, float x, float y) {
+  const uint64_t v = (uint64_t)__float_as_uint(x) | ((uint64_t)__float_as_uint(y) << 32);
+  asm volatile("st.relaxed.gpu.global.b64 [%0], %1;" ::"l"(addr), "l"(v) : "memory");
+}
+__device__ __forceinline__ bool poll_pair(const float2* addr, float2& out, volatile int* abort_flag) {
+  for (uint32_t spin = 0;; ++spin) {
+    uint64_t v;
+    asm volatile("ld.relaxed.gpu.global.b64 %0, [%1];" : "=l"(v) : "l"(addr) : "memory");
+    const float y = __uint_as_float((uint32_t)(v >> 32));
+    if (y == y) {
+      out = make_float2(__uint_as_float((uint32_t)v), y);
+      return true;
+    }
+    if (*abort_flag) return false;
+    if (spin > kSpinLimit) {
+      *abort_flag = 1;
+      return false;
+    }
+    __nanosleep(200);
+  }
 }
 
 // Shared-memory matrix descriptor: K-major operand, rows of 128 bytes, 128-byte
@@ -303,6 +352,42 @@ window_tc_kernel(const __grid_constant__ CUtensorMap tmap_k, const __grid_consta
     bool ok = true;
     for (int s = blockIdx.x; s < a.total && ok; s += gridDim.x) {
       const Item it = decode_item(a, s);
+      if (it.fin_unit >= 0) {
+        // combine the unit's per-item statistics, in item order, into (row max, 1 / row sum)
+        const int row = (warp - 2) * 32 + lane;
+        if (row < rows) {
+          const int uf = a.u0 + it.fin_unit;
+          const float2* part = reinterpret_cast<const float2*>(p.stat_part) + (size_t)uf * p.chunks_max * p.rows_pad;
+          float M = -INFINITY, z = 0.f;
+          for (int c0 = 0; c0 < a.chunks && ok; c0 += 8) {
+            uint64_t w[8];
+#pragma unroll
+            for (int i = 0; i < 8; ++i) {   // eight loads in flight, then consume in order
+              w[i] = ~0ull;
+              if (c0 + i < a.chunks)
+                asm volatile("ld.relaxed.gpu.global.b64 %0, [%1];"
+                             : "=l"(w[i]) : "l"(&part[(size_t)(c0 + i) * p.rows_pad + row]) : "memory");
+            }
+#pragma unroll
+            for (int i = 0; i < 8; ++i) {
+              if (c0 + i < a.chunks && ok) {
+                float2 o = make_float2(__uint_as_float((uint32_t)w[i]), __uint_as_float((uint32_t)(w[i] >> 32)));
+                if (o.y != o.y) ok = poll_pair(&part[(size_t)(c0 + i) * p.rows_pad + row], o, s_abort);
+                if (ok && o.x > -INFINITY) {
+                  const float Mn = fmaxf(M, o.x);
+                  z = fmaf(z, ex2(M - Mn), o.y * ex2(o.x - Mn));
+                  M = Mn;
+                }
+              }
+            }
+          }
+          if (ok)
+            publish_pair(reinterpret_cast<float2*>(p.stat) + (size_t)uf * p.rows_pad + row, z > 0.f ? M : 0.f,
+                         z > 0.f ? 1.0f / z : 0.f);
+        }
+        ok = __all_sync(0xffffffffu, ok);
+        if (!ok) break;
+      }
       if (!it.valid) continue;
       const int u = a.u0 + it.lu;
       const int key0 = it.ch * a.chunk_keys;
@@ -313,9 +398,13 @@ window_tc_kernel(const __grid_constant__ CUtensorMap tmap_k, const __grid_consta
       for (int rg = 0; rg < 4; ++rg) { m_run[rg] = -INFINITY; z_run[rg] = 0.f; }
       if (it.pass == 2) {
         __syncwarp();
-        for (int i = lane; i < rows; i += 32)
-          myStat[i] = reinterpret_cast<const float2*>(p.stat)[(size_t)u * p.rows_pad + i];
-        __syncwarp();
+        for (int i = lane; i < rows && ok; i += 32) {
+          float2 o;
+          ok = poll_pair(reinterpret_cast<const float2*>(p.stat) + (size_t)u * p.rows_pad + i, o, s_abort);
+          myStat[i] = o;
+        }
+        ok = __all_sync(0xffffffffu, ok);
+        if (!ok) break;
       }
       for (int t = 0; t < ntiles; ++t) {
         ok = mbar_wait(BAR(B_TFULL + acc), accphase, s_abort);
@@ -415,8 +504,8 @@ window_tc_kernel(const __grid_constant__ CUtensorMap tmap_k, const __grid_consta
             const float2 o = mg[w * 128 + tl];
             if (o.x > -INFINITY) z = fmaf(o.y, ex2(o.x - M), z);
           }
-          reinterpret_cast<float2*>(p.stat_part)[((size_t)u * p.chunks_max + it.ch) * p.rows_pad + tl] =
-              make_float2(M, z);
+          publish_pair(reinterpret_cast<float2*>(p.stat_part) + ((size_t)u * p.chunks_max + it.ch) * p.rows_pad + tl,
+                       M, z);
         }
         ++n_done;
       }
@@ -483,7 +572,9 @@ bool make_map(CUtensorMap* map, const void* base, int d, uint64_t rows_total, in
             CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
 }
 
-int g_tc_chunk = 2048;   // keys per work item
+int g_tc_mode = 0;       // 0: both passes in one launch; 1: one launch per pass
+int g_tc_chunk = 1024;   // keys per work item
+int g_tc_margin = 0;     // 0: from the SM count
 
 template <int D>
 cudaError_t launch_tc_d(const DeviceProblem& p, const WindowHostInfo& h, cudaStream_t s) {
@@ -497,6 +588,10 @@ cudaError_t launch_tc_d(const DeviceProblem& p, const WindowHostInfo& h, cudaStr
   const int smem = TcSmem<D>::kBytes;
   cudaError_t e = cudaFuncSetAttribute(window_tc_kernel<D>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem);
   if (e != cudaSuccess) return e;
+  // partial and final statistics start as NaN = "not written"
+  e = cudaMemsetAsync(p.stat_part, 0xFF, (size_t)p.U * p.chunks_max * p.rows_pad * sizeof(float2), s);
+  if (e == cudaSuccess) e = cudaMemsetAsync(p.stat, 0xFF, (size_t)p.U * p.rows_pad * sizeof(float2), s);
+  if (e != cudaSuccess) return e;
   const int per_seq = p.R * p.n_kv;
   for (int b = 0; b < h.batch; ++b) {
     const int N = h.seq_lens[b];
@@ -509,21 +604,33 @@ cudaError_t launch_tc_d(const DeviceProblem& p, const WindowHostInfo& h, cudaStr
     a.N = N;
     a.chunk_keys = g_tc_chunk < kTcChunk ? kTcChunk : g_tc_chunk / 128 * 128;
     a.chunks = (N + a.chunk_keys - 1) / a.chunk_keys;
-    a.total = a.n_local * a.chunks;
-    const int grid = a.total < n_sm ? a.total : n_sm;
-    a.pass = 1;
-    {
+    const int n1 = a.n_local * a.chunks;
+    // a round of the resident CTAs covers n_sm positions = n_sm / 2 items of each stream
+    const int margin = g_tc_margin > 0 ? g_tc_margin : n_sm / 2 + 8;
+    a.lag_r = margin;
+    a.lag2 = a.chunks + 2 * margin;
+    if (g_tc_mode == 0) {
+      a.mode = 0;
+      a.total = 2 * (n1 + a.lag2);
       LaunchScope ls(K_WINDOW_TC, s);
-      window_tc_kernel<D><<<grid, kThreads, smem, s>>>(mk, mq, p, a);
-    }
-    {
-      LaunchScope ls(K_WINDOW_REDUCE, s);
-      window_tc_reduce_kernel<<<per_seq, 128, 0, s>>>(p, a.u0, a.chunks);
-    }
-    a.pass = 2;
-    {
-      LaunchScope ls(K_WINDOW_TC, s);
-      window_tc_kernel<D><<<grid, kThreads, smem, s>>>(mk, mq, p, a);
+      window_tc_kernel<D><<<a.total < n_sm ? a.total : n_sm, kThreads, smem, s>>>(mk, mq, p, a);
+    } else {
+      a.total = n1;
+      const int grid = a.total < n_sm ? a.total : n_sm;
+      a.mode = 1;
+      {
+        LaunchScope ls(K_WINDOW_TC, s);
+        window_tc_kernel<D><<<grid, kThreads, smem, s>>>(mk, mq, p, a);
+      }
+      {
+        LaunchScope ls(K_WINDOW_REDUCE, s);
+        window_tc_reduce_kernel<<<per_seq, 128, 0, s>>>(p, a.u0, a.chunks);
+      }
+      a.mode = 2;
+      {
+        LaunchScope ls(K_WINDOW_TC, s);
+        window_tc_kernel<D><<<grid, kThreads, smem, s>>>(mk, mq, p, a);
+      }
     }
     e = cudaGetLastError();
     if (e != cudaSuccess) return e;
@@ -542,8 +649,10 @@ cudaError_t launch_window_scores_tc(const DeviceProblem& p, const WindowHostInfo
   return p.d == 64 ? launch_tc_d<64>(p, h, s) : launch_tc_d<128>(p, h, s);
 }
 
-void window_tc_set_mode(int, int chunk, int) {
+void window_tc_set_mode(int mode, int chunk, int margin) {
+  g_tc_mode = mode;
   if (chunk > 0) g_tc_chunk = chunk;
+  g_tc_margin = margin;
 }
 
 }  // namespace taskkv
