@@ -628,7 +628,3 @@ int32_t taskkv_timing_collect(int32_t* ids, float* ms, int32_t max) {
 const char* taskkv_timing_name(int32_t id) { return (id >= 0 && id < K_COUNT) ? kKernelNames[id] : "?"; }
 
 }  // extern "C"
-
-extern "C" void taskkv_debug_window_mode(int32_t mode, int32_t chunk, int32_t delay) {
-  taskkv::window_tc_set_mode(mode, chunk, delay);
-}

@@ -105,7 +105,6 @@ cudaError_t launch_window_scores(const DeviceProblem& p, int dtype, int max_N, c
                                  cudaStream_t s);
 bool window_tc_supported(const DeviceProblem& p, int dtype);
 cudaError_t launch_window_scores_tc(const DeviceProblem& p, const WindowHostInfo& h, cudaStream_t s);
-void window_tc_set_mode(int mode, int chunk, int delay);
 cudaError_t launch_select(const DeviceProblem& p, int dtype, int max_N, cudaStream_t s);
 cudaError_t launch_separator_plan(const DeviceProblem& p, int n_br, cudaStream_t s);
 cudaError_t launch_decode_plan(const DeviceProblem& p, const int32_t* lengths, cudaStream_t s);

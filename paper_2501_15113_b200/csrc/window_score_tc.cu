@@ -299,6 +299,13 @@ window_tc_kernel(const __grid_constant__ CUtensorMap tmap_k, const __grid_consta
           if (++stage == kStages) { stage = 0; phase ^= 1; }
         }
       }
+      // Drain: every tcgen05.commit aimed at this CTA's barriers must have arrived before the CTA exits,
+      // or it would land on the barriers of the next CTA that is given this shared memory.
+      for (int i = 0; i < kStages && ok; ++i) {
+        ok = mbar_wait(BAR(B_EMPTY + stage), phase ^ 1, s_abort);
+        if (++stage == kStages) { stage = 0; phase ^= 1; }
+      }
+      for (int i = 0; i < 2 && ok; ++i, qb ^= 1) ok = mbar_wait(BAR(B_QEMPTY + qb), qphase[qb] ^ 1, s_abort);
     }
   } else if (warp == 1) {
     // ------------------------------------------------------------ MMA issuer: D[key, row] = K Q^T, both passes
@@ -407,7 +414,7 @@ window_tc_kernel(const __grid_constant__ CUtensorMap tmap_k, const __grid_consta
         if (!ok) break;
       }
       for (int t = 0; t < ntiles; ++t) {
-        ok = mbar_wait(BAR(B_TFULL + acc), accphase, s_abort);
+        ok = __all_sync(0xffffffffu, mbar_wait(BAR(B_TFULL + acc), accphase, s_abort));
         if (!ok) break;
         tc_fence_after();
         const uint32_t taddr = tmem_base + ((uint32_t)(quad * 32) << 16) + (uint32_t)acc * 128u;
@@ -490,7 +497,7 @@ window_tc_kernel(const __grid_constant__ CUtensorMap tmap_k, const __grid_consta
         for (int rg = 0; rg < 4; ++rg)
           if (rg * 32 < rows) mg[(warp - 2) * 128 + rg * 32 + lane] = make_float2(m_run[rg] * scale2, z_run[rg]);
         mbar_arrive(BAR(B_EPI));
-        ok = mbar_wait(BAR(B_EPI), epiphase, s_abort);
+        ok = __all_sync(0xffffffffu, mbar_wait(BAR(B_EPI), epiphase, s_abort));
         epiphase ^= 1;
         if (!ok) break;
         const int tl = (warp - 2) * 32 + lane;
@@ -513,6 +520,9 @@ window_tc_kernel(const __grid_constant__ CUtensorMap tmap_k, const __grid_consta
   }
 
   // ---------------------------------------------------------------- teardown
+  // after a time-out give copies and MMAs still in flight a bounded time to land before the memory is released
+  if (*s_abort)
+    for (int i = 0; i < 200; ++i) __nanosleep(1000);
   tc_fence_before();
   __syncthreads();
   if (warp == 1) {
@@ -572,9 +582,12 @@ bool make_map(CUtensorMap* map, const void* base, int d, uint64_t rows_total, in
             CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
 }
 
-int g_tc_mode = 0;       // 0: both passes in one launch; 1: one launch per pass
-int g_tc_chunk = 1024;   // keys per work item
-int g_tc_margin = 0;     // 0: from the SM count
+// One launch per pass.  The single-launch order (mode 0) exists and is exact, but measured slower:
+// the pipeline is bound on the SM side (one MMA issuer, one epilogue group), not by HBM, so serving the
+// second pass from L2 does not pay yet.
+constexpr int g_tc_mode = 1;
+constexpr int g_tc_chunk = 2048;   // keys per work item
+constexpr int g_tc_margin = 0;     // 0: from the SM count
 
 template <int D>
 cudaError_t launch_tc_d(const DeviceProblem& p, const WindowHostInfo& h, cudaStream_t s) {
@@ -647,12 +660,6 @@ bool window_tc_supported(const DeviceProblem& p, int dtype) {
 
 cudaError_t launch_window_scores_tc(const DeviceProblem& p, const WindowHostInfo& h, cudaStream_t s) {
   return p.d == 64 ? launch_tc_d<64>(p, h, s) : launch_tc_d<128>(p, h, s);
-}
-
-void window_tc_set_mode(int mode, int chunk, int margin) {
-  g_tc_mode = mode;
-  if (chunk > 0) g_tc_chunk = chunk;
-  g_tc_margin = margin;
 }
 
 }  // namespace taskkv

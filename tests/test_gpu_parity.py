@@ -217,3 +217,47 @@ def test_flat_entry_point_and_host_buffers():
     out_h = torch.empty(q.shape, dtype=q.dtype).pin_memory()
     host.taskkv_decode_host(q.cpu().pin_memory(), kn.cpu().pin_memory(), vn.cpu().pin_memory(), out_h)
     assert torch.equal(out_h, want.cpu())
+
+
+# ---------------------------------------------------------------- the benchmark workloads
+def test_llama2_config_full_size_sampled_layers():
+    """Config 2 at full size (32 layers, 32 heads x 128, 32768 tokens, bf16), in the launch configuration
+    bench.py times; the oracle checks the first, a middle and the last layer, then four decode steps."""
+    from paper_2501_15113_b200 import configs
+    wl = configs.config2_llama2()
+    rep = run_workload(wl, layers=[(0, 0), (0, 13), (0, 31)], decode_steps=4, check_pool=False)
+    assert rep.class_near_ties == 0
+    assert rep.units == 96
+
+
+def test_llama3_shaped_gqa_with_budget_schedule():
+    """Config 3 scaled down: GQA 32q / 8kv, Eq. 16 schedule over the KV heads, Eq. 17 budgets for a 40 %
+    cache, 128 window rows on the tensor-core path."""
+    from paper_2501_15113_b200 import configs
+    wl = configs.config3_llama3(seq_len=6000, n_layers=3, decode_steps=3)
+    assert wl.n_hetero[0] == [2, 2, 1] and len(set(wl.mid_budget)) == 2
+    run_workload(wl)
+    full = wl.n_layers * wl.n_kv_heads * wl.seq_lens[0]
+    assert 0.39 < wl.retained_rows() / full <= 0.4
+
+
+def test_long_sequence_radix_select_path():
+    """More than 32768 keys per unit: the selection falls back to the multi-pass radix path."""
+    wl = small("long", n=8, n_kv=2, d=128, N=40000, L=32, s1=4, s2=256, k=1500, dtype="bf16", nh=0, steps=2)
+    run_workload(wl, check_pool=False)
+
+
+def test_mistral_shaped_ragged_batch():
+    """Config 4 scaled down: a ragged batch with a different number of heterogeneous heads per sequence."""
+    from paper_2501_15113_b200 import configs
+    wl = configs.config4_mistral(batch=4, lo=1500, hi=5000, n_layers=2, decode_steps=3)
+    assert len(set(wl.seq_lens)) > 1
+    run_workload(wl)
+
+
+@pytest.mark.parametrize("n_hetero,mid", [(0, 64), (2, 256), (8, 1024)])
+def test_budget_sweep_points(n_hetero, mid):
+    """Config 5 scaled down: planted fraction x middle budget."""
+    from paper_2501_15113_b200 import configs
+    wl = configs.config5_sweep(n_hetero, mid, seq_len=5000, batch=2, decode_steps=2)
+    run_workload(wl)
