@@ -137,7 +137,8 @@ def run_ours(args):
     peak, peak_kind = load_peaks()
 
     wl = get_workload(args.workload, args)
-    wl.seed += 1000 * rank            # weak scaling: every rank owns an independent replica of the batch
+    from paper_2501_15113_b200 import sharding
+    wl.seed = sharding.replica_seed(wl.seed, rank)   # weak scaling: every rank owns an independent replica
     wl.planted = W._choose_planted(wl)
     S = wl.decode_steps
     qs, ks, vs = W.materialize(wl, dev)
@@ -193,11 +194,11 @@ def run_ours(args):
     total_ms = t0.elapsed_time(t1)
     comp_ms = sum(e[0].elapsed_time(e[1]) for e in evs)
     dec_ms = sum(e[1].elapsed_time(e[2]) for e in evs)
-    if world > 1:
-        import torch.distributed as dist
-        t = torch.tensor([total_ms, comp_ms, dec_ms], device=dev, dtype=torch.float64)
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-        total_ms, comp_ms, dec_ms = t.tolist()
+    K = args.steps
+    # whole-job rates: units of all ranks over the slowest rank's time (one small all-reduce when N > 1)
+    value, dec_ms = sharding.job_throughput(K * S, dec_ms, device=dev)
+    comp_tps, comp_ms = sharding.job_throughput(K * sum(wl.seq_lens), comp_ms, device=dev)
+    _, total_ms = sharding.job_throughput(K, total_ms, device=dev)
 
     # per-kernel durations: one more identical pass with every launch bracketed by events on its stream
     tk.taskkv_timing_enable(True)
@@ -210,7 +211,6 @@ def run_ours(args):
         a[0] += 1
         a[1] += ms
 
-    K = args.steps
     tokens = sum(wl.seq_lens)
     es, d = wl.elem_size, wl.head_dim
     comp_bytes = algorithmic_bytes(wl, info)
@@ -219,8 +219,6 @@ def run_ours(args):
     dec_bytes_avg = 2 * d * es * (int(info.retained_rows) + U * (S + 1) / 2.0)
     dec_step_ms = dec_ms / (K * S)
     comp_pass_ms = comp_ms / K
-    value = world * 1e3 / dec_step_ms
-    comp_tps = world * tokens * 1e3 / comp_pass_ms
 
     kern = {}
     for name, (n, ms) in per.items():
@@ -384,7 +382,7 @@ def run_reference(args):
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
-    ap.add_argument("--steps", type=int, default=5)
+    ap.add_argument("--steps", type=int, default=10)
     ap.add_argument("--warmup", type=int, default=3)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--workload", default="llama2")
