@@ -234,7 +234,7 @@ def test_llama3_shaped_gqa_with_budget_schedule():
     """Config 3 scaled down: GQA 32q / 8kv, Eq. 16 schedule over the KV heads, Eq. 17 budgets for a 40 %
     cache, 128 window rows on the tensor-core path."""
     from paper_2501_15113_b200 import configs
-    wl = configs.config3_llama3(seq_len=6000, n_layers=3, decode_steps=3)
+    wl = configs.config3_llama3(seq_len=12000, n_layers=3, decode_steps=3)
     assert wl.n_hetero[0] == [2, 2, 1] and len(set(wl.mid_budget)) == 2
     run_workload(wl)
     full = wl.n_layers * wl.n_kv_heads * wl.seq_lens[0]
