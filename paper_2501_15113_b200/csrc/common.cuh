@@ -10,7 +10,7 @@
 
 namespace taskkv {
 
-constexpr int kDecodeChunk = 256;                 // rows of one split-K decode item
+constexpr int kDecodeChunk = 512;                 // rows of one split-K decode item
 constexpr int kGatherRows = 64;                   // rows of one gather item
 constexpr int kScoreChunk = 1024;                 // keys of one window-score work item (CUDA-core path)
 constexpr int kTcChunk = 1024;                    // keys of one window-score work item (tensor-core path)

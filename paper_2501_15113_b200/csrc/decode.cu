@@ -2,7 +2,7 @@
 // head, no mask): o_a = softmax(q_a K_u^T / sqrt(d)) V_u over the len_u rows of
 // the KV head's segment, for the G query heads that share it.
 //
-// Split-K: a unit's rows are cut into work items of kDecodeChunk rows, numbered
+// Split-K: a unit's rows are cut into work items of kDecodeChunk (512) rows, numbered
 // by an exclusive scan over the units (so a 32768-row full head and a 772-row
 // pruned head load the SMs alike).  Each item produces an un-normalised partial
 // (running max, sum, weighted V) per head with an online softmax in fp32; one
@@ -164,23 +164,30 @@ __global__ void __launch_bounds__(kAttnThreads) decode_attn_kernel(DeviceProblem
   }
 }
 
-// One warp per (unit, query head of the group): merge the unit's partials.
+// One block per (unit, query head of the group): merge the unit's partials.  First the block finds
+// the largest running maximum, then each warp accumulates every fourth partial against it (independent
+// loads, fixed order), and the four warps are summed in shared memory.
 template <typename T, int D, int G>
-__global__ void __launch_bounds__(256) decode_combine_kernel(DeviceProblem p, T* __restrict__ out) {
+__global__ void __launch_bounds__(kAttnThreads) decode_combine_kernel(DeviceProblem p, T* __restrict__ out) {
   constexpr int EPL = D / 32;
-  const int w = blockIdx.x * 8 + (threadIdx.x >> 5);
-  const int lane = threadIdx.x & 31;
-  if (w >= p.U * G) return;
-  const int u = w / G, g = w % G;
+  __shared__ float s_max[kAttnWarps];
+  __shared__ float s_l[kAttnWarps];
+  __shared__ float s_acc[kAttnWarps][D];
+  const int u = blockIdx.x / G, g = blockIdx.x % G;
+  const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
   const int i0 = p.dec_off[u], i1 = p.dec_off[u + 1];
   float M = -INFINITY;
-  for (int i = i0 + lane; i < i1; i += 32) M = fmaxf(M, p.part_ml[((size_t)i * G + g) * 2]);
+  for (int i = i0 + tid; i < i1; i += kAttnThreads) M = fmaxf(M, p.part_ml[((size_t)i * G + g) * 2]);
   M = warp_max(M);
+  if (lane == 0) s_max[warp] = M;
+  __syncthreads();
+  M = fmaxf(fmaxf(s_max[0], s_max[1]), fmaxf(s_max[2], s_max[3]));
   float acc[EPL];
 #pragma unroll
   for (int e = 0; e < EPL; ++e) acc[e] = 0.f;
   float L = 0.f;
-  for (int i = i0; i < i1; ++i) {
+#pragma unroll 4
+  for (int i = i0 + warp; i < i1; i += kAttnWarps) {
     const float mi = p.part_ml[((size_t)i * G + g) * 2];
     const float li = p.part_ml[((size_t)i * G + g) * 2 + 1];
     const float wgt = (mi == -INFINITY) ? 0.f : exp2f(mi - M);
@@ -189,16 +196,22 @@ __global__ void __launch_bounds__(256) decode_combine_kernel(DeviceProblem p, T*
 #pragma unroll
     for (int e = 0; e < EPL; ++e) acc[e] = fmaf(wgt, pa[e], acc[e]);
   }
-  const float inv = L > 0.f ? 1.0f / L : 0.f;
-  T* o = out + ((size_t)u * G + g) * D + lane * EPL;
 #pragma unroll
-  for (int e = 0; e < EPL; ++e) store_out(o + e, acc[e] * inv);
+  for (int e = 0; e < EPL; ++e) s_acc[warp][lane * EPL + e] = acc[e];
+  if (lane == 0) s_l[warp] = L;
+  __syncthreads();
+  if (tid < D) {
+    const float Lt = (s_l[0] + s_l[1]) + (s_l[2] + s_l[3]);
+    const float a = (s_acc[0][tid] + s_acc[1][tid]) + (s_acc[2][tid] + s_acc[3][tid]);
+    store_out(out + ((size_t)u * G + g) * D + tid, Lt > 0.f ? a / Lt : 0.f);
+  }
 }
 
 template <typename T, int D, int G>
 cudaError_t launch_typed(const DeviceProblem& p, const void* q, const int32_t* lengths, void* out,
                          cudaStream_t s) {
-  int64_t grid = p.max_items < 148 * 8 ? p.max_items : 148 * 8;
+  // persistent blocks: 16 per SM (measured best on B200 with 512-row items)
+  int64_t grid = p.max_items < 148 * 16 ? p.max_items : 148 * 16;
   if (grid < 1) grid = 1;
   {
     LaunchScope ls(K_DECODE_ATTN, s);
@@ -206,7 +219,7 @@ cudaError_t launch_typed(const DeviceProblem& p, const void* q, const int32_t* l
   }
   {
     LaunchScope ls(K_DECODE_COMBINE, s);
-    decode_combine_kernel<T, D, G><<<(unsigned)((p.U * G + 7) / 8), 256, 0, s>>>(p, static_cast<T*>(out));
+    decode_combine_kernel<T, D, G><<<(unsigned)(p.U * G), kAttnThreads, 0, s>>>(p, static_cast<T*>(out));
   }
   return cudaGetLastError();
 }
