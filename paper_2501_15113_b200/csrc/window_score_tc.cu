@@ -30,7 +30,7 @@ namespace {
 
 constexpr int kTile = 128;          // keys per tile (UMMA M in pass 2, key sub-tiles in pass 1)
 constexpr int kStages = 4;          // K tiles in flight per CTA
-constexpr int kThreads = 192;
+constexpr int kThreads = 224;       // producer, issuer, 4 epilogue warps, second issuer
 constexpr uint32_t kTmemCols = 256; // two accumulator stages of up to 128 columns
 constexpr uint32_t kSpinLimit = 1u << 22;
 
@@ -252,7 +252,7 @@ window_tc_kernel(const __grid_constant__ CUtensorMap tmap_k, const __grid_consta
     for (int i = 0; i < kStages; ++i) { mbar_init(BAR(B_FULL + i), 1); mbar_init(BAR(B_EMPTY + i), 1); }
     for (int i = 0; i < 2; ++i) {
       mbar_init(BAR(B_QFULL + i), 1);
-      mbar_init(BAR(B_QEMPTY + i), 1);
+      mbar_init(BAR(B_QEMPTY + i), 2);     // both issuers release a Q block
       mbar_init(BAR(B_TFULL + i), 1);
       mbar_init(BAR(B_TEMPTY + i), 4);
     }
@@ -307,11 +307,14 @@ window_tc_kernel(const __grid_constant__ CUtensorMap tmap_k, const __grid_consta
       }
       for (int i = 0; i < 2 && ok; ++i, qb ^= 1) ok = mbar_wait(BAR(B_QEMPTY + qb), qphase[qb] ^ 1, s_abort);
     }
-  } else if (warp == 1) {
-    // ------------------------------------------------------------ MMA issuer: D[key, row] = K Q^T, both passes
+  } else if (warp == 1 || warp == 6) {
+    // ------------------------------------------------------------ MMA issuers: D[key, row] = K Q^T, both passes.
+    // Two elected threads, one per accumulator: the issue -> commit -> hand-over chain of one tile
+    // overlaps with the other's.  Tiles are numbered n = 0, 1, ... per CTA; issuer n & 1 takes tile n.
     if (lane == 0) {
-      int stage = 0, acc = 0, qb = 0;
-      uint32_t phase = 0, accphase = 0, qphase[2] = {0, 0};
+      const int me = warp == 1 ? 0 : 1;
+      int qb = 0, n = 0;
+      uint32_t qphase[2] = {0, 0};
       const uint32_t idesc = instr_desc(128, rows);
       bool ok = true;
       for (int s = blockIdx.x; s < a.total && ok; s += gridDim.x) {
@@ -323,7 +326,10 @@ window_tc_kernel(const __grid_constant__ CUtensorMap tmap_k, const __grid_consta
         if (!ok) break;
         qphase[qb] ^= 1;
         const uint32_t qbase = smem_u32(sQ + (size_t)qb * TcSmem<D>::kQBlockBytes);
-        for (int t = 0; t < ntiles; ++t) {
+        for (int t = 0; t < ntiles; ++t, ++n) {
+          if ((n & 1) != me) continue;
+          const int stage = n % kStages, acc = n & 1;
+          const uint32_t phase = (uint32_t)((n / kStages) & 1), accphase = (uint32_t)((n >> 1) & 1);
           ok = mbar_wait(BAR(B_FULL + stage), phase, s_abort);
           if (!ok) break;
           ok = mbar_wait(BAR(B_TEMPTY + acc), accphase ^ 1, s_abort);
@@ -341,14 +347,13 @@ window_tc_kernel(const __grid_constant__ CUtensorMap tmap_k, const __grid_consta
             }
           tc_commit(BAR(B_EMPTY + stage));   // smem stage free once these MMAs have read it
           tc_commit(BAR(B_TFULL + acc));     // accumulator ready for the epilogue
-          if (++stage == kStages) { stage = 0; phase ^= 1; }
-          if (++acc == 2) { acc = 0; accphase ^= 1; }
         }
-        tc_commit(BAR(B_QEMPTY + qb));       // Q block free once the item's MMAs are done
+        if (!ok) break;
+        tc_commit(BAR(B_QEMPTY + qb));       // this issuer is done with the Q block
         qb ^= 1;
       }
     }
-  } else {
+  } else if (warp >= 2 && warp <= 5) {
     // ------------------------------------------------------------ epilogue: 4 warps, a TMEM lane is a key
     const int quad = warp & 3;                      // TMEM lane quadrant this warp may read
     float2* myStat = sStat + (warp - 2) * 128;
