@@ -29,9 +29,10 @@ namespace taskkv {
 namespace {
 
 constexpr int kTile = 128;          // keys per tile (UMMA M in pass 2, key sub-tiles in pass 1)
-constexpr int kStages = 4;          // K tiles in flight per CTA
-constexpr int kThreads = 224;       // producer, issuer, 4 epilogue warps, second issuer
-constexpr uint32_t kTmemCols = 256; // two accumulator stages of up to 128 columns
+constexpr int kMaxStages = 6;       // K tiles in flight per CTA (the count is fitted to shared memory)
+constexpr int kEpiWarps = 8;        // two groups of four epilogue warps, alternating tiles
+constexpr int kThreads = 352;       // warp 0 producer; 1, 6 MMA issuers; 2-5 and 7-10 epilogue groups
+constexpr uint32_t kTmemCols = 512; // four accumulators of up to 128 columns
 constexpr uint32_t kSpinLimit = 1u << 22;
 
 // Work items of one launch (one sequence): (pass, unit, chunk of chunk_keys keys).
@@ -208,55 +209,78 @@ __device__ __forceinline__ uint32_t instr_desc(int M, int N) {
   return (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(N >> 3) << 17) | ((uint32_t)(M >> 4) << 24);
 }
 
-template <int D>
-struct TcSmem {
-  static constexpr int KB = D / 64;                       // 128-byte k-blocks per row
-  static constexpr int kTileBytes = KB * kTile * 128;     // one K tile
-  static constexpr int kQBlockBytes = KB * 128 * 128;     // one Q block (up to 128 rows), double buffered
-  static constexpr int kStatBytes = 4 * 128 * (int)sizeof(float2);
-  static constexpr int kTransBytes = 4 * 32 * 33 * (int)sizeof(float);   // per-warp 32x32 transposition tiles
-  static constexpr int kMergeBytes = 2 * 4 * 128 * (int)sizeof(float2);  // [item parity][warp][row]
-  static constexpr int kBytes =
-      kStages * kTileBytes + 2 * kQBlockBytes + kStatBytes + kTransBytes + kMergeBytes + 256 + 1024;
+// Shared-memory plan, made on the host: the Q blocks and the per-warp areas scale with the number of
+// window rows; what is left of the 227 KB goes to K stages (an even count, so that each stage is always
+// consumed by the same issuer).
+struct TcLayout {
+  int stages;
+  int tile_bytes, q_block_bytes;
+  int off_q, off_stat, off_trans, off_merge, off_bars;
+  int total;
 };
+
+inline TcLayout make_layout(int D, int rows) {
+  TcLayout l;
+  const int KB = D / 64;
+  l.tile_bytes = KB * kTile * 128;
+  l.q_block_bytes = KB * rows * 128;
+  const int stat = kEpiWarps * rows * (int)sizeof(float2);
+  const int trans = kEpiWarps * 32 * 33 * (int)sizeof(float);
+  const int merge = 2 * kEpiWarps * rows * (int)sizeof(float2);
+  const int bars = 512;
+  const int budget = 232448 - 1024;     // dynamic shared memory of one CTA minus the alignment slack
+  int stages = (budget - 2 * l.q_block_bytes - stat - trans - merge - bars) / l.tile_bytes;
+  if (stages > kMaxStages) stages = kMaxStages;
+  l.stages = stages & ~1;
+  l.off_q = l.stages * l.tile_bytes;
+  l.off_stat = l.off_q + 2 * l.q_block_bytes;
+  l.off_trans = l.off_stat + stat;
+  l.off_merge = l.off_trans + trans;
+  l.off_bars = l.off_merge + merge;
+  l.total = l.off_bars + bars + 1024;
+  return l;
+}
 
 // barrier slots
 enum : int {
-  B_FULL = 0, B_EMPTY = 4, B_QFULL = 8, B_QEMPTY = 10, B_TFULL = 12, B_TEMPTY = 14, B_EPI = 16, B_COUNT = 17
+  B_FULL = 0, B_EMPTY = 8, B_QFULL = 16, B_QEMPTY = 18, B_TFULL = 20, B_TEMPTY = 24, B_EPI = 28, B_COUNT = 29
 };
 
 template <int D>
 __global__ void __launch_bounds__(kThreads, 1)
 window_tc_kernel(const __grid_constant__ CUtensorMap tmap_k, const __grid_constant__ CUtensorMap tmap_q,
-                 DeviceProblem p, TcArgs a) {
-  constexpr int KB = TcSmem<D>::KB;
+                 DeviceProblem p, TcArgs a, TcLayout lay) {
+  constexpr int KB = D / 64;
   extern __shared__ unsigned char smem_raw[];
   // 1024-byte alignment: the swizzle pattern is a function of the address bits
   unsigned char* smem = reinterpret_cast<unsigned char*>(((uintptr_t)smem_raw + 1023) & ~(uintptr_t)1023);
-  unsigned char* sK = smem;                                         // [kStages][KB][128 keys][128 B]
-  unsigned char* sQ = sK + kStages * TcSmem<D>::kTileBytes;         // [2][KB][rows][128 B]
-  float2* sStat = reinterpret_cast<float2*>(sQ + 2 * TcSmem<D>::kQBlockBytes);   // [4 warps][128]
-  float* sTrans = reinterpret_cast<float*>(reinterpret_cast<unsigned char*>(sStat) + TcSmem<D>::kStatBytes);
-  float2* sMerge = reinterpret_cast<float2*>(reinterpret_cast<unsigned char*>(sTrans) + TcSmem<D>::kTransBytes);
-  uint64_t* bars = reinterpret_cast<uint64_t*>(reinterpret_cast<unsigned char*>(sMerge) + TcSmem<D>::kMergeBytes);
+  unsigned char* sK = smem;                                         // [stages][KB][128 keys][128 B]
+  unsigned char* sQ = smem + lay.off_q;                             // [2][KB][rows][128 B]
+  float2* sStat = reinterpret_cast<float2*>(smem + lay.off_stat);   // [8 warps][rows]
+  float* sTrans = reinterpret_cast<float*>(smem + lay.off_trans);   // [8 warps][32][33]
+  float2* sMerge = reinterpret_cast<float2*>(smem + lay.off_merge); // [2][8 warps][rows]
+  uint64_t* bars = reinterpret_cast<uint64_t*>(smem + lay.off_bars);
   uint32_t* s_tmem = reinterpret_cast<uint32_t*>(bars + B_COUNT);
   volatile int* s_abort = reinterpret_cast<volatile int*>(s_tmem + 1);
 
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
   const int rows = p.rows;                  // 32, 64 or 128
   const int N = a.N, L = p.L;
+  const int S = lay.stages;
   const uint32_t bar0 = smem_u32(bars);
   auto BAR = [&](int i) { return bar0 + 8u * (uint32_t)i; };
 
   if (tid == 0) {
-    for (int i = 0; i < kStages; ++i) { mbar_init(BAR(B_FULL + i), 1); mbar_init(BAR(B_EMPTY + i), 1); }
+    for (int i = 0; i < kMaxStages; ++i) { mbar_init(BAR(B_FULL + i), 1); mbar_init(BAR(B_EMPTY + i), 1); }
+    for (int i = 0; i < 4; ++i) {
+      mbar_init(BAR(B_TFULL + i), 1);
+      mbar_init(BAR(B_TEMPTY + i), 4);     // the four warps of the group that reads the accumulator
+    }
     for (int i = 0; i < 2; ++i) {
       mbar_init(BAR(B_QFULL + i), 1);
       mbar_init(BAR(B_QEMPTY + i), 2);     // both issuers release a Q block
-      mbar_init(BAR(B_TFULL + i), 1);
-      mbar_init(BAR(B_TEMPTY + i), 4);
     }
-    mbar_init(BAR(B_EPI), 128);
+    mbar_init(BAR(B_EPI), 32 * kEpiWarps);
     *s_abort = 0;
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
   }
@@ -283,34 +307,35 @@ window_tc_kernel(const __grid_constant__ CUtensorMap tmap_k, const __grid_consta
         const int ntiles = (min(N, key0 + a.chunk_keys) - key0 + kTile - 1) / kTile;
         ok = mbar_wait(BAR(B_QEMPTY + qb), qphase[qb] ^ 1, s_abort);
         if (!ok) break;
-        mbar_expect_tx(BAR(B_QFULL + qb), (uint32_t)(KB * rows * 128));
+        mbar_expect_tx(BAR(B_QFULL + qb), (uint32_t)lay.q_block_bytes);
         for (int kb = 0; kb < KB; ++kb)
-          tma_load_2d(smem_u32(sQ + (size_t)qb * TcSmem<D>::kQBlockBytes + (size_t)kb * rows * 128), &tmap_q, kb * 64,
+          tma_load_2d(smem_u32(sQ + (size_t)qb * lay.q_block_bytes + (size_t)kb * rows * 128), &tmap_q, kb * 64,
                       it.lu * rows, BAR(B_QFULL + qb));
         qphase[qb] ^= 1;
         qb ^= 1;
         for (int t = 0; t < ntiles; ++t) {
           ok = mbar_wait(BAR(B_EMPTY + stage), phase ^ 1, s_abort);
           if (!ok) break;
-          mbar_expect_tx(BAR(B_FULL + stage), (uint32_t)TcSmem<D>::kTileBytes);
+          mbar_expect_tx(BAR(B_FULL + stage), (uint32_t)lay.tile_bytes);
           for (int kb = 0; kb < KB; ++kb)
-            tma_load_2d(smem_u32(sK + (size_t)stage * TcSmem<D>::kTileBytes + (size_t)kb * kTile * 128), &tmap_k,
+            tma_load_2d(smem_u32(sK + (size_t)stage * lay.tile_bytes + (size_t)kb * kTile * 128), &tmap_k,
                         kb * 64, it.lu * N + key0 + t * kTile, BAR(B_FULL + stage));
-          if (++stage == kStages) { stage = 0; phase ^= 1; }
+          if (++stage == S) { stage = 0; phase ^= 1; }
         }
       }
       // Drain: every tcgen05.commit aimed at this CTA's barriers must have arrived before the CTA exits,
       // or it would land on the barriers of the next CTA that is given this shared memory.
-      for (int i = 0; i < kStages && ok; ++i) {
+      for (int i = 0; i < S && ok; ++i) {
         ok = mbar_wait(BAR(B_EMPTY + stage), phase ^ 1, s_abort);
-        if (++stage == kStages) { stage = 0; phase ^= 1; }
+        if (++stage == S) { stage = 0; phase ^= 1; }
       }
       for (int i = 0; i < 2 && ok; ++i, qb ^= 1) ok = mbar_wait(BAR(B_QEMPTY + qb), qphase[qb] ^ 1, s_abort);
     }
   } else if (warp == 1 || warp == 6) {
     // ------------------------------------------------------------ MMA issuers: D[key, row] = K Q^T, both passes.
-    // Two elected threads, one per accumulator: the issue -> commit -> hand-over chain of one tile
-    // overlaps with the other's.  Tiles are numbered n = 0, 1, ... per CTA; issuer n & 1 takes tile n.
+    // Two elected threads: the issue -> commit -> hand-over chain of one tile overlaps with the other's.
+    // Tiles are numbered n = 0, 1, ... per CTA across items: issuer n & 1, smem stage n % stages, TMEM
+    // accumulator n & 3 (read by epilogue group n & 1).
     if (lane == 0) {
       const int me = warp == 1 ? 0 : 1;
       int qb = 0, n = 0;
@@ -325,18 +350,18 @@ window_tc_kernel(const __grid_constant__ CUtensorMap tmap_k, const __grid_consta
         ok = mbar_wait(BAR(B_QFULL + qb), qphase[qb], s_abort);
         if (!ok) break;
         qphase[qb] ^= 1;
-        const uint32_t qbase = smem_u32(sQ + (size_t)qb * TcSmem<D>::kQBlockBytes);
+        const uint32_t qbase = smem_u32(sQ + (size_t)qb * lay.q_block_bytes);
         for (int t = 0; t < ntiles; ++t, ++n) {
           if ((n & 1) != me) continue;
-          const int stage = n % kStages, acc = n & 1;
-          const uint32_t phase = (uint32_t)((n / kStages) & 1), accphase = (uint32_t)((n >> 1) & 1);
+          const int stage = n % S, acc = n & 3;
+          const uint32_t phase = (uint32_t)((n / S) & 1), accphase = (uint32_t)((n >> 2) & 1);
           ok = mbar_wait(BAR(B_FULL + stage), phase, s_abort);
           if (!ok) break;
           ok = mbar_wait(BAR(B_TEMPTY + acc), accphase ^ 1, s_abort);
           if (!ok) break;
           tc_fence_after();
           const uint32_t d_tmem = tmem_base + (uint32_t)acc * 128u;
-          const uint32_t kt = smem_u32(sK + (size_t)stage * TcSmem<D>::kTileBytes);
+          const uint32_t kt = smem_u32(sK + (size_t)stage * lay.tile_bytes);
 #pragma unroll
           for (int kb = 0; kb < KB; ++kb)
 #pragma unroll
@@ -353,20 +378,22 @@ window_tc_kernel(const __grid_constant__ CUtensorMap tmap_k, const __grid_consta
         qb ^= 1;
       }
     }
-  } else if (warp >= 2 && warp <= 5) {
-    // ------------------------------------------------------------ epilogue: 4 warps, a TMEM lane is a key
+  } else {
+    // ------------------------------------------------------------ epilogue: two groups of 4 warps (2-5 take
+    // even tiles, 7-10 odd tiles); a TMEM lane is a key
+    const int ew = warp < 6 ? warp - 2 : warp - 3;  // 0..7
+    const int grp = ew >> 2;
     const int quad = warp & 3;                      // TMEM lane quadrant this warp may read
-    float2* myStat = sStat + (warp - 2) * 128;
-    float* myT = sTrans + (warp - 2) * (32 * 33);
-    int acc = 0;
-    uint32_t accphase = 0, epiphase = 0;
-    int n_done = 0;
+    float2* myStat = sStat + ew * rows;
+    float* myT = sTrans + ew * (32 * 33);
+    uint32_t epiphase = 0;
+    int n = 0, n_done = 0;
     bool ok = true;
     for (int s = blockIdx.x; s < a.total && ok; s += gridDim.x) {
       const Item it = decode_item(a, s);
       if (it.fin_unit >= 0) {
         // combine the unit's per-item statistics, in item order, into (row max, 1 / row sum)
-        const int row = (warp - 2) * 32 + lane;
+        const int row = ew * 32 + lane;
         if (row < rows) {
           const int uf = a.u0 + it.fin_unit;
           const float2* part = reinterpret_cast<const float2*>(p.stat_part) + (size_t)uf * p.chunks_max * p.rows_pad;
@@ -418,7 +445,10 @@ window_tc_kernel(const __grid_constant__ CUtensorMap tmap_k, const __grid_consta
         ok = __all_sync(0xffffffffu, ok);
         if (!ok) break;
       }
-      for (int t = 0; t < ntiles; ++t) {
+      for (int t = 0; t < ntiles; ++t, ++n) {
+        if ((n & 1) != grp) continue;
+        const int acc = n & 3;
+        const uint32_t accphase = (uint32_t)((n >> 2) & 1);
         ok = __all_sync(0xffffffffu, mbar_wait(BAR(B_TFULL + acc), accphase, s_abort));
         if (!ok) break;
         tc_fence_after();
@@ -492,28 +522,27 @@ window_tc_kernel(const __grid_constant__ CUtensorMap tmap_k, const __grid_consta
         tc_fence_before();
         __syncwarp();
         if (lane == 0) mbar_arrive(BAR(B_TEMPTY + acc));
-        if (++acc == 2) { acc = 0; accphase ^= 1; }
       }
       if (!ok) break;
       if (it.pass == 1) {
-        // merge the four warps' (max, sum) per row in a fixed order; one slot per work item
-        float2* mg = sMerge + (n_done & 1) * (4 * 128);
+        // merge the eight warps' (max, sum) per row in a fixed order; one slot per work item
+        float2* mg = sMerge + (n_done & 1) * (kEpiWarps * rows);
 #pragma unroll
         for (int rg = 0; rg < 4; ++rg)
-          if (rg * 32 < rows) mg[(warp - 2) * 128 + rg * 32 + lane] = make_float2(m_run[rg] * scale2, z_run[rg]);
+          if (rg * 32 < rows) mg[ew * rows + rg * 32 + lane] = make_float2(m_run[rg] * scale2, z_run[rg]);
         mbar_arrive(BAR(B_EPI));
         ok = __all_sync(0xffffffffu, mbar_wait(BAR(B_EPI), epiphase, s_abort));
         epiphase ^= 1;
         if (!ok) break;
-        const int tl = (warp - 2) * 32 + lane;
+        const int tl = ew * 32 + lane;
         if (tl < rows) {
           float M = -INFINITY;
 #pragma unroll
-          for (int w = 0; w < 4; ++w) M = fmaxf(M, mg[w * 128 + tl].x);
+          for (int w = 0; w < kEpiWarps; ++w) M = fmaxf(M, mg[w * rows + tl].x);
           float z = 0.f;
 #pragma unroll
-          for (int w = 0; w < 4; ++w) {
-            const float2 o = mg[w * 128 + tl];
+          for (int w = 0; w < kEpiWarps; ++w) {
+            const float2 o = mg[w * rows + tl];
             if (o.x > -INFINITY) z = fmaf(o.y, ex2(o.x - M), z);
           }
           publish_pair(reinterpret_cast<float2*>(p.stat_part) + ((size_t)u * p.chunks_max + it.ch) * p.rows_pad + tl,
@@ -603,7 +632,9 @@ cudaError_t launch_tc_d(const DeviceProblem& p, const WindowHostInfo& h, cudaStr
     cudaDeviceGetAttribute(&n_sm, cudaDevAttrMultiProcessorCount, dev);
     if (n_sm <= 0) n_sm = 148;
   }
-  const int smem = TcSmem<D>::kBytes;
+  const TcLayout lay = make_layout(D, p.rows);
+  if (lay.stages < 2) return cudaErrorInvalidValue;
+  const int smem = lay.total;
   cudaError_t e = cudaFuncSetAttribute(window_tc_kernel<D>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem);
   if (e != cudaSuccess) return e;
   // partial and final statistics start as NaN = "not written"
@@ -631,14 +662,14 @@ cudaError_t launch_tc_d(const DeviceProblem& p, const WindowHostInfo& h, cudaStr
       a.mode = 0;
       a.total = 2 * (n1 + a.lag2);
       LaunchScope ls(K_WINDOW_TC, s);
-      window_tc_kernel<D><<<a.total < n_sm ? a.total : n_sm, kThreads, smem, s>>>(mk, mq, p, a);
+      window_tc_kernel<D><<<a.total < n_sm ? a.total : n_sm, kThreads, smem, s>>>(mk, mq, p, a, lay);
     } else {
       a.total = n1;
       const int grid = a.total < n_sm ? a.total : n_sm;
       a.mode = 1;
       {
         LaunchScope ls(K_WINDOW_TC, s);
-        window_tc_kernel<D><<<grid, kThreads, smem, s>>>(mk, mq, p, a);
+        window_tc_kernel<D><<<grid, kThreads, smem, s>>>(mk, mq, p, a, lay);
       }
       {
         LaunchScope ls(K_WINDOW_REDUCE, s);
@@ -647,7 +678,7 @@ cudaError_t launch_tc_d(const DeviceProblem& p, const WindowHostInfo& h, cudaStr
       a.mode = 2;
       {
         LaunchScope ls(K_WINDOW_TC, s);
-        window_tc_kernel<D><<<grid, kThreads, smem, s>>>(mk, mq, p, a);
+        window_tc_kernel<D><<<grid, kThreads, smem, s>>>(mk, mq, p, a, lay);
       }
     }
     e = cudaGetLastError();
