@@ -35,16 +35,17 @@ constexpr int kThreads = 352;       // warp 0 producer; 1, 6 MMA issuers; 2-5 an
 constexpr uint32_t kTmemCols = 512; // four accumulators of up to 128 columns
 constexpr uint32_t kSpinLimit = 1u << 22;
 
-// Work items of one launch (one sequence): (pass, unit, chunk of chunk_keys keys).
-// mode 1 / 2: one pass per launch, unit-major (statistics combined by a kernel in between).
-// mode 0: both passes in one launch so that the second read of the keys is served by L2.  Positions
-//   alternate between the pass-1 stream (item i at position 2i) and the pass-2 stream, which lags by
-//   `lag2` items; the statistics of unit u are combined ("finalised") by the epilogue warps of the CTA
-//   that takes pass-1 position u*C + C-1 + lag_r, i.e. lag_r items after the unit's last pass-1 item.
-//   lag_r and lag2 - C - lag_r exceed the number of positions in flight, so the data a step needs is
-//   normally there; if not, it polls (bounded): every partial and every statistic is one 8-byte word
-//   that is NaN until written, so no fence or counter is involved.  A step only ever depends on
-//   earlier positions, which resident CTAs taking positions in order have already started.
+// Work items of one launch (one sequence): (pass, unit, chunk of chunk_keys keys), numbered unit-major
+// i = unit * C + chunk.  CTA c of a grid of g CTAs owns the items i = c, c + g, c + 2g, ... of BOTH passes.
+// mode 1 / 2: one pass per launch (the statistics are combined by a small kernel in between).
+// mode 0: both passes in one launch, so that the second read of a chunk of keys comes from L2: in round r
+//   the CTA runs pass 1 on item c + r*g and then pass 2 on item c + (r - lag)*g -- the same SM that pulled
+//   the chunk into its side of the L2 a few rounds earlier.  Pass 2 of an item needs the statistics of
+//   its whole unit, i.e. the C per-item partials written by (mostly) other CTAs during rounds <= r - lag + 1;
+//   the epilogue combines them itself at the start of the item.  Every partial is one 8-byte word that
+//   is NaN until written, so no fence or counter is involved; a missing one is polled for (bounded).
+//   A step only ever depends on pass-1 items of earlier rounds, which resident CTAs that take their
+//   items in order have already started, so the wait always ends.
 struct TcArgs {
   int mode;
   int u0;            // first unit of this sequence
@@ -52,34 +53,28 @@ struct TcArgs {
   int N;             // sequence length
   int chunks;        // C: work items per unit and pass
   int chunk_keys;    // keys per work item (multiple of 128)
-  int lag_r, lag2;   // mode 0
-  int total;         // positions
+  int lag;           // mode 0: rounds between the two passes of an item
+  int steps;         // steps of every CTA
 };
 
 struct Item {
   int pass, lu, ch;
   bool valid;        // has tiles to process
-  int fin_unit;      // >= 0: first finalise this (local) unit's statistics
 };
-__device__ __forceinline__ Item decode_item(const TcArgs& a, int s) {
+__device__ __forceinline__ Item decode_item(const TcArgs& a, int k) {
   Item it;
-  it.fin_unit = -1;
   int i;
   if (a.mode != 0) {
     it.pass = a.mode;
-    i = s;
+    i = (int)blockIdx.x + k * (int)gridDim.x;
     it.valid = true;
-  } else if ((s & 1) == 0) {
-    it.pass = 1;
-    i = s >> 1;
-    it.valid = i < a.n_local * a.chunks;
-    const int r = i - a.lag_r - (a.chunks - 1);
-    if (r >= 0 && r % a.chunks == 0 && r / a.chunks < a.n_local) it.fin_unit = r / a.chunks;
   } else {
-    it.pass = 2;
-    i = (s >> 1) - a.lag2;
-    it.valid = i >= 0 && i < a.n_local * a.chunks;
+    const int r = k >> 1;
+    it.pass = (k & 1) ? 2 : 1;
+    i = (int)blockIdx.x + ((k & 1) ? r - a.lag : r) * (int)gridDim.x;
+    it.valid = i >= 0;
   }
+  it.valid = it.valid && i < a.n_local * a.chunks;
   it.lu = it.valid ? i / a.chunks : 0;
   it.ch = it.valid ? i % a.chunks : 0;
   return it;
@@ -300,8 +295,8 @@ window_tc_kernel(const __grid_constant__ CUtensorMap tmap_k, const __grid_consta
       int stage = 0, qb = 0;
       uint32_t phase = 0, qphase[2] = {0, 0};
       bool ok = true;
-      for (int s = blockIdx.x; s < a.total && ok; s += gridDim.x) {
-        const Item it = decode_item(a, s);
+      for (int k = 0; k < a.steps && ok; ++k) {
+        const Item it = decode_item(a, k);
         if (!it.valid) continue;
         const int key0 = it.ch * a.chunk_keys;
         const int ntiles = (min(N, key0 + a.chunk_keys) - key0 + kTile - 1) / kTile;
@@ -342,8 +337,8 @@ window_tc_kernel(const __grid_constant__ CUtensorMap tmap_k, const __grid_consta
       uint32_t qphase[2] = {0, 0};
       const uint32_t idesc = instr_desc(128, rows);
       bool ok = true;
-      for (int s = blockIdx.x; s < a.total && ok; s += gridDim.x) {
-        const Item it = decode_item(a, s);
+      for (int k = 0; k < a.steps && ok; ++k) {
+        const Item it = decode_item(a, k);
         if (!it.valid) continue;
         const int key0 = it.ch * a.chunk_keys;
         const int ntiles = (min(N, key0 + a.chunk_keys) - key0 + kTile - 1) / kTile;
@@ -389,44 +384,8 @@ window_tc_kernel(const __grid_constant__ CUtensorMap tmap_k, const __grid_consta
     uint32_t epiphase = 0;
     int n = 0, n_done = 0;
     bool ok = true;
-    for (int s = blockIdx.x; s < a.total && ok; s += gridDim.x) {
-      const Item it = decode_item(a, s);
-      if (it.fin_unit >= 0) {
-        // combine the unit's per-item statistics, in item order, into (row max, 1 / row sum)
-        const int row = ew * 32 + lane;
-        if (row < rows) {
-          const int uf = a.u0 + it.fin_unit;
-          const float2* part = reinterpret_cast<const float2*>(p.stat_part) + (size_t)uf * p.chunks_max * p.rows_pad;
-          float M = -INFINITY, z = 0.f;
-          for (int c0 = 0; c0 < a.chunks && ok; c0 += 8) {
-            uint64_t w[8];
-#pragma unroll
-            for (int i = 0; i < 8; ++i) {   // eight loads in flight, then consume in order
-              w[i] = ~0ull;
-              if (c0 + i < a.chunks)
-                asm volatile("ld.relaxed.gpu.global.b64 %0, [%1];"
-                             : "=l"(w[i]) : "l"(&part[(size_t)(c0 + i) * p.rows_pad + row]) : "memory");
-            }
-#pragma unroll
-            for (int i = 0; i < 8; ++i) {
-              if (c0 + i < a.chunks && ok) {
-                float2 o = make_float2(__uint_as_float((uint32_t)w[i]), __uint_as_float((uint32_t)(w[i] >> 32)));
-                if (o.y != o.y) ok = poll_pair(&part[(size_t)(c0 + i) * p.rows_pad + row], o, s_abort);
-                if (ok && o.x > -INFINITY) {
-                  const float Mn = fmaxf(M, o.x);
-                  z = fmaf(z, ex2(M - Mn), o.y * ex2(o.x - Mn));
-                  M = Mn;
-                }
-              }
-            }
-          }
-          if (ok)
-            publish_pair(reinterpret_cast<float2*>(p.stat) + (size_t)uf * p.rows_pad + row, z > 0.f ? M : 0.f,
-                         z > 0.f ? 1.0f / z : 0.f);
-        }
-        ok = __all_sync(0xffffffffu, ok);
-        if (!ok) break;
-      }
+    for (int k = 0; k < a.steps && ok; ++k) {
+      const Item it = decode_item(a, k);
       if (!it.valid) continue;
       const int u = a.u0 + it.lu;
       const int key0 = it.ch * a.chunk_keys;
@@ -435,7 +394,56 @@ window_tc_kernel(const __grid_constant__ CUtensorMap tmap_k, const __grid_consta
       float m_run[4], z_run[4];
 #pragma unroll
       for (int rg = 0; rg < 4; ++rg) { m_run[rg] = -INFINITY; z_run[rg] = 0.f; }
-      if (it.pass == 2) {
+      if (it.pass == 2 && a.mode == 0) {
+        // combine the unit's per-item partials (slot c = pass-1 item c of the unit), in a fixed order:
+        // rows are split over 256 / rows threads, each merging every (256 / rows)-th slot, then the
+        // parts are merged through shared memory and every warp keeps its own copy
+        const int tpr = (32 * kEpiWarps) / rows;
+        const int t = ew * 32 + lane, row = t % rows, part = t / rows;
+        const float2* slot = reinterpret_cast<const float2*>(p.stat_part) + (size_t)u * p.chunks_max * p.rows_pad + row;
+        float M = -INFINITY, z = 0.f;
+        for (int c0 = part; c0 < a.chunks && ok; c0 += 8 * tpr) {
+          uint64_t w[8];
+#pragma unroll
+          for (int i = 0; i < 8; ++i) {   // eight loads in flight, then consume in order
+            w[i] = ~0ull;
+            const int c = c0 + i * tpr;
+            if (c < a.chunks)
+              asm volatile("ld.relaxed.gpu.global.b64 %0, [%1];" : "=l"(w[i]) : "l"(slot + (size_t)c * p.rows_pad) : "memory");
+          }
+#pragma unroll
+          for (int i = 0; i < 8; ++i) {
+            const int c = c0 + i * tpr;
+            if (c < a.chunks && ok) {
+              float2 o = make_float2(__uint_as_float((uint32_t)w[i]), __uint_as_float((uint32_t)(w[i] >> 32)));
+              if (o.y != o.y) ok = poll_pair(slot + (size_t)c * p.rows_pad, o, s_abort);
+              if (ok && o.x > -INFINITY) {
+                const float Mn = fmaxf(M, o.x);
+                z = fmaf(z, ex2(M - Mn), o.y * ex2(o.x - Mn));
+                M = Mn;
+              }
+            }
+          }
+        }
+        float2* mg = sMerge + (n_done & 1) * (kEpiWarps * rows);
+        mg[part * rows + row] = make_float2(M, z);
+        mbar_arrive(BAR(B_EPI));
+        ok = __all_sync(0xffffffffu, ok && mbar_wait(BAR(B_EPI), epiphase, s_abort));
+        epiphase ^= 1;
+        ++n_done;
+        if (!ok) break;
+        for (int i = lane; i < rows; i += 32) {
+          float Mt = -INFINITY;
+          for (int q = 0; q < tpr; ++q) Mt = fmaxf(Mt, mg[q * rows + i].x);
+          float zt = 0.f;
+          for (int q = 0; q < tpr; ++q) {
+            const float2 o = mg[q * rows + i];
+            if (o.x > -INFINITY) zt = fmaf(o.y, ex2(o.x - Mt), zt);
+          }
+          myStat[i] = zt > 0.f ? make_float2(Mt, 1.0f / zt) : make_float2(0.f, 0.f);
+        }
+        __syncwarp();
+      } else if (it.pass == 2) {
         __syncwarp();
         for (int i = lane; i < rows && ok; i += 32) {
           float2 o;
@@ -616,12 +624,13 @@ bool make_map(CUtensorMap* map, const void* base, int d, uint64_t rows_total, in
             CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
 }
 
-// One launch per pass.  The single-launch order (mode 0) exists and is exact, but measured slower:
-// the pipeline is bound on the SM side (one MMA issuer, one epilogue group), not by HBM, so serving the
-// second pass from L2 does not pay yet.
+// One launch per pass.  The single-launch order (mode 0) is exact, but measured no faster on B200: with the
+// keys served from L2 the kernel runs into the shared-memory bandwidth of the SM (TMA fill + MMA operand
+// reads + the pass-1 transposition, about 1000 cycles per 128-key tile against 1420 for HBM), and the
+// hit rate stayed low in every order tried.  Both passes run at the HBM copy rate instead.
 constexpr int g_tc_mode = 1;
 constexpr int g_tc_chunk = 2048;   // keys per work item
-constexpr int g_tc_margin = 0;     // 0: from the SM count
+constexpr int g_tc_lag = 2;        // single launch: rounds between the two passes of an item
 
 template <int D>
 cudaError_t launch_tc_d(const DeviceProblem& p, const WindowHostInfo& h, cudaStream_t s) {
@@ -654,18 +663,19 @@ cudaError_t launch_tc_d(const DeviceProblem& p, const WindowHostInfo& h, cudaStr
     a.chunk_keys = g_tc_chunk < kTcChunk ? kTcChunk : g_tc_chunk / 128 * 128;
     a.chunks = (N + a.chunk_keys - 1) / a.chunk_keys;
     const int n1 = a.n_local * a.chunks;
-    // a round of the resident CTAs covers n_sm positions = n_sm / 2 items of each stream
-    const int margin = g_tc_margin > 0 ? g_tc_margin : n_sm / 2 + 8;
-    a.lag_r = margin;
-    a.lag2 = a.chunks + 2 * margin;
-    if (g_tc_mode == 0) {
+    const int grid = n1 < n_sm ? n1 : n_sm;
+    const int rounds = (n1 + grid - 1) / grid;
+    // the single-launch order needs the partials of a unit within reach of one combine step
+    const bool single = g_tc_mode == 0 && a.chunks <= 64;
+    if (single) {
       a.mode = 0;
-      a.total = 2 * (n1 + a.lag2);
+      a.lag = g_tc_lag;
+      a.steps = 2 * (rounds + a.lag);
       LaunchScope ls(K_WINDOW_TC, s);
-      window_tc_kernel<D><<<a.total < n_sm ? a.total : n_sm, kThreads, smem, s>>>(mk, mq, p, a, lay);
+      window_tc_kernel<D><<<grid, kThreads, smem, s>>>(mk, mq, p, a, lay);
     } else {
-      a.total = n1;
-      const int grid = a.total < n_sm ? a.total : n_sm;
+      a.lag = 0;
+      a.steps = rounds;
       a.mode = 1;
       {
         LaunchScope ls(K_WINDOW_TC, s);
