@@ -244,8 +244,9 @@ def run_ours(args):
             "decode_bytes_per_step": dec_bytes_avg, "compress_bytes": comp_bytes,
         },
         "roofline": {"bound": "hbm", "kernel": "decode_attn", "achieved": attn_gbs, "peak": peak, "unit": "GB/s",
-                     "frac": attn_gbs / peak, "peak_kind": peak_kind, "traffic": None,
-                     "avg_launch_ms": attn["avg_ms"]},
+                     "frac": attn_gbs / peak, "peak_kind": peak_kind,
+                     "traffic": ncu_traffic(wl, int(info.retained_rows)), "traffic_unit": "bytes per launch",
+                     "algorithmic_bytes": dec_bytes_avg, "avg_launch_ms": attn["avg_ms"]},
         "kernels": kern, "compress_kernel_ms": comp_kernel_ms,
         "gpu_launches": launches, "device_status": status, "clocks": clocks,
     }
@@ -260,6 +261,15 @@ def run_ours(args):
         import torch.distributed as dist
         dist.barrier()
         dist.destroy_process_group()
+
+
+def ncu_traffic(wl, retained_rows):
+    """DRAM bytes per decode_attn launch from the committed ncu capture (profiles/decode_attn_llama2_4layers.md):
+    382.09 MB read + written for 739,056 retained rows of 256 bytes, K and V.  Traffic grows in proportion to the
+    rows read, so it is scaled by rows; only the bf16, d = 128, one-query-head-per-KV-head shape was captured."""
+    if wl.dtype != "bf16" or wl.head_dim != 128 or wl.n_heads != wl.n_kv_heads:
+        return None
+    return 382.09e6 / 739056 * retained_rows
 
 
 def run_e2e(tk, wl, params, qs, ks, vs, steps_in, world):

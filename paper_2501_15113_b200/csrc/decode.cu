@@ -164,6 +164,200 @@ __global__ void __launch_bounds__(kAttnThreads) decode_attn_kernel(DeviceProblem
   }
 }
 
+// ---------------------------------------------------------------------------------------------
+// Grouped-query variant for bf16 (G >= 2 query heads per KV head): with several heads per row the
+// scalar kernel above runs out of issue slots long before HBM, so the two contractions go through
+// warp-level mma (m16n8k16, bf16 x bf16 -> fp32) on operands taken straight from 16-byte global
+// loads -- no shared-memory staging; the fragment layouts are met by permuting the contraction
+// index instead:
+//   S^T[head, row] = Q K^T   A = Q (heads on the 16 M rows, rows >= G zero), B = 8 cache rows.  Lane
+//       (g = lane/4, t = lane%4) owns cache row g and loads its 16-byte pieces i*4 + t; the two
+//       halves of piece i are the lane's operand words of k-chunks 2i and 2i+1.  Q is loaded with the
+//       same rule, so both sides agree on which d sits in which k slot.
+//   O^T[d, head] += V^T P^T   the accumulator fragment of S^T (head g, rows 2t, 2t+1) is already the
+//       B fragment of P^T; the A fragment needs pairs of consecutive rows at one d, built with one
+//       byte-permute from the lane's loads of rows 2t, 2t+1, 2t+8, 2t+9 (piece g of each 128-byte
+//       line).  Accumulator row (m-block mb, half hf) of lane g stands for d = pd(mb, hf, g).
+// P is rounded to bf16 for the second product (fp32 accumulation); the normaliser is summed in fp32.
+// Each warp walks 16-row blocks of the work item with its own running (max, sum, O^T); the four
+// warps are merged like the sub-groups of the scalar kernel and the partial goes to the same slots.
+__device__ __forceinline__ void mma_bf16_16816(float (&c)[4], uint32_t a0, uint32_t a1, uint32_t a2, uint32_t a3,
+                                               uint32_t b0, uint32_t b1) {
+  asm volatile(
+      "mma.sync.aligned.m16n8k16.row.col.f32.bf16.bf16.f32 {%0, %1, %2, %3}, {%4, %5, %6, %7}, {%8, %9}, "
+      "{%0, %1, %2, %3};"
+      : "+f"(c[0]), "+f"(c[1]), "+f"(c[2]), "+f"(c[3])
+      : "r"(a0), "r"(a1), "r"(a2), "r"(a3), "r"(b0), "r"(b1));
+}
+__device__ __forceinline__ uint32_t pack_bf16(float lo, float hi) {
+  __nv_bfloat162 v = __floats2bfloat162_rn(lo, hi);
+  return *reinterpret_cast<uint32_t*>(&v);
+}
+__device__ __forceinline__ uint32_t word_of(const uint4& v, int i) {
+  return i == 0 ? v.x : i == 1 ? v.y : i == 2 ? v.z : v.w;
+}
+
+template <int D, int G>
+__global__ void __launch_bounds__(kAttnThreads) decode_attn_mma_kernel(DeviceProblem p,
+                                                                       const __nv_bfloat16* __restrict__ q,
+                                                                       const int32_t* __restrict__ lengths) {
+  constexpr int ROW_BYTES = D * 2;
+  constexpr int KC = D / 16;            // k-chunks of the first product
+  constexpr int KP = D / 32;            // 16-byte pieces of a K row per lane
+  constexpr int MB = D / 16;            // m-blocks (16 d each) of the second product
+  constexpr int VP = D / 64;            // 16-byte pieces of a V row per lane
+  constexpr int kBlk = 16;              // cache rows per warp iteration
+
+  __shared__ float sm_m[kAttnWarps][G];
+  __shared__ float sm_l[kAttnWarps][G];
+  __shared__ __align__(16) float sm_acc[kAttnWarps][G][D];
+  __shared__ int s_unit;
+
+  const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+  const int g = lane >> 2, t = lane & 3;
+  const int total = p.dec_off[p.U];
+  const float scale2 = kLog2e * rsqrtf((float)D);
+  // d of accumulator row (mb, hf) of this lane's two output rows: e = hf * MB + mb, piece e / 8, element e % 8
+  auto pd = [&](int mb, int hf, int gg) { const int e = hf * MB + mb; return (e >> 3) * 64 + gg * 8 + (e & 7); };
+
+  for (int item = blockIdx.x; item < total; item += gridDim.x) {
+    __syncthreads();
+    if (tid == 0) s_unit = upper_unit(p.dec_off, p.U, item);
+    __syncthreads();
+    const int u = s_unit;
+    int len = p.len[u];
+    if (lengths) len = min(max(lengths[u], 0), len);
+    const int rbeg = (item - p.dec_off[u]) * kDecodeChunk;
+    const int rend = min(len, rbeg + kDecodeChunk);
+    const int64_t seg = p.seg_off[u];
+    const unsigned char* kp = static_cast<const unsigned char*>(p.k_pool) + (size_t)seg * ROW_BYTES;
+    const unsigned char* vp = static_cast<const unsigned char*>(p.v_pool) + (size_t)seg * ROW_BYTES;
+
+    // Q fragments: head g on M row g
+    uint32_t qa[KC][2];
+#pragma unroll
+    for (int i = 0; i < KP; ++i) {
+      uint4 raw = make_uint4(0, 0, 0, 0);
+      if (g < G) raw = *reinterpret_cast<const uint4*>(q + ((size_t)u * G + g) * D + (i * 4 + t) * 8);
+      qa[2 * i][0] = raw.x; qa[2 * i][1] = raw.y;
+      qa[2 * i + 1][0] = raw.z; qa[2 * i + 1][1] = raw.w;
+    }
+    float m_run = -INFINITY, l_run = 0.f;   // head g (this lane's share of the sum)
+    float o[MB][4];
+#pragma unroll
+    for (int mb = 0; mb < MB; ++mb)
+#pragma unroll
+      for (int e = 0; e < 4; ++e) o[mb][e] = 0.f;
+
+    for (int blk = rbeg + warp * kBlk; blk < rend; blk += kAttnWarps * kBlk) {   // warp-uniform
+      uint4 kraw[2][KP], vraw[4][VP];
+#pragma unroll
+      for (int j = 0; j < 2; ++j) {
+        const int r = blk + 8 * j + g;
+#pragma unroll
+        for (int i = 0; i < KP; ++i)
+          kraw[j][i] = r < rend ? *reinterpret_cast<const uint4*>(kp + (size_t)r * ROW_BYTES + (i * 4 + t) * 16)
+                                : make_uint4(0, 0, 0, 0);
+      }
+#pragma unroll
+      for (int x = 0; x < 4; ++x) {
+        const int r = blk + 2 * t + (x & 1) + 8 * (x >> 1);
+#pragma unroll
+        for (int i = 0; i < VP; ++i)
+          vraw[x][i] = r < rend ? *reinterpret_cast<const uint4*>(vp + (size_t)r * ROW_BYTES + i * 128 + g * 16)
+                                : make_uint4(0, 0, 0, 0);
+      }
+      // S^T for the two 8-row halves of the block
+      float sc[2][4];
+#pragma unroll
+      for (int j = 0; j < 2; ++j) {
+#pragma unroll
+        for (int e = 0; e < 4; ++e) sc[j][e] = 0.f;
+#pragma unroll
+        for (int i = 0; i < KP; ++i) {
+          mma_bf16_16816(sc[j], qa[2 * i][0], 0u, qa[2 * i][1], 0u, kraw[j][i].x, kraw[j][i].y);
+          mma_bf16_16816(sc[j], qa[2 * i + 1][0], 0u, qa[2 * i + 1][1], 0u, kraw[j][i].z, kraw[j][i].w);
+        }
+      }
+      // online softmax for head g over rows blk + 8j + 2t + {0, 1}
+      float tv[4];
+#pragma unroll
+      for (int j = 0; j < 2; ++j)
+#pragma unroll
+        for (int e = 0; e < 2; ++e) {
+          const int r = blk + 8 * j + 2 * t + e;
+          tv[2 * j + e] = r < rend ? sc[j][e] * scale2 : -INFINITY;
+        }
+      float mx = fmaxf(fmaxf(tv[0], tv[1]), fmaxf(tv[2], tv[3]));
+      mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, 1));
+      mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, 2));
+      const float mn = fmaxf(m_run, mx);
+      const float mu = (mn == -INFINITY) ? 0.f : mn;
+      const float corr = exp2f(m_run - mu);
+      float pw[4];
+#pragma unroll
+      for (int e = 0; e < 4; ++e) pw[e] = exp2f(tv[e] - mu);
+      l_run = l_run * corr + ((pw[0] + pw[1]) + (pw[2] + pw[3]));
+      m_run = mn;
+      // rescale O^T: its columns are heads 2t, 2t+1, whose factors live in lanes 8t and 8t + 4
+      const float ca = __shfl_sync(0xffffffffu, corr, 8 * t);
+      const float cb = __shfl_sync(0xffffffffu, corr, 8 * t + 4);
+      if (__any_sync(0xffffffffu, corr != 1.f)) {
+#pragma unroll
+        for (int mb = 0; mb < MB; ++mb) {
+          o[mb][0] *= ca; o[mb][1] *= cb; o[mb][2] *= ca; o[mb][3] *= cb;
+        }
+      }
+      const uint32_t pb0 = pack_bf16(pw[0], pw[1]);   // rows 2t, 2t+1
+      const uint32_t pb1 = pack_bf16(pw[2], pw[3]);   // rows 2t+8, 2t+9
+#pragma unroll
+      for (int mb = 0; mb < MB; ++mb) {
+        uint32_t a[4];
+#pragma unroll
+        for (int hf = 0; hf < 2; ++hf) {
+          const int e = hf * MB + mb, pc = e >> 3, wi = (e & 7) >> 1;
+          const uint32_t sel = (e & 1) ? 0x7632u : 0x5410u;
+          a[hf] = __byte_perm(word_of(vraw[0][pc], wi), word_of(vraw[1][pc], wi), sel);       // rows 2t, 2t+1
+          a[2 + hf] = __byte_perm(word_of(vraw[2][pc], wi), word_of(vraw[3][pc], wi), sel);   // rows 2t+8, 2t+9
+        }
+        mma_bf16_16816(o[mb], a[0], a[1], a[2], a[3], pb0, pb1);
+      }
+    }
+
+    // merge the four warps (same partial format as the scalar kernel)
+    l_run += __shfl_xor_sync(0xffffffffu, l_run, 1);
+    l_run += __shfl_xor_sync(0xffffffffu, l_run, 2);
+    if (t == 0 && g < G) { sm_m[warp][g] = m_run; sm_l[warp][g] = l_run; }
+#pragma unroll
+    for (int mb = 0; mb < MB; ++mb)
+#pragma unroll
+      for (int e = 0; e < 4; ++e) {
+        const int head = 2 * t + (e & 1);
+        if (head < G) sm_acc[warp][head][pd(mb, e >> 1, g)] = o[mb][e];
+      }
+    __syncthreads();
+    for (int i = tid; i < G * D; i += kAttnThreads) {
+      const int hh = i / D, dd = i % D;
+      float M = -INFINITY;
+#pragma unroll
+      for (int x = 0; x < kAttnWarps; ++x) M = fmaxf(M, sm_m[x][hh]);
+      float a = 0.f, ll = 0.f;
+#pragma unroll
+      for (int x = 0; x < kAttnWarps; ++x) {
+        const float mx = sm_m[x][hh];
+        const float w = (mx == -INFINITY) ? 0.f : exp2f(mx - M);
+        a = fmaf(w, sm_acc[x][hh][dd], a);
+        ll = fmaf(w, sm_l[x][hh], ll);
+      }
+      p.part_acc[((size_t)item * G + hh) * D + dd] = a;
+      if (dd == 0) {
+        p.part_ml[((size_t)item * G + hh) * 2 + 0] = M;
+        p.part_ml[((size_t)item * G + hh) * 2 + 1] = ll;
+      }
+    }
+  }
+}
+
 // One block per (unit, query head of the group): merge the unit's partials.  First the block finds
 // the largest running maximum, then each warp accumulates every fourth partial against it (independent
 // loads, fixed order), and the four warps are summed in shared memory.
@@ -215,7 +409,10 @@ cudaError_t launch_typed(const DeviceProblem& p, const void* q, const int32_t* l
   if (grid < 1) grid = 1;
   {
     LaunchScope ls(K_DECODE_ATTN, s);
-    decode_attn_kernel<T, D, G><<<(unsigned)grid, kAttnThreads, 0, s>>>(p, static_cast<const T*>(q), lengths);
+    if constexpr (G >= 2 && sizeof(T) == 2)
+      decode_attn_mma_kernel<D, G><<<(unsigned)grid, kAttnThreads, 0, s>>>(p, static_cast<const T*>(q), lengths);
+    else
+      decode_attn_kernel<T, D, G><<<(unsigned)grid, kAttnThreads, 0, s>>>(p, static_cast<const T*>(q), lengths);
   }
   {
     LaunchScope ls(K_DECODE_COMBINE, s);
