@@ -409,7 +409,7 @@ cudaError_t launch_typed(const DeviceProblem& p, const void* q, const int32_t* l
   if (grid < 1) grid = 1;
   {
     LaunchScope ls(K_DECODE_ATTN, s);
-    if constexpr (G >= 2 && sizeof(T) == 2)
+    if constexpr (sizeof(T) == 2)
       decode_attn_mma_kernel<D, G><<<(unsigned)grid, kAttnThreads, 0, s>>>(p, static_cast<const T*>(q), lengths);
     else
       decode_attn_kernel<T, D, G><<<(unsigned)grid, kAttnThreads, 0, s>>>(p, static_cast<const T*>(q), lengths);
