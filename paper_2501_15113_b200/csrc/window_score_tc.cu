@@ -220,8 +220,9 @@ inline TcLayout make_layout(int D, int rows) {
   l.tile_bytes = KB * kTile * 128;
   l.q_block_bytes = KB * rows * 128;
   const int stat = kEpiWarps * rows * (int)sizeof(float2);
-  const int trans = kEpiWarps * 32 * 33 * (int)sizeof(float);
-  const int merge = 2 * kEpiWarps * rows * (int)sizeof(float2);
+  // with 128 rows pass 1 puts the window rows on the TMEM lanes and needs no transposition
+  const int trans = rows == 128 ? 0 : kEpiWarps * 32 * 33 * (int)sizeof(float);
+  const int merge = 2 * (rows == 128 ? 2 : kEpiWarps) * rows * (int)sizeof(float2);
   const int bars = 512;
   const int budget = 232448 - 1024;     // dynamic shared memory of one CTA minus the alignment slack
   int stages = (budget - 2 * l.q_block_bytes - stat - trans - merge - bars) / l.tile_bytes;
@@ -363,7 +364,8 @@ window_tc_kernel(const __grid_constant__ CUtensorMap tmap_k, const __grid_consta
             for (int k = 0; k < 4; ++k) {
               const uint64_t ad = smem_desc(kt + (uint32_t)(kb * kTile * 128 + k * 32));
               const uint64_t bd = smem_desc(qbase + (uint32_t)(kb * rows * 128 + k * 32));
-              tc_mma(d_tmem, ad, bd, idesc, (kb | k) ? 1u : 0u);
+              if (it.pass == 1 && rows == 128) tc_mma(d_tmem, bd, ad, idesc, (kb | k) ? 1u : 0u);   // D[row, key]
+              else tc_mma(d_tmem, ad, bd, idesc, (kb | k) ? 1u : 0u);                               // D[key, row]
             }
           tc_commit(BAR(B_EMPTY + stage));   // smem stage free once these MMAs have read it
           tc_commit(BAR(B_TFULL + acc));     // accumulator ready for the epilogue
@@ -380,6 +382,7 @@ window_tc_kernel(const __grid_constant__ CUtensorMap tmap_k, const __grid_consta
     const int grp = ew >> 2;
     const int quad = warp & 3;                      // TMEM lane quadrant this warp may read
     float2* myStat = sStat + ew * rows;
+    const int mparts = rows == 128 ? 2 : kEpiWarps;   // contributors per row in a merge: the two groups, or all warps
     float* myT = sTrans + ew * (32 * 33);
     uint32_t epiphase = 0;
     int n = 0, n_done = 0;
@@ -425,7 +428,7 @@ window_tc_kernel(const __grid_constant__ CUtensorMap tmap_k, const __grid_consta
             }
           }
         }
-        float2* mg = sMerge + (n_done & 1) * (kEpiWarps * rows);
+        float2* mg = sMerge + (n_done & 1) * (mparts * rows);
         mg[part * rows + row] = make_float2(M, z);
         mbar_arrive(BAR(B_EPI));
         ok = __all_sync(0xffffffffu, ok && mbar_wait(BAR(B_EPI), epiphase, s_abort));
@@ -463,7 +466,42 @@ window_tc_kernel(const __grid_constant__ CUtensorMap tmap_k, const __grid_consta
         const uint32_t taddr = tmem_base + ((uint32_t)(quad * 32) << 16) + (uint32_t)acc * 128u;
         const int tbase = key0 + t * kTile;
         const bool tail = (tbase + kTile - 1 > N - L);   // some key of the tile is masked for some row
-        if (it.pass == 1) {
+        if (it.pass == 1 && rows == 128) {
+          // a TMEM lane is a window row (quad * 32 + lane), the 128 columns are the keys of the tile
+          const int pos = N - L + ((quad * 32 + lane) % L);   // last key this window row may see
+#pragma unroll
+          for (int cg = 0; cg < 4; ++cg) {
+            uint32_t r[32];
+            tc_ld32(taddr + (uint32_t)(cg * 32), r);
+            tc_wait_ld();
+            float x[32];
+            if (!tail) {
+#pragma unroll
+              for (int k = 0; k < 32; ++k) x[k] = __uint_as_float(r[k]);
+            } else {
+#pragma unroll
+              for (int k = 0; k < 32; ++k) {
+                const int j = tbase + cg * 32 + k;
+                x[k] = (j <= pos && j < N) ? __uint_as_float(r[k]) : -INFINITY;
+              }
+            }
+            float cm4[4] = {-INFINITY, -INFINITY, -INFINITY, -INFINITY};
+#pragma unroll
+            for (int k = 0; k < 32; ++k) cm4[k & 3] = fmaxf(cm4[k & 3], x[k]);
+            const float cm = fmaxf(fmaxf(cm4[0], cm4[1]), fmaxf(cm4[2], cm4[3]));
+            if (cm > m_run[0]) {
+              z_run[0] *= ex2((m_run[0] - cm) * scale2);
+              m_run[0] = cm;
+            }
+            if (m_run[0] > -INFINITY) {
+              const float ms = -m_run[0] * scale2;
+              float zs[4] = {0.f, 0.f, 0.f, 0.f};
+#pragma unroll
+              for (int k = 0; k < 32; ++k) zs[k & 3] += ex2(fmaf(x[k], scale2, ms));
+              z_run[0] += (zs[0] + zs[1]) + (zs[2] + zs[3]);
+            }
+          }
+        } else if (it.pass == 1) {
           const int jw = tbase + quad * 32;              // first key of this warp's 32 lanes
 #pragma unroll
           for (int rg = 0; rg < 4; ++rg) {
@@ -476,36 +514,39 @@ window_tc_kernel(const __grid_constant__ CUtensorMap tmap_k, const __grid_consta
               for (int c = 0; c < 32; ++c) myT[lane * 33 + c] = __uint_as_float(r[c]);
               __syncwarp();
               float x[32];
-              float cm = -INFINITY;
               if (!tail) {
 #pragma unroll
-                for (int k = 0; k < 32; ++k) { x[k] = myT[k * 33 + lane]; cm = fmaxf(cm, x[k]); }
+                for (int k = 0; k < 32; ++k) x[k] = myT[k * 33 + lane];
               } else {
                 const int pos = N - L + ((rg * 32 + lane) % L);   // last key this window row may see
 #pragma unroll
                 for (int k = 0; k < 32; ++k) {
                   const int j = jw + k;
                   x[k] = (j <= pos && j < N) ? myT[k * 33 + lane] : -INFINITY;
-                  cm = fmaxf(cm, x[k]);
                 }
               }
               __syncwarp();
+              // four interleaved chains: a single running max / sum would serialise on the ALU latency
+              float cm4[4] = {-INFINITY, -INFINITY, -INFINITY, -INFINITY};
+#pragma unroll
+              for (int k = 0; k < 32; ++k) cm4[k & 3] = fmaxf(cm4[k & 3], x[k]);
+              const float cm = fmaxf(fmaxf(cm4[0], cm4[1]), fmaxf(cm4[2], cm4[3]));
               if (cm > m_run[rg]) {
                 z_run[rg] *= ex2((m_run[rg] - cm) * scale2);
                 m_run[rg] = cm;
               }
               if (m_run[rg] > -INFINITY) {
                 const float ms = -m_run[rg] * scale2;
-                float zs = 0.f;
+                float zs[4] = {0.f, 0.f, 0.f, 0.f};
 #pragma unroll
-                for (int k = 0; k < 32; ++k) zs += ex2(fmaf(x[k], scale2, ms));
-                z_run[rg] += zs;
+                for (int k = 0; k < 32; ++k) zs[k & 3] += ex2(fmaf(x[k], scale2, ms));
+                z_run[rg] += (zs[0] + zs[1]) + (zs[2] + zs[3]);
               }
             }
           }
         } else {
           const int j = tbase + quad * 32 + lane;   // this thread's key
-          float csum = 0.f;
+          float cs[4] = {0.f, 0.f, 0.f, 0.f};   // four interleaved chains (FMA latency)
           for (int c0 = 0; c0 < rows; c0 += 32) {
             uint32_t r[32];
             tc_ld32(taddr + (uint32_t)c0, r);
@@ -514,17 +555,18 @@ window_tc_kernel(const __grid_constant__ CUtensorMap tmap_k, const __grid_consta
 #pragma unroll
               for (int c = 0; c < 32; ++c) {
                 const float2 ms = myStat[c0 + c];
-                csum = fmaf(ex2(fmaf(__uint_as_float(r[c]), scale2, -ms.x)), ms.y, csum);
+                cs[c & 3] = fmaf(ex2(fmaf(__uint_as_float(r[c]), scale2, -ms.x)), ms.y, cs[c & 3]);
               }
             } else {
 #pragma unroll
               for (int c = 0; c < 32; ++c) {
                 const float2 ms = myStat[c0 + c];
                 const bool vis = (j < N) && (j <= N - L + ((c0 + c) % L));
-                if (vis) csum = fmaf(ex2(fmaf(__uint_as_float(r[c]), scale2, -ms.x)), ms.y, csum);
+                if (vis) cs[c & 3] = fmaf(ex2(fmaf(__uint_as_float(r[c]), scale2, -ms.x)), ms.y, cs[c & 3]);
               }
             }
           }
+          const float csum = (cs[0] + cs[1]) + (cs[2] + cs[3]);
           if (j < N) p.C[p.c_off[u] + j] = csum * (1.0f / (float)rows);
         }
         tc_fence_before();
@@ -534,10 +576,15 @@ window_tc_kernel(const __grid_constant__ CUtensorMap tmap_k, const __grid_consta
       if (!ok) break;
       if (it.pass == 1) {
         // merge the eight warps' (max, sum) per row in a fixed order; one slot per work item
-        float2* mg = sMerge + (n_done & 1) * (kEpiWarps * rows);
+        const int nparts = mparts;
+        float2* mg = sMerge + (n_done & 1) * (nparts * rows);
+        if (rows == 128) {
+          mg[grp * rows + quad * 32 + lane] = make_float2(m_run[0] * scale2, z_run[0]);
+        } else {
 #pragma unroll
-        for (int rg = 0; rg < 4; ++rg)
-          if (rg * 32 < rows) mg[ew * rows + rg * 32 + lane] = make_float2(m_run[rg] * scale2, z_run[rg]);
+          for (int rg = 0; rg < 4; ++rg)
+            if (rg * 32 < rows) mg[ew * rows + rg * 32 + lane] = make_float2(m_run[rg] * scale2, z_run[rg]);
+        }
         mbar_arrive(BAR(B_EPI));
         ok = __all_sync(0xffffffffu, mbar_wait(BAR(B_EPI), epiphase, s_abort));
         epiphase ^= 1;
@@ -545,11 +592,9 @@ window_tc_kernel(const __grid_constant__ CUtensorMap tmap_k, const __grid_consta
         const int tl = ew * 32 + lane;
         if (tl < rows) {
           float M = -INFINITY;
-#pragma unroll
-          for (int w = 0; w < kEpiWarps; ++w) M = fmaxf(M, mg[w * rows + tl].x);
+          for (int w = 0; w < nparts; ++w) M = fmaxf(M, mg[w * rows + tl].x);
           float z = 0.f;
-#pragma unroll
-          for (int w = 0; w < kEpiWarps; ++w) {
+          for (int w = 0; w < nparts; ++w) {
             const float2 o = mg[w * rows + tl];
             if (o.x > -INFINITY) z = fmaf(o.y, ex2(o.x - M), z);
           }
