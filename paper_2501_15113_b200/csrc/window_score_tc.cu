@@ -249,7 +249,9 @@ window_tc_kernel(const __grid_constant__ CUtensorMap tmap_k, const __grid_consta
   constexpr int KB = D / 64;
   extern __shared__ unsigned char smem_raw[];
   // 1024-byte alignment: the swizzle pattern is a function of the address bits
-  unsigned char* smem = reinterpret_cast<unsigned char*>(((uintptr_t)smem_raw + 1023) & ~(uintptr_t)1023);
+  // (offset added to the array itself: a round trip through an integer would turn every access below into a
+  // generic-address load or store)
+  unsigned char* smem = smem_raw + ((1024u - (smem_u32(smem_raw) & 1023u)) & 1023u);
   unsigned char* sK = smem;                                         // [stages][KB][128 keys][128 B]
   unsigned char* sQ = smem + lay.off_q;                             // [2][KB][rows][128 B]
   float2* sStat = reinterpret_cast<float2*>(smem + lay.off_stat);   // [8 warps][rows]
@@ -552,10 +554,12 @@ window_tc_kernel(const __grid_constant__ CUtensorMap tmap_k, const __grid_consta
             tc_ld32(taddr + (uint32_t)c0, r);
             tc_wait_ld();
             if (!tail) {
+              const float4* st4 = reinterpret_cast<const float4*>(myStat + c0);   // two rows per 16-byte load
 #pragma unroll
-              for (int c = 0; c < 32; ++c) {
-                const float2 ms = myStat[c0 + c];
+              for (int c = 0; c < 32; c += 2) {
+                const float4 ms = st4[c >> 1];
                 cs[c & 3] = fmaf(ex2(fmaf(__uint_as_float(r[c]), scale2, -ms.x)), ms.y, cs[c & 3]);
+                cs[(c + 1) & 3] = fmaf(ex2(fmaf(__uint_as_float(r[c + 1]), scale2, -ms.z)), ms.w, cs[(c + 1) & 3]);
               }
             } else {
 #pragma unroll
