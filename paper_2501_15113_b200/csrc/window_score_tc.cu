@@ -116,6 +116,18 @@ __device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatil
     if (spin > 32) __nanosleep(128);
   }
 }
+// One lane of a converged warp.  The role loops below are run by all 32 lanes and only the TMA / MMA /
+// commit instructions sit under this predicate: address and descriptor arithmetic then stays warp-uniform
+// (uniform registers), which a loop inside `if (lane == 0)` does not allow.
+__device__ __forceinline__ bool elect_one() {
+  uint32_t pred;
+  asm volatile(
+      "{\n\t.reg .pred p;\n\t"
+      "elect.sync _|p, 0xffffffff;\n\t"
+      "selp.u32 %0, 1, 0, p;\n\t}"
+      : "=r"(pred));
+  return pred != 0;
+}
 __device__ __forceinline__ void tma_load_2d(uint32_t dst, const CUtensorMap* map, int x, int y, uint32_t bar) {
   asm volatile(
       "cp.async.bulk.tensor.2d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3}], [%4];"
@@ -293,8 +305,8 @@ window_tc_kernel(const __grid_constant__ CUtensorMap tmap_k, const __grid_consta
   const float scale2 = kLog2e * rsqrtf((float)D);
 
   if (warp == 0) {
-    // ------------------------------------------------------------ TMA producer
-    if (lane == 0) {
+    // ------------------------------------------------------------ TMA producer (whole warp, one lane issues)
+    {
       int stage = 0, qb = 0;
       uint32_t phase = 0, qphase[2] = {0, 0};
       bool ok = true;
@@ -303,38 +315,46 @@ window_tc_kernel(const __grid_constant__ CUtensorMap tmap_k, const __grid_consta
         if (!it.valid) continue;
         const int key0 = it.ch * a.chunk_keys;
         const int ntiles = (min(N, key0 + a.chunk_keys) - key0 + kTile - 1) / kTile;
-        ok = mbar_wait(BAR(B_QEMPTY + qb), qphase[qb] ^ 1, s_abort);
+        ok = __all_sync(0xffffffffu, mbar_wait(BAR(B_QEMPTY + qb), qphase[qb] ^ 1, s_abort));
         if (!ok) break;
-        mbar_expect_tx(BAR(B_QFULL + qb), (uint32_t)lay.q_block_bytes);
-        for (int kb = 0; kb < KB; ++kb)
-          tma_load_2d(smem_u32(sQ + (size_t)qb * lay.q_block_bytes + (size_t)kb * rows * 128), &tmap_q, kb * 64,
-                      it.lu * rows, BAR(B_QFULL + qb));
+        if (elect_one()) {
+          mbar_expect_tx(BAR(B_QFULL + qb), (uint32_t)lay.q_block_bytes);
+          for (int kb = 0; kb < KB; ++kb)
+            tma_load_2d(smem_u32(sQ + (size_t)qb * lay.q_block_bytes + (size_t)kb * rows * 128), &tmap_q, kb * 64,
+                        it.lu * rows, BAR(B_QFULL + qb));
+        }
+        __syncwarp();
         qphase[qb] ^= 1;
         qb ^= 1;
         for (int t = 0; t < ntiles; ++t) {
-          ok = mbar_wait(BAR(B_EMPTY + stage), phase ^ 1, s_abort);
+          ok = __all_sync(0xffffffffu, mbar_wait(BAR(B_EMPTY + stage), phase ^ 1, s_abort));
           if (!ok) break;
-          mbar_expect_tx(BAR(B_FULL + stage), (uint32_t)lay.tile_bytes);
-          for (int kb = 0; kb < KB; ++kb)
-            tma_load_2d(smem_u32(sK + (size_t)stage * lay.tile_bytes + (size_t)kb * kTile * 128), &tmap_k,
-                        kb * 64, it.lu * N + key0 + t * kTile, BAR(B_FULL + stage));
+          if (elect_one()) {
+            mbar_expect_tx(BAR(B_FULL + stage), (uint32_t)lay.tile_bytes);
+#pragma unroll
+            for (int kb = 0; kb < KB; ++kb)
+              tma_load_2d(smem_u32(sK + (size_t)stage * lay.tile_bytes + (size_t)kb * kTile * 128), &tmap_k,
+                          kb * 64, it.lu * N + key0 + t * kTile, BAR(B_FULL + stage));
+          }
+          __syncwarp();
           if (++stage == S) { stage = 0; phase ^= 1; }
         }
       }
       // Drain: every tcgen05.commit aimed at this CTA's barriers must have arrived before the CTA exits,
       // or it would land on the barriers of the next CTA that is given this shared memory.
       for (int i = 0; i < S && ok; ++i) {
-        ok = mbar_wait(BAR(B_EMPTY + stage), phase ^ 1, s_abort);
+        ok = __all_sync(0xffffffffu, mbar_wait(BAR(B_EMPTY + stage), phase ^ 1, s_abort));
         if (++stage == S) { stage = 0; phase ^= 1; }
       }
-      for (int i = 0; i < 2 && ok; ++i, qb ^= 1) ok = mbar_wait(BAR(B_QEMPTY + qb), qphase[qb] ^ 1, s_abort);
+      for (int i = 0; i < 2 && ok; ++i, qb ^= 1)
+        ok = __all_sync(0xffffffffu, mbar_wait(BAR(B_QEMPTY + qb), qphase[qb] ^ 1, s_abort));
     }
   } else if (warp == 1 || warp == 6) {
     // ------------------------------------------------------------ MMA issuers: D[key, row] = K Q^T, both passes.
     // Two elected threads: the issue -> commit -> hand-over chain of one tile overlaps with the other's.
     // Tiles are numbered n = 0, 1, ... per CTA across items: issuer n & 1, smem stage n % stages, TMEM
     // accumulator n & 3 (read by epilogue group n & 1).
-    if (lane == 0) {
+    {
       const int me = warp == 1 ? 0 : 1;
       int qb = 0, n = 0;
       uint32_t qphase[2] = {0, 0};
@@ -345,35 +365,40 @@ window_tc_kernel(const __grid_constant__ CUtensorMap tmap_k, const __grid_consta
         if (!it.valid) continue;
         const int key0 = it.ch * a.chunk_keys;
         const int ntiles = (min(N, key0 + a.chunk_keys) - key0 + kTile - 1) / kTile;
-        ok = mbar_wait(BAR(B_QFULL + qb), qphase[qb], s_abort);
+        ok = __all_sync(0xffffffffu, mbar_wait(BAR(B_QFULL + qb), qphase[qb], s_abort));
         if (!ok) break;
         qphase[qb] ^= 1;
         const uint32_t qbase = smem_u32(sQ + (size_t)qb * lay.q_block_bytes);
+        const bool swap = it.pass == 1 && rows == 128;   // D[row, key] instead of D[key, row]
         for (int t = 0; t < ntiles; ++t, ++n) {
           if ((n & 1) != me) continue;
           const int stage = n % S, acc = n & 3;
           const uint32_t phase = (uint32_t)((n / S) & 1), accphase = (uint32_t)((n >> 2) & 1);
-          ok = mbar_wait(BAR(B_FULL + stage), phase, s_abort);
+          ok = __all_sync(0xffffffffu, mbar_wait(BAR(B_FULL + stage), phase, s_abort));
           if (!ok) break;
-          ok = mbar_wait(BAR(B_TEMPTY + acc), accphase ^ 1, s_abort);
+          ok = __all_sync(0xffffffffu, mbar_wait(BAR(B_TEMPTY + acc), accphase ^ 1, s_abort));
           if (!ok) break;
           tc_fence_after();
           const uint32_t d_tmem = tmem_base + (uint32_t)acc * 128u;
           const uint32_t kt = smem_u32(sK + (size_t)stage * lay.tile_bytes);
+          if (elect_one()) {
 #pragma unroll
-          for (int kb = 0; kb < KB; ++kb)
+            for (int kb = 0; kb < KB; ++kb)
 #pragma unroll
-            for (int k = 0; k < 4; ++k) {
-              const uint64_t ad = smem_desc(kt + (uint32_t)(kb * kTile * 128 + k * 32));
-              const uint64_t bd = smem_desc(qbase + (uint32_t)(kb * rows * 128 + k * 32));
-              if (it.pass == 1 && rows == 128) tc_mma(d_tmem, bd, ad, idesc, (kb | k) ? 1u : 0u);   // D[row, key]
-              else tc_mma(d_tmem, ad, bd, idesc, (kb | k) ? 1u : 0u);                               // D[key, row]
-            }
-          tc_commit(BAR(B_EMPTY + stage));   // smem stage free once these MMAs have read it
-          tc_commit(BAR(B_TFULL + acc));     // accumulator ready for the epilogue
+              for (int k = 0; k < 4; ++k) {
+                const uint64_t ad = smem_desc(kt + (uint32_t)(kb * kTile * 128 + k * 32));
+                const uint64_t bd = smem_desc(qbase + (uint32_t)(kb * rows * 128 + k * 32));
+                if (swap) tc_mma(d_tmem, bd, ad, idesc, (kb | k) ? 1u : 0u);
+                else tc_mma(d_tmem, ad, bd, idesc, (kb | k) ? 1u : 0u);
+              }
+            tc_commit(BAR(B_EMPTY + stage));   // smem stage free once these MMAs have read it
+            tc_commit(BAR(B_TFULL + acc));     // accumulator ready for the epilogue
+          }
+          __syncwarp();
         }
         if (!ok) break;
-        tc_commit(BAR(B_QEMPTY + qb));       // this issuer is done with the Q block
+        if (elect_one()) tc_commit(BAR(B_QEMPTY + qb));   // this issuer is done with the Q block
+        __syncwarp();
         qb ^= 1;
       }
     }
