@@ -113,6 +113,10 @@ CASES = [
     dict(n=16, n_kv=4, d=128, N=2100, L=32, s1=4, s2=64, k=50, dtype="bf16"),
     dict(n=16, n_kv=2, d=64, N=900, L=16, s1=4, s2=64, k=50, dtype="f32", nh=0),
     dict(n=4, n_kv=1, d=128, N=700, L=32, s1=4, s2=64, k=50, dtype="bf16", nh=0),
+    # bf16 decode through warp mma: G = 8 and G = 2 at both head dims; segment lengths that end inside a 16-row block
+    dict(n=16, n_kv=2, d=64, N=1303, L=16, s1=4, s2=64, k=51, dtype="bf16", nh=0),   # G = 8, d = 64, 128 window rows
+    dict(n=8, n_kv=1, d=128, N=811, L=16, s1=4, s2=64, k=37, dtype="bf16", nh=0),    # G = 8, d = 128
+    dict(n=8, n_kv=4, d=64, N=1000, L=16, s1=3, s2=30, k=45, dtype="bf16"),          # G = 2, d = 64
     # degenerate budgets and windows
     dict(n=4, n_kv=4, d=64, N=90, L=8, s1=40, s2=60, k=10, dtype="f32"),          # N <= sink + recent
     dict(n=4, n_kv=4, d=64, N=600, L=8, s1=4, s2=32, k=0, dtype="f32"),           # no middle activations
