@@ -354,11 +354,16 @@ window_tc_kernel(const __grid_constant__ CUtensorMap tmap_k, const __grid_consta
     // Two elected threads: the issue -> commit -> hand-over chain of one tile overlaps with the other's.
     // Tiles are numbered n = 0, 1, ... per CTA across items: issuer n & 1, smem stage n % stages, TMEM
     // accumulator n & 3 (read by epilogue group n & 1).
+    // The per-tile bookkeeping is kept to counters that step by two (this issuer's tiles), and the
+    // descriptors to one add on a precomputed low word: a lone warp issues an instruction only every few cycles.
     {
       const int me = warp == 1 ? 0 : 1;
-      int qb = 0, n = 0;
+      int qb = 0, tiles_before = 0;
+      int stage = me, acc = me;                 // S is even: own stages me, me + 2, ...; accumulators me, me + 2
+      uint32_t sphase = 0, aphase = 0;
       uint32_t qphase[2] = {0, 0};
       const uint32_t idesc = instr_desc(128, rows);
+      const uint64_t desc_hi = smem_desc(0);    // everything but the start address
       bool ok = true;
       for (int k = 0; k < a.steps && ok; ++k) {
         const Item it = decode_item(a, k);
@@ -368,26 +373,22 @@ window_tc_kernel(const __grid_constant__ CUtensorMap tmap_k, const __grid_consta
         ok = __all_sync(0xffffffffu, mbar_wait(BAR(B_QFULL + qb), qphase[qb], s_abort));
         if (!ok) break;
         qphase[qb] ^= 1;
-        const uint32_t qbase = smem_u32(sQ + (size_t)qb * lay.q_block_bytes);
+        const uint32_t q_lo = smem_u32(sQ + (size_t)qb * lay.q_block_bytes) >> 4;
         const bool swap = it.pass == 1 && rows == 128;   // D[row, key] instead of D[key, row]
-        for (int t = 0; t < ntiles; ++t, ++n) {
-          if ((n & 1) != me) continue;
-          const int stage = n % S, acc = n & 3;
-          const uint32_t phase = (uint32_t)((n / S) & 1), accphase = (uint32_t)((n >> 2) & 1);
-          ok = __all_sync(0xffffffffu, mbar_wait(BAR(B_FULL + stage), phase, s_abort));
-          if (!ok) break;
-          ok = __all_sync(0xffffffffu, mbar_wait(BAR(B_TEMPTY + acc), accphase ^ 1, s_abort));
+        for (int t = (me ^ tiles_before) & 1; t < ntiles; t += 2) {
+          ok = __all_sync(0xffffffffu, mbar_wait(BAR(B_FULL + stage), sphase, s_abort) &&
+                                           mbar_wait(BAR(B_TEMPTY + acc), aphase ^ 1, s_abort));
           if (!ok) break;
           tc_fence_after();
           const uint32_t d_tmem = tmem_base + (uint32_t)acc * 128u;
-          const uint32_t kt = smem_u32(sK + (size_t)stage * lay.tile_bytes);
+          const uint32_t k_lo = smem_u32(sK + (size_t)stage * lay.tile_bytes) >> 4;
           if (elect_one()) {
 #pragma unroll
             for (int kb = 0; kb < KB; ++kb)
 #pragma unroll
               for (int k = 0; k < 4; ++k) {
-                const uint64_t ad = smem_desc(kt + (uint32_t)(kb * kTile * 128 + k * 32));
-                const uint64_t bd = smem_desc(qbase + (uint32_t)(kb * rows * 128 + k * 32));
+                const uint64_t ad = desc_hi | (uint64_t)(k_lo + (uint32_t)((kb * kTile * 128 + k * 32) >> 4));
+                const uint64_t bd = desc_hi | (uint64_t)(q_lo + (uint32_t)((kb * rows * 128 + k * 32) >> 4));
                 if (swap) tc_mma(d_tmem, bd, ad, idesc, (kb | k) ? 1u : 0u);
                 else tc_mma(d_tmem, ad, bd, idesc, (kb | k) ? 1u : 0u);
               }
@@ -395,8 +396,13 @@ window_tc_kernel(const __grid_constant__ CUtensorMap tmap_k, const __grid_consta
             tc_commit(BAR(B_TFULL + acc));     // accumulator ready for the epilogue
           }
           __syncwarp();
+          stage += 2;
+          if (stage >= S) { stage -= S; sphase ^= 1; }
+          acc ^= 2;
+          if (acc == me) aphase ^= 1;
         }
         if (!ok) break;
+        tiles_before += ntiles;
         if (elect_one()) tc_commit(BAR(B_QEMPTY + qb));   // this issuer is done with the Q block
         __syncwarp();
         qb ^= 1;
