@@ -110,7 +110,13 @@ taskkv_status make_plan(const taskkv_params* p, HostPlan& hp) {
   hp.c_total = c_total;
   hp.rows = G * p->window;
   hp.rows_pad = (hp.rows + 15) / 16 * 16;
-  hp.chunks_max = (hp.max_N + kTcChunk - 1) / kTcChunk;   // partial-statistic slots per unit (kTcChunk == kScoreChunk)
+  // partial-statistic slots per unit: one per 1024-key chunk on the CUDA-core path, one per epilogue warp and
+  // work item on the tensor-core path
+  {
+    const int generic = (hp.max_N + kScoreChunk - 1) / kScoreChunk;
+    const int tc = (hp.max_N + kTcChunk - 1) / kTcChunk * kTcParts;
+    hp.chunks_max = generic > tc ? generic : tc;
+  }
 
   const size_t es = p->dtype == TASKKV_F32 ? 4 : 2;
   const size_t d = p->head_dim;

@@ -13,7 +13,8 @@ namespace taskkv {
 constexpr int kDecodeChunk = 512;                 // rows of one split-K decode item
 constexpr int kGatherRows = 64;                   // rows of one gather item
 constexpr int kScoreChunk = 1024;                 // keys of one window-score work item (CUDA-core path)
-constexpr int kTcChunk = 1024;                    // keys of one window-score work item (tensor-core path)
+constexpr int kTcChunk = 2048;                    // fewest keys of one window-score work item (tensor-core path)
+constexpr int kTcParts = 8;                       // partial-statistic slots per work item (one per epilogue warp)
 constexpr float kLog2e = 1.4426950408889634f;
 
 // kernel ids for launch counting / timing
@@ -46,7 +47,7 @@ struct DeviceProblem {
   int32_t promote_center, force_class;
   int32_t max_new;
   int32_t idx_stride;   // ints per unit in idx
-  int32_t chunks_max;   // score chunks of the longest sequence
+  int32_t chunks_max;   // partial-statistic slots per unit (longest sequence)
   int64_t pool_rows;
   int64_t max_items;    // decode work items the scratch can hold
   // per unit tables

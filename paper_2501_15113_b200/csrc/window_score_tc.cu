@@ -4,22 +4,23 @@
 // The contraction S = Q_win K^T is 2*G*L*d flop per key (32-128 flop per byte of
 // K): too much for the CUDA cores next to an HBM-rate K stream, little for
 // tcgen05.  Each CTA is a persistent, warp-specialised pipeline:
-//   warp 0   TMA producer: K tiles of 128 keys (and the unit's Q rows) into
-//            128-byte-swizzled shared memory, completion on mbarriers
-//   warp 1   tcgen05.mma issuer (one elected thread), accumulators in TMEM,
-//            double buffered; tcgen05.commit frees the smem stage and hands the
-//            accumulator to the epilogue
-//   warps 2-5  epilogue: tcgen05.ld, softmax arithmetic in fp32 registers
-// Two passes, as Eq. 13 needs every row's normaliser before rows can be summed:
-//   pass 1 (row statistics)  D[row, key] = Q K^T: a TMEM lane is a window row, so
-//     the running max / exp-sum over keys stays inside one thread.  With fewer
-//     than 128 rows the Q block is replicated over the lane quadrants, each
-//     against its own sub-tile of keys, so all four epilogue warps share the work.
+//   warp 0        TMA producer: K tiles of 128 keys (and the unit's Q rows) into
+//                 128-byte-swizzled shared memory, completion on mbarriers
+//   warps 1, 6    tcgen05.mma issuers, alternating tiles; accumulators in TMEM (four of
+//                 them); tcgen05.commit frees the smem stage and hands the accumulator over
+//   warps 2-5, 7-10  two epilogue groups, alternating tiles: tcgen05.ld, softmax arithmetic
+//                 in fp32 registers
+// Two passes (two launches), as Eq. 13 needs every row's normaliser before rows can be summed:
+//   pass 1 (row statistics)  every epilogue warp keeps a running (max, exp-sum) per window row
+//     over the keys it sees in a work item and stores it as the warp's own partial; a small
+//     kernel folds the partials of a unit.  With up to 64 rows D[key, row] = K Q^T is used (a
+//     TMEM lane is a key) and the warp's 32x32 block is transposed through shared memory;
+//     with 128 rows the operands are swapped, D[row, key], and a lane owns a row outright.
 //   pass 2 (scores)  D[key, row] = K Q^T: a TMEM lane is a key, so
 //     C[key] = sum_rows exp2(s - max_row) / Z_row is a sum inside one thread.
-// Scores are kept in log2 units (scale log2(e)/sqrt(d)); exp is one ex2.approx.
-// Every wait is bounded: on time-out the CTA records TASKKV_ETIMEOUT, stops
-// issuing work, releases its TMEM and returns.
+// No warp ever waits for another epilogue warp.  Scores are kept in log2 units (scale
+// log2(e)/sqrt(d)); exp is one ex2.approx.  Every wait is bounded: on time-out the CTA records
+// TASKKV_ETIMEOUT, stops issuing work, releases its TMEM and returns.
 #include <cuda.h>
 
 #include "common.cuh"
@@ -31,50 +32,31 @@ namespace {
 constexpr int kTile = 128;          // keys per tile (UMMA M in pass 2, key sub-tiles in pass 1)
 constexpr int kMaxStages = 6;       // K tiles in flight per CTA (the count is fitted to shared memory)
 constexpr int kEpiWarps = 8;        // two groups of four epilogue warps, alternating tiles
+static_assert(kEpiWarps == kTcParts, "one partial-statistic slot per epilogue warp");
 constexpr int kThreads = 352;       // warp 0 producer; 1, 6 MMA issuers; 2-5 and 7-10 epilogue groups
 constexpr uint32_t kTmemCols = 512; // four accumulators of up to 128 columns
 constexpr uint32_t kSpinLimit = 1u << 22;
 
-// Work items of one launch (one sequence): (pass, unit, chunk of chunk_keys keys), numbered unit-major
-// i = unit * C + chunk.  CTA c of a grid of g CTAs owns the items i = c, c + g, c + 2g, ... of BOTH passes.
-// mode 1 / 2: one pass per launch (the statistics are combined by a small kernel in between).
-// mode 0: both passes in one launch, so that the second read of a chunk of keys comes from L2: in round r
-//   the CTA runs pass 1 on item c + r*g and then pass 2 on item c + (r - lag)*g -- the same SM that pulled
-//   the chunk into its side of the L2 a few rounds earlier.  Pass 2 of an item needs the statistics of
-//   its whole unit, i.e. the C per-item partials written by (mostly) other CTAs during rounds <= r - lag + 1;
-//   the epilogue combines them itself at the start of the item.  Every partial is one 8-byte word that
-//   is NaN until written, so no fence or counter is involved; a missing one is polled for (bounded).
-//   A step only ever depends on pass-1 items of earlier rounds, which resident CTAs that take their
-//   items in order have already started, so the wait always ends.
+// Work items of one launch (one sequence and one pass): (unit, chunk of chunk_keys keys), numbered
+// unit-major i = unit * chunks + chunk.  CTA c of a grid of g CTAs takes the items c, c + g, c + 2g, ...
 struct TcArgs {
-  int mode;
+  int pass;          // 1 = row statistics, 2 = scores
   int u0;            // first unit of this sequence
   int n_local;       // units in this launch (layers * kv heads)
   int N;             // sequence length
-  int chunks;        // C: work items per unit and pass
+  int chunks;        // work items per unit
   int chunk_keys;    // keys per work item (multiple of 128)
-  int lag;           // mode 0: rounds between the two passes of an item
-  int steps;         // steps of every CTA
+  int steps;         // items of the busiest CTA
 };
 
 struct Item {
-  int pass, lu, ch;
-  bool valid;        // has tiles to process
+  int lu, ch;
+  bool valid;
 };
 __device__ __forceinline__ Item decode_item(const TcArgs& a, int k) {
   Item it;
-  int i;
-  if (a.mode != 0) {
-    it.pass = a.mode;
-    i = (int)blockIdx.x + k * (int)gridDim.x;
-    it.valid = true;
-  } else {
-    const int r = k >> 1;
-    it.pass = (k & 1) ? 2 : 1;
-    i = (int)blockIdx.x + ((k & 1) ? r - a.lag : r) * (int)gridDim.x;
-    it.valid = i >= 0;
-  }
-  it.valid = it.valid && i < a.n_local * a.chunks;
+  const int i = (int)blockIdx.x + k * (int)gridDim.x;
+  it.valid = i < a.n_local * a.chunks;
   it.lu = it.valid ? i / a.chunks : 0;
   it.ch = it.valid ? i % a.chunks : 0;
   return it;
@@ -177,30 +159,6 @@ __device__ __forceinline__ float ex2(float x) {
   return y;
 }
 
-// (a, b) pairs that double as their own "written" flag: the buffers are filled with 0xFF bytes (NaN)
-// before the launch, a pair is published with one 8-byte store and read with one 8-byte load.
-__device__ __forceinline__ void publish_pair(float2* addr, float x, float y) {
-  const uint64_t v = (uint64_t)__float_as_uint(x) | ((uint64_t)__float_as_uint(y) << 32);
-  asm volatile("st.relaxed.gpu.global.b64 [%0], %1;" ::"l"(addr), "l"(v) : "memory");
-}
-__device__ __forceinline__ bool poll_pair(const float2* addr, float2& out, volatile int* abort_flag) {
-  for (uint32_t spin = 0;; ++spin) {
-    uint64_t v;
-    asm volatile("ld.relaxed.gpu.global.b64 %0, [%1];" : "=l"(v) : "l"(addr) : "memory");
-    const float y = __uint_as_float((uint32_t)(v >> 32));
-    if (y == y) {
-      out = make_float2(__uint_as_float((uint32_t)v), y);
-      return true;
-    }
-    if (*abort_flag) return false;
-    if (spin > kSpinLimit) {
-      *abort_flag = 1;
-      return false;
-    }
-    __nanosleep(200);
-  }
-}
-
 // Shared-memory matrix descriptor: K-major operand, rows of 128 bytes, 128-byte
 // swizzle, 8-row groups 1024 bytes apart.
 __device__ __forceinline__ uint64_t smem_desc(uint32_t saddr) {
@@ -222,7 +180,7 @@ __device__ __forceinline__ uint32_t instr_desc(int M, int N) {
 struct TcLayout {
   int stages;
   int tile_bytes, q_block_bytes;
-  int off_q, off_stat, off_trans, off_merge, off_bars;
+  int off_q, off_stat, off_trans, off_bars;
   int total;
 };
 
@@ -234,24 +192,22 @@ inline TcLayout make_layout(int D, int rows) {
   const int stat = kEpiWarps * rows * (int)sizeof(float2);
   // with 128 rows pass 1 puts the window rows on the TMEM lanes and needs no transposition
   const int trans = rows == 128 ? 0 : kEpiWarps * 32 * 33 * (int)sizeof(float);
-  const int merge = 2 * (rows == 128 ? 2 : kEpiWarps) * rows * (int)sizeof(float2);
   const int bars = 512;
   const int budget = 232448 - 1024;     // dynamic shared memory of one CTA minus the alignment slack
-  int stages = (budget - 2 * l.q_block_bytes - stat - trans - merge - bars) / l.tile_bytes;
+  int stages = (budget - 2 * l.q_block_bytes - stat - trans - bars) / l.tile_bytes;
   if (stages > kMaxStages) stages = kMaxStages;
   l.stages = stages & ~1;
   l.off_q = l.stages * l.tile_bytes;
   l.off_stat = l.off_q + 2 * l.q_block_bytes;
   l.off_trans = l.off_stat + stat;
-  l.off_merge = l.off_trans + trans;
-  l.off_bars = l.off_merge + merge;
+  l.off_bars = l.off_trans + trans;
   l.total = l.off_bars + bars + 1024;
   return l;
 }
 
 // barrier slots
 enum : int {
-  B_FULL = 0, B_EMPTY = 8, B_QFULL = 16, B_QEMPTY = 18, B_TFULL = 20, B_TEMPTY = 24, B_EPI = 28, B_COUNT = 29
+  B_FULL = 0, B_EMPTY = 8, B_QFULL = 16, B_QEMPTY = 18, B_TFULL = 20, B_TEMPTY = 24, B_COUNT = 28
 };
 
 template <int D>
@@ -268,7 +224,6 @@ window_tc_kernel(const __grid_constant__ CUtensorMap tmap_k, const __grid_consta
   unsigned char* sQ = smem + lay.off_q;                             // [2][KB][rows][128 B]
   float2* sStat = reinterpret_cast<float2*>(smem + lay.off_stat);   // [8 warps][rows]
   float* sTrans = reinterpret_cast<float*>(smem + lay.off_trans);   // [8 warps][32][33]
-  float2* sMerge = reinterpret_cast<float2*>(smem + lay.off_merge); // [2][8 warps][rows]
   uint64_t* bars = reinterpret_cast<uint64_t*>(smem + lay.off_bars);
   uint32_t* s_tmem = reinterpret_cast<uint32_t*>(bars + B_COUNT);
   volatile int* s_abort = reinterpret_cast<volatile int*>(s_tmem + 1);
@@ -290,7 +245,6 @@ window_tc_kernel(const __grid_constant__ CUtensorMap tmap_k, const __grid_consta
       mbar_init(BAR(B_QFULL + i), 1);
       mbar_init(BAR(B_QEMPTY + i), 2);     // both issuers release a Q block
     }
-    mbar_init(BAR(B_EPI), 32 * kEpiWarps);
     *s_abort = 0;
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
   }
@@ -374,7 +328,7 @@ window_tc_kernel(const __grid_constant__ CUtensorMap tmap_k, const __grid_consta
         if (!ok) break;
         qphase[qb] ^= 1;
         const uint32_t q_lo = smem_u32(sQ + (size_t)qb * lay.q_block_bytes) >> 4;
-        const bool swap = it.pass == 1 && rows == 128;   // D[row, key] instead of D[key, row]
+        const bool swap = a.pass == 1 && rows == 128;   // D[row, key] instead of D[key, row]
         for (int t = (me ^ tiles_before) & 1; t < ntiles; t += 2) {
           ok = __all_sync(0xffffffffu, mbar_wait(BAR(B_FULL + stage), sphase, s_abort) &&
                                            mbar_wait(BAR(B_TEMPTY + acc), aphase ^ 1, s_abort));
@@ -415,11 +369,20 @@ window_tc_kernel(const __grid_constant__ CUtensorMap tmap_k, const __grid_consta
     const int grp = ew >> 2;
     const int quad = warp & 3;                      // TMEM lane quadrant this warp may read
     float2* myStat = sStat + ew * rows;
-    const int mparts = rows == 128 ? 2 : kEpiWarps;   // contributors per row in a merge: the two groups, or all warps
     float* myT = sTrans + ew * (32 * 33);
-    uint32_t epiphase = 0;
-    int n = 0, n_done = 0;
+    int n = 0;
     bool ok = true;
+    // pass 2: (row max, 1 / row sum) of a unit, lane i holding rows i, i + 32, ...; loaded one item ahead
+    const float2* stat_g = reinterpret_cast<const float2*>(p.stat);
+    float2 pre[4];
+    auto fetch_stats = [&](int k) {
+      const Item nx = decode_item(a, k);
+#pragma unroll
+      for (int q = 0; q < 4; ++q)
+        pre[q] = (nx.valid && q * 32 + lane < rows) ? stat_g[(size_t)(a.u0 + nx.lu) * p.rows_pad + q * 32 + lane]
+                                                    : make_float2(0.f, 0.f);
+    };
+    if (a.pass == 2) fetch_stats(0);
     for (int k = 0; k < a.steps && ok; ++k) {
       const Item it = decode_item(a, k);
       if (!it.valid) continue;
@@ -430,64 +393,13 @@ window_tc_kernel(const __grid_constant__ CUtensorMap tmap_k, const __grid_consta
       float m_run[4], z_run[4];
 #pragma unroll
       for (int rg = 0; rg < 4; ++rg) { m_run[rg] = -INFINITY; z_run[rg] = 0.f; }
-      if (it.pass == 2 && a.mode == 0) {
-        // combine the unit's per-item partials (slot c = pass-1 item c of the unit), in a fixed order:
-        // rows are split over 256 / rows threads, each merging every (256 / rows)-th slot, then the
-        // parts are merged through shared memory and every warp keeps its own copy
-        const int tpr = (32 * kEpiWarps) / rows;
-        const int t = ew * 32 + lane, row = t % rows, part = t / rows;
-        const float2* slot = reinterpret_cast<const float2*>(p.stat_part) + (size_t)u * p.chunks_max * p.rows_pad + row;
-        float M = -INFINITY, z = 0.f;
-        for (int c0 = part; c0 < a.chunks && ok; c0 += 8 * tpr) {
-          uint64_t w[8];
+      if (a.pass == 2) {
+        __syncwarp();                       // the previous item's readers of myStat are done
 #pragma unroll
-          for (int i = 0; i < 8; ++i) {   // eight loads in flight, then consume in order
-            w[i] = ~0ull;
-            const int c = c0 + i * tpr;
-            if (c < a.chunks)
-              asm volatile("ld.relaxed.gpu.global.b64 %0, [%1];" : "=l"(w[i]) : "l"(slot + (size_t)c * p.rows_pad) : "memory");
-          }
-#pragma unroll
-          for (int i = 0; i < 8; ++i) {
-            const int c = c0 + i * tpr;
-            if (c < a.chunks && ok) {
-              float2 o = make_float2(__uint_as_float((uint32_t)w[i]), __uint_as_float((uint32_t)(w[i] >> 32)));
-              if (o.y != o.y) ok = poll_pair(slot + (size_t)c * p.rows_pad, o, s_abort);
-              if (ok && o.x > -INFINITY) {
-                const float Mn = fmaxf(M, o.x);
-                z = fmaf(z, ex2(M - Mn), o.y * ex2(o.x - Mn));
-                M = Mn;
-              }
-            }
-          }
-        }
-        float2* mg = sMerge + (n_done & 1) * (mparts * rows);
-        mg[part * rows + row] = make_float2(M, z);
-        mbar_arrive(BAR(B_EPI));
-        ok = __all_sync(0xffffffffu, ok && mbar_wait(BAR(B_EPI), epiphase, s_abort));
-        epiphase ^= 1;
-        ++n_done;
-        if (!ok) break;
-        for (int i = lane; i < rows; i += 32) {
-          float Mt = -INFINITY;
-          for (int q = 0; q < tpr; ++q) Mt = fmaxf(Mt, mg[q * rows + i].x);
-          float zt = 0.f;
-          for (int q = 0; q < tpr; ++q) {
-            const float2 o = mg[q * rows + i];
-            if (o.x > -INFINITY) zt = fmaf(o.y, ex2(o.x - Mt), zt);
-          }
-          myStat[i] = zt > 0.f ? make_float2(Mt, 1.0f / zt) : make_float2(0.f, 0.f);
-        }
+        for (int q = 0; q < 4; ++q)
+          if (q * 32 + lane < rows) myStat[q * 32 + lane] = pre[q];
         __syncwarp();
-      } else if (it.pass == 2) {
-        __syncwarp();
-        for (int i = lane; i < rows && ok; i += 32) {
-          float2 o;
-          ok = poll_pair(reinterpret_cast<const float2*>(p.stat) + (size_t)u * p.rows_pad + i, o, s_abort);
-          myStat[i] = o;
-        }
-        ok = __all_sync(0xffffffffu, ok);
-        if (!ok) break;
+        fetch_stats(k + 1);                 // in flight while this item's tiles are worked on
       }
       for (int t = 0; t < ntiles; ++t, ++n) {
         if ((n & 1) != grp) continue;
@@ -499,7 +411,7 @@ window_tc_kernel(const __grid_constant__ CUtensorMap tmap_k, const __grid_consta
         const uint32_t taddr = tmem_base + ((uint32_t)(quad * 32) << 16) + (uint32_t)acc * 128u;
         const int tbase = key0 + t * kTile;
         const bool tail = (tbase + kTile - 1 > N - L);   // some key of the tile is masked for some row
-        if (it.pass == 1 && rows == 128) {
+        if (a.pass == 1 && rows == 128) {
           // a TMEM lane is a window row (quad * 32 + lane), the 128 columns are the keys of the tile
           const int pos = N - L + ((quad * 32 + lane) % L);   // last key this window row may see
 #pragma unroll
@@ -534,7 +446,7 @@ window_tc_kernel(const __grid_constant__ CUtensorMap tmap_k, const __grid_consta
               z_run[0] += (zs[0] + zs[1]) + (zs[2] + zs[3]);
             }
           }
-        } else if (it.pass == 1) {
+        } else if (a.pass == 1) {
           const int jw = tbase + quad * 32;              // first key of this warp's 32 lanes
 #pragma unroll
           for (int rg = 0; rg < 4; ++rg) {
@@ -609,34 +521,17 @@ window_tc_kernel(const __grid_constant__ CUtensorMap tmap_k, const __grid_consta
         if (lane == 0) mbar_arrive(BAR(B_TEMPTY + acc));
       }
       if (!ok) break;
-      if (it.pass == 1) {
-        // merge the eight warps' (max, sum) per row in a fixed order; one slot per work item
-        const int nparts = mparts;
-        float2* mg = sMerge + (n_done & 1) * (nparts * rows);
+      if (a.pass == 1) {
+        // the warp's own partial of this item: slot (chunk, part), part = warp (group with 128 rows)
+        float2* slot = reinterpret_cast<float2*>(p.stat_part) +
+                       ((size_t)u * p.chunks_max + (size_t)it.ch * (rows == 128 ? 2 : kTcParts)) * p.rows_pad;
         if (rows == 128) {
-          mg[grp * rows + quad * 32 + lane] = make_float2(m_run[0] * scale2, z_run[0]);
+          slot[(size_t)grp * p.rows_pad + quad * 32 + lane] = make_float2(m_run[0] * scale2, z_run[0]);
         } else {
 #pragma unroll
           for (int rg = 0; rg < 4; ++rg)
-            if (rg * 32 < rows) mg[ew * rows + rg * 32 + lane] = make_float2(m_run[rg] * scale2, z_run[rg]);
+            if (rg * 32 < rows) slot[(size_t)ew * p.rows_pad + rg * 32 + lane] = make_float2(m_run[rg] * scale2, z_run[rg]);
         }
-        mbar_arrive(BAR(B_EPI));
-        ok = __all_sync(0xffffffffu, mbar_wait(BAR(B_EPI), epiphase, s_abort));
-        epiphase ^= 1;
-        if (!ok) break;
-        const int tl = ew * 32 + lane;
-        if (tl < rows) {
-          float M = -INFINITY;
-          for (int w = 0; w < nparts; ++w) M = fmaxf(M, mg[w * rows + tl].x);
-          float z = 0.f;
-          for (int w = 0; w < nparts; ++w) {
-            const float2 o = mg[w * rows + tl];
-            if (o.x > -INFINITY) z = fmaf(o.y, ex2(o.x - M), z);
-          }
-          publish_pair(reinterpret_cast<float2*>(p.stat_part) + ((size_t)u * p.chunks_max + it.ch) * p.rows_pad + tl,
-                       M, z);
-        }
-        ++n_done;
       }
     }
   }
@@ -654,21 +549,35 @@ window_tc_kernel(const __grid_constant__ CUtensorMap tmap_k, const __grid_consta
   if (tid == 0 && *s_abort) set_status(p.status, TASKKV_ETIMEOUT);
 }
 
-// Combine the per-item statistics of one unit, in item order: (row max, 1 / row sum).
-__global__ void window_tc_reduce_kernel(DeviceProblem p, int u0, int slots) {
+// Folds the partial statistics of one unit: slots (item, warp) of pass 1 -> (row max, 1 / row sum).
+// One warp per (unit, row): lanes take every 32nd slot, then a shuffle tree; the order is fixed.
+__global__ void __launch_bounds__(128) window_tc_reduce_kernel(DeviceProblem p, int u0, int slots) {
   const int u = u0 + blockIdx.x;
-  const int row = threadIdx.x;
-  if (row >= p.rows) return;
+  const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
   const float2* part = reinterpret_cast<const float2*>(p.stat_part) + (size_t)u * p.chunks_max * p.rows_pad;
-  float M = -INFINITY;
-  for (int c = 0; c < slots; ++c) M = fmaxf(M, part[(size_t)c * p.rows_pad + row].x);
-  float z = 0.f;
-  for (int c = 0; c < slots; ++c) {
-    const float2 o = part[(size_t)c * p.rows_pad + row];
-    if (o.x > -INFINITY) z = fmaf(o.y, exp2f(o.x - M), z);
+  const int row = blockIdx.y * 4 + warp;
+  if (row < p.rows) {
+    float M = -INFINITY, z = 0.f;
+    for (int c = lane; c < slots; c += 32) {
+      const float2 o = part[(size_t)c * p.rows_pad + row];
+      if (o.x > -INFINITY) {
+        const float Mn = fmaxf(M, o.x);
+        z = z * exp2f(M - Mn) + o.y * exp2f(o.x - Mn);
+        M = Mn;
+      }
+    }
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) {
+      const float M2 = __shfl_xor_sync(0xffffffffu, M, o);
+      const float z2 = __shfl_xor_sync(0xffffffffu, z, o);
+      const float Mn = fmaxf(M, M2);
+      if (Mn > -INFINITY) z = z * exp2f(M - Mn) + z2 * exp2f(M2 - Mn);
+      M = Mn;
+    }
+    if (lane == 0)
+      reinterpret_cast<float2*>(p.stat)[(size_t)u * p.rows_pad + row] =
+          z > 0.f ? make_float2(M, 1.0f / z) : make_float2(0.f, 0.f);
   }
-  reinterpret_cast<float2*>(p.stat)[(size_t)u * p.rows_pad + row] =
-      z > 0.f ? make_float2(M, 1.0f / z) : make_float2(0.f, 0.f);
 }
 
 typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
@@ -704,13 +613,12 @@ bool make_map(CUtensorMap* map, const void* base, int d, uint64_t rows_total, in
             CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
 }
 
-// One launch per pass.  The single-launch order (mode 0) is exact, but measured no faster on B200: with the
-// keys served from L2 the kernel runs into the shared-memory bandwidth of the SM (TMA fill + MMA operand
-// reads + the pass-1 transposition, about 1000 cycles per 128-key tile against 1420 for HBM), and the
-// hit rate stayed low in every order tried.  Both passes run at the HBM copy rate instead.
-constexpr int g_tc_mode = 1;
-constexpr int g_tc_chunk = 2048;   // keys per work item
-constexpr int g_tc_lag = 2;        // single launch: rounds between the two passes of an item
+// Keys per work item.  Every item costs a Q load and, in pass 2, a statistics load, so long items are
+// better as long as the CTAs still get a dozen items each; short sequences keep 2048-key items.
+inline int pick_chunk(int per_seq, int N, int n_sm) {
+  const int big = 2 * kTcChunk;
+  return (int64_t)per_seq * ((N + big - 1) / big) >= (int64_t)12 * n_sm ? big : kTcChunk;
+}
 
 template <int D>
 cudaError_t launch_tc_d(const DeviceProblem& p, const WindowHostInfo& h, cudaStream_t s) {
@@ -726,10 +634,6 @@ cudaError_t launch_tc_d(const DeviceProblem& p, const WindowHostInfo& h, cudaStr
   const int smem = lay.total;
   cudaError_t e = cudaFuncSetAttribute(window_tc_kernel<D>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem);
   if (e != cudaSuccess) return e;
-  // partial and final statistics start as NaN = "not written"
-  e = cudaMemsetAsync(p.stat_part, 0xFF, (size_t)p.U * p.chunks_max * p.rows_pad * sizeof(float2), s);
-  if (e == cudaSuccess) e = cudaMemsetAsync(p.stat, 0xFF, (size_t)p.U * p.rows_pad * sizeof(float2), s);
-  if (e != cudaSuccess) return e;
   const int per_seq = p.R * p.n_kv;
   for (int b = 0; b < h.batch; ++b) {
     const int N = h.seq_lens[b];
@@ -740,36 +644,25 @@ cudaError_t launch_tc_d(const DeviceProblem& p, const WindowHostInfo& h, cudaStr
     a.u0 = b * per_seq;
     a.n_local = per_seq;
     a.N = N;
-    a.chunk_keys = g_tc_chunk < kTcChunk ? kTcChunk : g_tc_chunk / 128 * 128;
+    a.chunk_keys = pick_chunk(per_seq, N, n_sm);
     a.chunks = (N + a.chunk_keys - 1) / a.chunk_keys;
     const int n1 = a.n_local * a.chunks;
     const int grid = n1 < n_sm ? n1 : n_sm;
-    const int rounds = (n1 + grid - 1) / grid;
-    // the single-launch order needs the partials of a unit within reach of one combine step
-    const bool single = g_tc_mode == 0 && a.chunks <= 64;
-    if (single) {
-      a.mode = 0;
-      a.lag = g_tc_lag;
-      a.steps = 2 * (rounds + a.lag);
+    a.steps = (n1 + grid - 1) / grid;
+    const int parts = p.rows == 128 ? 2 : kTcParts;
+    a.pass = 1;
+    {
       LaunchScope ls(K_WINDOW_TC, s);
       window_tc_kernel<D><<<grid, kThreads, smem, s>>>(mk, mq, p, a, lay);
-    } else {
-      a.lag = 0;
-      a.steps = rounds;
-      a.mode = 1;
-      {
-        LaunchScope ls(K_WINDOW_TC, s);
-        window_tc_kernel<D><<<grid, kThreads, smem, s>>>(mk, mq, p, a, lay);
-      }
-      {
-        LaunchScope ls(K_WINDOW_REDUCE, s);
-        window_tc_reduce_kernel<<<per_seq, 128, 0, s>>>(p, a.u0, a.chunks);
-      }
-      a.mode = 2;
-      {
-        LaunchScope ls(K_WINDOW_TC, s);
-        window_tc_kernel<D><<<grid, kThreads, smem, s>>>(mk, mq, p, a, lay);
-      }
+    }
+    {
+      LaunchScope ls(K_WINDOW_REDUCE, s);
+      window_tc_reduce_kernel<<<dim3(per_seq, (p.rows + 3) / 4), 128, 0, s>>>(p, a.u0, a.chunks * parts);
+    }
+    a.pass = 2;
+    {
+      LaunchScope ls(K_WINDOW_TC, s);
+      window_tc_kernel<D><<<grid, kThreads, smem, s>>>(mk, mq, p, a, lay);
     }
     e = cudaGetLastError();
     if (e != cudaSuccess) return e;
