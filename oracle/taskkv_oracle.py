@@ -22,6 +22,8 @@ in the paper's order and notation:
     Eq. 17   k = (B - N f(r))/(n - f(r)) - s1 - s2            mid_budget
     Eq. 1    decode row: softmax(q K^T / sqrt(d)) V           decode_attention
     Eq. 1-2  exact semantic vector from the N x N weights     exact_semantic_vector
+    Sec. V-G   the two other compensation methods compared    recent_only_indices,
+               with the middle activations                    mean_groups, compensated_cache
 
 Readings where the paper is silent or garbled are stated in each docstring.
 
@@ -30,7 +32,10 @@ here as "parity unpinned": the grouped-query rule of column_mean (mean over
 the group's G*L softmax rows), the zero-padded divisor-w pooling convention,
 round-half-up in hetero_count, floor in mid_budget and lowest-index tie-breaks
 are readings of this build, not statements of the paper; the paper prints no
-worked numeric example of C, v' or a distance.
+worked numeric example of C, v' or a distance.  Of the Sec. V-G variants the
+paper gives only a figure caption: the contiguous near-equal groups of
+mean_groups and the rounding of a compensation row to the cache's storage
+type are readings too.
 """
 from __future__ import annotations
 
@@ -253,18 +258,81 @@ def decode_attention(q: np.ndarray, k_cache: np.ndarray, v_cache: np.ndarray) ->
 
 
 # --------------------------------------------------------------------------
+# Sec. V-G: the two other information-compensation methods the paper compares
+# the middle activations with, at the same cache size
+# --------------------------------------------------------------------------
+MID_SELECT = 0   # middle activations (the method itself, Sec. IV-B)
+MID_RECENT = 1   # "No Cache": the budget is added to the recent window
+MID_MEAN = 2     # "Compressed Cache": one averaged compensation row per group
+
+
+def recent_only_indices(N: int, sink: int, recent: int, mid_budget: int) -> np.ndarray:
+    """"No Cache" of Sec. V-G: a non-heterogeneous head keeps the sinks and the
+    last recent + mid_budget positions, nothing from the middle."""
+    if N <= sink + recent:
+        return np.arange(N, dtype=np.int64)
+    extra = min(mid_budget, N - sink - recent)
+    return np.concatenate([np.arange(sink, dtype=np.int64),
+                           np.arange(N - recent - extra, N, dtype=np.int64)])
+
+
+def mean_groups(N: int, sink: int, recent: int, count: int) -> np.ndarray:
+    """"Compressed Cache" of Sec. V-G: the intermediate positions [sink, N - recent)
+    are divided into `count` groups.  Reading: contiguous groups in position
+    order whose sizes differ by at most one, group g starting at
+    sink + floor(g * M / count), M = N - sink - recent.  Returns the count + 1
+    boundaries (the last one is N - recent)."""
+    M = N - sink - recent
+    count = min(count, M)
+    return np.array([sink + (g * M) // count for g in range(count)] + [N - recent], dtype=np.int64)
+
+
+def round_to_storage(x: np.ndarray, dtype: str) -> np.ndarray:
+    """A float64 array rounded once, to nearest even, to the cache's element type
+    ("f32" or "bf16": 8 significant bits), returned as float64."""
+    x = np.asarray(x, dtype=F64)
+    if dtype == "f32":
+        return x.astype(np.float32).astype(F64)
+    m, e = np.frexp(x)
+    return np.ldexp(np.round(m * 256.0) / 256.0, e)
+
+
+def compensated_cache(k_u: np.ndarray, v_u: np.ndarray, sink: int, recent: int,
+                      count: int, dtype: str) -> tuple:
+    """"Compressed Cache" of Sec. V-G for one head: sinks, then one compensation
+    row per group (the arithmetic mean of the group's K rows resp. V rows, stored
+    in the cache's element type), then the recent window."""
+    k_u = np.asarray(k_u, dtype=F64)
+    v_u = np.asarray(v_u, dtype=F64)
+    N = k_u.shape[0]
+    if N <= sink + recent or count >= N - sink - recent:
+        return k_u.copy(), v_u.copy()
+    b = mean_groups(N, sink, recent, count)
+    out = []
+    for x in (k_u, v_u):
+        means = np.stack([x[b[g]:b[g + 1]].sum(axis=0) / (b[g + 1] - b[g]) for g in range(len(b) - 1)]) \
+            if count > 0 else np.zeros((0, x.shape[1]))
+        out.append(np.concatenate([x[:sink], round_to_storage(means, dtype), x[N - recent:]]))
+    return out[0], out[1]
+
+
+# --------------------------------------------------------------------------
 # The pipeline for one layer of one sequence, in the paper's order
 # --------------------------------------------------------------------------
 def compress_layer(q_win: np.ndarray, k: np.ndarray, v: np.ndarray, *,
                    n_hetero: int, sink: int, recent: int, mid: int,
                    top_t: int = 256, pool_kernel: int = 7,
-                   promote_center: bool = True, force_class: int = -1) -> dict:
+                   promote_center: bool = True, force_class: int = -1,
+                   mid_policy: int = MID_SELECT) -> dict:
     """Prefill-side compression of one layer (Sec. IV-A then IV-B).
 
     q_win: (n_heads, L, d) observation-window queries; k, v: (n_kv, N, d).
     Heads are classified per KV head (n = n_kv in Eq. 16/17) because V, and so
     the semantic vector of Eq. 15, exists once per KV head.
     force_class: -1 run the separator; 1 every head heterogeneous; 0 none.
+    mid_policy: what a non-heterogeneous head keeps besides sinks and recent
+    window (Sec. V-G): the middle activations, more recent positions, or
+    compensation rows (then "idx" lists the first position of each group).
     Returns C, top-t indices, semantic vectors, center, distances, classes,
     retained indices and lengths per KV head.
     """
@@ -284,8 +352,16 @@ def compress_layer(q_win: np.ndarray, k: np.ndarray, v: np.ndarray, *,
         cls = np.zeros(n_kv, dtype=np.uint8)
     else:
         cls = semantic_separator(dist, n_hetero, promote_center)
-    idx = [retained_indices(int(cls[u]), C[u], sink, recent, mid, pool_kernel)
-           for u in range(n_kv)]
+    def keep(u: int) -> np.ndarray:
+        if cls[u] != CLASS_NON_HETERO or mid_policy == MID_SELECT or N <= sink + recent:
+            return retained_indices(int(cls[u]), C[u], sink, recent, mid, pool_kernel)
+        if mid_policy == MID_RECENT:
+            return recent_only_indices(N, sink, recent, mid)
+        if mid >= N - sink - recent:
+            return np.arange(N, dtype=np.int64)
+        return np.concatenate([np.arange(sink, dtype=np.int64), mean_groups(N, sink, recent, mid)[:-1],
+                               np.arange(N - recent, N, dtype=np.int64)])
+    idx = [keep(u) for u in range(n_kv)]
     return {
         "C": C, "top": top, "sem": sem, "center": semantic_center(sem), "dist": dist,
         "cls": cls, "idx": idx, "len": np.array([len(i) for i in idx], dtype=np.int64),
@@ -296,6 +372,23 @@ def gather_cache(k: np.ndarray, v: np.ndarray, idx: list) -> tuple:
     """Sec. IV-B: the per-head compacted cache, rows in ascending position."""
     return ([np.asarray(k[u], dtype=F64)[idx[u]] for u in range(len(idx))],
             [np.asarray(v[u], dtype=F64)[idx[u]] for u in range(len(idx))])
+
+
+def gather_cache_policy(k: np.ndarray, v: np.ndarray, cls: np.ndarray, idx: list, *, mid_policy: int,
+                        sink: int, recent: int, mid: int, dtype: str) -> tuple:
+    """The per-head cache under a Sec. V-G policy: as gather_cache, except that
+    with MID_MEAN a non-heterogeneous head holds compensation rows."""
+    if mid_policy != MID_MEAN:
+        return gather_cache(k, v, idx)
+    kc, vc = [], []
+    for u in range(len(idx)):
+        if cls[u] == CLASS_NON_HETERO:
+            a, b = compensated_cache(k[u], v[u], sink, recent, mid, dtype)
+        else:
+            a, b = np.asarray(k[u], dtype=F64).copy(), np.asarray(v[u], dtype=F64).copy()
+        kc.append(a)
+        vc.append(b)
+    return kc, vc
 
 
 def decode_layer(q: np.ndarray, k_cache: list, v_cache: list) -> np.ndarray:

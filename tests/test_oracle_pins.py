@@ -314,3 +314,105 @@ def test_grouped_decode_and_append():
     ref = torch.nn.functional.scaled_dot_product_attention(
         torch.from_numpy(qd).reshape(n_kv, n // n_kv, d), torch.from_numpy(k_all), torch.from_numpy(v_all))
     np.testing.assert_allclose(got, ref.reshape(n, d).numpy(), rtol=0, atol=1e-13)
+
+
+# ---------------------------------------------------------------------------
+# Sec. V-G: the "No Cache" and "Compressed Cache" compensation methods
+# ---------------------------------------------------------------------------
+def test_recent_only_equals_masked_attention_with_a_longer_recent_window():
+    # "No Cache" at cache size c: the c extra positions join the recent window
+    q, k, v = _toy_layer(seed=21)
+    N, d = k.shape[1], k.shape[2]
+    s1, s2, c = 4, 16, 9
+    out = O.compress_layer(q, k, v, n_hetero=0, sink=s1, recent=s2, mid=c, top_t=64, promote_center=False,
+                           mid_policy=O.MID_RECENT)
+    for u in range(k.shape[0]):
+        assert out["idx"][u].tolist() == list(range(s1)) + list(range(N - s2 - c, N))
+    kc, vc = O.gather_cache(k, v, out["idx"])
+    qd = rng(22).normal(size=(8, d))
+    got = O.decode_layer(qd, kc, vc)
+    keep = np.zeros(N, dtype=bool)
+    keep[:s1] = True
+    keep[N - s2 - c:] = True
+    for a in range(8):
+        s = np.array([qd[a] @ k[a, j] / math.sqrt(d) if keep[j] else -np.inf for j in range(N)])
+        p = np.exp(s - s[keep].max())
+        p /= p.sum()
+        np.testing.assert_allclose(got[a], p @ v[a], rtol=0, atol=1e-13)
+
+
+@pytest.mark.parametrize("N,s1,s2,c", [(100, 4, 10, 7), (64, 0, 8, 56), (33, 3, 5, 1), (50, 4, 6, 40), (40, 4, 6, 1000)])
+def test_mean_groups_partition_the_middle(N, s1, s2, c):
+    b = O.mean_groups(N, s1, s2, c)
+    M = N - s1 - s2
+    cc = min(c, M)
+    assert len(b) == cc + 1 and b[0] == s1 and b[-1] == N - s2
+    sizes = np.diff(b)
+    assert sizes.sum() == M and sizes.min() >= M // cc and sizes.max() <= -(-M // cc)   # contiguous, near-equal
+    assert np.all(sizes > 0)
+
+
+def test_compensation_rows_by_hand_loops():
+    # every compensation row is the plain average of its group's rows (python loops, tiny case)
+    r = rng(23)
+    N, d, s1, s2, c = 23, 3, 2, 4, 5
+    k, v = r.normal(size=(N, d)), r.normal(size=(N, d))
+    kc, vc = O.compensated_cache(k, v, s1, s2, c, "f32")
+    assert kc.shape == (s1 + c + s2, d)
+    b = O.mean_groups(N, s1, s2, c)
+    for x, xc in ((k, kc), (v, vc)):
+        for g in range(c):
+            for e in range(d):
+                tot = 0.0
+                for j in range(int(b[g]), int(b[g + 1])):
+                    tot += x[j, e]
+                assert abs(xc[s1 + g, e] - np.float32(tot / (b[g + 1] - b[g]))) <= 1e-7 * abs(tot) + 1e-12
+        np.testing.assert_array_equal(xc[:s1], x[:s1])
+        np.testing.assert_array_equal(xc[s1 + c:], x[N - s2:])
+
+
+def test_compensation_special_cases():
+    r = rng(24)
+    N, d, s1, s2 = 40, 4, 3, 5
+    k, v = r.normal(size=(N, d)), r.normal(size=(N, d))
+    # one group per intermediate position (or more): nothing is averaged, the head keeps every row
+    for c in (N - s1 - s2, 1000):
+        kc, vc = O.compensated_cache(k, v, s1, s2, c, "f32")
+        np.testing.assert_array_equal(kc, k)
+        np.testing.assert_array_equal(vc, v)
+    # constant rows: every compensation row is that constant
+    kk = np.tile(np.array([[0.5, -1.25, 2.0, 3.0]]), (N, 1))
+    kc, _ = O.compensated_cache(kk, v, s1, s2, 6, "bf16")
+    np.testing.assert_array_equal(kc, np.tile(kk[:1], (s1 + 6 + s2, 1)))
+    # conservation: sizes x means add up to the sum of the intermediate rows
+    kc, _ = O.compensated_cache(k, v, s1, s2, 7, "f32")
+    sizes = np.diff(O.mean_groups(N, s1, s2, 7))
+    np.testing.assert_allclose((kc[s1:s1 + 7] * sizes[:, None]).sum(axis=0), k[s1:N - s2].sum(axis=0), rtol=1e-6)
+    # c = 0: sinks and recent window only
+    kc, _ = O.compensated_cache(k, v, s1, s2, 0, "f32")
+    np.testing.assert_array_equal(kc, np.concatenate([k[:s1], k[N - s2:]]))
+
+
+def test_round_to_storage_matches_library_casts():
+    x = rng(25).normal(size=4096) * np.exp(rng(26).normal(size=4096) * 3)
+    np.testing.assert_array_equal(O.round_to_storage(x, "bf16"),
+                                  torch.from_numpy(x).to(torch.bfloat16).double().numpy())
+    np.testing.assert_array_equal(O.round_to_storage(x, "f32"), torch.from_numpy(x).float().double().numpy())
+    # a tie goes to the even mantissa
+    assert O.round_to_storage(np.array([1.0 + 2.0 ** -8]), "bf16")[0] == 1.0
+    assert O.round_to_storage(np.array([1.0 + 3 * 2.0 ** -8]), "bf16")[0] == 1.0 + 2.0 ** -6
+
+
+def test_policy_pipeline_lengths_and_classes_do_not_depend_on_the_policy():
+    q, k, v = _toy_layer(seed=27)
+    base = O.compress_layer(q, k, v, n_hetero=2, sink=4, recent=16, mid=12, top_t=64)
+    for pol in (O.MID_RECENT, O.MID_MEAN):
+        out = O.compress_layer(q, k, v, n_hetero=2, sink=4, recent=16, mid=12, top_t=64, mid_policy=pol)
+        assert out["cls"].tolist() == base["cls"].tolist()
+        assert out["len"].tolist() == base["len"].tolist()
+        kc, vc = O.gather_cache_policy(k, v, out["cls"], out["idx"], mid_policy=pol, sink=4, recent=16, mid=12,
+                                       dtype="f32")
+        assert [len(x) for x in kc] == base["len"].tolist()
+        for u in range(k.shape[0]):
+            if out["cls"][u] != 0:
+                np.testing.assert_array_equal(kc[u], k[u])
