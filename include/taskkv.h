@@ -56,6 +56,19 @@ typedef int32_t taskkv_status;
 #define TASKKV_CLASS_HETERO     1
 #define TASKKV_CLASS_CENTER     2   /* the head closest to the center, promoted to a full cache */
 
+/* The information-compensation methods compared in Sec. V-G, at equal cache size (mid_budget rows):
+ *   SELECT  the middle activations of Sec. IV-B (the method itself; default)
+ *   RECENT  "No Cache": the budget goes to the recent window, nothing is kept from the middle
+ *   MEAN    "Compressed Cache": the intermediate positions [s1, N - s2) are cut into mid_budget contiguous
+ *           groups of near-equal size (group g starts at s1 + floor(g * M / mid_budget), M = N - s1 - s2) and
+ *           each group is replaced by one compensation row, the mean of its K rows resp. V rows (fp32
+ *           accumulation in position order, stored in the cache's element type).  In the retained-index
+ *           table a compensation row is listed with the first position of its group.
+ * Classes, lengths, capacities and every buffer size are the same under all three. */
+#define TASKKV_MID_SELECT 0
+#define TASKKV_MID_RECENT 1
+#define TASKKV_MID_MEAN   2
+
 #define TASKKV_MAX_TOP_T       1024
 #define TASKKV_MAX_KV_HEADS    64
 #define TASKKV_MAX_WINDOW_ROWS 128  /* G * window */
@@ -82,7 +95,7 @@ typedef struct taskkv_params {
   int32_t force_class;       /* -1: run the separator; 1: every head heterogeneous; 0: none */
   int32_t dtype;             /* TASKKV_F32 or TASKKV_BF16: element type of q, k, v, out and the pools */
   int32_t max_new_tokens;    /* rows reserved per unit for taskkv_append */
-  int32_t reserved_;
+  int32_t mid_policy;        /* TASKKV_MID_*: what a non-heterogeneous head keeps beside sinks and recent window */
   const int32_t* seq_lens;   /* host [batch]: N_b (ragged batches allowed) */
   const int32_t* mid_budget_per_layer;  /* host [n_layers] or NULL; overrides mid_budget */
   const int32_t* n_hetero;   /* host [batch][n_layers] or NULL; overrides Eq. 16 */

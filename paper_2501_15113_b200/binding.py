@@ -36,7 +36,7 @@ class taskkv_params(C.Structure):
         ("batch", C.c_int32), ("sink", C.c_int32), ("recent", C.c_int32), ("mid_budget", C.c_int32),
         ("window", C.c_int32), ("top_t", C.c_int32), ("pool_kernel", C.c_int32), ("m_top", C.c_int32),
         ("beta", C.c_float), ("promote_center", C.c_int32), ("force_class", C.c_int32), ("dtype", C.c_int32),
-        ("max_new_tokens", C.c_int32), ("reserved_", C.c_int32),
+        ("max_new_tokens", C.c_int32), ("mid_policy", C.c_int32),
         ("seq_lens", C.POINTER(C.c_int32)), ("mid_budget_per_layer", C.POINTER(C.c_int32)),
         ("n_hetero", C.POINTER(C.c_int32)),
     ]
@@ -139,7 +139,7 @@ class Params:
     def __init__(self, *, n_layers, n_heads, n_kv_heads, head_dim, seq_lens: Sequence[int], sink, recent,
                  mid_budget, window, dtype, top_t=256, pool_kernel=7, beta=0.25, m_top=4,
                  n_hetero: Optional[Sequence[Sequence[int]]] = None, promote_center=True, force_class=-1,
-                 max_new_tokens=0):
+                 max_new_tokens=0, mid_policy=0):
         p = taskkv_params()
         lib.taskkv_params_default(C.byref(p))
         p.n_layers, p.n_heads, p.n_kv_heads, p.head_dim = n_layers, n_heads, n_kv_heads, head_dim
@@ -165,6 +165,7 @@ class Params:
         p.force_class = force_class
         p.dtype = BF16 if dtype in (BF16, "bf16", torch.bfloat16) else F32
         p.max_new_tokens = max_new_tokens
+        p.mid_policy = int(mid_policy)
         self.c = p
 
     @property

@@ -54,6 +54,7 @@ taskkv_status make_plan(const taskkv_params* p, HostPlan& hp) {
   if (p->top_t < 1 || p->top_t > TASKKV_MAX_TOP_T) return TASKKV_EINVAL;
   if (p->pool_kernel < 1 || p->pool_kernel > 31 || p->pool_kernel % 2 == 0) return TASKKV_EINVAL;
   if (p->force_class < -1 || p->force_class > 1) return TASKKV_EINVAL;
+  if (p->mid_policy < TASKKV_MID_SELECT || p->mid_policy > TASKKV_MID_MEAN) return TASKKV_EINVAL;
   const int B = p->batch, R = p->n_layers, nkv = p->n_kv_heads;
   if ((int64_t)B * R * nkv > (1 << 20)) return TASKKV_EINVAL;
 
@@ -174,7 +175,7 @@ thread_local cudaEvent_t tl_start = nullptr;
 
 const char* kKernelNames[K_COUNT] = {
     "window_stats", "window_reduce", "window_scores", "select", "separator", "plan",
-    "gather", "append", "decode_plan", "decode_attn", "decode_combine", "window_tc"};
+    "gather", "append", "decode_plan", "decode_attn", "decode_combine", "window_tc", "compensate"};
 
 }  // namespace
 
@@ -237,6 +238,10 @@ void fill_device_problem(taskkv_cache* c) {
   d.recent = p.recent;
   d.promote_center = p.promote_center;
   d.force_class = p.force_class;
+  d.mid_policy = p.mid_policy;
+  d.max_mid = 0;
+  for (int32_t m : hp.mid) d.max_mid = m > d.max_mid ? m : d.max_mid;
+  if (d.max_mid > hp.max_N) d.max_mid = hp.max_N;
   d.max_new = p.max_new_tokens;
   d.idx_stride = hp.idx_stride;
   d.chunks_max = hp.chunks_max;
@@ -330,6 +335,7 @@ void taskkv_params_default(taskkv_params* p) {
   p->m_top = 4;
   p->promote_center = 1;
   p->force_class = -1;
+  p->mid_policy = TASKKV_MID_SELECT;
   p->dtype = TASKKV_BF16;
   p->max_new_tokens = 0;
 }
@@ -409,6 +415,7 @@ taskkv_status taskkv_compress_ex(const taskkv_params* p, const void* const* q_wi
   if (e == cudaSuccess) e = launch_select(c->dp, p->dtype, c->hp.max_N, s);
   if (e == cudaSuccess) e = launch_separator_plan(c->dp, p->batch * p->n_layers, s);
   if (e == cudaSuccess) e = launch_gather(c->dp, p->dtype, c->hp.info.gather_items, s);
+  if (e == cudaSuccess && p->mid_policy == TASKKV_MID_MEAN) e = launch_compensate(c->dp, p->dtype, s);
   if (e != cudaSuccess) {
     std::fprintf(stderr, "taskkv_compress_ex: CUDA error: %s\n", cudaGetErrorString(e));
     taskkv_cache_destroy(c);

@@ -31,6 +31,7 @@ enum KernelId : int32_t {
   K_DECODE_ATTN,
   K_DECODE_COMBINE,
   K_WINDOW_TC,
+  K_COMPENSATE,
   K_COUNT
 };
 
@@ -45,6 +46,8 @@ struct DeviceProblem {
   int32_t top_t, pool_w;
   int32_t sink, recent;
   int32_t promote_center, force_class;
+  int32_t mid_policy;   // TASKKV_MID_*
+  int32_t max_mid;      // largest middle budget of any layer
   int32_t max_new;
   int32_t idx_stride;   // ints per unit in idx
   int32_t chunks_max;   // partial-statistic slots per unit (longest sequence)
@@ -110,6 +113,7 @@ cudaError_t launch_select(const DeviceProblem& p, int dtype, int max_N, cudaStre
 cudaError_t launch_separator_plan(const DeviceProblem& p, int n_br, cudaStream_t s);
 cudaError_t launch_decode_plan(const DeviceProblem& p, const int32_t* lengths, cudaStream_t s);
 cudaError_t launch_gather(const DeviceProblem& p, int dtype, int64_t gather_items, cudaStream_t s);
+cudaError_t launch_compensate(const DeviceProblem& p, int dtype, cudaStream_t s);
 cudaError_t launch_append(const DeviceProblem& p, int dtype, const void* k_new, const void* v_new,
                           cudaStream_t s);
 cudaError_t launch_decode(const DeviceProblem& p, int dtype, const void* q, const int32_t* lengths, void* out,

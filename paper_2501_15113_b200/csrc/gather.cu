@@ -83,7 +83,72 @@ __global__ void __launch_bounds__(256) append_kernel(DeviceProblem p, const unsi
   }
 }
 
+// "Compressed Cache" of Sec. V-G: rows s1 .. s1 + c - 1 of a non-heterogeneous unit's segment become the
+// means of c contiguous groups of the intermediate positions (their first positions are in the index
+// table).  One thread per 16-byte column of one compensation row adds the group's rows in position order in
+// fp32 and stores the mean in the cache's element type; K and V alike.  Runs after the gather.
+template <typename T, int D>
+__global__ void __launch_bounds__(kGatherThreads) compensate_kernel(DeviceProblem p) {
+  constexpr int EPV = 16 / (int)sizeof(T);            // elements per 16-byte vector
+  constexpr int VPR = D / EPV;                        // vectors (threads) per row
+  constexpr int RPB = kGatherThreads / VPR;           // compensation rows per block
+  constexpr int ROW_BYTES = D * (int)sizeof(T);
+  const int u = blockIdx.y;
+  const int N = p.unit_N[u], len = p.len[u];
+  if (len == N) return;                               // the unit kept everything
+  const int s1 = p.sink, s2 = p.recent;
+  const int c = len - s1 - s2;                        // compensation rows
+  const int g = blockIdx.x * RPB + threadIdx.x / VPR;
+  if (g >= c) return;
+  const int vc = threadIdx.x % VPR;
+  const int64_t seg = p.seg_off[u];
+  if (seg + len > p.pool_rows) return;                // planning overflow, already flagged
+  const int32_t* idx = p.idx + (size_t)u * p.idx_stride;
+  int j0 = idx[s1 + g];
+  int j1 = (g + 1 < c) ? idx[s1 + g + 1] : N - s2;
+  j0 = min(max(j0, s1), N - s2);
+  j1 = min(max(j1, j0), N - s2);
+  const unsigned char* ksrc = static_cast<const unsigned char*>(p.k_ptr[u]) + vc * 16;
+  const unsigned char* vsrc = static_cast<const unsigned char*>(p.v_ptr[u]) + vc * 16;
+  float ka[EPV], va[EPV];
+#pragma unroll
+  for (int e = 0; e < EPV; ++e) { ka[e] = 0.f; va[e] = 0.f; }
+  for (int j = j0; j < j1; ++j) {
+    float kf[EPV], vf[EPV];
+    Vec16<T>::unpack(*reinterpret_cast<const uint4*>(ksrc + (size_t)j * ROW_BYTES), kf);
+    Vec16<T>::unpack(*reinterpret_cast<const uint4*>(vsrc + (size_t)j * ROW_BYTES), vf);
+#pragma unroll
+    for (int e = 0; e < EPV; ++e) { ka[e] += kf[e]; va[e] += vf[e]; }
+  }
+  const float cnt = (float)max(j1 - j0, 1);
+  T* kdst = reinterpret_cast<T*>(static_cast<unsigned char*>(p.k_pool) + ((size_t)seg + s1 + g) * ROW_BYTES) + vc * EPV;
+  T* vdst = reinterpret_cast<T*>(static_cast<unsigned char*>(p.v_pool) + ((size_t)seg + s1 + g) * ROW_BYTES) + vc * EPV;
+#pragma unroll
+  for (int e = 0; e < EPV; ++e) {
+    store_out(kdst + e, ka[e] / cnt);
+    store_out(vdst + e, va[e] / cnt);
+  }
+}
+
+template <typename T, int D>
+cudaError_t launch_compensate_typed(const DeviceProblem& p, int max_rows, cudaStream_t s) {
+  constexpr int RPB = kGatherThreads / (D * (int)sizeof(T) / 16);
+  const dim3 grid((unsigned)((max_rows + RPB - 1) / RPB), (unsigned)p.U);
+  compensate_kernel<T, D><<<grid, kGatherThreads, 0, s>>>(p);
+  return cudaGetLastError();
+}
+
 }  // namespace
+
+cudaError_t launch_compensate(const DeviceProblem& p, int dtype, cudaStream_t s) {
+  if (p.max_mid <= 0) return cudaSuccess;
+  LaunchScope ls(K_COMPENSATE, s);
+  if (dtype == TASKKV_F32)
+    return p.d == 64 ? launch_compensate_typed<float, 64>(p, p.max_mid, s)
+                     : launch_compensate_typed<float, 128>(p, p.max_mid, s);
+  return p.d == 64 ? launch_compensate_typed<__nv_bfloat16, 64>(p, p.max_mid, s)
+                   : launch_compensate_typed<__nv_bfloat16, 128>(p, p.max_mid, s);
+}
 
 cudaError_t launch_gather(const DeviceProblem& p, int dtype, int64_t gather_items, cudaStream_t s) {
   if (gather_items <= 0) return cudaSuccess;

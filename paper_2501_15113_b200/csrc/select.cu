@@ -215,6 +215,14 @@ __global__ void __launch_bounds__(kThreads) select_kernel(DeviceProblem p) {
   int* idx = p.idx + (size_t)u * p.idx_stride;
   for (int i = tid; i < s1; i += kThreads) idx[i] = i;
   for (int i = tid; i < s2; i += kThreads) idx[s1 + kmid + i] = N - s2 + i;
+  if (p.mid_policy != TASKKV_MID_SELECT) {
+    // Sec. V-G variants: the budget extends the recent window, or names the first position of each of the
+    // kmid contiguous groups whose mean becomes a compensation row (written after the gather)
+    for (int i = tid; i < kmid; i += kThreads)
+      idx[s1 + i] = p.mid_policy == TASKKV_MID_RECENT ? hi - kmid + i
+                                                     : lo + (int)(((int64_t)i * (hi - lo)) / kmid);
+    return;
+  }
   if (kmid > 0) {
     const PooledKey pkey{C, N, (p.pool_w - 1) / 2};
     __syncthreads();
@@ -387,6 +395,14 @@ __global__ void __launch_bounds__(kThreads, 1) select_fast_kernel(DeviceProblem 
   int* idx = p.idx + (size_t)u * p.idx_stride;
   for (int i = tid; i < s1; i += kThreads) idx[i] = i;
   for (int i = tid; i < s2; i += kThreads) idx[s1 + kmid + i] = N - s2 + i;
+  if (p.mid_policy != TASKKV_MID_SELECT) {
+    // Sec. V-G variants: the budget extends the recent window, or names the first position of each of the
+    // kmid contiguous groups whose mean becomes a compensation row (written after the gather)
+    for (int i = tid; i < kmid; i += kThreads)
+      idx[s1 + i] = p.mid_policy == TASKKV_MID_RECENT ? hi - kmid + i
+                                                     : lo + (int)(((int64_t)i * (hi - lo)) / kmid);
+    return;
+  }
   if (kmid == 0) return;
 
   // pooled window sums in ascending position: ext = [3 left neighbours][32 own][3 right neighbours]

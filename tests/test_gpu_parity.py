@@ -265,3 +265,73 @@ def test_budget_sweep_points(n_hetero, mid):
     from paper_2501_15113_b200 import configs
     wl = configs.config5_sweep(n_hetero, mid, seq_len=5000, batch=2, decode_steps=2)
     run_workload(wl)
+
+
+# ---------------------------------------------------------------------------
+# Sec. V-G: the other two compensation methods at the same cache size
+# ---------------------------------------------------------------------------
+POLICY_CASES = [
+    dict(n=4, n_kv=4, d=64, N=1500, L=16, s1=4, s2=32, k=37, dtype="f32"),
+    dict(n=4, n_kv=4, d=128, N=2341, L=32, s1=4, s2=64, k=100, dtype="bf16"),
+    dict(n=8, n_kv=2, d=128, N=3000, L=32, s1=3, s2=50, k=64, dtype="bf16", nh=0),      # grouped queries
+    dict(n=4, n_kv=4, d=64, N=700, L=8, s1=4, s2=32, k=0, dtype="bf16"),                # cache size 0
+    dict(n=4, n_kv=4, d=64, N=700, L=8, s1=4, s2=32, k=663, dtype="f32"),               # groups of one or two rows
+    dict(n=4, n_kv=4, d=64, N=700, L=8, s1=4, s2=32, k=10 ** 6, dtype="bf16"),          # budget covers the middle
+    dict(n=8, n_kv=4, d=128, N=0, L=32, s1=4, s2=128, k=200, dtype="bf16", R=2, seq_lens=[1500, 2049], nh=1),
+]
+
+
+@pytest.mark.parametrize("policy", [1, 2], ids=["recent", "mean"])
+@pytest.mark.parametrize("case", POLICY_CASES, ids=[f"case{i}" for i in range(len(POLICY_CASES))])
+def test_compensation_policies(case, policy):
+    tk, P = _tk(), _parity()
+    from oracle import taskkv_oracle as O
+    wl = small("policy", **case)
+    qs, ks, vs = W.materialize(wl, DEV)
+    steps = wl.decode_steps
+    params = tk.params_from_workload(wl, max_new_tokens=steps, mid_policy=policy)
+    cache = tk.taskkv_compress_ex(params, qs, ks, vs)
+    assert cache.status() == 0
+    lens, cls, idx_tab = cache.lengths(), cache.classes(), cache.query(tk.Q_INDICES)
+    step_inputs = [W.gen_decode_step(wl, s, DEV) for s in range(steps)]
+    outs = []
+    for (q, kn, vn) in step_inputs:
+        cache.taskkv_append(kn, vn)
+        outs.append(cache.taskkv_decode(q))
+    assert cache.status() == 0
+    ulp = 2.0 ** -7 if wl.dtype == "bf16" else 1e-6      # one unit in the last place of the stored row
+    worst = 0.0
+    for b in range(wl.batch):
+        N = wl.seq_lens[b]
+        for r in range(wl.n_layers):
+            k64, v64 = P.to64(ks[b][r]), P.to64(vs[b][r])
+            ref = O.compress_layer(P.to64(qs[b][r]), k64, v64, n_hetero=wl.n_hetero[b][r], sink=wl.sink,
+                                   recent=wl.recent, mid=wl.mid_budget[r], top_t=wl.top_t,
+                                   pool_kernel=wl.pool_kernel, promote_center=wl.promote_center, mid_policy=policy)
+            u0 = P.unit_index(wl, b, r, 0)
+            assert cls[u0:u0 + wl.n_kv_heads].tolist() == ref["cls"].tolist()
+            assert lens[u0:u0 + wl.n_kv_heads].tolist() == ref["len"].tolist()
+            kc, vc = O.gather_cache_policy(k64, v64, ref["cls"], ref["idx"], mid_policy=policy, sink=wl.sink,
+                                           recent=wl.recent, mid=wl.mid_budget[r], dtype=wl.dtype)
+            for h in range(wl.n_kv_heads):
+                u = u0 + h
+                if len(ref["idx"][h]) < N:      # positions (group starts for the averaged rows) are exact
+                    assert idx_tab[u, :lens[u]].tolist() == ref["idx"][h].tolist()
+                for name, want in (("k", kc[h]), ("v", vc[h])):
+                    got = P.to64(cache.pool_rows(name, u))[:len(want)]      # rows before the appended tokens
+                    exact = np.ones(len(want), dtype=bool)
+                    if policy == 2 and ref["cls"][h] == 0 and len(want) < N:
+                        exact[wl.sink:len(want) - wl.recent] = False
+                    np.testing.assert_array_equal(got[exact], want[exact])
+                    if (~exact).any():
+                        err = np.abs(got[~exact] - want[~exact])
+                        # fp32 sums in position order against the oracle's fp64 ones, then one rounding to storage
+                        assert np.all(err <= ulp * np.abs(want[~exact]) + 1e-5), f"unit {u} {name}: averaged rows"
+                        if wl.dtype == "bf16":
+                            assert np.mean(err > 0) < 0.01, "more than 1 % of the averaged values differ in the last place"
+            for (q, kn, vn), out in zip(step_inputs, outs):
+                O.append_layer(kc, vc, P.to64(kn[b, r]), P.to64(vn[b, r]))
+                want = O.decode_layer(P.to64(q[b, r]), kc, vc)
+                worst = max(worst, float(np.abs(P.to64(out[b, r]) - want).max()))
+    assert worst < P.TOL_OUT[wl.dtype], f"decode max abs err {worst:.3e}"
+    cache.close()
