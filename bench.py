@@ -105,8 +105,12 @@ class ClockSampler:
                 "samples": len(sm), "reasons": sorted(reasons)}
 
 
-def algorithmic_bytes(wl, info):
-    """Bytes the method itself must move: compress and one decode step."""
+POLICIES = {"select": 0, "recent": 1, "mean": 2}
+
+
+def algorithmic_bytes(wl, info, policy="select"):
+    """Bytes the method itself must move: compress and one decode step.  With averaged
+    compensation rows every intermediate K and V row of a non-heterogeneous head is read once more."""
     es, d = wl.elem_size, wl.head_dim
     G = wl.group
     comp = 0
@@ -117,6 +121,8 @@ def algorithmic_bytes(wl, info):
             kept = wl.kept_len(b, r)
             per_unit = N * d * es + G * wl.window * d * es + 12 * N + min(wl.top_t, N) * d * es
             comp += wl.n_kv_heads * per_unit + 4 * d * es * (h * N + (wl.n_kv_heads - h) * kept)
+            if policy == "mean" and kept < N:
+                comp += (wl.n_kv_heads - h) * 2 * d * es * (N - wl.sink - wl.recent)
     return comp
 
 
@@ -143,7 +149,7 @@ def run_ours(args):
     S = wl.decode_steps
     qs, ks, vs = W.materialize(wl, dev)
     steps_in = [W.gen_decode_step(wl, s, dev) for s in range(S)]
-    params = tk.params_from_workload(wl, max_new_tokens=S)
+    params = tk.params_from_workload(wl, max_new_tokens=S, mid_policy=POLICIES[args.policy])
     info = tk.taskkv_plan(params)
     cache_mem = torch.empty(int(info.cache_bytes), dtype=torch.uint8, device=dev)
     work_mem = torch.empty(int(info.workspace_bytes), dtype=torch.uint8, device=dev)
@@ -213,7 +219,7 @@ def run_ours(args):
 
     tokens = sum(wl.seq_lens)
     es, d = wl.elem_size, wl.head_dim
-    comp_bytes = algorithmic_bytes(wl, info)
+    comp_bytes = algorithmic_bytes(wl, info, args.policy)
     U = int(info.n_units)
     # decode step s (1-based) reads K and V rows of every segment once: retained rows + s appended per unit
     dec_bytes_avg = 2 * d * es * (int(info.retained_rows) + U * (S + 1) / 2.0)
@@ -232,7 +238,7 @@ def run_ours(args):
         "value": value, "unit": "steps/s", "n_gpus": world, "steps": K, "warmup": args.warmup,
         "ms_per_step": total_ms / K, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
         "dtype": wl.dtype, "data": "synthetic",
-        "config": dict(wl.describe(), l2="inputs (>=8 GB of K, >=3 GB retained cache) exceed the 126 MB L2",
+        "config": dict(wl.describe(), mid_policy=args.policy, l2="inputs (>=8 GB of K, >=3 GB retained cache) exceed the 126 MB L2",
                        step="compress all layers + decode_steps x (append + attention)"),
         "decode_ms_per_step": dec_step_ms, "compress_ms": comp_pass_ms, "compress_tokens_per_s": comp_tps,
         "hbm": {
@@ -253,7 +259,9 @@ def run_ours(args):
 
     if rank == 0 and not args.no_e2e:
         line["e2e"] = run_e2e(tk, wl, params, qs, ks, vs, steps_in, world)
-    if rank == 0 and world == 1 and not args.no_cpu:
+    if rank == 0 and world == 1 and not args.no_cpu and args.policy != "select":
+        line["cpu_baseline"] = None      # the oracle is timed on the method's own policy only
+    elif rank == 0 and world == 1 and not args.no_cpu:
         line["cpu_baseline"] = cpu_baseline(wl, qs, ks, vs, steps_in)
     if rank == 0:
         print(json.dumps(line))
@@ -399,6 +407,8 @@ def main():
     ap.add_argument("--seq-len", type=int, default=0)
     ap.add_argument("--layers", type=int, default=0)
     ap.add_argument("--decode-steps", type=int, default=0)
+    ap.add_argument("--policy", default="select", choices=sorted(POLICIES),
+                    help="what a non-heterogeneous head keeps beside sinks and recent window (Sec. V-G)")
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--no-cpu", action="store_true")
     args = ap.parse_args()
