@@ -198,7 +198,9 @@ def run_ours(args):
     for c in caches:
         c.close()
     total_ms = t0.elapsed_time(t1)
-    comp_ms = sum(e[0].elapsed_time(e[1]) for e in evs)
+    comp_each = [e[0].elapsed_time(e[1]) for e in evs]
+    dec_each = [e[1].elapsed_time(e[2]) / S for e in evs]       # per decode step, one value per timed pass
+    comp_ms = sum(comp_each)
     dec_ms = sum(e[1].elapsed_time(e[2]) for e in evs)
     K = args.steps
     # whole-job rates: units of all ranks over the slowest rank's time (one small all-reduce when N > 1)
@@ -241,6 +243,9 @@ def run_ours(args):
         "config": dict(wl.describe(), mid_policy=args.policy, l2="inputs (>=8 GB of K, >=3 GB retained cache) exceed the 126 MB L2",
                        step="compress all layers + decode_steps x (append + attention)"),
         "decode_ms_per_step": dec_step_ms, "compress_ms": comp_pass_ms, "compress_tokens_per_s": comp_tps,
+        "per_pass": {"compress_ms_median": statistics.median(comp_each), "compress_ms_min": min(comp_each),
+                     "decode_ms_per_step_median": statistics.median(dec_each),
+                     "decode_ms_per_step_min": min(dec_each), "passes": len(evs)},
         "hbm": {
             "peak_gbs": peak, "peak_kind": peak_kind, "nominal_gbs": NOMINAL_HBM_GBS,
             "decode_gbs": dec_bytes_avg / (dec_step_ms * 1e-3) / 1e9,
@@ -309,29 +314,38 @@ def run_e2e(tk, wl, params, qs, ks, vs, steps_in, world):
             "decode_ms_per_step": (t2 - t1) * 1e3 / S, "timing": "host wall clock around synchronous calls"}
 
 
-def oracle_sample(wl, qs, ks, vs, steps_in, n_units: int, n_steps: int):
-    """Times the oracle on the first n_units KV heads of layer 0 of sequence 0 and
-    n_steps decode steps of those units; returns seconds (compress, decode) and the scale factors."""
-    import numpy as np
+def oracle_sample(wl, qs, ks, vs, steps_in, n_units: int, n_steps: int, budget_s: float = 0.0):
+    """Times the oracle on the first n_units KV heads of sequence 0, layer after layer until budget_s seconds
+    of compression are spent (at least layer 0), then on decode steps of those layers (at most n_steps per
+    layer, same time budget).  Returns seconds (compress, decode), keys scanned and rows read."""
     from oracle import taskkv_oracle as O
     G = wl.group
     n_units = min(n_units, wl.n_kv_heads)
-    q = qs[0][0][:n_units * G].double().cpu().numpy()
-    k = ks[0][0][:n_units].double().cpu().numpy()
-    v = vs[0][0][:n_units].double().cpu().numpy()
+    caches, keys = [], 0
     t0 = time.perf_counter()
-    ref = O.compress_layer(q, k, v, n_hetero=min(wl.n_hetero[0][0], n_units), sink=wl.sink, recent=wl.recent,
-                           mid=wl.mid_budget[0], top_t=wl.top_t, pool_kernel=wl.pool_kernel,
-                           promote_center=wl.promote_center)
-    kc, vc = O.gather_cache(k, v, ref["idx"])
+    for r in range(wl.n_layers):
+        q = qs[0][r][:n_units * G].double().cpu().numpy()
+        k = ks[0][r][:n_units].double().cpu().numpy()
+        v = vs[0][r][:n_units].double().cpu().numpy()
+        ref = O.compress_layer(q, k, v, n_hetero=min(wl.n_hetero[0][r], n_units), sink=wl.sink, recent=wl.recent,
+                               mid=wl.mid_budget[r], top_t=wl.top_t, pool_kernel=wl.pool_kernel,
+                               promote_center=wl.promote_center)
+        caches.append((r, *O.gather_cache(k, v, ref["idx"])))
+        keys += n_units * wl.seq_lens[0]
+        if time.perf_counter() - t0 >= budget_s:
+            break
     t1 = time.perf_counter()
-    for s in range(n_steps):
-        qd, kn, vn = steps_in[s]
-        O.append_layer(kc, vc, kn[0, 0, :n_units].double().cpu().numpy(), vn[0, 0, :n_units].double().cpu().numpy())
-        O.decode_layer(qd[0, 0, :n_units * G].double().cpu().numpy(), kc, vc)
+    rows = 0
+    for (r, kc, vc) in caches:
+        for s in range(n_steps):
+            qd, kn, vn = steps_in[s]
+            O.append_layer(kc, vc, kn[0, r, :n_units].double().cpu().numpy(), vn[0, r, :n_units].double().cpu().numpy())
+            O.decode_layer(qd[0, r, :n_units * G].double().cpu().numpy(), kc, vc)
+            rows += int(sum(len(x) for x in kc))
+        if time.perf_counter() - t1 >= budget_s:
+            break
     t2 = time.perf_counter()
-    rows_sample = int(sum(len(i) for i in ref["idx"]))
-    return (t1 - t0), (t2 - t1), n_units, rows_sample
+    return (t1 - t0), (t2 - t1), keys, rows, len(caches)
 
 
 def cpu_threads():
@@ -345,16 +359,16 @@ def cpu_threads():
 
 def cpu_baseline(wl, qs, ks, vs, steps_in):
     n_steps = min(4, len(steps_in))
-    comp_s, dec_s, n_units, rows_sample = oracle_sample(wl, qs, ks, vs, steps_in, 8, n_steps)
-    U = wl.batch * wl.n_layers * wl.n_kv_heads
+    comp_s, dec_s, keys, rows, layers = oracle_sample(wl, qs, ks, vs, steps_in, wl.n_kv_heads, n_steps, budget_s=8.0)
     tokens_units = sum(wl.seq_lens[b] * wl.n_layers * wl.n_kv_heads for b in range(wl.batch))
     # compress cost scales with keys scanned; decode cost with rows read
-    comp_full = comp_s * tokens_units / (n_units * wl.seq_lens[0])
-    dec_full = (dec_s / n_steps) * wl.retained_rows() / rows_sample
+    comp_full = comp_s * tokens_units / keys
+    dec_full = dec_s * wl.retained_rows() / rows
     return {"value": 1.0 / dec_full, "unit": "steps/s", "cores": cpu_threads(), "kind": "oracle",
             "compress_tokens_per_s": sum(wl.seq_lens) / comp_full,
-            "sample": f"{n_units} KV heads of layer 0 (sequence 0): compress {comp_s:.2f} s, {n_steps} decode steps "
-                      f"{dec_s:.2f} s; scaled by keys scanned ({U} units) and by rows read ({wl.retained_rows()} rows)"}
+            "sample": f"all KV heads of {layers} layer(s) of sequence 0: compress {comp_s:.1f} s ({keys} keys), "
+                      f"decode steps {dec_s:.1f} s ({rows} rows read); scaled by keys scanned ({tokens_units}) and "
+                      f"by rows read per step ({wl.retained_rows()})"}
 
 
 def run_reference(args):
@@ -374,17 +388,18 @@ def run_reference(args):
     steps_in = [W.gen_decode_step(wl, s, "cpu") for s in range(2)]
     times = []
     for i in range(args.warmup + args.steps):
-        c, d, nu, rows = oracle_sample(sub, qs, ks, vs, steps_in, n_units, 2)
+        c, d, keys, rows, _ = oracle_sample(sub, qs, ks, vs, steps_in, n_units, 2)
         if i >= args.warmup:
-            times.append((c, d, nu, rows))
+            times.append((c, d, keys, rows))
     comp_s = statistics.mean(t[0] for t in times)
-    dec_s = statistics.mean(t[1] for t in times) / 2
-    nu, rows = times[0][2], times[0][3]
+    dec_s = statistics.mean(t[1] for t in times)
+    keys, rows = times[0][2], times[0][3]
     tokens_units = sum(wl.seq_lens[b] * wl.n_layers * wl.n_kv_heads for b in range(wl.batch))
-    comp_full = comp_s * tokens_units / (nu * wl.seq_lens[0])
+    comp_full = comp_s * tokens_units / keys
     dec_full = dec_s * wl.retained_rows() / rows
+    dec_s /= 2
     value = 1.0 / dec_full
-    sample = (f"{nu} KV heads of layer 0 per step: oracle compress {comp_s:.2f} s + 2 decode steps; scaled to the "
+    sample = (f"{n_units} KV heads of layer 0 per step: oracle compress {comp_s:.2f} s + 2 decode steps; scaled to the "
               f"whole workload by keys scanned and rows read")
     line = {"impl": "reference", "metric": "decode attn steps/s (compress tokens/s beside it)", "value": value,
             "unit": "steps/s", "n_gpus": args.gpus, "steps": args.steps, "warmup": args.warmup,
