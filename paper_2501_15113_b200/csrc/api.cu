@@ -29,7 +29,7 @@ struct HostPlan {
   size_t o_status, o_len, o_cap, o_seg, o_cls, o_dist, o_sem, o_idx, o_goff, o_doff, o_pacc, o_pml, o_kpool,
       o_vpool;
   // inside the workspace
-  size_t w_C, w_spart, w_stat, w_topt, w_sync;
+  size_t w_C, w_spart, w_stat, w_topt;
 };
 
 int32_t hetero_count_impl(int32_t n, float beta, int32_t m, int32_t R, int32_t r) {
@@ -151,7 +151,6 @@ taskkv_status make_plan(const taskkv_params* p, HostPlan& hp) {
   hp.w_spart = take((size_t)U * hp.chunks_max * hp.rows_pad * 8);
   hp.w_stat = take((size_t)U * hp.rows_pad * 8);
   hp.w_topt = take((size_t)U * p->top_t * 4);
-  hp.w_sync = take((size_t)U * 2 * 4);
   const size_t work_bytes = o;
 
   hp.info.n_units = U;
@@ -273,7 +272,6 @@ void fill_device_problem(taskkv_cache* c) {
     d.stat_part = reinterpret_cast<float*>(wm + hp.w_spart);
     d.stat = reinterpret_cast<float*>(wm + hp.w_stat);
     d.topt = reinterpret_cast<int32_t*>(wm + hp.w_topt);
-    d.tc_sync = reinterpret_cast<int32_t*>(wm + hp.w_sync);
   }
 }
 

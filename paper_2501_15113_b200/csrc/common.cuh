@@ -82,7 +82,6 @@ struct DeviceProblem {
   float* stat_part;           // [U][chunks_max][rows_pad][2]
   float* stat;                // [U][rows_pad][2]  (row max in log2 units, 1/Z)
   int32_t* topt;              // [U][top_t]
-  int32_t* tc_sync;           // [2][U] per-unit counters / flags of the tensor-core window path
 };
 
 // launch bookkeeping (api.cu)
