@@ -80,7 +80,7 @@ struct DeviceProblem {
   // workspace
   float* C;                   // scores, units concatenated
   float* stat_part;           // [U][chunks_max][rows_pad][2]
-  float* stat;                // [U][rows_pad][2]  (row max in log2 units, 1/Z)
+  float* stat;                // [U][rows_pad][2]  per row: (max in log2 units, 1/Z), or one offset (tensor-core path)
   int32_t* topt;              // [U][top_t]
 };
 

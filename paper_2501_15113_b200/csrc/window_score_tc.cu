@@ -10,6 +10,8 @@
 //                 them); tcgen05.commit frees the smem stage and hands the accumulator over
 //   warps 2-5, 7-10  two epilogue groups, alternating tiles: tcgen05.ld, softmax arithmetic
 //                 in fp32 registers
+// (A third epilogue group, with one accumulator per group and a single issuer so that every accumulator
+// keeps one issuer and one reader, was measured at the same speed with 128 rows and is not used.)
 // Two passes (two launches), as Eq. 13 needs every row's normaliser before rows can be summed:
 //   pass 1 (row statistics)  every epilogue warp keeps a running (max, exp-sum) per window row
 //     over the keys it sees in a work item and stores it as the warp's own partial; a small
@@ -368,19 +370,20 @@ window_tc_kernel(const __grid_constant__ CUtensorMap tmap_k, const __grid_consta
     const int ew = warp < 6 ? warp - 2 : warp - 3;  // 0..7
     const int grp = ew >> 2;
     const int quad = warp & 3;                      // TMEM lane quadrant this warp may read
-    float2* myStat = sStat + ew * rows;
+    float* myStat = reinterpret_cast<float*>(sStat) + ew * rows;
     float* myT = sTrans + ew * (32 * 33);
     int n = 0;
     bool ok = true;
-    // pass 2: (row max, 1 / row sum) of a unit, lane i holding rows i, i + 32, ...; loaded one item ahead
-    const float2* stat_g = reinterpret_cast<const float2*>(p.stat);
-    float2 pre[4];
+    // pass 2: the rows' offsets max + log2(sum) + log2(rows) of a unit (one subtraction then turns a raw score
+    // into its share of C), lane i holding rows i, i + 32, ...; loaded one item ahead
+    const float* stat_g = p.stat;
+    float pre[4];
     auto fetch_stats = [&](int k) {
       const Item nx = decode_item(a, k);
 #pragma unroll
       for (int q = 0; q < 4; ++q)
-        pre[q] = (nx.valid && q * 32 + lane < rows) ? stat_g[(size_t)(a.u0 + nx.lu) * p.rows_pad + q * 32 + lane]
-                                                    : make_float2(0.f, 0.f);
+        pre[q] = (nx.valid && q * 32 + lane < rows) ? stat_g[(size_t)(a.u0 + nx.lu) * (2 * p.rows_pad) + q * 32 + lane]
+                                                    : 0.f;
     };
     if (a.pass == 2) fetch_stats(0);
     for (int k = 0; k < a.steps && ok; ++k) {
@@ -497,24 +500,26 @@ window_tc_kernel(const __grid_constant__ CUtensorMap tmap_k, const __grid_consta
             tc_ld32(taddr + (uint32_t)c0, r);
             tc_wait_ld();
             if (!tail) {
-              const float4* st4 = reinterpret_cast<const float4*>(myStat + c0);   // two rows per 16-byte load
+              const float4* st4 = reinterpret_cast<const float4*>(myStat + c0);   // four rows per 16-byte load
 #pragma unroll
-              for (int c = 0; c < 32; c += 2) {
-                const float4 ms = st4[c >> 1];
-                cs[c & 3] = fmaf(ex2(fmaf(__uint_as_float(r[c]), scale2, -ms.x)), ms.y, cs[c & 3]);
-                cs[(c + 1) & 3] = fmaf(ex2(fmaf(__uint_as_float(r[c + 1]), scale2, -ms.z)), ms.w, cs[(c + 1) & 3]);
+              for (int c = 0; c < 32; c += 4) {
+                const float4 off = st4[c >> 2];
+                cs[0] += ex2(fmaf(__uint_as_float(r[c]), scale2, -off.x));
+                cs[1] += ex2(fmaf(__uint_as_float(r[c + 1]), scale2, -off.y));
+                cs[2] += ex2(fmaf(__uint_as_float(r[c + 2]), scale2, -off.z));
+                cs[3] += ex2(fmaf(__uint_as_float(r[c + 3]), scale2, -off.w));
               }
             } else {
 #pragma unroll
               for (int c = 0; c < 32; ++c) {
-                const float2 ms = myStat[c0 + c];
+                const float off = myStat[c0 + c];
                 const bool vis = (j < N) && (j <= N - L + ((c0 + c) % L));
-                if (vis) cs[c & 3] = fmaf(ex2(fmaf(__uint_as_float(r[c]), scale2, -ms.x)), ms.y, cs[c & 3]);
+                if (vis) cs[c & 3] += ex2(fmaf(__uint_as_float(r[c]), scale2, -off));
               }
             }
           }
           const float csum = (cs[0] + cs[1]) + (cs[2] + cs[3]);
-          if (j < N) p.C[p.c_off[u] + j] = csum * (1.0f / (float)rows);
+          if (j < N) p.C[p.c_off[u] + j] = csum;
         }
         tc_fence_before();
         __syncwarp();
@@ -549,7 +554,7 @@ window_tc_kernel(const __grid_constant__ CUtensorMap tmap_k, const __grid_consta
   if (tid == 0 && *s_abort) set_status(p.status, TASKKV_ETIMEOUT);
 }
 
-// Folds the partial statistics of one unit: slots (item, warp) of pass 1 -> (row max, 1 / row sum).
+// Folds the partial statistics of one unit: slots (item, warp) of pass 1 -> one offset per row.
 // One warp per (unit, row): lanes take every 32nd slot, then a shuffle tree; the order is fixed.
 __global__ void __launch_bounds__(128) window_tc_reduce_kernel(DeviceProblem p, int u0, int slots) {
   const int u = u0 + blockIdx.x;
@@ -574,9 +579,9 @@ __global__ void __launch_bounds__(128) window_tc_reduce_kernel(DeviceProblem p, 
       if (Mn > -INFINITY) z = z * exp2f(M - Mn) + z2 * exp2f(M2 - Mn);
       M = Mn;
     }
+    // one offset per row: score * scale - (max + log2(sum) + log2(rows)) is log2 of the row's share of C
     if (lane == 0)
-      reinterpret_cast<float2*>(p.stat)[(size_t)u * p.rows_pad + row] =
-          z > 0.f ? make_float2(M, 1.0f / z) : make_float2(0.f, 0.f);
+      p.stat[(size_t)u * (2 * p.rows_pad) + row] = z > 0.f ? M + log2f(z) + log2f((float)p.rows) : INFINITY;
   }
 }
 
