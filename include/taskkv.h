@@ -168,6 +168,19 @@ taskkv_status taskkv_append(taskkv_cache* c, const void* k_new, const void* v_ne
 taskkv_status taskkv_decode(const void* q, taskkv_cache* c, const int32_t* lengths, void* out,
                             taskkv_stream stream);
 
+/* The same two calls for layers [layer_begin, layer_begin + layer_count) of every
+ * sequence -- what a model's decode loop needs, since layer r's query exists only
+ * after layer r-1 has run (Eq. 1 is applied layer by layer).  k_new, v_new are
+ * [batch][layer_count][n_kv_heads][d], q and out [batch][layer_count][n_heads][d],
+ * lengths (optional) [batch][layer_count][n_kv_heads]; results are identical to the
+ * corresponding slices of the all-layer calls.  Calls on one cache share its
+ * split-K work buffers: issue them on one stream (or order them yourself).
+ * EINVAL if the range leaves [0, n_layers). */
+taskkv_status taskkv_append_ex(taskkv_cache* c, const void* k_new, const void* v_new,
+                               int32_t layer_begin, int32_t layer_count, taskkv_stream stream);
+taskkv_status taskkv_decode_ex(const void* q, taskkv_cache* c, const int32_t* lengths, void* out,
+                               int32_t layer_begin, int32_t layer_count, taskkv_stream stream);
+
 /* One decode step with HOST buffers: copies q, k_new, v_new in, appends,
  * attends and copies out back (k_new and v_new may both be NULL to skip the
  * append).  Synchronises the stream before returning. */

@@ -65,6 +65,10 @@ lib.taskkv_append.argtypes = [_vp, _vp, _vp, _vp]
 lib.taskkv_append.restype = C.c_int32
 lib.taskkv_decode.argtypes = [_vp, _vp, _vp, _vp, _vp]
 lib.taskkv_decode.restype = C.c_int32
+lib.taskkv_append_ex.argtypes = [_vp, _vp, _vp, C.c_int32, C.c_int32, _vp]
+lib.taskkv_append_ex.restype = C.c_int32
+lib.taskkv_decode_ex.argtypes = [_vp, _vp, _vp, _vp, C.c_int32, C.c_int32, _vp]
+lib.taskkv_decode_ex.restype = C.c_int32
 lib.taskkv_decode_host.argtypes = [_vp, _vp, _vp, _vp, _vp, _vp]
 lib.taskkv_decode_host.restype = C.c_int32
 lib.taskkv_decode_noalloc.argtypes = [_vp, _vp, _vp, _vp, _vp] + [C.c_int32] * 5 + [_vp, _vp]
@@ -223,6 +227,21 @@ class Cache:
         lp = lengths.data_ptr() if lengths is not None else None
         _check(lib.taskkv_decode(q.data_ptr(), self._h, lp, out.data_ptr(), _stream_handle(stream)),
                "taskkv_decode")
+        return out
+
+    def taskkv_append_ex(self, k_new: torch.Tensor, v_new: torch.Tensor, layer_begin: int, layer_count: int,
+                         stream=None) -> None:
+        _check(lib.taskkv_append_ex(self._h, k_new.data_ptr(), v_new.data_ptr(), layer_begin, layer_count,
+                                    _stream_handle(stream)), "taskkv_append_ex")
+
+    def taskkv_decode_ex(self, q: torch.Tensor, layer_begin: int, layer_count: int,
+                         out: Optional[torch.Tensor] = None, lengths: Optional[torch.Tensor] = None,
+                         stream=None) -> torch.Tensor:
+        if out is None:
+            out = torch.empty_like(q)
+        lp = lengths.data_ptr() if lengths is not None else None
+        _check(lib.taskkv_decode_ex(q.data_ptr(), self._h, lp, out.data_ptr(), layer_begin, layer_count,
+                                    _stream_handle(stream)), "taskkv_decode_ex")
         return out
 
     def taskkv_decode_host(self, q: torch.Tensor, k_new: Optional[torch.Tensor], v_new: Optional[torch.Tensor],

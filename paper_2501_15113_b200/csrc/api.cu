@@ -238,6 +238,9 @@ void fill_device_problem(taskkv_cache* c) {
   d.promote_center = p.promote_center;
   d.force_class = p.force_class;
   d.mid_policy = p.mid_policy;
+  d.view_l0 = 0;
+  d.view_nl = p.n_layers;
+  d.view_U = (int32_t)hp.info.n_units;
   d.max_mid = 0;
   for (int32_t m : hp.mid) d.max_mid = m > d.max_mid ? m : d.max_mid;
   if (d.max_mid > hp.max_N) d.max_mid = hp.max_N;
@@ -487,15 +490,43 @@ taskkv_status taskkv_compress_host(const taskkv_params* p, const void* const* q_
   return st;
 }
 
-taskkv_status taskkv_append(taskkv_cache* c, const void* k_new, const void* v_new, taskkv_stream stream) {
+namespace {
+// The cache's problem description restricted to layers [layer_begin, layer_begin + layer_count) of every sequence.
+bool layer_view(const taskkv_cache* c, int32_t layer_begin, int32_t layer_count, taskkv::DeviceProblem* out) {
+  if (layer_begin < 0 || layer_count < 1 || layer_begin + layer_count > c->dp.R) return false;
+  *out = c->dp;
+  out->view_l0 = layer_begin;
+  out->view_nl = layer_count;
+  out->view_U = c->prm.batch * layer_count * c->dp.n_kv;
+  return true;
+}
+}  // namespace
+
+taskkv_status taskkv_append_ex(taskkv_cache* c, const void* k_new, const void* v_new, int32_t layer_begin,
+                               int32_t layer_count, taskkv_stream stream) {
   if (!c || !k_new || !v_new || (((uintptr_t)k_new | (uintptr_t)v_new) & 15)) return TASKKV_EINVAL;
-  return cuda_status(launch_append(c->dp, c->prm.dtype, k_new, v_new, static_cast<cudaStream_t>(stream)));
+  taskkv::DeviceProblem view;
+  if (!layer_view(c, layer_begin, layer_count, &view)) return TASKKV_EINVAL;
+  return cuda_status(launch_append(view, c->prm.dtype, k_new, v_new, static_cast<cudaStream_t>(stream)));
+}
+
+taskkv_status taskkv_append(taskkv_cache* c, const void* k_new, const void* v_new, taskkv_stream stream) {
+  if (!c) return TASKKV_EINVAL;
+  return taskkv_append_ex(c, k_new, v_new, 0, c->dp.R, stream);
+}
+
+taskkv_status taskkv_decode_ex(const void* q, taskkv_cache* c, const int32_t* lengths, void* out,
+                               int32_t layer_begin, int32_t layer_count, taskkv_stream stream) {
+  if (!c || !q || !out || (((uintptr_t)q | (uintptr_t)out) & 15)) return TASKKV_EINVAL;
+  taskkv::DeviceProblem view;
+  if (!layer_view(c, layer_begin, layer_count, &view)) return TASKKV_EINVAL;
+  return cuda_status(launch_decode(view, c->prm.dtype, q, lengths, out, static_cast<cudaStream_t>(stream)));
 }
 
 taskkv_status taskkv_decode(const void* q, taskkv_cache* c, const int32_t* lengths, void* out,
                             taskkv_stream stream) {
-  if (!c || !q || !out || (((uintptr_t)q | (uintptr_t)out) & 15)) return TASKKV_EINVAL;
-  return cuda_status(launch_decode(c->dp, c->prm.dtype, q, lengths, out, static_cast<cudaStream_t>(stream)));
+  if (!c) return TASKKV_EINVAL;
+  return taskkv_decode_ex(q, c, lengths, out, 0, c->dp.R, stream);
 }
 
 taskkv_status taskkv_decode_host(const void* q, const void* k_new, const void* v_new, taskkv_cache* c,

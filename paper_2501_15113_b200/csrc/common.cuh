@@ -48,6 +48,9 @@ struct DeviceProblem {
   int32_t promote_center, force_class;
   int32_t mid_policy;   // TASKKV_MID_*
   int32_t max_mid;      // largest middle budget of any layer
+  // Append and decode address a range of layers of every sequence ("view"): view unit v = (b * view_nl + r') *
+  // n_kv + h stands for layer view_l0 + r'.  q, k_new, v_new, out and `lengths` are indexed by view unit.
+  int32_t view_l0, view_nl, view_U;
   int32_t max_new;
   int32_t idx_stride;   // ints per unit in idx
   int32_t chunks_max;   // partial-statistic slots per unit (longest sequence)
@@ -124,6 +127,13 @@ cudaError_t launch_decode(const DeviceProblem& p, int dtype, const void* q, cons
 __device__ __forceinline__ float to_float(float x) { return x; }
 __device__ __forceinline__ float to_float(__nv_bfloat16 x) { return __bfloat162float(x); }
 
+// Unit behind view unit v (identity when the view covers every layer).
+__device__ __forceinline__ int view_unit(const DeviceProblem& p, int v) {
+  if (p.view_nl == p.R) return v;
+  const int per = p.view_nl * p.n_kv;
+  const int b = v / per;
+  return (b * p.R + p.view_l0) * p.n_kv + (v - b * per);
+}
 __device__ __forceinline__ void store_out(float* p, float x) { *p = x; }
 __device__ __forceinline__ void store_out(__nv_bfloat16* p, float x) { *p = __float2bfloat16_rn(x); }
 

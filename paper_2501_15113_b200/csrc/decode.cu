@@ -35,17 +35,18 @@ __global__ void __launch_bounds__(kAttnThreads) decode_attn_kernel(DeviceProblem
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
   const int sg = lane / LPR, sl = lane % LPR;
   const int gsg = warp * RPW + sg;
-  const int total = p.dec_off[p.U];
+  const int total = p.dec_off[p.view_U];
   const float scale2 = kLog2e * rsqrtf((float)D);
 
   for (int item = blockIdx.x; item < total; item += gridDim.x) {
     __syncthreads();                                // previous item's shared state consumed
-    if (tid == 0) s_unit = upper_unit(p.dec_off, p.U, item);
+    if (tid == 0) s_unit = upper_unit(p.dec_off, p.view_U, item);
     __syncthreads();
-    const int u = s_unit;
+    const int vu = s_unit;                          // view unit: index into q, lengths, the work-item table
+    const int u = view_unit(p, vu);                 // unit: index into the cache
     int len = p.len[u];
-    if (lengths) len = min(max(lengths[u], 0), len);
-    const int rbeg = (item - p.dec_off[u]) * kDecodeChunk;
+    if (lengths) len = min(max(lengths[vu], 0), len);
+    const int rbeg = (item - p.dec_off[vu]) * kDecodeChunk;
     const int rend = min(len, rbeg + kDecodeChunk);
     const int64_t seg = p.seg_off[u];
     const unsigned char* kp = static_cast<const unsigned char*>(p.k_pool) + (size_t)seg * ROW_BYTES + sl * 16;
@@ -54,7 +55,7 @@ __global__ void __launch_bounds__(kAttnThreads) decode_attn_kernel(DeviceProblem
     float qf[G][EPL];
 #pragma unroll
     for (int g = 0; g < G; ++g) {
-      const uint4 raw = *reinterpret_cast<const uint4*>(q + ((size_t)u * G + g) * D + sl * EPL);
+      const uint4 raw = *reinterpret_cast<const uint4*>(q + ((size_t)vu * G + g) * D + sl * EPL);
       Vec16<T>::unpack(raw, qf[g]);
 #pragma unroll
       for (int e = 0; e < EPL; ++e) qf[g][e] *= scale2;
@@ -215,19 +216,20 @@ __global__ void __launch_bounds__(kAttnThreads) decode_attn_mma_kernel(DevicePro
 
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
   const int g = lane >> 2, t = lane & 3;
-  const int total = p.dec_off[p.U];
+  const int total = p.dec_off[p.view_U];
   const float scale2 = kLog2e * rsqrtf((float)D);
   // d of accumulator row (mb, hf) of this lane's two output rows: e = hf * MB + mb, piece e / 8, element e % 8
   auto pd = [&](int mb, int hf, int gg) { const int e = hf * MB + mb; return (e >> 3) * 64 + gg * 8 + (e & 7); };
 
   for (int item = blockIdx.x; item < total; item += gridDim.x) {
     __syncthreads();
-    if (tid == 0) s_unit = upper_unit(p.dec_off, p.U, item);
+    if (tid == 0) s_unit = upper_unit(p.dec_off, p.view_U, item);
     __syncthreads();
-    const int u = s_unit;
+    const int vu = s_unit;                          // view unit: index into q, lengths, the work-item table
+    const int u = view_unit(p, vu);                 // unit: index into the cache
     int len = p.len[u];
-    if (lengths) len = min(max(lengths[u], 0), len);
-    const int rbeg = (item - p.dec_off[u]) * kDecodeChunk;
+    if (lengths) len = min(max(lengths[vu], 0), len);
+    const int rbeg = (item - p.dec_off[vu]) * kDecodeChunk;
     const int rend = min(len, rbeg + kDecodeChunk);
     const int64_t seg = p.seg_off[u];
     const unsigned char* kp = static_cast<const unsigned char*>(p.k_pool) + (size_t)seg * ROW_BYTES;
@@ -238,7 +240,7 @@ __global__ void __launch_bounds__(kAttnThreads) decode_attn_mma_kernel(DevicePro
 #pragma unroll
     for (int i = 0; i < KP; ++i) {
       uint4 raw = make_uint4(0, 0, 0, 0);
-      if (g < G) raw = *reinterpret_cast<const uint4*>(q + ((size_t)u * G + g) * D + (i * 4 + t) * 8);
+      if (g < G) raw = *reinterpret_cast<const uint4*>(q + ((size_t)vu * G + g) * D + (i * 4 + t) * 8);
       qa[2 * i][0] = raw.x; qa[2 * i][1] = raw.y;
       qa[2 * i + 1][0] = raw.z; qa[2 * i + 1][1] = raw.w;
     }
@@ -358,7 +360,7 @@ __global__ void __launch_bounds__(kAttnThreads) decode_attn_mma_kernel(DevicePro
   }
 }
 
-// One block per (unit, query head of the group): merge the unit's partials.  First the block finds
+// One block per (view unit, query head of the group): merge the unit's partials.  First the block finds
 // the largest running maximum, then each warp accumulates every fourth partial against it (independent
 // loads, fixed order), and the four warps are summed in shared memory.
 template <typename T, int D, int G>
@@ -416,7 +418,7 @@ cudaError_t launch_typed(const DeviceProblem& p, const void* q, const int32_t* l
   }
   {
     LaunchScope ls(K_DECODE_COMBINE, s);
-    decode_combine_kernel<T, D, G><<<(unsigned)(p.U * G), kAttnThreads, 0, s>>>(p, static_cast<T*>(out));
+    decode_combine_kernel<T, D, G><<<(unsigned)(p.view_U * G), kAttnThreads, 0, s>>>(p, static_cast<T*>(out));
   }
   return cudaGetLastError();
 }

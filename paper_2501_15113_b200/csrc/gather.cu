@@ -61,16 +61,17 @@ template <int ROW_BYTES>
 __global__ void __launch_bounds__(256) append_kernel(DeviceProblem p, const unsigned char* k_new,
                                                      const unsigned char* v_new) {
   constexpr int VPR = ROW_BYTES / 16;
-  const int u = blockIdx.x * 8 + (threadIdx.x >> 5);
+  const int vu = blockIdx.x * 8 + (threadIdx.x >> 5);   // view unit: index into k_new, v_new
   const int lane = threadIdx.x & 31;
-  if (u >= p.U) return;
+  if (vu >= p.view_U) return;
+  const int u = view_unit(p, vu);
   const int len = p.len[u];
   const int64_t seg = p.seg_off[u];
   const bool ok = len < p.cap[u] && seg + len < p.pool_rows;
   __syncwarp();
   if (ok && lane < VPR) {
     const size_t dst = ((size_t)seg + len) * ROW_BYTES + lane * 16;
-    const size_t src = (size_t)u * ROW_BYTES + lane * 16;
+    const size_t src = (size_t)vu * ROW_BYTES + lane * 16;
     *reinterpret_cast<uint4*>(static_cast<unsigned char*>(p.k_pool) + dst) =
         *reinterpret_cast<const uint4*>(k_new + src);
     *reinterpret_cast<uint4*>(static_cast<unsigned char*>(p.v_pool) + dst) =
@@ -168,7 +169,7 @@ cudaError_t launch_append(const DeviceProblem& p, int dtype, const void* k_new, 
                           cudaStream_t s) {
   LaunchScope ls(K_APPEND, s);
   const int row_bytes = p.d * (dtype == TASKKV_F32 ? 4 : 2);
-  const unsigned grid = (unsigned)((p.U + 7) / 8);
+  const unsigned grid = (unsigned)((p.view_U + 7) / 8);
   const unsigned char* kn = static_cast<const unsigned char*>(k_new);
   const unsigned char* vn = static_cast<const unsigned char*>(v_new);
   switch (row_bytes) {

@@ -137,19 +137,20 @@ __global__ void __launch_bounds__(kPlanThreads) decode_plan_kernel(DeviceProblem
   __shared__ int64_t total;
   int64_t run = 0;
   const int tid = threadIdx.x;
-  for (int base = 0; base < p.U; base += kPlanThreads) {
-    const int u = base + tid;
+  for (int base = 0; base < p.view_U; base += kPlanThreads) {
+    const int v = base + tid;
     int items = 0;
-    if (u < p.U) {
-      const int len = lengths ? min(max(lengths[u], 0), p.len[u]) : p.len[u];
+    if (v < p.view_U) {
+      const int own = p.len[view_unit(p, v)];
+      const int len = lengths ? min(max(lengths[v], 0), own) : own;
       items = (len + kDecodeChunk - 1) / kDecodeChunk;
     }
     const int64_t o = block_excl_scan(items, warp_tot, &total);
-    if (u < p.U) p.dec_off[u] = (int32_t)(run + o);
+    if (v < p.view_U) p.dec_off[v] = (int32_t)(run + o);
     run += total;
   }
   if (tid == 0) {
-    p.dec_off[p.U] = (int32_t)min(run, p.max_items);
+    p.dec_off[p.view_U] = (int32_t)min(run, p.max_items);
     if (run > p.max_items) set_status(p.status, TASKKV_ESTATE);
   }
 }

@@ -335,3 +335,51 @@ def test_compensation_policies(case, policy):
                 worst = max(worst, float(np.abs(P.to64(out[b, r]) - want).max()))
     assert worst < P.TOL_OUT[wl.dtype], f"decode max abs err {worst:.3e}"
     cache.close()
+
+
+# ---------------------------------------------------------------------------
+# Layer-range append / decode: what a model's decode loop calls, layer after layer
+# ---------------------------------------------------------------------------
+@pytest.mark.parametrize("case", [
+    dict(n=8, n_kv=4, d=128, N=0, L=32, s1=4, s2=64, k=100, dtype="bf16", R=4, seq_lens=[1500, 2049, 777], nh=1),
+    dict(n=4, n_kv=4, d=64, N=900, L=16, s1=4, s2=32, k=50, dtype="f32", R=3),
+], ids=["bf16_gqa_ragged", "f32"])
+def test_layer_by_layer_decode_equals_all_layer_decode(case):
+    tk = _tk()
+    wl = small("layers", **case, steps=3)
+    qs, ks, vs = W.materialize(wl, DEV)
+    steps = wl.decode_steps
+    params = tk.params_from_workload(wl, max_new_tokens=steps)
+    whole = tk.taskkv_compress_ex(params, qs, ks, vs)
+    split = tk.taskkv_compress_ex(params, qs, ks, vs)
+    R = wl.n_layers
+    for s in range(steps):
+        q, kn, vn = W.gen_decode_step(wl, s, DEV)             # [B][R][heads][d]
+        whole.taskkv_append(kn, vn)
+        want = whole.taskkv_decode(q)
+        got = torch.empty_like(want)
+        # one layer at a time, then a range of two layers starting at 1 must reproduce the same slices
+        for r in range(R):
+            split.taskkv_append_ex(kn[:, r:r + 1].contiguous(), vn[:, r:r + 1].contiguous(), r, 1)
+            got[:, r:r + 1] = split.taskkv_decode_ex(q[:, r:r + 1].contiguous(), r, 1)
+        assert torch.equal(got.view(torch.uint8), want.view(torch.uint8)), f"step {s}: per-layer outputs differ"
+        pair = split.taskkv_decode_ex(q[:, 1:3].contiguous(), 1, 2)
+        assert torch.equal(pair.view(torch.uint8), want[:, 1:3].contiguous().view(torch.uint8))
+    assert whole.status() == 0 and split.status() == 0
+    assert np.array_equal(whole.lengths(), split.lengths())
+    # a prefix-length override is indexed like q: [B][layers in the call][n_kv]
+    lens = torch.from_numpy(split.lengths().reshape(wl.batch, R, wl.n_kv_heads)).to(DEV)
+    half = (lens[:, 2:3] // 2).to(torch.int32).contiguous()
+    full_half = lens.clone().to(torch.int32)
+    full_half[:, 2:3] = half
+    q, _, _ = W.gen_decode_step(wl, 0, DEV)
+    a = split.taskkv_decode_ex(q[:, 2:3].contiguous(), 2, 1, lengths=half)
+    b = whole.taskkv_decode(q, lengths=full_half.contiguous())[:, 2:3].contiguous()
+    assert torch.equal(a.view(torch.uint8), b.view(torch.uint8))
+    # out-of-range layers are refused before anything is launched
+    with pytest.raises(tk.TaskKVError):
+        split.taskkv_decode_ex(q[:, 0:1].contiguous(), R, 1)
+    with pytest.raises(tk.TaskKVError):
+        split.taskkv_append_ex(q[:, 0:1].contiguous(), q[:, 0:1].contiguous(), R - 1, 2)
+    whole.close()
+    split.close()
