@@ -262,6 +262,8 @@ def run_ours(args):
         "gpu_launches": launches, "device_status": status, "clocks": clocks,
     }
 
+    if rank == 0 and not args.no_latency:
+        line["latency_mode"] = run_latency_mode(tk, wl, qs, ks, vs, steps_in, args)
     if rank == 0 and not args.no_e2e:
         line["e2e"] = run_e2e(tk, wl, params, qs, ks, vs, steps_in, world)
     if rank == 0 and world == 1 and not args.no_cpu and args.policy != "select":
@@ -274,6 +276,53 @@ def run_ours(args):
         import torch.distributed as dist
         dist.barrier()
         dist.destroy_process_group()
+
+
+def run_latency_mode(tk, wl, qs, ks, vs, steps_in, args, n_steps=16):
+    """Decode as a model runs it: one append + attention call per layer (layer r's query depends on layer r-1),
+    n_steps tokens; first as plain launches, then with one token's 4 x n_layers launches replayed from a CUDA graph."""
+    import torch
+    R = wl.n_layers
+    params = tk.params_from_workload(wl, max_new_tokens=3 * n_steps + 4, mid_policy=POLICIES[args.policy])
+    cache = tk.taskkv_compress_ex(params, qs, ks, vs)
+    q, kn, vn = steps_in[0]
+    ql = [q[:, r:r + 1].contiguous() for r in range(R)]
+    kl = [kn[:, r:r + 1].contiguous() for r in range(R)]
+    vl = [vn[:, r:r + 1].contiguous() for r in range(R)]
+    ol = [torch.empty_like(x) for x in ql]
+    stream = torch.cuda.current_stream()
+
+    def token():
+        for r in range(R):
+            cache.taskkv_append_ex(kl[r], vl[r], r, 1)
+            cache.taskkv_decode_ex(ql[r], r, 1, out=ol[r])
+
+    def timed(fn, n):
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        torch.cuda.synchronize()
+        e0.record(stream)
+        for _ in range(n):
+            fn()
+        e1.record(stream)
+        torch.cuda.synchronize()
+        return e0.elapsed_time(e1) / n
+
+    for _ in range(3):
+        token()
+    eager_ms = timed(token, n_steps)
+    out = {"layers_per_token": R, "launches_per_token": 4 * R, "tokens_timed": n_steps,
+           "eager_ms_per_token": eager_ms, "graph_ms_per_token": None}
+    try:
+        g = torch.cuda.CUDAGraph()
+        with torch.cuda.graph(g):
+            token()
+        g.replay()
+        out["graph_ms_per_token"] = timed(g.replay, n_steps)
+    except Exception as exc:      # capture is an optimisation of the launch path only
+        out["graph_error"] = str(exc)[:200]
+    out["device_status"] = cache.status()
+    cache.close()
+    return out
 
 
 def ncu_traffic(wl, retained_rows):
@@ -424,6 +473,7 @@ def main():
     ap.add_argument("--decode-steps", type=int, default=0)
     ap.add_argument("--policy", default="select", choices=sorted(POLICIES),
                     help="what a non-heterogeneous head keeps beside sinks and recent window (Sec. V-G)")
+    ap.add_argument("--no-latency", action="store_true", help="skip the layer-by-layer decode measurement")
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--no-cpu", action="store_true")
     args = ap.parse_args()

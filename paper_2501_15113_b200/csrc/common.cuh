@@ -27,7 +27,6 @@ enum KernelId : int32_t {
   K_PLAN,
   K_GATHER,
   K_APPEND,
-  K_DECODE_PLAN,
   K_DECODE_ATTN,
   K_DECODE_COMBINE,
   K_WINDOW_TC,
@@ -113,7 +112,6 @@ bool window_tc_supported(const DeviceProblem& p, int dtype);
 cudaError_t launch_window_scores_tc(const DeviceProblem& p, const WindowHostInfo& h, cudaStream_t s);
 cudaError_t launch_select(const DeviceProblem& p, int dtype, int max_N, cudaStream_t s);
 cudaError_t launch_separator_plan(const DeviceProblem& p, int n_br, cudaStream_t s);
-cudaError_t launch_decode_plan(const DeviceProblem& p, const int32_t* lengths, cudaStream_t s);
 cudaError_t launch_gather(const DeviceProblem& p, int dtype, int64_t gather_items, cudaStream_t s);
 cudaError_t launch_compensate(const DeviceProblem& p, int dtype, cudaStream_t s);
 cudaError_t launch_append(const DeviceProblem& p, int dtype, const void* k_new, const void* v_new,
@@ -133,6 +131,24 @@ __device__ __forceinline__ int view_unit(const DeviceProblem& p, int v) {
   const int per = p.view_nl * p.n_kv;
   const int b = v / per;
   return (b * p.R + p.view_l0) * p.n_kv + (v - b * per);
+}
+// The split-K decode work items are numbered once, at compression, for every unit at its capacity and in
+// layer-major order w = (r * batch + b) * n_kv + h: a range of layers is then a contiguous range of items,
+// and a decode call needs no planning pass (an item whose rows lie beyond the segment's length is skipped).
+__device__ __forceinline__ int lm_batch(const DeviceProblem& p) { return p.U / (p.R * p.n_kv); }
+__device__ __forceinline__ int lm_index(const DeviceProblem& p, int u) {      // unit -> layer-major index
+  const int h = u % p.n_kv, br = u / p.n_kv;
+  return ((br % p.R) * lm_batch(p) + br / p.R) * p.n_kv + h;
+}
+struct LmUnit { int u, v; };                                                 // unit and view unit
+__device__ __forceinline__ LmUnit lm_unit(const DeviceProblem& p, int w) {   // layer-major index -> unit, view unit
+  const int B = lm_batch(p);
+  const int h = w % p.n_kv, rb = w / p.n_kv;
+  const int r = rb / B, b = rb % B;
+  LmUnit x;
+  x.u = (b * p.R + r) * p.n_kv + h;
+  x.v = (b * p.view_nl + (r - p.view_l0)) * p.n_kv + h;
+  return x;
 }
 __device__ __forceinline__ void store_out(float* p, float x) { *p = x; }
 __device__ __forceinline__ void store_out(__nv_bfloat16* p, float x) { *p = __float2bfloat16_rn(x); }

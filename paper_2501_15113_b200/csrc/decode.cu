@@ -2,9 +2,9 @@
 // head, no mask): o_a = softmax(q_a K_u^T / sqrt(d)) V_u over the len_u rows of
 // the KV head's segment, for the G query heads that share it.
 //
-// Split-K: a unit's rows are cut into work items of kDecodeChunk (512) rows, numbered
-// by an exclusive scan over the units (so a 32768-row full head and a 772-row
-// pruned head load the SMs alike).  Each item produces an un-normalised partial
+// Split-K: a unit's rows are cut into work items of kDecodeChunk (512) rows, numbered once at
+// compression for every unit at its capacity (so a 32768-row full head and a 772-row pruned head
+// load the SMs alike; items beyond a segment's current length are skipped).  Each item produces an un-normalised partial
 // (running max, sum, weighted V) per head with an online softmax in fp32; one
 // combine pass merges a unit's partials.  K/V rows are read once, as 16-byte
 // vectors, by all G heads.
@@ -35,18 +35,23 @@ __global__ void __launch_bounds__(kAttnThreads) decode_attn_kernel(DeviceProblem
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
   const int sg = lane / LPR, sl = lane % LPR;
   const int gsg = warp * RPW + sg;
-  const int total = p.dec_off[p.view_U];
+  // the view's layers are a contiguous range of layer-major indices, hence of work items
+  const int w0 = p.view_l0 * lm_batch(p) * p.n_kv, w1 = w0 + p.view_U;
+  const int item0 = p.dec_off[w0], item1 = p.dec_off[w1];
   const float scale2 = kLog2e * rsqrtf((float)D);
 
-  for (int item = blockIdx.x; item < total; item += gridDim.x) {
+  for (int item = item0 + blockIdx.x; item < item1; item += gridDim.x) {
     __syncthreads();                                // previous item's shared state consumed
-    if (tid == 0) s_unit = upper_unit(p.dec_off, p.view_U, item);
+    if (tid == 0) s_unit = w0 + upper_unit(p.dec_off + w0, p.view_U, item);
     __syncthreads();
-    const int vu = s_unit;                          // view unit: index into q, lengths, the work-item table
-    const int u = view_unit(p, vu);                 // unit: index into the cache
+    const int w = s_unit;
+    const LmUnit lu = lm_unit(p, w);
+    const int vu = lu.v;                            // view unit: index into q and lengths
+    const int u = lu.u;                             // unit: index into the cache
     int len = p.len[u];
     if (lengths) len = min(max(lengths[vu], 0), len);
-    const int rbeg = (item - p.dec_off[vu]) * kDecodeChunk;
+    const int rbeg = (item - p.dec_off[w]) * kDecodeChunk;
+    if (rbeg >= len) continue;                      // an item of the reserve beyond the segment's length
     const int rend = min(len, rbeg + kDecodeChunk);
     const int64_t seg = p.seg_off[u];
     const unsigned char* kp = static_cast<const unsigned char*>(p.k_pool) + (size_t)seg * ROW_BYTES + sl * 16;
@@ -216,20 +221,25 @@ __global__ void __launch_bounds__(kAttnThreads) decode_attn_mma_kernel(DevicePro
 
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
   const int g = lane >> 2, t = lane & 3;
-  const int total = p.dec_off[p.view_U];
+  // the view's layers are a contiguous range of layer-major indices, hence of work items
+  const int w0 = p.view_l0 * lm_batch(p) * p.n_kv, w1 = w0 + p.view_U;
+  const int item0 = p.dec_off[w0], item1 = p.dec_off[w1];
   const float scale2 = kLog2e * rsqrtf((float)D);
   // d of accumulator row (mb, hf) of this lane's two output rows: e = hf * MB + mb, piece e / 8, element e % 8
   auto pd = [&](int mb, int hf, int gg) { const int e = hf * MB + mb; return (e >> 3) * 64 + gg * 8 + (e & 7); };
 
-  for (int item = blockIdx.x; item < total; item += gridDim.x) {
+  for (int item = item0 + blockIdx.x; item < item1; item += gridDim.x) {
     __syncthreads();
-    if (tid == 0) s_unit = upper_unit(p.dec_off, p.view_U, item);
+    if (tid == 0) s_unit = w0 + upper_unit(p.dec_off + w0, p.view_U, item);
     __syncthreads();
-    const int vu = s_unit;                          // view unit: index into q, lengths, the work-item table
-    const int u = view_unit(p, vu);                 // unit: index into the cache
+    const int w = s_unit;
+    const LmUnit lu = lm_unit(p, w);
+    const int vu = lu.v;                            // view unit: index into q and lengths
+    const int u = lu.u;                             // unit: index into the cache
     int len = p.len[u];
     if (lengths) len = min(max(lengths[vu], 0), len);
-    const int rbeg = (item - p.dec_off[vu]) * kDecodeChunk;
+    const int rbeg = (item - p.dec_off[w]) * kDecodeChunk;
+    if (rbeg >= len) continue;                      // an item of the reserve beyond the segment's length
     const int rend = min(len, rbeg + kDecodeChunk);
     const int64_t seg = p.seg_off[u];
     const unsigned char* kp = static_cast<const unsigned char*>(p.k_pool) + (size_t)seg * ROW_BYTES;
@@ -364,14 +374,19 @@ __global__ void __launch_bounds__(kAttnThreads) decode_attn_mma_kernel(DevicePro
 // the largest running maximum, then each warp accumulates every fourth partial against it (independent
 // loads, fixed order), and the four warps are summed in shared memory.
 template <typename T, int D, int G>
-__global__ void __launch_bounds__(kAttnThreads) decode_combine_kernel(DeviceProblem p, T* __restrict__ out) {
+__global__ void __launch_bounds__(kAttnThreads) decode_combine_kernel(DeviceProblem p, const int32_t* __restrict__ lengths,
+                                                                      T* __restrict__ out) {
   constexpr int EPL = D / 32;
   __shared__ float s_max[kAttnWarps];
   __shared__ float s_l[kAttnWarps];
   __shared__ float s_acc[kAttnWarps][D];
-  const int u = blockIdx.x / G, g = blockIdx.x % G;
+  const int u = blockIdx.x / G, g = blockIdx.x % G;     // u: view unit
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
-  const int i0 = p.dec_off[u], i1 = p.dec_off[u + 1];
+  const int unit = view_unit(p, u);
+  int len = p.len[unit];
+  if (lengths) len = min(max(lengths[u], 0), len);
+  // the unit's items that hold rows (the table also numbers the reserve for appended tokens)
+  const int i0 = p.dec_off[lm_index(p, unit)], i1 = i0 + (len + kDecodeChunk - 1) / kDecodeChunk;
   float M = -INFINITY;
   for (int i = i0 + tid; i < i1; i += kAttnThreads) M = fmaxf(M, p.part_ml[((size_t)i * G + g) * 2]);
   M = warp_max(M);
@@ -418,7 +433,7 @@ cudaError_t launch_typed(const DeviceProblem& p, const void* q, const int32_t* l
   }
   {
     LaunchScope ls(K_DECODE_COMBINE, s);
-    decode_combine_kernel<T, D, G><<<(unsigned)(p.view_U * G), kAttnThreads, 0, s>>>(p, static_cast<T*>(out));
+    decode_combine_kernel<T, D, G><<<(unsigned)(p.view_U * G), kAttnThreads, 0, s>>>(p, lengths, static_cast<T*>(out));
   }
   return cudaGetLastError();
 }
@@ -439,8 +454,6 @@ cudaError_t launch_group(const DeviceProblem& p, const void* q, const int32_t* l
 
 cudaError_t launch_decode(const DeviceProblem& p, int dtype, const void* q, const int32_t* lengths, void* out,
                           cudaStream_t s) {
-  cudaError_t e = launch_decode_plan(p, lengths, s);
-  if (e != cudaSuccess) return e;
   if (dtype == TASKKV_F32)
     return p.d == 64 ? launch_group<float, 64>(p, q, lengths, out, s) : launch_group<float, 128>(p, q, lengths, out, s);
   return p.d == 64 ? launch_group<__nv_bfloat16, 64>(p, q, lengths, out, s)

@@ -129,29 +129,19 @@ __global__ void __launch_bounds__(kPlanThreads) plan_kernel(DeviceProblem p) {
     p.gather_off[p.U] = (int32_t)run_gather;
     if (run_rows > p.pool_rows) set_status(p.status, TASKKV_ESTATE);
   }
-}
-
-// Numbers the split-K decode work items: ceil(len_u / kDecodeChunk) per unit.
-__global__ void __launch_bounds__(kPlanThreads) decode_plan_kernel(DeviceProblem p, const int32_t* lengths) {
-  __shared__ int64_t warp_tot[32];
-  __shared__ int64_t total;
-  int64_t run = 0;
-  const int tid = threadIdx.x;
-  for (int base = 0; base < p.view_U; base += kPlanThreads) {
-    const int v = base + tid;
-    int items = 0;
-    if (v < p.view_U) {
-      const int own = p.len[view_unit(p, v)];
-      const int len = lengths ? min(max(lengths[v], 0), own) : own;
-      items = (len + kDecodeChunk - 1) / kDecodeChunk;
-    }
+  // decode work items: ceil(capacity / kDecodeChunk) per unit, numbered in layer-major order
+  __syncthreads();
+  int64_t run_items = 0;
+  for (int base = 0; base < p.U; base += kPlanThreads) {
+    const int w = base + tid;
+    const int items = (w < p.U) ? (p.cap[lm_unit(p, w).u] + kDecodeChunk - 1) / kDecodeChunk : 0;
     const int64_t o = block_excl_scan(items, warp_tot, &total);
-    if (v < p.view_U) p.dec_off[v] = (int32_t)(run + o);
-    run += total;
+    if (w < p.U) p.dec_off[w] = (int32_t)(run_items + o);
+    run_items += total;
   }
   if (tid == 0) {
-    p.dec_off[p.view_U] = (int32_t)min(run, p.max_items);
-    if (run > p.max_items) set_status(p.status, TASKKV_ESTATE);
+    p.dec_off[p.U] = (int32_t)min(run_items, p.max_items);
+    if (run_items > p.max_items) set_status(p.status, TASKKV_ESTATE);
   }
 }
 
@@ -166,12 +156,6 @@ cudaError_t launch_separator_plan(const DeviceProblem& p, int n_br, cudaStream_t
     LaunchScope ls(K_PLAN, s);
     plan_kernel<<<1, kPlanThreads, 0, s>>>(p);
   }
-  return cudaGetLastError();
-}
-
-cudaError_t launch_decode_plan(const DeviceProblem& p, const int32_t* lengths, cudaStream_t s) {
-  LaunchScope ls(K_DECODE_PLAN, s);
-  decode_plan_kernel<<<1, kPlanThreads, 0, s>>>(p, lengths);
   return cudaGetLastError();
 }
 
