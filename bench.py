@@ -264,6 +264,7 @@ def run_ours(args):
 
     if rank == 0 and not args.no_latency:
         line["latency_mode"] = run_latency_mode(tk, wl, qs, ks, vs, steps_in, args)
+        line["layer_streamed_compress"] = run_layer_streamed(tk, wl, qs, ks, vs, args)
     if rank == 0 and not args.no_e2e:
         line["e2e"] = run_e2e(tk, wl, params, qs, ks, vs, steps_in, world)
     if rank == 0 and world == 1 and not args.no_cpu and args.policy != "select":
@@ -323,6 +324,38 @@ def run_latency_mode(tk, wl, qs, ks, vs, steps_in, args, n_steps=16):
     out["device_status"] = cache.status()
     cache.close()
     return out
+
+
+def run_layer_streamed(tk, wl, qs, ks, vs, args):
+    """Compression as a prefill loop would issue it: one call per layer, each as soon as that layer's K and V
+    exist (here: back to back), every layer a one-layer problem with its own cache memory."""
+    import torch
+    params = tk.params_from_workload(wl, max_new_tokens=4, mid_policy=POLICIES[args.policy])
+    R = wl.n_layers
+    lp = [params.layer(r) for r in range(R)]
+    infos = [tk.taskkv_plan(x) for x in lp]
+    cmem = [torch.empty(int(i.cache_bytes), dtype=torch.uint8, device=qs[0].device) for i in infos]
+    wmem = torch.empty(max(int(i.workspace_bytes) for i in infos), dtype=torch.uint8, device=qs[0].device)
+    ins = [([x[r:r + 1] for x in qs], [x[r:r + 1] for x in ks], [x[r:r + 1] for x in vs]) for r in range(R)]
+    stream = torch.cuda.current_stream()
+
+    def all_layers():
+        caches = [tk.taskkv_compress_ex(lp[r], *ins[r], cache_mem=cmem[r], workspace_mem=wmem) for r in range(R)]
+        return caches
+
+    for c in all_layers():
+        c.close()
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    torch.cuda.synchronize()
+    e0.record(stream)
+    caches = all_layers()
+    e1.record(stream)
+    torch.cuda.synchronize()
+    status = max(c.status() for c in caches)
+    for c in caches:
+        c.close()
+    return {"calls": R, "total_ms": e0.elapsed_time(e1), "ms_per_layer": e0.elapsed_time(e1) / R,
+            "device_status": status}
 
 
 def ncu_traffic(wl, retained_rows):

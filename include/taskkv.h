@@ -141,6 +141,12 @@ taskkv_status taskkv_compress_ex(const taskkv_params* p, const void* const* q_wi
                                  void* workspace_mem, size_t workspace_bytes,
                                  taskkv_stream stream, taskkv_cache** out_cache);
 
+/* Layer at a time.  Nothing couples the layers of a sequence except the schedules of Eq. 16 / Eq. 17, which
+ * are known before any data: a prefill loop can therefore compress layer r as soon as its K and V exist, as a
+ * problem of its own with n_layers = 1, n_hetero = { f(r) } (taskkv_hetero_count with the model's R and r) and
+ * that layer's mid_budget, into its own cache memory, and free the layer's K and V afterwards.  Classes,
+ * lengths, retained positions and cache rows are those the all-layer call gives for layer r. */
+
 /* The flat form of the same call: one bf16 sequence, Sec. V-D defaults for
  * everything not listed, library-owned memory, max_new_tokens = 4096. */
 taskkv_status taskkv_compress(const void* q_win, const void* k, const void* v,

@@ -144,6 +144,11 @@ class Params:
                  mid_budget, window, dtype, top_t=256, pool_kernel=7, beta=0.25, m_top=4,
                  n_hetero: Optional[Sequence[Sequence[int]]] = None, promote_center=True, force_class=-1,
                  max_new_tokens=0, mid_policy=0):
+        self.kw = dict(n_layers=n_layers, n_heads=n_heads, n_kv_heads=n_kv_heads, head_dim=head_dim,
+                       seq_lens=list(seq_lens), sink=sink, recent=recent, mid_budget=mid_budget, window=window,
+                       dtype=dtype, top_t=top_t, pool_kernel=pool_kernel, beta=beta, m_top=m_top, n_hetero=n_hetero,
+                       promote_center=promote_center, force_class=force_class, max_new_tokens=max_new_tokens,
+                       mid_policy=mid_policy)
         p = taskkv_params()
         lib.taskkv_params_default(C.byref(p))
         p.n_layers, p.n_heads, p.n_kv_heads, p.head_dim = n_layers, n_heads, n_kv_heads, head_dim
@@ -175,6 +180,24 @@ class Params:
     @property
     def torch_dtype(self):
         return torch.bfloat16 if self.c.dtype == BF16 else torch.float32
+
+    def layer(self, r: int) -> "Params":
+        """The same problem restricted to layer r, as a one-layer problem of its own: Eq. 16's head count and the
+        layer's middle budget are fixed here, so that compressing layer r alone (as soon as its K and V exist,
+        while later layers are still being computed) gives exactly the cache rows the all-layer call gives."""
+        kw = dict(self.kw)
+        R = kw["n_layers"]
+        if not 0 <= r < R:
+            raise ValueError("layer out of range")
+        mid = kw["mid_budget"]
+        kw["mid_budget"] = int(mid[r]) if isinstance(mid, (list, tuple)) else int(mid)
+        if kw["n_hetero"] is not None:
+            kw["n_hetero"] = [[int(row[r])] for row in kw["n_hetero"]]
+        else:
+            f = int(lib.taskkv_hetero_count(kw["n_kv_heads"], kw["beta"], kw["m_top"], R, r))
+            kw["n_hetero"] = [[f] for _ in kw["seq_lens"]]
+        kw["n_layers"] = 1
+        return Params(**kw)
 
 
 def taskkv_plan(params: Params) -> taskkv_plan_info:

@@ -383,3 +383,40 @@ def test_layer_by_layer_decode_equals_all_layer_decode(case):
         split.taskkv_append_ex(q[:, 0:1].contiguous(), q[:, 0:1].contiguous(), R - 1, 2)
     whole.close()
     split.close()
+
+
+def test_layer_streamed_compression_equals_all_layer_compression():
+    """Compressing layer r alone (a one-layer problem with that layer's head count and budget) gives the same
+    classes, lengths, positions, cache rows and decode outputs as the all-layer call gives for layer r."""
+    tk = _tk()
+    wl = small("stream", n=8, n_kv=4, d=128, N=0, L=32, s1=4, s2=64, k=90, dtype="bf16", R=3,
+               seq_lens=[1400, 2100], nh=1, steps=2)
+    wl.mid_budget = [90, 40, 130]
+    wl.n_hetero = [[2, 1, 0], [1, 1, 2]]
+    wl.planted = W._choose_planted(wl)
+    qs, ks, vs = W.materialize(wl, DEV)
+    params = tk.params_from_workload(wl, max_new_tokens=wl.decode_steps)
+    whole = tk.taskkv_compress_ex(params, qs, ks, vs)
+    q, kn, vn = W.gen_decode_step(wl, 0, DEV)
+    whole.taskkv_append(kn, vn)
+    want_out = whole.taskkv_decode(q)
+    nkv = wl.n_kv_heads
+    for r in range(wl.n_layers):
+        one = tk.taskkv_compress_ex(params.layer(r), [x[r:r + 1].contiguous() for x in qs],
+                                    [x[r:r + 1].contiguous() for x in ks], [x[r:r + 1].contiguous() for x in vs])
+        assert one.status() == 0
+        for b in range(wl.batch):
+            for h in range(nkv):
+                u_all = (b * wl.n_layers + r) * nkv + h
+                u_one = b * nkv + h
+                assert int(one.classes()[u_one]) == int(whole.classes()[u_all])
+                n_all = int(whole.lengths()[u_all]) - 1          # the all-layer cache already holds one appended row
+                assert int(one.lengths()[u_one]) == n_all
+                for which in ("k", "v"):
+                    assert torch.equal(one.pool_rows(which, u_one).view(torch.uint8),
+                                       whole.pool_rows(which, u_all)[:n_all].contiguous().view(torch.uint8))
+        one.taskkv_append(kn[:, r:r + 1].contiguous(), vn[:, r:r + 1].contiguous())
+        got = one.taskkv_decode(q[:, r:r + 1].contiguous())
+        assert torch.equal(got.view(torch.uint8), want_out[:, r:r + 1].contiguous().view(torch.uint8))
+        one.close()
+    whole.close()
