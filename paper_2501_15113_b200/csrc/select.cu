@@ -246,7 +246,10 @@ struct FastSmem {
   uint32_t mn[kWarps], mx[kWarps];
   int scan[kWarps];
   int scan_tot;
+  int list_n;          // keys collected for the narrow phase of the bisection
+  uint32_t list_thr;   // its result
 };
+constexpr int kNarrow = 1024;  // the bisection runs over all keys until at most this many lie in the undecided range
 
 __device__ __forceinline__ int block_count_ge(const uint32_t (&key)[kEpt], uint32_t cand, int* slot) {
   int c = 0;
@@ -260,7 +263,12 @@ __device__ __forceinline__ int block_count_ge(const uint32_t (&key)[kEpt], uint3
 }
 
 // k-th largest key (1 <= want <= number of non-zero keys) and how many keys equal to it belong to the top `want`.
-__device__ void block_bisect(FastSmem& fs, const uint32_t (&key)[kEpt], int want, uint32_t& thr, int& need_eq) {
+// Every step over all keys also tells how many keys still lie in the undecided range [t, t + 2^(bit+1)); once
+// they are few, they are collected into `list` (shared memory, `cap` entries, any order) and one warp settles
+// the remaining bits on them.  With many near-equal scores that moment may never come and the bisection simply
+// stays on all keys.  The result is the same key either way.
+__device__ void block_bisect(FastSmem& fs, const uint32_t (&key)[kEpt], int want, uint32_t* list, int cap,
+                             uint32_t& thr, int& need_eq) {
   const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
   // bits above the highest bit in which the non-zero keys differ are common to the answer
   uint32_t lo = 0xffffffffu, hi = 0u;
@@ -270,6 +278,7 @@ __device__ void block_bisect(FastSmem& fs, const uint32_t (&key)[kEpt], int want
   lo = __reduce_min_sync(0xffffffffu, lo);
   hi = __reduce_max_sync(0xffffffffu, hi);
   if (lane == 0) { fs.mn[warp] = lo; fs.mx[warp] = hi; }
+  if (threadIdx.x == 0) fs.list_n = 0;
   __syncthreads();
   lo = __reduce_min_sync(0xffffffffu, fs.mn[lane]);
   hi = __reduce_max_sync(0xffffffffu, fs.mx[lane]);
@@ -277,10 +286,37 @@ __device__ void block_bisect(FastSmem& fs, const uint32_t (&key)[kEpt], int want
   int bit = diff ? 31 - __clz(diff) : -1;
   uint32_t t = diff ? (hi & ~((2u << bit) - 1u)) : hi;
   int par = 0;
-  for (; bit >= 0; --bit) {
+  int above = 0;           // keys >= t + 2^(bit+1): the last count that fell short of `want`
+  int at_least = 1 << 30;  // keys >= t: the last count that reached `want` (unknown before the first one)
+  const int narrow = min(cap, kNarrow);
+  for (; bit >= 0 && at_least - above > narrow; --bit) {
     const uint32_t cand = t | (1u << bit);
-    if (block_count_ge(key, cand, fs.cnt[par]) >= want) t = cand;
+    const int c = block_count_ge(key, cand, fs.cnt[par]);
+    if (c >= want) { t = cand; at_least = c; } else above = c;
     par ^= 1;
+  }
+  if (bit >= 0) {
+    const uint32_t top = t + (2u << bit);            // end of the undecided range (0 if it wraps: no upper bound)
+    const int alive = at_least - above;
+    {
+#pragma unroll
+      for (int e = 0; e < kEpt; ++e)
+        if (key[e] >= t && (top == 0u || key[e] < top)) list[atomicAdd(&fs.list_n, 1)] = key[e];
+      __syncthreads();
+      if (warp == 0) {
+        const int want2 = want - above;               // rank inside the collected keys
+        for (; bit >= 0; --bit) {
+          const uint32_t cand = t | (1u << bit);
+          int c = 0;
+          for (int i = lane; i < alive; i += 32) c += list[i] >= cand;
+          c = __reduce_add_sync(0xffffffffu, c);
+          if (c >= want2) t = cand;
+        }
+        if (lane == 0) fs.list_thr = t;
+      }
+      __syncthreads();
+      t = fs.list_thr;
+    }
   }
   const int n_gt = (t == 0xffffffffu) ? 0 : block_count_ge(key, t + 1u, fs.cnt[par]);
   thr = t;
@@ -356,7 +392,8 @@ __global__ void __launch_bounds__(kThreads, 1) select_fast_kernel(DeviceProblem 
   const int t = min(p.top_t, N);
   uint32_t thr;
   int need_eq;
-  block_bisect(fs, key, t, thr, need_eq);
+  uint32_t* scratch = reinterpret_cast<uint32_t*>(&red[0][0]);   // free until the semantic vector is summed
+  block_bisect(fs, key, t, scratch, kWarps * D, thr, need_eq);
   int* topt = p.topt + (size_t)u * p.top_t;
   block_compact_regs(fs, key, base, thr, need_eq, [&](int pos, int j, int e) {
     sel[pos] = j;
@@ -432,7 +469,7 @@ __global__ void __launch_bounds__(kThreads, 1) select_fast_kernel(DeviceProblem 
     }
   }
   __syncthreads();
-  block_bisect(fs, key, kmid, thr, need_eq);
+  block_bisect(fs, key, kmid, scratch, kWarps * D, thr, need_eq);
   block_compact_regs(fs, key, base, thr, need_eq, [&](int pos, int j, int) { idx[s1 + pos] = j; });
 }
 
