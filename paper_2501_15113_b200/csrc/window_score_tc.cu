@@ -39,28 +39,41 @@ constexpr int kThreads = 352;       // warp 0 producer; 1, 6 MMA issuers; 2-5 an
 constexpr uint32_t kTmemCols = 512; // four accumulators of up to 128 columns
 constexpr uint32_t kSpinLimit = 1u << 22;
 
-// Work items of one launch (one sequence and one pass): (unit, chunk of chunk_keys keys), numbered
-// unit-major i = unit * chunks + chunk.  CTA c of a grid of g CTAs takes the items c, c + g, c + 2g, ...
+// Work items of one launch (one pass over up to kMaxSeq sequences): (sequence, unit, chunk of chunk_keys keys),
+// numbered sequence-major, then unit-major: i = item_off[s] + unit * chunks[s] + chunk.  CTA c of a grid of g
+// CTAs takes the items c, c + g, c + 2g, ...  Short sequences share a launch so that every SM has work.
+constexpr int kMaxSeq = 8;
+struct TcMaps {
+  CUtensorMap k[kMaxSeq];   // [units * N][d] of each sequence
+  CUtensorMap q[kMaxSeq];   // [units * rows][d]
+};
 struct TcArgs {
-  int pass;          // 1 = row statistics, 2 = scores
-  int u0;            // first unit of this sequence
-  int n_local;       // units in this launch (layers * kv heads)
-  int N;             // sequence length
-  int chunks;        // work items per unit
-  int chunk_keys;    // keys per work item (multiple of 128)
-  int steps;         // items of the busiest CTA
+  int pass;                 // 1 = row statistics, 2 = scores
+  int n_seq;                // sequences in this launch
+  int n_local;              // units per sequence (layers * kv heads)
+  int chunk_keys;           // keys per work item (multiple of 128)
+  int steps;                // items of the busiest CTA
+  int u0[kMaxSeq];          // first unit of each sequence
+  int N[kMaxSeq];           // sequence length
+  int chunks[kMaxSeq];      // work items per unit
+  int item_off[kMaxSeq + 1];
 };
 
 struct Item {
-  int lu, ch;
+  int seq, lu, ch;
   bool valid;
 };
 __device__ __forceinline__ Item decode_item(const TcArgs& a, int k) {
   Item it;
   const int i = (int)blockIdx.x + k * (int)gridDim.x;
-  it.valid = i < a.n_local * a.chunks;
-  it.lu = it.valid ? i / a.chunks : 0;
-  it.ch = it.valid ? i % a.chunks : 0;
+  it.valid = i < a.item_off[a.n_seq];
+  it.seq = 0;
+#pragma unroll
+  for (int s = 1; s < kMaxSeq; ++s)
+    if (s < a.n_seq && i >= a.item_off[s]) it.seq = s;
+  const int local = it.valid ? i - a.item_off[it.seq] : 0;
+  it.lu = local / a.chunks[it.seq];
+  it.ch = local % a.chunks[it.seq];
   return it;
 }
 
@@ -214,8 +227,8 @@ enum : int {
 
 template <int D>
 __global__ void __launch_bounds__(kThreads, 1)
-window_tc_kernel(const __grid_constant__ CUtensorMap tmap_k, const __grid_constant__ CUtensorMap tmap_q,
-                 DeviceProblem p, TcArgs a, TcLayout lay) {
+window_tc_kernel(const __grid_constant__ TcMaps maps, DeviceProblem p, const __grid_constant__ TcArgs a,
+                 TcLayout lay) {
   constexpr int KB = D / 64;
   extern __shared__ unsigned char smem_raw[];
   // 1024-byte alignment: the swizzle pattern is a function of the address bits
@@ -232,7 +245,7 @@ window_tc_kernel(const __grid_constant__ CUtensorMap tmap_k, const __grid_consta
 
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
   const int rows = p.rows;                  // 32, 64 or 128
-  const int N = a.N, L = p.L;
+  const int L = p.L;
   const int S = lay.stages;
   const uint32_t bar0 = smem_u32(bars);
   auto BAR = [&](int i) { return bar0 + 8u * (uint32_t)i; };
@@ -269,6 +282,7 @@ window_tc_kernel(const __grid_constant__ CUtensorMap tmap_k, const __grid_consta
       for (int k = 0; k < a.steps && ok; ++k) {
         const Item it = decode_item(a, k);
         if (!it.valid) continue;
+        const int N = a.N[it.seq];
         const int key0 = it.ch * a.chunk_keys;
         const int ntiles = (min(N, key0 + a.chunk_keys) - key0 + kTile - 1) / kTile;
         ok = __all_sync(0xffffffffu, mbar_wait(BAR(B_QEMPTY + qb), qphase[qb] ^ 1, s_abort));
@@ -276,8 +290,8 @@ window_tc_kernel(const __grid_constant__ CUtensorMap tmap_k, const __grid_consta
         if (elect_one()) {
           mbar_expect_tx(BAR(B_QFULL + qb), (uint32_t)lay.q_block_bytes);
           for (int kb = 0; kb < KB; ++kb)
-            tma_load_2d(smem_u32(sQ + (size_t)qb * lay.q_block_bytes + (size_t)kb * rows * 128), &tmap_q, kb * 64,
-                        it.lu * rows, BAR(B_QFULL + qb));
+            tma_load_2d(smem_u32(sQ + (size_t)qb * lay.q_block_bytes + (size_t)kb * rows * 128), &maps.q[it.seq],
+                        kb * 64, it.lu * rows, BAR(B_QFULL + qb));
         }
         __syncwarp();
         qphase[qb] ^= 1;
@@ -289,7 +303,7 @@ window_tc_kernel(const __grid_constant__ CUtensorMap tmap_k, const __grid_consta
             mbar_expect_tx(BAR(B_FULL + stage), (uint32_t)lay.tile_bytes);
 #pragma unroll
             for (int kb = 0; kb < KB; ++kb)
-              tma_load_2d(smem_u32(sK + (size_t)stage * lay.tile_bytes + (size_t)kb * kTile * 128), &tmap_k,
+              tma_load_2d(smem_u32(sK + (size_t)stage * lay.tile_bytes + (size_t)kb * kTile * 128), &maps.k[it.seq],
                           kb * 64, it.lu * N + key0 + t * kTile, BAR(B_FULL + stage));
           }
           __syncwarp();
@@ -324,6 +338,7 @@ window_tc_kernel(const __grid_constant__ CUtensorMap tmap_k, const __grid_consta
       for (int k = 0; k < a.steps && ok; ++k) {
         const Item it = decode_item(a, k);
         if (!it.valid) continue;
+        const int N = a.N[it.seq];
         const int key0 = it.ch * a.chunk_keys;
         const int ntiles = (min(N, key0 + a.chunk_keys) - key0 + kTile - 1) / kTile;
         ok = __all_sync(0xffffffffu, mbar_wait(BAR(B_QFULL + qb), qphase[qb], s_abort));
@@ -382,14 +397,15 @@ window_tc_kernel(const __grid_constant__ CUtensorMap tmap_k, const __grid_consta
       const Item nx = decode_item(a, k);
 #pragma unroll
       for (int q = 0; q < 4; ++q)
-        pre[q] = (nx.valid && q * 32 + lane < rows) ? stat_g[(size_t)(a.u0 + nx.lu) * (2 * p.rows_pad) + q * 32 + lane]
+        pre[q] = (nx.valid && q * 32 + lane < rows) ? stat_g[(size_t)(a.u0[nx.seq] + nx.lu) * (2 * p.rows_pad) + q * 32 + lane]
                                                     : 0.f;
     };
     if (a.pass == 2) fetch_stats(0);
     for (int k = 0; k < a.steps && ok; ++k) {
       const Item it = decode_item(a, k);
       if (!it.valid) continue;
-      const int u = a.u0 + it.lu;
+      const int u = a.u0[it.seq] + it.lu;
+      const int N = a.N[it.seq];
       const int key0 = it.ch * a.chunk_keys;
       const int ntiles = (min(N, key0 + a.chunk_keys) - key0 + kTile - 1) / kTile;
       // pass 1 state: after the transposition lane = window row (rg * 32 + lane); raw (unscaled) maxima
@@ -556,8 +572,9 @@ window_tc_kernel(const __grid_constant__ CUtensorMap tmap_k, const __grid_consta
 
 // Folds the partial statistics of one unit: slots (item, warp) of pass 1 -> one offset per row.
 // One warp per (unit, row): lanes take every 32nd slot, then a shuffle tree; the order is fixed.
-__global__ void __launch_bounds__(128) window_tc_reduce_kernel(DeviceProblem p, int u0, int slots) {
+__global__ void __launch_bounds__(128) window_tc_reduce_kernel(DeviceProblem p, int u0, int chunk_keys, int parts) {
   const int u = u0 + blockIdx.x;
+  const int slots = (p.unit_N[u] + chunk_keys - 1) / chunk_keys * parts;
   const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
   const float2* part = reinterpret_cast<const float2*>(p.stat_part) + (size_t)u * p.chunks_max * p.rows_pad;
   const int row = blockIdx.y * 4 + warp;
@@ -619,10 +636,10 @@ bool make_map(CUtensorMap* map, const void* base, int d, uint64_t rows_total, in
 }
 
 // Keys per work item.  Every item costs a Q load and, in pass 2, a statistics load, so long items are
-// better as long as the CTAs still get a dozen items each; short sequences keep 2048-key items.
-inline int pick_chunk(int per_seq, int N, int n_sm) {
+// better as long as the CTAs still get a dozen items each; short inputs keep 2048-key items.
+inline int pick_chunk(int64_t units_times_keys, int n_sm) {
   const int big = 2 * kTcChunk;
-  return (int64_t)per_seq * ((N + big - 1) / big) >= (int64_t)12 * n_sm ? big : kTcChunk;
+  return units_times_keys / big >= (int64_t)12 * n_sm ? big : kTcChunk;
 }
 
 template <int D>
@@ -640,34 +657,44 @@ cudaError_t launch_tc_d(const DeviceProblem& p, const WindowHostInfo& h, cudaStr
   cudaError_t e = cudaFuncSetAttribute(window_tc_kernel<D>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem);
   if (e != cudaSuccess) return e;
   const int per_seq = p.R * p.n_kv;
-  for (int b = 0; b < h.batch; ++b) {
-    const int N = h.seq_lens[b];
-    CUtensorMap mk, mq;
-    if (!make_map(&mk, h.k[b], D, (uint64_t)per_seq * (uint64_t)N, kTile)) return cudaErrorUnknown;
-    if (!make_map(&mq, h.q[b], D, (uint64_t)per_seq * (uint64_t)p.rows, p.rows)) return cudaErrorUnknown;
+  const int parts = p.rows == 128 ? 2 : kTcParts;
+  // up to kMaxSeq sequences per pair of launches
+  for (int b0 = 0; b0 < h.batch; b0 += kMaxSeq) {
+    const int nb = h.batch - b0 < kMaxSeq ? h.batch - b0 : kMaxSeq;
+    TcMaps maps;
     TcArgs a;
-    a.u0 = b * per_seq;
+    int64_t keys = 0;
+    for (int i = 0; i < nb; ++i) keys += (int64_t)per_seq * h.seq_lens[b0 + i];
+    a.n_seq = nb;
     a.n_local = per_seq;
-    a.N = N;
-    a.chunk_keys = pick_chunk(per_seq, N, n_sm);
-    a.chunks = (N + a.chunk_keys - 1) / a.chunk_keys;
-    const int n1 = a.n_local * a.chunks;
+    a.chunk_keys = pick_chunk(keys, n_sm);
+    a.item_off[0] = 0;
+    for (int i = 0; i < kMaxSeq; ++i) {
+      const int b = b0 + (i < nb ? i : 0);                  // unused slots repeat the first sequence
+      const int N = h.seq_lens[b];
+      if (!make_map(&maps.k[i], h.k[b], D, (uint64_t)per_seq * (uint64_t)N, kTile)) return cudaErrorUnknown;
+      if (!make_map(&maps.q[i], h.q[b], D, (uint64_t)per_seq * (uint64_t)p.rows, p.rows)) return cudaErrorUnknown;
+      a.u0[i] = b * per_seq;
+      a.N[i] = N;
+      a.chunks[i] = (N + a.chunk_keys - 1) / a.chunk_keys;
+      a.item_off[i + 1] = a.item_off[i] + (i < nb ? per_seq * a.chunks[i] : 0);
+    }
+    const int n1 = a.item_off[nb];
     const int grid = n1 < n_sm ? n1 : n_sm;
     a.steps = (n1 + grid - 1) / grid;
-    const int parts = p.rows == 128 ? 2 : kTcParts;
     a.pass = 1;
     {
       LaunchScope ls(K_WINDOW_TC, s);
-      window_tc_kernel<D><<<grid, kThreads, smem, s>>>(mk, mq, p, a, lay);
+      window_tc_kernel<D><<<grid, kThreads, smem, s>>>(maps, p, a, lay);
     }
     {
       LaunchScope ls(K_WINDOW_REDUCE, s);
-      window_tc_reduce_kernel<<<dim3(per_seq, (p.rows + 3) / 4), 128, 0, s>>>(p, a.u0, a.chunks * parts);
+      window_tc_reduce_kernel<<<dim3(nb * per_seq, (p.rows + 3) / 4), 128, 0, s>>>(p, b0 * per_seq, a.chunk_keys, parts);
     }
     a.pass = 2;
     {
       LaunchScope ls(K_WINDOW_TC, s);
-      window_tc_kernel<D><<<grid, kThreads, smem, s>>>(mk, mq, p, a, lay);
+      window_tc_kernel<D><<<grid, kThreads, smem, s>>>(maps, p, a, lay);
     }
     e = cudaGetLastError();
     if (e != cudaSuccess) return e;
