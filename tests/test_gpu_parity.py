@@ -259,6 +259,13 @@ def test_mistral_shaped_ragged_batch():
     run_workload(wl)
 
 
+def test_ragged_batch_of_eleven_sequences():
+    """More sequences than one window-score launch takes (eight): a full group and a partial one."""
+    from paper_2501_15113_b200 import configs
+    wl = configs.config4_mistral(batch=11, lo=700, hi=2600, n_layers=1, decode_steps=2)
+    run_workload(wl)
+
+
 @pytest.mark.parametrize("n_hetero,mid", [(0, 64), (2, 256), (8, 1024)])
 def test_budget_sweep_points(n_hetero, mid):
     """Config 5 scaled down: planted fraction x middle budget."""
