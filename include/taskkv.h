@@ -187,6 +187,16 @@ taskkv_status taskkv_append_ex(taskkv_cache* c, const void* k_new, const void* v
 taskkv_status taskkv_decode_ex(const void* q, taskkv_cache* c, const int32_t* lengths, void* out,
                                int32_t layer_begin, int32_t layer_count, taskkv_stream stream);
 
+/* One decode step in one call: taskkv_append_ex followed by taskkv_decode_ex on the same layers, fused -- the new
+ * token's k, v rows are read by the attention kernel straight from k_new, v_new (and stored in the segments by
+ * it), and the lengths are raised by its combine pass; outputs, cache rows and lengths afterwards are those of
+ * the two separate calls, bit for bit.  A unit already at capacity attends over its existing rows only and
+ * the sticky status becomes ESTATE.  taskkv_decode_step covers every layer. */
+taskkv_status taskkv_decode_step_ex(const void* q, const void* k_new, const void* v_new, taskkv_cache* c,
+                                    void* out, int32_t layer_begin, int32_t layer_count, taskkv_stream stream);
+taskkv_status taskkv_decode_step(const void* q, const void* k_new, const void* v_new, taskkv_cache* c,
+                                 void* out, taskkv_stream stream);
+
 /* One decode step with HOST buffers: copies q, k_new, v_new in, appends,
  * attends and copies out back (k_new and v_new may both be NULL to skip the
  * append).  Synchronises the stream before returning. */

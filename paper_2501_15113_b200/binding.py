@@ -69,6 +69,10 @@ lib.taskkv_append_ex.argtypes = [_vp, _vp, _vp, C.c_int32, C.c_int32, _vp]
 lib.taskkv_append_ex.restype = C.c_int32
 lib.taskkv_decode_ex.argtypes = [_vp, _vp, _vp, _vp, C.c_int32, C.c_int32, _vp]
 lib.taskkv_decode_ex.restype = C.c_int32
+lib.taskkv_decode_step_ex.argtypes = [_vp, _vp, _vp, _vp, _vp, C.c_int32, C.c_int32, _vp]
+lib.taskkv_decode_step_ex.restype = C.c_int32
+lib.taskkv_decode_step.argtypes = [_vp, _vp, _vp, _vp, _vp, _vp]
+lib.taskkv_decode_step.restype = C.c_int32
 lib.taskkv_decode_host.argtypes = [_vp, _vp, _vp, _vp, _vp, _vp]
 lib.taskkv_decode_host.restype = C.c_int32
 lib.taskkv_decode_noalloc.argtypes = [_vp, _vp, _vp, _vp, _vp] + [C.c_int32] * 5 + [_vp, _vp]
@@ -265,6 +269,22 @@ class Cache:
         lp = lengths.data_ptr() if lengths is not None else None
         _check(lib.taskkv_decode_ex(q.data_ptr(), self._h, lp, out.data_ptr(), layer_begin, layer_count,
                                     _stream_handle(stream)), "taskkv_decode_ex")
+        return out
+
+    def taskkv_decode_step(self, q: torch.Tensor, k_new: torch.Tensor, v_new: torch.Tensor,
+                           out: Optional[torch.Tensor] = None, stream=None) -> torch.Tensor:
+        if out is None:
+            out = torch.empty_like(q)
+        _check(lib.taskkv_decode_step(q.data_ptr(), k_new.data_ptr(), v_new.data_ptr(), self._h, out.data_ptr(),
+                                      _stream_handle(stream)), "taskkv_decode_step")
+        return out
+
+    def taskkv_decode_step_ex(self, q: torch.Tensor, k_new: torch.Tensor, v_new: torch.Tensor, layer_begin: int,
+                              layer_count: int, out: Optional[torch.Tensor] = None, stream=None) -> torch.Tensor:
+        if out is None:
+            out = torch.empty_like(q)
+        _check(lib.taskkv_decode_step_ex(q.data_ptr(), k_new.data_ptr(), v_new.data_ptr(), self._h, out.data_ptr(),
+                                         layer_begin, layer_count, _stream_handle(stream)), "taskkv_decode_step_ex")
         return out
 
     def taskkv_decode_host(self, q: torch.Tensor, k_new: Optional[torch.Tensor], v_new: Optional[torch.Tensor],

@@ -26,7 +26,7 @@ struct HostPlan {
   std::vector<int32_t> full;                    // [B*R] full-cache heads
   // byte offsets inside the cache memory
   size_t o_unit_N, o_unit_mid, o_nhet, o_c_off, o_qp, o_kp, o_vp, meta_bytes;
-  size_t o_status, o_len, o_cap, o_seg, o_cls, o_dist, o_sem, o_idx, o_goff, o_doff, o_pacc, o_pml, o_kpool,
+  size_t o_status, o_len, o_cap, o_seg, o_cls, o_dist, o_sem, o_idx, o_goff, o_doff, o_step, o_pacc, o_pml, o_kpool,
       o_vpool;
   // inside the workspace
   size_t w_C, w_spart, w_stat, w_topt;
@@ -141,6 +141,7 @@ taskkv_status make_plan(const taskkv_params* p, HostPlan& hp) {
   hp.o_idx = take((size_t)U * hp.idx_stride * 4);
   hp.o_goff = take((U + 1) * 4);
   hp.o_doff = take((U + 1) * 4);
+  hp.o_step = take(U * 4);
   hp.o_pacc = take((size_t)ditems * G * d * 4);
   hp.o_pml = take((size_t)ditems * G * 2 * 4);
   hp.o_kpool = take((size_t)pool * d * es);
@@ -266,6 +267,7 @@ void fill_device_problem(taskkv_cache* c) {
   d.idx = reinterpret_cast<int32_t*>(cm + hp.o_idx);
   d.gather_off = reinterpret_cast<int32_t*>(cm + hp.o_goff);
   d.dec_off = reinterpret_cast<int32_t*>(cm + hp.o_doff);
+  d.step_cnt = reinterpret_cast<int32_t*>(cm + hp.o_step);
   d.part_acc = reinterpret_cast<float*>(cm + hp.o_pacc);
   d.part_ml = reinterpret_cast<float*>(cm + hp.o_pml);
   d.k_pool = cm + hp.o_kpool;
@@ -407,6 +409,7 @@ taskkv_status taskkv_compress_ex(const taskkv_params* p, const void* const* q_wi
 
   cudaError_t e = cudaMemcpyAsync(c->cache_mem, c->meta.data(), c->hp.meta_bytes, cudaMemcpyHostToDevice, s);
   if (e == cudaSuccess) e = cudaMemsetAsync(c->dp.status, 0, 64, s);
+  if (e == cudaSuccess) e = cudaMemsetAsync(c->dp.step_cnt, 0, (size_t)c->dp.U * 4, s);
   WindowHostInfo wh;
   wh.batch = p->batch;
   wh.seq_lens = c->hp.seq_lens.data();
@@ -520,7 +523,24 @@ taskkv_status taskkv_decode_ex(const void* q, taskkv_cache* c, const int32_t* le
   if (!c || !q || !out || (((uintptr_t)q | (uintptr_t)out) & 15)) return TASKKV_EINVAL;
   taskkv::DeviceProblem view;
   if (!layer_view(c, layer_begin, layer_count, &view)) return TASKKV_EINVAL;
-  return cuda_status(launch_decode(view, c->prm.dtype, q, lengths, out, static_cast<cudaStream_t>(stream)));
+  return cuda_status(launch_decode(view, c->prm.dtype, q, lengths, nullptr, nullptr, out,
+                                   static_cast<cudaStream_t>(stream)));
+}
+
+taskkv_status taskkv_decode_step_ex(const void* q, const void* k_new, const void* v_new, taskkv_cache* c, void* out,
+                                    int32_t layer_begin, int32_t layer_count, taskkv_stream stream) {
+  if (!c || !q || !out || !k_new || !v_new) return TASKKV_EINVAL;
+  if (((uintptr_t)q | (uintptr_t)out | (uintptr_t)k_new | (uintptr_t)v_new) & 15) return TASKKV_EINVAL;
+  taskkv::DeviceProblem view;
+  if (!layer_view(c, layer_begin, layer_count, &view)) return TASKKV_EINVAL;
+  return cuda_status(launch_decode(view, c->prm.dtype, q, nullptr, k_new, v_new, out,
+                                   static_cast<cudaStream_t>(stream)));
+}
+
+taskkv_status taskkv_decode_step(const void* q, const void* k_new, const void* v_new, taskkv_cache* c, void* out,
+                                 taskkv_stream stream) {
+  if (!c) return TASKKV_EINVAL;
+  return taskkv_decode_step_ex(q, k_new, v_new, c, out, 0, c->dp.R, stream);
 }
 
 taskkv_status taskkv_decode(const void* q, taskkv_cache* c, const int32_t* lengths, void* out,
@@ -555,9 +575,9 @@ taskkv_status taskkv_decode_host(const void* q, const void* k_new, const void* v
   if (k_new && e == cudaSuccess) {
     e = cudaMemcpyAsync(dkn, k_new, k_bytes, cudaMemcpyHostToDevice, s);
     if (e == cudaSuccess) e = cudaMemcpyAsync(dvn, v_new, k_bytes, cudaMemcpyHostToDevice, s);
-    if (e == cudaSuccess) e = launch_append(c->dp, c->prm.dtype, dkn, dvn, s);
   }
-  if (e == cudaSuccess) e = launch_decode(c->dp, c->prm.dtype, dq, nullptr, dout, s);
+  if (e == cudaSuccess)
+    e = launch_decode(c->dp, c->prm.dtype, dq, nullptr, k_new ? dkn : nullptr, k_new ? dvn : nullptr, dout, s);
   if (e == cudaSuccess) e = cudaMemcpyAsync(out, dout, q_bytes, cudaMemcpyDeviceToHost, s);
   if (e == cudaSuccess) e = cudaStreamSynchronize(s);
   return cuda_status(e);

@@ -74,6 +74,7 @@ struct DeviceProblem {
   int32_t* idx;               // [U][idx_stride]
   int32_t* gather_off;        // [U+1] gather work items
   int32_t* dec_off;           // [U+1] decode work items
+  int32_t* step_cnt;          // [U] combine blocks of a unit that finished the current fused step (0 between calls)
   void* k_pool;
   void* v_pool;
   // decode scratch
@@ -116,8 +117,8 @@ cudaError_t launch_gather(const DeviceProblem& p, int dtype, int64_t gather_item
 cudaError_t launch_compensate(const DeviceProblem& p, int dtype, cudaStream_t s);
 cudaError_t launch_append(const DeviceProblem& p, int dtype, const void* k_new, const void* v_new,
                           cudaStream_t s);
-cudaError_t launch_decode(const DeviceProblem& p, int dtype, const void* q, const int32_t* lengths, void* out,
-                          cudaStream_t s);
+cudaError_t launch_decode(const DeviceProblem& p, int dtype, const void* q, const int32_t* lengths,
+                          const void* k_new, const void* v_new, void* out, cudaStream_t s);
 
 // ---------------------------------------------------------------- device helpers
 #ifdef __CUDACC__

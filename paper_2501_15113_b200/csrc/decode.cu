@@ -8,6 +8,8 @@
 // (running max, sum, weighted V) per head with an online softmax in fp32; one
 // combine pass merges a unit's partials.  K/V rows are read once, as 16-byte
 // vectors, by all G heads.
+#include <type_traits>
+
 #include "common.cuh"
 
 namespace taskkv {
@@ -20,7 +22,9 @@ constexpr int kUnroll = 4;
 
 template <typename T, int D, int G>
 __global__ void __launch_bounds__(kAttnThreads) decode_attn_kernel(DeviceProblem p, const T* __restrict__ q,
-                                                                   const int32_t* __restrict__ lengths) {
+                                                                   const int32_t* __restrict__ lengths,
+                                                                   const unsigned char* __restrict__ k_new,
+                                                                   const unsigned char* __restrict__ v_new) {
   constexpr int EPL = 16 / (int)sizeof(T);          // elements per lane (one 16-byte vector)
   constexpr int LPR = D / EPL;                      // lanes per row
   constexpr int RPW = 32 / LPR;                     // rows per warp instruction
@@ -49,11 +53,23 @@ __global__ void __launch_bounds__(kAttnThreads) decode_attn_kernel(DeviceProblem
     const int vu = lu.v;                            // view unit: index into q and lengths
     const int u = lu.u;                             // unit: index into the cache
     int len = p.len[u];
+    // fused step: the new token's row sits at index len; it is read from k_new / v_new and the item that holds
+    // it also stores it in the segment (the length itself is raised by the combine pass)
+    const int new_r = (k_new != nullptr && len < p.cap[u]) ? len : -1;
+    if (new_r >= 0) ++len;
     if (lengths) len = min(max(lengths[vu], 0), len);
     const int rbeg = (item - p.dec_off[w]) * kDecodeChunk;
     if (rbeg >= len) continue;                      // an item of the reserve beyond the segment's length
     const int rend = min(len, rbeg + kDecodeChunk);
     const int64_t seg = p.seg_off[u];
+    const unsigned char* kn_row = k_new + (size_t)vu * ROW_BYTES;
+    const unsigned char* vn_row = v_new + (size_t)vu * ROW_BYTES;
+    if (new_r >= rbeg && new_r < rend && tid < ROW_BYTES / 16) {
+      unsigned char* kd = static_cast<unsigned char*>(p.k_pool) + ((size_t)seg + new_r) * ROW_BYTES + tid * 16;
+      unsigned char* vd = static_cast<unsigned char*>(p.v_pool) + ((size_t)seg + new_r) * ROW_BYTES + tid * 16;
+      *reinterpret_cast<uint4*>(kd) = *reinterpret_cast<const uint4*>(kn_row + tid * 16);
+      *reinterpret_cast<uint4*>(vd) = *reinterpret_cast<const uint4*>(vn_row + tid * 16);
+    }
     const unsigned char* kp = static_cast<const unsigned char*>(p.k_pool) + (size_t)seg * ROW_BYTES + sl * 16;
     const unsigned char* vp = static_cast<const unsigned char*>(p.v_pool) + (size_t)seg * ROW_BYTES + sl * 16;
 
@@ -74,6 +90,8 @@ __global__ void __launch_bounds__(kAttnThreads) decode_attn_kernel(DeviceProblem
       for (int e = 0; e < EPL; ++e) acc[g][e] = 0.f;
     }
 
+    // two copies of the row loop: only the item that holds the new token's row pays for telling it apart
+    auto rows_loop = [&](auto has_new) {
     for (int base = rbeg; base < rend; base += NSG * kUnroll) {   // warp-uniform trip count
       const int r0 = base + gsg;
       uint4 kraw[kUnroll], vraw[kUnroll];
@@ -81,8 +99,10 @@ __global__ void __launch_bounds__(kAttnThreads) decode_attn_kernel(DeviceProblem
       for (int i = 0; i < kUnroll; ++i) {
         const int r = r0 + i * NSG;
         if (r < rend) {
-          kraw[i] = *reinterpret_cast<const uint4*>(kp + (size_t)r * ROW_BYTES);
-          vraw[i] = *reinterpret_cast<const uint4*>(vp + (size_t)r * ROW_BYTES);
+          kraw[i] = *reinterpret_cast<const uint4*>((decltype(has_new)::value && r == new_r) ? kn_row + sl * 16
+                                                                                             : kp + (size_t)r * ROW_BYTES);
+          vraw[i] = *reinterpret_cast<const uint4*>((decltype(has_new)::value && r == new_r) ? vn_row + sl * 16
+                                                                                             : vp + (size_t)r * ROW_BYTES);
         } else {
           kraw[i] = make_uint4(0, 0, 0, 0);
           vraw[i] = make_uint4(0, 0, 0, 0);
@@ -139,6 +159,9 @@ __global__ void __launch_bounds__(kAttnThreads) decode_attn_kernel(DeviceProblem
           for (int e = 0; e < EPL; ++e) acc[g][e] = fmaf(pw[i][g], vf[e], acc[g][e]);
       }
     }
+
+    };
+    if (new_r >= rbeg && new_r < rend) rows_loop(std::true_type{}); else rows_loop(std::false_type{});
 
     // merge the block's sub-groups
 #pragma unroll
@@ -206,7 +229,9 @@ __device__ __forceinline__ uint32_t word_of(const uint4& v, int i) {
 template <int D, int G>
 __global__ void __launch_bounds__(kAttnThreads) decode_attn_mma_kernel(DeviceProblem p,
                                                                        const __nv_bfloat16* __restrict__ q,
-                                                                       const int32_t* __restrict__ lengths) {
+                                                                       const int32_t* __restrict__ lengths,
+                                                                       const unsigned char* __restrict__ k_new,
+                                                                       const unsigned char* __restrict__ v_new) {
   constexpr int ROW_BYTES = D * 2;
   constexpr int KC = D / 16;            // k-chunks of the first product
   constexpr int KP = D / 32;            // 16-byte pieces of a K row per lane
@@ -237,11 +262,23 @@ __global__ void __launch_bounds__(kAttnThreads) decode_attn_mma_kernel(DevicePro
     const int vu = lu.v;                            // view unit: index into q and lengths
     const int u = lu.u;                             // unit: index into the cache
     int len = p.len[u];
+    // fused step: the new token's row sits at index len; it is read from k_new / v_new and the item that holds
+    // it also stores it in the segment (the length itself is raised by the combine pass)
+    const int new_r = (k_new != nullptr && len < p.cap[u]) ? len : -1;
+    if (new_r >= 0) ++len;
     if (lengths) len = min(max(lengths[vu], 0), len);
     const int rbeg = (item - p.dec_off[w]) * kDecodeChunk;
     if (rbeg >= len) continue;                      // an item of the reserve beyond the segment's length
     const int rend = min(len, rbeg + kDecodeChunk);
     const int64_t seg = p.seg_off[u];
+    const unsigned char* kn_row = k_new + (size_t)vu * ROW_BYTES;
+    const unsigned char* vn_row = v_new + (size_t)vu * ROW_BYTES;
+    if (new_r >= rbeg && new_r < rend && tid < ROW_BYTES / 16) {
+      unsigned char* kd = static_cast<unsigned char*>(p.k_pool) + ((size_t)seg + new_r) * ROW_BYTES + tid * 16;
+      unsigned char* vd = static_cast<unsigned char*>(p.v_pool) + ((size_t)seg + new_r) * ROW_BYTES + tid * 16;
+      *reinterpret_cast<uint4*>(kd) = *reinterpret_cast<const uint4*>(kn_row + tid * 16);
+      *reinterpret_cast<uint4*>(vd) = *reinterpret_cast<const uint4*>(vn_row + tid * 16);
+    }
     const unsigned char* kp = static_cast<const unsigned char*>(p.k_pool) + (size_t)seg * ROW_BYTES;
     const unsigned char* vp = static_cast<const unsigned char*>(p.v_pool) + (size_t)seg * ROW_BYTES;
 
@@ -261,6 +298,8 @@ __global__ void __launch_bounds__(kAttnThreads) decode_attn_mma_kernel(DevicePro
 #pragma unroll
       for (int e = 0; e < 4; ++e) o[mb][e] = 0.f;
 
+    // two copies of the row loop: only the item that holds the new token's row pays for telling it apart
+    auto rows_loop = [&](auto has_new) {
     for (int blk = rbeg + warp * kBlk; blk < rend; blk += kAttnWarps * kBlk) {   // warp-uniform
       uint4 kraw[2][KP], vraw[4][VP];
 #pragma unroll
@@ -268,7 +307,9 @@ __global__ void __launch_bounds__(kAttnThreads) decode_attn_mma_kernel(DevicePro
         const int r = blk + 8 * j + g;
 #pragma unroll
         for (int i = 0; i < KP; ++i)
-          kraw[j][i] = r < rend ? *reinterpret_cast<const uint4*>(kp + (size_t)r * ROW_BYTES + (i * 4 + t) * 16)
+          kraw[j][i] = r < rend ? *reinterpret_cast<const uint4*>(((decltype(has_new)::value && r == new_r)
+                                                                       ? kn_row : kp + (size_t)r * ROW_BYTES) +
+                                                                  (i * 4 + t) * 16)
                                 : make_uint4(0, 0, 0, 0);
       }
 #pragma unroll
@@ -276,7 +317,9 @@ __global__ void __launch_bounds__(kAttnThreads) decode_attn_mma_kernel(DevicePro
         const int r = blk + 2 * t + (x & 1) + 8 * (x >> 1);
 #pragma unroll
         for (int i = 0; i < VP; ++i)
-          vraw[x][i] = r < rend ? *reinterpret_cast<const uint4*>(vp + (size_t)r * ROW_BYTES + i * 128 + g * 16)
+          vraw[x][i] = r < rend ? *reinterpret_cast<const uint4*>(((decltype(has_new)::value && r == new_r)
+                                                                       ? vn_row : vp + (size_t)r * ROW_BYTES) +
+                                                                  i * 128 + g * 16)
                                 : make_uint4(0, 0, 0, 0);
       }
       // S^T for the two 8-row halves of the block
@@ -336,6 +379,9 @@ __global__ void __launch_bounds__(kAttnThreads) decode_attn_mma_kernel(DevicePro
       }
     }
 
+    };
+    if (new_r >= rbeg && new_r < rend) rows_loop(std::true_type{}); else rows_loop(std::false_type{});
+
     // merge the four warps (same partial format as the scalar kernel)
     l_run += __shfl_xor_sync(0xffffffffu, l_run, 1);
     l_run += __shfl_xor_sync(0xffffffffu, l_run, 2);
@@ -375,7 +421,7 @@ __global__ void __launch_bounds__(kAttnThreads) decode_attn_mma_kernel(DevicePro
 // loads, fixed order), and the four warps are summed in shared memory.
 template <typename T, int D, int G>
 __global__ void __launch_bounds__(kAttnThreads) decode_combine_kernel(DeviceProblem p, const int32_t* __restrict__ lengths,
-                                                                      T* __restrict__ out) {
+                                                                      int fused_step, T* __restrict__ out) {
   constexpr int EPL = D / 32;
   __shared__ float s_max[kAttnWarps];
   __shared__ float s_l[kAttnWarps];
@@ -384,6 +430,9 @@ __global__ void __launch_bounds__(kAttnThreads) decode_combine_kernel(DeviceProb
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
   const int unit = view_unit(p, u);
   int len = p.len[unit];
+  const bool grown = fused_step && len < p.cap[unit];   // the attention pass has appended the new token's row
+  const int len_next = len + (grown ? 1 : 0);
+  len = len_next;
   if (lengths) len = min(max(lengths[u], 0), len);
   // the unit's items that hold rows (the table also numbers the reserve for appended tokens)
   const int i0 = p.dec_off[lm_index(p, unit)], i1 = i0 + (len + kDecodeChunk - 1) / kDecodeChunk;
@@ -416,48 +465,59 @@ __global__ void __launch_bounds__(kAttnThreads) decode_combine_kernel(DeviceProb
     const float a = (s_acc[0][tid] + s_acc[1][tid]) + (s_acc[2][tid] + s_acc[3][tid]);
     store_out(out + ((size_t)u * G + g) * D + tid, Lt > 0.f ? a / Lt : 0.f);
   }
+  // fused step: the last of the unit's G blocks (each has read the old length by now) raises the length
+  if (fused_step && tid == 0) {
+    if (atomicAdd(&p.step_cnt[unit], 1) == G - 1) {
+      p.step_cnt[unit] = 0;
+      if (grown) p.len[unit] = len_next;
+      else set_status(p.status, TASKKV_ESTATE);
+    }
+  }
 }
 
 template <typename T, int D, int G>
-cudaError_t launch_typed(const DeviceProblem& p, const void* q, const int32_t* lengths, void* out,
-                         cudaStream_t s) {
+cudaError_t launch_typed(const DeviceProblem& p, const void* q, const int32_t* lengths, const void* k_new,
+                         const void* v_new, void* out, cudaStream_t s) {
+  const unsigned char* kn = static_cast<const unsigned char*>(k_new);
+  const unsigned char* vn = static_cast<const unsigned char*>(v_new);
   // persistent blocks: 16 per SM (measured best on B200 with 512-row items)
   int64_t grid = p.max_items < 148 * 16 ? p.max_items : 148 * 16;
   if (grid < 1) grid = 1;
   {
     LaunchScope ls(K_DECODE_ATTN, s);
     if constexpr (sizeof(T) == 2)
-      decode_attn_mma_kernel<D, G><<<(unsigned)grid, kAttnThreads, 0, s>>>(p, static_cast<const T*>(q), lengths);
+      decode_attn_mma_kernel<D, G><<<(unsigned)grid, kAttnThreads, 0, s>>>(p, static_cast<const T*>(q), lengths, kn, vn);
     else
-      decode_attn_kernel<T, D, G><<<(unsigned)grid, kAttnThreads, 0, s>>>(p, static_cast<const T*>(q), lengths);
+      decode_attn_kernel<T, D, G><<<(unsigned)grid, kAttnThreads, 0, s>>>(p, static_cast<const T*>(q), lengths, kn, vn);
   }
   {
     LaunchScope ls(K_DECODE_COMBINE, s);
-    decode_combine_kernel<T, D, G><<<(unsigned)(p.view_U * G), kAttnThreads, 0, s>>>(p, lengths, static_cast<T*>(out));
+    decode_combine_kernel<T, D, G><<<(unsigned)(p.view_U * G), kAttnThreads, 0, s>>>(p, lengths, k_new != nullptr ? 1 : 0,
+                                                                                     static_cast<T*>(out));
   }
   return cudaGetLastError();
 }
 
 template <typename T, int D>
-cudaError_t launch_group(const DeviceProblem& p, const void* q, const int32_t* lengths, void* out,
-                         cudaStream_t s) {
+cudaError_t launch_group(const DeviceProblem& p, const void* q, const int32_t* lengths, const void* k_new,
+                         const void* v_new, void* out, cudaStream_t s) {
   switch (p.G) {
-    case 1: return launch_typed<T, D, 1>(p, q, lengths, out, s);
-    case 2: return launch_typed<T, D, 2>(p, q, lengths, out, s);
-    case 4: return launch_typed<T, D, 4>(p, q, lengths, out, s);
-    case 8: return launch_typed<T, D, 8>(p, q, lengths, out, s);
+    case 1: return launch_typed<T, D, 1>(p, q, lengths, k_new, v_new, out, s);
+    case 2: return launch_typed<T, D, 2>(p, q, lengths, k_new, v_new, out, s);
+    case 4: return launch_typed<T, D, 4>(p, q, lengths, k_new, v_new, out, s);
+    case 8: return launch_typed<T, D, 8>(p, q, lengths, k_new, v_new, out, s);
     default: return cudaErrorInvalidValue;
   }
 }
 
 }  // namespace
 
-cudaError_t launch_decode(const DeviceProblem& p, int dtype, const void* q, const int32_t* lengths, void* out,
-                          cudaStream_t s) {
+cudaError_t launch_decode(const DeviceProblem& p, int dtype, const void* q, const int32_t* lengths,
+                          const void* k_new, const void* v_new, void* out, cudaStream_t s) {
   if (dtype == TASKKV_F32)
-    return p.d == 64 ? launch_group<float, 64>(p, q, lengths, out, s) : launch_group<float, 128>(p, q, lengths, out, s);
-  return p.d == 64 ? launch_group<__nv_bfloat16, 64>(p, q, lengths, out, s)
-                   : launch_group<__nv_bfloat16, 128>(p, q, lengths, out, s);
+    return p.d == 64 ? launch_group<float, 64>(p, q, lengths, k_new, v_new, out, s) : launch_group<float, 128>(p, q, lengths, k_new, v_new, out, s);
+  return p.d == 64 ? launch_group<__nv_bfloat16, 64>(p, q, lengths, k_new, v_new, out, s)
+                   : launch_group<__nv_bfloat16, 128>(p, q, lengths, k_new, v_new, out, s);
 }
 
 }  // namespace taskkv

@@ -427,3 +427,44 @@ def test_layer_streamed_compression_equals_all_layer_compression():
         assert torch.equal(got.view(torch.uint8), want_out[:, r:r + 1].contiguous().view(torch.uint8))
         one.close()
     whole.close()
+
+
+@pytest.mark.parametrize("case", [
+    dict(n=8, n_kv=2, d=128, N=0, L=32, s1=4, s2=64, k=100, dtype="bf16", R=2, seq_lens=[1500, 1023], nh=1),
+    dict(n=4, n_kv=4, d=128, N=2047, L=32, s1=4, s2=64, k=60, dtype="bf16", R=2),     # appended rows cross a 512-row item
+    dict(n=4, n_kv=4, d=64, N=900, L=16, s1=4, s2=32, k=50, dtype="f32", R=3),
+], ids=["bf16_gqa_ragged", "bf16_item_boundary", "f32"])
+def test_fused_decode_step_equals_append_then_decode(case):
+    tk = _tk()
+    wl = small("step", **case, steps=4)
+    qs, ks, vs = W.materialize(wl, DEV)
+    params = tk.params_from_workload(wl, max_new_tokens=3)          # the 4th token does not fit
+    two = tk.taskkv_compress_ex(params, qs, ks, vs)
+    one = tk.taskkv_compress_ex(params, qs, ks, vs)
+    for s in range(3):
+        q, kn, vn = W.gen_decode_step(wl, s, DEV)
+        two.taskkv_append(kn, vn)
+        want = two.taskkv_decode(q)
+        if s == 1:      # layer by layer
+            got = torch.empty_like(want)
+            for r in range(wl.n_layers):
+                got[:, r:r + 1] = one.taskkv_decode_step_ex(q[:, r:r + 1].contiguous(), kn[:, r:r + 1].contiguous(),
+                                                            vn[:, r:r + 1].contiguous(), r, 1)
+        else:
+            got = one.taskkv_decode_step(q, kn, vn)
+        assert torch.equal(got.view(torch.uint8), want.view(torch.uint8)), f"step {s}"
+        assert np.array_equal(one.lengths(), two.lengths())
+    assert one.status() == 0
+    for u in (0, int(one.info.n_units) - 1):
+        for which in ("k", "v"):
+            assert torch.equal(one.pool_rows(which, u).view(torch.uint8), two.pool_rows(which, u).view(torch.uint8))
+    # at capacity: the step attends over the rows it has, keeps the lengths and raises the sticky status
+    q, kn, vn = W.gen_decode_step(wl, 3, DEV)
+    before = one.lengths().copy()
+    got = one.taskkv_decode_step(q, kn, vn)
+    want = two.taskkv_decode(q)
+    assert torch.equal(got.view(torch.uint8), want.view(torch.uint8))
+    assert np.array_equal(one.lengths(), before)
+    assert one.status() == tk.ESTATE
+    one.close()
+    two.close()
