@@ -259,6 +259,17 @@ def test_mistral_shaped_ragged_batch():
     run_workload(wl)
 
 
+@pytest.mark.parametrize("case", [
+    dict(n=8, n_kv=8, d=128, N=0, L=32, s1=4, s2=64, k=120, dtype="bf16", R=4, seq_lens=[9000, 7001, 12345], nh=2),
+    dict(n=8, n_kv=4, d=64, N=0, L=32, s1=4, s2=64, k=120, dtype="bf16", R=6, seq_lens=[16384, 15000], nh=1),
+], ids=["32rows_ragged", "64rows_d64"])
+def test_window_scores_many_items_per_cta(case):
+    """Large enough for every CTA of the window-score kernel to run through several work items of several
+    sequences: ragged ends, units that straddle the grid, both tensor-core row counts below 128."""
+    wl = small("rounds", **case, steps=1)
+    run_workload(wl, layers=[(b, r) for b in range(wl.batch) for r in (0, wl.n_layers - 1)])
+
+
 def test_ragged_batch_of_eleven_sequences():
     """More sequences than one window-score launch takes (eight): a full group and a partial one."""
     from paper_2501_15113_b200 import configs
