@@ -109,7 +109,8 @@ POLICIES = {"select": 0, "recent": 1, "mean": 2}
 
 
 def algorithmic_bytes(wl, info, policy="select"):
-    """Bytes the method itself must move: compress and one decode step.  With averaged
+    """Bytes the method itself must move: K once, Q_win, C written once and read about twice, the top-t V rows, and
+    the retained K/V rows read and written by the gather; per decode step every retained K/V row once.  With averaged
     compensation rows every intermediate K and V row of a non-heterogeneous head is read once more."""
     es, d = wl.elem_size, wl.head_dim
     G = wl.group
