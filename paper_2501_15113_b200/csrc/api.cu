@@ -29,7 +29,7 @@ struct HostPlan {
   size_t o_status, o_len, o_cap, o_seg, o_cls, o_dist, o_sem, o_idx, o_goff, o_doff, o_step, o_pacc, o_pml, o_kpool,
       o_vpool;
   // inside the workspace
-  size_t w_C, w_spart, w_stat, w_topt;
+  size_t w_C, w_pool, w_spart, w_stat, w_topt;
 };
 
 int32_t hetero_count_impl(int32_t n, float beta, int32_t m, int32_t R, int32_t r) {
@@ -149,6 +149,8 @@ taskkv_status make_plan(const taskkv_params* p, HostPlan& hp) {
   const size_t cache_bytes = o;
   o = 0;
   hp.w_C = take((size_t)c_total * 4);
+  // the streaming selection of long units keeps the pooled scores beside C
+  hp.w_pool = take(hp.max_N > 32768 || (p->pool_kernel != 7 && p->pool_kernel != 1) ? (size_t)c_total * 4 : 0);
   hp.w_spart = take((size_t)U * hp.chunks_max * hp.rows_pad * 8);
   hp.w_stat = take((size_t)U * hp.rows_pad * 8);
   hp.w_topt = take((size_t)U * p->top_t * 4);
@@ -274,6 +276,7 @@ void fill_device_problem(taskkv_cache* c) {
   d.v_pool = cm + hp.o_vpool;
   if (wm) {
     d.C = reinterpret_cast<float*>(wm + hp.w_C);
+    d.pooled = reinterpret_cast<float*>(wm + hp.w_pool);
     d.stat_part = reinterpret_cast<float*>(wm + hp.w_spart);
     d.stat = reinterpret_cast<float*>(wm + hp.w_stat);
     d.topt = reinterpret_cast<int32_t*>(wm + hp.w_topt);

@@ -82,6 +82,7 @@ struct DeviceProblem {
   float* part_ml;             // [items][G][2]
   // workspace
   float* C;                   // scores, units concatenated
+  float* pooled;              // [sum N] pooling-window sums of C (only for units too long for the register path)
   float* stat_part;           // [U][chunks_max][rows_pad][2]
   float* stat;                // [U][rows_pad][2]  per row: (max in log2 units, 1/Z), or one offset (tensor-core path)
   int32_t* topt;              // [U][top_t]

@@ -3,9 +3,11 @@
 //   the k middle activations: top-k of the average-pooled scores over the
 //   intermediate positions [s1, N - s2) (Sec. IV-B, pooling of Sec. V-D), written
 //   with the sinks and the recent window as the unit's ascending index list.
-// Both selections are an exact block-level radix select on order-preserving
-// 32-bit keys (4 passes of 8 bits) followed by an ordered compaction; of equal
-// scores the lower position wins.
+// Both selections find the exact k-th largest order-preserving 32-bit key by bisection
+// over the key bits, followed by an ordered compaction; of equal scores the lower
+// position wins.  Up to 32768 positions the keys live in registers (select_fast_kernel);
+// longer units stream them from L2 once per bisection step until few enough survive to
+// be collected in shared memory (select_kernel).
 #include "common.cuh"
 
 namespace taskkv {
@@ -28,135 +30,166 @@ struct ScoreKey {          // key of C[j]
   __device__ __forceinline__ uint32_t operator()(int j) const { return ordered_key(C[j]); }
 };
 
-struct PooledKey {         // key of the pooling-window sum around j (zeros outside [0, N))
-  const float* C;
-  int N, half;
-  __device__ __forceinline__ uint32_t operator()(int j) const {
-    float s = 0.f;
-    for (int o = -half; o <= half; ++o) {
-      const int q = j + o;
-      s += (q >= 0 && q < N) ? C[q] : 0.f;
-    }
-    return ordered_key(s);
-  }
+struct SelectSmem {
+  int cnt[2][kWarps];
+  int cnt3[2][3][kWarps];
+  uint32_t mn[kWarps], mx[kWarps];
+  long long scan[kWarps];
+  int list_n;
+  uint32_t list_thr;
 };
 
-struct SelectSmem {
-  int hist[256];
-  int warp_tot[kWarps];
-  uint32_t prefix;
-  int remaining;
-  int run_gt, run_eq, tile_tot;
-};
+// #(key(j) >= cand), j in [lo, hi), over the whole block: one coalesced pass over the keys.
+template <class KeyFn>
+__device__ int stream_count_ge(int lo, int hi, const KeyFn& key, uint32_t cand, int* slot) {
+  int c = 0;
+#pragma unroll 8    // several loads in flight per thread: the pass is bound by L2 latency otherwise
+  for (int j = lo + (int)threadIdx.x; j < hi; j += kThreads) c += key(j) >= cand;
+  c = __reduce_add_sync(0xffffffffu, c);
+  const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+  if (lane == 0) slot[warp] = c;
+  __syncthreads();
+  return __reduce_add_sync(0xffffffffu, slot[lane]);
+}
 
 // Finds the key `thr` of the `want`-th largest element of key(j), j in [lo, hi)
 // (1 <= want <= hi - lo), and how many elements equal to thr belong to the top
 // `want` (need_eq); elements with key > thr number want - need_eq.
+// Bisection over the key bits, one pass over the keys per step, which also tells how many keys still lie in
+// the undecided range [t, t + 2^(bit+1)); once they fit into `list` (shared memory, `cap` entries) they are
+// collected there and one warp settles the remaining bits.
 template <class KeyFn>
-__device__ void block_radix_select(SelectSmem& sm, int lo, int hi, int want, const KeyFn& key,
-                                   uint32_t& thr, int& need_eq) {
-  const int tid = threadIdx.x, lane = tid & 31;
-  if (tid == 0) { sm.prefix = 0u; sm.remaining = want; }
-  uint32_t mask = 0u;
-  const int trips = (hi - lo + kThreads - 1) / kThreads;
-  for (int shift = 24; shift >= 0; shift -= 8) {
-    for (int i = tid; i < 256; i += kThreads) sm.hist[i] = 0;
-    __syncthreads();
-    const uint32_t prefix = sm.prefix;
-    for (int it = 0; it < trips; ++it) {
-      const int j = lo + it * kThreads + tid;
-      int digit = 256;                       // lanes without a candidate element
-      if (j < hi) {
-        const uint32_t kx = key(j);
-        if ((kx & mask) == prefix) digit = (kx >> shift) & 255;
-      }
-      // warp-aggregated histogram: one atomic per distinct digit per warp
-      const unsigned peers = __match_any_sync(0xffffffffu, digit);
-      if (digit < 256 && lane == (__ffs(peers) - 1)) atomicAdd(&sm.hist[digit], __popc(peers));
-    }
-    __syncthreads();
-    if (tid < 32) {
-      // lane l owns bins 255-8l .. 248-8l (descending); find the bin holding the `remaining`-th largest
-      const int remaining = sm.remaining;
-      int local[8], tot = 0;
-#pragma unroll
-      for (int b = 0; b < 8; ++b) { local[b] = sm.hist[255 - 8 * lane - b]; tot += local[b]; }
-      int incl = tot;
-#pragma unroll
-      for (int o = 1; o < 32; o <<= 1) {
-        const int y = __shfl_up_sync(0xffffffffu, incl, o);
-        if (lane >= o) incl += y;
-      }
-      int above = incl - tot;   // elements in bins owned by lower lanes (= larger digits)
-      if (above < remaining && remaining <= incl) {
-#pragma unroll
-        for (int b = 0; b < 8; ++b) {
-          if (above < remaining && remaining <= above + local[b]) {
-            sm.prefix = prefix | ((uint32_t)(255 - 8 * lane - b) << shift);
-            sm.remaining = remaining - above;
-          }
-          above += local[b];
-        }
-      }
-    }
-    mask |= 255u << shift;
-    __syncthreads();
+__device__ void block_stream_select(SelectSmem& sm, int lo, int hi, int want, const KeyFn& key, uint32_t* list,
+                                    int cap, uint32_t& thr, int& need_eq) {
+  const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+  uint32_t kmin = 0xffffffffu, kmax = 0u;
+#pragma unroll 8
+  for (int j = lo + tid; j < hi; j += kThreads) {
+    const uint32_t kx = key(j);
+    kmin = min(kmin, kx);
+    kmax = max(kmax, kx);
   }
-  thr = sm.prefix;
-  need_eq = sm.remaining;
+  kmin = __reduce_min_sync(0xffffffffu, kmin);
+  kmax = __reduce_max_sync(0xffffffffu, kmax);
+  if (lane == 0) { sm.mn[warp] = kmin; sm.mx[warp] = kmax; }
+  if (tid == 0) sm.list_n = 0;
+  __syncthreads();
+  kmin = __reduce_min_sync(0xffffffffu, sm.mn[lane]);
+  kmax = __reduce_max_sync(0xffffffffu, sm.mx[lane]);
+  // bits above the highest bit in which the keys differ are common to the answer
+  const uint32_t diff = kmin ^ kmax;
+  int bit = diff ? 31 - __clz(diff) : -1;
+  uint32_t t = diff ? (kmax & ~((2u << bit) - 1u)) : kmax;
+  int par = 0;
+  int above = 0;             // keys >= t + 2^(bit+1): the last count that fell short of `want`
+  int at_least = hi - lo;    // keys >= t: all of them at the start, then the last count that reached `want`
+  // two bits per pass over the keys (the pass is bound by the L2 stream, three compares per key are free)
+  for (; bit >= 1 && at_least - above > cap; bit -= 2) {
+    const uint32_t c10 = t | (2u << (bit - 1)), c11 = t | (3u << (bit - 1)), c01 = t | (1u << (bit - 1));
+    int n10 = 0, n11 = 0, n01 = 0;
+#pragma unroll 8
+    for (int j = lo + tid; j < hi; j += kThreads) {
+      const uint32_t kx = key(j);
+      n10 += kx >= c10;
+      n11 += kx >= c11;
+      n01 += kx >= c01;
+    }
+    n10 = __reduce_add_sync(0xffffffffu, n10);
+    n11 = __reduce_add_sync(0xffffffffu, n11);
+    n01 = __reduce_add_sync(0xffffffffu, n01);
+    if (lane == 0) { sm.cnt3[par][0][warp] = n10; sm.cnt3[par][1][warp] = n11; sm.cnt3[par][2][warp] = n01; }
+    __syncthreads();
+    n10 = __reduce_add_sync(0xffffffffu, sm.cnt3[par][0][lane]);
+    n11 = __reduce_add_sync(0xffffffffu, sm.cnt3[par][1][lane]);
+    n01 = __reduce_add_sync(0xffffffffu, sm.cnt3[par][2][lane]);
+    par ^= 1;
+    if (n10 >= want) {
+      if (n11 >= want) { t = c11; at_least = n11; } else { t = c10; at_least = n10; above = n11; }
+    } else {
+      if (n01 >= want) { t = c01; at_least = n01; above = n10; } else above = n01;
+    }
+  }
+  for (; bit >= 0 && at_least - above > cap; --bit) {   // an odd bit left over
+    const uint32_t cand = t | (1u << bit);
+    const int c = stream_count_ge(lo, hi, key, cand, sm.cnt[par]);
+    if (c >= want) { t = cand; at_least = c; } else above = c;
+    par ^= 1;
+  }
+  if (bit >= 0) {
+    const uint32_t top = t + (2u << bit);            // end of the undecided range (0 if it wraps: no upper bound)
+    const int alive = at_least - above;
+#pragma unroll 8
+    for (int j = lo + tid; j < hi; j += kThreads) {
+      const uint32_t kx = key(j);
+      if (kx >= t && (top == 0u || kx < top)) list[atomicAdd(&sm.list_n, 1)] = kx;
+    }
+    __syncthreads();
+    if (warp == 0) {
+      const int want2 = want - above;                 // rank inside the collected keys
+      for (; bit >= 0; --bit) {
+        const uint32_t cand = t | (1u << bit);
+        int c = 0;
+        for (int i = lane; i < alive; i += 32) c += list[i] >= cand;
+        c = __reduce_add_sync(0xffffffffu, c);
+        if (c >= want2) t = cand;
+      }
+      if (lane == 0) sm.list_thr = t;
+    }
+    __syncthreads();
+    t = sm.list_thr;
+  }
+  const int n_gt = (t == 0xffffffffu) ? 0 : stream_count_ge(lo, hi, key, t + 1u, sm.cnt[par]);
+  thr = t;
+  need_eq = want - n_gt;
   __syncthreads();
 }
 
 // Writes, ascending, every j in [lo, hi) with key > thr plus the first need_eq
-// with key == thr.  emit(pos, j) receives the output slot.
+// with key == thr.  emit(pos, j) receives the output slot.  Every warp owns a contiguous stretch of positions
+// and walks it 32 at a time (coalesced): one pass counts, one block scan places the stretches, one pass
+// ranks by ballot and writes.
 template <class KeyFn, class Emit>
 __device__ void block_compact(SelectSmem& sm, int lo, int hi, uint32_t thr, int need_eq, const KeyFn& key,
                               const Emit& emit) {
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
-  if (tid == 0) { sm.run_gt = 0; sm.run_eq = 0; }
-  __syncthreads();
-  const int trips = (hi - lo + kThreads - 1) / kThreads;
-  for (int it = 0; it < trips; ++it) {
-    const int j = lo + it * kThreads + tid;
-    int gt = 0, eq = 0;
-    if (j < hi) {
-      const uint32_t kx = key(j);
-      gt = kx > thr;
-      eq = kx == thr;
-    }
-    // block exclusive scan of the packed pair (gt in the low half, eq in the high half)
-    const int packed = gt | (eq << 16);
-    int incl = packed;
-#pragma unroll
-    for (int o = 1; o < 32; o <<= 1) {
-      const int y = __shfl_up_sync(0xffffffffu, incl, o);
-      if (lane >= o) incl += y;
-    }
-    if (lane == 31) sm.warp_tot[warp] = incl;
-    __syncthreads();
-    if (warp == 0) {
-      const int w = sm.warp_tot[lane];
-      int wi = w;
-#pragma unroll
-      for (int o = 1; o < 32; o <<= 1) {
-        const int y = __shfl_up_sync(0xffffffffu, wi, o);
-        if (lane >= o) wi += y;
-      }
-      sm.warp_tot[lane] = wi - w;   // exclusive prefix of the warp totals
-      if (lane == 31) sm.tile_tot = wi;
-    }
-    __syncthreads();
-    const int excl = incl - packed + sm.warp_tot[warp];
-    const int gt_before = sm.run_gt + (excl & 0xffff);
-    const int eq_before = sm.run_eq + (excl >> 16);
-    if (gt || (eq && eq_before < need_eq)) emit(gt_before + min(eq_before, need_eq), j);
-    __syncthreads();
-    if (tid == 0) {
-      sm.run_gt += sm.tile_tot & 0xffff;
-      sm.run_eq += sm.tile_tot >> 16;
-    }
-    __syncthreads();
+  const int stretch = ((hi - lo + kWarps - 1) / kWarps + 31) & ~31;
+  const int j0 = min(hi, lo + warp * stretch), j1 = min(hi, j0 + stretch);
+  int gt = 0, eq = 0;
+#pragma unroll 4
+  for (int j = j0 + lane; j < j1; j += 32) {
+    const uint32_t kx = key(j);
+    gt += kx > thr;
+    eq += kx == thr;
   }
+  gt = __reduce_add_sync(0xffffffffu, gt);
+  eq = __reduce_add_sync(0xffffffffu, eq);
+  if (lane == 0) sm.scan[warp] = (long long)gt | ((long long)eq << 32);
+  __syncthreads();
+  const long long wp = sm.scan[lane];
+  long long wi = wp;
+#pragma unroll
+  for (int o = 1; o < 32; o <<= 1) {
+    const long long y = __shfl_up_sync(0xffffffffu, wi, o);
+    if (lane >= o) wi += y;
+  }
+  const long long wexcl = __shfl_sync(0xffffffffu, wi - wp, warp);
+  int gt_before = (int)(wexcl & 0xffffffffll), eq_before = (int)(wexcl >> 32);
+  const unsigned lt = (1u << lane) - 1u;
+  for (int jb = j0; jb < j1; jb += 32) {              // warp-uniform trip count
+    const int j = jb + lane;
+    bool g = false, q = false;
+    if (j < j1) {
+      const uint32_t kx = key(j);
+      g = kx > thr;
+      q = kx == thr;
+    }
+    const unsigned gm = __ballot_sync(0xffffffffu, g), qm = __ballot_sync(0xffffffffu, q);
+    const int my_gt = gt_before + __popc(gm & lt), my_eq = eq_before + __popc(qm & lt);
+    if (g || (q && my_eq < need_eq)) emit(my_gt + min(my_eq, need_eq), j);
+    gt_before += __popc(gm);
+    eq_before += __popc(qm);
+  }
+  __syncthreads();
 }
 
 template <typename T, int D>
@@ -175,7 +208,8 @@ __global__ void __launch_bounds__(kThreads) select_kernel(DeviceProblem p) {
   uint32_t thr;
   int need_eq;
   const ScoreKey skey{C};
-  block_radix_select(sm, 0, N, t, skey, thr, need_eq);
+  uint32_t* scratch = reinterpret_cast<uint32_t*>(&red[0][0]);   // free until the semantic vector is summed
+  block_stream_select(sm, 0, N, t, skey, scratch, kWarps * D, thr, need_eq);
   int* topt = p.topt + (size_t)u * p.top_t;
   block_compact(sm, 0, N, thr, need_eq, skey, [&](int pos, int j) {
     sel[pos] = j;
@@ -224,10 +258,30 @@ __global__ void __launch_bounds__(kThreads) select_kernel(DeviceProblem p) {
     return;
   }
   if (kmid > 0) {
-    const PooledKey pkey{C, N, (p.pool_w - 1) / 2};
+    // the pooling-window sums once, into the unit's scratch row, then selected like plain scores
+    const int half = (p.pool_w - 1) / 2;
+    float* P = p.pooled + p.c_off[u];
+#pragma unroll 2
+    for (int j = tid; j < N; j += kThreads) {
+      float sum = 0.f;                      // added in ascending position, zeros outside [0, N)
+      if (j >= half && j + half < N) {
+        if (half == 3) {
+          sum = C[j - 3]; sum += C[j - 2]; sum += C[j - 1]; sum += C[j]; sum += C[j + 1]; sum += C[j + 2]; sum += C[j + 3];
+        } else {
+          for (int o = -half; o <= half; ++o) sum += C[j + o];
+        }
+      } else {
+        for (int o = -half; o <= half; ++o) {
+          const int q = j + o;
+          sum += (q >= 0 && q < N) ? C[q] : 0.f;
+        }
+      }
+      P[j] = sum;
+    }
     __syncthreads();
-    block_radix_select(sm, lo, hi, kmid, pkey, thr, need_eq);
-    block_compact(sm, lo, hi, thr, need_eq, pkey, [&](int pos, int j) { idx[s1 + pos] = j; });
+    const ScoreKey qkey{P};
+    block_stream_select(sm, lo, hi, kmid, qkey, scratch, kWarps * D, thr, need_eq);
+    block_compact(sm, lo, hi, thr, need_eq, qkey, [&](int pos, int j) { idx[s1 + pos] = j; });
   }
 }
 

@@ -128,6 +128,9 @@ CASES = [
     dict(n=4, n_kv=4, d=64, N=1000, L=8, s1=4, s2=32, k=20, dtype="bf16", nh=0, promote=False),
     # several layers and a ragged batch
     dict(n=16, n_kv=4, d=128, N=0, L=32, s1=4, s2=128, k=256, dtype="bf16", R=3, seq_lens=[1500, 2049, 1024], nh=1),
+    # pooling kernels other than 1 and 7 take the streaming selection: all keys collected at once / after some steps
+    dict(n=4, n_kv=4, d=64, N=1900, L=16, s1=4, s2=32, k=77, dtype="bf16", pool=5),
+    dict(n=4, n_kv=4, d=64, N=9000, L=16, s1=5, s2=33, k=1500, dtype="f32", pool=3),
 ]
 
 
