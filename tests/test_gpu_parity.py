@@ -482,3 +482,25 @@ def test_fused_decode_step_equals_append_then_decode(case):
     assert one.status() == tk.ESTATE
     one.close()
     two.close()
+
+
+def _random_case(seed: int) -> dict:
+    r = np.random.default_rng(seed)
+    n_kv = int(r.choice([1, 2, 4, 8]))
+    G = int(r.choice([1, 2, 4, 8]))
+    L = int(r.choice([l for l in (1, 8, 16, 32) if G * l <= 128]))
+    d = int(r.choice([64, 128]))
+    s1, s2 = int(r.integers(0, 9)), int(r.integers(1, 81))
+    B = int(r.integers(1, 4))
+    lens = [int(r.integers(max(L, s1 + s2 + 2, 40), 4000)) for _ in range(B)]
+    return dict(n=n_kv * G, n_kv=n_kv, d=d, N=0, L=L, s1=s1, s2=s2, k=int(r.integers(0, 300)),
+                dtype=str(r.choice(["bf16", "f32"])), R=int(r.integers(1, 3)), seq_lens=lens,
+                pool=int(r.choice([1, 3, 5, 7])), nh=int(r.integers(0, n_kv + 1)), seed=100 + seed)
+
+
+@pytest.mark.parametrize("seed", list(range(16)))
+def test_random_shapes(seed):
+    """Seeded random problem shapes (head counts, group sizes, window, pooling kernel, ragged batch, budgets)."""
+    case = _random_case(seed)
+    wl = small(f"random{seed}", **case, steps=2)
+    run_workload(wl)
