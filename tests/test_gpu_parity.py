@@ -237,6 +237,35 @@ def test_llama2_config_full_size_sampled_layers():
     assert rep.units == 96
 
 
+def test_llama3_config_full_size_sampled_layers():
+    """Config 3 at full size (32 layers, 32 query / 8 KV heads, 131072 tokens, bf16, 40 % budget), in the launch
+    configuration bench.py times: 128 window rows, streaming selection, warp-mma decode with four heads per KV
+    head.  The oracle checks one layer of each budget (Eq. 16 gives 2 far heads up to layer 19, then 1), then
+    two decode steps."""
+    from paper_2501_15113_b200 import configs
+    wl = configs.config3_llama3()
+    rep = run_workload(wl, layers=[(0, 1), (0, 30)], decode_steps=2, check_pool=False)
+    assert rep.class_near_ties == 0
+    assert rep.units == 16
+
+
+def test_sweep_config_full_size_sampled_sequences():
+    """Config 5 at full size (8 sequences of 65536 tokens, one layer, 2 planted heads, 256 middle positions):
+    the oracle checks two of the sequences."""
+    from paper_2501_15113_b200 import configs
+    wl = configs.config5_sweep(2, 256, decode_steps=2)
+    rep = run_workload(wl, layers=[(0, 0), (5, 0)], decode_steps=2, check_pool=False)
+    assert rep.class_near_ties == 0
+
+
+def test_mistral_config_full_size_sampled_layers():
+    """Config 4 at full size (16 ragged sequences of 8192-32768 tokens, 32 layers, grouped queries): the oracle
+    checks one layer of three sequences, then two decode steps."""
+    from paper_2501_15113_b200 import configs
+    wl = configs.config4_mistral(decode_steps=2)
+    run_workload(wl, layers=[(0, 0), (7, 17), (15, 31)], decode_steps=2, check_pool=False)
+
+
 def test_llama3_shaped_gqa_with_budget_schedule():
     """Config 3 scaled down: GQA 32q / 8kv, Eq. 16 schedule over the KV heads, Eq. 17 budgets for a 40 %
     cache, 128 window rows on the tensor-core path."""
