@@ -167,6 +167,13 @@ __device__ __forceinline__ void tc_ld32(uint32_t taddr, uint32_t* r) {
       : "r"(taddr)
       : "memory");
 }
+__device__ __forceinline__ void tc_ld64(uint32_t taddr, uint32_t* r) {
+  asm volatile(
+      "tcgen05.ld.sync.aligned.32x32b.x64.b32 {%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15, %16, %17, %18, %19, %20, %21, %22, %23, %24, %25, %26, %27, %28, %29, %30, %31, %32, %33, %34, %35, %36, %37, %38, %39, %40, %41, %42, %43, %44, %45, %46, %47, %48, %49, %50, %51, %52, %53, %54, %55, %56, %57, %58, %59, %60, %61, %62, %63}, [%64];"
+      : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7]), "=r"(r[8]), "=r"(r[9]), "=r"(r[10]), "=r"(r[11]), "=r"(r[12]), "=r"(r[13]), "=r"(r[14]), "=r"(r[15]), "=r"(r[16]), "=r"(r[17]), "=r"(r[18]), "=r"(r[19]), "=r"(r[20]), "=r"(r[21]), "=r"(r[22]), "=r"(r[23]), "=r"(r[24]), "=r"(r[25]), "=r"(r[26]), "=r"(r[27]), "=r"(r[28]), "=r"(r[29]), "=r"(r[30]), "=r"(r[31]), "=r"(r[32]), "=r"(r[33]), "=r"(r[34]), "=r"(r[35]), "=r"(r[36]), "=r"(r[37]), "=r"(r[38]), "=r"(r[39]), "=r"(r[40]), "=r"(r[41]), "=r"(r[42]), "=r"(r[43]), "=r"(r[44]), "=r"(r[45]), "=r"(r[46]), "=r"(r[47]), "=r"(r[48]), "=r"(r[49]), "=r"(r[50]), "=r"(r[51]), "=r"(r[52]), "=r"(r[53]), "=r"(r[54]), "=r"(r[55]), "=r"(r[56]), "=r"(r[57]), "=r"(r[58]), "=r"(r[59]), "=r"(r[60]), "=r"(r[61]), "=r"(r[62]), "=r"(r[63])
+      : "r"(taddr)
+      : "memory");
+}
 __device__ __forceinline__ void tc_wait_ld() { asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory"); }
 __device__ __forceinline__ float ex2(float x) {
   float y;
@@ -434,24 +441,24 @@ window_tc_kernel(const __grid_constant__ TcMaps maps, DeviceProblem p, const __g
           // a TMEM lane is a window row (quad * 32 + lane), the 128 columns are the keys of the tile
           const int pos = N - L + ((quad * 32 + lane) % L);   // last key this window row may see
 #pragma unroll
-          for (int cg = 0; cg < 4; ++cg) {
-            uint32_t r[32];
-            tc_ld32(taddr + (uint32_t)(cg * 32), r);
+          for (int cg = 0; cg < 2; ++cg) {               // 64 keys per TMEM load
+            uint32_t r[64];
+            tc_ld64(taddr + (uint32_t)(cg * 64), r);
             tc_wait_ld();
-            float x[32];
+            float x[64];
             if (!tail) {
 #pragma unroll
-              for (int k = 0; k < 32; ++k) x[k] = __uint_as_float(r[k]);
+              for (int k = 0; k < 64; ++k) x[k] = __uint_as_float(r[k]);
             } else {
 #pragma unroll
-              for (int k = 0; k < 32; ++k) {
-                const int j = tbase + cg * 32 + k;
+              for (int k = 0; k < 64; ++k) {
+                const int j = tbase + cg * 64 + k;
                 x[k] = (j <= pos && j < N) ? __uint_as_float(r[k]) : -INFINITY;
               }
             }
             float cm4[4] = {-INFINITY, -INFINITY, -INFINITY, -INFINITY};
 #pragma unroll
-            for (int k = 0; k < 32; ++k) cm4[k & 3] = fmaxf(cm4[k & 3], x[k]);
+            for (int k = 0; k < 64; ++k) cm4[k & 3] = fmaxf(cm4[k & 3], x[k]);
             const float cm = fmaxf(fmaxf(cm4[0], cm4[1]), fmaxf(cm4[2], cm4[3]));
             if (cm > m_run[0]) {
               z_run[0] *= ex2((m_run[0] - cm) * scale2);
@@ -461,7 +468,7 @@ window_tc_kernel(const __grid_constant__ TcMaps maps, DeviceProblem p, const __g
               const float ms = -m_run[0] * scale2;
               float zs[4] = {0.f, 0.f, 0.f, 0.f};
 #pragma unroll
-              for (int k = 0; k < 32; ++k) zs[k & 3] += ex2(fmaf(x[k], scale2, ms));
+              for (int k = 0; k < 64; ++k) zs[k & 3] += ex2(fmaf(x[k], scale2, ms));
               z_run[0] += (zs[0] + zs[1]) + (zs[2] + zs[3]);
             }
           }
@@ -511,6 +518,23 @@ window_tc_kernel(const __grid_constant__ TcMaps maps, DeviceProblem p, const __g
         } else {
           const int j = tbase + quad * 32 + lane;   // this thread's key
           float cs[4] = {0.f, 0.f, 0.f, 0.f};   // four interleaved chains (FMA latency)
+          if (rows >= 64 && !tail) {
+            // 64 columns per TMEM load: half the load / wait round trips of the 32-column walk below
+            for (int c0 = 0; c0 < rows; c0 += 64) {
+              uint32_t r[64];
+              tc_ld64(taddr + (uint32_t)c0, r);
+              tc_wait_ld();
+              const float4* st4 = reinterpret_cast<const float4*>(myStat + c0);   // four rows per 16-byte load
+#pragma unroll
+              for (int c = 0; c < 64; c += 4) {
+                const float4 off = st4[c >> 2];
+                cs[0] += ex2(fmaf(__uint_as_float(r[c]), scale2, -off.x));
+                cs[1] += ex2(fmaf(__uint_as_float(r[c + 1]), scale2, -off.y));
+                cs[2] += ex2(fmaf(__uint_as_float(r[c + 2]), scale2, -off.z));
+                cs[3] += ex2(fmaf(__uint_as_float(r[c + 3]), scale2, -off.w));
+              }
+            }
+          } else
           for (int c0 = 0; c0 < rows; c0 += 32) {
             uint32_t r[32];
             tc_ld32(taddr + (uint32_t)c0, r);
