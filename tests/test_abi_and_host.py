@@ -84,7 +84,7 @@ def test_invalid_arguments_are_rejected_before_any_launch(tk):
     tk.taskkv_plan(tk.Params(**good))
     bad = [dict(head_dim=96), dict(n_kv_heads=3), dict(window=0), dict(window=1024), dict(seq_lens=[8]),
            dict(top_t=5000), dict(pool_kernel=4), dict(sink=-1), dict(n_heads=8 * 16, n_kv_heads=8),
-           dict(mid_budget=-2), dict(force_class=7), dict(seq_lens=[0])]
+           dict(mid_budget=-2), dict(force_class=7), dict(seq_lens=[0]), dict(mid_policy=3), dict(mid_policy=-1)]
     for override in bad:
         kw = dict(good)
         kw.update(override)
@@ -96,6 +96,10 @@ def test_invalid_arguments_are_rejected_before_any_launch(tk):
     assert tk.lib.taskkv_compress_ex(None, None, None, None, None, 0, None, 0, None, C.byref(h)) == tk.EINVAL
     assert tk.lib.taskkv_decode(None, None, None, None, None) == tk.EINVAL
     assert tk.lib.taskkv_append(None, None, None, None) == tk.EINVAL
+    assert tk.lib.taskkv_append_ex(None, None, None, 0, 1, None) == tk.EINVAL
+    assert tk.lib.taskkv_decode_ex(None, None, None, None, 0, 1, None) == tk.EINVAL
+    assert tk.lib.taskkv_decode_step(None, None, None, None, None, None) == tk.EINVAL
+    assert tk.lib.taskkv_decode_step_ex(None, None, None, None, None, 0, 1, None) == tk.EINVAL
     assert tk.lib.taskkv_cache_query(None, 0, None, 0) == tk.EINVAL
     assert tk.lib.taskkv_status_str(tk.ESTATE) == b"cache in wrong state"
     assert wl.retained_rows() == 3 * 512 + 5 * 68
