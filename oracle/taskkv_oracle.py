@@ -77,6 +77,21 @@ def window_attention(q_win: np.ndarray, k: np.ndarray) -> np.ndarray:
     return e / e.sum(axis=1, keepdims=True)
 
 
+def window_lse(q_win: np.ndarray, k: np.ndarray) -> np.ndarray:
+    """Natural-log normaliser of every row of Eq. 12: lse_i = log sum_j exp(s_ij) over the keys row i may see, so
+    that A'[i, j] = exp(s_ij - lse_i).  This is what an attention kernel run over the prompt returns as its
+    log-sum-exp for the last L query rows; a caller that has it can hand it over instead of having it recomputed."""
+    q_win = np.asarray(q_win, dtype=F64)
+    k = np.asarray(k, dtype=F64)
+    L, d = q_win.shape
+    N = k.shape[0]
+    s = (q_win @ k.T) / math.sqrt(d)
+    pos = N - L + np.arange(L)
+    s = np.where(np.arange(N)[None, :] > pos[:, None], -np.inf, s)
+    m = s.max(axis=1)
+    return m + np.log(np.exp(s - m[:, None]).sum(axis=1))
+
+
 def column_mean(a_rows: np.ndarray) -> np.ndarray:
     """Eq. 13: C = sum_i A'[i,:] / L, a vector of length N.
 

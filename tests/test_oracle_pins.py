@@ -416,3 +416,19 @@ def test_policy_pipeline_lengths_and_classes_do_not_depend_on_the_policy():
         for u in range(k.shape[0]):
             if out["cls"][u] != 0:
                 np.testing.assert_array_equal(kc[u], k[u])
+
+
+def test_window_lse_is_the_normaliser_of_eq12():
+    r = rng(31)
+    L, N, d = 6, 40, 8
+    q, k = r.normal(size=(L, d)) * 2, r.normal(size=(N, d)) * 2
+    lse = O.window_lse(q, k)
+    a = O.window_attention(q, k)
+    s = (q @ k.T) / math.sqrt(d)
+    for i in range(L):
+        p_i = N - L + i
+        # library cross-check on the visible keys of row i, and A' = exp(s - lse) entry by entry
+        ref = torch.logsumexp(torch.from_numpy(s[i, :p_i + 1]), dim=0).item()
+        assert abs(lse[i] - ref) < 1e-12
+        np.testing.assert_allclose(np.exp(s[i, :p_i + 1] - lse[i]), a[i, :p_i + 1], rtol=1e-12, atol=0)
+        assert np.all(a[i, p_i + 1:] == 0)
