@@ -141,6 +141,19 @@ taskkv_status taskkv_compress_ex(const taskkv_params* p, const void* const* q_wi
                                  void* workspace_mem, size_t workspace_bytes,
                                  taskkv_stream stream, taskkv_cache** out_cache);
 
+/* As taskkv_compress_ex, for callers that already hold the normalisers of the observation window's rows:
+ *   window_lse[b]  device fp32 [n_layers][n_heads][L], lse_i = ln sum_j exp(q_i . k_j / sqrt(d)) over the keys
+ *                  j <= position of window row i -- what an attention kernel run over the prompt returns as the
+ *                  log-sum-exp of its last L query rows.
+ * With them A'[i, j] = exp(s_ij - lse_i) (Eq. 12) needs no pass over K for the row sums, so the window scores
+ * read K once instead of twice.  Results equal those of taskkv_compress_ex up to the rounding of the supplied
+ * values.  window_lse itself is a host array of `batch` device pointers. */
+taskkv_status taskkv_compress_lse(const taskkv_params* p, const void* const* q_win, const void* const* k,
+                                  const void* const* v, const void* const* window_lse,
+                                  void* cache_mem, size_t cache_bytes,
+                                  void* workspace_mem, size_t workspace_bytes,
+                                  taskkv_stream stream, taskkv_cache** out_cache);
+
 /* Layer at a time.  Nothing couples the layers of a sequence except the schedules of Eq. 16 / Eq. 17, which
  * are known before any data: a prefill loop can therefore compress layer r as soon as its K and V exist, as a
  * problem of its own with n_layers = 1, n_hetero = { f(r) } (taskkv_hetero_count with the model's R and r) and

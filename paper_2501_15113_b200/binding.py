@@ -57,6 +57,9 @@ lib.taskkv_plan.restype = C.c_int32
 lib.taskkv_compress_ex.argtypes = [C.POINTER(taskkv_params), _pp, _pp, _pp, _vp, C.c_size_t, _vp, C.c_size_t,
                                    _vp, C.POINTER(_vp)]
 lib.taskkv_compress_ex.restype = C.c_int32
+lib.taskkv_compress_lse.argtypes = [C.POINTER(taskkv_params), _pp, _pp, _pp, _pp, _vp, C.c_size_t, _vp, C.c_size_t,
+                                    _vp, C.POINTER(_vp)]
+lib.taskkv_compress_lse.restype = C.c_int32
 lib.taskkv_compress.argtypes = [_vp, _vp, _vp] + [C.c_int32] * 9 + [_vp, C.POINTER(_vp)]
 lib.taskkv_compress.restype = C.c_int32
 lib.taskkv_compress_host.argtypes = [C.POINTER(taskkv_params), _pp, _pp, _pp, _vp, C.POINTER(_vp)]
@@ -349,9 +352,11 @@ class Cache:
 
 def taskkv_compress_ex(params: Params, q_win: Sequence[torch.Tensor], k: Sequence[torch.Tensor],
                        v: Sequence[torch.Tensor], stream=None, cache_mem: Optional[torch.Tensor] = None,
-                       workspace_mem: Optional[torch.Tensor] = None) -> Cache:
+                       workspace_mem: Optional[torch.Tensor] = None,
+                       window_lse: Optional[Sequence[torch.Tensor]] = None) -> Cache:
     """q_win[b]: [R, n, L, d]; k[b], v[b]: [R, n_kv, N_b, d] contiguous CUDA tensors.
-    Cache and workspace memory are torch allocations unless supplied."""
+    Cache and workspace memory are torch allocations unless supplied.  window_lse[b] (fp32 [R, n, L], optional):
+    the log-sum-exp of the window rows from the prompt's attention; then taskkv_compress_lse is called."""
     info = taskkv_plan(params)
     dev = k[0].device
     if cache_mem is None:
@@ -363,6 +368,15 @@ def taskkv_compress_ex(params: Params, q_win: Sequence[torch.Tensor], k: Sequenc
             raise ValueError("inputs must be contiguous CUDA tensors")
     qa, ka, va = _ptr_array(q_win), _ptr_array(k), _ptr_array(v)
     h = C.c_void_p()
+    if window_lse is not None:
+        for t in window_lse:
+            if not t.is_contiguous() or not t.is_cuda or t.dtype != torch.float32:
+                raise ValueError("window_lse must be contiguous fp32 CUDA tensors")
+        la = _ptr_array(window_lse)
+        _check(lib.taskkv_compress_lse(C.byref(params.c), qa, ka, va, la, cache_mem.data_ptr(), cache_mem.numel(),
+                                       workspace_mem.data_ptr(), workspace_mem.numel(), _stream_handle(stream),
+                                       C.byref(h)), "taskkv_compress_lse")
+        return Cache(h.value, params, {"cache": cache_mem, "workspace": workspace_mem, "lse": list(window_lse)})
     _check(lib.taskkv_compress_ex(C.byref(params.c), qa, ka, va, cache_mem.data_ptr(), cache_mem.numel(),
                                   workspace_mem.data_ptr(), workspace_mem.numel(), _stream_handle(stream),
                                   C.byref(h)), "taskkv_compress_ex")

@@ -355,10 +355,35 @@ taskkv_status taskkv_plan(const taskkv_params* p, taskkv_plan_info* out) {
   return TASKKV_OK;
 }
 
+namespace {
+taskkv_status compress_impl(const taskkv_params* p, const void* const* q_win, const void* const* k,
+                            const void* const* v, const void* const* window_lse, void* cache_mem,
+                            size_t cache_bytes, void* workspace_mem, size_t workspace_bytes, taskkv_stream stream,
+                            taskkv_cache** out_cache);
+}  // namespace
+
 taskkv_status taskkv_compress_ex(const taskkv_params* p, const void* const* q_win, const void* const* k,
                                  const void* const* v, void* cache_mem, size_t cache_bytes,
                                  void* workspace_mem, size_t workspace_bytes, taskkv_stream stream,
                                  taskkv_cache** out_cache) {
+  return compress_impl(p, q_win, k, v, nullptr, cache_mem, cache_bytes, workspace_mem, workspace_bytes, stream,
+                       out_cache);
+}
+
+taskkv_status taskkv_compress_lse(const taskkv_params* p, const void* const* q_win, const void* const* k,
+                                  const void* const* v, const void* const* window_lse, void* cache_mem,
+                                  size_t cache_bytes, void* workspace_mem, size_t workspace_bytes,
+                                  taskkv_stream stream, taskkv_cache** out_cache) {
+  if (!window_lse) return TASKKV_EINVAL;
+  return compress_impl(p, q_win, k, v, window_lse, cache_mem, cache_bytes, workspace_mem, workspace_bytes, stream,
+                       out_cache);
+}
+
+namespace {
+taskkv_status compress_impl(const taskkv_params* p, const void* const* q_win, const void* const* k,
+                            const void* const* v, const void* const* window_lse, void* cache_mem,
+                            size_t cache_bytes, void* workspace_mem, size_t workspace_bytes, taskkv_stream stream,
+                            taskkv_cache** out_cache) {
   if (!p || !q_win || !k || !v || !out_cache) return TASKKV_EINVAL;
   *out_cache = nullptr;
   taskkv_cache* c = new (std::nothrow) taskkv_cache();
@@ -367,6 +392,10 @@ taskkv_status taskkv_compress_ex(const taskkv_params* p, const void* const* q_wi
   if (st != TASKKV_OK) { delete c; return st; }
   for (int b = 0; b < p->batch; ++b) {
     if (!q_win[b] || !k[b] || !v[b] || ((uintptr_t)q_win[b] | (uintptr_t)k[b] | (uintptr_t)v[b]) & 15) {
+      delete c;
+      return TASKKV_EINVAL;
+    }
+    if (window_lse && (!window_lse[b] || ((uintptr_t)window_lse[b] & 3))) {
       delete c;
       return TASKKV_EINVAL;
     }
@@ -418,6 +447,7 @@ taskkv_status taskkv_compress_ex(const taskkv_params* p, const void* const* q_wi
   wh.seq_lens = c->hp.seq_lens.data();
   wh.q = q_win;
   wh.k = k;
+  wh.lse = window_lse;
   if (e == cudaSuccess) e = launch_window_scores(c->dp, p->dtype, c->hp.max_N, wh, s);
   if (e == cudaSuccess) e = launch_select(c->dp, p->dtype, c->hp.max_N, s);
   if (e == cudaSuccess) e = launch_separator_plan(c->dp, p->batch * p->n_layers, s);
@@ -431,6 +461,7 @@ taskkv_status taskkv_compress_ex(const taskkv_params* p, const void* const* q_wi
   *out_cache = c;
   return TASKKV_OK;
 }
+}  // namespace
 
 taskkv_status taskkv_compress(const void* q_win, const void* k, const void* v, int32_t n_layers,
                               int32_t n_heads, int32_t n_kv_heads, int32_t head_dim, int32_t seq_len,

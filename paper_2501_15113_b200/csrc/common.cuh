@@ -105,7 +105,13 @@ struct WindowHostInfo {
   const int32_t* seq_lens;      // host [batch]
   const void* const* q;         // host [batch] device pointers: [R][n][L][d]
   const void* const* k;         // host [batch] device pointers: [R][n_kv][N_b][d]
+  const void* const* lse;       // host [batch] device pointers to fp32 [R][n][L] natural-log normalisers of the
+                                // window rows, or nullptr: then pass 1 computes them
 };
+
+// Row statistics from caller-supplied normalisers (replaces pass 1): units [u0, u0 + n_units) of one sequence.
+cudaError_t launch_lse_to_stat(const DeviceProblem& p, int u0, int n_units, const float* lse, bool tensor_core_format,
+                               cudaStream_t s);
 
 // kernel launchers (one per translation unit)
 cudaError_t launch_window_scores(const DeviceProblem& p, int dtype, int max_N, const WindowHostInfo& h,

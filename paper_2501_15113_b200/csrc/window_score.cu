@@ -155,8 +155,20 @@ __global__ void window_reduce_kernel(DeviceProblem p) {
   reinterpret_cast<float2*>(p.stat)[(size_t)u * p.rows_pad + row] = out;
 }
 
+// Caller-supplied normalisers lse_i = ln sum_j exp(s_ij) of the window rows, in place of pass 1.  A unit's G*L rows
+// are contiguous in [R][n][L].  Tensor-core path: one offset per row, lse * log2(e) + log2(rows); here: the pair
+// (reference, 1 / sum relative to it) = (lse * log2(e), 1).
+__global__ void lse_to_stat_kernel(DeviceProblem p, int u0, const float* __restrict__ lse, int tc_format) {
+  const int lu = blockIdx.x, row = threadIdx.x;
+  if (row >= p.rows) return;
+  const float v = lse[(size_t)lu * p.rows + row] * kLog2e;
+  const size_t u = (size_t)(u0 + lu);
+  if (tc_format) p.stat[u * (2 * p.rows_pad) + row] = v + log2f((float)p.rows);
+  else reinterpret_cast<float2*>(p.stat)[u * p.rows_pad + row] = make_float2(v, 1.0f);
+}
+
 template <typename T, int D>
-cudaError_t launch_generic(const DeviceProblem& p, int max_N, cudaStream_t s) {
+cudaError_t launch_generic(const DeviceProblem& p, int max_N, const WindowHostInfo& h, cudaStream_t s) {
   const size_t smem = (size_t)p.rows_pad * D * sizeof(float) + (size_t)kTile * WinSmem<T, D>::kRowBytes +
                       (size_t)p.rows_pad * 4 * sizeof(float2);
   cudaError_t e;
@@ -165,13 +177,21 @@ cudaError_t launch_generic(const DeviceProblem& p, int max_N, cudaStream_t s) {
   e = cudaFuncSetAttribute(window_pass_kernel<T, D, 2>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
   if (e != cudaSuccess) return e;
   const dim3 grid((max_N + kScoreChunk - 1) / kScoreChunk, p.U);
-  {
-    LaunchScope ls(K_WINDOW_STATS, s);
-    window_pass_kernel<T, D, 1><<<grid, kTile, smem, s>>>(p);
-  }
-  {
-    LaunchScope ls(K_WINDOW_REDUCE, s);
-    window_reduce_kernel<<<p.U, p.rows_pad, 0, s>>>(p);
+  if (h.lse) {
+    const int per_seq = p.R * p.n_kv;
+    for (int b = 0; b < h.batch; ++b) {
+      e = launch_lse_to_stat(p, b * per_seq, per_seq, static_cast<const float*>(h.lse[b]), false, s);
+      if (e != cudaSuccess) return e;
+    }
+  } else {
+    {
+      LaunchScope ls(K_WINDOW_STATS, s);
+      window_pass_kernel<T, D, 1><<<grid, kTile, smem, s>>>(p);
+    }
+    {
+      LaunchScope ls(K_WINDOW_REDUCE, s);
+      window_reduce_kernel<<<p.U, p.rows_pad, 0, s>>>(p);
+    }
   }
   {
     LaunchScope ls(K_WINDOW_SCORES, s);
@@ -182,15 +202,22 @@ cudaError_t launch_generic(const DeviceProblem& p, int max_N, cudaStream_t s) {
 
 }  // namespace
 
+cudaError_t launch_lse_to_stat(const DeviceProblem& p, int u0, int n_units, const float* lse, bool tensor_core_format,
+                               cudaStream_t s) {
+  LaunchScope ls(K_WINDOW_REDUCE, s);
+  lse_to_stat_kernel<<<n_units, 128, 0, s>>>(p, u0, lse, tensor_core_format ? 1 : 0);
+  return cudaGetLastError();
+}
+
 cudaError_t launch_window_scores(const DeviceProblem& p, int dtype, int max_N, const WindowHostInfo& h,
                                  cudaStream_t s) {
   // bf16 with 32 / 64 / 128 window rows runs on the tensor cores; everything else here
   if (window_tc_supported(p, dtype)) return launch_window_scores_tc(p, h, s);
   if (dtype == TASKKV_F32) {
-    return p.d == 64 ? launch_generic<float, 64>(p, max_N, s) : launch_generic<float, 128>(p, max_N, s);
+    return p.d == 64 ? launch_generic<float, 64>(p, max_N, h, s) : launch_generic<float, 128>(p, max_N, h, s);
   }
-  return p.d == 64 ? launch_generic<__nv_bfloat16, 64>(p, max_N, s)
-                   : launch_generic<__nv_bfloat16, 128>(p, max_N, s);
+  return p.d == 64 ? launch_generic<__nv_bfloat16, 64>(p, max_N, h, s)
+                   : launch_generic<__nv_bfloat16, 128>(p, max_N, h, s);
 }
 
 }  // namespace taskkv

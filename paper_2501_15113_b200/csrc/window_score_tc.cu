@@ -706,14 +706,22 @@ cudaError_t launch_tc_d(const DeviceProblem& p, const WindowHostInfo& h, cudaStr
     const int n1 = a.item_off[nb];
     const int grid = n1 < n_sm ? n1 : n_sm;
     a.steps = (n1 + grid - 1) / grid;
-    a.pass = 1;
-    {
-      LaunchScope ls(K_WINDOW_TC, s);
-      window_tc_kernel<D><<<grid, kThreads, smem, s>>>(maps, p, a, lay);
-    }
-    {
-      LaunchScope ls(K_WINDOW_REDUCE, s);
-      window_tc_reduce_kernel<<<dim3(nb * per_seq, (p.rows + 3) / 4), 128, 0, s>>>(p, b0 * per_seq, a.chunk_keys, parts);
+    if (h.lse) {
+      // the caller already has the rows' normalisers: no pass 1
+      for (int i = 0; i < nb; ++i) {
+        e = launch_lse_to_stat(p, (b0 + i) * per_seq, per_seq, static_cast<const float*>(h.lse[b0 + i]), true, s);
+        if (e != cudaSuccess) return e;
+      }
+    } else {
+      a.pass = 1;
+      {
+        LaunchScope ls(K_WINDOW_TC, s);
+        window_tc_kernel<D><<<grid, kThreads, smem, s>>>(maps, p, a, lay);
+      }
+      {
+        LaunchScope ls(K_WINDOW_REDUCE, s);
+        window_tc_reduce_kernel<<<dim3(nb * per_seq, (p.rows + 3) / 4), 128, 0, s>>>(p, b0 * per_seq, a.chunk_keys, parts);
+      }
     }
     a.pass = 2;
     {

@@ -533,3 +533,45 @@ def test_random_shapes(seed):
     case = _random_case(seed)
     wl = small(f"random{seed}", **case, steps=2)
     run_workload(wl)
+
+
+@pytest.mark.parametrize("case", [
+    dict(n=4, n_kv=4, d=128, N=2341, L=32, s1=4, s2=64, k=100, dtype="bf16"),            # tensor-core path, 32 rows
+    dict(n=8, n_kv=2, d=128, N=0, L=32, s1=4, s2=64, k=150, dtype="bf16", R=2, seq_lens=[3000, 1777], nh=1),  # 128 rows
+    dict(n=4, n_kv=4, d=64, N=1500, L=16, s1=4, s2=32, k=77, dtype="f32"),               # CUDA-core path
+], ids=["tc32", "tc128_ragged", "f32"])
+def test_compress_with_supplied_window_lse(case):
+    """With the window rows' log-sum-exp handed in (here: the oracle's, rounded to fp32) pass 1 is skipped; scores,
+    selections, classes, rows and decode outputs must match the oracle exactly as in the full computation."""
+    tk, P = _tk(), _parity()
+    from oracle import taskkv_oracle as O
+    wl = small("lse", **case)
+    qs, ks, vs = W.materialize(wl, DEV)
+    G = wl.group
+    lse = []
+    for b in range(wl.batch):
+        per_layer = []
+        for r in range(wl.n_layers):
+            q64, k64 = P.to64(qs[b][r]), P.to64(ks[b][r])
+            per_layer.append(np.stack([O.window_lse(q64[a], k64[a // G]) for a in range(wl.n_heads)]))
+        lse.append(torch.from_numpy(np.stack(per_layer)).float().to(DEV).contiguous())
+    steps = wl.decode_steps
+    params = tk.params_from_workload(wl, max_new_tokens=steps)
+    cache = tk.taskkv_compress_ex(params, qs, ks, vs, window_lse=lse)
+    assert cache.status() == 0
+    rep = P.Report()
+    scores, topt = cache.query(tk.Q_SCORES), cache.query(tk.Q_TOPT)
+    refs = {}
+    for b in range(wl.batch):
+        for r in range(wl.n_layers):
+            refs[(b, r)] = P.oracle_layer(wl, b, r, qs[b][r], ks[b][r], vs[b][r])
+            P.compare_layer(cache, wl, b, r, refs[(b, r)], rep, scores=scores, topt=topt)
+            P.compare_pool_rows(cache, wl, b, r, ks[b][r], vs[b][r])
+    step_inputs = [W.gen_decode_step(wl, s, DEV) for s in range(steps)]
+    outs = [cache.taskkv_decode_step(q, kn, vn) for (q, kn, vn) in step_inputs]
+    for (b, r), ref in refs.items():
+        want = P.oracle_decode_steps(wl, b, r, ks[b][r], vs[b][r], ref["idx"], step_inputs)
+        for s in range(steps):
+            assert float(np.abs(P.to64(outs[s][b, r]) - want[s]).max()) < P.TOL_OUT[wl.dtype]
+    assert rep.class_near_ties == 0
+    cache.close()
