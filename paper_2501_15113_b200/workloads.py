@@ -50,6 +50,8 @@ class Workload:
     plant_signed: bool = True       # random sign per (head, dim); False: +offset on every dim
     planted: Optional[List[List[List[int]]]] = None  # [batch][layer] -> kv heads
     sink_key_scale: float = 1.0
+    heavy_keys: int = 0             # keys per head, at seeded positions, scaled by heavy_scale ("heavy hitters")
+    heavy_scale: float = 1.0
     note: str = ""
 
     @property
@@ -150,6 +152,11 @@ def gen_layer(wl: Workload, b: int, r: int, device="cpu"):
     v *= (std * uv).to(device)[:, None, None]
     if wl.sink_key_scale != 1.0:
         k[:, 0, :] *= wl.sink_key_scale
+    if wl.heavy_keys > 0:
+        gh = _cpu_gen(wl.seed, 606, b, r)
+        for h in range(wl.n_kv_heads):
+            pos = torch.randint(0, N, (wl.heavy_keys,), generator=gh).to(device)
+            k[h, pos, :] *= wl.heavy_scale
     planted = wl.planted[b][r] if wl.planted is not None else []
     for h in planted:
         if wl.plant_signed:

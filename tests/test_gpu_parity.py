@@ -302,6 +302,63 @@ def test_window_scores_many_items_per_cta(case):
     run_workload(wl, layers=[(b, r) for b in range(wl.batch) for r in (0, wl.n_layers - 1)])
 
 
+SINGLE_READ_CASES = [
+    # cluster sizes 2, 4, 8, 16 of the kernel that keeps a unit's scores in tensor memory; slices of unequal
+    # tile counts, ragged last tiles, a last tile shorter than the window
+    dict(n=4, n_kv=4, d=128, N=4000, L=32, s1=4, s2=64, k=100, dtype="bf16"),
+    dict(n=4, n_kv=4, d=128, N=8200, L=32, s1=4, s2=64, k=100, dtype="bf16"),
+    dict(n=4, n_kv=4, d=64, N=16397, L=32, s1=4, s2=64, k=300, dtype="bf16"),
+    dict(n=2, n_kv=2, d=128, N=32768, L=32, s1=4, s2=256, k=512, dtype="bf16"),
+    dict(n=2, n_kv=2, d=128, N=30001, L=32, s1=4, s2=256, k=512, dtype="bf16", nh=0),
+    # two query heads per KV head with a 16-row window: 32 rows, causal limit by row % 16
+    dict(n=8, n_kv=4, d=128, N=5003, L=16, s1=4, s2=64, k=100, dtype="bf16"),
+    # a batch whose sequences need different slice sizes in one launch, more units than clusters
+    dict(n=8, n_kv=8, d=128, N=0, L=32, s1=4, s2=64, k=120, dtype="bf16", R=3, seq_lens=[9000, 300, 16000, 2100], nh=2),
+]
+
+
+@pytest.mark.parametrize("case", SINGLE_READ_CASES, ids=[f"case{i}" for i in range(len(SINGLE_READ_CASES))])
+def test_window_scores_single_read(case):
+    wl = small("single_read", **case, steps=1)
+    run_workload(wl, layers=[(b, r) for b in range(wl.batch) for r in (0, wl.n_layers - 1)])
+
+
+def test_window_scores_single_read_moderate_heavy_keys():
+    """A few keys per head well above the rest (scores stay within fp32 range of one another): full parity."""
+    wl = small("heavy", n=4, n_kv=4, d=128, N=9000, L=32, s1=4, s2=64, k=100, dtype="bf16", steps=1)
+    wl.heavy_keys, wl.heavy_scale = 5, 6.0
+    run_workload(wl)
+
+
+def test_window_scores_single_read_extreme_keys_fall_back_to_exact_maxima():
+    """Keys hundreds of score units above the rest: a warp's running sums, taken relative to an ordinary key,
+    overflow and the warp redoes its tiles with its exact row maxima.  Almost all of the softmax mass sits on a few
+    keys, the rest is below fp32 range, so only the scores are compared here (absolute, against the largest)."""
+    tk, P = _tk(), _parity()
+    from oracle import taskkv_oracle as O
+    wl = small("extreme", n=2, n_kv=2, d=128, N=9000, L=32, s1=4, s2=64, k=100, dtype="bf16", steps=0, nh=0)
+    wl.heavy_keys, wl.heavy_scale = 5, 600.0
+    qs, ks, vs = W.materialize(wl, DEV)
+    cache = tk.taskkv_compress_ex(tk.params_from_workload(wl, max_new_tokens=0), qs, ks, vs)
+    assert cache.status() == 0
+    got = cache.query(tk.Q_SCORES).astype(np.float64)
+    off = P.score_offsets(wl)
+    spread = 0.0
+    for h in range(wl.n_kv_heads):
+        q64, k64 = P.to64(qs[0][0][h:h + 1]), P.to64(ks[0][0][h])
+        s = (q64[0] @ k64.T) / np.sqrt(wl.head_dim)
+        spread = max(spread, float(s.max() - np.median(s)))
+        want = O.window_scores(q64, k64)
+        c = got[off[h]:off[h] + wl.seq_lens[0]]
+        assert np.isfinite(c).all()
+        # scores of several hundred: the fp32 rounding of a score (relative 6e-8 per operation) is ~1e-4 absolute in
+        # the exponent, hence the wider bound than for ordinary inputs
+        assert np.abs(c - want).max() < 1e-3 * want.max()
+        assert abs(c.sum() - 1.0) < 1e-3
+    assert spread > 150.0      # beyond what exp2 in fp32 holds relative to an ordinary key: the fast path cannot apply
+    cache.close()
+
+
 def test_ragged_batch_of_eleven_sequences():
     """More sequences than one window-score launch takes (eight): a full group and a partial one."""
     from paper_2501_15113_b200 import configs
