@@ -303,7 +303,7 @@ struct FastSmem {
   int list_n;          // keys collected for the narrow phase of the bisection
   uint32_t list_thr;   // its result
 };
-constexpr int kNarrow = 1024;  // the bisection runs over all keys until at most this many lie in the undecided range
+constexpr int kNarrow = 1023;  // the bisection runs over all keys until at most this many lie in the undecided range
 
 __device__ __forceinline__ int block_count_ge(const uint32_t (&key)[kEpt], uint32_t cand, int* slot) {
   int c = 0;
@@ -357,19 +357,26 @@ __device__ void block_bisect(FastSmem& fs, const uint32_t (&key)[kEpt], int want
       for (int e = 0; e < kEpt; ++e)
         if (key[e] >= t && (top == 0u || key[e] < top)) list[atomicAdd(&fs.list_n, 1)] = key[e];
       __syncthreads();
-      if (warp == 0) {
-        const int want2 = want - above;               // rank inside the collected keys
-        for (; bit >= 0; --bit) {
-          const uint32_t cand = t | (1u << bit);
-          int c = 0;
-          for (int i = lane; i < alive; i += 32) c += list[i] >= cand;
-          c = __reduce_add_sync(0xffffffffu, c);
-          if (c >= want2) t = cand;
-        }
-        if (lane == 0) fs.list_thr = t;
+      // every thread takes one collected key (there are at most as many as threads); two bits per step: the
+      // counts above the three thresholds travel packed in one word (10 bits each hold a count <= 1023)
+      static_assert(kNarrow <= kThreads && kNarrow < (1 << 10), "one key per thread, three counts per word");
+      const uint32_t mine = (int)threadIdx.x < alive ? list[threadIdx.x] : 0u;
+      const int want2 = want - above;                 // rank inside the collected keys
+      while (bit >= 0) {
+        const uint32_t b_hi = 1u << bit, b_lo = bit > 0 ? 1u << (bit - 1) : 0u;
+        const uint32_t c10 = t | b_hi, c11 = c10 | b_lo, c01 = t | b_lo;
+        int v = (int)(mine >= c10) | ((int)(mine >= c11) << 10) | ((int)(b_lo != 0u && mine >= c01) << 20);
+        v = __reduce_add_sync(0xffffffffu, v);
+        if (lane == 0) fs.cnt[par][warp] = v;
+        __syncthreads();
+        v = __reduce_add_sync(0xffffffffu, fs.cnt[par][lane]);
+        par ^= 1;
+        const int n10 = v & 0x3ff, n11 = (v >> 10) & 0x3ff, n01 = (v >> 20) & 0x3ff;
+        if (b_lo != 0u && n11 >= want2) t = c11;
+        else if (n10 >= want2) t = c10;
+        else if (b_lo != 0u && n01 >= want2) t = c01;
+        bit -= 2;
       }
-      __syncthreads();
-      t = fs.list_thr;
     }
   }
   const int n_gt = (t == 0xffffffffu) ? 0 : block_count_ge(key, t + 1u, fs.cnt[par]);
@@ -378,14 +385,21 @@ __device__ void block_bisect(FastSmem& fs, const uint32_t (&key)[kEpt], int want
   __syncthreads();
 }
 
-// Ordered compaction of this thread's 32 consecutive positions [base, base + 32).
+// Ordered compaction of this thread's 32 consecutive positions [base, base + 32): emit(rank, position) for every
+// key above thr and for the first need_eq keys equal to it (lower position first).  The comparisons are made once,
+// into two bit masks; the selected keys are few per thread, so the emitting loop walks set bits only.
 template <class Emit>
 __device__ void block_compact_regs(FastSmem& fs, const uint32_t (&key)[kEpt], int base, uint32_t thr, int need_eq,
                                    const Emit& emit) {
+  static_assert(kEpt == 32, "one mask bit per key");
   const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
-  int gt = 0, eq = 0;
+  uint32_t m_gt = 0u, m_ge = 0u;
 #pragma unroll
-  for (int e = 0; e < kEpt; ++e) { gt += key[e] > thr; eq += key[e] == thr; }
+  for (int e = 0; e < kEpt; ++e) {
+    m_gt |= (uint32_t)(key[e] > thr) << e;
+    m_ge |= (uint32_t)(key[e] >= thr) << e;
+  }
+  const int gt = __popc(m_gt), eq = __popc(m_ge) - gt;
   const int packed = gt | (eq << 16);
   int incl = packed;
 #pragma unroll
@@ -405,12 +419,12 @@ __device__ void block_compact_regs(FastSmem& fs, const uint32_t (&key)[kEpt], in
   const int wexcl = __shfl_sync(0xffffffffu, wi - wp, warp);
   const int excl = incl - packed + wexcl;
   int gt_before = excl & 0xffff, eq_before = excl >> 16;
-#pragma unroll
-  for (int e = 0; e < kEpt; ++e) {
-    const bool g = key[e] > thr, q = key[e] == thr;
-    if (g || (q && eq_before < need_eq)) emit(gt_before + min(eq_before, need_eq), base + e, e);
+  for (uint32_t m = m_ge; m != 0u; m &= m - 1u) {
+    const int e = __ffs((int)m) - 1;
+    const bool g = (m_gt >> e) & 1u;
+    if (g || eq_before < need_eq) emit(gt_before + min(eq_before, need_eq), base + e);
     gt_before += g;
-    eq_before += q;
+    eq_before += !g;
   }
   __syncthreads();
 }
@@ -449,9 +463,9 @@ __global__ void __launch_bounds__(kThreads, 1) select_fast_kernel(DeviceProblem 
   uint32_t* scratch = reinterpret_cast<uint32_t*>(&red[0][0]);   // free until the semantic vector is summed
   block_bisect(fs, key, t, scratch, kWarps * D, thr, need_eq);
   int* topt = p.topt + (size_t)u * p.top_t;
-  block_compact_regs(fs, key, base, thr, need_eq, [&](int pos, int j, int e) {
+  block_compact_regs(fs, key, base, thr, need_eq, [&](int pos, int j) {
     sel[pos] = j;
-    selw[pos] = key_score(key[e]);
+    selw[pos] = C[j];
     topt[pos] = j;
   });
   for (int i = t + tid; i < p.top_t; i += kThreads) topt[i] = -1;
@@ -524,7 +538,7 @@ __global__ void __launch_bounds__(kThreads, 1) select_fast_kernel(DeviceProblem 
   }
   __syncthreads();
   block_bisect(fs, key, kmid, scratch, kWarps * D, thr, need_eq);
-  block_compact_regs(fs, key, base, thr, need_eq, [&](int pos, int j, int) { idx[s1 + pos] = j; });
+  block_compact_regs(fs, key, base, thr, need_eq, [&](int pos, int j) { idx[s1 + pos] = j; });
 }
 
 template <typename T, int D>
