@@ -141,6 +141,25 @@ taskkv_status taskkv_compress_ex(const taskkv_params* p, const void* const* q_wi
                                  void* workspace_mem, size_t workspace_bytes,
                                  taskkv_stream stream, taskkv_cache** out_cache);
 
+/*
+ * The exact semantic vectors of Sec. III-A (Eq. 1-2) of one sequence: for every KV head
+ *   C[j] = (1 / (G N)) sum over the G query heads of the group and all N query rows i of A[i, j],
+ *          A = softmax(Q K^T / sqrt(d) + causal mask) row by row (G = 1: exactly the column mean of Eq. 2),
+ *   v    = sum_j C[j] V[j, :],
+ * i.e. what the observation window, the top-t selection and Eq. 15 approximate.  The cost is quadratic in N (two
+ * tensor-core passes over the causal half of Q K^T); this is an analysis routine beside the compression path.
+ *   q        device bf16 [n_layers][n_heads][N][d]     every query row (post-RoPE), 16-byte aligned
+ *   k, v     device bf16 [n_layers][n_kv_heads][N][d]
+ *   sem_out  device fp32 [n_layers][n_kv_heads][d]     v
+ *   c_out    device fp32 [n_layers][n_kv_heads][N], or NULL if the column means are not wanted
+ * head_dim 64 or 128, bf16 only.  Scratch (up to ~1.5 GB) comes from the stream's memory pool (cudaMallocAsync) and
+ * goes back to it; the call returns after the stream has finished the work.  Errors: EINVAL (arguments), EALLOC,
+ * ECUDA, ETIMEOUT (a bounded wait inside a kernel ran out).
+ */
+taskkv_status taskkv_exact_semantic(const void* q, const void* k, const void* v, int32_t n_layers, int32_t n_heads,
+                                    int32_t n_kv_heads, int32_t head_dim, int32_t seq_len, float* sem_out,
+                                    float* c_out, taskkv_stream stream);
+
 /* As taskkv_compress_ex, for callers that already hold the normalisers of the observation window's rows:
  *   window_lse[b]  device fp32 [n_layers][n_heads][L], lse_i = ln sum_j exp(q_i . k_j / sqrt(d)) over the keys
  *                  j <= position of window row i -- what an attention kernel run over the prompt returns as the

@@ -177,7 +177,7 @@ thread_local cudaEvent_t tl_start = nullptr;
 
 const char* kKernelNames[K_COUNT] = {
     "window_stats", "window_reduce", "window_scores", "select", "separator", "plan",
-    "gather", "append", "decode_attn", "decode_combine", "window_tc", "compensate"};
+    "gather", "append", "decode_attn", "decode_combine", "window_tc", "compensate", "exact_sum"};
 
 }  // namespace
 

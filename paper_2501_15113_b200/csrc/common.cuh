@@ -31,6 +31,7 @@ enum KernelId : int32_t {
   K_DECODE_COMBINE,
   K_WINDOW_TC,
   K_COMPENSATE,
+  K_EXACT_SUM,
   K_COUNT
 };
 
@@ -118,6 +119,8 @@ cudaError_t launch_window_scores(const DeviceProblem& p, int dtype, int max_N, c
                                  cudaStream_t s);
 bool window_tc_supported(const DeviceProblem& p, int dtype);
 cudaError_t launch_window_scores_tc(const DeviceProblem& p, const WindowHostInfo& h, cudaStream_t s);
+cudaError_t launch_window_prefix(const DeviceProblem& p, const void* q, const void* k, int heads, int group, int N,
+                                 cudaStream_t s);
 int window_res_team(const DeviceProblem& p, const WindowHostInfo& h);
 cudaError_t launch_window_scores_res(const DeviceProblem& p, const WindowHostInfo& h, int team, cudaStream_t s);
 cudaError_t launch_select(const DeviceProblem& p, int dtype, int max_N, cudaStream_t s);

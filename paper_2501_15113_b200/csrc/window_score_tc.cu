@@ -88,6 +88,11 @@ struct TcArgs {
   int n_local;              // units per sequence (layers * kv heads)
   int chunk_keys;           // keys per work item (multiple of 128)
   int steps;                // items of the busiest CTA
+  // Prefix mode (the column sums of the full causal attention matrix, Eq. 1-2 of Sec. III-A): unit lu stands for the
+  // 128 query rows [128 b, 128 b + 128) of query head lu / prefix_blocks, b = lu % prefix_blocks, as a window
+  // over the first 128 (b + 1) keys of that head's KV head.  0: every unit has its own N keys and rows.
+  int prefix_blocks;
+  int group;                // query heads per KV head (prefix mode)
   int u0[kMaxSeq];          // first unit of each sequence
   int N[kMaxSeq];           // sequence length
   int chunks[kMaxSeq];      // work items per unit
@@ -96,9 +101,11 @@ struct TcArgs {
 
 struct Item {
   int seq, lu, ch;
+  int N;                    // keys of the unit
+  int krow0, qrow0;         // first row of the unit in the K and Q tensor maps
   bool valid;
 };
-__device__ __forceinline__ Item decode_item(const TcArgs& a, int k) {
+__device__ __forceinline__ Item decode_item(const TcArgs& a, int k, int rows) {
   Item it;
   const int i = (int)blockIdx.x + k * (int)gridDim.x;
   it.valid = i < a.item_off[a.n_seq];
@@ -109,6 +116,18 @@ __device__ __forceinline__ Item decode_item(const TcArgs& a, int k) {
   const int local = it.valid ? i - a.item_off[it.seq] : 0;
   it.lu = local / a.chunks[it.seq];
   it.ch = local % a.chunks[it.seq];
+  const int N = a.N[it.seq];
+  if (a.prefix_blocks > 0) {
+    const int head = it.lu / a.prefix_blocks, b = it.lu % a.prefix_blocks;
+    it.N = (b + 1) * kTile;                 // may run past the sequence end: those rows and keys are neutralised
+    it.krow0 = (head / a.group) * N;
+    it.qrow0 = head * N + b * kTile;
+    it.valid = it.valid && it.ch * a.chunk_keys < it.N;
+  } else {
+    it.N = N;
+    it.krow0 = it.lu * N;
+    it.qrow0 = it.lu * rows;
+  }
   return it;
 }
 
@@ -203,9 +222,9 @@ window_tc_kernel(const __grid_constant__ TcMaps maps, DeviceProblem p, const __g
       uint32_t phase = 0, qphase[2] = {0, 0};
       bool ok = true;
       for (int k = 0; k < a.steps && ok; ++k) {
-        const Item it = decode_item(a, k);
+        const Item it = decode_item(a, k, rows);
         if (!it.valid) continue;
-        const int N = a.N[it.seq];
+        const int N = it.N;
         const int key0 = it.ch * a.chunk_keys;
         const int ntiles = (min(N, key0 + a.chunk_keys) - key0 + kTile - 1) / kTile;
         ok = __all_sync(0xffffffffu, mbar_wait(BAR(B_QEMPTY + qb), qphase[qb] ^ 1, s_abort));
@@ -214,7 +233,7 @@ window_tc_kernel(const __grid_constant__ TcMaps maps, DeviceProblem p, const __g
           mbar_expect_tx(BAR(B_QFULL + qb), (uint32_t)lay.q_block_bytes);
           for (int kb = 0; kb < KB; ++kb)
             tma_load_2d(smem_u32(sQ + (size_t)qb * lay.q_block_bytes + (size_t)kb * rows * 128), &maps.q[it.seq],
-                        kb * 64, it.lu * rows, BAR(B_QFULL + qb));
+                        kb * 64, it.qrow0, BAR(B_QFULL + qb));
         }
         __syncwarp();
         qphase[qb] ^= 1;
@@ -227,7 +246,7 @@ window_tc_kernel(const __grid_constant__ TcMaps maps, DeviceProblem p, const __g
 #pragma unroll
             for (int kb = 0; kb < KB; ++kb)
               tma_load_2d(smem_u32(sK + (size_t)stage * lay.tile_bytes + (size_t)kb * kTile * 128), &maps.k[it.seq],
-                          kb * 64, it.lu * N + key0 + t * kTile, BAR(B_FULL + stage));
+                          kb * 64, it.krow0 + key0 + t * kTile, BAR(B_FULL + stage));
           }
           __syncwarp();
           if (++stage == S) { stage = 0; phase ^= 1; }
@@ -259,9 +278,9 @@ window_tc_kernel(const __grid_constant__ TcMaps maps, DeviceProblem p, const __g
       const uint64_t desc_hi = smem_desc(0);    // everything but the start address
       bool ok = true;
       for (int k = 0; k < a.steps && ok; ++k) {
-        const Item it = decode_item(a, k);
+        const Item it = decode_item(a, k, rows);
         if (!it.valid) continue;
-        const int N = a.N[it.seq];
+        const int N = it.N;
         const int key0 = it.ch * a.chunk_keys;
         const int ntiles = (min(N, key0 + a.chunk_keys) - key0 + kTile - 1) / kTile;
         ok = __all_sync(0xffffffffu, mbar_wait(BAR(B_QFULL + qb), qphase[qb], s_abort));
@@ -317,7 +336,7 @@ window_tc_kernel(const __grid_constant__ TcMaps maps, DeviceProblem p, const __g
     const float* stat_g = p.stat;
     float pre[4];
     auto fetch_stats = [&](int k) {
-      const Item nx = decode_item(a, k);
+      const Item nx = decode_item(a, k, rows);
 #pragma unroll
       for (int q = 0; q < 4; ++q)
         pre[q] = (nx.valid && q * 32 + lane < rows) ? stat_g[(size_t)(a.u0[nx.seq] + nx.lu) * (2 * p.rows_pad) + q * 32 + lane]
@@ -325,10 +344,13 @@ window_tc_kernel(const __grid_constant__ TcMaps maps, DeviceProblem p, const __g
     };
     if (a.pass == 2) fetch_stats(0);
     for (int k = 0; k < a.steps && ok; ++k) {
-      const Item it = decode_item(a, k);
-      if (!it.valid) continue;
+      const Item it = decode_item(a, k, rows);
+      if (!it.valid) {
+        if (a.pass == 2) fetch_stats(k + 1);   // (prefix mode skips items in mid-run: keep the prefetch one ahead)
+        continue;
+      }
       const int u = a.u0[it.seq] + it.lu;
-      const int N = a.N[it.seq];
+      const int N = it.N;
       const int key0 = it.ch * a.chunk_keys;
       const int ntiles = (min(N, key0 + a.chunk_keys) - key0 + kTile - 1) / kTile;
       // pass 1 state: after the transposition lane = window row (rg * 32 + lane); raw (unscaled) maxima
@@ -512,7 +534,8 @@ window_tc_kernel(const __grid_constant__ TcMaps maps, DeviceProblem p, const __g
 
 // Folds the partial statistics of one unit: slots (item, warp) of pass 1 -> one offset per row.
 // One warp per (unit, row): lanes take every 32nd slot, then a shuffle tree; the order is fixed.
-__global__ void __launch_bounds__(128) window_tc_reduce_kernel(DeviceProblem p, int u0, int chunk_keys, int parts) {
+__global__ void __launch_bounds__(128) window_tc_reduce_kernel(DeviceProblem p, int u0, int chunk_keys, int parts,
+                                                               int n_real) {
   const int u = u0 + blockIdx.x;
   const int slots = (p.unit_N[u] + chunk_keys - 1) / chunk_keys * parts;
   const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
@@ -537,8 +560,12 @@ __global__ void __launch_bounds__(128) window_tc_reduce_kernel(DeviceProblem p, 
       M = Mn;
     }
     // one offset per row: score * scale - (max + log2(sum) + log2(rows)) is log2 of the row's share of C
+    // prefix mode (n_real > 0): a query row at or beyond the end of the sequence does not exist; an infinite
+    // offset takes it out of every column sum
+    const bool absent = n_real > 0 && p.unit_N[u] - p.rows + row >= n_real;
     if (lane == 0)
-      p.stat[(size_t)u * (2 * p.rows_pad) + row] = z > 0.f ? M + log2f(z) + log2f((float)p.rows) : INFINITY;
+      p.stat[(size_t)u * (2 * p.rows_pad) + row] =
+          (z > 0.f && !absent) ? M + log2f(z) + log2f((float)p.rows) : INFINITY;
   }
 }
 
@@ -574,6 +601,8 @@ cudaError_t launch_tc_d(const DeviceProblem& p, const WindowHostInfo& h, cudaStr
     for (int i = 0; i < nb; ++i) keys += (int64_t)per_seq * h.seq_lens[b0 + i];
     a.n_seq = nb;
     a.n_local = per_seq;
+    a.prefix_blocks = 0;
+    a.group = 1;
     a.chunk_keys = pick_chunk(keys, n_sm);
     a.item_off[0] = 0;
     for (int i = 0; i < kMaxSeq; ++i) {
@@ -603,7 +632,7 @@ cudaError_t launch_tc_d(const DeviceProblem& p, const WindowHostInfo& h, cudaStr
       }
       {
         LaunchScope ls(K_WINDOW_REDUCE, s);
-        window_tc_reduce_kernel<<<dim3(nb * per_seq, (p.rows + 3) / 4), 128, 0, s>>>(p, b0 * per_seq, a.chunk_keys, parts);
+        window_tc_reduce_kernel<<<dim3(nb * per_seq, (p.rows + 3) / 4), 128, 0, s>>>(p, b0 * per_seq, a.chunk_keys, parts, 0);
       }
     }
     a.pass = 2;
@@ -617,11 +646,66 @@ cudaError_t launch_tc_d(const DeviceProblem& p, const WindowHostInfo& h, cudaStr
   return cudaSuccess;
 }
 
+// Prefix mode: p describes heads * blocks virtual units of 128 window rows (rows = L = 128; unit_N, c_off, stat,
+// stat_part sized for them); q is [heads][N][d], k is [heads / group][N][d].
+template <int D>
+cudaError_t launch_prefix_d(const DeviceProblem& p, const void* q, const void* k, int heads, int group, int N,
+                            cudaStream_t s) {
+  int dev = 0, n_sm = 0;
+  cudaGetDevice(&dev);
+  cudaDeviceGetAttribute(&n_sm, cudaDevAttrMultiProcessorCount, dev);
+  if (n_sm <= 0) n_sm = 148;
+  const TcLayout lay = make_layout(D, p.rows);
+  if (lay.stages < 2) return cudaErrorInvalidValue;
+  cudaError_t e = cudaFuncSetAttribute(window_tc_kernel<D>, cudaFuncAttributeMaxDynamicSharedMemorySize, lay.total);
+  if (e != cudaSuccess) return e;
+  const int blocks = (N + kTile - 1) / kTile;
+  TcMaps maps;
+  TcArgs a;
+  a.n_seq = 1;
+  a.n_local = heads * blocks;
+  a.prefix_blocks = blocks;
+  a.group = group;
+  a.chunk_keys = kTcChunk;
+  a.item_off[0] = 0;
+  for (int i = 0; i < kMaxSeq; ++i) {
+    if (!make_tensor_map_2d(&maps.k[i], k, D, (uint64_t)(heads / group) * (uint64_t)N, kTile)) return cudaErrorUnknown;
+    if (!make_tensor_map_2d(&maps.q[i], q, D, (uint64_t)heads * (uint64_t)N, p.rows)) return cudaErrorUnknown;
+    a.u0[i] = 0;
+    a.N[i] = N;
+    a.chunks[i] = (blocks * kTile + a.chunk_keys - 1) / a.chunk_keys;
+    a.item_off[i + 1] = a.item_off[i] + (i == 0 ? a.n_local * a.chunks[i] : 0);
+  }
+  const int n1 = a.item_off[1];
+  const int grid = n1 < n_sm ? n1 : n_sm;
+  a.steps = (n1 + grid - 1) / grid;
+  a.pass = 1;
+  {
+    LaunchScope ls(K_WINDOW_TC, s);
+    window_tc_kernel<D><<<grid, kThreads, lay.total, s>>>(maps, p, a, lay);
+  }
+  {
+    LaunchScope ls(K_WINDOW_REDUCE, s);
+    window_tc_reduce_kernel<<<dim3(a.n_local, (p.rows + 3) / 4), 128, 0, s>>>(p, 0, a.chunk_keys, 2, N);
+  }
+  a.pass = 2;
+  {
+    LaunchScope ls(K_WINDOW_TC, s);
+    window_tc_kernel<D><<<grid, kThreads, lay.total, s>>>(maps, p, a, lay);
+  }
+  return cudaGetLastError();
+}
+
 }  // namespace
 
 bool window_tc_supported(const DeviceProblem& p, int dtype) {
   return dtype == TASKKV_BF16 && (p.rows == 32 || p.rows == 64 || p.rows == 128) && p.L <= p.rows &&
          encode_fn() != nullptr;
+}
+
+cudaError_t launch_window_prefix(const DeviceProblem& p, const void* q, const void* k, int heads, int group, int N,
+                                 cudaStream_t s) {
+  return p.d == 64 ? launch_prefix_d<64>(p, q, k, heads, group, N, s) : launch_prefix_d<128>(p, q, k, heads, group, N, s);
 }
 
 cudaError_t launch_window_scores_tc(const DeviceProblem& p, const WindowHostInfo& h, cudaStream_t s) {

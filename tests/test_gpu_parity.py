@@ -632,3 +632,43 @@ def test_compress_with_supplied_window_lse(case):
             assert float(np.abs(P.to64(outs[s][b, r]) - want[s]).max()) < P.TOL_OUT[wl.dtype]
     assert rep.class_near_ties == 0
     cache.close()
+
+
+EXACT_CASES = [
+    dict(R=1, n=2, n_kv=2, d=128, N=700),      # a ragged last block of query rows
+    dict(R=2, n=4, n_kv=2, d=64, N=1000),      # two query heads per KV head, d = 64
+    dict(R=1, n=2, n_kv=1, d=128, N=128),      # exactly one block
+    dict(R=1, n=1, n_kv=1, d=128, N=100),      # shorter than a block
+    dict(R=1, n=2, n_kv=2, d=128, N=4500),     # several work items per prefix window, 36 blocks
+]
+
+
+@pytest.mark.parametrize("case", EXACT_CASES, ids=[f"case{i}" for i in range(len(EXACT_CASES))])
+def test_exact_semantic_vector(case):
+    """Eq. 1-2 on the GPU (prefix windows on the tensor cores) against the oracle's full causal attention."""
+    tk, P = _tk(), _parity()
+    from oracle import taskkv_oracle as O
+    R, n, n_kv, d, N = (case[x] for x in ("R", "n", "n_kv", "d", "N"))
+    G = n // n_kv
+    g = torch.Generator(device="cpu").manual_seed(1234 + N)
+    std = float(d) ** -0.25
+    q = (torch.randn(R, n, N, d, generator=g) * std).to(torch.bfloat16).to(DEV)
+    k = (torch.randn(R, n_kv, N, d, generator=g) * std).to(torch.bfloat16).to(DEV)
+    v = (torch.randn(R, n_kv, N, d, generator=g) * std).to(torch.bfloat16).to(DEV)
+    k[:, :, N // 3, :] *= 6.0                          # one heavy key per head
+    sem, c = tk.taskkv_exact_semantic(q, k, v)
+    sem_only, none = tk.taskkv_exact_semantic(q, k, v, want_scores=False)
+    assert none is None and torch.equal(sem, sem_only)
+    for r in range(R):
+        for h in range(n_kv):
+            q64 = P.to64(q[r, h * G:(h + 1) * G])
+            k64, v64 = P.to64(k[r, h]), P.to64(v[r, h])
+            want_c = O.window_scores(q64, k64)           # the window is the whole sequence: L = N
+            got_c = P.to64(c[r, h])
+            assert np.abs(got_c - want_c).max() < P.TOL_SCORE_REL * want_c.max()
+            assert abs(got_c.sum() - 1.0) < 1e-5
+            want_v = want_c @ v64
+            if G == 1:
+                np.testing.assert_allclose(want_v, O.exact_semantic_vector(q64[0], k64, v64), rtol=0, atol=1e-13)
+            bound = P.TOL_SCORE_REL * (want_c[:, None] * np.abs(v64)).sum(axis=0).max()
+            assert np.abs(P.to64(sem[r, h]) - want_v).max() < bound

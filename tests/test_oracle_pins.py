@@ -432,3 +432,18 @@ def test_window_lse_is_the_normaliser_of_eq12():
         assert abs(lse[i] - ref) < 1e-12
         np.testing.assert_allclose(np.exp(s[i, :p_i + 1] - lse[i]), a[i, :p_i + 1], rtol=1e-12, atol=0)
         assert np.all(a[i, p_i + 1:] == 0)
+
+
+def test_exact_semantic_vector_closed_forms():
+    """Eq. 1-2 with all keys equal: row i of the causal softmax is uniform over its i + 1 keys, so the column mean is
+    C[j] = (1/N) sum_{i >= j} 1/(i + 1); with all value rows equal to c the semantic vector is c itself."""
+    rng = np.random.default_rng(5)
+    N, d = 37, 8
+    q = rng.normal(size=(N, d))
+    k = np.tile(rng.normal(size=(1, d)), (N, 1))
+    v = rng.normal(size=(N, d))
+    c_closed = np.array([sum(1.0 / (i + 1) for i in range(j, N)) / N for j in range(N)])
+    np.testing.assert_allclose(O.window_scores(q[None], k), c_closed, rtol=0, atol=1e-14)
+    np.testing.assert_allclose(O.exact_semantic_vector(q, k, v), c_closed @ v, rtol=0, atol=1e-14)
+    const = np.tile(rng.normal(size=(1, d)), (N, 1))
+    np.testing.assert_allclose(O.exact_semantic_vector(q, rng.normal(size=(N, d)), const), const[0], rtol=0, atol=1e-14)
