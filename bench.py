@@ -266,6 +266,8 @@ def run_ours(args):
         line["latency_mode"] = run_latency_mode(tk, wl, qs, ks, vs, steps_in, args)
         line["layer_streamed_compress"] = run_layer_streamed(tk, wl, qs, ks, vs, args)
         line["compress_with_window_lse"] = run_with_window_lse(tk, wl, qs, ks, vs, args, comp_bytes, peak)
+        if wl.seq_lens[0] <= 32768:
+            line["exact_semantic"] = run_exact_semantic(tk, wl, qs, ks, vs)
     if rank == 0 and not args.no_e2e:
         line["e2e"] = run_e2e(tk, wl, params, qs, ks, vs, steps_in, world)
     if rank == 0 and world == 1 and not args.no_cpu and args.policy != "select":
@@ -356,6 +358,63 @@ def run_layer_streamed(tk, wl, qs, ks, vs, args):
         c.close()
     return {"calls": R, "total_ms": e0.elapsed_time(e1), "ms_per_layer": e0.elapsed_time(e1) / R,
             "device_status": status}
+
+
+def run_exact_semantic(tk, wl, qs, ks, vs):
+    """The exact semantic vector of Eq. 1-2 (full causal attention, quadratic in N) for layer 0 of sequence 0, beside
+    the window approximation of Eq. 12-15 that compression uses.  The query rows before the window are seeded random
+    rows with the workload's scale; the last L rows are the workload's own window."""
+    import numpy as np
+    import torch
+    N, d, n, L = wl.seq_lens[0], wl.head_dim, wl.n_heads, wl.window
+    g = torch.Generator(device=qs[0].device).manual_seed(wl.seed * 7919 + 17)
+    q = torch.randn(1, n, N, d, generator=g, device=qs[0].device, dtype=torch.float32) * (wl.variance ** 0.5)
+    q = q.to(torch.bfloat16)
+    q[0, :, N - L:, :] = qs[0][0]
+    k, v = ks[0][0:1].contiguous(), vs[0][0:1].contiguous()
+    stream = torch.cuda.current_stream()
+    ws = torch.empty(int(tk.lib.taskkv_exact_semantic_bytes(1, n, wl.n_kv_heads, d, N)), dtype=torch.uint8,
+                     device=qs[0].device)
+    times = []
+    for i in range(1 + 3):
+        tk.taskkv_timing_enable(i == 3)
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        e0.record(stream)
+        sem, _ = tk.taskkv_exact_semantic(q, k, v, want_scores=False, workspace_mem=ws)
+        e1.record(stream)
+        torch.cuda.synchronize()
+        if i >= 1:
+            times.append(e0.elapsed_time(e1))
+    kern = {}
+    for name, t in tk.taskkv_timing_collect():
+        kern[name] = round(kern.get(name, 0.0) + t, 3)
+    tk.taskkv_timing_enable(False)
+    ms = statistics.median(times)
+    nb = (N + 127) // 128
+    scores = n * 128 * 128 * nb * (nb + 1) // 2            # per pass: the causal half in 128 x 128 tiles
+    tflops = 2 * scores * 2 * d / (ms * 1e-3) / 1e12
+    try:
+        with open(os.path.join(ROOT, "MEASURED_PEAKS.json")) as fh:
+            tpeak, kind = float(json.load(fh)["bf16_tflops"]), "measured"
+    except Exception:
+        tpeak, kind = 1590.0, "fallback"
+    out = {"layers": 1, "query_heads": n, "seq_len": N, "ms": ms, "tflops": tflops, "tensor_peak_tflops": tpeak,
+           "tensor_frac": tflops / tpeak, "peak_kind": kind, "exp_per_s": 2 * scores / (ms * 1e-3), "kernel_ms": kern,
+           "note": "two passes (row normalisers, column sums) over the causal half of Q K^T; one exponential per "
+                   "score and pass bounds it before the tensor pipe does"}
+    # how far the window's v' is from v, and whether the two pick the same far heads (one layer, one sequence)
+    if wl.batch == 1:
+        one = tk.params_from_workload(wl, max_new_tokens=0).layer(0)
+        c = tk.taskkv_compress_ex(one, [qs[0][0:1].contiguous()], [k], [v])
+        approx = c.query(tk.Q_SEMVEC).reshape(wl.n_kv_heads, d).astype(np.float64)
+        c.close()
+        exact = sem[0].double().cpu().numpy()
+        rel = np.linalg.norm(approx - exact, axis=1) / np.linalg.norm(exact, axis=1)
+        f = wl.n_hetero[0][0]
+        far = lambda x: set(np.argsort(-np.linalg.norm(x - x.mean(0), axis=1), kind="stable")[:f].tolist())
+        out.update({"window_vs_exact_rel_dist_median": float(np.median(rel)),
+                    "far_heads_agree": len(far(approx) & far(exact)), "far_heads": f})
+    return out
 
 
 def run_with_window_lse(tk, wl, qs, ks, vs, args, comp_bytes, peak):

@@ -152,13 +152,19 @@ taskkv_status taskkv_compress_ex(const taskkv_params* p, const void* const* q_wi
  *   k, v     device bf16 [n_layers][n_kv_heads][N][d]
  *   sem_out  device fp32 [n_layers][n_kv_heads][d]     v
  *   c_out    device fp32 [n_layers][n_kv_heads][N], or NULL if the column means are not wanted
- * head_dim 64 or 128, bf16 only.  Scratch (up to ~1.5 GB) comes from the stream's memory pool (cudaMallocAsync) and
- * goes back to it; the call returns after the stream has finished the work.  Errors: EINVAL (arguments), EALLOC,
- * ECUDA, ETIMEOUT (a bounded wait inside a kernel ran out).
+ *   workspace_mem  device scratch, 256-byte aligned, owned by the caller, or NULL: then up to ~1.5 GB come from the
+ *            stream's memory pool (cudaMallocAsync) and go back to it, which can cost more than the kernels.
+ *            taskkv_exact_semantic_bytes gives the size with which all heads (or as many as fit 1.5 GB) go through
+ *            in one round; with less, fewer heads go per round; EALLOC if not even one KV group fits.
+ * head_dim 64 or 128, bf16 only.  The call returns after the stream has finished the work.
+ * Errors: EINVAL (arguments), EALLOC, ECUDA, ETIMEOUT (a bounded wait inside a kernel ran out).
  */
 taskkv_status taskkv_exact_semantic(const void* q, const void* k, const void* v, int32_t n_layers, int32_t n_heads,
                                     int32_t n_kv_heads, int32_t head_dim, int32_t seq_len, float* sem_out,
-                                    float* c_out, taskkv_stream stream);
+                                    float* c_out, void* workspace_mem, size_t workspace_bytes, taskkv_stream stream);
+/* Scratch size for taskkv_exact_semantic (host only; 0 for arguments it would reject). */
+size_t taskkv_exact_semantic_bytes(int32_t n_layers, int32_t n_heads, int32_t n_kv_heads, int32_t head_dim,
+                                   int32_t seq_len);
 
 /* As taskkv_compress_ex, for callers that already hold the normalisers of the observation window's rows:
  *   window_lse[b]  device fp32 [n_layers][n_heads][L], lse_i = ln sum_j exp(q_i . k_j / sqrt(d)) over the keys

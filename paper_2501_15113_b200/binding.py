@@ -60,8 +60,11 @@ lib.taskkv_compress_ex.restype = C.c_int32
 lib.taskkv_compress_lse.argtypes = [C.POINTER(taskkv_params), _pp, _pp, _pp, _pp, _vp, C.c_size_t, _vp, C.c_size_t,
                                     _vp, C.POINTER(_vp)]
 lib.taskkv_compress_lse.restype = C.c_int32
-lib.taskkv_exact_semantic.argtypes = [_vp, _vp, _vp, C.c_int32, C.c_int32, C.c_int32, C.c_int32, C.c_int32, _vp, _vp, _vp]
+lib.taskkv_exact_semantic.argtypes = [_vp, _vp, _vp, C.c_int32, C.c_int32, C.c_int32, C.c_int32, C.c_int32, _vp, _vp, _vp,
+                                      C.c_size_t, _vp]
 lib.taskkv_exact_semantic.restype = C.c_int32
+lib.taskkv_exact_semantic_bytes.argtypes = [C.c_int32] * 5
+lib.taskkv_exact_semantic_bytes.restype = C.c_size_t
 lib.taskkv_compress.argtypes = [_vp, _vp, _vp] + [C.c_int32] * 9 + [_vp, C.POINTER(_vp)]
 lib.taskkv_compress.restype = C.c_int32
 lib.taskkv_compress_host.argtypes = [C.POINTER(taskkv_params), _pp, _pp, _pp, _vp, C.POINTER(_vp)]
@@ -395,9 +398,10 @@ def taskkv_compress_host(params: Params, q_win: Sequence[torch.Tensor], k: Seque
     return Cache(h.value, params, {})
 
 
-def taskkv_exact_semantic(q: torch.Tensor, k: torch.Tensor, v: torch.Tensor, want_scores: bool = True, stream=None):
+def taskkv_exact_semantic(q: torch.Tensor, k: torch.Tensor, v: torch.Tensor, want_scores: bool = True, stream=None,
+                          workspace_mem: Optional[torch.Tensor] = None):
     """Eq. 1-2 for one sequence.  q: [R, n, N, d], k, v: [R, n_kv, N, d], contiguous bf16 CUDA tensors.
-    Returns (sem [R, n_kv, d] fp32, C [R, n_kv, N] fp32 or None)."""
+    Returns (sem [R, n_kv, d] fp32, C [R, n_kv, N] fp32 or None).  The scratch is a torch allocation unless supplied."""
     for t in (q, k, v):
         if not t.is_contiguous() or not t.is_cuda or t.dtype != torch.bfloat16:
             raise ValueError("inputs must be contiguous bf16 CUDA tensors")
@@ -407,9 +411,12 @@ def taskkv_exact_semantic(q: torch.Tensor, k: torch.Tensor, v: torch.Tensor, wan
         raise ValueError("k and v must be [R, n_kv, N, d] with q's R, N and d")
     sem = torch.empty(R, n_kv, d, dtype=torch.float32, device=q.device)
     c = torch.empty(R, n_kv, N, dtype=torch.float32, device=q.device) if want_scores else None
+    if workspace_mem is None:
+        workspace_mem = torch.empty(int(lib.taskkv_exact_semantic_bytes(R, n, n_kv, d, N)), dtype=torch.uint8,
+                                    device=q.device)
     _check(lib.taskkv_exact_semantic(q.data_ptr(), k.data_ptr(), v.data_ptr(), R, n, n_kv, d, N, sem.data_ptr(),
-                                     c.data_ptr() if c is not None else None, _stream_handle(stream)),
-           "taskkv_exact_semantic")
+                                     c.data_ptr() if c is not None else None, workspace_mem.data_ptr(),
+                                     workspace_mem.numel(), _stream_handle(stream)), "taskkv_exact_semantic")
     return sem, c
 
 

@@ -75,42 +75,93 @@ size_t align256(size_t x) { return (x + 255) / 256 * 256; }
 
 using namespace taskkv;
 
-extern "C" taskkv_status taskkv_exact_semantic(const void* q, const void* k, const void* v, int32_t n_layers,
-                                               int32_t n_heads, int32_t n_kv_heads, int32_t head_dim, int32_t seq_len,
-                                               float* sem_out, float* c_out, taskkv_stream stream) {
-  if (!q || !k || !v || !sem_out) return TASKKV_EINVAL;
-  if (n_layers < 1 || n_heads < 1 || n_kv_heads < 1 || n_heads % n_kv_heads != 0) return TASKKV_EINVAL;
-  if (head_dim != 64 && head_dim != 128) return TASKKV_EINVAL;
-  if (seq_len < 1 || seq_len > (1 << 20)) return TASKKV_EINVAL;
-  if (((uintptr_t)q | (uintptr_t)k | (uintptr_t)v) & 15) return TASKKV_EINVAL;
-  cudaStream_t s = static_cast<cudaStream_t>(stream);
-  const int N = seq_len, d = head_dim, G = n_heads / n_kv_heads;
-  const int nb = (N + kBlockRows - 1) / kBlockRows;
-  const int64_t q_heads = (int64_t)n_layers * n_heads, kv_heads = (int64_t)n_layers * n_kv_heads;
-  const int chunks = (nb * kBlockRows + kTcChunk - 1) / kTcChunk;
-  const int slices = (N + kSliceKeys - 1) / kSliceKeys;
-  if ((int64_t)nb * G * chunks > (1 << 24)) return TASKKV_EINVAL;
+namespace {
 
-  // query heads per round: whole KV groups, within ~1.5 GB of scratch, and a work-item count that fits an int
-  const size_t per_head = (size_t)block_off(nb) * 4 + (size_t)nb * chunks * 2 * kBlockRows * 8 +
-                          (size_t)nb * 2 * kBlockRows * 4 + (size_t)nb * 16;
-  int64_t hb = (int64_t)((size_t)1536 << 20) / (int64_t)per_head / G * G;
-  hb = std::max<int64_t>(G, std::min<int64_t>(hb, q_heads));
-  while (hb > G && hb * nb * chunks > (1 << 30)) hb -= G;
+struct ExactLayout {
+  size_t o_status, o_unit_N, o_c_off, o_Cb, o_spart, o_stat, o_cfull, o_part, total;
+};
+// Scratch for rounds of hb query heads (a multiple of G).
+ExactLayout exact_layout(int64_t hb, int nb, int chunks, int G, int N, int d, int slices, bool own_scores) {
+  ExactLayout l;
   const int64_t U = hb * nb;
-
   size_t o = 0;
   auto take = [&](size_t bytes) { size_t at = o; o = align256(o + bytes); return at; };
-  const size_t o_status = take(64);
-  const size_t o_unit_N = take((size_t)U * 4);
-  const size_t o_c_off = take((size_t)(U + 1) * 8);
-  const size_t o_Cb = take((size_t)hb * block_off(nb) * 4);
-  const size_t o_spart = take((size_t)U * chunks * 2 * kBlockRows * 8);
-  const size_t o_stat = take((size_t)U * 2 * kBlockRows * 4);
-  const size_t o_cfull = take(c_out ? 0 : (size_t)(hb / G) * N * 4);
-  const size_t o_part = take((size_t)(hb / G) * slices * d * 4);
-  unsigned char* ws = nullptr;
-  if (cudaMallocAsync(reinterpret_cast<void**>(&ws), o, s) != cudaSuccess) {
+  l.o_status = take(64);
+  l.o_unit_N = take((size_t)U * 4);
+  l.o_c_off = take((size_t)(U + 1) * 8);
+  l.o_Cb = take((size_t)hb * block_off(nb) * 4);
+  l.o_spart = take((size_t)U * chunks * 2 * kBlockRows * 8);
+  l.o_stat = take((size_t)U * 2 * kBlockRows * 4);
+  l.o_cfull = take(own_scores ? (size_t)(hb / G) * N * 4 : 0);
+  l.o_part = take((size_t)(hb / G) * slices * d * 4);
+  l.total = o;
+  return l;
+}
+
+struct ExactShape {
+  int N, d, G, nb, chunks, slices;
+  int64_t q_heads;
+  bool ok;
+};
+ExactShape exact_shape(int32_t n_layers, int32_t n_heads, int32_t n_kv_heads, int32_t head_dim, int32_t seq_len) {
+  ExactShape x = {};
+  if (n_layers < 1 || n_heads < 1 || n_kv_heads < 1 || n_heads % n_kv_heads != 0) return x;
+  if (head_dim != 64 && head_dim != 128) return x;
+  if (seq_len < 1 || seq_len > (1 << 20)) return x;
+  x.N = seq_len;
+  x.d = head_dim;
+  x.G = n_heads / n_kv_heads;
+  x.nb = (x.N + kBlockRows - 1) / kBlockRows;
+  x.chunks = (x.nb * kBlockRows + kTcChunk - 1) / kTcChunk;
+  x.slices = (x.N + kSliceKeys - 1) / kSliceKeys;
+  x.q_heads = (int64_t)n_layers * n_heads;
+  x.ok = (int64_t)x.nb * x.G * x.chunks <= (1 << 24);
+  return x;
+}
+// Most query heads per round: whole KV groups, a work-item count that fits an int, scratch within `budget` bytes
+// (0 if not even one group fits).
+int64_t exact_heads_per_round(const ExactShape& x, size_t budget) {
+  int64_t hb = x.q_heads;
+  while (hb > x.G && hb * x.nb * x.chunks > (1 << 30)) hb -= x.G;
+  while (hb > x.G && exact_layout(hb, x.nb, x.chunks, x.G, x.N, x.d, x.slices, true).total > budget)
+    hb = std::max<int64_t>(x.G, hb / 2 / x.G * x.G);
+  return exact_layout(hb, x.nb, x.chunks, x.G, x.N, x.d, x.slices, true).total <= budget ? hb : 0;
+}
+constexpr size_t kOwnBudget = (size_t)1536 << 20;   // what the library asks the stream's pool for by itself
+
+}  // namespace
+
+extern "C" size_t taskkv_exact_semantic_bytes(int32_t n_layers, int32_t n_heads, int32_t n_kv_heads, int32_t head_dim,
+                                              int32_t seq_len) {
+  const ExactShape x = exact_shape(n_layers, n_heads, n_kv_heads, head_dim, seq_len);
+  if (!x.ok) return 0;
+  int64_t hb = exact_heads_per_round(x, kOwnBudget);
+  if (hb == 0) hb = x.G;                              // one KV group is the least a round can do
+  return exact_layout(hb, x.nb, x.chunks, x.G, x.N, x.d, x.slices, true).total;
+}
+
+extern "C" taskkv_status taskkv_exact_semantic(const void* q, const void* k, const void* v, int32_t n_layers,
+                                               int32_t n_heads, int32_t n_kv_heads, int32_t head_dim, int32_t seq_len,
+                                               float* sem_out, float* c_out, void* workspace_mem,
+                                               size_t workspace_bytes, taskkv_stream stream) {
+  if (!q || !k || !v || !sem_out) return TASKKV_EINVAL;
+  const ExactShape x = exact_shape(n_layers, n_heads, n_kv_heads, head_dim, seq_len);
+  if (!x.ok) return TASKKV_EINVAL;
+  if (((uintptr_t)q | (uintptr_t)k | (uintptr_t)v) & 15) return TASKKV_EINVAL;
+  if (workspace_mem && ((uintptr_t)workspace_mem & 255)) return TASKKV_EINVAL;
+  cudaStream_t s = static_cast<cudaStream_t>(stream);
+  const int N = x.N, d = x.d, G = x.G, nb = x.nb, chunks = x.chunks, slices = x.slices;
+  const int64_t q_heads = x.q_heads;
+
+  int64_t hb = exact_heads_per_round(x, workspace_mem ? workspace_bytes : kOwnBudget);
+  if (hb == 0 && !workspace_mem) hb = G;
+  if (hb == 0) return TASKKV_EALLOC;
+  const ExactLayout lay = exact_layout(hb, nb, chunks, G, N, d, slices, true);
+  const size_t o_status = lay.o_status, o_unit_N = lay.o_unit_N, o_c_off = lay.o_c_off, o_Cb = lay.o_Cb,
+               o_spart = lay.o_spart, o_stat = lay.o_stat, o_cfull = lay.o_cfull, o_part = lay.o_part;
+  const int64_t U = hb * nb;
+  unsigned char* ws = static_cast<unsigned char*>(workspace_mem);
+  if (!ws && cudaMallocAsync(reinterpret_cast<void**>(&ws), lay.total, s) != cudaSuccess) {
     cudaGetLastError();
     return TASKKV_EALLOC;
   }
@@ -169,7 +220,7 @@ extern "C" taskkv_status taskkv_exact_semantic(const void* q, const void* k, con
   }
   int32_t dev_status = 0;
   if (e == cudaSuccess) e = cudaMemcpyAsync(&dev_status, ws + o_status, 4, cudaMemcpyDeviceToHost, s);
-  cudaFreeAsync(ws, s);
+  if (!workspace_mem) cudaFreeAsync(ws, s);
   if (e == cudaSuccess) e = cudaStreamSynchronize(s);
   if (e != cudaSuccess) {
     cudaGetLastError();

@@ -101,10 +101,15 @@ def test_invalid_arguments_are_rejected_before_any_launch(tk):
     assert tk.lib.taskkv_decode_step(None, None, None, None, None, None) == tk.EINVAL
     assert tk.lib.taskkv_decode_step_ex(None, None, None, None, None, 0, 1, None) == tk.EINVAL
     assert tk.lib.taskkv_cache_query(None, 0, None, 0) == tk.EINVAL
-    assert tk.lib.taskkv_exact_semantic(None, None, None, 1, 8, 8, 128, 512, None, None, None) == tk.EINVAL
+    assert tk.lib.taskkv_exact_semantic(None, None, None, 1, 8, 8, 128, 512, None, None, None, 0, None) == tk.EINVAL
     # argument checks come before any device work: a head dimension or a head grouping the kernels do not take
-    assert tk.lib.taskkv_exact_semantic(16, 16, 16, 1, 8, 8, 96, 512, 16, None, None) == tk.EINVAL
-    assert tk.lib.taskkv_exact_semantic(16, 16, 16, 1, 8, 3, 128, 512, 16, None, None) == tk.EINVAL
-    assert tk.lib.taskkv_exact_semantic(16, 16, 16, 1, 8, 8, 128, 0, 16, None, None) == tk.EINVAL
+    assert tk.lib.taskkv_exact_semantic(16, 16, 16, 1, 8, 8, 96, 512, 16, None, None, 0, None) == tk.EINVAL
+    assert tk.lib.taskkv_exact_semantic(16, 16, 16, 1, 8, 3, 128, 512, 16, None, None, 0, None) == tk.EINVAL
+    assert tk.lib.taskkv_exact_semantic(16, 16, 16, 1, 8, 8, 128, 0, 16, None, None, 0, None) == tk.EINVAL
+    assert tk.lib.taskkv_exact_semantic_bytes(1, 8, 8, 96, 512) == 0
+    # one round over all 64 query heads: the blocks' scores (64 b (b + 1) floats per head for b = 4 blocks) dominate
+    assert tk.lib.taskkv_exact_semantic_bytes(2, 32, 8, 128, 512) >= 64 * 64 * 4 * 5 * 4
+    # a scratch too small for even one KV group is refused before any device work
+    assert tk.lib.taskkv_exact_semantic(256, 256, 256, 1, 8, 8, 128, 4096, 256, None, 256, 1024, None) == tk.EALLOC
     assert tk.lib.taskkv_status_str(tk.ESTATE) == b"cache in wrong state"
     assert wl.retained_rows() == 3 * 512 + 5 * 68
