@@ -323,6 +323,14 @@ def test_window_scores_single_read(case):
     run_workload(wl, layers=[(b, r) for b in range(wl.batch) for r in (0, wl.n_layers - 1)])
 
 
+def test_window_scores_single_read_batch_of_ten_sequences():
+    """More sequences than one launch of the single-read kernel takes (eight), of very different lengths: the cluster
+    size follows the longest, short sequences leave most CTAs of a cluster without a tile."""
+    lens = [300, 9000, 1500, 4097, 129, 2048, 7000, 640, 5121, 3333]
+    wl = small("ten", n=4, n_kv=4, d=128, N=0, L=32, s1=4, s2=64, k=60, dtype="bf16", seq_lens=lens, steps=1)
+    run_workload(wl)
+
+
 def test_window_scores_single_read_moderate_heavy_keys():
     """A few keys per head well above the rest (scores stay within fp32 range of one another): full parity."""
     wl = small("heavy", n=4, n_kv=4, d=128, N=9000, L=32, s1=4, s2=64, k=100, dtype="bf16", steps=1)
