@@ -121,8 +121,8 @@ bool window_tc_supported(const DeviceProblem& p, int dtype);
 cudaError_t launch_window_scores_tc(const DeviceProblem& p, const WindowHostInfo& h, cudaStream_t s);
 cudaError_t launch_window_prefix(const DeviceProblem& p, const void* q, const void* k, int heads, int group, int N,
                                  cudaStream_t s);
-int window_res_team(const DeviceProblem& p, const WindowHostInfo& h);
-cudaError_t launch_window_scores_res(const DeviceProblem& p, const WindowHostInfo& h, int team, cudaStream_t s);
+bool window_res_supported(const DeviceProblem& p, const WindowHostInfo& h);
+cudaError_t launch_window_scores_res(const DeviceProblem& p, const WindowHostInfo& h, cudaStream_t s);
 cudaError_t launch_select(const DeviceProblem& p, int dtype, int max_N, cudaStream_t s);
 cudaError_t launch_separator_plan(const DeviceProblem& p, int n_br, cudaStream_t s);
 cudaError_t launch_gather(const DeviceProblem& p, int dtype, int64_t gather_items, cudaStream_t s);

@@ -4,9 +4,10 @@
 //
 // Eq. 13 sums the rows of the window's softmax, so every row's normaliser (over all N keys) is needed before
 // any column can be finished.  The two-launch kernel of window_score_tc.cu reads K a second time for that.
-// Here a thread-block cluster of T CTAs (T = 1, 2, 4, 8 or 16) owns one unit at a time; CTA c takes the
-// c-th slice of the unit's 128-key tiles (at most 16 of them) and keeps S^T[key, row] = K Q^T of every tile in
-// its own 32 columns of TMEM: 16 tiles x 32 columns x 128 lanes = all 512 columns.  Per unit:
+// Here a thread-block cluster of T CTAs (T = 1, 2, 4, 8 or 16, the smallest that holds the sequence) owns one unit
+// at a time; CTA c takes the c-th slice of the unit's 128-key tiles (at most 16 of them) and keeps
+// S^T[key, row] = K Q^T of every tile in its own 32 columns of TMEM: 16 tiles x 32 columns x 128 lanes = all 512
+// columns.  Per unit:
 //   step 1  as each tile's MMAs complete, the epilogue warps add exp2(s - c_row) into per-thread row sums
 //           (a TMEM lane is a key; c_row is the score of one visible key of the warp, so the sum holds a
 //           term equal to 1 and cannot vanish; should a sum overflow, or should the warp's reference key
@@ -510,77 +511,91 @@ inline int team_for(int max_tiles) {
   return team;
 }
 
+inline int seq_team(int N) { return team_for((N + kTile - 1) / kTile); }
+
+// One launch per cluster size in use and per eight sequences of it: a sequence is handled by the smallest cluster
+// that holds it, so that short sequences of a ragged batch do not leave most CTAs of a large cluster without a tile.
 template <int D>
-cudaError_t launch_res_d(const DeviceProblem& p, const WindowHostInfo& h, int team, cudaStream_t s) {
+cudaError_t launch_res_d(const DeviceProblem& p, const WindowHostInfo& h, cudaStream_t s) {
   const ResLayout lay = make_layout(D);
-  const int n_cl = max_clusters<D>(team, lay.total);
-  if (n_cl <= 0) return cudaErrorInvalidConfiguration;
   const int per_seq = p.R * p.n_kv;
-  for (int b0 = 0; b0 < h.batch; b0 += kMaxSeq) {
-    const int nb = h.batch - b0 < kMaxSeq ? h.batch - b0 : kMaxSeq;
-    ResMaps maps;
-    ResArgs a;
-    a.n_seq = nb;
-    a.item_off[0] = 0;
-    for (int i = 0; i < kMaxSeq; ++i) {
-      const int b = b0 + (i < nb ? i : 0);                  // unused slots repeat the first sequence
-      const int N = h.seq_lens[b];
-      if (!make_tensor_map_2d(&maps.k[i], h.k[b], D, (uint64_t)per_seq * (uint64_t)N, kTile)) return cudaErrorUnknown;
-      if (!make_tensor_map_2d(&maps.q[i], h.q[b], D, (uint64_t)per_seq * (uint64_t)kRows, kRows)) return cudaErrorUnknown;
-      a.u0[i] = b * per_seq;
-      a.N[i] = N;
-      a.tiles[i] = (N + kTile - 1) / kTile;
-      a.item_off[i + 1] = a.item_off[i] + (i < nb ? per_seq : 0);
+  for (int team = 1; team <= kMaxTeam; team *= 2) {
+    int b_next = 0;
+    for (;;) {
+      int seqs[kMaxSeq], nb = 0;
+      while (b_next < h.batch && nb < kMaxSeq) {
+        if (seq_team(h.seq_lens[b_next]) == team) seqs[nb++] = b_next;
+        ++b_next;
+      }
+      if (nb == 0) break;
+      const int n_cl = max_clusters<D>(team, lay.total);
+      if (n_cl <= 0) return cudaErrorInvalidConfiguration;
+      ResMaps maps;
+      ResArgs a;
+      a.n_seq = nb;
+      a.item_off[0] = 0;
+      for (int i = 0; i < kMaxSeq; ++i) {
+        const int b = seqs[i < nb ? i : 0];                   // unused slots repeat the first sequence
+        const int N = h.seq_lens[b];
+        if (!make_tensor_map_2d(&maps.k[i], h.k[b], D, (uint64_t)per_seq * (uint64_t)N, kTile)) return cudaErrorUnknown;
+        if (!make_tensor_map_2d(&maps.q[i], h.q[b], D, (uint64_t)per_seq * (uint64_t)kRows, kRows))
+          return cudaErrorUnknown;
+        a.u0[i] = b * per_seq;
+        a.N[i] = N;
+        a.tiles[i] = (N + kTile - 1) / kTile;
+        a.item_off[i + 1] = a.item_off[i] + (i < nb ? per_seq : 0);
+      }
+      a.n_items = a.item_off[nb];
+      const int clusters = a.n_items < n_cl ? a.n_items : n_cl;
+      a.steps = (a.n_items + clusters - 1) / clusters;
+      cudaLaunchConfig_t cfg = {};
+      cfg.gridDim = dim3(clusters * team, 1, 1);
+      cfg.blockDim = dim3(kThreads, 1, 1);
+      cfg.dynamicSmemBytes = lay.total;
+      cfg.stream = s;
+      cudaLaunchAttribute attr;
+      attr.id = cudaLaunchAttributeClusterDimension;
+      attr.val.clusterDim.x = team;
+      attr.val.clusterDim.y = 1;
+      attr.val.clusterDim.z = 1;
+      cfg.attrs = &attr;
+      cfg.numAttrs = 1;
+      cudaError_t e;
+      {
+        LaunchScope ls(K_WINDOW_TC, s);
+        e = cudaLaunchKernelEx(&cfg, window_res_kernel<D>, maps, p, a, lay);
+      }
+      if (e != cudaSuccess) return e;
     }
-    a.n_items = a.item_off[nb];
-    const int clusters = a.n_items < n_cl ? a.n_items : n_cl;
-    a.steps = (a.n_items + clusters - 1) / clusters;
-    cudaLaunchConfig_t cfg = {};
-    cfg.gridDim = dim3(clusters * team, 1, 1);
-    cfg.blockDim = dim3(kThreads, 1, 1);
-    cfg.dynamicSmemBytes = lay.total;
-    cfg.stream = s;
-    cudaLaunchAttribute attr;
-    attr.id = cudaLaunchAttributeClusterDimension;
-    attr.val.clusterDim.x = team;
-    attr.val.clusterDim.y = 1;
-    attr.val.clusterDim.z = 1;
-    cfg.attrs = &attr;
-    cfg.numAttrs = 1;
-    cudaError_t e;
-    {
-      LaunchScope ls(K_WINDOW_TC, s);
-      e = cudaLaunchKernelEx(&cfg, window_res_kernel<D>, maps, p, a, lay);
-    }
-    if (e != cudaSuccess) return e;
   }
   return cudaSuccess;
 }
 
 }  // namespace
 
-// Cluster size for this problem, or 0 when the single-read kernel does not take it: 32 window rows, every
-// sequence within 16 CTAs x 16 tiles, and a device that co-schedules enough clusters of that size to fill it.
-int window_res_team(const DeviceProblem& p, const WindowHostInfo& h) {
-  if (p.rows != kRows || p.L > kRows || h.lse != nullptr) return 0;
-  int max_tiles = 0;
-  for (int b = 0; b < h.batch; ++b) {
-    const int tiles = (h.seq_lens[b] + kTile - 1) / kTile;
-    if (tiles > max_tiles) max_tiles = tiles;
-  }
-  if (max_tiles > kMaxTeam * kSlots) return 0;
-  const int team = team_for(max_tiles);
-  const int smem = make_layout(p.d).total;
-  const int n_cl = p.d == 64 ? max_clusters<64>(team, smem) : max_clusters<128>(team, smem);
+// Whether the single-read kernel takes this problem: 32 window rows, every sequence within 16 CTAs x 16 tiles, and a
+// device that co-schedules enough clusters of every size in use to fill three quarters of its SMs.
+bool window_res_supported(const DeviceProblem& p, const WindowHostInfo& h) {
+  if (p.rows != kRows || p.L > kRows || h.lse != nullptr) return false;
   int dev = 0, n_sm = 0;
   cudaGetDevice(&dev);
   cudaDeviceGetAttribute(&n_sm, cudaDevAttrMultiProcessorCount, dev);
-  // worth it only when the clusters cover most of the device
-  return n_cl * team * 4 >= n_sm * 3 ? team : 0;
+  const int smem = make_layout(p.d).total;
+  bool checked[kMaxTeam + 1] = {false};
+  for (int b = 0; b < h.batch; ++b) {
+    const int tiles = (h.seq_lens[b] + kTile - 1) / kTile;
+    if (tiles > kMaxTeam * kSlots) return false;
+    const int team = team_for(tiles);
+    if (checked[team]) continue;
+    checked[team] = true;
+    const int n_cl = p.d == 64 ? max_clusters<64>(team, smem) : max_clusters<128>(team, smem);
+    if (n_cl * team * 4 < n_sm * 3) return false;
+  }
+  return true;
 }
 
-cudaError_t launch_window_scores_res(const DeviceProblem& p, const WindowHostInfo& h, int team, cudaStream_t s) {
-  return p.d == 64 ? launch_res_d<64>(p, h, team, s) : launch_res_d<128>(p, h, team, s);
+cudaError_t launch_window_scores_res(const DeviceProblem& p, const WindowHostInfo& h, cudaStream_t s) {
+  return p.d == 64 ? launch_res_d<64>(p, h, s) : launch_res_d<128>(p, h, s);
 }
 
 }  // namespace taskkv

@@ -710,7 +710,7 @@ cudaError_t launch_window_prefix(const DeviceProblem& p, const void* q, const vo
 
 cudaError_t launch_window_scores_tc(const DeviceProblem& p, const WindowHostInfo& h, cudaStream_t s) {
   // 32 window rows and sequences short enough for a unit's scores to stay in tensor memory: K is read once
-  if (const int team = window_res_team(p, h)) return launch_window_scores_res(p, h, team, s);
+  if (window_res_supported(p, h)) return launch_window_scores_res(p, h, s);
   return p.d == 64 ? launch_tc_d<64>(p, h, s) : launch_tc_d<128>(p, h, s);
 }
 
