@@ -8,15 +8,18 @@
 // at a time; CTA c takes the c-th slice of the unit's 128-key tiles (at most 16 of them) and keeps
 // S^T[key, row] = K Q^T of every tile in its own 32 columns of TMEM: 16 tiles x 32 columns x 128 lanes = all 512
 // columns.  Per unit:
-//   step 1  as each tile's MMAs complete, the epilogue warps add exp2(s - c_row) into per-thread row sums
-//           (a TMEM lane is a key; c_row is the score of one visible key of the warp, so the sum holds a
-//           term equal to 1 and cannot vanish; should a sum overflow, or should the warp's reference key
-//           fall into the causally masked tail, the warp redoes its tiles with its exact row maxima);
+//   step 1  as each tile's MMAs complete, an epilogue warp replaces its scores in place (tcgen05.ld, ex2,
+//           tcgen05.st) by e = exp2(s - c_row) and adds them into per-thread row sums (a TMEM lane is a key;
+//           c_row is the score of one visible key of the warp, so the sum holds a term equal to 1 and loses
+//           nothing that matters to underflow; should a term come near the top of the fp32 range, or should
+//           the warp's reference key fall into the causally masked tail, the warp walks its tiles again with
+//           its exact row maxima); masked scores become 0;
 //   exchange  the warps' partial (c, sum) pairs are merged per CTA and sent to every CTA of the cluster
 //           through distributed shared memory (st.async completing bytes on the receiver's mbarrier);
-//   step 2  every warp folds the T pairs of each row into one offset, walks its tiles in TMEM again
-//           and writes C[key] = sum_rows exp2(s - offset_row); each tile's columns are then handed back
-//           to the MMA issuer for the next unit.
+//   step 2  every warp folds the T pairs of each row into the row's offset, turns it into one weight per row,
+//           w = exp2(c_row - offset_row), walks its tiles in TMEM again and writes C[key] = sum_rows e w
+//           (no second exponential); each tile's columns are then handed back to the MMA issuer for the
+//           next unit.
 // K tiles of the next unit keep streaming into the shared-memory ring during exchange and step 2.
 // Warp roles: 0 TMA producer, 1 MMA issuer, 2-9 epilogue (two groups of four, alternating tiles).
 // Every wait inside the pipeline is bounded; after a time-out the CTA stops, its cluster peers run into
