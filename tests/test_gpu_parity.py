@@ -312,6 +312,8 @@ SINGLE_READ_CASES = [
     dict(n=2, n_kv=2, d=128, N=30001, L=32, s1=4, s2=256, k=512, dtype="bf16", nh=0),
     # two query heads per KV head with a 16-row window: 32 rows, causal limit by row % 16
     dict(n=8, n_kv=4, d=128, N=5003, L=16, s1=4, s2=64, k=100, dtype="bf16"),
+    # four query heads per KV head with an 8-row window
+    dict(n=8, n_kv=2, d=64, N=2500, L=8, s1=4, s2=64, k=100, dtype="bf16", nh=0),
     # a batch whose sequences need different slice sizes in one launch, more units than clusters
     dict(n=8, n_kv=8, d=128, N=0, L=32, s1=4, s2=64, k=120, dtype="bf16", R=3, seq_lens=[9000, 300, 16000, 2100], nh=2),
 ]
