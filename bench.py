@@ -402,6 +402,11 @@ def run_exact_semantic(tk, wl, qs, ks, vs):
            "tensor_frac": tflops / tpeak, "peak_kind": kind, "exp_per_s": 2 * scores / (ms * 1e-3), "kernel_ms": kern,
            "note": "two passes (row normalisers, column sums) over the causal half of Q K^T; one exponential per "
                    "score and pass bounds it before the tensor pipe does"}
+    # the share of the exact column means held by the t largest of them (the premise of Eq. 14), median over heads
+    _, c_exact = tk.taskkv_exact_semantic(q, k, v, want_scores=True, workspace_mem=ws)
+    top = torch.sort(c_exact[0], dim=1, descending=True).values.cumsum(dim=1)
+    out["top_t_mass"] = {str(t): float(top[:, min(t, N) - 1].median()) for t in (64, 256, 1024, 4096)}
+    del c_exact, top
     # how far the window's v' is from v, and whether the two pick the same far heads (one layer, one sequence)
     if wl.batch == 1:
         one = tk.params_from_workload(wl, max_new_tokens=0).layer(0)
