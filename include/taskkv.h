@@ -155,7 +155,7 @@ taskkv_status taskkv_compress_ex(const taskkv_params* p, const void* const* q_wi
  *   workspace_mem  device scratch, 256-byte aligned, owned by the caller, or NULL: then up to ~1.5 GB come from the
  *            stream's memory pool (cudaMallocAsync) and go back to it, which can cost more than the kernels.
  *            taskkv_exact_semantic_bytes gives the size with which all heads (or as many as fit 1.5 GB) go through
- *            in one round; with less, fewer heads go per round; EALLOC if not even one KV group fits.
+ *            in one batch; with less, fewer heads go per batch; EALLOC if not even one KV group fits.
  * head_dim 64 or 128, bf16 only.  The call returns after the stream has finished the work.
  * Errors: EINVAL (arguments), EALLOC, ECUDA, ETIMEOUT (a bounded wait inside a kernel ran out).
  */

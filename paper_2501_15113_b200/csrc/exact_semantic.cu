@@ -80,7 +80,7 @@ namespace {
 struct ExactLayout {
   size_t o_status, o_unit_N, o_c_off, o_Cb, o_spart, o_stat, o_cfull, o_part, total;
 };
-// Scratch for rounds of hb query heads (a multiple of G).
+// Scratch for batches of hb query heads (a multiple of G).
 ExactLayout exact_layout(int64_t hb, int nb, int chunks, int G, int N, int d, int slices, bool own_scores) {
   ExactLayout l;
   const int64_t U = hb * nb;
@@ -118,9 +118,9 @@ ExactShape exact_shape(int32_t n_layers, int32_t n_heads, int32_t n_kv_heads, in
   x.ok = (int64_t)x.nb * x.G * x.chunks <= (1 << 24);
   return x;
 }
-// Most query heads per round: whole KV groups, a work-item count that fits an int, scratch within `budget` bytes
+// Most query heads per batch: whole KV groups, a work-item count that fits an int, scratch within `budget` bytes
 // (0 if not even one group fits).
-int64_t exact_heads_per_round(const ExactShape& x, size_t budget) {
+int64_t exact_heads_per_batch(const ExactShape& x, size_t budget) {
   int64_t hb = x.q_heads;
   while (hb > x.G && hb * x.nb * x.chunks > (1 << 30)) hb -= x.G;
   while (hb > x.G && exact_layout(hb, x.nb, x.chunks, x.G, x.N, x.d, x.slices, true).total > budget)
@@ -135,8 +135,8 @@ extern "C" size_t taskkv_exact_semantic_bytes(int32_t n_layers, int32_t n_heads,
                                               int32_t seq_len) {
   const ExactShape x = exact_shape(n_layers, n_heads, n_kv_heads, head_dim, seq_len);
   if (!x.ok) return 0;
-  int64_t hb = exact_heads_per_round(x, kOwnBudget);
-  if (hb == 0) hb = x.G;                              // one KV group is the least a round can do
+  int64_t hb = exact_heads_per_batch(x, kOwnBudget);
+  if (hb == 0) hb = x.G;                              // one KV group is the least a batch can be
   return exact_layout(hb, x.nb, x.chunks, x.G, x.N, x.d, x.slices, true).total;
 }
 
@@ -153,7 +153,7 @@ extern "C" taskkv_status taskkv_exact_semantic(const void* q, const void* k, con
   const int N = x.N, d = x.d, G = x.G, nb = x.nb, chunks = x.chunks, slices = x.slices;
   const int64_t q_heads = x.q_heads;
 
-  int64_t hb = exact_heads_per_round(x, workspace_mem ? workspace_bytes : kOwnBudget);
+  int64_t hb = exact_heads_per_batch(x, workspace_mem ? workspace_bytes : kOwnBudget);
   if (hb == 0 && !workspace_mem) hb = G;
   if (hb == 0) return TASKKV_EALLOC;
   const ExactLayout lay = exact_layout(hb, nb, chunks, G, N, d, slices, true);
@@ -187,7 +187,7 @@ extern "C" taskkv_status taskkv_exact_semantic(const void* q, const void* k, con
   cudaError_t e = cudaMemsetAsync(ws + o_status, 0, 64, s);
   const size_t es = 2;
   for (int64_t h0 = 0; h0 < q_heads && e == cudaSuccess; h0 += hb) {
-    const int64_t hn = std::min<int64_t>(hb, q_heads - h0);          // query heads of this round (a multiple of G)
+    const int64_t hn = std::min<int64_t>(hb, q_heads - h0);          // query heads of this batch (a multiple of G)
     const int64_t kv0 = h0 / G, kvn = hn / G;
     p.U = (int32_t)(hn * nb);
     {
