@@ -540,9 +540,14 @@ cudaError_t launch_res_d(const DeviceProblem& p, const WindowHostInfo& h, cudaSt
       for (int i = 0; i < kMaxSeq; ++i) {
         const int b = seqs[i < nb ? i : 0];                   // unused slots repeat the first sequence
         const int N = h.seq_lens[b];
-        if (!make_tensor_map_2d(&maps.k[i], h.k[b], D, (uint64_t)per_seq * (uint64_t)N, kTile)) return cudaErrorUnknown;
-        if (!make_tensor_map_2d(&maps.q[i], h.q[b], D, (uint64_t)per_seq * (uint64_t)kRows, kRows))
-          return cudaErrorUnknown;
+        if (i >= nb) {
+          maps.k[i] = maps.k[0];
+          maps.q[i] = maps.q[0];
+        } else {
+          if (!make_tensor_map_2d(&maps.k[i], h.k[b], D, (uint64_t)per_seq * (uint64_t)N, kTile)) return cudaErrorUnknown;
+          if (!make_tensor_map_2d(&maps.q[i], h.q[b], D, (uint64_t)per_seq * (uint64_t)kRows, kRows))
+            return cudaErrorUnknown;
+        }
         a.u0[i] = b * per_seq;
         a.N[i] = N;
         a.tiles[i] = (N + kTile - 1) / kTile;

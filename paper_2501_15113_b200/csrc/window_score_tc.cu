@@ -608,8 +608,14 @@ cudaError_t launch_tc_d(const DeviceProblem& p, const WindowHostInfo& h, cudaStr
     for (int i = 0; i < kMaxSeq; ++i) {
       const int b = b0 + (i < nb ? i : 0);                  // unused slots repeat the first sequence
       const int N = h.seq_lens[b];
-      if (!make_tensor_map_2d(&maps.k[i], h.k[b], D, (uint64_t)per_seq * (uint64_t)N, kTile)) return cudaErrorUnknown;
-      if (!make_tensor_map_2d(&maps.q[i], h.q[b], D, (uint64_t)per_seq * (uint64_t)p.rows, p.rows)) return cudaErrorUnknown;
+      if (i >= nb) {
+        maps.k[i] = maps.k[0];
+        maps.q[i] = maps.q[0];
+      } else {
+        if (!make_tensor_map_2d(&maps.k[i], h.k[b], D, (uint64_t)per_seq * (uint64_t)N, kTile)) return cudaErrorUnknown;
+        if (!make_tensor_map_2d(&maps.q[i], h.q[b], D, (uint64_t)per_seq * (uint64_t)p.rows, p.rows))
+          return cudaErrorUnknown;
+      }
       a.u0[i] = b * per_seq;
       a.N[i] = N;
       a.chunks[i] = (N + a.chunk_keys - 1) / a.chunk_keys;
@@ -669,8 +675,13 @@ cudaError_t launch_prefix_d(const DeviceProblem& p, const void* q, const void* k
   a.chunk_keys = kTcChunk;
   a.item_off[0] = 0;
   for (int i = 0; i < kMaxSeq; ++i) {
-    if (!make_tensor_map_2d(&maps.k[i], k, D, (uint64_t)(heads / group) * (uint64_t)N, kTile)) return cudaErrorUnknown;
-    if (!make_tensor_map_2d(&maps.q[i], q, D, (uint64_t)heads * (uint64_t)N, p.rows)) return cudaErrorUnknown;
+    if (i > 0) {
+      maps.k[i] = maps.k[0];
+      maps.q[i] = maps.q[0];
+    } else {
+      if (!make_tensor_map_2d(&maps.k[i], k, D, (uint64_t)(heads / group) * (uint64_t)N, kTile)) return cudaErrorUnknown;
+      if (!make_tensor_map_2d(&maps.q[i], q, D, (uint64_t)heads * (uint64_t)N, p.rows)) return cudaErrorUnknown;
+    }
     a.u0[i] = 0;
     a.N[i] = N;
     a.chunks[i] = (blocks * kTile + a.chunk_keys - 1) / a.chunk_keys;
