@@ -203,6 +203,72 @@ void note_launch_end(int32_t id, cudaStream_t s) {
 }
 }  // namespace taskkv
 
+namespace {
+// Window scores and selection of different layers overlapped.  The single-read window kernel is bound by the K stream
+// and its clusters leave part of the SMs empty; the selection is bound by integer work on scores that sit in L2.  So the
+// layers are cut into chunks: the window kernel of chunk i+1 runs on the caller's stream while the selection of chunk i
+// runs on a side stream of the library (one per device, created on first use), joined back before the separator.
+constexpr int kMaxChunks = 8;
+struct SideStream {
+  cudaStream_t stream = nullptr;
+  cudaEvent_t ev[kMaxChunks + 1] = {};
+  bool ok = false, tried = false;
+};
+std::mutex g_side_mu;
+SideStream g_side[64];
+
+SideStream* side_stream() {   // call with g_side_mu held
+  int dev = 0;
+  if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) return nullptr;
+  SideStream& ss = g_side[dev];
+  if (!ss.tried) {
+    ss.tried = true;
+    ss.ok = cudaStreamCreateWithFlags(&ss.stream, cudaStreamNonBlocking) == cudaSuccess;
+    for (int i = 0; ss.ok && i <= kMaxChunks; ++i)
+      ss.ok = cudaEventCreateWithFlags(&ss.ev[i], cudaEventDisableTiming) == cudaSuccess;
+    if (!ss.ok) cudaGetLastError();
+  }
+  return ss.ok ? &ss : nullptr;
+}
+
+// How many chunks of layers to overlap (1 = do not): only where the single-read window kernel and the
+// register-resident selection run, with enough units per chunk to fill the window kernel's clusters many times over,
+// and not while per-kernel durations are being recorded (they are meant to be those of a kernel running alone).
+int overlap_chunks(const DeviceProblem& dp, int dtype, const WindowHostInfo& wh) {
+  if (g_timing.load(std::memory_order_relaxed)) return 1;
+  if (!window_tc_supported(dp, dtype) || !window_res_supported(dp, wh)) return 1;
+  const int batch = wh.batch;
+  int chunks = 1;
+  while (chunks * 2 <= kMaxChunks && chunks * 2 <= dp.R && (int64_t)(dp.R / (chunks * 2)) * dp.n_kv * batch >= 256)
+    chunks *= 2;
+  return chunks;
+}
+
+cudaError_t window_select_overlapped(const DeviceProblem& dp, int dtype, int max_N, const WindowHostInfo& wh,
+                                     int n_chunks, cudaStream_t s) {
+  std::lock_guard<std::mutex> lk(g_side_mu);
+  SideStream* ss = side_stream();
+  if (!ss) {
+    cudaError_t e = launch_window_scores(dp, dtype, max_N, wh, s);
+    return e == cudaSuccess ? launch_select(dp, dtype, max_N, s) : e;
+  }
+  const int per_seq = dp.R * dp.n_kv;
+  cudaError_t e = cudaSuccess;
+  for (int ch = 0; ch < n_chunks && e == cudaSuccess; ++ch) {
+    const int l0 = (int)((int64_t)dp.R * ch / n_chunks), l1 = (int)((int64_t)dp.R * (ch + 1) / n_chunks);
+    e = launch_window_scores_res(dp, wh, s, l0, l1 - l0);
+    if (e == cudaSuccess) e = cudaEventRecord(ss->ev[ch], s);
+    if (e == cudaSuccess) e = cudaStreamWaitEvent(ss->stream, ss->ev[ch], 0);
+    const UnitRange ur{l0 * dp.n_kv, (l1 - l0) * dp.n_kv, per_seq, wh.batch * (l1 - l0) * dp.n_kv};
+    if (e == cudaSuccess) e = launch_select(dp, dtype, max_N, ss->stream, &ur);
+  }
+  // always join, so that nothing of this call is left running on the side stream when the caller's stream moves on
+  cudaError_t j = cudaEventRecord(ss->ev[kMaxChunks], ss->stream);
+  if (j == cudaSuccess) j = cudaStreamWaitEvent(s, ss->ev[kMaxChunks], 0);
+  return e != cudaSuccess ? e : j;
+}
+}  // namespace
+
 struct taskkv_cache {
   taskkv_params prm;
   HostPlan hp;
@@ -448,8 +514,15 @@ taskkv_status compress_impl(const taskkv_params* p, const void* const* q_win, co
   wh.q = q_win;
   wh.k = k;
   wh.lse = window_lse;
-  if (e == cudaSuccess) e = launch_window_scores(c->dp, p->dtype, c->hp.max_N, wh, s);
-  if (e == cudaSuccess) e = launch_select(c->dp, p->dtype, c->hp.max_N, s);
+  if (e == cudaSuccess) {
+    const int n_chunks = overlap_chunks(c->dp, p->dtype, wh);
+    if (n_chunks > 1) {
+      e = window_select_overlapped(c->dp, p->dtype, c->hp.max_N, wh, n_chunks, s);
+    } else {
+      e = launch_window_scores(c->dp, p->dtype, c->hp.max_N, wh, s);
+      if (e == cudaSuccess) e = launch_select(c->dp, p->dtype, c->hp.max_N, s);
+    }
+  }
   if (e == cudaSuccess) e = launch_separator_plan(c->dp, p->batch * p->n_layers, s);
   if (e == cudaSuccess) e = launch_gather(c->dp, p->dtype, c->hp.info.gather_items, s);
   if (e == cudaSuccess && p->mid_policy == TASKKV_MID_MEAN) e = launch_compensate(c->dp, p->dtype, s);

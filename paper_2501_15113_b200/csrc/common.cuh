@@ -100,6 +100,13 @@ struct LaunchScope {
   ~LaunchScope() { note_launch_end(id, s); }
 };
 
+// A launch over part of the units: `count` consecutive units starting at `first` inside every sequence's block of
+// `per_seq` units (units are numbered [sequence][layer][kv head], so this is a range of layers of every sequence).
+struct UnitRange {
+  int32_t first, count, per_seq, blocks;   // blocks = sequences * count
+  __host__ __device__ int unit(int block) const { return (block / count) * per_seq + first + block % count; }
+};
+
 // Host-side view of the inputs, for launchers that build per-sequence descriptors.
 struct WindowHostInfo {
   int batch;
@@ -122,8 +129,11 @@ cudaError_t launch_window_scores_tc(const DeviceProblem& p, const WindowHostInfo
 cudaError_t launch_window_prefix(const DeviceProblem& p, const void* q, const void* k, int heads, int group, int N,
                                  cudaStream_t s);
 bool window_res_supported(const DeviceProblem& p, const WindowHostInfo& h);
-cudaError_t launch_window_scores_res(const DeviceProblem& p, const WindowHostInfo& h, cudaStream_t s);
-cudaError_t launch_select(const DeviceProblem& p, int dtype, int max_N, cudaStream_t s);
+// layers [layer0, layer0 + n_layers) of every sequence; n_layers < 0: all of them
+cudaError_t launch_window_scores_res(const DeviceProblem& p, const WindowHostInfo& h, cudaStream_t s, int layer0 = 0,
+                                     int n_layers = -1);
+cudaError_t launch_select(const DeviceProblem& p, int dtype, int max_N, cudaStream_t s,
+                          const UnitRange* range = nullptr);
 cudaError_t launch_separator_plan(const DeviceProblem& p, int n_br, cudaStream_t s);
 cudaError_t launch_gather(const DeviceProblem& p, int dtype, int64_t gather_items, cudaStream_t s);
 cudaError_t launch_compensate(const DeviceProblem& p, int dtype, cudaStream_t s);

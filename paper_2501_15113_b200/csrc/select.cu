@@ -5,10 +5,16 @@
 //   with the sinks and the recent window as the unit's ascending index list.
 // Both selections find the exact k-th largest order-preserving 32-bit key by bisection
 // over the key bits, followed by an ordered compaction; of equal scores the lower
-// position wins.  Up to 32768 positions the keys live in registers (select_fast_kernel);
-// longer units stream them from L2 once per bisection step until few enough survive to
-// be collected in shared memory (select_kernel).
+// position wins.  Up to 32768 positions the keys live in the registers of one block
+// (select_fast_kernel), up to 262144 in those of a thread-block cluster
+// (select_cluster_kernel); longer units, or other pooling kernels, stream them from L2
+// once per bisection step until few enough survive to be collected in shared memory
+// (select_kernel).
+#include <cooperative_groups.h>
+
 #include "common.cuh"
+
+namespace cg = cooperative_groups;
 
 namespace taskkv {
 
@@ -193,12 +199,12 @@ __device__ void block_compact(SelectSmem& sm, int lo, int hi, uint32_t thr, int 
 }
 
 template <typename T, int D>
-__global__ void __launch_bounds__(kThreads) select_kernel(DeviceProblem p) {
+__global__ void __launch_bounds__(kThreads) select_kernel(DeviceProblem p, UnitRange ur) {
   __shared__ SelectSmem sm;
   __shared__ int sel[TASKKV_MAX_TOP_T];
   __shared__ float red[kWarps][D];
 
-  const int u = blockIdx.x;
+  const int u = ur.unit(blockIdx.x);
   const int N = p.unit_N[u];
   const float* C = p.C + p.c_off[u];
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
@@ -430,13 +436,13 @@ __device__ void block_compact_regs(FastSmem& fs, const uint32_t (&key)[kEpt], in
 }
 
 template <typename T, int D, int POOL_HALF>
-__global__ void __launch_bounds__(kThreads, 1) select_fast_kernel(DeviceProblem p) {
+__global__ void __launch_bounds__(kThreads, 1) select_fast_kernel(DeviceProblem p, UnitRange ur) {
   __shared__ FastSmem fs;
   __shared__ int sel[TASKKV_MAX_TOP_T];
   __shared__ float selw[TASKKV_MAX_TOP_T];
   __shared__ float red[kWarps][D];
 
-  const int u = blockIdx.x;
+  const int u = ur.unit(blockIdx.x);
   const int N = p.unit_N[u];
   const float* C = p.C + p.c_off[u];
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
@@ -541,30 +547,337 @@ __global__ void __launch_bounds__(kThreads, 1) select_fast_kernel(DeviceProblem 
   block_compact_regs(fs, key, base, thr, need_eq, [&](int pos, int j) { idx[s1 + pos] = j; });
 }
 
+// ---------------------------------------------------------------------------
+// Cluster variant for 32768 < N <= 262144 (and pooling kernel 1 or 7): a thread-block cluster of 2, 4 or 8 CTAs
+// owns a unit, CTA c keeps positions [32768 c, 32768 (c + 1)) in registers exactly as select_fast_kernel does, and
+// every block-wide count becomes a cluster-wide one: each warp leaves its count in a slot of every CTA's shared
+// memory (distributed shared memory), one cluster barrier, and every thread adds up all slots.  The slots are
+// double-buffered by step parity: a slot is rewritten two barriers after it was read.  Same results as the other
+// two kernels: exact k-th key, lower position first among equal keys, pooled sums added in ascending position.
+constexpr int kMaxCS = 8;
+
+struct ClusterSmem {
+  int cnt[2][kMaxCS][kWarps];
+  uint32_t mn[kMaxCS][kWarps], mx[kMaxCS][kWarps];
+  int tot[2][kMaxCS][2];     // per compaction and CTA: keys above the threshold, keys equal to it
+  int scan[kWarps];
+  int list_n;
+};
+
+// Sum over the whole cluster of one int per warp (v: this warp's value, already reduced over the warp).
+__device__ __forceinline__ int cluster_sum(cg::cluster_group& cl, ClusterSmem& cs, int cs_n, int rank, int par, int v) {
+  const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+  if (lane < cs_n) cl.map_shared_rank(&cs.cnt[par][rank][warp], lane)[0] = v;
+  cl.sync();
+  int acc = 0;
+  for (int r = 0; r < cs_n; ++r) acc += cs.cnt[par][r][lane];
+  return __reduce_add_sync(0xffffffffu, acc);
+}
+
+__device__ __forceinline__ int cluster_count_ge(cg::cluster_group& cl, ClusterSmem& cs, int cs_n, int rank, int par,
+                                                const uint32_t (&key)[kEpt], uint32_t cand) {
+  int c = 0;
+#pragma unroll
+  for (int e = 0; e < kEpt; ++e) c += (key[e] >= cand) ? 1 : 0;
+  c = __reduce_add_sync(0xffffffffu, c);
+  return cluster_sum(cl, cs, cs_n, rank, par, c);
+}
+
+// block_bisect over the keys of the whole cluster.  In the narrow phase every CTA collects its own surviving keys
+// (at most kNarrow in the whole cluster, so at most one per thread) and the packed counts are summed over the cluster.
+__device__ void cluster_bisect(cg::cluster_group& cl, ClusterSmem& cs, int cs_n, int rank, const uint32_t (&key)[kEpt],
+                               int want, uint32_t* list, int cap, uint32_t& thr, int& need_eq) {
+  const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+  uint32_t lo = 0xffffffffu, hi = 0u;
+#pragma unroll
+  for (int e = 0; e < kEpt; ++e)
+    if (key[e]) { lo = min(lo, key[e]); hi = max(hi, key[e]); }
+  lo = __reduce_min_sync(0xffffffffu, lo);
+  hi = __reduce_max_sync(0xffffffffu, hi);
+  if (lane < cs_n) {
+    cl.map_shared_rank(&cs.mn[rank][warp], lane)[0] = lo;
+    cl.map_shared_rank(&cs.mx[rank][warp], lane)[0] = hi;
+  }
+  if (threadIdx.x == 0) cs.list_n = 0;
+  cl.sync();
+  lo = 0xffffffffu; hi = 0u;
+  for (int r = 0; r < cs_n; ++r) { lo = min(lo, cs.mn[r][lane]); hi = max(hi, cs.mx[r][lane]); }
+  lo = __reduce_min_sync(0xffffffffu, lo);
+  hi = __reduce_max_sync(0xffffffffu, hi);
+  const uint32_t diff = lo ^ hi;
+  int bit = diff ? 31 - __clz(diff) : -1;
+  uint32_t t = diff ? (hi & ~((2u << bit) - 1u)) : hi;
+  int par = 0;
+  int above = 0;
+  int at_least = 1 << 30;
+  const int narrow = min(cap, kNarrow);
+  for (; bit >= 0 && at_least - above > narrow; --bit) {
+    const uint32_t cand = t | (1u << bit);
+    const int c = cluster_count_ge(cl, cs, cs_n, rank, par, key, cand);
+    if (c >= want) { t = cand; at_least = c; } else above = c;
+    par ^= 1;
+  }
+  if (bit >= 0) {
+    const uint32_t top = t + (2u << bit);            // end of the undecided range (0 if it wraps: no upper bound)
+#pragma unroll
+    for (int e = 0; e < kEpt; ++e)
+      if (key[e] >= t && (top == 0u || key[e] < top)) list[atomicAdd(&cs.list_n, 1)] = key[e];
+    __syncthreads();
+    const int alive = cs.list_n;                     // this CTA's share of the at most kNarrow survivors
+    const uint32_t mine = (int)threadIdx.x < alive ? list[threadIdx.x] : 0u;
+    const int want2 = want - above;                  // rank inside the collected keys
+    while (bit >= 0) {
+      const uint32_t b_hi = 1u << bit, b_lo = bit > 0 ? 1u << (bit - 1) : 0u;
+      const uint32_t c10 = t | b_hi, c11 = c10 | b_lo, c01 = t | b_lo;
+      int v = (int)(mine >= c10) | ((int)(mine >= c11) << 10) | ((int)(b_lo != 0u && mine >= c01) << 20);
+      v = __reduce_add_sync(0xffffffffu, v);
+      v = cluster_sum(cl, cs, cs_n, rank, par, v);
+      par ^= 1;
+      const int n10 = v & 0x3ff, n11 = (v >> 10) & 0x3ff, n01 = (v >> 20) & 0x3ff;
+      if (b_lo != 0u && n11 >= want2) t = c11;
+      else if (n10 >= want2) t = c10;
+      else if (b_lo != 0u && n01 >= want2) t = c01;
+      bit -= 2;
+    }
+  }
+  const int n_gt = (t == 0xffffffffu) ? 0 : cluster_count_ge(cl, cs, cs_n, rank, par, key, t + 1u);
+  thr = t;
+  need_eq = want - n_gt;
+  __syncthreads();
+}
+
+// block_compact_regs with the ranks continued across the CTAs of the cluster (`which` names the totals' slot).
+template <class Emit>
+__device__ void cluster_compact_regs(cg::cluster_group& cl, ClusterSmem& cs, int cs_n, int rank, int which,
+                                     const uint32_t (&key)[kEpt], int base, uint32_t thr, int need_eq,
+                                     const Emit& emit) {
+  static_assert(kEpt == 32, "one mask bit per key");
+  const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+  uint32_t m_gt = 0u, m_ge = 0u;
+#pragma unroll
+  for (int e = 0; e < kEpt; ++e) {
+    m_gt |= (uint32_t)(key[e] > thr) << e;
+    m_ge |= (uint32_t)(key[e] >= thr) << e;
+  }
+  const int gt = __popc(m_gt), eq = __popc(m_ge) - gt;
+  const int packed = gt | (eq << 16);                 // a CTA holds 32768 keys: both fields stay below 2^16
+  int incl = packed;
+#pragma unroll
+  for (int o = 1; o < 32; o <<= 1) {
+    const int y = __shfl_up_sync(0xffffffffu, incl, o);
+    if (lane >= o) incl += y;
+  }
+  if (lane == 31) cs.scan[warp] = incl;
+  __syncthreads();
+  int wp = cs.scan[lane];
+  int wi = wp;
+#pragma unroll
+  for (int o = 1; o < 32; o <<= 1) {
+    const int y = __shfl_up_sync(0xffffffffu, wi, o);
+    if (lane >= o) wi += y;
+  }
+  const int wexcl = __shfl_sync(0xffffffffu, wi - wp, warp);
+  const int excl = incl - packed + wexcl;
+  const int total = __shfl_sync(0xffffffffu, wi, 31);   // this CTA's totals
+  if (warp == 0 && lane < cs_n) {
+    int* dst = cl.map_shared_rank(&cs.tot[which][rank][0], lane);
+    dst[0] = total & 0xffff;
+    dst[1] = (int)((uint32_t)total >> 16);            // 32768 equal keys fill the sign bit of the packed word
+  }
+  cl.sync();
+  int gt_before = excl & 0xffff, eq_before = excl >> 16;
+  for (int r = 0; r < rank; ++r) { gt_before += cs.tot[which][r][0]; eq_before += cs.tot[which][r][1]; }
+  for (uint32_t m = m_ge; m != 0u; m &= m - 1u) {
+    const int e = __ffs((int)m) - 1;
+    const bool g = (m_gt >> e) & 1u;
+    if (g || eq_before < need_eq) emit(gt_before + min(eq_before, need_eq), base + e);
+    gt_before += g;
+    eq_before += !g;
+  }
+  __syncthreads();
+}
+
+template <typename T, int D, int POOL_HALF>
+__global__ void __launch_bounds__(kThreads, 1) select_cluster_kernel(DeviceProblem p, UnitRange ur) {
+  __shared__ ClusterSmem cs;
+  __shared__ int sel[TASKKV_MAX_TOP_T];
+  __shared__ float selw[TASKKV_MAX_TOP_T];
+  __shared__ float red[kWarps][D];
+  __shared__ float vpart[kMaxCS][D];
+
+  cg::cluster_group cl = cg::this_cluster();
+  const int cs_n = (int)cl.num_blocks();
+  const int rank = (int)cl.block_rank();
+  const int u = ur.unit(blockIdx.x / cs_n);
+  const int N = p.unit_N[u];
+  const float* C = p.C + p.c_off[u];
+  const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+  const int base = (rank * kThreads + tid) * kEpt;
+
+  uint32_t key[kEpt];
+  if (base + kEpt <= N && ((reinterpret_cast<uintptr_t>(C + base) & 15) == 0)) {
+#pragma unroll
+    for (int e = 0; e < kEpt; e += 4) {
+      const float4 v = *reinterpret_cast<const float4*>(C + base + e);
+      key[e] = ordered_key(v.x); key[e + 1] = ordered_key(v.y);
+      key[e + 2] = ordered_key(v.z); key[e + 3] = ordered_key(v.w);
+    }
+  } else {
+#pragma unroll
+    for (int e = 0; e < kEpt; ++e) key[e] = (base + e < N) ? ordered_key(C[base + e]) : 0u;
+  }
+
+  // ---- Eq. 14: I = top-min(t, N) of C; every CTA receives the whole list
+  const int t = min(p.top_t, N);
+  uint32_t thr;
+  int need_eq;
+  uint32_t* scratch = reinterpret_cast<uint32_t*>(&red[0][0]);   // free until the semantic vector is summed
+  cluster_bisect(cl, cs, cs_n, rank, key, t, scratch, kWarps * D, thr, need_eq);
+  int* topt = p.topt + (size_t)u * p.top_t;
+  cluster_compact_regs(cl, cs, cs_n, rank, 0, key, base, thr, need_eq, [&](int pos, int j) {
+    const float w = C[j];
+    for (int r = 0; r < cs_n; ++r) {
+      cl.map_shared_rank(&sel[pos], r)[0] = j;
+      cl.map_shared_rank(&selw[pos], r)[0] = w;
+    }
+    topt[pos] = j;
+  });
+  if (rank == 0)
+    for (int i = t + tid; i < p.top_t; i += kThreads) topt[i] = -1;
+  cl.sync();
+
+  // ---- Eq. 15: v' = sum_{j in I} C[j] V[j,:]: the CTAs share the t rows, fixed summation order
+  constexpr int EPL = D / 32;
+  float acc[EPL];
+#pragma unroll
+  for (int e = 0; e < EPL; ++e) acc[e] = 0.f;
+  const T* V = static_cast<const T*>(p.v_ptr[u]);
+  for (int i = rank * kWarps + warp; i < t; i += cs_n * kWarps) {
+    const float w = selw[i];
+    const T* row = V + (size_t)sel[i] * D + lane * EPL;
+#pragma unroll
+    for (int e = 0; e < EPL; ++e) acc[e] = fmaf(w, to_float(row[e]), acc[e]);
+  }
+#pragma unroll
+  for (int e = 0; e < EPL; ++e) red[warp][lane * EPL + e] = acc[e];
+  __syncthreads();
+  if (tid < D) {
+    float s = 0.f;
+    for (int w = 0; w < kWarps; ++w) s += red[w][tid];
+    cl.map_shared_rank(&vpart[rank][tid], 0)[0] = s;
+  }
+  cl.sync();
+  if (rank == 0 && tid < D) {
+    float s = 0.f;
+    for (int r = 0; r < cs_n; ++r) s += vpart[r][tid];
+    p.sem[(size_t)u * D + tid] = s;
+  }
+
+  // ---- Sec. IV-B: sinks, middle activations (top-k of the pooled scores), recent window
+  // (every condition below depends on the unit alone, so the CTAs of a cluster leave together)
+  const int s1 = p.sink, s2 = p.recent;
+  if (N <= s1 + s2) return;
+  const int lo = s1, hi = N - s2;
+  const int kmid = min(p.unit_mid[u], hi - lo);
+  if (kmid >= hi - lo) return;
+  int* idx = p.idx + (size_t)u * p.idx_stride;
+  const int ctid = rank * kThreads + tid, cthreads = cs_n * kThreads;
+  for (int i = ctid; i < s1; i += cthreads) idx[i] = i;
+  for (int i = ctid; i < s2; i += cthreads) idx[s1 + kmid + i] = N - s2 + i;
+  if (p.mid_policy != TASKKV_MID_SELECT) {
+    for (int i = ctid; i < kmid; i += cthreads)
+      idx[s1 + i] = p.mid_policy == TASKKV_MID_RECENT ? hi - kmid + i
+                                                     : lo + (int)(((int64_t)i * (hi - lo)) / kmid);
+    return;
+  }
+  if (kmid == 0) return;
+
+  if (POOL_HALF > 0) {
+    float ext[kEpt + 2 * POOL_HALF];
+#pragma unroll
+    for (int h = 0; h < POOL_HALF; ++h) {
+      const int jl = base - POOL_HALF + h, jr = base + kEpt + h;
+      ext[h] = (jl >= 0 && jl < N) ? C[jl] : 0.f;
+      ext[POOL_HALF + kEpt + h] = (jr < N) ? C[jr] : 0.f;
+    }
+#pragma unroll
+    for (int e = 0; e < kEpt; ++e) ext[POOL_HALF + e] = (base + e < N) ? key_score(key[e]) : 0.f;
+#pragma unroll
+    for (int e = 0; e < kEpt; ++e) {
+      float sum = 0.f;
+#pragma unroll
+      for (int o = 0; o <= 2 * POOL_HALF; ++o) sum += ext[e + o];
+      const int j = base + e;
+      key[e] = (j >= lo && j < hi) ? ordered_key(sum) : 0u;
+    }
+  } else {
+#pragma unroll
+    for (int e = 0; e < kEpt; ++e) {
+      const int j = base + e;
+      if (!(j >= lo && j < hi)) key[e] = 0u;
+    }
+  }
+  __syncthreads();
+  cluster_bisect(cl, cs, cs_n, rank, key, kmid, scratch, kWarps * D, thr, need_eq);
+  cluster_compact_regs(cl, cs, cs_n, rank, 1, key, base, thr, need_eq, [&](int pos, int j) { idx[s1 + pos] = j; });
+}
+
+template <typename T, int D, int POOL_HALF>
+cudaError_t launch_cluster_k(const DeviceProblem& p, const UnitRange& ur, int cs_n, cudaStream_t s) {
+  cudaLaunchConfig_t cfg = {};
+  cfg.gridDim = dim3((unsigned)(ur.blocks * cs_n), 1, 1);
+  cfg.blockDim = dim3(kThreads, 1, 1);
+  cfg.dynamicSmemBytes = 0;
+  cfg.stream = s;
+  cudaLaunchAttribute attr;
+  attr.id = cudaLaunchAttributeClusterDimension;
+  attr.val.clusterDim.x = (unsigned)cs_n;
+  attr.val.clusterDim.y = 1;
+  attr.val.clusterDim.z = 1;
+  cfg.attrs = &attr;
+  cfg.numAttrs = 1;
+  return cudaLaunchKernelEx(&cfg, select_cluster_kernel<T, D, POOL_HALF>, p, ur);
+}
+
 template <typename T, int D>
-void launch_fast(const DeviceProblem& p, cudaStream_t s) {
-  if (p.pool_w == 7) select_fast_kernel<T, D, 3><<<p.U, kThreads, 0, s>>>(p);
-  else select_fast_kernel<T, D, 0><<<p.U, kThreads, 0, s>>>(p);
+cudaError_t launch_cluster(const DeviceProblem& p, const UnitRange& ur, int cs_n, cudaStream_t s) {
+  return p.pool_w == 7 ? launch_cluster_k<T, D, 3>(p, ur, cs_n, s) : launch_cluster_k<T, D, 0>(p, ur, cs_n, s);
+}
+
+template <typename T, int D>
+void launch_fast(const DeviceProblem& p, const UnitRange& ur, cudaStream_t s) {
+  if (p.pool_w == 7) select_fast_kernel<T, D, 3><<<ur.blocks, kThreads, 0, s>>>(p, ur);
+  else select_fast_kernel<T, D, 0><<<ur.blocks, kThreads, 0, s>>>(p, ur);
 }
 
 }  // namespace
 
-cudaError_t launch_select(const DeviceProblem& p, int dtype, int max_N, cudaStream_t s) {
+cudaError_t launch_select(const DeviceProblem& p, int dtype, int max_N, cudaStream_t s, const UnitRange* range) {
   LaunchScope ls(K_SELECT, s);
+  const UnitRange ur = range ? *range : UnitRange{0, p.U, p.U, p.U};
+  if (ur.blocks <= 0) return cudaSuccess;
   if (max_N <= kThreads * kEpt && (p.pool_w == 7 || p.pool_w == 1)) {
     if (dtype == TASKKV_F32) {
-      if (p.d == 64) launch_fast<float, 64>(p, s); else launch_fast<float, 128>(p, s);
+      if (p.d == 64) launch_fast<float, 64>(p, ur, s); else launch_fast<float, 128>(p, ur, s);
     } else {
-      if (p.d == 64) launch_fast<__nv_bfloat16, 64>(p, s); else launch_fast<__nv_bfloat16, 128>(p, s);
+      if (p.d == 64) launch_fast<__nv_bfloat16, 64>(p, ur, s); else launch_fast<__nv_bfloat16, 128>(p, ur, s);
     }
     return cudaGetLastError();
   }
+  if (max_N <= kMaxCS * kThreads * kEpt && (p.pool_w == 7 || p.pool_w == 1)) {
+    int cs_n = 2;
+    while (cs_n * kThreads * kEpt < max_N) cs_n *= 2;
+    if (dtype == TASKKV_F32)
+      return p.d == 64 ? launch_cluster<float, 64>(p, ur, cs_n, s) : launch_cluster<float, 128>(p, ur, cs_n, s);
+    return p.d == 64 ? launch_cluster<__nv_bfloat16, 64>(p, ur, cs_n, s)
+                     : launch_cluster<__nv_bfloat16, 128>(p, ur, cs_n, s);
+  }
   if (dtype == TASKKV_F32) {
-    if (p.d == 64) select_kernel<float, 64><<<p.U, kThreads, 0, s>>>(p);
-    else select_kernel<float, 128><<<p.U, kThreads, 0, s>>>(p);
+    if (p.d == 64) select_kernel<float, 64><<<ur.blocks, kThreads, 0, s>>>(p, ur);
+    else select_kernel<float, 128><<<ur.blocks, kThreads, 0, s>>>(p, ur);
   } else {
-    if (p.d == 64) select_kernel<__nv_bfloat16, 64><<<p.U, kThreads, 0, s>>>(p);
-    else select_kernel<__nv_bfloat16, 128><<<p.U, kThreads, 0, s>>>(p);
+    if (p.d == 64) select_kernel<__nv_bfloat16, 64><<<ur.blocks, kThreads, 0, s>>>(p, ur);
+    else select_kernel<__nv_bfloat16, 128><<<ur.blocks, kThreads, 0, s>>>(p, ur);
   }
   return cudaGetLastError();
 }

@@ -519,9 +519,12 @@ inline int seq_team(int N) { return team_for((N + kTile - 1) / kTile); }
 // One launch per cluster size in use and per eight sequences of it: a sequence is handled by the smallest cluster
 // that holds it, so that short sequences of a ragged batch do not leave most CTAs of a large cluster without a tile.
 template <int D>
-cudaError_t launch_res_d(const DeviceProblem& p, const WindowHostInfo& h, cudaStream_t s) {
+cudaError_t launch_res_d(const DeviceProblem& p, const WindowHostInfo& h, cudaStream_t s, int layer0, int n_layers) {
   const ResLayout lay = make_layout(D);
-  const int per_seq = p.R * p.n_kv;
+  const int per_seq_all = p.R * p.n_kv;
+  const int first = layer0 * p.n_kv;               // the launch covers units [first, first + per_seq) of every sequence
+  const int per_seq = n_layers * p.n_kv;
+  if (per_seq <= 0) return cudaSuccess;
   for (int team = 1; team <= kMaxTeam; team *= 2) {
     int b_next = 0;
     for (;;) {
@@ -544,11 +547,13 @@ cudaError_t launch_res_d(const DeviceProblem& p, const WindowHostInfo& h, cudaSt
           maps.k[i] = maps.k[0];
           maps.q[i] = maps.q[0];
         } else {
-          if (!make_tensor_map_2d(&maps.k[i], h.k[b], D, (uint64_t)per_seq * (uint64_t)N, kTile)) return cudaErrorUnknown;
-          if (!make_tensor_map_2d(&maps.q[i], h.q[b], D, (uint64_t)per_seq * (uint64_t)kRows, kRows))
+          const char* kb = static_cast<const char*>(h.k[b]) + (size_t)first * (size_t)N * D * sizeof(__nv_bfloat16);
+          const char* qb = static_cast<const char*>(h.q[b]) + (size_t)first * kRows * D * sizeof(__nv_bfloat16);
+          if (!make_tensor_map_2d(&maps.k[i], kb, D, (uint64_t)per_seq * (uint64_t)N, kTile)) return cudaErrorUnknown;
+          if (!make_tensor_map_2d(&maps.q[i], qb, D, (uint64_t)per_seq * (uint64_t)kRows, kRows))
             return cudaErrorUnknown;
         }
-        a.u0[i] = b * per_seq;
+        a.u0[i] = b * per_seq_all + first;
         a.N[i] = N;
         a.tiles[i] = (N + kTile - 1) / kTile;
         a.item_off[i + 1] = a.item_off[i] + (i < nb ? per_seq : 0);
@@ -602,8 +607,10 @@ bool window_res_supported(const DeviceProblem& p, const WindowHostInfo& h) {
   return true;
 }
 
-cudaError_t launch_window_scores_res(const DeviceProblem& p, const WindowHostInfo& h, cudaStream_t s) {
-  return p.d == 64 ? launch_res_d<64>(p, h, s) : launch_res_d<128>(p, h, s);
+cudaError_t launch_window_scores_res(const DeviceProblem& p, const WindowHostInfo& h, cudaStream_t s, int layer0,
+                                     int n_layers) {
+  if (n_layers < 0) { layer0 = 0; n_layers = p.R; }
+  return p.d == 64 ? launch_res_d<64>(p, h, s, layer0, n_layers) : launch_res_d<128>(p, h, s, layer0, n_layers);
 }
 
 }  // namespace taskkv

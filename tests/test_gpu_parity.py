@@ -277,10 +277,52 @@ def test_llama3_shaped_gqa_with_budget_schedule():
     assert 0.39 < wl.retained_rows() / full <= 0.4
 
 
-def test_long_sequence_radix_select_path():
-    """More than 32768 keys per unit: the selection falls back to the multi-pass radix path."""
-    wl = small("long", n=8, n_kv=2, d=128, N=40000, L=32, s1=4, s2=256, k=1500, dtype="bf16", nh=0, steps=2)
+def test_long_sequence_streaming_select_path():
+    """More than 32768 keys per unit with a pooling kernel other than 1 and 7: the selection streams the keys from
+    L2 once per bisection step."""
+    wl = small("long", n=8, n_kv=2, d=128, N=40000, L=32, s1=4, s2=256, k=1500, dtype="bf16", nh=0, steps=2, pool=5)
     run_workload(wl, check_pool=False)
+
+
+CLUSTER_SELECT_CASES = [
+    # 32768 < N <= 262144: a thread-block cluster of 2, 4 or 8 CTAs keeps a unit's keys in registers
+    dict(n=8, n_kv=2, d=128, N=40000, L=32, s1=4, s2=256, k=1500, dtype="bf16", nh=0),                  # 2 CTAs
+    dict(n=2, n_kv=2, d=64, N=70001, L=32, s1=4, s2=256, k=36000, dtype="bf16", nh=0),                  # 4, k > one CTA
+    dict(n=2, n_kv=2, d=64, N=98304, L=32, s1=16, s2=300, k=700, dtype="bf16", nh=0, pool=1, t=100),    # 4, 3 of them used
+    dict(n=2, n_kv=1, d=64, N=140000, L=16, s1=4, s2=256, k=5000, dtype="bf16", nh=0),                  # 8 CTAs
+    # ragged batch: the cluster size follows the longest sequence, the short one leaves CTAs without a key
+    dict(n=4, n_kv=4, d=64, N=0, L=32, s1=4, s2=128, k=900, dtype="bf16", R=2, seq_lens=[50000, 3000, 33000], nh=1),
+    dict(n=2, n_kv=2, d=64, N=33000, L=8, s1=4, s2=64, k=200, dtype="f32", nh=1),
+]
+
+
+@pytest.mark.parametrize("case", CLUSTER_SELECT_CASES, ids=[f"case{i}" for i in range(len(CLUSTER_SELECT_CASES))])
+def test_cluster_select(case):
+    wl = small("cluster_select", **case, steps=1)
+    run_workload(wl, check_pool=False)
+
+
+def test_cluster_select_equal_scores_keep_the_lower_positions():
+    """All keys of a head equal: every score before the window is the same number (on the GPU and in the oracle
+    alike), so both selections are decided by position alone, and the run of equal keys that is kept crosses from one
+    CTA of the cluster into the next (36000 middle positions, 32768 keys per CTA)."""
+    tk = _tk()
+    N, k, s1, s2 = 70000, 36000, 4, 256
+    wl = small("equal", n=2, n_kv=2, d=64, N=N, L=32, s1=s1, s2=s2, k=k, dtype="bf16", nh=0, steps=0, promote=False)
+    qs, ks, vs = W.materialize(wl, DEV)
+    for h in range(2):
+        ks[0][0][h][:] = ks[0][0][h][0:1].clone()
+    cache = tk.taskkv_compress_ex(tk.params_from_workload(wl, max_new_tokens=0), qs, ks, vs)
+    assert cache.status() == 0
+    topt = cache.query(tk.Q_TOPT)
+    idx = cache.query(tk.Q_INDICES)
+    lens = cache.lengths()
+    want = list(range(s1 + k)) + list(range(N - s2, N))
+    for u in range(2):
+        assert topt[u].tolist() == list(range(256))
+        assert lens[u] == s1 + k + s2
+        assert idx[u, :lens[u]].tolist() == want
+    cache.close()
 
 
 def test_mistral_shaped_ragged_batch():
@@ -331,6 +373,15 @@ def test_window_scores_single_read_batch_of_ten_sequences():
     lens = [300, 9000, 1500, 4097, 129, 2048, 7000, 640, 5121, 3333]
     wl = small("ten", n=4, n_kv=4, d=128, N=0, L=32, s1=4, s2=64, k=60, dtype="bf16", seq_lens=lens, steps=1)
     run_workload(wl)
+
+
+def test_window_scores_and_selection_overlapped_by_layer_chunks():
+    """Enough units for the library to cut the layers into chunks and run the selection of one chunk beside the
+    window scores of the next (a side stream): two ragged sequences, 16 layers x 32 heads, so 4 chunks of 4 layers.
+    Layers of every chunk and both sequences are checked, the chunk borders included."""
+    wl = small("chunks", n=32, n_kv=32, d=64, N=0, L=32, s1=4, s2=64, k=90, dtype="bf16", R=16,
+               seq_lens=[1500, 2100], nh=3, steps=1)
+    run_workload(wl, layers=[(b, r) for b in range(2) for r in (0, 3, 4, 8, 11, 12, 15)])
 
 
 def test_window_scores_single_read_moderate_heavy_keys():
