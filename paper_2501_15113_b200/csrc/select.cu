@@ -558,6 +558,7 @@ constexpr int kMaxCS = 8;
 
 struct ClusterSmem {
   int cnt[2][kMaxCS][kWarps];
+  int loc[2][kWarps];        // block-local counts of the narrow phase (peers never write here)
   uint32_t mn[kMaxCS][kWarps], mx[kMaxCS][kWarps];
   int tot[2][kMaxCS][2];     // per compaction and CTA: keys above the threshold, keys equal to it
   int scan[kWarps];
@@ -583,8 +584,8 @@ __device__ __forceinline__ int cluster_count_ge(cg::cluster_group& cl, ClusterSm
   return cluster_sum(cl, cs, cs_n, rank, par, c);
 }
 
-// block_bisect over the keys of the whole cluster.  In the narrow phase every CTA collects its own surviving keys
-// (at most kNarrow in the whole cluster, so at most one per thread) and the packed counts are summed over the cluster.
+// block_bisect over the keys of the whole cluster.  For the narrow phase every CTA sends its surviving keys to all
+// CTAs (at most kNarrow in the whole cluster, so at most one per thread), and each settles the rest on its own copy.
 __device__ void cluster_bisect(cg::cluster_group& cl, ClusterSmem& cs, int cs_n, int rank, const uint32_t (&key)[kEpt],
                                int want, uint32_t* list, int cap, uint32_t& thr, int& need_eq) {
   const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
@@ -619,26 +620,41 @@ __device__ void cluster_bisect(cg::cluster_group& cl, ClusterSmem& cs, int cs_n,
   }
   if (bit >= 0) {
     const uint32_t top = t + (2u << bit);            // end of the undecided range (0 if it wraps: no upper bound)
+    const int alive = at_least - above;              // survivors in the whole cluster: at most one per thread
 #pragma unroll
     for (int e = 0; e < kEpt; ++e)
-      if (key[e] >= t && (top == 0u || key[e] < top)) list[atomicAdd(&cs.list_n, 1)] = key[e];
-    __syncthreads();
-    const int alive = cs.list_n;                     // this CTA's share of the at most kNarrow survivors
+      if (key[e] >= t && (top == 0u || key[e] < top))
+        for (int r = 0; r < cs_n; ++r)
+          cl.map_shared_rank(list, r)[atomicAdd(cl.map_shared_rank(&cs.list_n, r), 1)] = key[e];
+    cl.sync();
+    // from here on every CTA settles the remaining bits on its own copy, with block barriers only
     const uint32_t mine = (int)threadIdx.x < alive ? list[threadIdx.x] : 0u;
     const int want2 = want - above;                  // rank inside the collected keys
+    int lpar = 0;
     while (bit >= 0) {
       const uint32_t b_hi = 1u << bit, b_lo = bit > 0 ? 1u << (bit - 1) : 0u;
       const uint32_t c10 = t | b_hi, c11 = c10 | b_lo, c01 = t | b_lo;
       int v = (int)(mine >= c10) | ((int)(mine >= c11) << 10) | ((int)(b_lo != 0u && mine >= c01) << 20);
       v = __reduce_add_sync(0xffffffffu, v);
-      v = cluster_sum(cl, cs, cs_n, rank, par, v);
-      par ^= 1;
+      if (lane == 0) cs.loc[lpar][warp] = v;
+      __syncthreads();
+      v = __reduce_add_sync(0xffffffffu, cs.loc[lpar][lane]);
+      lpar ^= 1;
       const int n10 = v & 0x3ff, n11 = (v >> 10) & 0x3ff, n01 = (v >> 20) & 0x3ff;
       if (b_lo != 0u && n11 >= want2) t = c11;
       else if (n10 >= want2) t = c10;
       else if (b_lo != 0u && n01 >= want2) t = c01;
       bit -= 2;
     }
+    // keys above the threshold: those above the undecided range plus the survivors above it (no pass over all keys)
+    int g = __reduce_add_sync(0xffffffffu, (int)(mine > t));
+    if (lane == 0) cs.loc[lpar][warp] = g;
+    __syncthreads();
+    g = __reduce_add_sync(0xffffffffu, cs.loc[lpar][lane]);
+    thr = t;
+    need_eq = want - (above + g);
+    __syncthreads();
+    return;
   }
   const int n_gt = (t == 0xffffffffu) ? 0 : cluster_count_ge(cl, cs, cs_n, rank, par, key, t + 1u);
   thr = t;
