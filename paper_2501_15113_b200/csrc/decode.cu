@@ -20,6 +20,28 @@ constexpr int kAttnThreads = 128;
 constexpr int kAttnWarps = kAttnThreads / 32;
 constexpr int kUnroll = 4;
 
+// Programmatic dependent launch: a kernel launched with launch_dependent() may be set up, and its blocks may become
+// resident, while the kernel before it in the stream is still draining; grid_dependency_wait() at its start returns
+// once that kernel has completed and its writes are visible, so the stream's order of effects is unchanged.  (Without
+// the launch attribute the wait returns at once.)  This takes the launch latency out of the attention -> combine ->
+// attention chain of a layer-by-layer decode loop.
+__device__ __forceinline__ void grid_dependency_wait() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
+
+template <class... KArgs, class... Args>
+cudaError_t launch_dependent(void (*kernel)(KArgs...), unsigned grid, cudaStream_t s, Args... args) {
+  cudaLaunchConfig_t cfg = {};
+  cfg.gridDim = dim3(grid, 1, 1);
+  cfg.blockDim = dim3(kAttnThreads, 1, 1);
+  cfg.dynamicSmemBytes = 0;
+  cfg.stream = s;
+  cudaLaunchAttribute attr;
+  attr.id = cudaLaunchAttributeProgrammaticStreamSerialization;
+  attr.val.programmaticStreamSerializationAllowed = 1;
+  cfg.attrs = &attr;
+  cfg.numAttrs = 1;
+  return cudaLaunchKernelEx(&cfg, kernel, static_cast<KArgs>(args)...);
+}
+
 template <typename T, int D, int G>
 __global__ void __launch_bounds__(kAttnThreads) decode_attn_kernel(DeviceProblem p, const T* __restrict__ q,
                                                                    const int32_t* __restrict__ lengths,
@@ -36,6 +58,7 @@ __global__ void __launch_bounds__(kAttnThreads) decode_attn_kernel(DeviceProblem
   __shared__ __align__(16) float sm_acc[NSG][G][D];
   __shared__ int s_unit;
 
+  grid_dependency_wait();
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
   const int sg = lane / LPR, sl = lane % LPR;
   const int gsg = warp * RPW + sg;
@@ -244,6 +267,7 @@ __global__ void __launch_bounds__(kAttnThreads) decode_attn_mma_kernel(DevicePro
   __shared__ __align__(16) float sm_acc[kAttnWarps][G][D];
   __shared__ int s_unit;
 
+  grid_dependency_wait();
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
   const int g = lane >> 2, t = lane & 3;
   // the view's layers are a contiguous range of layer-major indices, hence of work items
@@ -426,6 +450,7 @@ __global__ void __launch_bounds__(kAttnThreads) decode_combine_kernel(DeviceProb
   __shared__ float s_max[kAttnWarps];
   __shared__ float s_l[kAttnWarps];
   __shared__ float s_acc[kAttnWarps][D];
+  grid_dependency_wait();
   const int u = blockIdx.x / G, g = blockIdx.x % G;     // u: view unit
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
   const int unit = view_unit(p, u);
@@ -483,19 +508,21 @@ cudaError_t launch_typed(const DeviceProblem& p, const void* q, const int32_t* l
   // persistent blocks: 16 per SM (measured best on B200 with 512-row items)
   int64_t grid = p.max_items < 148 * 16 ? p.max_items : 148 * 16;
   if (grid < 1) grid = 1;
+  cudaError_t e;
   {
     LaunchScope ls(K_DECODE_ATTN, s);
     if constexpr (sizeof(T) == 2)
-      decode_attn_mma_kernel<D, G><<<(unsigned)grid, kAttnThreads, 0, s>>>(p, static_cast<const T*>(q), lengths, kn, vn);
+      e = launch_dependent(decode_attn_mma_kernel<D, G>, (unsigned)grid, s, p, static_cast<const T*>(q), lengths, kn, vn);
     else
-      decode_attn_kernel<T, D, G><<<(unsigned)grid, kAttnThreads, 0, s>>>(p, static_cast<const T*>(q), lengths, kn, vn);
+      e = launch_dependent(decode_attn_kernel<T, D, G>, (unsigned)grid, s, p, static_cast<const T*>(q), lengths, kn, vn);
   }
+  if (e != cudaSuccess) return e;
   {
     LaunchScope ls(K_DECODE_COMBINE, s);
-    decode_combine_kernel<T, D, G><<<(unsigned)(p.view_U * G), kAttnThreads, 0, s>>>(p, lengths, k_new != nullptr ? 1 : 0,
-                                                                                     static_cast<T*>(out));
+    e = launch_dependent(decode_combine_kernel<T, D, G>, (unsigned)(p.view_U * G), s, p, lengths,
+                         k_new != nullptr ? 1 : 0, static_cast<T*>(out));
   }
-  return cudaGetLastError();
+  return e;
 }
 
 template <typename T, int D>
