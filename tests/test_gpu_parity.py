@@ -384,6 +384,45 @@ def test_window_scores_and_selection_overlapped_by_layer_chunks():
     run_workload(wl, layers=[(b, r) for b in range(2) for r in (0, 3, 4, 8, 11, 12, 15)])
 
 
+def test_overlapped_compression_equals_the_one_launch_order_bit_for_bit():
+    """The chunked, two-stream order of window scores and selection against the plain order (one launch each over all
+    layers, which the library takes while per-kernel timing is switched on): scores, top-t lists, semantic vectors,
+    classes, lengths, retained positions and both pools must be the same bits, three times in a row, also when the
+    caller's stream is not the default one.  A race between the two streams would show here."""
+    tk = _tk()
+    wl = small("chunks_bits", n=32, n_kv=32, d=128, N=0, L=32, s1=4, s2=64, k=150, dtype="bf16", R=8,
+               seq_lens=[2500, 1100], nh=2, steps=0)
+    qs, ks, vs = W.materialize(wl, DEV)
+    what = (tk.Q_SCORES, tk.Q_TOPT, tk.Q_SEMVEC, tk.Q_CLASSES, tk.Q_LENGTHS, tk.Q_INDICES, tk.Q_KPOOL, tk.Q_VPOOL)
+
+    def run(stream=None):
+        params = tk.params_from_workload(wl, max_new_tokens=0)
+        if stream is None:
+            cache = tk.taskkv_compress_ex(params, qs, ks, vs)
+        else:
+            with torch.cuda.stream(stream):
+                cache = tk.taskkv_compress_ex(params, qs, ks, vs)
+            stream.synchronize()
+        assert cache.status() == 0
+        got = [cache.query(w).copy() for w in what]
+        lens, idx = got[4], got[5]
+        for u in range(idx.shape[0]):
+            idx[u, min(lens[u], wl.sink + 150 + wl.recent):] = -1   # slots past sinks + middle + recent are never written
+        cache.close()
+        return got
+
+    tk.taskkv_timing_enable(True)
+    try:
+        plain = run()
+    finally:
+        tk.taskkv_timing_enable(False)
+        tk.taskkv_timing_collect()
+    side = torch.cuda.Stream()
+    for stream in (None, side, None):
+        for a, b in zip(plain, run(stream)):
+            assert np.array_equal(a, b)
+
+
 def test_window_scores_single_read_moderate_heavy_keys():
     """A few keys per head well above the rest (scores stay within fp32 range of one another): full parity."""
     wl = small("heavy", n=4, n_kv=4, d=128, N=9000, L=32, s1=4, s2=64, k=100, dtype="bf16", steps=1)
