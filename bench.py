@@ -497,11 +497,11 @@ def run_with_window_lse(tk, wl, qs, ks, vs, args, comp_bytes, peak):
 
 def ncu_traffic(wl, retained_rows):
     """DRAM bytes per decode_attn launch from the committed ncu capture (profiles/decode_attn_llama2_4layers.md):
-    382.92 MB read + written for 739,056 retained rows of 256 bytes, K and V.  Traffic grows in proportion to the
+    383.07 MB read + written for 739,056 retained rows of 256 bytes, K and V.  Traffic grows in proportion to the
     rows read, so it is scaled by rows; only the bf16, d = 128, one-query-head-per-KV-head shape was captured."""
     if wl.dtype != "bf16" or wl.head_dim != 128 or wl.n_heads != wl.n_kv_heads:
         return None
-    return 382.92e6 / 739056 * retained_rows
+    return 383.07e6 / 739056 * retained_rows
 
 
 def run_e2e(tk, wl, params, qs, ks, vs, steps_in, world):
