@@ -134,6 +134,13 @@ taskkv_status taskkv_plan(const taskkv_params* p, taskkv_plan_info* out);
  * On success *out_cache holds the compacted cache: per unit a segment of
  * retained rows in ascending position, its length, class, distance and
  * semantic vector.  Errors: EINVAL (arguments), EALLOC, ECUDA.
+ * Streams: all work is ordered after what `stream` holds at the call and is
+ * complete, for every later operation on `stream`, when the call's last kernel is.
+ * For large bf16 problems with 32 window rows the selection of one chunk of
+ * layers runs beside the window scores of the next on a stream the library
+ * owns (one per device, created by the first such call: make that call before
+ * capturing `stream` into a graph); it is forked from and joined back into
+ * `stream` with events, and calls that use it are serialised on the host.
  */
 taskkv_status taskkv_compress_ex(const taskkv_params* p, const void* const* q_win,
                                  const void* const* k, const void* const* v,
