@@ -24,6 +24,7 @@ struct HostPlan {
   int32_t chunks_max = 0, rows = 0, rows_pad = 0, idx_stride = 0;
   std::vector<int32_t> seq_lens, mid, nhet;     // [B], [R], [B*R]
   std::vector<int32_t> full;                    // [B*R] full-cache heads
+  std::vector<int64_t> layer_items;             // [R] split-K decode items of a layer over all sequences, at capacity
   // byte offsets inside the cache memory
   size_t o_unit_N, o_unit_mid, o_nhet, o_c_off, o_qp, o_kp, o_vp, meta_bytes;
   size_t o_status, o_len, o_cap, o_seg, o_cls, o_dist, o_sem, o_idx, o_goff, o_doff, o_step, o_pacc, o_pml, o_kpool,
@@ -91,6 +92,7 @@ taskkv_status make_plan(const taskkv_params* p, HostPlan& hp) {
   const int s1 = p->sink, s2 = p->recent, mn = p->max_new_tokens;
   int64_t pool = 0, kept_rows = 0, gitems = 0, ditems = 0, c_total = 0;
   int32_t stride = 1;
+  hp.layer_items.assign((size_t)R, 0);
   for (int b = 0; b < B; ++b) {
     const int64_t N = hp.seq_lens[b];
     for (int r = 0; r < R; ++r) {
@@ -101,8 +103,10 @@ taskkv_status make_plan(const taskkv_params* p, HostPlan& hp) {
       pool += h * (N + mn) + (nkv - h) * (kept + mn);
       kept_rows += h * N + (nkv - h) * kept;
       gitems += h * ((N + kGatherRows - 1) / kGatherRows) + (nkv - h) * ((kept + kGatherRows - 1) / kGatherRows);
-      ditems += h * ((N + mn + kDecodeChunk - 1) / kDecodeChunk) +
-                (nkv - h) * ((kept + mn + kDecodeChunk - 1) / kDecodeChunk);
+      const int64_t li = h * ((N + mn + kDecodeChunk - 1) / kDecodeChunk) +
+                         (nkv - h) * ((kept + mn + kDecodeChunk - 1) / kDecodeChunk);
+      ditems += li;
+      hp.layer_items[(size_t)r] += li;
       c_total += (int64_t)nkv * ((N + 3) / 4 * 4);
     }
   }
@@ -608,6 +612,10 @@ bool layer_view(const taskkv_cache* c, int32_t layer_begin, int32_t layer_count,
   out->view_l0 = layer_begin;
   out->view_nl = layer_count;
   out->view_U = c->prm.batch * layer_count * c->dp.n_kv;
+  // the attention grid is sized by the work items of the layers in view, not of the whole cache
+  int64_t items = 0;
+  for (int32_t r = layer_begin; r < layer_begin + layer_count; ++r) items += c->hp.layer_items[(size_t)r];
+  out->max_items = items;
   return true;
 }
 }  // namespace
