@@ -855,6 +855,34 @@ cudaError_t launch_cluster_k(const DeviceProblem& p, const UnitRange& ur, int cs
   return cudaLaunchKernelEx(&cfg, select_cluster_kernel<T, D, POOL_HALF>, p, ur);
 }
 
+// Whether the device can co-schedule at least one cluster of cs_n such CTAs (asked once per cluster size).
+template <typename T, int D, int POOL_HALF>
+bool cluster_fits(int cs_n) {
+  static int cached[kMaxCS + 1] = {0};      // 0 unknown, 1 yes, -1 no
+  if (cached[cs_n] == 0) {
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = dim3((unsigned)cs_n, 1, 1);
+    cfg.blockDim = dim3(kThreads, 1, 1);
+    cudaLaunchAttribute attr;
+    attr.id = cudaLaunchAttributeClusterDimension;
+    attr.val.clusterDim.x = (unsigned)cs_n;
+    attr.val.clusterDim.y = 1;
+    attr.val.clusterDim.z = 1;
+    cfg.attrs = &attr;
+    cfg.numAttrs = 1;
+    int n = 0;
+    if (cudaOccupancyMaxActiveClusters(&n, select_cluster_kernel<T, D, POOL_HALF>, &cfg) != cudaSuccess) n = 0;
+    cudaGetLastError();
+    cached[cs_n] = n > 0 ? 1 : -1;
+  }
+  return cached[cs_n] > 0;
+}
+
+template <typename T, int D>
+bool cluster_supported(const DeviceProblem& p, int cs_n) {
+  return p.pool_w == 7 ? cluster_fits<T, D, 3>(cs_n) : cluster_fits<T, D, 0>(cs_n);
+}
+
 template <typename T, int D>
 cudaError_t launch_cluster(const DeviceProblem& p, const UnitRange& ur, int cs_n, cudaStream_t s) {
   return p.pool_w == 7 ? launch_cluster_k<T, D, 3>(p, ur, cs_n, s) : launch_cluster_k<T, D, 0>(p, ur, cs_n, s);
@@ -883,10 +911,17 @@ cudaError_t launch_select(const DeviceProblem& p, int dtype, int max_N, cudaStre
   if (max_N <= kMaxCS * kThreads * kEpt && (p.pool_w == 7 || p.pool_w == 1)) {
     int cs_n = 2;
     while (cs_n * kThreads * kEpt < max_N) cs_n *= 2;
-    if (dtype == TASKKV_F32)
-      return p.d == 64 ? launch_cluster<float, 64>(p, ur, cs_n, s) : launch_cluster<float, 128>(p, ur, cs_n, s);
-    return p.d == 64 ? launch_cluster<__nv_bfloat16, 64>(p, ur, cs_n, s)
-                     : launch_cluster<__nv_bfloat16, 128>(p, ur, cs_n, s);
+    const bool fits = dtype == TASKKV_F32
+                          ? (p.d == 64 ? cluster_supported<float, 64>(p, cs_n) : cluster_supported<float, 128>(p, cs_n))
+                          : (p.d == 64 ? cluster_supported<__nv_bfloat16, 64>(p, cs_n)
+                                       : cluster_supported<__nv_bfloat16, 128>(p, cs_n));
+    if (fits) {
+      if (dtype == TASKKV_F32)
+        return p.d == 64 ? launch_cluster<float, 64>(p, ur, cs_n, s) : launch_cluster<float, 128>(p, ur, cs_n, s);
+      return p.d == 64 ? launch_cluster<__nv_bfloat16, 64>(p, ur, cs_n, s)
+                       : launch_cluster<__nv_bfloat16, 128>(p, ur, cs_n, s);
+    }
+    // a device that cannot place such a cluster streams the keys instead (below)
   }
   if (dtype == TASKKV_F32) {
     if (p.d == 64) select_kernel<float, 64><<<ur.blocks, kThreads, 0, s>>>(p, ur);
