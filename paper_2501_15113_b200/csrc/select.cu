@@ -562,7 +562,9 @@ struct ClusterSmem {
   uint32_t mn[kMaxCS][kWarps], mx[kMaxCS][kWarps];
   int tot[2][kMaxCS][2];     // per compaction and CTA: keys above the threshold, keys equal to it
   int scan[kWarps];
-  int list_n;
+  int list_n;                // survivors received from all CTAs
+  int loc_n;                 // this CTA's own survivors
+  int base[kMaxCS];          // where they go in each CTA's list
 };
 
 // Sum over the whole cluster of one int per warp (v: this warp's value, already reduced over the warp).
@@ -586,6 +588,7 @@ __device__ __forceinline__ int cluster_count_ge(cg::cluster_group& cl, ClusterSm
 
 // block_bisect over the keys of the whole cluster.  For the narrow phase every CTA sends its surviving keys to all
 // CTAs (at most kNarrow in the whole cluster, so at most one per thread), and each settles the rest on its own copy.
+// `list` must hold 2 (kNarrow + 1) words.
 __device__ void cluster_bisect(cg::cluster_group& cl, ClusterSmem& cs, int cs_n, int rank, const uint32_t (&key)[kEpt],
                                int want, uint32_t* list, int cap, uint32_t& thr, int& need_eq) {
   const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
@@ -599,7 +602,7 @@ __device__ void cluster_bisect(cg::cluster_group& cl, ClusterSmem& cs, int cs_n,
     cl.map_shared_rank(&cs.mn[rank][warp], lane)[0] = lo;
     cl.map_shared_rank(&cs.mx[rank][warp], lane)[0] = hi;
   }
-  if (threadIdx.x == 0) cs.list_n = 0;
+  if (threadIdx.x == 0) { cs.list_n = 0; cs.loc_n = 0; }
   cl.sync();
   lo = 0xffffffffu; hi = 0u;
   for (int r = 0; r < cs_n; ++r) { lo = min(lo, cs.mn[r][lane]); hi = max(hi, cs.mx[r][lane]); }
@@ -611,7 +614,7 @@ __device__ void cluster_bisect(cg::cluster_group& cl, ClusterSmem& cs, int cs_n,
   int par = 0;
   int above = 0;
   int at_least = 1 << 30;
-  const int narrow = min(cap, kNarrow);
+  const int narrow = min(cap - (kNarrow + 1), kNarrow);   // lower half of `list`: the cluster's survivors; upper half: staging
   for (; bit >= 0 && at_least - above > narrow; --bit) {
     const uint32_t cand = t | (1u << bit);
     const int c = cluster_count_ge(cl, cs, cs_n, rank, par, key, cand);
@@ -621,11 +624,20 @@ __device__ void cluster_bisect(cg::cluster_group& cl, ClusterSmem& cs, int cs_n,
   if (bit >= 0) {
     const uint32_t top = t + (2u << bit);            // end of the undecided range (0 if it wraps: no upper bound)
     const int alive = at_least - above;              // survivors in the whole cluster: at most one per thread
+    // this CTA's survivors are staged in the upper half of `list`, then copied into every CTA's lower half at an
+    // offset reserved with one remote atomic per CTA (any order: only counts matter)
+    uint32_t* stage = list + kNarrow + 1;
 #pragma unroll
     for (int e = 0; e < kEpt; ++e)
-      if (key[e] >= t && (top == 0u || key[e] < top))
-        for (int r = 0; r < cs_n; ++r)
-          cl.map_shared_rank(list, r)[atomicAdd(cl.map_shared_rank(&cs.list_n, r), 1)] = key[e];
+      if (key[e] >= t && (top == 0u || key[e] < top)) stage[atomicAdd(&cs.loc_n, 1)] = key[e];
+    __syncthreads();
+    const int n_loc = cs.loc_n;
+    if ((int)threadIdx.x < cs_n) cs.base[threadIdx.x] = atomicAdd(cl.map_shared_rank(&cs.list_n, threadIdx.x), n_loc);
+    __syncthreads();
+    for (int r = 0; r < cs_n; ++r) {
+      uint32_t* dst = cl.map_shared_rank(list, r) + cs.base[r];
+      for (int i = threadIdx.x; i < n_loc; i += kThreads) dst[i] = stage[i];
+    }
     cl.sync();
     // from here on every CTA settles the remaining bits on its own copy, with block barriers only
     const uint32_t mine = (int)threadIdx.x < alive ? list[threadIdx.x] : 0u;
