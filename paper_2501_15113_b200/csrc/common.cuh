@@ -142,6 +142,30 @@ cudaError_t launch_append(const DeviceProblem& p, int dtype, const void* k_new, 
 cudaError_t launch_decode(const DeviceProblem& p, int dtype, const void* q, const int32_t* lengths,
                           const void* k_new, const void* v_new, void* out, cudaStream_t s);
 
+// Programmatic dependent launch: a kernel launched with launch_dependent() may be set up, and its blocks may become
+// resident, while the kernel before it in the stream is still draining; grid_dependency_wait() at its start returns
+// once that kernel has completed and its writes are visible, so the stream's order of effects is unchanged.  (Without
+// the launch attribute the wait returns at once.)  This takes the launch latency out of chains of short dependent
+// kernels: attention -> combine -> attention of a layer-by-layer decode loop, separator -> plan -> gather.
+#ifdef __CUDACC__
+__device__ __forceinline__ void grid_dependency_wait() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
+
+template <class... KArgs, class... Args>
+cudaError_t launch_dependent(void (*kernel)(KArgs...), unsigned grid, unsigned block, cudaStream_t s, Args... args) {
+  cudaLaunchConfig_t cfg = {};
+  cfg.gridDim = dim3(grid, 1, 1);
+  cfg.blockDim = dim3(block, 1, 1);
+  cfg.dynamicSmemBytes = 0;
+  cfg.stream = s;
+  cudaLaunchAttribute attr;
+  attr.id = cudaLaunchAttributeProgrammaticStreamSerialization;
+  attr.val.programmaticStreamSerializationAllowed = 1;
+  cfg.attrs = &attr;
+  cfg.numAttrs = 1;
+  return cudaLaunchKernelEx(&cfg, kernel, static_cast<KArgs>(args)...);
+}
+#endif
+
 // ---------------------------------------------------------------- device helpers
 #ifdef __CUDACC__
 

@@ -20,28 +20,6 @@ constexpr int kAttnThreads = 128;
 constexpr int kAttnWarps = kAttnThreads / 32;
 constexpr int kUnroll = 4;
 
-// Programmatic dependent launch: a kernel launched with launch_dependent() may be set up, and its blocks may become
-// resident, while the kernel before it in the stream is still draining; grid_dependency_wait() at its start returns
-// once that kernel has completed and its writes are visible, so the stream's order of effects is unchanged.  (Without
-// the launch attribute the wait returns at once.)  This takes the launch latency out of the attention -> combine ->
-// attention chain of a layer-by-layer decode loop.
-__device__ __forceinline__ void grid_dependency_wait() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
-
-template <class... KArgs, class... Args>
-cudaError_t launch_dependent(void (*kernel)(KArgs...), unsigned grid, cudaStream_t s, Args... args) {
-  cudaLaunchConfig_t cfg = {};
-  cfg.gridDim = dim3(grid, 1, 1);
-  cfg.blockDim = dim3(kAttnThreads, 1, 1);
-  cfg.dynamicSmemBytes = 0;
-  cfg.stream = s;
-  cudaLaunchAttribute attr;
-  attr.id = cudaLaunchAttributeProgrammaticStreamSerialization;
-  attr.val.programmaticStreamSerializationAllowed = 1;
-  cfg.attrs = &attr;
-  cfg.numAttrs = 1;
-  return cudaLaunchKernelEx(&cfg, kernel, static_cast<KArgs>(args)...);
-}
-
 template <typename T, int D, int G>
 __global__ void __launch_bounds__(kAttnThreads) decode_attn_kernel(DeviceProblem p, const T* __restrict__ q,
                                                                    const int32_t* __restrict__ lengths,
@@ -512,14 +490,14 @@ cudaError_t launch_typed(const DeviceProblem& p, const void* q, const int32_t* l
   {
     LaunchScope ls(K_DECODE_ATTN, s);
     if constexpr (sizeof(T) == 2)
-      e = launch_dependent(decode_attn_mma_kernel<D, G>, (unsigned)grid, s, p, static_cast<const T*>(q), lengths, kn, vn);
+      e = launch_dependent(decode_attn_mma_kernel<D, G>, (unsigned)grid, kAttnThreads, s, p, static_cast<const T*>(q), lengths, kn, vn);
     else
-      e = launch_dependent(decode_attn_kernel<T, D, G>, (unsigned)grid, s, p, static_cast<const T*>(q), lengths, kn, vn);
+      e = launch_dependent(decode_attn_kernel<T, D, G>, (unsigned)grid, kAttnThreads, s, p, static_cast<const T*>(q), lengths, kn, vn);
   }
   if (e != cudaSuccess) return e;
   {
     LaunchScope ls(K_DECODE_COMBINE, s);
-    e = launch_dependent(decode_combine_kernel<T, D, G>, (unsigned)(p.view_U * G), s, p, lengths,
+    e = launch_dependent(decode_combine_kernel<T, D, G>, (unsigned)(p.view_U * G), kAttnThreads, s, p, lengths,
                          k_new != nullptr ? 1 : 0, static_cast<T*>(out));
   }
   return e;

@@ -17,6 +17,7 @@ __global__ void __launch_bounds__(kGatherThreads) gather_kernel(DeviceProblem p)
   constexpr int RPP = kGatherThreads / VPR;           // rows per pass
   constexpr int PASSES = kGatherRows / RPP;
   __shared__ int s_unit;
+  grid_dependency_wait();
   const int item = blockIdx.x;
   if (threadIdx.x == 0) s_unit = (item < p.gather_off[p.U]) ? upper_unit(p.gather_off, p.U, item) : -1;
   __syncthreads();
@@ -157,12 +158,11 @@ cudaError_t launch_gather(const DeviceProblem& p, int dtype, int64_t gather_item
   const int row_bytes = p.d * (dtype == TASKKV_F32 ? 4 : 2);
   const unsigned grid = (unsigned)gather_items;
   switch (row_bytes) {
-    case 128: gather_kernel<128><<<grid, kGatherThreads, 0, s>>>(p); break;
-    case 256: gather_kernel<256><<<grid, kGatherThreads, 0, s>>>(p); break;
-    case 512: gather_kernel<512><<<grid, kGatherThreads, 0, s>>>(p); break;
+    case 128: return launch_dependent(gather_kernel<128>, grid, (unsigned)kGatherThreads, s, p);
+    case 256: return launch_dependent(gather_kernel<256>, grid, (unsigned)kGatherThreads, s, p);
+    case 512: return launch_dependent(gather_kernel<512>, grid, (unsigned)kGatherThreads, s, p);
     default: return cudaErrorInvalidValue;
   }
-  return cudaGetLastError();
 }
 
 cudaError_t launch_append(const DeviceProblem& p, int dtype, const void* k_new, const void* v_new,

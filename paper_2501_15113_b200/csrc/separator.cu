@@ -14,6 +14,7 @@ namespace taskkv {
 namespace {
 
 __global__ void __launch_bounds__(128) separator_kernel(DeviceProblem p) {
+  grid_dependency_wait();
   __shared__ double center[128];
   __shared__ double dist[TASKKV_MAX_KV_HEADS];
   __shared__ int cls[TASKKV_MAX_KV_HEADS];
@@ -97,6 +98,7 @@ __device__ int64_t block_excl_scan(int64_t v, int64_t* warp_tot, int64_t* total)
 }
 
 __global__ void __launch_bounds__(kPlanThreads) plan_kernel(DeviceProblem p) {
+  grid_dependency_wait();
   __shared__ int64_t warp_tot[32];
   __shared__ int64_t total;
   int64_t run_rows = 0, run_gather = 0;
@@ -148,15 +150,17 @@ __global__ void __launch_bounds__(kPlanThreads) plan_kernel(DeviceProblem p) {
 }  // namespace
 
 cudaError_t launch_separator_plan(const DeviceProblem& p, int n_br, cudaStream_t s) {
+  cudaError_t e;
   {
     LaunchScope ls(K_SEPARATOR, s);
-    separator_kernel<<<n_br, 128, 0, s>>>(p);
+    e = launch_dependent(separator_kernel, (unsigned)n_br, 128u, s, p);
   }
+  if (e != cudaSuccess) return e;
   {
     LaunchScope ls(K_PLAN, s);
-    plan_kernel<<<1, kPlanThreads, 0, s>>>(p);
+    e = launch_dependent(plan_kernel, 1u, (unsigned)kPlanThreads, s, p);
   }
-  return cudaGetLastError();
+  return e;
 }
 
 }  // namespace taskkv
