@@ -3,12 +3,20 @@ seeded inputs as the CUDA library and compares stage by stage.
 
 Index rule: retained positions must be identical, except at a selection
 boundary where the oracle's own scores are tied to within 1e-5 relative (the
-GPU ranks fp32 scores, the oracle fp64 ones); such differences are counted and
-returned so that tests can report and bound them.
+GPU ranks fp32 scores, the oracle fp64 ones); such differences are counted,
+bounded (Report.check_bounds) and, when the environment variable
+TASKKV_PARITY_REPORT names a file, appended to it as one JSON line per test.
+Head classes must be identical; the one exception is a layer whose deciding
+distance gap (the f-th against the (f+1)-th farthest head, or the nearest
+against the second-nearest of the rest) is below CLASS_TIE_REL in the oracle,
+which is counted per (sequence, layer) and must be named by the test that
+expects it.
 """
 from __future__ import annotations
 
 import dataclasses
+import json
+import os
 from typing import Dict, List
 
 import numpy as np
@@ -19,6 +27,9 @@ from paper_2501_15113_b200 import binding as tk
 from paper_2501_15113_b200 import workloads as W
 
 TIE_REL = 1e-5
+# distances are sums of fp32 scores (2e-5) times stored values, accumulated in fp32: two oracle distances closer than
+# this cannot be ranked by the fp32 path, and only the gap that decides a class may be that close
+CLASS_TIE_REL = 1e-4
 TOL_OUT = {"f32": 1e-5, "bf16": 2e-2}
 # C is computed in fp32 from exact products: fp32 accumulation over d <= 128 terms, one ex2 on an fp32 argument and
 # tree-summed row normalisers keep the result within this bound of the fp64 oracle (measured 2e-7 .. 8e-6)
@@ -31,10 +42,39 @@ class Report:
     topt_ties: int = 0
     mid_ties: int = 0
     class_near_ties: int = 0
+    selected: int = 0                # positions chosen by the selections that were compared (top-t + middle)
+    class_diff: Dict = dataclasses.field(default_factory=dict)     # (b, r) -> KV heads of a counted class near-tie
     max_score_rel: float = 0.0
     max_sem_rel: float = 0.0
     max_out_abs: float = 0.0
-    notes: List[str] = dataclasses.field(default_factory=list)
+
+    def tie_bound(self) -> int:
+        """At most one boundary tie per 10,000 selected positions, and one for any sample smaller than that."""
+        return 1 + self.selected // 10000
+
+    def summary(self) -> str:
+        return (f"units={self.units} selected={self.selected} topt_ties={self.topt_ties} mid_ties={self.mid_ties} "
+                f"class_near_ties={self.class_near_ties} {self.class_diff if self.class_diff else ''} "
+                f"max_score_rel={self.max_score_rel:.2e} max_sem_rel={self.max_sem_rel:.2e} "
+                f"max_out_abs={self.max_out_abs:.2e}")
+
+    def check_bounds(self, name: str, expect_class_ties=()) -> None:
+        """Every caller ends here: class near-ties only at the (b, r) the test names, boundary ties within the bound."""
+        assert sorted(self.class_diff) == sorted(expect_class_ties), f"[{name}] unexpected class near-ties: {self.summary()}"
+        assert self.topt_ties + self.mid_ties <= self.tie_bound(), \
+            f"[{name}] more boundary ties than {self.tie_bound()}: {self.summary()}"
+
+
+def write_report(name: str, rep: "Report") -> None:
+    path = os.environ.get("TASKKV_PARITY_REPORT")
+    if not path:
+        return
+    rec = {"test": name, "units": rep.units, "selected": rep.selected, "topt_ties": rep.topt_ties,
+           "mid_ties": rep.mid_ties, "tie_bound": rep.tie_bound(), "class_near_ties": rep.class_near_ties,
+           "class_diff": {f"{b},{r}": h for (b, r), h in rep.class_diff.items()},
+           "max_score_rel": rep.max_score_rel, "max_sem_rel": rep.max_sem_rel, "max_out_abs": rep.max_out_abs}
+    with open(path, "a") as fh:
+        fh.write(json.dumps(rec) + "\n")
 
 
 def to64(t: torch.Tensor) -> np.ndarray:
@@ -76,9 +116,44 @@ def score_offsets(wl: W.Workload) -> np.ndarray:
     return np.array(off, dtype=np.int64)
 
 
+def classes_valid_up_to(dist: np.ndarray, got_cls: np.ndarray, f: int, promote: bool, tol: float) -> bool:
+    """Sec. IV-A on the oracle's distances: is `got_cls` a correct answer if distances closer than `tol` relative
+    cannot be told apart?  Only the two deciding gaps count: every head marked heterogeneous must be at least as far
+    as every head left out (the f-th against the (f+1)-th distance), and the promoted head must be the nearest of the
+    rest (smallest against second-smallest remaining distance)."""
+    n = dist.shape[0]
+    f = max(0, min(int(f), n))
+    far = np.flatnonzero(got_cls == O.CLASS_HETERO)
+    rest = np.flatnonzero(got_cls != O.CLASS_HETERO)
+    if len(far) != f:
+        return False
+    if len(far) and len(rest) and dist[far].min() < dist[rest].max() * (1.0 - tol):
+        return False
+    centre = np.flatnonzero(got_cls == O.CLASS_CENTER)
+    if not (promote and f < n):
+        return len(centre) == 0
+    return len(centre) == 1 and dist[centre[0]] <= dist[rest].min() * (1.0 + tol)
+
+
+@dataclasses.dataclass
+class LayerCheck:
+    """What compare_layer found for one (sequence, layer)."""
+    skip_heads: set          # KV heads whose class legitimately differs from the oracle's (a counted near-tie)
+    idx: List[np.ndarray]    # per KV head: the retained positions to decode over (the oracle's, or the library's
+    #                          where it differs from them only by counted boundary ties)
+
+
 def compare_layer(cache: tk.Cache, wl: W.Workload, b: int, r: int, ref: Dict, rep: Report,
-                  scores: np.ndarray = None, topt: np.ndarray = None) -> None:
-    """Stage-by-stage comparison of one (sequence, layer) against the oracle result `ref`."""
+                  scores: np.ndarray = None, topt: np.ndarray = None, v=None, force_class: int = -1) -> LayerCheck:
+    """Stage-by-stage comparison of one (sequence, layer) against the oracle result `ref`.
+
+    Index rule: a selection may differ from the oracle's only by swaps among positions whose oracle scores are within
+    TIE_REL of the selection boundary; such swaps are counted.  A counted top-t swap changes which V rows enter
+    Eq. 15, so when one occurred (and `v`, the layer's values, is given) the oracle's semantic vectors, distances
+    and classes are recomputed from the oracle's own scores with the library's validated top-t lists, and the
+    comparison continues against those.  Classes must then be equal, except where the distance gap that decides
+    the difference is below CLASS_TIE_REL; those layers are counted in rep.class_near_ties, listed in
+    rep.class_diff, and only the heads concerned are left out of the later stages."""
     N = wl.seq_lens[b]
     nkv = wl.n_kv_heads
     lens = cache.lengths()
@@ -88,6 +163,8 @@ def compare_layer(cache: tk.Cache, wl: W.Workload, b: int, r: int, ref: Dict, re
     idx_tab = cache.query(tk.Q_INDICES)
     coff = score_offsets(wl)
     u0 = unit_index(wl, b, r, 0)
+    want_sem = np.array(ref["sem"], dtype=np.float64)
+    unresolved = set()              # heads whose semantic vector cannot be compared (tie swap and no V given)
     flips_in_layer = 0
     for h in range(nkv):
         u = u0 + h
@@ -100,7 +177,6 @@ def compare_layer(cache: tk.Cache, wl: W.Workload, b: int, r: int, ref: Dict, re
             assert rel.max() < TOL_SCORE_REL, f"unit {u}: scores off by {rel.max():.3e} relative"
             assert abs(c_gpu.sum() - 1.0) < 1e-4
         # Eq. 14: top-t set
-        flips = 0
         if topt is not None:
             got = topt[u]
             got = got[got >= 0]
@@ -108,31 +184,52 @@ def compare_layer(cache: tk.Cache, wl: W.Workload, b: int, r: int, ref: Dict, re
             assert np.all(np.diff(got) > 0), f"unit {u}: top-t list not ascending"
             rep.topt_ties += flips
             flips_in_layer += flips
-        # Eq. 15: semantic vector (comparable only when the same positions were summed)
-        if flips == 0:
-            scale = max(np.abs(ref["sem"][h]).max(), 1e-30)
-            rel = float(np.abs(sem[u].astype(np.float64) - ref["sem"][h]).max() / scale)
-            rep.max_sem_rel = max(rep.max_sem_rel, rel)
-            assert rel < 1e-4, f"unit {u}: semantic vector off by {rel:.3e} of its largest component"
+            if flips:
+                if v is not None:
+                    want_sem[h] = O.semantic_vector(ref["C"][h], to64(v[h]), got.astype(np.int64))
+                else:
+                    unresolved.add(h)
+    rep.selected += nkv * min(wl.top_t, N)
+    # Eq. 15: semantic vectors (after a counted tie swap: the oracle's sum over the library's validated positions)
+    for h in range(nkv):
+        if h in unresolved:
+            continue
+        scale = max(np.abs(want_sem[h]).max(), 1e-30)
+        rel = float(np.abs(sem[u0 + h].astype(np.float64) - want_sem[h]).max() / scale)
+        rep.max_sem_rel = max(rep.max_sem_rel, rel)
+        assert rel < 1e-4, f"unit {u0 + h}: semantic vector off by {rel:.3e} of its largest component"
     # Eq. 7-8 / Sec. IV-A: distances and classes
-    ref_cls = ref["cls"]
+    f = wl.n_hetero[b][r]
+    if flips_in_layer and not unresolved:
+        want_dist = O.center_distances(want_sem)
+        if force_class == -1:
+            want_cls = O.semantic_separator(want_dist, f, wl.promote_center)
+        else:
+            want_cls = ref["cls"]
+    else:
+        want_dist, want_cls = ref["dist"], ref["cls"]
+    if not unresolved:
+        np.testing.assert_allclose(dist[u0:u0 + nkv], want_dist, rtol=1e-4, atol=1e-30)
     got_cls = cls[u0:u0 + nkv]
-    if flips_in_layer == 0:
-        np.testing.assert_allclose(dist[u0:u0 + nkv], ref["dist"], rtol=1e-4, atol=1e-30)
-    if got_cls.tolist() != ref_cls.tolist():
-        # legitimate only if the oracle's own ranking margin is below what the fp32 scores can resolve
-        d = np.sort(ref["dist"])
-        gaps = np.diff(d) / d[1:]
-        assert flips_in_layer > 0 or gaps.min() < 1e-4, \
-            f"(b={b}, r={r}): classes {got_cls.tolist()} differ from the oracle's {ref_cls.tolist()}"
+    skip = set()
+    if got_cls.tolist() != want_cls.tolist():
+        ok = force_class == -1 and not unresolved and \
+            classes_valid_up_to(want_dist, got_cls, f, wl.promote_center, CLASS_TIE_REL)
+        assert ok, (f"(b={b}, r={r}): classes {got_cls.tolist()} differ from the oracle's {want_cls.tolist()} and the "
+                    f"deciding distance gap is not below {CLASS_TIE_REL} (distances {want_dist.tolist()})")
+        skip = {h for h in range(nkv) if int(got_cls[h]) != int(want_cls[h])}
         rep.class_near_ties += 1
-        rep.notes.append(f"class near-tie at b={b} r={r}")
-        return
+        rep.class_diff[(b, r)] = sorted(skip)
     # Sec. IV-B: lengths and retained positions
-    assert lens[u0:u0 + nkv].tolist() == ref["len"].tolist(), f"(b={b}, r={r}): lengths differ"
+    out_idx = []
     for h in range(nkv):
         u = u0 + h
-        want = ref["idx"][h]
+        want = ref["idx"][h] if int(want_cls[h]) == int(ref["cls"][h]) else \
+            O.retained_indices(int(want_cls[h]), ref["C"][h], wl.sink, wl.recent, wl.mid_budget[r], wl.pool_kernel)
+        out_idx.append(want)
+        if h in skip:
+            continue
+        assert int(lens[u]) == len(want), f"(b={b}, r={r}) head {h}: length {int(lens[u])}, oracle keeps {len(want)}"
         if len(want) == N:
             continue
         got = idx_tab[u, :lens[u]].astype(np.int64)
@@ -140,7 +237,12 @@ def compare_layer(cache: tk.Cache, wl: W.Workload, b: int, r: int, ref: Dict, re
         s1, s2 = wl.sink, wl.recent
         assert got[:s1].tolist() == list(range(s1)) and got[len(got) - s2:].tolist() == list(range(N - s2, N))
         pooled = O.average_pool(ref["C"][h], wl.pool_kernel)
-        rep.mid_ties += check_selection(got[s1:len(got) - s2], want[s1:len(want) - s2], pooled, f"unit {u} middle")
+        ties = check_selection(got[s1:len(got) - s2], want[s1:len(want) - s2], pooled, f"unit {u} middle")
+        rep.mid_ties += ties
+        rep.selected += len(got) - s1 - s2
+        if ties:
+            out_idx[h] = got            # equal to the oracle's list up to the counted boundary ties
+    return LayerCheck(skip_heads=skip, idx=out_idx)
 
 
 def compare_pool_rows(cache: tk.Cache, wl: W.Workload, b: int, r: int, k, v) -> None:
