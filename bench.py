@@ -11,7 +11,12 @@ Prints ONE JSON line.  `value` is decode attention steps per second (all layers
 per step), measured on the device with inputs resident in HBM; compression
 tokens per second is reported beside it, and `e2e` repeats the measurement
 through the host-buffer entry points with the copies inside the timed region.
-`--impl reference` times the CPU oracle on a bounded sample instead.
+On one GPU the line also carries, under `workloads`, the same device-timed
+measurement of the other single-GPU workloads: the Llama-3-8B-shaped
+grouped-query stack, the Mistral-7B-shaped ragged batch and the 15 points of
+the budget sweep (`--no-extra` skips them).
+`--impl reference` times the CPU oracle on a bounded sample instead; that arm
+never builds or loads the CUDA library.
 """
 from __future__ import annotations
 
@@ -43,14 +48,15 @@ def load_peaks():
         return FALLBACK_HBM_GBS, "fallback"
 
 
-def get_workload(name: str, args):
+def get_workload(name: str, args, helpers=None):
+    """helpers: (hetero_count, mid_budget) for Eq. 16 / Eq. 17; None takes the library's own host helpers."""
     from paper_2501_15113_b200 import configs
     if name == "llama2":
         return configs.config2_llama2(seq_len=args.seq_len or 32768, n_layers=args.layers or 32,
                                       decode_steps=args.decode_steps or 256)
     if name == "llama3":
         return configs.config3_llama3(seq_len=args.seq_len or 131072, n_layers=args.layers or 32,
-                                      decode_steps=args.decode_steps or 128)
+                                      decode_steps=args.decode_steps or 128, helpers=helpers)
     if name == "mistral":
         return configs.config4_mistral(n_layers=args.layers or 32, decode_steps=args.decode_steps or 512)
     if name == "toy":
@@ -127,6 +133,162 @@ def algorithmic_bytes(wl, info, policy="select"):
     return comp
 
 
+def measure_workload(tk, W, wl, dev, steps, warmup, policy, peak, peak_kind, sampler_gpu, world=1):
+    """Device-timed measurement of one workload: `warmup` untimed and `steps` timed passes (compress every layer, then
+    the workload's decode steps as fused append + attention calls), then one more pass with every kernel launch
+    bracketed by events.  Returns (result dict, live objects the caller may keep using)."""
+    from paper_2501_15113_b200 import sharding
+    S = wl.decode_steps
+    qs, ks, vs = W.materialize(wl, dev)
+    steps_in = [W.gen_decode_step(wl, s, dev) for s in range(S)]
+    params = tk.params_from_workload(wl, max_new_tokens=S, mid_policy=POLICIES[policy])
+    info = tk.taskkv_plan(params)
+    cache_mem = torch.empty(int(info.cache_bytes), dtype=torch.uint8, device=dev)
+    work_mem = torch.empty(int(info.workspace_bytes), dtype=torch.uint8, device=dev)
+    out = torch.empty_like(steps_in[0][0])
+    stream = torch.cuda.current_stream()
+
+    def one_pass(ev=None):
+        if ev:
+            ev[0].record(stream)
+        cache = tk.taskkv_compress_ex(params, qs, ks, vs, cache_mem=cache_mem, workspace_mem=work_mem)
+        if ev:
+            ev[1].record(stream)
+        for (q, kn, vn) in steps_in:
+            cache.taskkv_decode_step(q, kn, vn, out=out)        # append + attention, fused
+        if ev:
+            ev[2].record(stream)
+        return cache
+
+    for _ in range(warmup):
+        one_pass().close()
+    torch.cuda.synchronize()
+
+    def barrier():
+        if world > 1:
+            import torch.distributed as dist
+            dist.barrier()
+        torch.cuda.synchronize()
+
+    sampler = ClockSampler(sampler_gpu)
+    launches0 = tk.taskkv_launch_count()
+    evs = [[torch.cuda.Event(enable_timing=True) for _ in range(3)] for _ in range(steps)]
+    barrier()
+    sampler.start()
+    t0 = torch.cuda.Event(enable_timing=True)
+    t1 = torch.cuda.Event(enable_timing=True)
+    t0.record(stream)
+    caches = []
+    for i in range(steps):
+        caches.append(one_pass(evs[i]))
+    t1.record(stream)
+    barrier()
+    clocks = sampler.stop()
+    launches = tk.taskkv_launch_count() - launches0
+    status = caches[-1].status()
+    for c in caches:
+        c.close()
+    total_ms = t0.elapsed_time(t1)
+    comp_each = [e[0].elapsed_time(e[1]) for e in evs]
+    dec_each = [e[1].elapsed_time(e[2]) / S for e in evs]       # per decode step, one value per timed pass
+    comp_ms = sum(comp_each)
+    dec_ms = sum(e[1].elapsed_time(e[2]) for e in evs)
+    K = steps
+    # whole-job rates: units of all ranks over the slowest rank's time (one small all-reduce when N > 1)
+    value, dec_ms = sharding.job_throughput(K * S, dec_ms, device=dev)
+    comp_tps, comp_ms = sharding.job_throughput(K * sum(wl.seq_lens), comp_ms, device=dev)
+    _, total_ms = sharding.job_throughput(K, total_ms, device=dev)
+
+    # per-kernel durations: one more identical pass with every launch bracketed by events on its stream
+    tk.taskkv_timing_enable(True)
+    one_pass().close()
+    recs = tk.taskkv_timing_collect()
+    tk.taskkv_timing_enable(False)
+    per = {}
+    for name, ms in recs:
+        a = per.setdefault(name, [0, 0.0])
+        a[0] += 1
+        a[1] += ms
+
+    es, d = wl.elem_size, wl.head_dim
+    comp_bytes = algorithmic_bytes(wl, info, policy)
+    U = int(info.n_units)
+    # decode step s (1-based) reads K and V rows of every segment once: retained rows + s appended per unit
+    dec_bytes_avg = 2 * d * es * (int(info.retained_rows) + U * (S + 1) / 2.0)
+    dec_step_ms = dec_ms / (K * S)
+    comp_pass_ms = comp_ms / K
+
+    kern = {}
+    for name, (n, ms) in per.items():
+        kern[name] = {"launches": n, "avg_ms": ms / n, "total_ms": ms}
+    attn = kern.get("decode_attn", {"avg_ms": float("nan")})
+    attn_gbs = dec_bytes_avg / (attn["avg_ms"] * 1e-3) / 1e9
+    comp_kernel_ms = sum(v["total_ms"] for k, v in kern.items() if not k.startswith(("decode", "append")))
+    dec_gbs = dec_bytes_avg / (dec_step_ms * 1e-3) / 1e9
+    comp_gbs = comp_bytes / (comp_pass_ms * 1e-3) / 1e9
+    traffic, traffic_src = ncu_traffic(wl, int(info.retained_rows))
+    res = {
+        "value": value, "ms_per_step": total_ms / K,
+        "decode_ms_per_step": dec_step_ms, "compress_ms": comp_pass_ms, "compress_tokens_per_s": comp_tps,
+        "per_pass": {"compress_ms_median": statistics.median(comp_each), "compress_ms_min": min(comp_each),
+                     "decode_ms_per_step_median": statistics.median(dec_each),
+                     "decode_ms_per_step_min": min(dec_each), "passes": len(evs)},
+        "hbm": {
+            "peak_gbs": peak, "peak_kind": peak_kind, "nominal_gbs": NOMINAL_HBM_GBS,
+            "decode_gbs": dec_gbs, "decode_frac": dec_gbs / peak, "decode_frac_of_nominal": dec_gbs / NOMINAL_HBM_GBS,
+            "compress_gbs": comp_gbs, "compress_frac": comp_gbs / peak,
+            "compress_frac_of_nominal": comp_gbs / NOMINAL_HBM_GBS,
+            "decode_bytes_per_step": dec_bytes_avg, "compress_bytes": comp_bytes,
+        },
+        "roofline": {"bound": "hbm", "kernel": "decode_attn", "achieved": attn_gbs, "peak": peak, "unit": "GB/s",
+                     "frac": attn_gbs / peak, "frac_of_nominal": attn_gbs / NOMINAL_HBM_GBS, "peak_kind": peak_kind,
+                     "traffic": traffic, "traffic_unit": "bytes per launch", "traffic_source": traffic_src,
+                     "algorithmic_bytes": dec_bytes_avg, "avg_launch_ms": attn["avg_ms"]},
+        "kernels": kern, "compress_kernel_ms": comp_kernel_ms,
+        "gpu_launches": launches, "device_status": status, "clocks": clocks,
+    }
+    live = {"qs": qs, "ks": ks, "vs": vs, "steps_in": steps_in, "params": params, "comp_bytes": comp_bytes}
+    return res, live
+
+
+EXTRA_WORKLOADS = ["llama3", "mistral"] + [f"sweep:{h}:{k}" for h in (0, 1, 2, 4, 8) for k in (64, 256, 1024)]
+
+
+def run_extra_workloads(tk, W, args, dev, peak, peak_kind, gpu):
+    """The other single-GPU workloads, each measured like the headline one (3 warm-up and 3 timed passes, per-kernel
+    pass, clocks sampled): the grouped-query stack, the ragged serving batch, and the 15 budget-sweep points."""
+    out = {}
+    for name in EXTRA_WORKLOADS:
+        if name == args.workload:
+            continue
+        wl = get_workload(name, args)
+        wl.planted = W._choose_planted(wl)
+        try:
+            res, live = measure_workload(tk, W, wl, dev, steps=3, warmup=3, policy=args.policy, peak=peak,
+                                         peak_kind=peak_kind, sampler_gpu=gpu)
+        except Exception as exc:            # one workload failing must not lose the headline line
+            out[name] = {"workload": wl.name, "error": f"{type(exc).__name__}: {str(exc)[:200]}"}
+            torch.cuda.empty_cache()
+            continue
+        del live
+        torch.cuda.empty_cache()
+        k = res["kernels"]
+        out[name] = {
+            "workload": wl.name, "decode_steps": wl.decode_steps, "passes": 3,
+            "compress_ms": res["compress_ms"], "compress_tokens_per_s": res["compress_tokens_per_s"],
+            "decode_ms_per_step": res["decode_ms_per_step"], "decode_steps_per_s": res["value"],
+            "hbm": {x: res["hbm"][x] for x in ("compress_frac", "decode_frac", "compress_frac_of_nominal",
+                                               "decode_frac_of_nominal", "compress_gbs", "decode_gbs",
+                                               "compress_bytes", "decode_bytes_per_step")},
+            "decode_attn": {x: res["roofline"][x] for x in ("achieved", "frac", "traffic", "avg_launch_ms")},
+            "kernel_ms": {n: round(v["total_ms"], 4) for n, v in k.items() if not n.startswith(("decode", "append"))},
+            "kernel_ms_per_decode_launch": {n: round(v["avg_ms"], 4) for n, v in k.items()
+                                            if n.startswith(("decode", "append"))},
+            "gpu_launches": res["gpu_launches"], "device_status": res["device_status"], "clocks": res["clocks"],
+        }
+    return out
+
+
 def run_ours(args):
     import __graft_entry__ as ge
     ge.build()
@@ -147,120 +309,20 @@ def run_ours(args):
     from paper_2501_15113_b200 import sharding
     wl.seed = sharding.replica_seed(wl.seed, rank)   # weak scaling: every rank owns an independent replica
     wl.planted = W._choose_planted(wl)
-    S = wl.decode_steps
-    qs, ks, vs = W.materialize(wl, dev)
-    steps_in = [W.gen_decode_step(wl, s, dev) for s in range(S)]
-    params = tk.params_from_workload(wl, max_new_tokens=S, mid_policy=POLICIES[args.policy])
-    info = tk.taskkv_plan(params)
-    cache_mem = torch.empty(int(info.cache_bytes), dtype=torch.uint8, device=dev)
-    work_mem = torch.empty(int(info.workspace_bytes), dtype=torch.uint8, device=dev)
-    out = torch.empty_like(steps_in[0][0])
-    stream = torch.cuda.current_stream()
-
-    def one_pass(ev=None):
-        if ev:
-            ev[0].record(stream)
-        cache = tk.taskkv_compress_ex(params, qs, ks, vs, cache_mem=cache_mem, workspace_mem=work_mem)
-        if ev:
-            ev[1].record(stream)
-        for (q, kn, vn) in steps_in:
-            cache.taskkv_decode_step(q, kn, vn, out=out)        # append + attention, fused
-        if ev:
-            ev[2].record(stream)
-        return cache
-
-    for _ in range(args.warmup):
-        one_pass().close()
-    torch.cuda.synchronize()
-
-    def barrier():
-        if world > 1:
-            import torch.distributed as dist
-            dist.barrier()
-        torch.cuda.synchronize()
-
-    sampler = ClockSampler(local)
-    launches0 = tk.taskkv_launch_count()
-    evs = [[torch.cuda.Event(enable_timing=True) for _ in range(3)] for _ in range(args.steps)]
-    barrier()
-    sampler.start()
-    t0 = torch.cuda.Event(enable_timing=True)
-    t1 = torch.cuda.Event(enable_timing=True)
-    t0.record(stream)
-    caches = []
-    for i in range(args.steps):
-        caches.append(one_pass(evs[i]))
-    t1.record(stream)
-    barrier()
-    clocks = sampler.stop()
-    launches = tk.taskkv_launch_count() - launches0
-    status = caches[-1].status()
-    for c in caches:
-        c.close()
-    total_ms = t0.elapsed_time(t1)
-    comp_each = [e[0].elapsed_time(e[1]) for e in evs]
-    dec_each = [e[1].elapsed_time(e[2]) / S for e in evs]       # per decode step, one value per timed pass
-    comp_ms = sum(comp_each)
-    dec_ms = sum(e[1].elapsed_time(e[2]) for e in evs)
-    K = args.steps
-    # whole-job rates: units of all ranks over the slowest rank's time (one small all-reduce when N > 1)
-    value, dec_ms = sharding.job_throughput(K * S, dec_ms, device=dev)
-    comp_tps, comp_ms = sharding.job_throughput(K * sum(wl.seq_lens), comp_ms, device=dev)
-    _, total_ms = sharding.job_throughput(K, total_ms, device=dev)
-
-    # per-kernel durations: one more identical pass with every launch bracketed by events on its stream
-    tk.taskkv_timing_enable(True)
-    one_pass().close()
-    recs = tk.taskkv_timing_collect()
-    tk.taskkv_timing_enable(False)
-    per = {}
-    for name, ms in recs:
-        a = per.setdefault(name, [0, 0.0])
-        a[0] += 1
-        a[1] += ms
-
-    tokens = sum(wl.seq_lens)
-    es, d = wl.elem_size, wl.head_dim
-    comp_bytes = algorithmic_bytes(wl, info, args.policy)
-    U = int(info.n_units)
-    # decode step s (1-based) reads K and V rows of every segment once: retained rows + s appended per unit
-    dec_bytes_avg = 2 * d * es * (int(info.retained_rows) + U * (S + 1) / 2.0)
-    dec_step_ms = dec_ms / (K * S)
-    comp_pass_ms = comp_ms / K
-
-    kern = {}
-    for name, (n, ms) in per.items():
-        kern[name] = {"launches": n, "avg_ms": ms / n, "total_ms": ms}
-    attn = kern.get("decode_attn", {"avg_ms": float("nan")})
-    attn_gbs = dec_bytes_avg / (attn["avg_ms"] * 1e-3) / 1e9
-    comp_kernel_ms = sum(v["total_ms"] for k, v in kern.items() if not k.startswith(("decode", "append")))
+    res, live = measure_workload(tk, W, wl, dev, steps=args.steps, warmup=args.warmup, policy=args.policy, peak=peak,
+                                 peak_kind=peak_kind, sampler_gpu=local, world=world)
+    qs, ks, vs, steps_in, params = (live[x] for x in ("qs", "ks", "vs", "steps_in", "params"))
+    comp_bytes = live["comp_bytes"]
 
     line = {
         "metric": "decode attn steps/s (compress tokens/s beside it)",
-        "value": value, "unit": "steps/s", "n_gpus": world, "steps": K, "warmup": args.warmup,
-        "ms_per_step": total_ms / K, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
+        "value": res["value"], "unit": "steps/s", "n_gpus": world, "steps": args.steps, "warmup": args.warmup,
+        "ms_per_step": res["ms_per_step"], "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
         "dtype": wl.dtype, "data": "synthetic",
         "config": dict(wl.describe(), mid_policy=args.policy, l2="inputs (>=8 GB of K, >=3 GB retained cache) exceed the 126 MB L2",
                        step="compress all layers + decode_steps x (append + attention, one fused call)"),
-        "decode_ms_per_step": dec_step_ms, "compress_ms": comp_pass_ms, "compress_tokens_per_s": comp_tps,
-        "per_pass": {"compress_ms_median": statistics.median(comp_each), "compress_ms_min": min(comp_each),
-                     "decode_ms_per_step_median": statistics.median(dec_each),
-                     "decode_ms_per_step_min": min(dec_each), "passes": len(evs)},
-        "hbm": {
-            "peak_gbs": peak, "peak_kind": peak_kind, "nominal_gbs": NOMINAL_HBM_GBS,
-            "decode_gbs": dec_bytes_avg / (dec_step_ms * 1e-3) / 1e9,
-            "decode_frac": dec_bytes_avg / (dec_step_ms * 1e-3) / 1e9 / peak,
-            "compress_gbs": comp_bytes / (comp_pass_ms * 1e-3) / 1e9,
-            "compress_frac": comp_bytes / (comp_pass_ms * 1e-3) / 1e9 / peak,
-            "decode_bytes_per_step": dec_bytes_avg, "compress_bytes": comp_bytes,
-        },
-        "roofline": {"bound": "hbm", "kernel": "decode_attn", "achieved": attn_gbs, "peak": peak, "unit": "GB/s",
-                     "frac": attn_gbs / peak, "peak_kind": peak_kind,
-                     "traffic": ncu_traffic(wl, int(info.retained_rows)), "traffic_unit": "bytes per launch",
-                     "algorithmic_bytes": dec_bytes_avg, "avg_launch_ms": attn["avg_ms"]},
-        "kernels": kern, "compress_kernel_ms": comp_kernel_ms,
-        "gpu_launches": launches, "device_status": status, "clocks": clocks,
     }
+    line.update({k: v for k, v in res.items() if k not in ("value", "ms_per_step")})
 
     if rank == 0 and not args.no_latency:
         line["latency_mode"] = run_latency_mode(tk, wl, qs, ks, vs, steps_in, args)
@@ -274,6 +336,10 @@ def run_ours(args):
         line["cpu_baseline"] = None      # the oracle is timed on the method's own policy only
     elif rank == 0 and world == 1 and not args.no_cpu:
         line["cpu_baseline"] = cpu_baseline(wl, qs, ks, vs, steps_in)
+    del qs, ks, vs, steps_in, params, live
+    torch.cuda.empty_cache()
+    if rank == 0 and world == 1 and not args.no_extra:
+        line["workloads"] = run_extra_workloads(tk, W, args, dev, peak, peak_kind, local)
     if rank == 0:
         print(json.dumps(line))
     if world > 1:
@@ -496,12 +562,15 @@ def run_with_window_lse(tk, wl, qs, ks, vs, args, comp_bytes, peak):
 
 
 def ncu_traffic(wl, retained_rows):
-    """DRAM bytes per decode_attn launch from the committed ncu capture (profiles/decode_attn_llama2_4layers.md):
-    383.07 MB read + written for 739,056 retained rows of 256 bytes, K and V.  Traffic grows in proportion to the
-    rows read, so it is scaled by rows; only the bf16, d = 128, one-query-head-per-KV-head shape was captured."""
-    if wl.dtype != "bf16" or wl.head_dim != 128 or wl.n_heads != wl.n_kv_heads:
-        return None
-    return 383.07e6 / 739056 * retained_rows
+    """DRAM bytes per decode_attn launch, from the committed ncu captures of the kernel as it is now, scaled by the
+    rows a launch reads (traffic grows in proportion to them; a full-size launch holds too much on the device for a
+    multi-pass capture).  Returns (bytes or None, the capture it comes from)."""
+    if wl.dtype != "bf16" or wl.head_dim != 128:
+        return None, None
+    if wl.n_heads == wl.n_kv_heads:
+        # 378.44 MB read + 4.63 MB written for 739,056 retained rows of 256 bytes, K and V
+        return 383.07e6 / 739056 * retained_rows, "profiles/decode_attn_llama2_4layers.md (one query head per KV head)"
+    return None, None
 
 
 def run_e2e(tk, wl, params, qs, ks, vs, steps_in, world):
@@ -584,6 +653,7 @@ def cpu_baseline(wl, qs, ks, vs, steps_in):
     comp_full = comp_s * tokens_units / keys
     dec_full = dec_s * wl.retained_rows() / rows
     return {"value": 1.0 / dec_full, "unit": "steps/s", "cores": cpu_threads(), "kind": "oracle",
+            "threads": "single-process numpy float64; only its BLAS matrix products run on `cores` threads",
             "compress_tokens_per_s": sum(wl.seq_lens) / comp_full,
             "sample": f"all KV heads of {layers} layer(s) of sequence 0: compress {comp_s:.1f} s ({keys} keys), "
                       f"decode steps {dec_s:.1f} s ({rows} rows read); scaled by keys scanned ({tokens_units}) and "
@@ -595,8 +665,9 @@ def run_reference(args):
     rank = int(os.environ.get("RANK", "0"))
     if rank != 0:
         return
+    from oracle import taskkv_oracle as O
     from paper_2501_15113_b200 import workloads as W
-    wl = get_workload(args.workload, args)
+    wl = get_workload(args.workload, args, helpers=(O.hetero_count, O.mid_budget))   # no CUDA library on this arm
     n_units = 4
     sub = W.Workload(**{**wl.__dict__})
     qs, ks, vs = [], [], []
@@ -626,7 +697,8 @@ def run_reference(args):
             "vs_baseline": None, "dtype": "f64", "data": "synthetic", "config": wl.describe(),
             "compress_tokens_per_s": sum(wl.seq_lens) / comp_full,
             "cpu_baseline": {"value": value, "unit": "steps/s", "cores": cpu_threads(), "kind": "oracle",
-                             "sample": sample},
+                             "threads": "single-process numpy float64; only its BLAS matrix products run on `cores` "
+                                        "threads", "sample": sample},
             "e2e": {"value": value, "unit": "steps/s", "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0}}
     print(json.dumps(line))
 
@@ -646,9 +718,8 @@ def main():
     ap.add_argument("--no-latency", action="store_true", help="skip the layer-by-layer decode measurement")
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--no-cpu", action="store_true")
+    ap.add_argument("--no-extra", action="store_true", help="skip the other workloads (grouped-query, batch, sweep)")
     args = ap.parse_args()
-    import __graft_entry__ as ge
-    ge.build()          # the workload tables use the library's host-only schedule / budget helpers
     if args.impl == "reference":
         run_reference(args)
     else:
