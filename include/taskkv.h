@@ -202,7 +202,9 @@ taskkv_status taskkv_compress(const void* q_win, const void* k, const void* v,
 /* As taskkv_compress_ex, but q_win[b], k[b], v[b] are HOST buffers (pinned
  * memory gives asynchronous copies).  Layers are staged through device
  * buffers the library allocates, so the host-to-device copies are part of the
- * call.  Cache memory is library-owned. */
+ * call.  Cache memory is library-owned.  The call synchronises the stream and
+ * then reads the cache's sticky device status: if a kernel recorded an error
+ * (ETIMEOUT) the cache is destroyed, *out_cache is NULL and that code is returned. */
 taskkv_status taskkv_compress_host(const taskkv_params* p, const void* const* q_win,
                                    const void* const* k, const void* const* v,
                                    taskkv_stream stream, taskkv_cache** out_cache);
@@ -244,7 +246,10 @@ taskkv_status taskkv_decode_step(const void* q, const void* k_new, const void* v
 
 /* One decode step with HOST buffers: copies q, k_new, v_new in, appends,
  * attends and copies out back (k_new and v_new may both be NULL to skip the
- * append).  Synchronises the stream before returning. */
+ * append).  Synchronises the stream before returning, and returns the cache's
+ * sticky device status if it is not TASKKV_OK (ESTATE: a unit was already at
+ * capacity, its row was not appended, `out` is still the attention over the
+ * rows it holds; ETIMEOUT: a bounded device-side wait ran out). */
 taskkv_status taskkv_decode_host(const void* q, const void* k_new, const void* v_new, taskkv_cache* c,
                                  void* out, taskkv_stream stream);
 
@@ -260,7 +265,8 @@ taskkv_status taskkv_decode_host(const void* q, const void* k_new, const void* v
  *   q, out    [n_units * group][head_dim] in `dtype`; unit u serves query heads u*group .. u*group+group-1
  *   k_pool, v_pool   rows of head_dim elements; unit u owns rows seg_off[u] .. seg_off[u] + lengths[u] - 1
  *   seg_off   device int64 [n_units];  lengths  device int32 [n_units]
- *   max_len   host-side upper bound of every lengths[u] (sets the work split)
+ *   max_len   host-side upper bound of every lengths[u] (sets the work split); a unit whose length is larger
+ *             attends over its first max_len rows only (the length is clamped, never read past)
  * Limits: group in {1,2,4,8}, head_dim in {64,128}, and
  * n_units * group * (head_dim + 2) * 4 bytes must fit the 32 MiB scratch;
  * beyond that the call returns TASKKV_EINVAL (with a line on stderr) and
@@ -304,6 +310,22 @@ int32_t taskkv_hetero_count(int32_t n, float beta, int32_t m, int32_t R, int32_t
  * of the layer, the quotient floored, clamped to [0, N - s1 - s2].  Host only. */
 int32_t taskkv_mid_budget(double budget_tokens, int32_t N, int32_t h_full, int32_t n,
                           int32_t sink, int32_t recent);
+
+/* Eq. 17 from Eq. 16's head count f = f(r).  literal = 0: h = f plus the promoted closest head (if promote_center
+ * and f < n), i.e. the heads that really keep a full cache, so the layer total stays within the budget;
+ * literal = 1: h = f, Eq. 17 exactly as printed.  Host only. */
+int32_t taskkv_mid_budget_ex(double budget_tokens, int32_t N, int32_t f, int32_t n, int32_t sink, int32_t recent,
+                             int32_t promote_center, int32_t literal);
+
+/* Self-test of the bounded device-side waits (no counterpart in the paper).  The tensor-core kernels wait on
+ * shared-memory barriers with an iteration limit; when a wait runs out the block raises an abort flag, every other
+ * wait of the block returns at once, and the kernel records TASKKV_ETIMEOUT in its status word and exits normally.
+ * This call runs that wait, in a one-block kernel with nothing else in flight, on a barrier that nobody completes,
+ * with a limit of `max_polls` polls (clamped to [1, 65536]; a few milliseconds at most), then a second wait that
+ * must return at once because of the abort flag.  Synchronises `stream`.  Returns TASKKV_ETIMEOUT when the wait
+ * gave up as designed (the expected result), TASKKV_OK if it did not, TASKKV_ECUDA on a runtime error;
+ * *polls_out (host, optional) receives the polls the first wait made. */
+taskkv_status taskkv_selftest_bounded_wait(int32_t max_polls, int32_t* polls_out, taskkv_stream stream);
 
 /* Kernel launches issued by this library in this process so far. */
 int64_t taskkv_launch_count(void);

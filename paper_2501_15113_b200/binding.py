@@ -99,6 +99,10 @@ lib.taskkv_hetero_count.argtypes = [C.c_int32, C.c_float, C.c_int32, C.c_int32, 
 lib.taskkv_hetero_count.restype = C.c_int32
 lib.taskkv_mid_budget.argtypes = [C.c_double] + [C.c_int32] * 5
 lib.taskkv_mid_budget.restype = C.c_int32
+lib.taskkv_mid_budget_ex.argtypes = [C.c_double] + [C.c_int32] * 7
+lib.taskkv_mid_budget_ex.restype = C.c_int32
+lib.taskkv_selftest_bounded_wait.argtypes = [C.c_int32, C.POINTER(C.c_int32), _vp]
+lib.taskkv_selftest_bounded_wait.restype = C.c_int32
 lib.taskkv_launch_count.argtypes = []
 lib.taskkv_launch_count.restype = C.c_int64
 lib.taskkv_timing_enable.argtypes = [C.c_int32]
@@ -126,6 +130,19 @@ def taskkv_hetero_count(n: int, beta: float, m: int, R: int, r: int) -> int:
 
 def taskkv_mid_budget(budget_tokens: float, N: int, h_full: int, n: int, sink: int, recent: int) -> int:
     return int(lib.taskkv_mid_budget(budget_tokens, N, h_full, n, sink, recent))
+
+
+def taskkv_mid_budget_ex(budget_tokens: float, N: int, f: int, n: int, sink: int, recent: int,
+                         promote_center: bool = True, literal: bool = False) -> int:
+    return int(lib.taskkv_mid_budget_ex(budget_tokens, N, f, n, sink, recent, 1 if promote_center else 0,
+                                        1 if literal else 0))
+
+
+def taskkv_selftest_bounded_wait(max_polls: int = 2000, stream=None):
+    """(status, polls): status is ETIMEOUT when the bounded wait gave up as designed."""
+    polls = C.c_int32(0)
+    st = int(lib.taskkv_selftest_bounded_wait(max_polls, C.byref(polls), _stream_handle(stream)))
+    return st, int(polls.value)
 
 
 def taskkv_launch_count() -> int:
@@ -440,14 +457,35 @@ def taskkv_decode_noalloc(q: torch.Tensor, k_pool: torch.Tensor, v_pool: torch.T
     """Decode attention over caller-held pools with the library's fixed scratch: no
     allocation happens inside the call (`out` is allocated here, by torch, only if
     the caller passes none).  q: [n_units * group, d]; pools: [rows, d];
-    seg_off int64 [n_units]; lengths int32 [n_units]; max_len >= lengths.max()."""
+    seg_off int64 [n_units]; lengths int32 [n_units]; a length above max_len is
+    clamped to max_len.  The C side sees only pointers, so shapes, types and
+    devices are checked here."""
+    if q.dtype not in (torch.bfloat16, torch.float32):
+        raise ValueError("q must be bf16 or fp32")
     if out is None:
         out = torch.empty_like(q)
-    d = q.shape[-1]
     n_units = lengths.numel()
+    if q.dim() != 2 or q.shape[0] != n_units * group:
+        raise ValueError("q must be [n_units * group, head_dim]")
+    d = q.shape[1]
+    if out.shape != q.shape or out.dtype != q.dtype:
+        raise ValueError("out must match q")
+    for name, t in (("k_pool", k_pool), ("v_pool", v_pool)):
+        if t.dim() != 2 or t.shape[1] != d or t.dtype != q.dtype:
+            raise ValueError(f"{name} must be [rows, head_dim] in q's dtype")
+    if k_pool.shape != v_pool.shape:
+        raise ValueError("k_pool and v_pool must have the same shape")
+    if seg_off.dtype != torch.int64 or seg_off.numel() != n_units:
+        raise ValueError("seg_off must be int64 [n_units]")
+    if lengths.dtype != torch.int32:
+        raise ValueError("lengths must be int32 [n_units]")
+    for name, t in (("q", q), ("out", out), ("k_pool", k_pool), ("v_pool", v_pool), ("seg_off", seg_off),
+                    ("lengths", lengths)):
+        if not t.is_cuda or t.device != q.device or not t.is_contiguous():
+            raise ValueError(f"{name} must be a contiguous CUDA tensor on q's device")
     dtype = BF16 if q.dtype == torch.bfloat16 else F32
     _check(lib.taskkv_decode_noalloc(q.data_ptr(), k_pool.data_ptr(), v_pool.data_ptr(), seg_off.data_ptr(),
-                                     lengths.data_ptr(), n_units, group, d, dtype, max_len, out.data_ptr(),
+                                     lengths.data_ptr(), n_units, group, d, dtype, int(max_len), out.data_ptr(),
                                      _stream_handle(stream)), "taskkv_decode_noalloc")
     return out
 

@@ -11,7 +11,7 @@ ROOT = os.path.dirname(HERE)
 CSRC = os.path.join(HERE, "csrc")
 OBJ = os.path.join(ROOT, "_build")
 LIB = os.path.join(HERE, "libtaskkv.so")
-SOURCES = ["api.cu", "window_score.cu", "window_score_tc.cu", "window_score_res.cu", "exact_semantic.cu", "select.cu", "separator.cu", "gather.cu", "decode.cu", "decode_noalloc.cu"]
+SOURCES = ["api.cu", "window_score.cu", "window_score_tc.cu", "window_score_res.cu", "exact_semantic.cu", "select.cu", "separator.cu", "gather.cu", "decode.cu", "decode_noalloc.cu", "selftest.cu"]
 NVCC = os.environ.get("NVCC", "/usr/local/cuda/bin/nvcc")
 FLAGS = ["-gencode", "arch=compute_100a,code=sm_100a", "-lineinfo", "-O3", "-std=c++17",
          "-Xcompiler", "-fPIC", "-I", os.path.join(ROOT, "include"), "-I", CSRC]

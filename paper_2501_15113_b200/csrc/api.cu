@@ -181,7 +181,7 @@ thread_local cudaEvent_t tl_start = nullptr;
 
 const char* kKernelNames[K_COUNT] = {
     "window_stats", "window_reduce", "window_scores", "select", "separator", "plan",
-    "gather", "append", "decode_attn", "decode_combine", "window_tc", "compensate", "exact_sum"};
+    "gather", "append", "decode_attn", "decode_combine", "window_tc", "compensate", "exact_sum", "selftest"};
 
 }  // namespace
 
@@ -391,6 +391,16 @@ void build_meta(taskkv_cache* c, const void* const* q_win, const void* const* k,
 
 taskkv_status cuda_status(cudaError_t e) { return e == cudaSuccess ? TASKKV_OK : TASKKV_ECUDA; }
 
+// The cache's sticky device status word, read after everything on `s` has finished (the synchronising entry points
+// report it; the asynchronous ones leave it to the next synchronising call or to taskkv_cache_query).
+taskkv_status sticky_status(const taskkv_cache* c, cudaStream_t s) {
+  int32_t word = 0;
+  cudaError_t e = cudaMemcpyAsync(&word, c->dp.status, sizeof(word), cudaMemcpyDeviceToHost, s);
+  if (e == cudaSuccess) e = cudaStreamSynchronize(s);
+  if (e != cudaSuccess) return TASKKV_ECUDA;
+  return (taskkv_status)word;
+}
+
 }  // namespace
 
 // ================================================================ exported calls
@@ -596,10 +606,12 @@ taskkv_status taskkv_compress_host(const taskkv_params* p, const void* const* q_
   st = taskkv_compress_ex(p, dq.data(), dk.data(), dv.data(), nullptr, 0, nullptr, 0, stream, out_cache);
   e = cudaStreamSynchronize(s);
   release();
-  if (st == TASKKV_OK && e != cudaSuccess) {
+  if (st == TASKKV_OK && e != cudaSuccess) st = TASKKV_ECUDA;
+  // a kernel that gave up on a bounded wait leaves its code in the cache's status word: the cache is then unusable
+  if (st == TASKKV_OK) st = sticky_status(*out_cache, s);
+  if (st != TASKKV_OK && *out_cache) {
     taskkv_cache_destroy(*out_cache);
     *out_cache = nullptr;
-    return TASKKV_ECUDA;
   }
   return st;
 }
@@ -694,8 +706,8 @@ taskkv_status taskkv_decode_host(const void* q, const void* k_new, const void* v
   if (e == cudaSuccess)
     e = launch_decode(c->dp, c->prm.dtype, dq, nullptr, k_new ? dkn : nullptr, k_new ? dvn : nullptr, dout, s);
   if (e == cudaSuccess) e = cudaMemcpyAsync(out, dout, q_bytes, cudaMemcpyDeviceToHost, s);
-  if (e == cudaSuccess) e = cudaStreamSynchronize(s);
-  return cuda_status(e);
+  if (e != cudaSuccess) return TASKKV_ECUDA;
+  return sticky_status(c, s);      // synchronises; ESTATE if a unit was at capacity, ETIMEOUT after a device time-out
 }
 
 int64_t taskkv_cache_query_bytes(const taskkv_cache* c, int32_t what) {
@@ -781,6 +793,14 @@ int32_t taskkv_mid_budget(double budget_tokens, int32_t N, int32_t h_full, int32
   if (k < 0) k = 0;
   if (k > room) k = room;
   return (int32_t)k;
+}
+
+int32_t taskkv_mid_budget_ex(double budget_tokens, int32_t N, int32_t f, int32_t n, int32_t sink, int32_t recent,
+                             int32_t promote_center, int32_t literal) {
+  if (f < 0) f = 0;
+  if (f > n) f = n;
+  const int32_t h = literal ? f : std::min(n, f + ((promote_center && f < n) ? 1 : 0));
+  return taskkv_mid_budget(budget_tokens, N, h, n, sink, recent);
 }
 
 int64_t taskkv_launch_count(void) { return g_launches.load(); }

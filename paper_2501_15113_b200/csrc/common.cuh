@@ -32,6 +32,7 @@ enum KernelId : int32_t {
   K_WINDOW_TC,
   K_COMPENSATE,
   K_EXACT_SUM,
+  K_SELFTEST,
   K_COUNT
 };
 

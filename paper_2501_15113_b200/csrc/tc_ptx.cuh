@@ -39,17 +39,22 @@ static __device__ __forceinline__ uint32_t mbar_try_wait(uint32_t bar, uint32_t 
       : "memory");
   return ok;
 }
-// Bounded wait: false if the CTA is aborting or the limit ran out (which raises the abort flag).
-static __device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile int* abort_flag) {
+// Bounded wait: false if the CTA is aborting or the limit of polls ran out (which raises the abort flag).
+static __device__ __forceinline__ bool mbar_wait_limit(uint32_t bar, uint32_t parity, volatile int* abort_flag,
+                                                        uint32_t limit, uint32_t* polls = nullptr) {
   for (uint32_t spin = 0;; ++spin) {
+    if (polls) *polls = spin;
     if (mbar_try_wait(bar, parity)) return true;
     if (*abort_flag) return false;
-    if (spin > kSpinLimit) {
+    if (spin > limit) {
       *abort_flag = 1;
       return false;
     }
     if (spin > 32) __nanosleep(128);
   }
+}
+static __device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile int* abort_flag) {
+  return mbar_wait_limit(bar, parity, abort_flag, kSpinLimit);
 }
 // One lane of a converged warp.  The role loops below are run by all 32 lanes and only the TMA / MMA /
 // commit instructions sit under this predicate: address and descriptor arithmetic then stays warp-uniform

@@ -60,6 +60,27 @@ def test_mid_budget_matches_oracle(tk):
                 assert tk.taskkv_mid_budget(B, N, h, n, 4, 256) == O.mid_budget(B, N, h, n, 4, 256)
 
 
+def test_mid_budget_from_far_head_count_and_literal_reading(tk):
+    """Eq. 17 from f(r): the default counts the promoted head among the full caches (the layer total stays within
+    the budget); literal = 1 is Eq. 17 exactly as printed, h = f(r)."""
+    for N in (512, 30000, 131072):
+        for n in (8, 32):
+            for f in (0, 1, 2, n - 1, n):
+                for frac in (0.1, 0.4, 0.6, 1.0):
+                    B = frac * n * N
+                    assert tk.taskkv_mid_budget_ex(B, N, f, n, 4, 256, literal=True) == O.mid_budget(B, N, f, n, 4, 256)
+                    h = min(n, f + 1)
+                    assert tk.taskkv_mid_budget_ex(B, N, f, n, 4, 256) == O.mid_budget(B, N, h, n, 4, 256)
+                    assert tk.taskkv_mid_budget_ex(B, N, f, n, 4, 256, promote_center=False) == \
+                        O.mid_budget(B, N, f, n, 4, 256)
+    # the printed form overshoots the budget once the promoted head is stored in full; the default does not
+    N, n, f = 131072, 8, 2
+    B = 0.4 * n * N
+    k_lit = tk.taskkv_mid_budget_ex(B, N, f, n, 4, 256, literal=True)
+    k_def = tk.taskkv_mid_budget_ex(B, N, f, n, 4, 256)
+    assert (f + 1) * N + (n - f - 1) * (k_lit + 260) > B >= (f + 1) * N + (n - f - 1) * (k_def + 260)
+
+
 def test_plan_matches_closed_forms(tk):
     from paper_2501_15113_b200 import configs
     for wl in (configs.config1_toy(), configs.config2_llama2(), configs.config3_llama3(),

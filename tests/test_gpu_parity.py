@@ -783,3 +783,46 @@ def test_exact_semantic_vector(case):
                 np.testing.assert_allclose(want_v, O.exact_semantic_vector(q64[0], k64, v64), rtol=0, atol=1e-13)
             bound = P.TOL_SCORE_REL * (want_c[:, None] * np.abs(v64)).sum(axis=0).max()
             assert np.abs(P.to64(sem[r, h]) - want_v).max() < bound
+
+
+# ---------------------------------------------------------------------------
+# Error reporting across the boundary
+# ---------------------------------------------------------------------------
+def test_bounded_device_wait_runs_out_and_reports_timeout():
+    """The waits inside the tensor-core kernels have an iteration limit.  The library's self-test runs that wait in a
+    one-block kernel on a barrier nothing completes (no copy or MMA in flight): the wait gives up after the limit,
+    the block's later waits return at once, the kernel exits normally and leaves ETIMEOUT in its status word.  The
+    context stays usable: a regular compression runs right after it."""
+    tk = _tk()
+    st, polls = tk.taskkv_selftest_bounded_wait(2000)
+    assert st == tk.ETIMEOUT
+    assert 2000 <= polls <= 2002
+    st, polls = tk.taskkv_selftest_bounded_wait(1)
+    assert st == tk.ETIMEOUT and polls <= 3
+    wl = small("after_timeout", n=4, n_kv=4, d=128, N=1500, L=32, s1=4, s2=64, k=50, dtype="bf16", steps=1)
+    run_workload(wl)
+
+
+def test_host_buffer_calls_return_the_sticky_device_status():
+    """taskkv_decode_host synchronises, so it can and does return what the kernels left in the cache's status word:
+    a step beyond a unit's capacity is reported as ESTATE by the call itself (the attention over the rows the unit
+    holds is still delivered), and stays reported until the cache is destroyed."""
+    tk = _tk()
+    wl = small("host_status", n=4, n_kv=4, d=64, N=300, L=8, s1=4, s2=32, k=20, dtype="f32")
+    qs, ks, vs = W.materialize(wl, "cpu")
+    params = tk.params_from_workload(wl, max_new_tokens=1)
+    cache = tk.taskkv_compress_host(params, [t.pin_memory() for t in qs], [t.pin_memory() for t in ks],
+                                    [t.pin_memory() for t in vs])
+    q, kn, vn = (t.pin_memory() for t in W.gen_decode_step(wl, 0, "cpu"))
+    out = torch.empty_like(q).pin_memory()
+    cache.taskkv_decode_host(q, kn, vn, out)                     # fits: one reserved row per unit
+    assert cache.status() == 0
+    first = out.clone()
+    with pytest.raises(tk.TaskKVError) as ei:
+        cache.taskkv_decode_host(q, kn, vn, out)                 # no room left
+    assert ei.value.status == tk.ESTATE
+    assert torch.equal(out, first)                               # same rows attended, nothing appended
+    with pytest.raises(tk.TaskKVError) as ei:
+        cache.taskkv_decode_host(q, None, None, out)             # sticky
+    assert ei.value.status == tk.ESTATE
+    cache.close()
