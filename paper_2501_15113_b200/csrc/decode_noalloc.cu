@@ -68,6 +68,7 @@ struct NaArgs {
   float* part_acc;     // [n_units * splits][G][D]   (inside the static scratch)
   float* part_ml;      // [n_units * splits][G][2]
   int32_t n_units, splits, rows_per_split;
+  int32_t max_len;     // lengths above it are clamped to it
 };
 
 template <typename T, int D, int G>
@@ -92,7 +93,7 @@ __global__ void __launch_bounds__(kNaThreads) na_attn_kernel(NaArgs a) {
   for (int item = blockIdx.x; item < total; item += gridDim.x) {
     __syncthreads();
     const int u = item / a.splits, sp = item % a.splits;
-    const int len = max(a.lengths[u], 0);
+    const int len = min(max(a.lengths[u], 0), a.max_len);
     const int rbeg = min(len, sp * a.rows_per_split);
     const int rend = min(len, rbeg + a.rows_per_split);
     const int64_t seg = a.seg_off[u];
@@ -228,8 +229,16 @@ template <typename T, int D, int G>
 cudaError_t na_launch(const NaArgs& a, cudaStream_t s) {
   const int64_t total = (int64_t)a.n_units * a.splits;
   const unsigned grid = (unsigned)(total < 148 * 8 ? total : 148 * 8);
-  na_attn_kernel<T, D, G><<<grid, kNaThreads, 0, s>>>(a);
-  na_combine_kernel<T, D, G><<<(unsigned)((a.n_units * G + 7) / 8), 256, 0, s>>>(a);
+  {
+    LaunchScope ls(K_DECODE_ATTN, s);
+    na_attn_kernel<T, D, G><<<grid, kNaThreads, 0, s>>>(a);
+  }
+  cudaError_t e = cudaGetLastError();
+  if (e != cudaSuccess) return e;      // no combine over partials that were never written
+  {
+    LaunchScope ls(K_DECODE_COMBINE, s);
+    na_combine_kernel<T, D, G><<<(unsigned)((a.n_units * G + 7) / 8), 256, 0, s>>>(a);
+  }
   return cudaGetLastError();
 }
 
@@ -291,6 +300,7 @@ extern "C" taskkv_status taskkv_decode_noalloc(const void* q, const void* k_pool
   a.n_units = n_units;
   a.splits = (int32_t)splits;
   a.rows_per_split = (int32_t)rps;
+  a.max_len = max_len;
   const size_t items = (size_t)n_units * (size_t)splits;
   a.part_acc = static_cast<float*>(scratch);
   a.part_ml = reinterpret_cast<float*>(static_cast<unsigned char*>(scratch) +
