@@ -99,6 +99,11 @@ typedef struct taskkv_params {
   const int32_t* seq_lens;   /* host [batch]: N_b (ragged batches allowed) */
   const int32_t* mid_budget_per_layer;  /* host [n_layers] or NULL; overrides mid_budget */
   const int32_t* n_hetero;   /* host [batch][n_layers] or NULL; overrides Eq. 16 */
+  float   budget_frac;       /* 0: mid_budget (or mid_budget_per_layer) is used as given.  In (0, 1]: the KV budget of
+                                Sec. IV-B as a fraction of the full cache; every (sequence, layer) then gets the middle
+                                budget of Eq. 17, k = floor((B - N h) / (n - h)) - s1 - s2 with B = fraction * n_kv * N_b
+                                and h the heads of that layer that keep everything, computed on the device (and, for
+                                the exact sizing of the pools, by the same formula on the host) */
 } taskkv_params;
 
 typedef struct taskkv_plan_info {
@@ -136,11 +141,13 @@ taskkv_status taskkv_plan(const taskkv_params* p, taskkv_plan_info* out);
  * semantic vector.  Errors: EINVAL (arguments), EALLOC, ECUDA.
  * Streams: all work is ordered after what `stream` holds at the call and is
  * complete, for every later operation on `stream`, when the call's last kernel is.
- * For large bf16 problems with 32 window rows the selection of one chunk of
- * layers runs beside the window scores of the next on a stream the library
- * owns (one per device, created by the first such call: make that call before
- * capturing `stream` into a graph); it is forked from and joined back into
- * `stream` with events, and calls that use it are serialised on the host.
+ * For large bf16 problems the steps of different chunks of layers overlap on
+ * streams the library owns (with 32 window rows the selection of one chunk
+ * beside the window scores of the next; with more window rows the gather of
+ * one chunk beside window scores and selection of the next; two streams per
+ * device, created by the first such call: make that call before capturing
+ * `stream` into a graph); they are forked from and joined back into `stream`
+ * with events, and calls that use them are serialised on the host.
  */
 taskkv_status taskkv_compress_ex(const taskkv_params* p, const void* const* q_win,
                                  const void* const* k, const void* const* v,
@@ -186,11 +193,30 @@ taskkv_status taskkv_compress_lse(const taskkv_params* p, const void* const* q_w
                                   void* workspace_mem, size_t workspace_bytes,
                                   taskkv_stream stream, taskkv_cache** out_cache);
 
-/* Layer at a time.  Nothing couples the layers of a sequence except the schedules of Eq. 16 / Eq. 17, which
- * are known before any data: a prefill loop can therefore compress layer r as soon as its K and V exist, as a
- * problem of its own with n_layers = 1, n_hetero = { f(r) } (taskkv_hetero_count with the model's R and r) and
- * that layer's mid_budget, into its own cache memory, and free the layer's K and V afterwards.  Classes,
- * lengths, retained positions and cache rows are those the all-layer call gives for layer r. */
+/* Layer at a time, into ONE cache.  Nothing couples the layers of a sequence except the schedules of Eq. 16 /
+ * Eq. 17, which are known before any data, and Eq. 16 also fixes how many heads of a layer keep everything, so
+ * the place of every layer's segments in the pools is known in advance.  A prefill loop can therefore create the
+ * cache first and compress layer r as soon as its K and V exist, then free them:
+ *   taskkv_cache_create    plans the whole problem (all layers, all sequences), takes or allocates cache and
+ *                          workspace memory exactly as taskkv_compress_ex does, uploads the tables and zeroes the
+ *                          state: every unit has length 0 until its layer is compressed.
+ *   taskkv_compress_layer  steps a1-a5 for layer `layer` of every sequence:
+ *                            q_win[b]  device [n_heads][L][d]       the layer's last L query rows
+ *                            k[b],v[b] device [n_kv_heads][N_b][d]  the layer's keys / values
+ *                            window_lse[b] device fp32 [n_heads][L] or window_lse == NULL (see taskkv_compress_lse)
+ *                          Each layer may be compressed once (ESTATE otherwise), in any order, all on one stream (or
+ *                          ordered by the caller: the calls share the workspace).  Classes, lengths, retained
+ *                          positions, cache rows, segment offsets and work lists are bit for bit those the all-layer
+ *                          call produces; once every layer is in, the cache is the same object, and
+ *                          taskkv_decode_step and the other decode calls work on it as usual (a layer-range decode
+ *                          may already run on layers that are in).
+ * Errors: EINVAL (arguments, layer out of range, cache without workspace), ESTATE, ECUDA. */
+taskkv_status taskkv_cache_create(const taskkv_params* p, void* cache_mem, size_t cache_bytes,
+                                  void* workspace_mem, size_t workspace_bytes, taskkv_stream stream,
+                                  taskkv_cache** out_cache);
+taskkv_status taskkv_compress_layer(taskkv_cache* c, int32_t layer, const void* const* q_win,
+                                    const void* const* k, const void* const* v, const void* const* window_lse,
+                                    taskkv_stream stream);
 
 /* The flat form of the same call: one bf16 sequence, Sec. V-D defaults for
  * everything not listed, library-owned memory, max_new_tokens = 4096. */

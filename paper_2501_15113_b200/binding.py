@@ -38,7 +38,7 @@ class taskkv_params(C.Structure):
         ("beta", C.c_float), ("promote_center", C.c_int32), ("force_class", C.c_int32), ("dtype", C.c_int32),
         ("max_new_tokens", C.c_int32), ("mid_policy", C.c_int32),
         ("seq_lens", C.POINTER(C.c_int32)), ("mid_budget_per_layer", C.POINTER(C.c_int32)),
-        ("n_hetero", C.POINTER(C.c_int32)),
+        ("n_hetero", C.POINTER(C.c_int32)), ("budget_frac", C.c_float),
     ]
 
 
@@ -57,6 +57,10 @@ lib.taskkv_plan.restype = C.c_int32
 lib.taskkv_compress_ex.argtypes = [C.POINTER(taskkv_params), _pp, _pp, _pp, _vp, C.c_size_t, _vp, C.c_size_t,
                                    _vp, C.POINTER(_vp)]
 lib.taskkv_compress_ex.restype = C.c_int32
+lib.taskkv_cache_create.argtypes = [C.POINTER(taskkv_params), _vp, C.c_size_t, _vp, C.c_size_t, _vp, C.POINTER(_vp)]
+lib.taskkv_cache_create.restype = C.c_int32
+lib.taskkv_compress_layer.argtypes = [_vp, C.c_int32, _pp, _pp, _pp, _pp, _vp]
+lib.taskkv_compress_layer.restype = C.c_int32
 lib.taskkv_compress_lse.argtypes = [C.POINTER(taskkv_params), _pp, _pp, _pp, _pp, _vp, C.c_size_t, _vp, C.c_size_t,
                                     _vp, C.POINTER(_vp)]
 lib.taskkv_compress_lse.restype = C.c_int32
@@ -172,12 +176,12 @@ class Params:
     def __init__(self, *, n_layers, n_heads, n_kv_heads, head_dim, seq_lens: Sequence[int], sink, recent,
                  mid_budget, window, dtype, top_t=256, pool_kernel=7, beta=0.25, m_top=4,
                  n_hetero: Optional[Sequence[Sequence[int]]] = None, promote_center=True, force_class=-1,
-                 max_new_tokens=0, mid_policy=0):
+                 max_new_tokens=0, mid_policy=0, budget_frac=0.0):
         self.kw = dict(n_layers=n_layers, n_heads=n_heads, n_kv_heads=n_kv_heads, head_dim=head_dim,
                        seq_lens=list(seq_lens), sink=sink, recent=recent, mid_budget=mid_budget, window=window,
                        dtype=dtype, top_t=top_t, pool_kernel=pool_kernel, beta=beta, m_top=m_top, n_hetero=n_hetero,
                        promote_center=promote_center, force_class=force_class, max_new_tokens=max_new_tokens,
-                       mid_policy=mid_policy)
+                       mid_policy=mid_policy, budget_frac=budget_frac)
         p = taskkv_params()
         lib.taskkv_params_default(C.byref(p))
         p.n_layers, p.n_heads, p.n_kv_heads, p.head_dim = n_layers, n_heads, n_kv_heads, head_dim
@@ -204,6 +208,7 @@ class Params:
         p.dtype = BF16 if dtype in (BF16, "bf16", torch.bfloat16) else F32
         p.max_new_tokens = max_new_tokens
         p.mid_policy = int(mid_policy)
+        p.budget_frac = float(budget_frac)
         self.c = p
 
     @property
@@ -266,6 +271,23 @@ class Cache:
             self.close()
         except Exception:
             pass
+
+    def taskkv_compress_layer(self, layer: int, q_win: Sequence[torch.Tensor], k: Sequence[torch.Tensor],
+                              v: Sequence[torch.Tensor], window_lse: Optional[Sequence[torch.Tensor]] = None,
+                              stream=None) -> None:
+        """Steps a1-a5 for one layer of every sequence of a cache made by taskkv_cache_create.
+        q_win[b]: [n, L, d]; k[b], v[b]: [n_kv, N_b, d] of that layer, contiguous CUDA tensors."""
+        for t in list(q_win) + list(k) + list(v):
+            if not t.is_contiguous() or not t.is_cuda:
+                raise ValueError("inputs must be contiguous CUDA tensors")
+        la = None
+        if window_lse is not None:
+            for t in window_lse:
+                if not t.is_contiguous() or not t.is_cuda or t.dtype != torch.float32:
+                    raise ValueError("window_lse must be contiguous fp32 CUDA tensors")
+            la = _ptr_array(window_lse)
+        _check(lib.taskkv_compress_layer(self._h, layer, _ptr_array(q_win), _ptr_array(k), _ptr_array(v), la,
+                                         _stream_handle(stream)), "taskkv_compress_layer")
 
     # -- the decode-side calls
     def taskkv_append(self, k_new: torch.Tensor, v_new: torch.Tensor, stream=None) -> None:
@@ -405,6 +427,23 @@ def taskkv_compress_ex(params: Params, q_win: Sequence[torch.Tensor], k: Sequenc
     return Cache(h.value, params, {"cache": cache_mem, "workspace": workspace_mem})
 
 
+def taskkv_cache_create(params: Params, device, stream=None, cache_mem: Optional[torch.Tensor] = None,
+                        workspace_mem: Optional[torch.Tensor] = None) -> Cache:
+    """An empty cache for the whole problem (every layer of every sequence); layers are then compressed one at a
+    time with Cache.taskkv_compress_layer.  Cache and workspace memory are torch allocations unless supplied."""
+    info = taskkv_plan(params)
+    if cache_mem is None:
+        cache_mem = torch.empty(int(info.cache_bytes), dtype=torch.uint8, device=device)
+    if workspace_mem is None:
+        workspace_mem = torch.empty(int(info.workspace_bytes), dtype=torch.uint8, device=device)
+    h = C.c_void_p()
+    with torch.cuda.device(cache_mem.device):
+        _check(lib.taskkv_cache_create(C.byref(params.c), cache_mem.data_ptr(), cache_mem.numel(),
+                                       workspace_mem.data_ptr(), workspace_mem.numel(), _stream_handle(stream),
+                                       C.byref(h)), "taskkv_cache_create")
+    return Cache(h.value, params, {"cache": cache_mem, "workspace": workspace_mem})
+
+
 def taskkv_compress_host(params: Params, q_win: Sequence[torch.Tensor], k: Sequence[torch.Tensor],
                          v: Sequence[torch.Tensor], stream=None) -> Cache:
     """Same call with HOST tensors (pinned for asynchronous copies)."""
@@ -495,6 +534,7 @@ def params_from_workload(wl, max_new_tokens: Optional[int] = None, **overrides) 
               seq_lens=wl.seq_lens, sink=wl.sink, recent=wl.recent, mid_budget=list(wl.mid_budget),
               window=wl.window, dtype=wl.dtype, top_t=wl.top_t, pool_kernel=wl.pool_kernel,
               n_hetero=wl.n_hetero, promote_center=wl.promote_center,
+              budget_frac=getattr(wl, "budget_frac", 0.0),
               max_new_tokens=wl.decode_steps if max_new_tokens is None else max_new_tokens)
     kw.update(overrides)
     return Params(**kw)

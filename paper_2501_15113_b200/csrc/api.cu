@@ -1,8 +1,10 @@
 // Host side of the Task-KV library: argument validation, exact buffer planning,
 // the cache handle, and the kernel sequences behind the exported calls.
+#include <algorithm>
 #include <atomic>
 #include <cmath>
 #include <cstdio>
+#include <cstdlib>
 #include <cstring>
 #include <mutex>
 #include <new>
@@ -22,11 +24,15 @@ struct HostPlan {
   int64_t c_total = 0;
   int32_t max_N = 0, min_N = 0;
   int32_t chunks_max = 0, rows = 0, rows_pad = 0, idx_stride = 0;
-  std::vector<int32_t> seq_lens, mid, nhet;     // [B], [R], [B*R]
+  std::vector<int32_t> seq_lens, mid, nhet;     // [B], [B*R] middle budget of a (sequence, layer), [B*R]
   std::vector<int32_t> full;                    // [B*R] full-cache heads
   std::vector<int64_t> layer_items;             // [R] split-K decode items of a layer over all sequences, at capacity
+  // where each (sequence, layer) block starts: pool rows (block b * R + r), gather and decode work items (block
+  // r * B + b, layer-major); one entry more than blocks
+  std::vector<int64_t> seg_base;
+  std::vector<int32_t> gather_base, dec_base;
   // byte offsets inside the cache memory
-  size_t o_unit_N, o_unit_mid, o_nhet, o_c_off, o_qp, o_kp, o_vp, meta_bytes;
+  size_t o_unit_N, o_unit_mid, o_nhet, o_c_off, o_seg_base, o_gbase, o_dbase, o_qp, o_kp, o_vp, meta_bytes;
   size_t o_status, o_len, o_cap, o_seg, o_cls, o_dist, o_sem, o_idx, o_goff, o_doff, o_step, o_pacc, o_pml, o_kpool,
       o_vpool;
   // inside the workspace
@@ -40,6 +46,17 @@ int32_t hetero_count_impl(int32_t n, float beta, int32_t m, int32_t R, int32_t r
   if (f < 0) f = 0;
   if (f > n) f = n;
   return (int32_t)f;
+}
+
+// Eq. 17 with h full-cache heads: floor((B - N h) / (n - h)) - s1 - s2, clamped to [0, N - s1 - s2].
+int32_t mid_budget_impl(double budget_tokens, int32_t N, int32_t h_full, int32_t n, int32_t sink, int32_t recent) {
+  if (n <= h_full) return 0;
+  const double per_head = std::floor((budget_tokens - (double)N * (double)h_full) / (double)(n - h_full));
+  double k = per_head - (double)sink - (double)recent;
+  const double room = std::max(0, N - sink - recent);
+  if (k < 0) k = 0;
+  if (k > room) k = room;
+  return (int32_t)k;
 }
 
 taskkv_status make_plan(const taskkv_params* p, HostPlan& hp) {
@@ -56,6 +73,7 @@ taskkv_status make_plan(const taskkv_params* p, HostPlan& hp) {
   if (p->pool_kernel < 1 || p->pool_kernel > 31 || p->pool_kernel % 2 == 0) return TASKKV_EINVAL;
   if (p->force_class < -1 || p->force_class > 1) return TASKKV_EINVAL;
   if (p->mid_policy < TASKKV_MID_SELECT || p->mid_policy > TASKKV_MID_MEAN) return TASKKV_EINVAL;
+  if (!(p->budget_frac >= 0.f) || p->budget_frac > 1.f) return TASKKV_EINVAL;
   const int B = p->batch, R = p->n_layers, nkv = p->n_kv_heads;
   if ((int64_t)B * R * nkv > (1 << 20)) return TASKKV_EINVAL;
 
@@ -69,10 +87,11 @@ taskkv_status make_plan(const taskkv_params* p, HostPlan& hp) {
     hp.min_N = std::min(hp.min_N, N);
   }
   if (p->window > hp.min_N) return TASKKV_EINVAL;
-  hp.mid.resize(R);
+  hp.mid.resize((size_t)B * R);
   for (int r = 0; r < R; ++r) {
-    hp.mid[r] = p->mid_budget_per_layer ? p->mid_budget_per_layer[r] : p->mid_budget;
-    if (hp.mid[r] < 0) return TASKKV_EINVAL;
+    const int32_t m = p->mid_budget_per_layer ? p->mid_budget_per_layer[r] : p->mid_budget;
+    if (m < 0) return TASKKV_EINVAL;
+    for (int b = 0; b < B; ++b) hp.mid[(size_t)b * R + r] = m;
   }
   hp.nhet.resize((size_t)B * R);
   hp.full.resize((size_t)B * R);
@@ -86,6 +105,11 @@ taskkv_status make_plan(const taskkv_params* p, HostPlan& hp) {
       if (p->force_class == 1) h = nkv;
       if (p->force_class == 0) h = 0;
       hp.full[(size_t)b * R + r] = h;
+      // a budget given as a fraction of the full cache: Eq. 17 per (sequence, layer), with the heads that really
+      // keep everything (the device computes the same number for its own table, see budget_kernel)
+      if (p->budget_frac > 0.f)
+        hp.mid[(size_t)b * R + r] = mid_budget_impl((double)p->budget_frac * (double)nkv * (double)hp.seq_lens[b],
+                                                    hp.seq_lens[b], h, nkv, p->sink, p->recent);
     }
 
   const int64_t U = (int64_t)B * R * nkv;
@@ -93,24 +117,46 @@ taskkv_status make_plan(const taskkv_params* p, HostPlan& hp) {
   int64_t pool = 0, kept_rows = 0, gitems = 0, ditems = 0, c_total = 0;
   int32_t stride = 1;
   hp.layer_items.assign((size_t)R, 0);
+  hp.seg_base.assign((size_t)B * R + 1, 0);
+  std::vector<int64_t> blk_g((size_t)B * R, 0), blk_d((size_t)B * R, 0);   // per block b * R + r
   for (int b = 0; b < B; ++b) {
     const int64_t N = hp.seq_lens[b];
     for (int r = 0; r < R; ++r) {
-      const int64_t h = hp.full[(size_t)b * R + r];
+      const size_t br = (size_t)b * R + r;
+      const int64_t h = hp.full[br];
       int64_t kept = N;
-      if (N > (int64_t)s1 + s2) kept = s1 + s2 + std::min<int64_t>(hp.mid[r], N - s1 - s2);
+      if (N > (int64_t)s1 + s2) kept = s1 + s2 + std::min<int64_t>(hp.mid[br], N - s1 - s2);
       if (kept < N) stride = std::max<int32_t>(stride, (int32_t)kept);
+      hp.seg_base[br] = pool;
       pool += h * (N + mn) + (nkv - h) * (kept + mn);
       kept_rows += h * N + (nkv - h) * kept;
-      gitems += h * ((N + kGatherRows - 1) / kGatherRows) + (nkv - h) * ((kept + kGatherRows - 1) / kGatherRows);
+      blk_g[br] = h * ((N + kGatherRows - 1) / kGatherRows) + (nkv - h) * ((kept + kGatherRows - 1) / kGatherRows);
+      gitems += blk_g[br];
       const int64_t li = h * ((N + mn + kDecodeChunk - 1) / kDecodeChunk) +
                          (nkv - h) * ((kept + mn + kDecodeChunk - 1) / kDecodeChunk);
+      blk_d[br] = li;
       ditems += li;
       hp.layer_items[(size_t)r] += li;
       c_total += (int64_t)nkv * ((N + 3) / 4 * 4);
     }
   }
+  hp.seg_base[(size_t)B * R] = pool;
   if (gitems > 0x7fffffff || ditems > 0x7fffffff) return TASKKV_EINVAL;
+  // gather and decode work items are numbered layer-major: block r * B + b
+  hp.gather_base.assign((size_t)R * B + 1, 0);
+  hp.dec_base.assign((size_t)R * B + 1, 0);
+  {
+    int64_t g = 0, dd = 0;
+    for (int r = 0; r < R; ++r)
+      for (int b = 0; b < B; ++b) {
+        hp.gather_base[(size_t)r * B + b] = (int32_t)g;
+        hp.dec_base[(size_t)r * B + b] = (int32_t)dd;
+        g += blk_g[(size_t)b * R + r];
+        dd += blk_d[(size_t)b * R + r];
+      }
+    hp.gather_base[(size_t)R * B] = (int32_t)g;
+    hp.dec_base[(size_t)R * B] = (int32_t)dd;
+  }
   hp.idx_stride = (stride + 3) / 4 * 4;
   hp.c_total = c_total;
   hp.rows = G * p->window;
@@ -131,6 +177,9 @@ taskkv_status make_plan(const taskkv_params* p, HostPlan& hp) {
   hp.o_unit_mid = take(U * 4);
   hp.o_nhet = take((size_t)B * R * 4);
   hp.o_c_off = take((U + 1) * 8);
+  hp.o_seg_base = take(((size_t)B * R + 1) * 8);
+  hp.o_gbase = take(((size_t)B * R + 1) * 4);
+  hp.o_dbase = take(((size_t)B * R + 1) * 4);
   hp.o_qp = take(U * 8);
   hp.o_kp = take(U * 8);
   hp.o_vp = take(U * 8);
@@ -207,15 +256,39 @@ void note_launch_end(int32_t id, cudaStream_t s) {
 }
 }  // namespace taskkv
 
+struct taskkv_cache {
+  taskkv_params prm;
+  HostPlan hp;
+  DeviceProblem dp;
+  std::vector<unsigned char> meta;
+  void* cache_mem = nullptr;
+  void* work_mem = nullptr;
+  bool own_cache = false, own_work = false;
+  // staging for the host-buffer decode path
+  void* stage = nullptr;
+  size_t stage_bytes = 0;
+  std::vector<unsigned char> layer_done;   // [R] layers compressed so far (layer-streamed caches)
+};
+
 namespace {
-// Window scores and selection of different layers overlapped.  The single-read window kernel is bound by the K stream
-// and its clusters leave part of the SMs empty; the selection is bound by integer work on scores that sit in L2.  So the
-// layers are cut into chunks: the window kernel of chunk i+1 runs on the caller's stream while the selection of chunk i
-// runs on a side stream of the library (one per device, created on first use), joined back before the separator.
+// Two ways of overlapping the steps of different layers, both over chunks of layers and with streams the library
+// owns (per device, created on first use):
+//  (1) Multi-head attention (32 window rows): the single-read window kernel is bound by the K stream and its clusters
+//      leave part of the SMs empty; the selection is bound by integer work on scores that sit in L2.  The window
+//      kernel of chunk i+1 runs on the caller's stream while the selection of chunk i runs on a side stream, joined
+//      back before the separator.
+//  (2) Grouped queries (64 / 128 window rows): the two-pass window kernel is bound by its epilogue (one exponential
+//      per score and pass) and leaves two fifths of the HBM bandwidth unused, while the gather is a pure copy whose
+//      blocks need few registers and no shared memory.  Window scores and selection of chunk i+1 run on a
+//      high-priority stream; separator, plan and gather of chunk i run beside them on the caller's stream, their
+//      blocks placed on the same SMs as the (persistent, one per SM) window CTAs.  Every (sequence, layer) is planned
+//      on its own (the host knows where its block of segments starts), which is what lets a chunk be gathered
+//      before later layers are classified.
 constexpr int kMaxChunks = 8;
 struct SideStream {
-  cudaStream_t stream = nullptr;
-  cudaEvent_t ev[kMaxChunks + 1] = {};
+  cudaStream_t stream = nullptr;      // selection beside window scores (1)
+  cudaStream_t hi = nullptr;          // window scores + selection, above the caller's gather in priority (2)
+  cudaEvent_t ev[kMaxChunks + 2] = {};
   bool ok = false, tried = false;
 };
 std::mutex g_side_mu;
@@ -227,15 +300,18 @@ SideStream* side_stream() {   // call with g_side_mu held
   SideStream& ss = g_side[dev];
   if (!ss.tried) {
     ss.tried = true;
-    ss.ok = cudaStreamCreateWithFlags(&ss.stream, cudaStreamNonBlocking) == cudaSuccess;
-    for (int i = 0; ss.ok && i <= kMaxChunks; ++i)
+    int lo = 0, hi = 0;
+    ss.ok = cudaDeviceGetStreamPriorityRange(&lo, &hi) == cudaSuccess;
+    ss.ok = ss.ok && cudaStreamCreateWithFlags(&ss.stream, cudaStreamNonBlocking) == cudaSuccess;
+    ss.ok = ss.ok && cudaStreamCreateWithPriority(&ss.hi, cudaStreamNonBlocking, hi) == cudaSuccess;
+    for (int i = 0; ss.ok && i < kMaxChunks + 2; ++i)
       ss.ok = cudaEventCreateWithFlags(&ss.ev[i], cudaEventDisableTiming) == cudaSuccess;
     if (!ss.ok) cudaGetLastError();
   }
   return ss.ok ? &ss : nullptr;
 }
 
-// How many chunks of layers to overlap (1 = do not): only where the single-read window kernel and the
+// How many chunks of layers to overlap as in (1) (1 = do not): only where the single-read window kernel and the
 // register-resident selection run, with enough units per chunk to fill the window kernel's clusters many times over,
 // and not while per-kernel durations are being recorded (they are meant to be those of a kernel running alone).
 int overlap_chunks(const DeviceProblem& dp, int dtype, const WindowHostInfo& wh) {
@@ -248,43 +324,109 @@ int overlap_chunks(const DeviceProblem& dp, int dtype, const WindowHostInfo& wh)
   return chunks;
 }
 
-cudaError_t window_select_overlapped(const DeviceProblem& dp, int dtype, int max_N, const WindowHostInfo& wh,
-                                     int n_chunks, cudaStream_t s) {
+// Chunks for (2): the two-pass tensor-core window kernel, at least 32 units and 2 layers... per chunk.
+int gather_overlap_chunks(const DeviceProblem& dp, int dtype, const WindowHostInfo& wh) {
+  if (g_timing.load(std::memory_order_relaxed)) return 1;
+  if (!window_tc_supported(dp, dtype) || window_res_supported(dp, wh)) return 1;
+  static int forced = -1;
+  if (forced < 0) {
+    const char* e = std::getenv("TASKKV_GATHER_CHUNKS");
+    forced = e ? std::atoi(e) : 0;
+  }
+  int chunks = 1;
+  const int cap = forced > 0 ? forced : kMaxChunks;
+  while (chunks * 2 <= cap && chunks * 2 <= dp.R && (int64_t)(dp.R / (chunks * 2)) * dp.n_kv * wh.batch >= 32)
+    chunks *= 2;
+  return chunks;
+}
+
+// Steps a1-a5 for layers [l0, l0 + nl) of every sequence, one after the other on `s`.
+cudaError_t compress_layers(taskkv_cache* c, const WindowHostInfo& wh, int l0, int nl, cudaStream_t s) {
+  const DeviceProblem& dp = c->dp;
+  const int dtype = c->prm.dtype, B = c->prm.batch;
+  const UnitRange ur = layer_range(dp, B, l0, nl);
+  cudaError_t e = launch_budget(dp, B, l0, nl, s);
+  if (e == cudaSuccess) e = launch_window_scores(dp, dtype, c->hp.max_N, wh, s, l0, nl);
+  if (e == cudaSuccess) e = launch_select(dp, dtype, c->hp.max_N, s, &ur);
+  if (e == cudaSuccess) e = launch_separator_plan(dp, B, l0, nl, s);
+  const int64_t g0 = c->hp.gather_base[(size_t)l0 * B], g1 = c->hp.gather_base[(size_t)(l0 + nl) * B];
+  if (e == cudaSuccess) e = launch_gather(dp, dtype, B, l0, nl, g0, g1 - g0, s);
+  if (e == cudaSuccess && c->prm.mid_policy == TASKKV_MID_MEAN) e = launch_compensate(dp, dtype, ur, s);
+  return e;
+}
+
+// (1): window scores of chunk i+1 beside the selection of chunk i; then separator, plan and gather of everything.
+cudaError_t compress_window_select_overlapped(taskkv_cache* c, const WindowHostInfo& wh, int n_chunks, cudaStream_t s) {
+  const DeviceProblem& dp = c->dp;
+  const int dtype = c->prm.dtype, B = c->prm.batch, R = dp.R;
   std::lock_guard<std::mutex> lk(g_side_mu);
   SideStream* ss = side_stream();
-  if (!ss) {
-    cudaError_t e = launch_window_scores(dp, dtype, max_N, wh, s);
-    return e == cudaSuccess ? launch_select(dp, dtype, max_N, s) : e;
-  }
-  const int per_seq = dp.R * dp.n_kv;
-  cudaError_t e = cudaSuccess;
+  if (!ss) return compress_layers(c, wh, 0, R, s);
+  cudaError_t e = launch_budget(dp, B, 0, R, s);
   for (int ch = 0; ch < n_chunks && e == cudaSuccess; ++ch) {
-    const int l0 = (int)((int64_t)dp.R * ch / n_chunks), l1 = (int)((int64_t)dp.R * (ch + 1) / n_chunks);
+    const int l0 = (int)((int64_t)R * ch / n_chunks), l1 = (int)((int64_t)R * (ch + 1) / n_chunks);
     e = launch_window_scores_res(dp, wh, s, l0, l1 - l0);
     if (e == cudaSuccess) e = cudaEventRecord(ss->ev[ch], s);
     if (e == cudaSuccess) e = cudaStreamWaitEvent(ss->stream, ss->ev[ch], 0);
-    const UnitRange ur{l0 * dp.n_kv, (l1 - l0) * dp.n_kv, per_seq, wh.batch * (l1 - l0) * dp.n_kv};
-    if (e == cudaSuccess) e = launch_select(dp, dtype, max_N, ss->stream, &ur);
+    const UnitRange ur = layer_range(dp, B, l0, l1 - l0);
+    if (e == cudaSuccess) e = launch_select(dp, dtype, c->hp.max_N, ss->stream, &ur);
   }
   // always join, so that nothing of this call is left running on the side stream when the caller's stream moves on
   cudaError_t j = cudaEventRecord(ss->ev[kMaxChunks], ss->stream);
   if (j == cudaSuccess) j = cudaStreamWaitEvent(s, ss->ev[kMaxChunks], 0);
-  return e != cudaSuccess ? e : j;
+  if (e == cudaSuccess) e = j;
+  if (e == cudaSuccess) e = launch_separator_plan(dp, B, 0, R, s);
+  if (e == cudaSuccess) e = launch_gather(dp, dtype, B, 0, R, 0, c->hp.info.gather_items, s);
+  if (e == cudaSuccess && c->prm.mid_policy == TASKKV_MID_MEAN) e = launch_compensate(dp, dtype, layer_range(dp, B, 0, R), s);
+  return e;
+}
+
+// (2): window scores and selection of chunk i+1 (high-priority stream) beside separator, plan and gather of chunk i
+// (caller's stream).
+cudaError_t compress_gather_overlapped(taskkv_cache* c, const WindowHostInfo& wh, int n_chunks, cudaStream_t s) {
+  const DeviceProblem& dp = c->dp;
+  const int dtype = c->prm.dtype, B = c->prm.batch, R = dp.R;
+  std::lock_guard<std::mutex> lk(g_side_mu);
+  SideStream* ss = side_stream();
+  if (!ss) return compress_layers(c, wh, 0, R, s);
+  // fork: the library's stream starts after everything the caller's stream holds (table upload included)
+  cudaError_t e = cudaEventRecord(ss->ev[kMaxChunks + 1], s);
+  if (e == cudaSuccess) e = cudaStreamWaitEvent(ss->hi, ss->ev[kMaxChunks + 1], 0);
+  if (e != cudaSuccess) return e;
+  e = launch_budget(dp, B, 0, R, ss->hi);
+  int joined = -1;
+  for (int ch = 0; ch < n_chunks && e == cudaSuccess; ++ch) {
+    const int l0 = (int)((int64_t)R * ch / n_chunks), l1 = (int)((int64_t)R * (ch + 1) / n_chunks);
+    const UnitRange ur = layer_range(dp, B, l0, l1 - l0);
+    e = launch_window_scores(dp, dtype, c->hp.max_N, wh, ss->hi, l0, l1 - l0);
+    if (e == cudaSuccess) e = launch_select(dp, dtype, c->hp.max_N, ss->hi, &ur);
+    if (e == cudaSuccess) e = cudaEventRecord(ss->ev[ch], ss->hi);
+    if (e == cudaSuccess) e = cudaStreamWaitEvent(s, ss->ev[ch], 0);
+    if (e != cudaSuccess) break;
+    joined = ch;
+    e = launch_separator_plan(dp, B, l0, l1 - l0, s);
+    const int64_t g0 = c->hp.gather_base[(size_t)l0 * B], g1 = c->hp.gather_base[(size_t)l1 * B];
+    if (e == cudaSuccess) e = launch_gather(dp, dtype, B, l0, l1 - l0, g0, g1 - g0, s);
+    if (e == cudaSuccess && c->prm.mid_policy == TASKKV_MID_MEAN) e = launch_compensate(dp, dtype, ur, s);
+  }
+  // always join: nothing of this call may be left running on the library's stream when the caller's stream moves on
+  if (joined != n_chunks - 1) {
+    cudaError_t j = cudaEventRecord(ss->ev[kMaxChunks], ss->hi);
+    if (j == cudaSuccess) j = cudaStreamWaitEvent(s, ss->ev[kMaxChunks], 0);
+    if (e == cudaSuccess) e = j;
+  }
+  return e;
+}
+
+// Every layer of every sequence, in the order that suits the shape.
+cudaError_t compress_all(taskkv_cache* c, const WindowHostInfo& wh, cudaStream_t s) {
+  const int n1 = overlap_chunks(c->dp, c->prm.dtype, wh);
+  if (n1 > 1) return compress_window_select_overlapped(c, wh, n1, s);
+  const int n2 = gather_overlap_chunks(c->dp, c->prm.dtype, wh);
+  if (n2 > 1) return compress_gather_overlapped(c, wh, n2, s);
+  return compress_layers(c, wh, 0, c->dp.R, s);
 }
 }  // namespace
-
-struct taskkv_cache {
-  taskkv_params prm;
-  HostPlan hp;
-  DeviceProblem dp;
-  std::vector<unsigned char> meta;
-  void* cache_mem = nullptr;
-  void* work_mem = nullptr;
-  bool own_cache = false, own_work = false;
-  // staging for the host-buffer decode path
-  void* stage = nullptr;
-  size_t stage_bytes = 0;
-};
 
 namespace {
 
@@ -323,7 +465,11 @@ void fill_device_problem(taskkv_cache* c) {
   d.pool_rows = hp.info.pool_rows;
   d.max_items = hp.info.max_decode_items;
   d.unit_N = reinterpret_cast<const int32_t*>(cm + hp.o_unit_N);
-  d.unit_mid = reinterpret_cast<const int32_t*>(cm + hp.o_unit_mid);
+  d.unit_mid = reinterpret_cast<int32_t*>(cm + hp.o_unit_mid);
+  d.seg_base = reinterpret_cast<const int64_t*>(cm + hp.o_seg_base);
+  d.gather_base = reinterpret_cast<const int32_t*>(cm + hp.o_gbase);
+  d.dec_base = reinterpret_cast<const int32_t*>(cm + hp.o_dbase);
+  d.budget_frac = p.budget_frac;
   d.nhet = reinterpret_cast<const int32_t*>(cm + hp.o_nhet);
   d.c_off = reinterpret_cast<const int64_t*>(cm + hp.o_c_off);
   d.q_ptr = reinterpret_cast<const void* const*>(cm + hp.o_qp);
@@ -353,23 +499,21 @@ void fill_device_problem(taskkv_cache* c) {
   }
 }
 
-void build_meta(taskkv_cache* c, const void* const* q_win, const void* const* k, const void* const* v) {
+// Host copy of the tables at the head of the cache memory: everything but the per-unit input pointers.
+void fill_tables(taskkv_cache* c) {
   const taskkv_params& p = c->prm;
   const HostPlan& hp = c->hp;
   const int B = p.batch, R = p.n_layers, nkv = p.n_kv_heads;
-  const int G = p.n_heads / nkv;
-  const size_t es = p.dtype == TASKKV_F32 ? 4 : 2;
-  const size_t d = p.head_dim;
   c->meta.assign(hp.meta_bytes, 0);
   unsigned char* m = c->meta.data();
   int32_t* unit_N = reinterpret_cast<int32_t*>(m + hp.o_unit_N);
   int32_t* unit_mid = reinterpret_cast<int32_t*>(m + hp.o_unit_mid);
   int32_t* nhet = reinterpret_cast<int32_t*>(m + hp.o_nhet);
   int64_t* c_off = reinterpret_cast<int64_t*>(m + hp.o_c_off);
-  const void** qp = reinterpret_cast<const void**>(m + hp.o_qp);
-  const void** kp = reinterpret_cast<const void**>(m + hp.o_kp);
-  const void** vp = reinterpret_cast<const void**>(m + hp.o_vp);
   std::memcpy(nhet, hp.nhet.data(), hp.nhet.size() * 4);
+  std::memcpy(m + hp.o_seg_base, hp.seg_base.data(), hp.seg_base.size() * 8);
+  std::memcpy(m + hp.o_gbase, hp.gather_base.data(), hp.gather_base.size() * 4);
+  std::memcpy(m + hp.o_dbase, hp.dec_base.data(), hp.dec_base.size() * 4);
   int64_t coff = 0;
   size_t u = 0;
   for (int b = 0; b < B; ++b) {
@@ -377,16 +521,38 @@ void build_meta(taskkv_cache* c, const void* const* q_win, const void* const* k,
     for (int r = 0; r < R; ++r)
       for (int h = 0; h < nkv; ++h, ++u) {
         unit_N[u] = (int32_t)N;
-        unit_mid[u] = hp.mid[r];
+        unit_mid[u] = hp.mid[(size_t)b * R + r];
         c_off[u] = coff;
         coff += (int64_t)((N + 3) / 4 * 4);
-        qp[u] = static_cast<const unsigned char*>(q_win[b]) +
-                (((size_t)r * p.n_heads + (size_t)h * G) * p.window) * d * es;
-        kp[u] = static_cast<const unsigned char*>(k[b]) + (((size_t)r * nkv + h) * N) * d * es;
-        vp[u] = static_cast<const unsigned char*>(v[b]) + (((size_t)r * nkv + h) * N) * d * es;
       }
   }
   c_off[u] = coff;
+}
+
+// Per-unit input pointers of layers [layer0, layer0 + n_layers): q_win[b], k[b], v[b] point at layer layer0 of
+// sequence b ([n_layers][n][L][d] resp. [n_layers][n_kv][N_b][d], contiguous).
+void set_layer_pointers(taskkv_cache* c, int layer0, int n_layers, const void* const* q_win, const void* const* k,
+                        const void* const* v) {
+  const taskkv_params& p = c->prm;
+  const HostPlan& hp = c->hp;
+  const int B = p.batch, R = p.n_layers, nkv = p.n_kv_heads;
+  const int G = p.n_heads / nkv;
+  const size_t es = p.dtype == TASKKV_F32 ? 4 : 2;
+  const size_t d = p.head_dim;
+  unsigned char* m = c->meta.data();
+  const void** qp = reinterpret_cast<const void**>(m + hp.o_qp);
+  const void** kp = reinterpret_cast<const void**>(m + hp.o_kp);
+  const void** vp = reinterpret_cast<const void**>(m + hp.o_vp);
+  for (int b = 0; b < B; ++b) {
+    const size_t N = hp.seq_lens[b];
+    for (int i = 0; i < n_layers; ++i)
+      for (int h = 0; h < nkv; ++h) {
+        const size_t u = ((size_t)b * R + layer0 + i) * nkv + h;
+        qp[u] = static_cast<const unsigned char*>(q_win[b]) + (((size_t)i * p.n_heads + (size_t)h * G) * p.window) * d * es;
+        kp[u] = static_cast<const unsigned char*>(k[b]) + (((size_t)i * nkv + h) * N) * d * es;
+        vp[u] = static_cast<const unsigned char*>(v[b]) + (((size_t)i * nkv + h) * N) * d * es;
+      }
+  }
 }
 
 taskkv_status cuda_status(cudaError_t e) { return e == cudaSuccess ? TASKKV_OK : TASKKV_ECUDA; }
@@ -460,31 +626,21 @@ taskkv_status taskkv_compress_lse(const taskkv_params* p, const void* const* q_w
 }
 
 namespace {
-taskkv_status compress_impl(const taskkv_params* p, const void* const* q_win, const void* const* k,
-                            const void* const* v, const void* const* window_lse, void* cache_mem,
-                            size_t cache_bytes, void* workspace_mem, size_t workspace_bytes, taskkv_stream stream,
-                            taskkv_cache** out_cache) {
-  if (!p || !q_win || !k || !v || !out_cache) return TASKKV_EINVAL;
+// Plans the problem, takes or allocates the memory, and puts the tables and a clean state on the device (enqueued
+// on `s`); no layer is compressed yet.
+taskkv_status cache_create_impl(const taskkv_params* p, void* cache_mem, size_t cache_bytes, void* workspace_mem,
+                                size_t workspace_bytes, cudaStream_t s, taskkv_cache** out_cache) {
+  if (!p || !out_cache) return TASKKV_EINVAL;
   *out_cache = nullptr;
   taskkv_cache* c = new (std::nothrow) taskkv_cache();
   if (!c) return TASKKV_EALLOC;
   taskkv_status st = make_plan(p, c->hp);
   if (st != TASKKV_OK) { delete c; return st; }
-  for (int b = 0; b < p->batch; ++b) {
-    if (!q_win[b] || !k[b] || !v[b] || ((uintptr_t)q_win[b] | (uintptr_t)k[b] | (uintptr_t)v[b]) & 15) {
-      delete c;
-      return TASKKV_EINVAL;
-    }
-    if (window_lse && (!window_lse[b] || ((uintptr_t)window_lse[b] & 3))) {
-      delete c;
-      return TASKKV_EINVAL;
-    }
-  }
   c->prm = *p;
   c->prm.seq_lens = c->hp.seq_lens.data();
-  c->prm.mid_budget_per_layer = c->hp.mid.data();
+  c->prm.mid_budget_per_layer = nullptr;          // the per-(sequence, layer) budgets live in the plan
   c->prm.n_hetero = c->hp.nhet.data();
-  cudaStream_t s = static_cast<cudaStream_t>(stream);
+  c->layer_done.assign((size_t)p->n_layers, 0);
 
   if (cache_mem) {
     if (cache_bytes < (size_t)c->hp.info.cache_bytes || ((uintptr_t)cache_mem & (kAlign - 1))) {
@@ -517,38 +673,101 @@ taskkv_status compress_impl(const taskkv_params* p, const void* const* q_win, co
     c->own_work = true;
   }
   fill_device_problem(c);
-  build_meta(c, q_win, k, v);
-
+  fill_tables(c);
+  // the tables, then zeros over everything between them and the pools: status word, lengths, capacities, offsets,
+  // classes, work lists (a layer that has not been compressed yet has length 0 everywhere)
   cudaError_t e = cudaMemcpyAsync(c->cache_mem, c->meta.data(), c->hp.meta_bytes, cudaMemcpyHostToDevice, s);
-  if (e == cudaSuccess) e = cudaMemsetAsync(c->dp.status, 0, 64, s);
-  if (e == cudaSuccess) e = cudaMemsetAsync(c->dp.step_cnt, 0, (size_t)c->dp.U * 4, s);
-  WindowHostInfo wh;
-  wh.batch = p->batch;
-  wh.seq_lens = c->hp.seq_lens.data();
-  wh.q = q_win;
-  wh.k = k;
-  wh.lse = window_lse;
-  if (e == cudaSuccess) {
-    const int n_chunks = overlap_chunks(c->dp, p->dtype, wh);
-    if (n_chunks > 1) {
-      e = window_select_overlapped(c->dp, p->dtype, c->hp.max_N, wh, n_chunks, s);
-    } else {
-      e = launch_window_scores(c->dp, p->dtype, c->hp.max_N, wh, s);
-      if (e == cudaSuccess) e = launch_select(c->dp, p->dtype, c->hp.max_N, s);
-    }
-  }
-  if (e == cudaSuccess) e = launch_separator_plan(c->dp, p->batch * p->n_layers, s);
-  if (e == cudaSuccess) e = launch_gather(c->dp, p->dtype, c->hp.info.gather_items, s);
-  if (e == cudaSuccess && p->mid_policy == TASKKV_MID_MEAN) e = launch_compensate(c->dp, p->dtype, s);
+  if (e == cudaSuccess)
+    e = cudaMemsetAsync(static_cast<unsigned char*>(c->cache_mem) + c->hp.o_status, 0, c->hp.o_pacc - c->hp.o_status, s);
   if (e != cudaSuccess) {
-    std::fprintf(stderr, "taskkv_compress_ex: CUDA error: %s\n", cudaGetErrorString(e));
+    cudaGetLastError();
     taskkv_cache_destroy(c);
     return TASKKV_ECUDA;
   }
   *out_cache = c;
   return TASKKV_OK;
 }
+
+// Uploads the per-unit input pointer tables (three adjacent arrays of the table area).
+cudaError_t upload_pointers(taskkv_cache* c, cudaStream_t s) {
+  const HostPlan& hp = c->hp;
+  return cudaMemcpyAsync(static_cast<unsigned char*>(c->cache_mem) + hp.o_qp, c->meta.data() + hp.o_qp,
+                         hp.meta_bytes - hp.o_qp, cudaMemcpyHostToDevice, s);
+}
+
+bool pointers_ok(const taskkv_params* p, const void* const* q_win, const void* const* k, const void* const* v,
+                 const void* const* window_lse) {
+  for (int b = 0; b < p->batch; ++b) {
+    if (!q_win[b] || !k[b] || !v[b] || ((uintptr_t)q_win[b] | (uintptr_t)k[b] | (uintptr_t)v[b]) & 15) return false;
+    if (window_lse && (!window_lse[b] || ((uintptr_t)window_lse[b] & 3))) return false;
+  }
+  return true;
+}
+
+taskkv_status compress_impl(const taskkv_params* p, const void* const* q_win, const void* const* k,
+                            const void* const* v, const void* const* window_lse, void* cache_mem,
+                            size_t cache_bytes, void* workspace_mem, size_t workspace_bytes, taskkv_stream stream,
+                            taskkv_cache** out_cache) {
+  if (!p || !q_win || !k || !v || !out_cache) return TASKKV_EINVAL;
+  *out_cache = nullptr;
+  if (p->batch < 1 || !pointers_ok(p, q_win, k, v, window_lse)) return TASKKV_EINVAL;
+  cudaStream_t s = static_cast<cudaStream_t>(stream);
+  taskkv_cache* c = nullptr;
+  const taskkv_status st = cache_create_impl(p, cache_mem, cache_bytes, workspace_mem, workspace_bytes, s, &c);
+  if (st != TASKKV_OK) return st;
+  set_layer_pointers(c, 0, p->n_layers, q_win, k, v);
+  cudaError_t e = upload_pointers(c, s);
+  WindowHostInfo wh;
+  wh.batch = p->batch;
+  wh.seq_lens = c->hp.seq_lens.data();
+  wh.q = q_win;
+  wh.k = k;
+  wh.lse = window_lse;
+  wh.base_layer = 0;
+  if (e == cudaSuccess) e = compress_all(c, wh, s);
+  if (e != cudaSuccess) {
+    std::fprintf(stderr, "taskkv_compress_ex: CUDA error: %s\n", cudaGetErrorString(e));
+    cudaGetLastError();
+    taskkv_cache_destroy(c);
+    return TASKKV_ECUDA;
+  }
+  std::fill(c->layer_done.begin(), c->layer_done.end(), (unsigned char)1);
+  *out_cache = c;
+  return TASKKV_OK;
+}
 }  // namespace
+
+taskkv_status taskkv_cache_create(const taskkv_params* p, void* cache_mem, size_t cache_bytes, void* workspace_mem,
+                                  size_t workspace_bytes, taskkv_stream stream, taskkv_cache** out_cache) {
+  return cache_create_impl(p, cache_mem, cache_bytes, workspace_mem, workspace_bytes,
+                           static_cast<cudaStream_t>(stream), out_cache);
+}
+
+taskkv_status taskkv_compress_layer(taskkv_cache* c, int32_t layer, const void* const* q_win, const void* const* k,
+                                    const void* const* v, const void* const* window_lse, taskkv_stream stream) {
+  if (!c || !q_win || !k || !v) return TASKKV_EINVAL;
+  if (layer < 0 || layer >= c->prm.n_layers || !c->work_mem) return TASKKV_EINVAL;
+  if (!pointers_ok(&c->prm, q_win, k, v, window_lse)) return TASKKV_EINVAL;
+  if (c->layer_done[(size_t)layer]) return TASKKV_ESTATE;      // a layer's segments are written once
+  cudaStream_t s = static_cast<cudaStream_t>(stream);
+  set_layer_pointers(c, layer, 1, q_win, k, v);
+  cudaError_t e = upload_pointers(c, s);
+  WindowHostInfo wh;
+  wh.batch = c->prm.batch;
+  wh.seq_lens = c->hp.seq_lens.data();
+  wh.q = q_win;
+  wh.k = k;
+  wh.lse = window_lse;
+  wh.base_layer = layer;
+  if (e == cudaSuccess) e = compress_layers(c, wh, layer, 1, s);
+  if (e != cudaSuccess) {
+    std::fprintf(stderr, "taskkv_compress_layer: CUDA error: %s\n", cudaGetErrorString(e));
+    cudaGetLastError();
+    return TASKKV_ECUDA;
+  }
+  c->layer_done[(size_t)layer] = 1;
+  return TASKKV_OK;
+}
 
 taskkv_status taskkv_compress(const void* q_win, const void* k, const void* v, int32_t n_layers,
                               int32_t n_heads, int32_t n_kv_heads, int32_t head_dim, int32_t seq_len,
@@ -786,13 +1005,7 @@ int32_t taskkv_hetero_count(int32_t n, float beta, int32_t m, int32_t R, int32_t
 
 int32_t taskkv_mid_budget(double budget_tokens, int32_t N, int32_t h_full, int32_t n, int32_t sink,
                           int32_t recent) {
-  if (n <= h_full) return 0;
-  const double per_head = std::floor((budget_tokens - (double)N * (double)h_full) / (double)(n - h_full));
-  double k = per_head - (double)sink - (double)recent;
-  const double room = std::max(0, N - sink - recent);
-  if (k < 0) k = 0;
-  if (k > room) k = room;
-  return (int32_t)k;
+  return mid_budget_impl(budget_tokens, N, h_full, n, sink, recent);
 }
 
 int32_t taskkv_mid_budget_ex(double budget_tokens, int32_t N, int32_t f, int32_t n, int32_t sink, int32_t recent,

@@ -53,15 +53,23 @@ struct DeviceProblem {
   // n_kv + h stands for layer view_l0 + r'.  q, k_new, v_new, out and `lengths` are indexed by view unit.
   int32_t view_l0, view_nl, view_U;
   int32_t max_new;
+  float budget_frac;    // > 0: the middle budget follows Eq. 17 from this fraction of the full cache
   int32_t idx_stride;   // ints per unit in idx
   int32_t chunks_max;   // partial-statistic slots per unit (longest sequence)
   int64_t pool_rows;
   int64_t max_items;    // decode work items the scratch can hold
   // per unit tables
   const int32_t* unit_N;      // [U] sequence length
-  const int32_t* unit_mid;    // [U] middle budget k of the unit's layer
+  int32_t* unit_mid;          // [U] middle budget k of the unit's (sequence, layer): from the host's table, or
+                              // written by budget_kernel when the budget is given as a fraction (Eq. 17)
   const int32_t* nhet;        // [B*R] far heads per (sequence, layer)
   const int64_t* c_off;       // [U+1] offset of the unit's scores in C
+  // Where each (sequence, layer) block of n_kv units starts.  The number of full-cache heads of a block is fixed by
+  // Eq. 16 (only which heads is data dependent), so these are known on the host before any kernel runs, and a
+  // layer can be planned and gathered without the layers before it.
+  const int64_t* seg_base;    // [B*R+1] first pool row of block b * R + r
+  const int32_t* gather_base; // [R*B+1] first gather work item of block r * B + b (layer-major)
+  const int32_t* dec_base;    // [R*B+1] first decode work item of block r * B + b (layer-major)
   const void* const* q_ptr;   // [U] -> [rows][d]
   const void* const* k_ptr;   // [U] -> [N][d]
   const void* const* v_ptr;   // [U] -> [N][d]
@@ -74,8 +82,8 @@ struct DeviceProblem {
   float* dist;                // [U]
   float* sem;                 // [U][d]
   int32_t* idx;               // [U][idx_stride]
-  int32_t* gather_off;        // [U+1] gather work items
-  int32_t* dec_off;           // [U+1] decode work items
+  int32_t* gather_off;        // [U+1] gather work items, indexed layer-major like dec_off
+  int32_t* dec_off;           // [U+1] decode work items, indexed by w = (r * B + b) * n_kv + h
   int32_t* step_cnt;          // [U] combine blocks of a unit that finished the current fused step (0 between calls)
   void* k_pool;
   void* v_pool;
@@ -112,21 +120,30 @@ struct UnitRange {
 struct WindowHostInfo {
   int batch;
   const int32_t* seq_lens;      // host [batch]
-  const void* const* q;         // host [batch] device pointers: [R][n][L][d]
-  const void* const* k;         // host [batch] device pointers: [R][n_kv][N_b][d]
-  const void* const* lse;       // host [batch] device pointers to fp32 [R][n][L] natural-log normalisers of the
+  const void* const* q;         // host [batch] device pointers: [layers][n][L][d], first layer = base_layer
+  const void* const* k;         // host [batch] device pointers: [layers][n_kv][N_b][d], first layer = base_layer
+  const void* const* lse;       // host [batch] device pointers to fp32 [layers][n][L] natural-log normalisers of the
                                 // window rows, or nullptr: then pass 1 computes them
+  int base_layer = 0;           // the layer q[b], k[b], lse[b] point at (0: the tensors hold every layer; r: the
+                                // caller passed layer r alone)
 };
+
+// The units of layers [layer0, layer0 + n_layers) of every sequence.
+inline UnitRange layer_range(const DeviceProblem& p, int batch, int layer0, int n_layers) {
+  return UnitRange{layer0 * p.n_kv, n_layers * p.n_kv, p.R * p.n_kv, batch * n_layers * p.n_kv};
+}
 
 // Row statistics from caller-supplied normalisers (replaces pass 1): units [u0, u0 + n_units) of one sequence.
 cudaError_t launch_lse_to_stat(const DeviceProblem& p, int u0, int n_units, const float* lse, bool tensor_core_format,
                                cudaStream_t s);
 
-// kernel launchers (one per translation unit)
+// kernel launchers (one per translation unit).  Where a launcher takes (layer0, n_layers) it works on those layers
+// of every sequence; n_layers < 0 means all of them.
 cudaError_t launch_window_scores(const DeviceProblem& p, int dtype, int max_N, const WindowHostInfo& h,
-                                 cudaStream_t s);
+                                 cudaStream_t s, int layer0 = 0, int n_layers = -1);
 bool window_tc_supported(const DeviceProblem& p, int dtype);
-cudaError_t launch_window_scores_tc(const DeviceProblem& p, const WindowHostInfo& h, cudaStream_t s);
+cudaError_t launch_window_scores_tc(const DeviceProblem& p, const WindowHostInfo& h, cudaStream_t s, int layer0 = 0,
+                                    int n_layers = -1);
 cudaError_t launch_window_prefix(const DeviceProblem& p, const void* q, const void* k, int heads, int group, int N,
                                  cudaStream_t s);
 bool window_res_supported(const DeviceProblem& p, const WindowHostInfo& h);
@@ -135,9 +152,13 @@ cudaError_t launch_window_scores_res(const DeviceProblem& p, const WindowHostInf
                                      int n_layers = -1);
 cudaError_t launch_select(const DeviceProblem& p, int dtype, int max_N, cudaStream_t s,
                           const UnitRange* range = nullptr);
-cudaError_t launch_separator_plan(const DeviceProblem& p, int n_br, cudaStream_t s);
-cudaError_t launch_gather(const DeviceProblem& p, int dtype, int64_t gather_items, cudaStream_t s);
-cudaError_t launch_compensate(const DeviceProblem& p, int dtype, cudaStream_t s);
+cudaError_t launch_separator_plan(const DeviceProblem& p, int batch, int layer0, int n_layers, cudaStream_t s);
+// Eq. 17 on the device for the units of a range of layers (nothing to do unless budget_frac > 0)
+cudaError_t launch_budget(const DeviceProblem& p, int batch, int layer0, int n_layers, cudaStream_t s);
+// gather work items [item0, item0 + n_items) = those of layers [layer0, layer0 + n_layers) (layer-major numbering)
+cudaError_t launch_gather(const DeviceProblem& p, int dtype, int batch, int layer0, int n_layers, int64_t item0,
+                          int64_t n_items, cudaStream_t s);
+cudaError_t launch_compensate(const DeviceProblem& p, int dtype, const UnitRange& ur, cudaStream_t s);
 cudaError_t launch_append(const DeviceProblem& p, int dtype, const void* k_new, const void* v_new,
                           cudaStream_t s);
 cudaError_t launch_decode(const DeviceProblem& p, int dtype, const void* q, const int32_t* lengths,

@@ -41,8 +41,9 @@ __global__ void __launch_bounds__(kAttnThreads) decode_attn_kernel(DeviceProblem
   const int sg = lane / LPR, sl = lane % LPR;
   const int gsg = warp * RPW + sg;
   // the view's layers are a contiguous range of layer-major indices, hence of work items
-  const int w0 = p.view_l0 * lm_batch(p) * p.n_kv, w1 = w0 + p.view_U;
-  const int item0 = p.dec_off[w0], item1 = p.dec_off[w1];
+  const int w0 = p.view_l0 * lm_batch(p) * p.n_kv;
+  // (from the host's table of block starts: it does not depend on which layers have been compressed so far)
+  const int item0 = p.dec_base[p.view_l0 * lm_batch(p)], item1 = p.dec_base[(p.view_l0 + p.view_nl) * lm_batch(p)];
   const float scale2 = kLog2e * rsqrtf((float)D);
 
   for (int item = item0 + blockIdx.x; item < item1; item += gridDim.x) {
@@ -249,8 +250,9 @@ __global__ void __launch_bounds__(kAttnThreads) decode_attn_mma_kernel(DevicePro
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
   const int g = lane >> 2, t = lane & 3;
   // the view's layers are a contiguous range of layer-major indices, hence of work items
-  const int w0 = p.view_l0 * lm_batch(p) * p.n_kv, w1 = w0 + p.view_U;
-  const int item0 = p.dec_off[w0], item1 = p.dec_off[w1];
+  const int w0 = p.view_l0 * lm_batch(p) * p.n_kv;
+  // (from the host's table of block starts: it does not depend on which layers have been compressed so far)
+  const int item0 = p.dec_base[p.view_l0 * lm_batch(p)], item1 = p.dec_base[(p.view_l0 + p.view_nl) * lm_batch(p)];
   const float scale2 = kLog2e * rsqrtf((float)D);
   // d of accumulator row (mb, hf) of this lane's two output rows: e = hf * MB + mb, piece e / 8, element e % 8
   auto pd = [&](int mb, int hf, int gg) { const int e = hf * MB + mb; return (e >> 3) * 64 + gg * 8 + (e & 7); };

@@ -8,24 +8,34 @@ namespace taskkv {
 
 namespace {
 
-constexpr int kGatherThreads = 256;
+constexpr int kGatherThreads = 128;   // also the block size of the compensation kernel
 
 // One block copies kGatherRows consecutive segment rows of one unit, K and V.
+// Work items are numbered layer-major (gather_off[w], w = (r * B + b) * n_kv + h), so the items of layers
+// [layer0, layer0 + n_layers) are the contiguous range [item0, item0 + gridDim.x) and belong to the units
+// w0 .. w0 + wn - 1; only those entries of the table are read (later layers may not be planned yet).
+// 128 threads and at most 48 registers each: a block then fits beside a resident CTA of the window-score kernel
+// (which holds most of an SM's registers and shared memory but leaves HBM bandwidth unused), so that the gather of
+// one chunk of layers can run under the window scores of the next.  A block moves its 64 rows in rounds of
+// kGatherInFlight 16-byte loads per thread and array, all loads of a round issued before its stores.
+constexpr int kGatherInFlight = 4;
 template <int ROW_BYTES>
-__global__ void __launch_bounds__(kGatherThreads) gather_kernel(DeviceProblem p) {
+__global__ void __launch_bounds__(kGatherThreads, 10) gather_kernel(DeviceProblem p, int item0, int w0, int wn) {
   constexpr int VPR = ROW_BYTES / 16;                 // vectors (threads) per row
   constexpr int RPP = kGatherThreads / VPR;           // rows per pass
   constexpr int PASSES = kGatherRows / RPP;
-  __shared__ int s_unit;
+  constexpr int ROUND = PASSES < kGatherInFlight ? PASSES : kGatherInFlight;
+  static_assert(PASSES % ROUND == 0, "rows per block must be a whole number of rounds");
+  __shared__ int s_w;
   grid_dependency_wait();
-  const int item = blockIdx.x;
-  if (threadIdx.x == 0) s_unit = (item < p.gather_off[p.U]) ? upper_unit(p.gather_off, p.U, item) : -1;
+  const int item = item0 + (int)blockIdx.x;
+  if (threadIdx.x == 0) s_w = w0 + upper_unit(p.gather_off + w0, wn, item);
   __syncthreads();
-  const int u = s_unit;
-  if (u < 0) return;
+  const int w = s_w;
+  const int u = lm_unit(p, w).u;
   const int len = p.len[u];
   const int N = p.unit_N[u];
-  const int r0 = (item - p.gather_off[u]) * kGatherRows;
+  const int r0 = (item - p.gather_off[w]) * kGatherRows;
   const int64_t seg = p.seg_off[u];
   if (seg + len > p.pool_rows) return;                // planning overflow, already flagged
   const bool identity = (len == N);
@@ -36,23 +46,25 @@ __global__ void __launch_bounds__(kGatherThreads) gather_kernel(DeviceProblem p)
   unsigned char* vdst = static_cast<unsigned char*>(p.v_pool) + (size_t)seg * ROW_BYTES;
   const int rr = threadIdx.x / VPR, vc = threadIdx.x % VPR;
 
-  uint4 kreg[PASSES], vreg[PASSES];
+  for (int base = 0; base < PASSES; base += ROUND) {
+    uint4 kreg[ROUND], vreg[ROUND];
 #pragma unroll
-  for (int ps = 0; ps < PASSES; ++ps) {
-    const int r = r0 + ps * RPP + rr;
-    if (r < len) {
-      int src = identity ? r : idx[r];
-      src = min(max(src, 0), N - 1);
-      kreg[ps] = *reinterpret_cast<const uint4*>(ksrc + (size_t)src * ROW_BYTES + vc * 16);
-      vreg[ps] = *reinterpret_cast<const uint4*>(vsrc + (size_t)src * ROW_BYTES + vc * 16);
+    for (int ps = 0; ps < ROUND; ++ps) {
+      const int r = r0 + (base + ps) * RPP + rr;
+      if (r < len) {
+        int src = identity ? r : idx[r];
+        src = min(max(src, 0), N - 1);
+        kreg[ps] = *reinterpret_cast<const uint4*>(ksrc + (size_t)src * ROW_BYTES + vc * 16);
+        vreg[ps] = *reinterpret_cast<const uint4*>(vsrc + (size_t)src * ROW_BYTES + vc * 16);
+      }
     }
-  }
 #pragma unroll
-  for (int ps = 0; ps < PASSES; ++ps) {
-    const int r = r0 + ps * RPP + rr;
-    if (r < len) {
-      *reinterpret_cast<uint4*>(kdst + (size_t)r * ROW_BYTES + vc * 16) = kreg[ps];
-      *reinterpret_cast<uint4*>(vdst + (size_t)r * ROW_BYTES + vc * 16) = vreg[ps];
+    for (int ps = 0; ps < ROUND; ++ps) {
+      const int r = r0 + (base + ps) * RPP + rr;
+      if (r < len) {
+        *reinterpret_cast<uint4*>(kdst + (size_t)r * ROW_BYTES + vc * 16) = kreg[ps];
+        *reinterpret_cast<uint4*>(vdst + (size_t)r * ROW_BYTES + vc * 16) = vreg[ps];
+      }
     }
   }
 }
@@ -90,12 +102,12 @@ __global__ void __launch_bounds__(256) append_kernel(DeviceProblem p, const unsi
 // table).  One thread per 16-byte column of one compensation row adds the group's rows in position order in
 // fp32 and stores the mean in the cache's element type; K and V alike.  Runs after the gather.
 template <typename T, int D>
-__global__ void __launch_bounds__(kGatherThreads) compensate_kernel(DeviceProblem p) {
+__global__ void __launch_bounds__(kGatherThreads) compensate_kernel(DeviceProblem p, UnitRange ur) {
   constexpr int EPV = 16 / (int)sizeof(T);            // elements per 16-byte vector
   constexpr int VPR = D / EPV;                        // vectors (threads) per row
   constexpr int RPB = kGatherThreads / VPR;           // compensation rows per block
   constexpr int ROW_BYTES = D * (int)sizeof(T);
-  const int u = blockIdx.y;
+  const int u = ur.unit(blockIdx.y);
   const int N = p.unit_N[u], len = p.len[u];
   if (len == N) return;                               // the unit kept everything
   const int s1 = p.sink, s2 = p.recent;
@@ -133,34 +145,36 @@ __global__ void __launch_bounds__(kGatherThreads) compensate_kernel(DeviceProble
 }
 
 template <typename T, int D>
-cudaError_t launch_compensate_typed(const DeviceProblem& p, int max_rows, cudaStream_t s) {
+cudaError_t launch_compensate_typed(const DeviceProblem& p, int max_rows, const UnitRange& ur, cudaStream_t s) {
   constexpr int RPB = kGatherThreads / (D * (int)sizeof(T) / 16);
-  const dim3 grid((unsigned)((max_rows + RPB - 1) / RPB), (unsigned)p.U);
-  compensate_kernel<T, D><<<grid, kGatherThreads, 0, s>>>(p);
+  const dim3 grid((unsigned)((max_rows + RPB - 1) / RPB), (unsigned)ur.blocks);
+  compensate_kernel<T, D><<<grid, kGatherThreads, 0, s>>>(p, ur);
   return cudaGetLastError();
 }
 
 }  // namespace
 
-cudaError_t launch_compensate(const DeviceProblem& p, int dtype, cudaStream_t s) {
-  if (p.max_mid <= 0) return cudaSuccess;
+cudaError_t launch_compensate(const DeviceProblem& p, int dtype, const UnitRange& ur, cudaStream_t s) {
+  if (p.max_mid <= 0 || ur.blocks <= 0) return cudaSuccess;
   LaunchScope ls(K_COMPENSATE, s);
   if (dtype == TASKKV_F32)
-    return p.d == 64 ? launch_compensate_typed<float, 64>(p, p.max_mid, s)
-                     : launch_compensate_typed<float, 128>(p, p.max_mid, s);
-  return p.d == 64 ? launch_compensate_typed<__nv_bfloat16, 64>(p, p.max_mid, s)
-                   : launch_compensate_typed<__nv_bfloat16, 128>(p, p.max_mid, s);
+    return p.d == 64 ? launch_compensate_typed<float, 64>(p, p.max_mid, ur, s)
+                     : launch_compensate_typed<float, 128>(p, p.max_mid, ur, s);
+  return p.d == 64 ? launch_compensate_typed<__nv_bfloat16, 64>(p, p.max_mid, ur, s)
+                   : launch_compensate_typed<__nv_bfloat16, 128>(p, p.max_mid, ur, s);
 }
 
-cudaError_t launch_gather(const DeviceProblem& p, int dtype, int64_t gather_items, cudaStream_t s) {
-  if (gather_items <= 0) return cudaSuccess;
+cudaError_t launch_gather(const DeviceProblem& p, int dtype, int batch, int layer0, int n_layers, int64_t item0,
+                          int64_t n_items, cudaStream_t s) {
+  if (n_items <= 0) return cudaSuccess;
   LaunchScope ls(K_GATHER, s);
   const int row_bytes = p.d * (dtype == TASKKV_F32 ? 4 : 2);
-  const unsigned grid = (unsigned)gather_items;
+  const unsigned grid = (unsigned)n_items;
+  const int first = (int)item0, w0 = layer0 * batch * p.n_kv, wn = n_layers * batch * p.n_kv;
   switch (row_bytes) {
-    case 128: return launch_dependent(gather_kernel<128>, grid, (unsigned)kGatherThreads, s, p);
-    case 256: return launch_dependent(gather_kernel<256>, grid, (unsigned)kGatherThreads, s, p);
-    case 512: return launch_dependent(gather_kernel<512>, grid, (unsigned)kGatherThreads, s, p);
+    case 128: return launch_dependent(gather_kernel<128>, grid, (unsigned)kGatherThreads, s, p, first, w0, wn);
+    case 256: return launch_dependent(gather_kernel<256>, grid, (unsigned)kGatherThreads, s, p, first, w0, wn);
+    case 512: return launch_dependent(gather_kernel<512>, grid, (unsigned)kGatherThreads, s, p, first, w0, wn);
     default: return cudaErrorInvalidValue;
   }
 }

@@ -4,21 +4,25 @@
 //     from the center (Eq. 7), heads are ranked far -> near, the first f are
 //     heterogeneous (class 1) and the closest of the rest is promoted (class 2).
 //     n_kv * d values: done in double precision by one small block.
-//   plan: per unit the retained length (N for classes 1/2, sinks + recent +
-//     middle budget otherwise), the capacity, and exclusive scans that place the
-//     segments in the pools and number the gather / decode work items.
+//   plan: the same block then gives every unit of its (sequence, layer) the
+//     retained length (N for classes 1/2, sinks + recent + middle budget
+//     otherwise), the capacity, its place in the pools and its gather / decode
+//     work items.  Where the block starts in each of these is known on the host
+//     (Eq. 16 fixes how many heads keep everything), so blocks are independent:
+//     a layer is planned as soon as its own semantic vectors exist.
 #include "common.cuh"
 
 namespace taskkv {
 
 namespace {
 
-__global__ void __launch_bounds__(128) separator_kernel(DeviceProblem p) {
+__global__ void __launch_bounds__(128) separator_plan_kernel(DeviceProblem p, int layer0, int n_layers) {
   grid_dependency_wait();
   __shared__ double center[128];
   __shared__ double dist[TASKKV_MAX_KV_HEADS];
   __shared__ int cls[TASKKV_MAX_KV_HEADS];
-  const int br = blockIdx.x;               // b * R + r
+  const int b_seq = blockIdx.x / n_layers, r_lay = layer0 + blockIdx.x % n_layers;
+  const int br = b_seq * p.R + r_lay;
   const int n = p.n_kv, d = p.d;
   const int tid = threadIdx.x;
   const float* sem = p.sem + (size_t)br * n * d;
@@ -53,8 +57,9 @@ __global__ void __launch_bounds__(128) separator_kernel(DeviceProblem p) {
     cls[tid] = rank < f ? TASKKV_CLASS_HETERO : TASKKV_CLASS_NON_HETERO;
   }
   __syncthreads();
+  int c = TASKKV_CLASS_NON_HETERO;
   if (tid < n) {
-    int c = cls[tid];
+    c = cls[tid];
     if (promote && c == TASKKV_CLASS_NON_HETERO) {
       const double me = dist[tid];
       int nearer = 0;
@@ -65,102 +70,95 @@ __global__ void __launch_bounds__(128) separator_kernel(DeviceProblem p) {
     p.cls[(size_t)br * n + tid] = c;
     p.dist[(size_t)br * n + tid] = (float)dist[tid];
   }
+  __syncthreads();                 // every thread has read the far / not-far marks
+  if (tid < n) cls[tid] = c;
+  __syncthreads();
+
+  // ---- plan of this block's units
+  __shared__ int s_cap[TASKKV_MAX_KV_HEADS], s_git[TASKKV_MAX_KV_HEADS], s_dit[TASKKV_MAX_KV_HEADS];
+  const int B = lm_batch(p);
+  const int lm_block = r_lay * B + b_seq;
+  int len = 0;
+  if (tid < n) {
+    const int u = br * n + tid;
+    const int N = p.unit_N[u];
+    len = N;
+    if (cls[tid] == TASKKV_CLASS_NON_HETERO && N > p.sink + p.recent)
+      len = p.sink + p.recent + min(p.unit_mid[u], N - p.sink - p.recent);
+    const int cap = len + p.max_new;
+    p.len[u] = len;
+    p.cap[u] = cap;
+    s_cap[tid] = cap;
+    s_git[tid] = (len + kGatherRows - 1) / kGatherRows;
+    s_dit[tid] = (cap + kDecodeChunk - 1) / kDecodeChunk;
+  }
+  __syncthreads();
+  if (tid < n) {
+    int64_t rows_before = 0;
+    int git_before = 0, dit_before = 0;
+    for (int h = 0; h < tid; ++h) { rows_before += s_cap[h]; git_before += s_git[h]; dit_before += s_dit[h]; }
+    const int u = br * n + tid, w = lm_block * n + tid;
+    p.seg_off[u] = p.seg_base[br] + rows_before;
+    p.gather_off[w] = p.gather_base[lm_block] + git_before;
+    p.dec_off[w] = p.dec_base[lm_block] + dit_before;
+    if (tid == n - 1) {
+      // the block must end exactly where the host placed the next one
+      const bool fits = p.seg_base[br] + rows_before + s_cap[tid] == p.seg_base[br + 1] &&
+                        p.gather_base[lm_block] + git_before + s_git[tid] == p.gather_base[lm_block + 1] &&
+                        p.dec_base[lm_block] + dit_before + s_dit[tid] == p.dec_base[lm_block + 1];
+      if (!fits) set_status(p.status, TASKKV_ESTATE);
+      if (br == B * p.R - 1) p.seg_off[p.U] = p.seg_base[br + 1];
+      if (lm_block == B * p.R - 1) {
+        p.gather_off[p.U] = p.gather_base[lm_block + 1];
+        p.dec_off[p.U] = p.dec_base[lm_block + 1];
+      }
+    }
+  }
 }
 
-constexpr int kPlanThreads = 1024;
-
-// Block-wide exclusive scan of one int64 per thread; the block total is left in
-// *total (shared) until the next call.
-__device__ int64_t block_excl_scan(int64_t v, int64_t* warp_tot, int64_t* total) {
-  const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
-  int64_t incl = v;
-#pragma unroll
-  for (int o = 1; o < 32; o <<= 1) {
-    const int64_t y = __shfl_up_sync(0xffffffffu, incl, o);
-    if (lane >= o) incl += y;
+// Eq. 17 with the budget given as a fraction of the full cache: k = floor((B - N h) / (n - h)) - s1 - s2 with
+// B = fraction * n * N token-heads and h the heads of the block that keep everything (Eq. 16's f plus the promoted
+// one), clamped to [0, N - s1 - s2].  Every operation is rounded on its own (no fused multiply-add), so the host's
+// plan, which sizes the pools from the same formula, gets the same integer.
+__global__ void __launch_bounds__(128) budget_kernel(DeviceProblem p, UnitRange ur) {
+  const int i = blockIdx.x * blockDim.x + threadIdx.x;
+  if (i >= ur.blocks) return;
+  const int u = ur.unit(i);
+  const int n = p.n_kv, br = u / n;
+  const int N = p.unit_N[u];
+  int f = max(0, min(p.nhet[br], n));
+  int h = min(n, f + ((p.promote_center && f < n) ? 1 : 0));
+  if (p.force_class == 1) h = n;
+  if (p.force_class == 0) h = 0;
+  int k = 0;
+  if (n > h) {
+    const double budget = __dmul_rn(__dmul_rn((double)p.budget_frac, (double)n), (double)N);
+    const double per_head = floor(__ddiv_rn(__dsub_rn(budget, __dmul_rn((double)N, (double)h)), (double)(n - h)));
+    double kk = per_head - (double)p.sink - (double)p.recent;
+    const double room = (double)max(0, N - p.sink - p.recent);
+    kk = kk < 0.0 ? 0.0 : kk;
+    kk = kk > room ? room : kk;
+    k = (int)kk;
   }
-  __syncthreads();                 // readers of the previous call's warp_tot / total are done
-  if (lane == 31) warp_tot[warp] = incl;
-  __syncthreads();
-  if (warp == 0) {
-    const int64_t w = warp_tot[lane];
-    int64_t wi = w;
-#pragma unroll
-    for (int o = 1; o < 32; o <<= 1) {
-      const int64_t y = __shfl_up_sync(0xffffffffu, wi, o);
-      if (lane >= o) wi += y;
-    }
-    warp_tot[lane] = wi - w;
-    if (lane == 31) *total = wi;
-  }
-  __syncthreads();
-  return incl - v + warp_tot[warp];
-}
-
-__global__ void __launch_bounds__(kPlanThreads) plan_kernel(DeviceProblem p) {
-  grid_dependency_wait();
-  __shared__ int64_t warp_tot[32];
-  __shared__ int64_t total;
-  int64_t run_rows = 0, run_gather = 0;
-  const int tid = threadIdx.x;
-  for (int base = 0; base < p.U; base += kPlanThreads) {
-    const int u = base + tid;
-    int len = 0, cap = 0;
-    if (u < p.U) {
-      const int N = p.unit_N[u];
-      len = N;
-      if (p.cls[u] == TASKKV_CLASS_NON_HETERO && N > p.sink + p.recent)
-        len = p.sink + p.recent + min(p.unit_mid[u], N - p.sink - p.recent);
-      cap = len + p.max_new;
-      p.len[u] = len;
-      p.cap[u] = cap;
-    }
-    const int64_t ro = block_excl_scan(cap, warp_tot, &total);
-    const int64_t tot_rows = total;
-    const int64_t go = block_excl_scan((len + kGatherRows - 1) / kGatherRows, warp_tot, &total);
-    const int64_t tot_gather = total;
-    if (u < p.U) {
-      p.seg_off[u] = run_rows + ro;
-      p.gather_off[u] = (int32_t)(run_gather + go);
-    }
-    run_rows += tot_rows;
-    run_gather += tot_gather;
-  }
-  if (tid == 0) {
-    p.seg_off[p.U] = run_rows;
-    p.gather_off[p.U] = (int32_t)run_gather;
-    if (run_rows > p.pool_rows) set_status(p.status, TASKKV_ESTATE);
-  }
-  // decode work items: ceil(capacity / kDecodeChunk) per unit, numbered in layer-major order
-  __syncthreads();
-  int64_t run_items = 0;
-  for (int base = 0; base < p.U; base += kPlanThreads) {
-    const int w = base + tid;
-    const int items = (w < p.U) ? (p.cap[lm_unit(p, w).u] + kDecodeChunk - 1) / kDecodeChunk : 0;
-    const int64_t o = block_excl_scan(items, warp_tot, &total);
-    if (w < p.U) p.dec_off[w] = (int32_t)(run_items + o);
-    run_items += total;
-  }
-  if (tid == 0) {
-    p.dec_off[p.U] = (int32_t)min(run_items, p.max_items);
-    if (run_items > p.max_items) set_status(p.status, TASKKV_ESTATE);
-  }
+  p.unit_mid[u] = k;
 }
 
 }  // namespace
 
-cudaError_t launch_separator_plan(const DeviceProblem& p, int n_br, cudaStream_t s) {
-  cudaError_t e;
-  {
-    LaunchScope ls(K_SEPARATOR, s);
-    e = launch_dependent(separator_kernel, (unsigned)n_br, 128u, s, p);
-  }
-  if (e != cudaSuccess) return e;
-  {
-    LaunchScope ls(K_PLAN, s);
-    e = launch_dependent(plan_kernel, 1u, (unsigned)kPlanThreads, s, p);
-  }
-  return e;
+cudaError_t launch_budget(const DeviceProblem& p, int batch, int layer0, int n_layers, cudaStream_t s) {
+  if (!(p.budget_frac > 0.f)) return cudaSuccess;
+  if (n_layers < 0) { layer0 = 0; n_layers = p.R; }
+  const UnitRange ur = layer_range(p, batch, layer0, n_layers);
+  if (ur.blocks <= 0) return cudaSuccess;
+  LaunchScope ls(K_PLAN, s);
+  budget_kernel<<<(ur.blocks + 127) / 128, 128, 0, s>>>(p, ur);
+  return cudaGetLastError();
+}
+
+cudaError_t launch_separator_plan(const DeviceProblem& p, int batch, int layer0, int n_layers, cudaStream_t s) {
+  if (n_layers < 0) { layer0 = 0; n_layers = p.R; }
+  LaunchScope ls(K_SEPARATOR, s);
+  return launch_dependent(separator_plan_kernel, (unsigned)(batch * n_layers), 128u, s, p, layer0, n_layers);
 }
 
 }  // namespace taskkv

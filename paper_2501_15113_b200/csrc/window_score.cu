@@ -23,8 +23,8 @@ struct WinSmem {
 };
 
 template <typename T, int D, int PASS>
-__global__ void __launch_bounds__(kTile) window_pass_kernel(DeviceProblem p) {
-  const int u = blockIdx.y;
+__global__ void __launch_bounds__(kTile) window_pass_kernel(DeviceProblem p, UnitRange ur) {
+  const int u = ur.unit(blockIdx.y);
   const int N = p.unit_N[u];
   const int key0 = blockIdx.x * kScoreChunk;
   if (key0 >= N) return;
@@ -136,8 +136,8 @@ __global__ void __launch_bounds__(kTile) window_pass_kernel(DeviceProblem p) {
 }
 
 // Combine the chunk partials of one unit: (max, sum) -> (max, 1/sum) per window row.
-__global__ void window_reduce_kernel(DeviceProblem p) {
-  const int u = blockIdx.x;
+__global__ void window_reduce_kernel(DeviceProblem p, UnitRange ur) {
+  const int u = ur.unit(blockIdx.x);
   const int row = threadIdx.x;
   if (row >= p.rows_pad) return;
   const int N = p.unit_N[u];
@@ -168,7 +168,8 @@ __global__ void lse_to_stat_kernel(DeviceProblem p, int u0, const float* __restr
 }
 
 template <typename T, int D>
-cudaError_t launch_generic(const DeviceProblem& p, int max_N, const WindowHostInfo& h, cudaStream_t s) {
+cudaError_t launch_generic(const DeviceProblem& p, int max_N, const WindowHostInfo& h, cudaStream_t s, int layer0,
+                           int n_layers) {
   const size_t smem = (size_t)p.rows_pad * D * sizeof(float) + (size_t)kTile * WinSmem<T, D>::kRowBytes +
                       (size_t)p.rows_pad * 4 * sizeof(float2);
   cudaError_t e;
@@ -176,26 +177,28 @@ cudaError_t launch_generic(const DeviceProblem& p, int max_N, const WindowHostIn
   if (e != cudaSuccess) return e;
   e = cudaFuncSetAttribute(window_pass_kernel<T, D, 2>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
   if (e != cudaSuccess) return e;
-  const dim3 grid((max_N + kScoreChunk - 1) / kScoreChunk, p.U);
+  const UnitRange ur = layer_range(p, h.batch, layer0, n_layers);
+  const dim3 grid((max_N + kScoreChunk - 1) / kScoreChunk, ur.blocks);
   if (h.lse) {
     const int per_seq = p.R * p.n_kv;
+    const size_t lse_skip = (size_t)(layer0 - h.base_layer) * p.n_heads * p.L;
     for (int b = 0; b < h.batch; ++b) {
-      e = launch_lse_to_stat(p, b * per_seq, per_seq, static_cast<const float*>(h.lse[b]), false, s);
+      e = launch_lse_to_stat(p, b * per_seq + ur.first, ur.count, static_cast<const float*>(h.lse[b]) + lse_skip, false, s);
       if (e != cudaSuccess) return e;
     }
   } else {
     {
       LaunchScope ls(K_WINDOW_STATS, s);
-      window_pass_kernel<T, D, 1><<<grid, kTile, smem, s>>>(p);
+      window_pass_kernel<T, D, 1><<<grid, kTile, smem, s>>>(p, ur);
     }
     {
       LaunchScope ls(K_WINDOW_REDUCE, s);
-      window_reduce_kernel<<<p.U, p.rows_pad, 0, s>>>(p);
+      window_reduce_kernel<<<ur.blocks, p.rows_pad, 0, s>>>(p, ur);
     }
   }
   {
     LaunchScope ls(K_WINDOW_SCORES, s);
-    window_pass_kernel<T, D, 2><<<grid, kTile, smem, s>>>(p);
+    window_pass_kernel<T, D, 2><<<grid, kTile, smem, s>>>(p, ur);
   }
   return cudaGetLastError();
 }
@@ -210,14 +213,16 @@ cudaError_t launch_lse_to_stat(const DeviceProblem& p, int u0, int n_units, cons
 }
 
 cudaError_t launch_window_scores(const DeviceProblem& p, int dtype, int max_N, const WindowHostInfo& h,
-                                 cudaStream_t s) {
+                                 cudaStream_t s, int layer0, int n_layers) {
+  if (n_layers < 0) { layer0 = 0; n_layers = p.R; }
   // bf16 with 32 / 64 / 128 window rows runs on the tensor cores; everything else here
-  if (window_tc_supported(p, dtype)) return launch_window_scores_tc(p, h, s);
+  if (window_tc_supported(p, dtype)) return launch_window_scores_tc(p, h, s, layer0, n_layers);
   if (dtype == TASKKV_F32) {
-    return p.d == 64 ? launch_generic<float, 64>(p, max_N, h, s) : launch_generic<float, 128>(p, max_N, h, s);
+    return p.d == 64 ? launch_generic<float, 64>(p, max_N, h, s, layer0, n_layers)
+                     : launch_generic<float, 128>(p, max_N, h, s, layer0, n_layers);
   }
-  return p.d == 64 ? launch_generic<__nv_bfloat16, 64>(p, max_N, h, s)
-                   : launch_generic<__nv_bfloat16, 128>(p, max_N, h, s);
+  return p.d == 64 ? launch_generic<__nv_bfloat16, 64>(p, max_N, h, s, layer0, n_layers)
+                   : launch_generic<__nv_bfloat16, 128>(p, max_N, h, s, layer0, n_layers);
 }
 
 }  // namespace taskkv

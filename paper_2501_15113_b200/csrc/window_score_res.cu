@@ -547,8 +547,10 @@ cudaError_t launch_res_d(const DeviceProblem& p, const WindowHostInfo& h, cudaSt
           maps.k[i] = maps.k[0];
           maps.q[i] = maps.q[0];
         } else {
-          const char* kb = static_cast<const char*>(h.k[b]) + (size_t)first * (size_t)N * D * sizeof(__nv_bfloat16);
-          const char* qb = static_cast<const char*>(h.q[b]) + (size_t)first * kRows * D * sizeof(__nv_bfloat16);
+          // h.k[b], h.q[b] point at layer h.base_layer
+          const size_t skip = (size_t)(first - h.base_layer * p.n_kv);
+          const char* kb = static_cast<const char*>(h.k[b]) + skip * (size_t)N * D * sizeof(__nv_bfloat16);
+          const char* qb = static_cast<const char*>(h.q[b]) + skip * kRows * D * sizeof(__nv_bfloat16);
           if (!make_tensor_map_2d(&maps.k[i], kb, D, (uint64_t)per_seq * (uint64_t)N, kTile)) return cudaErrorUnknown;
           if (!make_tensor_map_2d(&maps.q[i], qb, D, (uint64_t)per_seq * (uint64_t)kRows, kRows))
             return cudaErrorUnknown;

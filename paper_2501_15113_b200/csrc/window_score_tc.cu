@@ -534,9 +534,9 @@ window_tc_kernel(const __grid_constant__ TcMaps maps, DeviceProblem p, const __g
 
 // Folds the partial statistics of one unit: slots (item, warp) of pass 1 -> one offset per row.
 // One warp per (unit, row): lanes take every 32nd slot, then a shuffle tree; the order is fixed.
-__global__ void __launch_bounds__(128) window_tc_reduce_kernel(DeviceProblem p, int u0, int chunk_keys, int parts,
-                                                               int n_real) {
-  const int u = u0 + blockIdx.x;
+__global__ void __launch_bounds__(128) window_tc_reduce_kernel(DeviceProblem p, UnitRange ur, int chunk_keys,
+                                                               int parts, int n_real) {
+  const int u = ur.unit(blockIdx.x);
   const int slots = (p.unit_N[u] + chunk_keys - 1) / chunk_keys * parts;
   const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
   const float2* part = reinterpret_cast<const float2*>(p.stat_part) + (size_t)u * p.chunks_max * p.rows_pad;
@@ -577,7 +577,7 @@ inline int pick_chunk(int64_t units_times_keys, int n_sm) {
 }
 
 template <int D>
-cudaError_t launch_tc_d(const DeviceProblem& p, const WindowHostInfo& h, cudaStream_t s) {
+cudaError_t launch_tc_d(const DeviceProblem& p, const WindowHostInfo& h, cudaStream_t s, int layer0, int n_layers) {
   static int n_sm = 0;
   if (n_sm == 0) {
     int dev = 0;
@@ -590,7 +590,11 @@ cudaError_t launch_tc_d(const DeviceProblem& p, const WindowHostInfo& h, cudaStr
   const int smem = lay.total;
   cudaError_t e = cudaFuncSetAttribute(window_tc_kernel<D>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem);
   if (e != cudaSuccess) return e;
-  const int per_seq = p.R * p.n_kv;
+  const int per_seq_all = p.R * p.n_kv;
+  const int first = layer0 * p.n_kv;               // the launch covers units [first, first + per_seq) of every sequence
+  const int per_seq = n_layers * p.n_kv;
+  const int skip = (layer0 - h.base_layer) * p.n_kv;   // units between what h.q / h.k point at and the first one
+  if (per_seq <= 0) return cudaSuccess;
   const int parts = p.rows == 128 ? 2 : kTcParts;
   // up to kMaxSeq sequences per pair of launches
   for (int b0 = 0; b0 < h.batch; b0 += kMaxSeq) {
@@ -612,11 +616,13 @@ cudaError_t launch_tc_d(const DeviceProblem& p, const WindowHostInfo& h, cudaStr
         maps.k[i] = maps.k[0];
         maps.q[i] = maps.q[0];
       } else {
-        if (!make_tensor_map_2d(&maps.k[i], h.k[b], D, (uint64_t)per_seq * (uint64_t)N, kTile)) return cudaErrorUnknown;
-        if (!make_tensor_map_2d(&maps.q[i], h.q[b], D, (uint64_t)per_seq * (uint64_t)p.rows, p.rows))
+        const char* kb = static_cast<const char*>(h.k[b]) + (size_t)skip * (size_t)N * D * sizeof(__nv_bfloat16);
+        const char* qb = static_cast<const char*>(h.q[b]) + (size_t)skip * p.rows * D * sizeof(__nv_bfloat16);
+        if (!make_tensor_map_2d(&maps.k[i], kb, D, (uint64_t)per_seq * (uint64_t)N, kTile)) return cudaErrorUnknown;
+        if (!make_tensor_map_2d(&maps.q[i], qb, D, (uint64_t)per_seq * (uint64_t)p.rows, p.rows))
           return cudaErrorUnknown;
       }
-      a.u0[i] = b * per_seq;
+      a.u0[i] = b * per_seq_all + first;
       a.N[i] = N;
       a.chunks[i] = (N + a.chunk_keys - 1) / a.chunk_keys;
       a.item_off[i + 1] = a.item_off[i] + (i < nb ? per_seq * a.chunks[i] : 0);
@@ -626,8 +632,10 @@ cudaError_t launch_tc_d(const DeviceProblem& p, const WindowHostInfo& h, cudaStr
     a.steps = (n1 + grid - 1) / grid;
     if (h.lse) {
       // the caller already has the rows' normalisers: no pass 1
+      const size_t lse_skip = (size_t)(layer0 - h.base_layer) * p.n_heads * p.L;
       for (int i = 0; i < nb; ++i) {
-        e = launch_lse_to_stat(p, (b0 + i) * per_seq, per_seq, static_cast<const float*>(h.lse[b0 + i]), true, s);
+        e = launch_lse_to_stat(p, (b0 + i) * per_seq_all + first, per_seq,
+                               static_cast<const float*>(h.lse[b0 + i]) + lse_skip, true, s);
         if (e != cudaSuccess) return e;
       }
     } else {
@@ -638,7 +646,8 @@ cudaError_t launch_tc_d(const DeviceProblem& p, const WindowHostInfo& h, cudaStr
       }
       {
         LaunchScope ls(K_WINDOW_REDUCE, s);
-        window_tc_reduce_kernel<<<dim3(nb * per_seq, (p.rows + 3) / 4), 128, 0, s>>>(p, b0 * per_seq, a.chunk_keys, parts, 0);
+        const UnitRange ur{b0 * per_seq_all + first, per_seq, per_seq_all, nb * per_seq};
+        window_tc_reduce_kernel<<<dim3(nb * per_seq, (p.rows + 3) / 4), 128, 0, s>>>(p, ur, a.chunk_keys, parts, 0);
       }
     }
     a.pass = 2;
@@ -697,7 +706,8 @@ cudaError_t launch_prefix_d(const DeviceProblem& p, const void* q, const void* k
   }
   {
     LaunchScope ls(K_WINDOW_REDUCE, s);
-    window_tc_reduce_kernel<<<dim3(a.n_local, (p.rows + 3) / 4), 128, 0, s>>>(p, 0, a.chunk_keys, 2, N);
+    const UnitRange ur{0, a.n_local, a.n_local, a.n_local};
+    window_tc_reduce_kernel<<<dim3(a.n_local, (p.rows + 3) / 4), 128, 0, s>>>(p, ur, a.chunk_keys, 2, N);
   }
   a.pass = 2;
   {
@@ -719,10 +729,12 @@ cudaError_t launch_window_prefix(const DeviceProblem& p, const void* q, const vo
   return p.d == 64 ? launch_prefix_d<64>(p, q, k, heads, group, N, s) : launch_prefix_d<128>(p, q, k, heads, group, N, s);
 }
 
-cudaError_t launch_window_scores_tc(const DeviceProblem& p, const WindowHostInfo& h, cudaStream_t s) {
+cudaError_t launch_window_scores_tc(const DeviceProblem& p, const WindowHostInfo& h, cudaStream_t s, int layer0,
+                                    int n_layers) {
+  if (n_layers < 0) { layer0 = 0; n_layers = p.R; }
   // 32 window rows and sequences short enough for a unit's scores to stay in tensor memory: K is read once
-  if (window_res_supported(p, h)) return launch_window_scores_res(p, h, s);
-  return p.d == 64 ? launch_tc_d<64>(p, h, s) : launch_tc_d<128>(p, h, s);
+  if (window_res_supported(p, h)) return launch_window_scores_res(p, h, s, layer0, n_layers);
+  return p.d == 64 ? launch_tc_d<64>(p, h, s, layer0, n_layers) : launch_tc_d<128>(p, h, s, layer0, n_layers);
 }
 
 }  // namespace taskkv

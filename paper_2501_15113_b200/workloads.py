@@ -53,6 +53,8 @@ class Workload:
     heavy_keys: int = 0             # keys per head, at seeded positions, scaled by heavy_scale ("heavy hitters")
     heavy_scale: float = 1.0
     note: str = ""
+    mid_by_seq: Optional[List[List[int]]] = None   # [batch][layer]: overrides mid_budget where budgets differ by sequence
+    budget_frac: float = 0.0        # > 0: the library derives the budgets itself (Eq. 17) from this fraction
 
     @property
     def group(self) -> int:
@@ -70,12 +72,16 @@ class Workload:
         f = self.n_hetero[b][r]
         return min(self.n_kv_heads, f + (1 if self.promote_center and f < self.n_kv_heads else 0))
 
+    def mid_of(self, b: int, r: int) -> int:
+        """Middle budget of (sequence, layer)."""
+        return self.mid_by_seq[b][r] if self.mid_by_seq is not None else self.mid_budget[r]
+
     def kept_len(self, b: int, r: int) -> int:
         """Rows a non-full head keeps after compression (before any append)."""
         N = self.seq_lens[b]
         if N <= self.sink + self.recent:
             return N
-        return self.sink + self.recent + min(self.mid_budget[r], N - self.sink - self.recent)
+        return self.sink + self.recent + min(self.mid_of(b, r), N - self.sink - self.recent)
 
     def retained_rows(self) -> int:
         tot = 0

@@ -99,7 +99,7 @@ def check_selection(got: np.ndarray, want: np.ndarray, score: np.ndarray, what: 
 
 def oracle_layer(wl: W.Workload, b: int, r: int, q, k, v, force_class: int = -1) -> Dict:
     return O.compress_layer(to64(q), to64(k), to64(v), n_hetero=wl.n_hetero[b][r], sink=wl.sink,
-                            recent=wl.recent, mid=wl.mid_budget[r], top_t=wl.top_t,
+                            recent=wl.recent, mid=wl.mid_of(b, r), top_t=wl.top_t,
                             pool_kernel=wl.pool_kernel, promote_center=wl.promote_center,
                             force_class=force_class)
 
@@ -225,7 +225,7 @@ def compare_layer(cache: tk.Cache, wl: W.Workload, b: int, r: int, ref: Dict, re
     for h in range(nkv):
         u = u0 + h
         want = ref["idx"][h] if int(want_cls[h]) == int(ref["cls"][h]) else \
-            O.retained_indices(int(want_cls[h]), ref["C"][h], wl.sink, wl.recent, wl.mid_budget[r], wl.pool_kernel)
+            O.retained_indices(int(want_cls[h]), ref["C"][h], wl.sink, wl.recent, wl.mid_of(b, r), wl.pool_kernel)
         out_idx.append(want)
         if h in skip:
             continue

@@ -524,13 +524,13 @@ def test_compensation_policies(case, policy):
         for r in range(wl.n_layers):
             k64, v64 = P.to64(ks[b][r]), P.to64(vs[b][r])
             ref = O.compress_layer(P.to64(qs[b][r]), k64, v64, n_hetero=wl.n_hetero[b][r], sink=wl.sink,
-                                   recent=wl.recent, mid=wl.mid_budget[r], top_t=wl.top_t,
+                                   recent=wl.recent, mid=wl.mid_of(b, r), top_t=wl.top_t,
                                    pool_kernel=wl.pool_kernel, promote_center=wl.promote_center, mid_policy=policy)
             u0 = P.unit_index(wl, b, r, 0)
             assert cls[u0:u0 + wl.n_kv_heads].tolist() == ref["cls"].tolist()
             assert lens[u0:u0 + wl.n_kv_heads].tolist() == ref["len"].tolist()
             kc, vc = O.gather_cache_policy(k64, v64, ref["cls"], ref["idx"], mid_policy=policy, sink=wl.sink,
-                                           recent=wl.recent, mid=wl.mid_budget[r], dtype=wl.dtype)
+                                           recent=wl.recent, mid=wl.mid_of(b, r), dtype=wl.dtype)
             for h in range(wl.n_kv_heads):
                 u = u0 + h
                 if len(ref["idx"][h]) < N:      # positions (group starts for the averaged rows) are exact
@@ -603,8 +603,8 @@ def test_layer_by_layer_decode_equals_all_layer_decode(case):
     split.close()
 
 
-def test_layer_streamed_compression_equals_all_layer_compression():
-    """Compressing layer r alone (a one-layer problem with that layer's head count and budget) gives the same
+def test_one_layer_problems_equal_the_all_layer_compression():
+    """Compressing layer r alone as a problem of its own (Params.layer: that layer's head count and budget) gives the same
     classes, lengths, positions, cache rows and decode outputs as the all-layer call gives for layer r."""
     tk = _tk()
     wl = small("stream", n=8, n_kv=4, d=128, N=0, L=32, s1=4, s2=64, k=90, dtype="bf16", R=3,
@@ -638,6 +638,171 @@ def test_layer_streamed_compression_equals_all_layer_compression():
         assert torch.equal(got.view(torch.uint8), want_out[:, r:r + 1].contiguous().view(torch.uint8))
         one.close()
     whole.close()
+
+
+WHAT_CACHE_HOLDS = ("Q_SEMVEC", "Q_DIST", "Q_CLASSES", "Q_LENGTHS", "Q_CAPACITY", "Q_OFFSETS", "Q_KPOOL", "Q_VPOOL")
+
+
+def _cache_state(tk, cache, wl):
+    """Everything a cache holds after compression, as arrays that can be compared bit for bit."""
+    got = {w: cache.query(getattr(tk, w)).copy() for w in WHAT_CACHE_HOLDS}
+    lens = got["Q_LENGTHS"]
+    idx = cache.query(tk.Q_INDICES).copy()
+    for u in range(idx.shape[0]):          # slots past a unit's retained positions are never written
+        b, r = u // (wl.n_layers * wl.n_kv_heads), (u // wl.n_kv_heads) % wl.n_layers
+        idx[u, min(int(lens[u]), wl.kept_len(b, r)) if lens[u] < wl.seq_lens[b] else 0:] = -1
+    got["Q_INDICES"] = idx
+    # of the pools only the rows a unit holds (the reserve for appended tokens is not written by compression)
+    off = got["Q_OFFSETS"]
+    row = wl.head_dim * wl.elem_size
+    for name in ("Q_KPOOL", "Q_VPOOL"):
+        raw = got[name]
+        got[name] = np.concatenate([raw[int(off[u]) * row:(int(off[u]) + int(lens[u])) * row] for u in range(len(lens))])
+    return got
+
+
+STREAM_CASES = [
+    # grouped queries, 128 window rows (two-pass tensor-core window kernel), ragged batch, layer schedules
+    dict(n=8, n_kv=2, d=128, N=0, L=32, s1=4, s2=64, k=90, dtype="bf16", R=4, seq_lens=[1400, 2100, 900], nh=1),
+    # one query head per KV head, 32 window rows (single-read window kernel)
+    dict(n=8, n_kv=8, d=128, N=0, L=32, s1=4, s2=64, k=120, dtype="bf16", R=3, seq_lens=[3000, 4500], nh=2),
+    # fp32 on the CUDA cores
+    dict(n=4, n_kv=4, d=64, N=0, L=16, s1=4, s2=32, k=50, dtype="f32", R=3, seq_lens=[900, 700], nh=1),
+]
+
+
+@pytest.mark.parametrize("case", STREAM_CASES, ids=["bf16_gqa_ragged", "bf16_mha", "f32"])
+def test_layers_streamed_into_one_cache_equal_the_all_layer_call(case):
+    """taskkv_cache_create + one taskkv_compress_layer per layer, in a scrambled order and with every layer's
+    tensors in allocations of their own, against taskkv_compress_ex over all layers: semantic vectors, distances,
+    classes, lengths, capacities, segment offsets, retained positions and both pools are the same bits; so are the
+    outputs of decode steps over all layers and layer by layer.  One layer is also checked against the oracle, and
+    a layer-range decode runs before the last layer is in."""
+    tk, P = _tk(), _parity()
+    wl = small("stream_one_cache", **case, steps=2)
+    R = wl.n_layers
+    wl.mid_budget = [case["k"] + 13 * r for r in range(R)]
+    wl.n_hetero = [[(b + r) % (wl.n_kv_heads - 1) for r in range(R)] for b in range(wl.batch)]
+    wl.planted = W._choose_planted(wl)
+    qs, ks, vs = W.materialize(wl, DEV)
+    params = tk.params_from_workload(wl, max_new_tokens=wl.decode_steps)
+    whole = tk.taskkv_compress_ex(params, qs, ks, vs)
+    want = _cache_state(tk, whole, wl)
+
+    streamed = tk.taskkv_cache_create(params, DEV)
+    assert streamed.lengths().tolist() == [0] * (wl.batch * R * wl.n_kv_heads)
+    order = list(range(R))[::-1] if R < 4 else [2, 0, 3, 1]
+    layer_inputs = {r: ([x[r].clone() for x in qs], [x[r].clone() for x in ks], [x[r].clone() for x in vs])
+                    for r in range(R)}
+    q0, kn0, vn0 = W.gen_decode_step(wl, 0, DEV)
+    for i, r in enumerate(order):
+        ql, kl, vl = layer_inputs.pop(r)
+        streamed.taskkv_compress_layer(r, ql, kl, vl)
+        del ql, kl, vl                      # the caller may free a layer's K and V once the stream has passed
+        if i == 0:
+            # a layer that is in can be decoded while the others are still missing
+            early = streamed.taskkv_decode_ex(q0[:, r:r + 1].contiguous(), r, 1)
+            ref = whole.taskkv_decode_ex(q0[:, r:r + 1].contiguous(), r, 1)
+            assert torch.equal(early.view(torch.uint8), ref.view(torch.uint8))
+    with pytest.raises(tk.TaskKVError) as ei:
+        streamed.taskkv_compress_layer(order[0], [x[order[0]].contiguous() for x in qs],
+                                       [x[order[0]].contiguous() for x in ks], [x[order[0]].contiguous() for x in vs])
+    assert ei.value.status == tk.ESTATE                 # a layer goes in once
+    with pytest.raises(tk.TaskKVError):
+        streamed.taskkv_compress_layer(R, [x[0].contiguous() for x in qs], [x[0].contiguous() for x in ks],
+                                       [x[0].contiguous() for x in vs])
+    assert streamed.status() == 0
+    got = _cache_state(tk, streamed, wl)
+    for name in want:
+        assert np.array_equal(want[name], got[name]), f"{name} differs between the streamed and the all-layer cache"
+    # the oracle on one (sequence, layer) of the streamed cache
+    rep = P.Report()
+    b, r = wl.batch - 1, order[0]
+    ref = P.oracle_layer(wl, b, r, qs[b][r], ks[b][r], vs[b][r])
+    P.compare_layer(streamed, wl, b, r, ref, rep, v=vs[b][r])
+    rep.check_bounds(wl.name)
+    # decode over the streamed cache: all layers at once, then layer by layer
+    for s_ in range(wl.decode_steps):
+        q, kn, vn = W.gen_decode_step(wl, s_, DEV)
+        a = whole.taskkv_decode_step(q, kn, vn)
+        if s_ == 0:
+            bb = streamed.taskkv_decode_step(q, kn, vn)
+        else:
+            bb = torch.empty_like(a)
+            for r in range(R):
+                bb[:, r:r + 1] = streamed.taskkv_decode_step_ex(q[:, r:r + 1].contiguous(), kn[:, r:r + 1].contiguous(),
+                                                                vn[:, r:r + 1].contiguous(), r, 1)
+        assert torch.equal(a.view(torch.uint8), bb.view(torch.uint8)), f"decode step {s_}"
+    assert np.array_equal(whole.lengths(), streamed.lengths())
+    assert whole.status() == 0 and streamed.status() == 0
+    whole.close()
+    streamed.close()
+
+
+def test_gather_overlapped_compression_equals_the_plain_order_bit_for_bit():
+    """Grouped queries with enough layers for the library to cut them into chunks and gather one chunk beside the
+    window scores and the selection of the next (two streams): against the plain order (one launch of every step
+    over all layers, which the library takes while per-kernel timing is switched on) everything a cache holds must
+    be the same bits, three times in a row, also when the caller's stream is not the default one."""
+    tk = _tk()
+    wl = small("gather_chunks", n=32, n_kv=8, d=128, N=0, L=32, s1=4, s2=64, k=150, dtype="bf16", R=8,
+               seq_lens=[2500, 1100], nh=2, steps=0)
+    wl.mid_budget = [150 + 7 * r for r in range(8)]
+    qs, ks, vs = W.materialize(wl, DEV)
+
+    def run(stream=None):
+        params = tk.params_from_workload(wl, max_new_tokens=2)
+        if stream is None:
+            cache = tk.taskkv_compress_ex(params, qs, ks, vs)
+        else:
+            with torch.cuda.stream(stream):
+                cache = tk.taskkv_compress_ex(params, qs, ks, vs)
+            stream.synchronize()
+        assert cache.status() == 0
+        got = _cache_state(tk, cache, wl)
+        got["scores"] = cache.query(tk.Q_SCORES).copy()
+        got["topt"] = cache.query(tk.Q_TOPT).copy()
+        cache.close()
+        return got
+
+    tk.taskkv_timing_enable(True)
+    try:
+        plain = run()
+    finally:
+        tk.taskkv_timing_enable(False)
+        tk.taskkv_timing_collect()
+    side = torch.cuda.Stream()
+    for stream in (None, side, None):
+        got = run(stream)
+        for name in plain:
+            assert np.array_equal(plain[name], got[name]), name
+    # and the oracle on layers of different chunks
+    run_workload(wl, layers=[(0, 0), (1, 3), (0, 4), (1, 7)], decode_steps=1)
+
+
+def test_budget_given_as_a_fraction_of_the_full_cache():
+    """budget_frac: the middle budget of every (sequence, layer) follows Eq. 17 from 40 % of the full cache, computed
+    by the library (on the device, and by the same formula on the host for the pool sizes).  A ragged batch, so the
+    budgets differ by sequence as well as by layer; the oracle is given the budgets of its own Eq. 17."""
+    tk = _tk()
+    wl = small("budget_frac", n=16, n_kv=8, d=128, N=0, L=32, s1=4, s2=64, k=0, dtype="bf16", R=3,
+               seq_lens=[3000, 5200, 1700], nh=1, steps=2)
+    wl.n_hetero = [[2, 1, 0], [1, 3, 2], [0, 0, 7]]
+    wl.planted = W._choose_planted(wl)
+    frac = 0.4
+    wl.mid_by_seq = [[O.mid_budget(frac * 8 * wl.seq_lens[b], wl.seq_lens[b], wl.full_heads(b, r), 8, wl.sink, wl.recent)
+                      for r in range(3)] for b in range(3)]
+    assert len({m for row in wl.mid_by_seq for m in row}) >= 6
+    wl.budget_frac = frac
+    rep = run_workload(wl)
+    assert rep.units == 72
+    # the cache holds at most 40 % of the rows of every (sequence, layer), and misses it by less than one row per head
+    for b in range(3):
+        for r in range(3):
+            h = wl.full_heads(b, r)
+            rows = h * wl.seq_lens[b] + (8 - h) * wl.kept_len(b, r)
+            if wl.mid_of(b, r) > 0:
+                assert 0 <= frac * 8 * wl.seq_lens[b] - rows < 8 - h
 
 
 @pytest.mark.parametrize("case", [
