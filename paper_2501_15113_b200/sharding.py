@@ -4,6 +4,12 @@ Every (sequence, layer) is independent of every other (the separator couples onl
 one layer), so a job is split across ranks by whole (sequence, layer) pairs -- or, as bench.py does for
 weak scaling, every rank runs its own replica of the batch.  The only exchange is the timing reduce:
 throughput of the whole job = units all ranks processed / the slowest rank's time.
+
+Sharding by KV head (tensor-parallel style, where every rank holds some heads of every layer) does need one
+exchange: the center of Eq. 8 is the mean over ALL heads of a layer, so the ranks all-gather their heads'
+semantic vectors (n_kv_local x d fp32 per sequence and layer) and each runs the separator of Sec. IV-A on the full
+set, redundantly; everything before (window scores, top-t, Eq. 15) and after (allocation, gather, decode) is per
+head.  `shard_heads`, `allgather_semantic_vectors` and `shard_pool_rows_bound` are the host side of that variant.
 """
 from __future__ import annotations
 
@@ -35,3 +41,36 @@ def job_throughput(units_this_rank: float, ms_this_rank: float, device=None) -> 
     dist.all_reduce(t, op=dist.ReduceOp.MAX)
     dist.all_reduce(n, op=dist.ReduceOp.SUM)
     return float(n.item()) * 1e3 / float(t.item()), float(t.item())
+
+
+def shard_heads(n_kv_heads: int, rank: int, world: int) -> range:
+    """KV heads owned by `rank`: a contiguous, balanced block (query heads follow their KV head)."""
+    lo = n_kv_heads * rank // world
+    hi = n_kv_heads * (rank + 1) // world
+    return range(lo, hi)
+
+
+def allgather_semantic_vectors(local: torch.Tensor, n_kv_heads: int) -> torch.Tensor:
+    """local: [..., n_local, d] fp32 semantic vectors (Eq. 15) of this rank's heads, in `shard_heads` order.
+    Returns [..., n_kv_heads, d] with every rank's block in place, identical on all ranks.  Blocks may differ in
+    size by one head, so each is padded to the largest before the collective (into local memory: the result is an
+    ordinary tensor of this rank)."""
+    if not (dist.is_available() and dist.is_initialized()) or dist.get_world_size() == 1:
+        return local
+    world = dist.get_world_size()
+    sizes = [len(shard_heads(n_kv_heads, r, world)) for r in range(world)]
+    pad = max(sizes)
+    lead, d = local.shape[:-2], local.shape[-1]
+    buf = torch.zeros(*lead, pad, d, dtype=local.dtype, device=local.device)
+    buf[..., :local.shape[-2], :] = local
+    parts = [torch.empty_like(buf) for _ in range(world)]
+    dist.all_gather(parts, buf.contiguous())
+    return torch.cat([parts[r][..., :sizes[r], :] for r in range(world)], dim=-2)
+
+
+def shard_pool_rows_bound(seq_len: int, n_local: int, full_heads: int, kept_len: int, max_new_tokens: int = 0) -> int:
+    """Pool rows a rank must reserve for one (sequence, layer) when heads are sharded: how many heads of the layer
+    keep everything is fixed by Eq. 16, but which rank they land on is not, so a rank plans for as many of them as it
+    has heads."""
+    h = min(full_heads, n_local)
+    return h * (seq_len + max_new_tokens) + (n_local - h) * (kept_len + max_new_tokens)
