@@ -4,7 +4,6 @@
 #include <atomic>
 #include <cmath>
 #include <cstdio>
-#include <cstdlib>
 #include <cstring>
 #include <mutex>
 #include <new>
@@ -324,18 +323,14 @@ int overlap_chunks(const DeviceProblem& dp, int dtype, const WindowHostInfo& wh)
   return chunks;
 }
 
-// Chunks for (2): the two-pass tensor-core window kernel, at least 32 units and 2 layers... per chunk.
+// Chunks for (2): where the two-pass tensor-core window kernel runs, up to four chunks of at least 64 units each
+// (measured on the 131072-key and the ragged-batch shapes: two chunks hide less of the gather, eight add launches
+// and part-filled grids for nothing), and not while per-kernel durations are being recorded.
 int gather_overlap_chunks(const DeviceProblem& dp, int dtype, const WindowHostInfo& wh) {
   if (g_timing.load(std::memory_order_relaxed)) return 1;
   if (!window_tc_supported(dp, dtype) || window_res_supported(dp, wh)) return 1;
-  static int forced = -1;
-  if (forced < 0) {
-    const char* e = std::getenv("TASKKV_GATHER_CHUNKS");
-    forced = e ? std::atoi(e) : 0;
-  }
   int chunks = 1;
-  const int cap = forced > 0 ? forced : kMaxChunks;
-  while (chunks * 2 <= cap && chunks * 2 <= dp.R && (int64_t)(dp.R / (chunks * 2)) * dp.n_kv * wh.batch >= 32)
+  while (chunks * 2 <= 4 && chunks * 2 <= dp.R && (int64_t)(dp.R / (chunks * 2)) * dp.n_kv * wh.batch >= 64)
     chunks *= 2;
   return chunks;
 }
