@@ -204,8 +204,10 @@ taskkv_status taskkv_compress_lse(const taskkv_params* p, const void* const* q_w
  *                            q_win[b]  device [n_heads][L][d]       the layer's last L query rows
  *                            k[b],v[b] device [n_kv_heads][N_b][d]  the layer's keys / values
  *                            window_lse[b] device fp32 [n_heads][L] or window_lse == NULL (see taskkv_compress_lse)
- *                          Each layer may be compressed once (ESTATE otherwise), in any order, all on one stream (or
- *                          ordered by the caller: the calls share the workspace).  Classes, lengths, retained
+ *                          Each layer may be compressed once (ESTATE otherwise), in any order.  Calls for different
+ *                          layers work on disjoint parts of the cache and of the workspace, so they may be issued on
+ *                          different streams (each ordered after taskkv_cache_create) and then overlap on the GPU;
+ *                          host-side the calls on one cache are not re-entrant.  Classes, lengths, retained
  *                          positions, cache rows, segment offsets and work lists are bit for bit those the all-layer
  *                          call produces; once every layer is in, the cache is the same object, and
  *                          taskkv_decode_step and the other decode calls work on it as usual (a layer-range decode

@@ -467,9 +467,9 @@ void fill_device_problem(taskkv_cache* c) {
   d.budget_frac = p.budget_frac;
   d.nhet = reinterpret_cast<const int32_t*>(cm + hp.o_nhet);
   d.c_off = reinterpret_cast<const int64_t*>(cm + hp.o_c_off);
-  d.q_ptr = reinterpret_cast<const void* const*>(cm + hp.o_qp);
-  d.k_ptr = reinterpret_cast<const void* const*>(cm + hp.o_kp);
-  d.v_ptr = reinterpret_cast<const void* const*>(cm + hp.o_vp);
+  d.q_ptr = reinterpret_cast<const void**>(cm + hp.o_qp);
+  d.k_ptr = reinterpret_cast<const void**>(cm + hp.o_kp);
+  d.v_ptr = reinterpret_cast<const void**>(cm + hp.o_vp);
   d.status = reinterpret_cast<int32_t*>(cm + hp.o_status);
   d.len = reinterpret_cast<int32_t*>(cm + hp.o_len);
   d.cap = reinterpret_cast<int32_t*>(cm + hp.o_cap);
@@ -745,8 +745,8 @@ taskkv_status taskkv_compress_layer(taskkv_cache* c, int32_t layer, const void* 
   if (!pointers_ok(&c->prm, q_win, k, v, window_lse)) return TASKKV_EINVAL;
   if (c->layer_done[(size_t)layer]) return TASKKV_ESTATE;      // a layer's segments are written once
   cudaStream_t s = static_cast<cudaStream_t>(stream);
-  set_layer_pointers(c, layer, 1, q_win, k, v);
-  cudaError_t e = upload_pointers(c, s);
+  // this layer's entries of the pointer tables, written on the device: calls for other layers touch other words
+  cudaError_t e = launch_set_layer_pointers(c->dp, c->prm.batch, layer, c->prm.dtype == TASKKV_F32 ? 4 : 2, q_win, k, v, s);
   WindowHostInfo wh;
   wh.batch = c->prm.batch;
   wh.seq_lens = c->hp.seq_lens.data();

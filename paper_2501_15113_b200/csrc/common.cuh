@@ -70,9 +70,9 @@ struct DeviceProblem {
   const int64_t* seg_base;    // [B*R+1] first pool row of block b * R + r
   const int32_t* gather_base; // [R*B+1] first gather work item of block r * B + b (layer-major)
   const int32_t* dec_base;    // [R*B+1] first decode work item of block r * B + b (layer-major)
-  const void* const* q_ptr;   // [U] -> [rows][d]
-  const void* const* k_ptr;   // [U] -> [N][d]
-  const void* const* v_ptr;   // [U] -> [N][d]
+  const void** q_ptr;         // [U] -> [rows][d]
+  const void** k_ptr;         // [U] -> [N][d]
+  const void** v_ptr;         // [U] -> [N][d]
   // results
   int32_t* status;            // sticky status word
   int32_t* len;               // [U]
@@ -153,6 +153,10 @@ cudaError_t launch_window_scores_res(const DeviceProblem& p, const WindowHostInf
 cudaError_t launch_select(const DeviceProblem& p, int dtype, int max_N, cudaStream_t s,
                           const UnitRange* range = nullptr);
 cudaError_t launch_separator_plan(const DeviceProblem& p, int batch, int layer0, int n_layers, cudaStream_t s);
+// Per-unit input pointers of one layer written on the device from the per-sequence bases of that layer
+// (q_win[b]: [n][L][d], k[b], v[b]: [n_kv][N_b][d]); host arrays of `batch` device pointers.
+cudaError_t launch_set_layer_pointers(const DeviceProblem& p, int batch, int layer, int elem_size, const void* const* q_win,
+                                      const void* const* k, const void* const* v, cudaStream_t s);
 // Eq. 17 on the device for the units of a range of layers (nothing to do unless budget_frac > 0)
 cudaError_t launch_budget(const DeviceProblem& p, int batch, int layer0, int n_layers, cudaStream_t s);
 // gather work items [item0, item0 + n_items) = those of layers [layer0, layer0 + n_layers) (layer-major numbering)

@@ -143,7 +143,42 @@ __global__ void __launch_bounds__(128) budget_kernel(DeviceProblem p, UnitRange 
   p.unit_mid[u] = k;
 }
 
+// The input pointers of one layer's units, from the layer's per-sequence base pointers (passed by value, up to
+// kPtrSeqs sequences per launch): only this layer's entries of the tables are written, so calls for different
+// layers never touch the same words.
+constexpr int kPtrSeqs = 64;
+struct LayerBases {
+  const void* q[kPtrSeqs];
+  const void* k[kPtrSeqs];
+  const void* v[kPtrSeqs];
+};
+__global__ void __launch_bounds__(128) set_layer_pointers_kernel(DeviceProblem p, const __grid_constant__ LayerBases bases,
+                                                                 int b0, int nb, int layer, int elem_size) {
+  const int i = blockIdx.x * blockDim.x + threadIdx.x;
+  if (i >= nb * p.n_kv) return;
+  const int bi = i / p.n_kv, h = i % p.n_kv;
+  const size_t u = ((size_t)(b0 + bi) * p.R + layer) * p.n_kv + h;
+  const size_t N = (size_t)p.unit_N[u], row = (size_t)p.d * elem_size;
+  p.q_ptr[u] = static_cast<const unsigned char*>(bases.q[bi]) + (size_t)h * p.rows * row;
+  p.k_ptr[u] = static_cast<const unsigned char*>(bases.k[bi]) + (size_t)h * N * row;
+  p.v_ptr[u] = static_cast<const unsigned char*>(bases.v[bi]) + (size_t)h * N * row;
+}
+
 }  // namespace
+
+cudaError_t launch_set_layer_pointers(const DeviceProblem& p, int batch, int layer, int elem_size, const void* const* q_win,
+                                      const void* const* k, const void* const* v, cudaStream_t s) {
+  for (int b0 = 0; b0 < batch; b0 += kPtrSeqs) {
+    const int nb = batch - b0 < kPtrSeqs ? batch - b0 : kPtrSeqs;
+    LayerBases bases = {};
+    for (int i = 0; i < nb; ++i) { bases.q[i] = q_win[b0 + i]; bases.k[i] = k[b0 + i]; bases.v[i] = v[b0 + i]; }
+    LaunchScope ls(K_PLAN, s);
+    set_layer_pointers_kernel<<<(nb * p.n_kv + 127) / 128, 128, 0, s>>>(p, bases, b0, nb, layer, elem_size);
+    const cudaError_t e = cudaGetLastError();
+    if (e != cudaSuccess) return e;
+  }
+  return cudaSuccess;
+}
 
 cudaError_t launch_budget(const DeviceProblem& p, int batch, int layer0, int n_layers, cudaStream_t s) {
   if (!(p.budget_frac > 0.f)) return cudaSuccess;

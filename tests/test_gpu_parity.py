@@ -698,6 +698,7 @@ def test_layers_streamed_into_one_cache_equal_the_all_layer_call(case):
     for i, r in enumerate(order):
         ql, kl, vl = layer_inputs.pop(r)
         streamed.taskkv_compress_layer(r, ql, kl, vl)
+        torch.cuda.current_stream().synchronize()
         del ql, kl, vl                      # the caller may free a layer's K and V once the stream has passed
         if i == 0:
             # a layer that is in can be decoded while the others are still missing
@@ -737,6 +738,46 @@ def test_layers_streamed_into_one_cache_equal_the_all_layer_call(case):
     assert whole.status() == 0 and streamed.status() == 0
     whole.close()
     streamed.close()
+
+
+def test_layers_streamed_on_several_streams_equal_the_all_layer_call():
+    """Calls for different layers touch disjoint parts of the cache and of the workspace, so a prefill loop may issue
+    them on different streams: six layers go round-robin to three streams, which are then joined; the cache must be
+    the all-layer one bit for bit, three times in a row (a race between two layers' kernels would show)."""
+    tk = _tk()
+    wl = small("stream_streams", n=16, n_kv=4, d=128, N=0, L=32, s1=4, s2=64, k=110, dtype="bf16", R=6,
+               seq_lens=[2300, 1500], nh=1, steps=1)
+    wl.mid_budget = [110 + 9 * r for r in range(6)]
+    qs, ks, vs = W.materialize(wl, DEV)
+    params = tk.params_from_workload(wl, max_new_tokens=1)
+    whole = tk.taskkv_compress_ex(params, qs, ks, vs)
+    want = _cache_state(tk, whole, wl)
+    ins = [([x[r].contiguous() for x in qs], [x[r].contiguous() for x in ks], [x[r].contiguous() for x in vs])
+           for r in range(6)]
+    streams = [torch.cuda.Stream() for _ in range(3)]
+    main = torch.cuda.current_stream()
+    for _ in range(3):
+        cache = tk.taskkv_cache_create(params, DEV)
+        created = torch.cuda.Event()
+        created.record(main)
+        for st in streams:
+            st.wait_event(created)
+        for r in range(6):
+            cache.taskkv_compress_layer(r, *ins[r], stream=streams[r % 3])
+        for st in streams:
+            done = torch.cuda.Event()
+            done.record(st)
+            main.wait_event(done)
+        assert cache.status() == 0
+        got = _cache_state(tk, cache, wl)
+        for name in want:
+            assert np.array_equal(want[name], got[name]), name
+        q, kn, vn = W.gen_decode_step(wl, 0, DEV)
+        a = cache.taskkv_decode_step(q, kn, vn)
+        cache.close()
+    b = whole.taskkv_decode_step(q, kn, vn)
+    assert torch.equal(a.view(torch.uint8), b.view(torch.uint8))
+    whole.close()
 
 
 def test_gather_overlapped_compression_equals_the_plain_order_bit_for_bit():
