@@ -104,6 +104,10 @@ typedef struct taskkv_params {
                                 budget of Eq. 17, k = floor((B - N h) / (n - h)) - s1 - s2 with B = fraction * n_kv * N_b
                                 and h the heads of that layer that keep everything, computed on the device (and, for
                                 the exact sizing of the pools, by the same formula on the host) */
+  int32_t shard_kv_heads;    /* 0: the problem holds every KV head of the model.  > 0: head sharding -- the model has this
+                                many KV heads per layer and this problem holds n_kv_heads of them, starting at shard_first
+                                (and their query heads); see taskkv_compress_shard_begin */
+  int32_t shard_first;
 } taskkv_params;
 
 typedef struct taskkv_plan_info {
@@ -219,6 +223,29 @@ taskkv_status taskkv_cache_create(const taskkv_params* p, void* cache_mem, size_
 taskkv_status taskkv_compress_layer(taskkv_cache* c, int32_t layer, const void* const* q_win,
                                     const void* const* k, const void* const* v, const void* const* window_lse,
                                     taskkv_stream stream);
+
+/* Head sharding (tensor-parallel style): every rank holds some KV heads of every layer.  Window scores, top-t and
+ * semantic vectors (Eq. 12-15) are per head; the center of Eq. 8 and the ranking of Sec. IV-A are over ALL heads of a
+ * layer; allocation, gather and decode are per head again.  So a rank runs
+ *   taskkv_compress_shard_begin   steps a1-a2 for its heads (params with shard_kv_heads > 0; n_heads, n_kv_heads and the
+ *                                 q_win / k / v tensors are the rank's own; Eq. 16, Eq. 17 and an n_hetero override
+ *                                 count over the model's shard_kv_heads heads),
+ *   taskkv_cache_semantic         device pointer to its vectors, fp32 [batch][n_layers][n_kv_heads][d] -- the ranks
+ *                                 all-gather these into [batch][n_layers][shard_kv_heads][d] in head order (any
+ *                                 collective; into this GPU's own memory),
+ *   taskkv_compress_shard_finish  separator over the gathered vectors (every rank computes every head's class and keeps
+ *                                 its own), plan and gather for its heads.
+ * Which rank the layer's full-cache heads land on is data dependent, so a shard's pools are sized for the most it can
+ * get, min(full heads of the layer, n_kv_heads) per (sequence, layer): pool_rows, retained_rows and cache_bytes of
+ * taskkv_plan are then upper bounds, and the lengths tell what is used.  Classes, lengths, retained positions, cache
+ * rows and decode outputs of a head are those of the unsharded problem.  The decode calls work on a shard's cache as on
+ * any other.  finish without begin, or begin's cache used before finish, is ESTATE / undefined lengths of 0. */
+taskkv_status taskkv_compress_shard_begin(const taskkv_params* p, const void* const* q_win, const void* const* k,
+                                          const void* const* v, const void* const* window_lse,
+                                          void* cache_mem, size_t cache_bytes, void* workspace_mem,
+                                          size_t workspace_bytes, taskkv_stream stream, taskkv_cache** out_cache);
+taskkv_status taskkv_cache_semantic(const taskkv_cache* c, const float** device_ptr, int64_t* n_floats);
+taskkv_status taskkv_compress_shard_finish(taskkv_cache* c, const float* sem_all, taskkv_stream stream);
 
 /* The flat form of the same call: one bf16 sequence, Sec. V-D defaults for
  * everything not listed, library-owned memory, max_new_tokens = 4096. */

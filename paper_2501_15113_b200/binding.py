@@ -39,6 +39,7 @@ class taskkv_params(C.Structure):
         ("max_new_tokens", C.c_int32), ("mid_policy", C.c_int32),
         ("seq_lens", C.POINTER(C.c_int32)), ("mid_budget_per_layer", C.POINTER(C.c_int32)),
         ("n_hetero", C.POINTER(C.c_int32)), ("budget_frac", C.c_float),
+        ("shard_kv_heads", C.c_int32), ("shard_first", C.c_int32),
     ]
 
 
@@ -61,6 +62,13 @@ lib.taskkv_cache_create.argtypes = [C.POINTER(taskkv_params), _vp, C.c_size_t, _
 lib.taskkv_cache_create.restype = C.c_int32
 lib.taskkv_compress_layer.argtypes = [_vp, C.c_int32, _pp, _pp, _pp, _pp, _vp]
 lib.taskkv_compress_layer.restype = C.c_int32
+lib.taskkv_compress_shard_begin.argtypes = [C.POINTER(taskkv_params), _pp, _pp, _pp, _pp, _vp, C.c_size_t, _vp, C.c_size_t,
+                                            _vp, C.POINTER(_vp)]
+lib.taskkv_compress_shard_begin.restype = C.c_int32
+lib.taskkv_cache_semantic.argtypes = [_vp, C.POINTER(_vp), C.POINTER(C.c_int64)]
+lib.taskkv_cache_semantic.restype = C.c_int32
+lib.taskkv_compress_shard_finish.argtypes = [_vp, _vp, _vp]
+lib.taskkv_compress_shard_finish.restype = C.c_int32
 lib.taskkv_compress_lse.argtypes = [C.POINTER(taskkv_params), _pp, _pp, _pp, _pp, _vp, C.c_size_t, _vp, C.c_size_t,
                                     _vp, C.POINTER(_vp)]
 lib.taskkv_compress_lse.restype = C.c_int32
@@ -176,12 +184,13 @@ class Params:
     def __init__(self, *, n_layers, n_heads, n_kv_heads, head_dim, seq_lens: Sequence[int], sink, recent,
                  mid_budget, window, dtype, top_t=256, pool_kernel=7, beta=0.25, m_top=4,
                  n_hetero: Optional[Sequence[Sequence[int]]] = None, promote_center=True, force_class=-1,
-                 max_new_tokens=0, mid_policy=0, budget_frac=0.0):
+                 max_new_tokens=0, mid_policy=0, budget_frac=0.0, shard_kv_heads=0, shard_first=0):
         self.kw = dict(n_layers=n_layers, n_heads=n_heads, n_kv_heads=n_kv_heads, head_dim=head_dim,
                        seq_lens=list(seq_lens), sink=sink, recent=recent, mid_budget=mid_budget, window=window,
                        dtype=dtype, top_t=top_t, pool_kernel=pool_kernel, beta=beta, m_top=m_top, n_hetero=n_hetero,
                        promote_center=promote_center, force_class=force_class, max_new_tokens=max_new_tokens,
-                       mid_policy=mid_policy, budget_frac=budget_frac)
+                       mid_policy=mid_policy, budget_frac=budget_frac, shard_kv_heads=shard_kv_heads,
+                       shard_first=shard_first)
         p = taskkv_params()
         lib.taskkv_params_default(C.byref(p))
         p.n_layers, p.n_heads, p.n_kv_heads, p.head_dim = n_layers, n_heads, n_kv_heads, head_dim
@@ -209,6 +218,7 @@ class Params:
         p.max_new_tokens = max_new_tokens
         p.mid_policy = int(mid_policy)
         p.budget_frac = float(budget_frac)
+        p.shard_kv_heads, p.shard_first = int(shard_kv_heads), int(shard_first)
         self.c = p
 
     @property
@@ -288,6 +298,25 @@ class Cache:
             la = _ptr_array(window_lse)
         _check(lib.taskkv_compress_layer(self._h, layer, _ptr_array(q_win), _ptr_array(k), _ptr_array(v), la,
                                          _stream_handle(stream)), "taskkv_compress_layer")
+
+    def semantic_vectors(self) -> torch.Tensor:
+        """The cache's semantic vectors (Eq. 15) as a view of its device memory: fp32 [batch * n_layers, n_kv, d]."""
+        ptr, n = C.c_void_p(), C.c_int64()
+        _check(lib.taskkv_cache_semantic(self._h, C.byref(ptr), C.byref(n)), "taskkv_cache_semantic")
+        mem = self._keep["cache"]
+        off = ptr.value - mem.data_ptr()
+        d = self.params.c.head_dim
+        return mem[off:off + 4 * n.value].view(torch.float32).view(-1, self.params.c.n_kv_heads, d)
+
+    def taskkv_compress_shard_finish(self, sem_all: torch.Tensor, stream=None) -> None:
+        """sem_all: fp32 [batch * n_layers, shard_kv_heads, d], every shard's vectors in head order."""
+        if sem_all.dtype != torch.float32 or not sem_all.is_cuda or not sem_all.is_contiguous():
+            raise ValueError("sem_all must be a contiguous fp32 CUDA tensor")
+        p = self.params.c
+        if sem_all.numel() != p.batch * p.n_layers * p.shard_kv_heads * p.head_dim:
+            raise ValueError("sem_all must hold batch * n_layers * shard_kv_heads * d floats")
+        _check(lib.taskkv_compress_shard_finish(self._h, sem_all.data_ptr(), _stream_handle(stream)),
+               "taskkv_compress_shard_finish")
 
     # -- the decode-side calls
     def taskkv_append(self, k_new: torch.Tensor, v_new: torch.Tensor, stream=None) -> None:
@@ -441,6 +470,25 @@ def taskkv_cache_create(params: Params, device, stream=None, cache_mem: Optional
         _check(lib.taskkv_cache_create(C.byref(params.c), cache_mem.data_ptr(), cache_mem.numel(),
                                        workspace_mem.data_ptr(), workspace_mem.numel(), _stream_handle(stream),
                                        C.byref(h)), "taskkv_cache_create")
+    return Cache(h.value, params, {"cache": cache_mem, "workspace": workspace_mem})
+
+
+def taskkv_compress_shard_begin(params: Params, q_win: Sequence[torch.Tensor], k: Sequence[torch.Tensor],
+                                v: Sequence[torch.Tensor], stream=None) -> Cache:
+    """Steps a1-a2 for the KV heads of one shard (params.shard_kv_heads > 0).  The tensors hold the shard's own heads:
+    q_win[b]: [R, n_local * G, L, d]; k[b], v[b]: [R, n_local, N_b, d]."""
+    info = taskkv_plan(params)
+    dev = k[0].device
+    cache_mem = torch.empty(int(info.cache_bytes), dtype=torch.uint8, device=dev)
+    workspace_mem = torch.empty(int(info.workspace_bytes), dtype=torch.uint8, device=dev)
+    for t in list(q_win) + list(k) + list(v):
+        if not t.is_contiguous() or not t.is_cuda:
+            raise ValueError("inputs must be contiguous CUDA tensors")
+    h = C.c_void_p()
+    _check(lib.taskkv_compress_shard_begin(C.byref(params.c), _ptr_array(q_win), _ptr_array(k), _ptr_array(v), None,
+                                           cache_mem.data_ptr(), cache_mem.numel(), workspace_mem.data_ptr(),
+                                           workspace_mem.numel(), _stream_handle(stream), C.byref(h)),
+           "taskkv_compress_shard_begin")
     return Cache(h.value, params, {"cache": cache_mem, "workspace": workspace_mem})
 
 

@@ -73,7 +73,10 @@ taskkv_status make_plan(const taskkv_params* p, HostPlan& hp) {
   if (p->force_class < -1 || p->force_class > 1) return TASKKV_EINVAL;
   if (p->mid_policy < TASKKV_MID_SELECT || p->mid_policy > TASKKV_MID_MEAN) return TASKKV_EINVAL;
   if (!(p->budget_frac >= 0.f) || p->budget_frac > 1.f) return TASKKV_EINVAL;
+  if (p->shard_kv_heads < 0 || p->shard_kv_heads > TASKKV_MAX_KV_HEADS) return TASKKV_EINVAL;
+  if (p->shard_kv_heads > 0 && (p->shard_first < 0 || p->shard_first + p->n_kv_heads > p->shard_kv_heads)) return TASKKV_EINVAL;
   const int B = p->batch, R = p->n_layers, nkv = p->n_kv_heads;
+  const int n_model = p->shard_kv_heads > 0 ? p->shard_kv_heads : nkv;      // heads Eq. 16 / Eq. 17 count over
   if ((int64_t)B * R * nkv > (1 << 20)) return TASKKV_EINVAL;
 
   hp.seq_lens.assign(p->seq_lens, p->seq_lens + B);
@@ -96,19 +99,20 @@ taskkv_status make_plan(const taskkv_params* p, HostPlan& hp) {
   hp.full.resize((size_t)B * R);
   for (int b = 0; b < B; ++b)
     for (int r = 0; r < R; ++r) {
-      int f = p->n_hetero ? p->n_hetero[(size_t)b * R + r] : hetero_count_impl(nkv, p->beta, p->m_top, R, r);
+      int f = p->n_hetero ? p->n_hetero[(size_t)b * R + r] : hetero_count_impl(n_model, p->beta, p->m_top, R, r);
       if (f < 0) return TASKKV_EINVAL;
-      f = std::min(f, nkv);
+      f = std::min(f, n_model);
       hp.nhet[(size_t)b * R + r] = f;
-      int h = std::min(nkv, f + ((p->promote_center && f < nkv) ? 1 : 0));
-      if (p->force_class == 1) h = nkv;
+      int h = std::min(n_model, f + ((p->promote_center && f < n_model) ? 1 : 0));
+      if (p->force_class == 1) h = n_model;
       if (p->force_class == 0) h = 0;
-      hp.full[(size_t)b * R + r] = h;
+      // a shard plans for as many of the layer's full-cache heads as it has heads (which ones it gets is data dependent)
+      hp.full[(size_t)b * R + r] = std::min(h, nkv);
       // a budget given as a fraction of the full cache: Eq. 17 per (sequence, layer), with the heads that really
       // keep everything (the device computes the same number for its own table, see budget_kernel)
       if (p->budget_frac > 0.f)
-        hp.mid[(size_t)b * R + r] = mid_budget_impl((double)p->budget_frac * (double)nkv * (double)hp.seq_lens[b],
-                                                    hp.seq_lens[b], h, nkv, p->sink, p->recent);
+        hp.mid[(size_t)b * R + r] = mid_budget_impl((double)p->budget_frac * (double)n_model * (double)hp.seq_lens[b],
+                                                    hp.seq_lens[b], h, n_model, p->sink, p->recent);
     }
 
   const int64_t U = (int64_t)B * R * nkv;
@@ -267,6 +271,7 @@ struct taskkv_cache {
   void* stage = nullptr;
   size_t stage_bytes = 0;
   std::vector<unsigned char> layer_done;   // [R] layers compressed so far (layer-streamed caches)
+  int shard_stage = 0;                     // head-sharded caches: 1 after begin (vectors ready), 2 after finish
 };
 
 namespace {
@@ -465,6 +470,9 @@ void fill_device_problem(taskkv_cache* c) {
   d.gather_base = reinterpret_cast<const int32_t*>(cm + hp.o_gbase);
   d.dec_base = reinterpret_cast<const int32_t*>(cm + hp.o_dbase);
   d.budget_frac = p.budget_frac;
+  d.n_kv_model = p.shard_kv_heads > 0 ? p.shard_kv_heads : p.n_kv_heads;
+  d.kv_first = p.shard_kv_heads > 0 ? p.shard_first : 0;
+  d.sem_all = nullptr;
   d.nhet = reinterpret_cast<const int32_t*>(cm + hp.o_nhet);
   d.c_off = reinterpret_cast<const int64_t*>(cm + hp.o_c_off);
   d.q_ptr = reinterpret_cast<const void**>(cm + hp.o_qp);
@@ -706,6 +714,7 @@ taskkv_status compress_impl(const taskkv_params* p, const void* const* q_win, co
   if (!p || !q_win || !k || !v || !out_cache) return TASKKV_EINVAL;
   *out_cache = nullptr;
   if (p->batch < 1 || !pointers_ok(p, q_win, k, v, window_lse)) return TASKKV_EINVAL;
+  if (p->shard_kv_heads > 0) return TASKKV_EINVAL;      // a shard needs the other shards' vectors: begin / finish
   cudaStream_t s = static_cast<cudaStream_t>(stream);
   taskkv_cache* c = nullptr;
   const taskkv_status st = cache_create_impl(p, cache_mem, cache_bytes, workspace_mem, workspace_bytes, s, &c);
@@ -734,13 +743,79 @@ taskkv_status compress_impl(const taskkv_params* p, const void* const* q_win, co
 
 taskkv_status taskkv_cache_create(const taskkv_params* p, void* cache_mem, size_t cache_bytes, void* workspace_mem,
                                   size_t workspace_bytes, taskkv_stream stream, taskkv_cache** out_cache) {
+  if (p && p->shard_kv_heads > 0) return TASKKV_EINVAL;
   return cache_create_impl(p, cache_mem, cache_bytes, workspace_mem, workspace_bytes,
                            static_cast<cudaStream_t>(stream), out_cache);
+}
+
+taskkv_status taskkv_compress_shard_begin(const taskkv_params* p, const void* const* q_win, const void* const* k,
+                                          const void* const* v, const void* const* window_lse, void* cache_mem,
+                                          size_t cache_bytes, void* workspace_mem, size_t workspace_bytes,
+                                          taskkv_stream stream, taskkv_cache** out_cache) {
+  if (!p || !q_win || !k || !v || !out_cache) return TASKKV_EINVAL;
+  *out_cache = nullptr;
+  if (p->batch < 1 || p->shard_kv_heads < 1 || !pointers_ok(p, q_win, k, v, window_lse)) return TASKKV_EINVAL;
+  cudaStream_t s = static_cast<cudaStream_t>(stream);
+  taskkv_cache* c = nullptr;
+  const taskkv_status st = cache_create_impl(p, cache_mem, cache_bytes, workspace_mem, workspace_bytes, s, &c);
+  if (st != TASKKV_OK) return st;
+  set_layer_pointers(c, 0, p->n_layers, q_win, k, v);
+  cudaError_t e = upload_pointers(c, s);
+  WindowHostInfo wh;
+  wh.batch = p->batch;
+  wh.seq_lens = c->hp.seq_lens.data();
+  wh.q = q_win;
+  wh.k = k;
+  wh.lse = window_lse;
+  wh.base_layer = 0;
+  // Eq. 12-15 for this shard's heads: window scores, top-t, semantic vectors (and the middle top-k, which the select
+  // kernels produce in the same pass for every unit; only non-heterogeneous heads will use it)
+  if (e == cudaSuccess) e = launch_budget(c->dp, p->batch, 0, p->n_layers, s);
+  if (e == cudaSuccess) e = launch_window_scores(c->dp, p->dtype, c->hp.max_N, wh, s);
+  if (e == cudaSuccess) e = launch_select(c->dp, p->dtype, c->hp.max_N, s);
+  if (e != cudaSuccess) {
+    std::fprintf(stderr, "taskkv_compress_shard_begin: CUDA error: %s\n", cudaGetErrorString(e));
+    cudaGetLastError();
+    taskkv_cache_destroy(c);
+    return TASKKV_ECUDA;
+  }
+  c->shard_stage = 1;
+  *out_cache = c;
+  return TASKKV_OK;
+}
+
+taskkv_status taskkv_cache_semantic(const taskkv_cache* c, const float** device_ptr, int64_t* n_floats) {
+  if (!c || !device_ptr) return TASKKV_EINVAL;
+  *device_ptr = c->dp.sem;
+  if (n_floats) *n_floats = (int64_t)c->dp.U * c->dp.d;
+  return TASKKV_OK;
+}
+
+taskkv_status taskkv_compress_shard_finish(taskkv_cache* c, const float* sem_all, taskkv_stream stream) {
+  if (!c || !sem_all || ((uintptr_t)sem_all & 3)) return TASKKV_EINVAL;
+  if (c->shard_stage != 1) return TASKKV_ESTATE;
+  cudaStream_t s = static_cast<cudaStream_t>(stream);
+  const int B = c->prm.batch, R = c->prm.n_layers;
+  c->dp.sem_all = sem_all;         // only the separator reads it; the cache keeps no reference afterwards
+  cudaError_t e = launch_separator_plan(c->dp, B, 0, R, s);
+  c->dp.sem_all = nullptr;
+  if (e == cudaSuccess) e = launch_gather(c->dp, c->prm.dtype, B, 0, R, 0, c->hp.info.gather_items, s);
+  if (e == cudaSuccess && c->prm.mid_policy == TASKKV_MID_MEAN)
+    e = launch_compensate(c->dp, c->prm.dtype, layer_range(c->dp, B, 0, R), s);
+  if (e != cudaSuccess) {
+    std::fprintf(stderr, "taskkv_compress_shard_finish: CUDA error: %s\n", cudaGetErrorString(e));
+    cudaGetLastError();
+    return TASKKV_ECUDA;
+  }
+  c->shard_stage = 2;
+  std::fill(c->layer_done.begin(), c->layer_done.end(), (unsigned char)1);
+  return TASKKV_OK;
 }
 
 taskkv_status taskkv_compress_layer(taskkv_cache* c, int32_t layer, const void* const* q_win, const void* const* k,
                                     const void* const* v, const void* const* window_lse, taskkv_stream stream) {
   if (!c || !q_win || !k || !v) return TASKKV_EINVAL;
+  if (c->prm.shard_kv_heads > 0) return TASKKV_EINVAL;
   if (layer < 0 || layer >= c->prm.n_layers || !c->work_mem) return TASKKV_EINVAL;
   if (!pointers_ok(&c->prm, q_win, k, v, window_lse)) return TASKKV_EINVAL;
   if (c->layer_done[(size_t)layer]) return TASKKV_ESTATE;      // a layer's segments are written once

@@ -54,6 +54,12 @@ struct DeviceProblem {
   int32_t view_l0, view_nl, view_U;
   int32_t max_new;
   float budget_frac;    // > 0: the middle budget follows Eq. 17 from this fraction of the full cache
+  // Head sharding: this problem holds KV heads [kv_first, kv_first + n_kv) of a model with n_kv_model per layer.
+  // Eq. 8 / Eq. 16 / Eq. 17 count over the model's heads; the separator then reads every head's semantic vector
+  // from sem_all ([B*R][n_kv_model][d], gathered from all shards).  Unsharded: n_kv_model = n_kv, kv_first = 0,
+  // sem_all = nullptr (the cache's own vectors).
+  int32_t n_kv_model, kv_first;
+  const float* sem_all;
   int32_t idx_stride;   // ints per unit in idx
   int32_t chunks_max;   // partial-statistic slots per unit (longest sequence)
   int64_t pool_rows;

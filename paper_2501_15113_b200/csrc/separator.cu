@@ -23,9 +23,10 @@ __global__ void __launch_bounds__(128) separator_plan_kernel(DeviceProblem p, in
   __shared__ int cls[TASKKV_MAX_KV_HEADS];
   const int b_seq = blockIdx.x / n_layers, r_lay = layer0 + blockIdx.x % n_layers;
   const int br = b_seq * p.R + r_lay;
-  const int n = p.n_kv, d = p.d;
+  const int nl = p.n_kv, d = p.d;          // heads of this problem (a shard holds nl of the model's n)
+  const int n = p.n_kv_model, h0 = p.kv_first;
   const int tid = threadIdx.x;
-  const float* sem = p.sem + (size_t)br * n * d;
+  const float* sem = p.sem_all ? p.sem_all + (size_t)br * n * d : p.sem + (size_t)br * nl * d;
 
   if (tid < d) {
     double s = 0.0;
@@ -67,23 +68,25 @@ __global__ void __launch_bounds__(128) separator_plan_kernel(DeviceProblem p, in
         if (cls[h] == TASKKV_CLASS_NON_HETERO) nearer += (dist[h] < me) || (dist[h] == me && h < tid);
       if (nearer == 0) c = TASKKV_CLASS_CENTER;
     }
-    p.cls[(size_t)br * n + tid] = c;
-    p.dist[(size_t)br * n + tid] = (float)dist[tid];
+    if (tid >= h0 && tid < h0 + nl) {      // this problem's own heads
+      p.cls[(size_t)br * nl + tid - h0] = c;
+      p.dist[(size_t)br * nl + tid - h0] = (float)dist[tid];
+    }
   }
   __syncthreads();                 // every thread has read the far / not-far marks
   if (tid < n) cls[tid] = c;
   __syncthreads();
 
-  // ---- plan of this block's units
+  // ---- plan of this block's units (the problem's own heads)
   __shared__ int s_cap[TASKKV_MAX_KV_HEADS], s_git[TASKKV_MAX_KV_HEADS], s_dit[TASKKV_MAX_KV_HEADS];
   const int B = lm_batch(p);
   const int lm_block = r_lay * B + b_seq;
   int len = 0;
-  if (tid < n) {
-    const int u = br * n + tid;
+  if (tid < nl) {
+    const int u = br * nl + tid;
     const int N = p.unit_N[u];
     len = N;
-    if (cls[tid] == TASKKV_CLASS_NON_HETERO && N > p.sink + p.recent)
+    if (cls[h0 + tid] == TASKKV_CLASS_NON_HETERO && N > p.sink + p.recent)
       len = p.sink + p.recent + min(p.unit_mid[u], N - p.sink - p.recent);
     const int cap = len + p.max_new;
     p.len[u] = len;
@@ -93,19 +96,26 @@ __global__ void __launch_bounds__(128) separator_plan_kernel(DeviceProblem p, in
     s_dit[tid] = (cap + kDecodeChunk - 1) / kDecodeChunk;
   }
   __syncthreads();
-  if (tid < n) {
+  if (tid < nl) {
     int64_t rows_before = 0;
     int git_before = 0, dit_before = 0;
     for (int h = 0; h < tid; ++h) { rows_before += s_cap[h]; git_before += s_git[h]; dit_before += s_dit[h]; }
-    const int u = br * n + tid, w = lm_block * n + tid;
+    const int u = br * nl + tid, w = lm_block * nl + tid;
     p.seg_off[u] = p.seg_base[br] + rows_before;
     p.gather_off[w] = p.gather_base[lm_block] + git_before;
     p.dec_off[w] = p.dec_base[lm_block] + dit_before;
-    if (tid == n - 1) {
-      // the block must end exactly where the host placed the next one
-      const bool fits = p.seg_base[br] + rows_before + s_cap[tid] == p.seg_base[br + 1] &&
-                        p.gather_base[lm_block] + git_before + s_git[tid] == p.gather_base[lm_block + 1] &&
-                        p.dec_base[lm_block] + dit_before + s_dit[tid] == p.dec_base[lm_block + 1];
+    if (tid == nl - 1) {
+      // The block must end exactly where the host placed the next one.  (A shard cannot know how many of the layer's
+      // full-cache heads it will hold, so its blocks are sized for the most it can get and may end early: rows and
+      // work items between a block's end and the next block's start stay unused, and the kernels skip such items.)
+      const int64_t end_rows = p.seg_base[br] + rows_before + s_cap[tid];
+      const int end_git = p.gather_base[lm_block] + git_before + s_git[tid];
+      const int end_dit = p.dec_base[lm_block] + dit_before + s_dit[tid];
+      const bool sharded = n != nl;
+      const bool fits = sharded ? (end_rows <= p.seg_base[br + 1] && end_git <= p.gather_base[lm_block + 1] &&
+                                   end_dit <= p.dec_base[lm_block + 1])
+                                : (end_rows == p.seg_base[br + 1] && end_git == p.gather_base[lm_block + 1] &&
+                                   end_dit == p.dec_base[lm_block + 1]);
       if (!fits) set_status(p.status, TASKKV_ESTATE);
       if (br == B * p.R - 1) p.seg_off[p.U] = p.seg_base[br + 1];
       if (lm_block == B * p.R - 1) {
@@ -124,7 +134,7 @@ __global__ void __launch_bounds__(128) budget_kernel(DeviceProblem p, UnitRange 
   const int i = blockIdx.x * blockDim.x + threadIdx.x;
   if (i >= ur.blocks) return;
   const int u = ur.unit(i);
-  const int n = p.n_kv, br = u / n;
+  const int n = p.n_kv_model, br = u / p.n_kv;      // Eq. 16 and Eq. 17 count over the model's heads
   const int N = p.unit_N[u];
   int f = max(0, min(p.nhet[br], n));
   int h = min(n, f + ((p.promote_center && f < n) ? 1 : 0));

@@ -74,3 +74,19 @@ def shard_pool_rows_bound(seq_len: int, n_local: int, full_heads: int, kept_len:
     has heads."""
     h = min(full_heads, n_local)
     return h * (seq_len + max_new_tokens) + (n_local - h) * (kept_len + max_new_tokens)
+
+
+def compress_head_sharded(params, q_win, k, v, stream=None):
+    """One rank's part of a head-sharded compression: Eq. 12-15 for its own heads, the all-gather of the semantic
+    vectors, then separator, allocation and gather.  `params` is a binding.Params with shard_kv_heads > 0 and
+    shard_first = shard_heads(...)[0]; the tensors hold this rank's heads.  Returns the rank's cache."""
+    from . import binding as tk
+    cache = tk.taskkv_compress_shard_begin(params, q_win, k, v, stream=stream)
+    local = cache.semantic_vectors()
+    if stream is not None:
+        stream.synchronize()                     # the collective runs on the process group's own stream
+    else:
+        torch.cuda.current_stream().synchronize()
+    sem_all = allgather_semantic_vectors(local, params.c.shard_kv_heads).contiguous()
+    cache.taskkv_compress_shard_finish(sem_all, stream=stream)
+    return cache

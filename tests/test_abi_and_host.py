@@ -122,6 +122,11 @@ def test_invalid_arguments_are_rejected_before_any_launch(tk):
     assert tk.lib.taskkv_decode_step(None, None, None, None, None, None) == tk.EINVAL
     assert tk.lib.taskkv_decode_step_ex(None, None, None, None, None, 0, 1, None) == tk.EINVAL
     assert tk.lib.taskkv_cache_query(None, 0, None, 0) == tk.EINVAL
+    assert tk.lib.taskkv_cache_create(None, None, 0, None, 0, None, C.byref(h)) == tk.EINVAL
+    assert tk.lib.taskkv_compress_layer(None, 0, None, None, None, None, None) == tk.EINVAL
+    assert tk.lib.taskkv_compress_shard_begin(None, None, None, None, None, None, 0, None, 0, None, C.byref(h)) == tk.EINVAL
+    assert tk.lib.taskkv_compress_shard_finish(None, None, None) == tk.EINVAL
+    assert tk.lib.taskkv_cache_semantic(None, None, None) == tk.EINVAL
     assert tk.lib.taskkv_exact_semantic(None, None, None, 1, 8, 8, 128, 512, None, None, None, 0, None) == tk.EINVAL
     # argument checks come before any device work: a head dimension or a head grouping the kernels do not take
     assert tk.lib.taskkv_exact_semantic(16, 16, 16, 1, 8, 8, 96, 512, 16, None, None, 0, None) == tk.EINVAL
@@ -134,3 +139,35 @@ def test_invalid_arguments_are_rejected_before_any_launch(tk):
     assert tk.lib.taskkv_exact_semantic(256, 256, 256, 1, 8, 8, 128, 4096, 256, None, 256, 1024, None) == tk.EALLOC
     assert tk.lib.taskkv_status_str(tk.ESTATE) == b"cache in wrong state"
     assert wl.retained_rows() == 3 * 512 + 5 * 68
+
+
+def test_plan_of_a_head_shard_is_the_upper_bound(tk):
+    """A shard cannot know how many of a layer's full-cache heads it will hold: its pools are planned for
+    min(full heads of the layer, its own heads) per (sequence, layer), Eq. 16 and Eq. 17 counting over the model's heads."""
+    from paper_2501_15113_b200 import sharding
+    n_model, R, lens, s1, s2, k, mn = 8, 4, [3000, 1700], 4, 64, 100, 5
+    nh = [[tk.taskkv_hetero_count(n_model, 0.3, 1, R, r) for r in range(R)]] * 2       # 2, 2, 1, 1 far heads of 8
+    for (h0, h1) in ((0, 3), (3, 8), (0, 1)):
+        nl = h1 - h0
+        p = tk.Params(n_layers=R, n_heads=2 * nl, n_kv_heads=nl, head_dim=128, seq_lens=lens, sink=s1, recent=s2,
+                      mid_budget=k, window=32, dtype="bf16", beta=0.3, m_top=1, max_new_tokens=mn,
+                      shard_kv_heads=n_model, shard_first=h0)
+        info = tk.taskkv_plan(p)
+        want = sum(sharding.shard_pool_rows_bound(N, nl, nh[0][r] + 1, s1 + s2 + k, mn) for N in lens for r in range(R))
+        assert info.pool_rows == want and info.n_units == 2 * R * nl
+    # out-of-range shards are refused
+    for bad in (dict(shard_kv_heads=8, shard_first=6), dict(shard_kv_heads=2, shard_first=0), dict(shard_kv_heads=-1)):
+        kw = dict(n_layers=R, n_heads=6, n_kv_heads=3, head_dim=128, seq_lens=lens, sink=s1, recent=s2, mid_budget=k,
+                  window=32, dtype="bf16")
+        kw.update(bad)
+        with pytest.raises(tk.TaskKVError):
+            tk.taskkv_plan(tk.Params(**kw))
+    # budgets from a fraction count the model's heads too
+    p = tk.Params(n_layers=1, n_heads=4, n_kv_heads=2, head_dim=128, seq_lens=[4000], sink=s1, recent=s2, mid_budget=0,
+                  window=32, dtype="bf16", n_hetero=[[2]], budget_frac=0.5, shard_kv_heads=8, shard_first=2)
+    kmid = O.mid_budget(0.5 * 8 * 4000, 4000, 3, 8, s1, s2)
+    assert tk.taskkv_plan(p).pool_rows == 2 * 4000            # both of its heads may be full ones
+    p0 = tk.Params(n_layers=1, n_heads=4, n_kv_heads=2, head_dim=128, seq_lens=[4000], sink=s1, recent=s2, mid_budget=0,
+                   window=32, dtype="bf16", n_hetero=[[0]], promote_center=False, budget_frac=0.5, shard_kv_heads=8,
+                   shard_first=2)
+    assert tk.taskkv_plan(p0).pool_rows == 2 * (s1 + s2 + O.mid_budget(0.5 * 8 * 4000, 4000, 0, 8, s1, s2)) and kmid > 0

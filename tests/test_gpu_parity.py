@@ -1032,3 +1032,92 @@ def test_host_buffer_calls_return_the_sticky_device_status():
         cache.taskkv_decode_host(q, None, None, out)             # sticky
     assert ei.value.status == tk.ESTATE
     cache.close()
+
+
+# ---------------------------------------------------------------------------
+# Head sharding: the KV heads of every layer split over ranks (here: over caches on one GPU, one after the other)
+# ---------------------------------------------------------------------------
+@pytest.mark.parametrize("case", [
+    dict(G=2, splits=[(0, 3), (3, 8)], dtype="bf16", frac=0.0),          # uneven shards, 64 window rows
+    dict(G=4, splits=[(0, 2), (2, 4), (4, 8)], dtype="bf16", frac=0.35),  # three shards, 128 rows, budget as a fraction
+    dict(G=1, splits=[(0, 4), (4, 8)], dtype="f32", frac=0.0),            # CUDA-core path
+], ids=["g2_uneven", "g4_three_budget_frac", "f32"])
+def test_head_sharded_compression_equals_the_unsharded_call(case):
+    """Every shard runs Eq. 12-15 for its own heads (taskkv_compress_shard_begin), the semantic vectors of all shards
+    are put side by side in head order (what the ranks' all-gather produces), and every shard finishes with the
+    separator over all of them.  Vectors, distances, classes, lengths, retained positions, cache rows and decode
+    outputs of every head must be those of the unsharded call, bit for bit; so must the layer's heterogeneous heads,
+    wherever they land (one shard gets none of them in some layers, all of them in others)."""
+    tk, P = _tk(), _parity()
+    G, n_kv = case["G"], 8
+    wl = small("sharded", n=n_kv * G, n_kv=n_kv, d=128 if case["dtype"] == "bf16" else 64, N=0, L=32 if G < 4 else 32,
+               s1=4, s2=64, k=140, dtype=case["dtype"], R=3, seq_lens=[2100, 1300], nh=2, steps=2)
+    wl.mid_budget = [140, 60, 200]
+    wl.n_hetero = [[2, 0, 5], [1, 3, 7]]
+    wl.planted = W._choose_planted(wl)
+    if case["frac"] > 0:
+        wl.budget_frac = case["frac"]
+        wl.mid_by_seq = [[O.mid_budget(case["frac"] * n_kv * wl.seq_lens[b], wl.seq_lens[b], wl.full_heads(b, r), n_kv,
+                                       wl.sink, wl.recent) for r in range(3)] for b in range(2)]
+    qs, ks, vs = W.materialize(wl, DEV)
+    whole = tk.taskkv_compress_ex(tk.params_from_workload(wl, max_new_tokens=wl.decode_steps), qs, ks, vs)
+    assert whole.status() == 0
+    w_cls, w_len, w_dist = whole.classes(), whole.lengths(), whole.query(tk.Q_DIST)
+    w_sem, w_idx = whole.query(tk.Q_SEMVEC), whole.query(tk.Q_INDICES)
+
+    shards = []
+    for (h0, h1) in case["splits"]:
+        params = tk.params_from_workload(wl, max_new_tokens=wl.decode_steps, n_heads=(h1 - h0) * G, n_kv_heads=h1 - h0,
+                                         shard_kv_heads=n_kv, shard_first=h0)
+        ql = [x[:, h0 * G:h1 * G].contiguous() for x in qs]
+        kl = [x[:, h0:h1].contiguous() for x in ks]
+        vl = [x[:, h0:h1].contiguous() for x in vs]
+        shards.append((h0, h1, tk.taskkv_compress_shard_begin(params, ql, kl, vl), (ql, kl, vl)))
+    # what an all-gather of the shards' vectors gives every rank
+    sem_all = torch.cat([c.semantic_vectors() for (_, _, c, _) in shards], dim=1).contiguous()
+    assert np.array_equal(sem_all.cpu().numpy().reshape(-1, sem_all.shape[-1]), w_sem)
+    for (_, _, c, _) in shards:
+        with pytest.raises(tk.TaskKVError):
+            tk.taskkv_compress_ex(c.params, *shards[0][3])           # a shard cannot be compressed in one call
+        c.taskkv_compress_shard_finish(sem_all)
+        assert c.status() == 0
+    with pytest.raises(tk.TaskKVError) as ei:
+        shards[0][2].taskkv_compress_shard_finish(sem_all)
+    assert ei.value.status == tk.ESTATE
+
+    R = wl.n_layers
+    full_seen = set()
+    for (h0, h1, c, _) in shards:
+        nl = h1 - h0
+        cls, lens, dist, idx = c.classes(), c.lengths(), c.query(tk.Q_DIST), c.query(tk.Q_INDICES)
+        assert int(lens.sum()) <= int(c.info.retained_rows)          # the plan is an upper bound for a shard
+        for b in range(wl.batch):
+            for r in range(R):
+                full_seen.add(int((cls[(b * R + r) * nl:(b * R + r + 1) * nl] != 0).sum()))
+                for h in range(h0, h1):
+                    u, us = (b * R + r) * n_kv + h, (b * R + r) * nl + h - h0
+                    assert int(cls[us]) == int(w_cls[u]) and int(lens[us]) == int(w_len[u])
+                    assert dist[us] == w_dist[u]
+                    if lens[us] < wl.seq_lens[b]:
+                        assert np.array_equal(idx[us, :lens[us]], w_idx[u, :lens[us]])
+                    for which in ("k", "v"):
+                        assert torch.equal(c.pool_rows(which, us).view(torch.uint8),
+                                           whole.pool_rows(which, u).view(torch.uint8))
+    assert 0 in full_seen and max(full_seen) >= 3                    # shards without and with many full heads
+    # and the unsharded result is the oracle's
+    rep = P.Report()
+    ref = P.oracle_layer(wl, 1, 2, qs[1][2], ks[1][2], vs[1][2])
+    P.compare_layer(whole, wl, 1, 2, ref, rep, v=vs[1][2])
+    rep.check_bounds(wl.name)
+    # decode: a shard's outputs are the unsharded outputs of its query heads
+    for s_ in range(wl.decode_steps):
+        q, kn, vn = W.gen_decode_step(wl, s_, DEV)
+        want = whole.taskkv_decode_step(q, kn, vn)
+        for (h0, h1, c, _) in shards:
+            got = c.taskkv_decode_step(q[:, :, h0 * G:h1 * G].contiguous(), kn[:, :, h0:h1].contiguous(),
+                                       vn[:, :, h0:h1].contiguous())
+            assert torch.equal(got.view(torch.uint8), want[:, :, h0 * G:h1 * G].contiguous().view(torch.uint8))
+            assert c.status() == 0
+    whole.close()
+    for (_, _, c, _) in shards:
+        c.close()
