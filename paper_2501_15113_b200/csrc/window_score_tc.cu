@@ -365,6 +365,11 @@ window_tc_kernel(const __grid_constant__ TcMaps maps, DeviceProblem p, const __g
         __syncwarp();
         fetch_stats(k + 1);                 // in flight while this item's tiles are worked on
       }
+      // Which of the item's tiles this group takes depends on how many tiles the CTA has seen before (n): with n even
+      // at the item's start it is the even ones.  The partial statistics below are filed under that parity, not under
+      // the group, so that a slot always holds the same tiles (and keys) whatever else the CTA worked on before:
+      // results do not depend on how a problem is cut into launches.
+      const int par = grp ^ (n & 1);                 // parity, within the item, of the tiles this warp takes
       for (int t = 0; t < ntiles; ++t, ++n) {
         if ((n & 1) != grp) continue;
         const int acc = n & 3;
@@ -505,15 +510,17 @@ window_tc_kernel(const __grid_constant__ TcMaps maps, DeviceProblem p, const __g
       }
       if (!ok) break;
       if (a.pass == 1) {
-        // the warp's own partial of this item: slot (chunk, part), part = warp (group with 128 rows)
+        // the warp's partial of this item: slot (chunk, part), part = (tile parity, lane quadrant); with 128 rows a
+        // quadrant is a set of rows, so there part = tile parity
         float2* slot = reinterpret_cast<float2*>(p.stat_part) +
                        ((size_t)u * p.chunks_max + (size_t)it.ch * (rows == 128 ? 2 : kTcParts)) * p.rows_pad;
         if (rows == 128) {
-          slot[(size_t)grp * p.rows_pad + quad * 32 + lane] = make_float2(m_run[0] * scale2, z_run[0]);
+          slot[(size_t)par * p.rows_pad + quad * 32 + lane] = make_float2(m_run[0] * scale2, z_run[0]);
         } else {
 #pragma unroll
           for (int rg = 0; rg < 4; ++rg)
-            if (rg * 32 < rows) slot[(size_t)ew * p.rows_pad + rg * 32 + lane] = make_float2(m_run[rg] * scale2, z_run[rg]);
+            if (rg * 32 < rows)
+              slot[(size_t)(par * 4 + quad) * p.rows_pad + rg * 32 + lane] = make_float2(m_run[rg] * scale2, z_run[rg]);
         }
       }
     }

@@ -477,12 +477,13 @@ def test_ragged_batch_of_eleven_sequences():
     run_workload(wl)
 
 
-@pytest.mark.parametrize("n_hetero,mid", [(0, 64), (2, 256), (8, 1024)])
+@pytest.mark.parametrize("n_hetero,mid", [(h, k) for h in W.SWEEP_HETERO for k in W.SWEEP_MID])
 def test_budget_sweep_points(n_hetero, mid):
-    """Config 5 scaled down: planted fraction x middle budget."""
+    """Config 5 scaled down, all 15 points: planted fraction (0, 1, 2, 4, 8 of 8 heads) x middle budget (64, 256, 1024)."""
     from paper_2501_15113_b200 import configs
     wl = configs.config5_sweep(n_hetero, mid, seq_len=5000, batch=2, decode_steps=2)
-    run_workload(wl)
+    rep = run_workload(wl)
+    assert rep.units == 16
 
 
 # ---------------------------------------------------------------------------
@@ -668,10 +669,14 @@ STREAM_CASES = [
     dict(n=8, n_kv=8, d=128, N=0, L=32, s1=4, s2=64, k=120, dtype="bf16", R=3, seq_lens=[3000, 4500], nh=2),
     # fp32 on the CUDA cores
     dict(n=4, n_kv=4, d=64, N=0, L=16, s1=4, s2=32, k=50, dtype="f32", R=3, seq_lens=[900, 700], nh=1),
+    # 64 window rows, enough units for every CTA of the all-layer window-score launch to work through several items
+    # whose tile counts are odd (9 and 19 tiles), while the per-layer launches give every CTA one item: the partial
+    # row statistics must not depend on what a CTA worked on before
+    dict(n=16, n_kv=8, d=64, N=0, L=32, s1=4, s2=64, k=70, dtype="bf16", R=8, seq_lens=[2400, 1150, 3300], nh=1),
 ]
 
 
-@pytest.mark.parametrize("case", STREAM_CASES, ids=["bf16_gqa_ragged", "bf16_mha", "f32"])
+@pytest.mark.parametrize("case", STREAM_CASES, ids=["bf16_gqa_ragged", "bf16_mha", "f32", "bf16_64rows_many_items"])
 def test_layers_streamed_into_one_cache_equal_the_all_layer_call(case):
     """taskkv_cache_create + one taskkv_compress_layer per layer, in a scrambled order and with every layer's
     tensors in allocations of their own, against taskkv_compress_ex over all layers: semantic vectors, distances,
@@ -691,7 +696,7 @@ def test_layers_streamed_into_one_cache_equal_the_all_layer_call(case):
 
     streamed = tk.taskkv_cache_create(params, DEV)
     assert streamed.lengths().tolist() == [0] * (wl.batch * R * wl.n_kv_heads)
-    order = list(range(R))[::-1] if R < 4 else [2, 0, 3, 1]
+    order = list(range(R))[::-1] if R != 4 else [2, 0, 3, 1]
     layer_inputs = {r: ([x[r].clone() for x in qs], [x[r].clone() for x in ks], [x[r].clone() for x in vs])
                     for r in range(R)}
     q0, kn0, vn0 = W.gen_decode_step(wl, 0, DEV)
