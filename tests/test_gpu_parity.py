@@ -604,6 +604,45 @@ def test_layer_by_layer_decode_equals_all_layer_decode(case):
     split.close()
 
 
+def test_layer_decode_equals_all_layer_decode_with_many_work_items():
+    """Layer-range calls against the all-layer call on a cache with 640 split-K work items per layer (every head keeps
+    40447 rows): a layer's grid is sized by its own items, the all-layer grid by all 2560, so blocks walk the items in
+    different orders; the outputs must be the same bits, for plain decode, for prefix lengths and for the fused step,
+    whose appended rows sit in the last item of every unit."""
+    tk = _tk()
+    wl = small("by_warp", n=16, n_kv=8, d=128, N=40447, L=32, s1=4, s2=64, k=100, dtype="bf16", R=4, nh=0, steps=3)
+    qs, ks, vs = W.materialize(wl, DEV)
+    params = tk.params_from_workload(wl, max_new_tokens=3, force_class=1)      # every head keeps all 40447 rows
+    whole = tk.taskkv_compress_ex(params, qs, ks, vs)
+    split = tk.taskkv_compress_ex(params, qs, ks, vs)
+    assert int(whole.info.max_decode_items) == 4 * 8 * 80          # (40447 + 3 reserved rows) / 512, rounded up
+    R = wl.n_layers
+    q, kn, vn = W.gen_decode_step(wl, 0, DEV)
+    want = whole.taskkv_decode(q)
+    for r in range(R):
+        got = split.taskkv_decode_ex(q[:, r:r + 1].contiguous(), r, 1)
+        assert torch.equal(got.view(torch.uint8), want[:, r:r + 1].contiguous().view(torch.uint8)), f"layer {r}"
+    lens = torch.from_numpy(whole.lengths().reshape(1, R, 8)).to(DEV).to(torch.int32)
+    part = (lens * 2 // 3).contiguous()
+    want = whole.taskkv_decode(q, lengths=part)
+    got = split.taskkv_decode_ex(q[:, 2:3].contiguous(), 2, 1, lengths=part[:, 2:3].contiguous())
+    assert torch.equal(got.view(torch.uint8), want[:, 2:3].contiguous().view(torch.uint8))
+    for s_ in range(3):
+        q, kn, vn = W.gen_decode_step(wl, s_, DEV)
+        want = whole.taskkv_decode_step(q, kn, vn)
+        for r in range(R):
+            got = split.taskkv_decode_step_ex(q[:, r:r + 1].contiguous(), kn[:, r:r + 1].contiguous(),
+                                              vn[:, r:r + 1].contiguous(), r, 1)
+            assert torch.equal(got.view(torch.uint8), want[:, r:r + 1].contiguous().view(torch.uint8)), f"step {s_} layer {r}"
+        assert np.array_equal(whole.lengths(), split.lengths())
+    for u in (0, 13, 31):
+        for which in ("k", "v"):
+            assert torch.equal(whole.pool_rows(which, u)[-4:].view(torch.uint8), split.pool_rows(which, u)[-4:].view(torch.uint8))
+    assert whole.status() == 0 and split.status() == 0
+    whole.close()
+    split.close()
+
+
 def test_one_layer_problems_equal_the_all_layer_compression():
     """Compressing layer r alone as a problem of its own (Params.layer: that layer's head count and budget) gives the same
     classes, lengths, positions, cache rows and decode outputs as the all-layer call gives for layer r."""
