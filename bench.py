@@ -328,6 +328,7 @@ def run_ours(args):
         line["latency_mode"] = run_latency_mode(tk, wl, qs, ks, vs, steps_in, args)
         line["layer_streamed_compress"] = run_layer_streamed(tk, wl, qs, ks, vs, args, steps_in)
         line["compress_with_window_lse"] = run_with_window_lse(tk, wl, qs, ks, vs, args, comp_bytes, peak)
+        line["paged_cache"] = run_paged(tk, wl, qs, ks, vs, steps_in, args, comp_bytes, res["hbm"]["decode_bytes_per_step"], peak)
         if wl.seq_lens[0] <= 32768:
             line["exact_semantic"] = run_exact_semantic(tk, wl, qs, ks, vs)
     if rank == 0 and not args.no_e2e:
@@ -392,6 +393,53 @@ def run_latency_mode(tk, wl, qs, ks, vs, steps_in, args, n_steps=16):
     out["device_status"] = cache.status()
     cache.close()
     return out
+
+
+def run_paged(tk, wl, qs, ks, vs, steps_in, args, comp_bytes, decode_bytes, peak):
+    """The same compression and decode steps with the rows in pages of a shared pool (block tables), as a serving
+    engine would hold them: compression time, time of a fused decode step, both against the same algorithmic bytes
+    as the contiguous cache."""
+    import torch
+    n_dec = len(steps_in)
+    params = tk.params_from_workload(wl, max_new_tokens=4 * n_dec + 4, mid_policy=POLICIES[args.policy])
+    P = args.page_rows
+    info, pages = tk.taskkv_plan_paged(params, P)
+    pool = tk.Pool(P, pages + 2 * int(info.n_units), wl.head_dim, wl.dtype, qs[0].device)
+    stream = torch.cuda.current_stream()
+
+    def timed(fn):
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        torch.cuda.synchronize()
+        e0.record(stream)
+        r = fn()
+        e1.record(stream)
+        torch.cuda.synchronize()
+        return e0.elapsed_time(e1), r
+
+    comp, dec = [], []
+    status = 0
+    for it in range(4):
+        ms, cache = timed(lambda: tk.taskkv_compress_paged(params, qs, ks, vs, pool))
+        out = torch.empty_like(steps_in[0][0])
+
+        def steps():
+            for (q, kn, vn) in steps_in:
+                cache.taskkv_decode_step(q, kn, vn, out=out)
+
+        msd, _ = timed(steps)
+        if it:
+            comp.append(ms)
+            dec.append(msd / n_dec)
+        status = max(status, cache.status())
+        cache.close()
+    free_after = pool.free_pages()
+    n_pages = pool.n_pages
+    pool.close()
+    cms, dms = statistics.median(comp), statistics.median(dec)
+    return {"page_rows": P, "pages": pages, "pool_pages": n_pages, "all_pages_returned": free_after == n_pages,
+            "compress_ms": cms, "compress_frac_of_peak": comp_bytes / (cms * 1e-3) / 1e9 / peak,
+            "decode_ms_per_step": dms, "decode_frac_of_peak": decode_bytes / (dms * 1e-3) / 1e9 / peak,
+            "device_status": status}
 
 
 def run_layer_streamed(tk, wl, qs, ks, vs, args, steps_in):
@@ -734,6 +782,7 @@ def main():
     ap.add_argument("--policy", default="select", choices=sorted(POLICIES),
                     help="what a non-heterogeneous head keeps beside sinks and recent window (Sec. V-G)")
     ap.add_argument("--no-latency", action="store_true", help="skip the layer-by-layer decode measurement")
+    ap.add_argument("--page-rows", type=int, default=256, help="page size of the paged-cache measurement")
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--no-cpu", action="store_true")
     ap.add_argument("--no-extra", action="store_true", help="skip the other workloads (grouped-query, batch, sweep)")

@@ -247,6 +247,37 @@ taskkv_status taskkv_compress_shard_begin(const taskkv_params* p, const void* co
 taskkv_status taskkv_cache_semantic(const taskkv_cache* c, const float** device_ptr, int64_t* n_floats);
 taskkv_status taskkv_compress_shard_finish(taskkv_cache* c, const float* sem_all, taskkv_stream stream);
 
+/* Paged cache (block tables), for serving.  Per-head caches of different and growing lengths fragment memory when
+ * every batch owns contiguous pools with a reserve per unit; here the K and V rows of every cache live in pages of
+ * page_rows rows taken from one pool, each unit has a table of its pages, pages for appended tokens are taken when a
+ * unit's last page is full, and destroying a cache returns its pages for the next one.
+ *   taskkv_pool_create    a pool of n_pages pages of page_rows rows (a multiple of 64) of head_dim elements of
+ *                         `dtype`, for K and for V, in `mem` (device, 256-byte aligned, at least
+ *                         taskkv_pool_bytes(...) bytes, owned by the caller) or, with mem == NULL, in memory the
+ *                         library allocates.
+ *   taskkv_compress_paged as taskkv_compress_ex, with the compacted rows going to pages of `pool`; cache_mem then
+ *                         holds only tables (taskkv_plan_paged gives the sizes and the pages the compression takes).
+ *                         max_new_tokens still bounds how far a unit may grow (it sizes the page tables and the
+ *                         decode work lists) but reserves no rows.
+ * Every other call (append, decode, decode_step, layer ranges, queries, destroy) works on a paged cache as on any
+ * other; results are bit for bit those of the contiguous layout.  The library keeps count of the pool's free pages on
+ * the host (how many pages a call takes follows from the schedules, not from the data) and refuses a compression or an
+ * append that would not fit with EALLOC before anything is launched.  Calls that use one pool -- compressions,
+ * appends and decode steps of its caches, and their destruction -- must be ordered with respect to one another by the
+ * caller (one stream, or events); the pool must outlive its caches.
+ * A paged cache cannot be head-sharded or filled layer by layer (EINVAL). */
+typedef struct taskkv_pool taskkv_pool;
+size_t        taskkv_pool_bytes(int32_t page_rows, int32_t n_pages, int32_t head_dim, int32_t dtype);
+taskkv_status taskkv_pool_create(int32_t page_rows, int32_t n_pages, int32_t head_dim, int32_t dtype, void* mem,
+                                 size_t bytes, taskkv_stream stream, taskkv_pool** out_pool);
+int32_t       taskkv_pool_free_pages(const taskkv_pool* pool);      /* the host's count; -1 for a NULL pool */
+void          taskkv_pool_destroy(taskkv_pool* pool);
+taskkv_status taskkv_plan_paged(const taskkv_params* p, int32_t page_rows, taskkv_plan_info* out, int64_t* pages_needed);
+taskkv_status taskkv_compress_paged(const taskkv_params* p, const void* const* q_win, const void* const* k,
+                                    const void* const* v, taskkv_pool* pool, void* cache_mem, size_t cache_bytes,
+                                    void* workspace_mem, size_t workspace_bytes, taskkv_stream stream,
+                                    taskkv_cache** out_cache);
+
 /* The flat form of the same call: one bf16 sequence, Sec. V-D defaults for
  * everything not listed, library-owned memory, max_new_tokens = 4096. */
 taskkv_status taskkv_compress(const void* q_win, const void* k, const void* v,
@@ -350,6 +381,8 @@ taskkv_status taskkv_decode_noalloc(const void* q, const void* k_pool, const voi
 #define TASKKV_Q_KPOOL     9   /* raw K pool bytes */
 #define TASKKV_Q_VPOOL    10   /* raw V pool bytes */
 #define TASKKV_Q_CAPACITY 11   /* int32 [n_units] */
+#define TASKKV_Q_PAGETAB  12   /* int32 [n_units][page_stride]: page ids of each unit's rows, in order (paged caches);
+                                  with it TASKKV_Q_KPOOL / TASKKV_Q_VPOOL return the pool's pages */
 int64_t       taskkv_cache_query_bytes(const taskkv_cache* c, int32_t what);
 taskkv_status taskkv_cache_query(const taskkv_cache* c, int32_t what, void* host_dst, size_t bytes);
 taskkv_status taskkv_cache_plan(const taskkv_cache* c, taskkv_plan_info* out);

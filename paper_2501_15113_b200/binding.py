@@ -27,7 +27,7 @@ lib = C.CDLL(LIB_PATH)
 OK, EINVAL, EALLOC, ECUDA, ETIMEOUT, ESTATE = 0, -1, -2, -3, -4, -5
 F32, BF16 = 0, 1
 (Q_LENGTHS, Q_CLASSES, Q_DIST, Q_SEMVEC, Q_OFFSETS, Q_INDICES, Q_SCORES, Q_TOPT, Q_STATUS, Q_KPOOL,
- Q_VPOOL, Q_CAPACITY) = range(12)
+ Q_VPOOL, Q_CAPACITY, Q_PAGETAB) = range(13)
 
 
 class taskkv_params(C.Structure):
@@ -69,6 +69,19 @@ lib.taskkv_cache_semantic.argtypes = [_vp, C.POINTER(_vp), C.POINTER(C.c_int64)]
 lib.taskkv_cache_semantic.restype = C.c_int32
 lib.taskkv_compress_shard_finish.argtypes = [_vp, _vp, _vp]
 lib.taskkv_compress_shard_finish.restype = C.c_int32
+lib.taskkv_pool_bytes.argtypes = [C.c_int32] * 4
+lib.taskkv_pool_bytes.restype = C.c_size_t
+lib.taskkv_pool_create.argtypes = [C.c_int32] * 4 + [_vp, C.c_size_t, _vp, C.POINTER(_vp)]
+lib.taskkv_pool_create.restype = C.c_int32
+lib.taskkv_pool_free_pages.argtypes = [_vp]
+lib.taskkv_pool_free_pages.restype = C.c_int32
+lib.taskkv_pool_destroy.argtypes = [_vp]
+lib.taskkv_pool_destroy.restype = None
+lib.taskkv_plan_paged.argtypes = [C.POINTER(taskkv_params), C.c_int32, C.POINTER(taskkv_plan_info), C.POINTER(C.c_int64)]
+lib.taskkv_plan_paged.restype = C.c_int32
+lib.taskkv_compress_paged.argtypes = [C.POINTER(taskkv_params), _pp, _pp, _pp, _vp, _vp, C.c_size_t, _vp, C.c_size_t,
+                                      _vp, C.POINTER(_vp)]
+lib.taskkv_compress_paged.restype = C.c_int32
 lib.taskkv_compress_lse.argtypes = [C.POINTER(taskkv_params), _pp, _pp, _pp, _pp, _vp, C.c_size_t, _vp, C.c_size_t,
                                     _vp, C.POINTER(_vp)]
 lib.taskkv_compress_lse.restype = C.c_int32
@@ -382,6 +395,8 @@ class Cache:
         U = int(self.info.n_units)
         if what in (Q_LENGTHS, Q_CLASSES, Q_CAPACITY, Q_STATUS):
             return buf.view(np.int32)
+        if what == Q_PAGETAB:
+            return buf.view(np.int32).reshape(U, -1)
         if what == Q_DIST:
             return buf.view(np.float32)
         if what == Q_SEMVEC:
@@ -406,15 +421,26 @@ class Cache:
         return int(self.query(Q_STATUS)[0])
 
     def pool_rows(self, which: str, u: int) -> torch.Tensor:
-        """Rows of unit u's K ('k') or V ('v') segment as a CPU tensor [len_u, d]."""
-        off = self.query(Q_OFFSETS)
-        ln = self.query(Q_LENGTHS)
-        raw = self.query(Q_KPOOL if which == "k" else Q_VPOOL)
+        """Rows of unit u's K ('k') or V ('v') segment as a CPU tensor [len_u, d] (for a paged cache: gathered from
+        the unit's pages in order)."""
+        ln = int(self.query(Q_LENGTHS)[u])
         d = self.params.c.head_dim
         es = 2 if self.params.c.dtype == BF16 else 4
-        seg = raw[int(off[u]) * d * es:(int(off[u]) + int(ln[u])) * d * es]
+        raw = self.query(Q_KPOOL if which == "k" else Q_VPOOL)
+        if self._keep is not None and "pool" in self._keep:
+            P = self._keep["pool"].page_rows
+            tab = self.query(Q_PAGETAB)[u]
+            parts = []
+            for i in range((ln + P - 1) // P):
+                rows = min(P, ln - i * P)
+                start = int(tab[i]) * P * d * es
+                parts.append(raw[start:start + rows * d * es])
+            seg = np.concatenate(parts) if parts else raw[:0]
+        else:
+            off = self.query(Q_OFFSETS)
+            seg = raw[int(off[u]) * d * es:(int(off[u]) + ln) * d * es]
         t = torch.from_numpy(seg.copy())
-        return t.view(self.params.torch_dtype).reshape(int(ln[u]), d)
+        return t.view(self.params.torch_dtype).reshape(ln, d)
 
     def retained_indices(self, u: int, N: int) -> np.ndarray:
         ln = int(self.query(Q_LENGTHS)[u])
@@ -490,6 +516,58 @@ def taskkv_compress_shard_begin(params: Params, q_win: Sequence[torch.Tensor], k
                                            workspace_mem.numel(), _stream_handle(stream), C.byref(h)),
            "taskkv_compress_shard_begin")
     return Cache(h.value, params, {"cache": cache_mem, "workspace": workspace_mem})
+
+
+class Pool:
+    """A page pool for paged caches (taskkv_pool*) plus the torch buffer backing it."""
+
+    def __init__(self, page_rows: int, n_pages: int, head_dim: int, dtype, device, stream=None):
+        dt = BF16 if dtype in (BF16, "bf16", torch.bfloat16) else F32
+        nbytes = int(lib.taskkv_pool_bytes(page_rows, n_pages, head_dim, dt))
+        if nbytes == 0:
+            raise TaskKVError(EINVAL, "taskkv_pool_bytes")
+        self.mem = torch.empty(nbytes, dtype=torch.uint8, device=device)
+        self.page_rows, self.n_pages = page_rows, n_pages
+        h = C.c_void_p()
+        with torch.cuda.device(self.mem.device):
+            _check(lib.taskkv_pool_create(page_rows, n_pages, head_dim, dt, self.mem.data_ptr(), nbytes,
+                                          _stream_handle(stream), C.byref(h)), "taskkv_pool_create")
+        self._h = h
+
+    def free_pages(self) -> int:
+        return int(lib.taskkv_pool_free_pages(self._h))
+
+    def close(self):
+        if self._h:
+            lib.taskkv_pool_destroy(self._h)
+            self._h = None
+            self.mem = None
+
+
+def taskkv_plan_paged(params: Params, page_rows: int):
+    """(plan info, pages the compression takes) for a paged cache."""
+    info = taskkv_plan_info()
+    pages = C.c_int64()
+    _check(lib.taskkv_plan_paged(C.byref(params.c), page_rows, C.byref(info), C.byref(pages)), "taskkv_plan_paged")
+    return info, int(pages.value)
+
+
+def taskkv_compress_paged(params: Params, q_win: Sequence[torch.Tensor], k: Sequence[torch.Tensor],
+                          v: Sequence[torch.Tensor], pool: Pool, stream=None) -> Cache:
+    """As taskkv_compress_ex, the compacted rows going to pages of `pool`."""
+    info, _ = taskkv_plan_paged(params, pool.page_rows)
+    dev = k[0].device
+    cache_mem = torch.empty(int(info.cache_bytes), dtype=torch.uint8, device=dev)
+    workspace_mem = torch.empty(int(info.workspace_bytes), dtype=torch.uint8, device=dev)
+    for t in list(q_win) + list(k) + list(v):
+        if not t.is_contiguous() or not t.is_cuda:
+            raise ValueError("inputs must be contiguous CUDA tensors")
+    h = C.c_void_p()
+    _check(lib.taskkv_compress_paged(C.byref(params.c), _ptr_array(q_win), _ptr_array(k), _ptr_array(v), pool._h,
+                                     cache_mem.data_ptr(), cache_mem.numel(), workspace_mem.data_ptr(),
+                                     workspace_mem.numel(), _stream_handle(stream), C.byref(h)),
+           "taskkv_compress_paged")
+    return Cache(h.value, params, {"cache": cache_mem, "workspace": workspace_mem, "pool": pool})
 
 
 def taskkv_compress_host(params: Params, q_win: Sequence[torch.Tensor], k: Sequence[torch.Tensor],

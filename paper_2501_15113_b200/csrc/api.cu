@@ -30,6 +30,12 @@ struct HostPlan {
   // r * B + b, layer-major); one entry more than blocks
   std::vector<int64_t> seg_base;
   std::vector<int32_t> gather_base, dec_base;
+  // paged cache: rows per page (0: contiguous pools inside the cache memory), table entries per unit, pages the
+  // compression takes, rows a unit of each kind holds right after compression ([B*R] full / kept lengths)
+  int32_t page_rows = 0, page_stride = 0;
+  int64_t pages_compress = 0;
+  std::vector<int32_t> kept_len;
+  size_t o_ptab = 0;
   // byte offsets inside the cache memory
   size_t o_unit_N, o_unit_mid, o_nhet, o_c_off, o_seg_base, o_gbase, o_dbase, o_qp, o_kp, o_vp, meta_bytes;
   size_t o_status, o_len, o_cap, o_seg, o_cls, o_dist, o_sem, o_idx, o_goff, o_doff, o_step, o_pacc, o_pml, o_kpool,
@@ -58,7 +64,10 @@ int32_t mid_budget_impl(double budget_tokens, int32_t N, int32_t h_full, int32_t
   return (int32_t)k;
 }
 
-taskkv_status make_plan(const taskkv_params* p, HostPlan& hp) {
+taskkv_status make_plan(const taskkv_params* p, HostPlan& hp, int32_t page_rows = 0) {
+  if (page_rows < 0 || page_rows % kGatherRows != 0) return TASKKV_EINVAL;
+  if (page_rows > 0 && p && p->shard_kv_heads > 0) return TASKKV_EINVAL;
+  hp.page_rows = page_rows;
   if (!p || !p->seq_lens) return TASKKV_EINVAL;
   if (p->n_layers < 1 || p->batch < 1 || p->n_heads < 1 || p->n_kv_heads < 1) return TASKKV_EINVAL;
   if (p->n_kv_heads > TASKKV_MAX_KV_HEADS || p->n_heads % p->n_kv_heads != 0) return TASKKV_EINVAL;
@@ -121,6 +130,9 @@ taskkv_status make_plan(const taskkv_params* p, HostPlan& hp) {
   int32_t stride = 1;
   hp.layer_items.assign((size_t)R, 0);
   hp.seg_base.assign((size_t)B * R + 1, 0);
+  hp.kept_len.assign((size_t)B * R, 0);
+  hp.pages_compress = 0;
+  hp.page_stride = 0;
   std::vector<int64_t> blk_g((size_t)B * R, 0), blk_d((size_t)B * R, 0);   // per block b * R + r
   for (int b = 0; b < B; ++b) {
     const int64_t N = hp.seq_lens[b];
@@ -131,6 +143,11 @@ taskkv_status make_plan(const taskkv_params* p, HostPlan& hp) {
       if (N > (int64_t)s1 + s2) kept = s1 + s2 + std::min<int64_t>(hp.mid[br], N - s1 - s2);
       if (kept < N) stride = std::max<int32_t>(stride, (int32_t)kept);
       hp.seg_base[br] = pool;
+      hp.kept_len[br] = (int32_t)kept;
+      if (page_rows > 0) {
+        hp.pages_compress += h * ((N + page_rows - 1) / page_rows) + (nkv - h) * ((kept + page_rows - 1) / page_rows);
+        hp.page_stride = std::max<int32_t>(hp.page_stride, (int32_t)((N + mn + page_rows - 1) / page_rows));
+      }
       pool += h * (N + mn) + (nkv - h) * (kept + mn);
       kept_rows += h * N + (nkv - h) * kept;
       blk_g[br] = h * ((N + kGatherRows - 1) / kGatherRows) + (nkv - h) * ((kept + kGatherRows - 1) / kGatherRows);
@@ -200,8 +217,9 @@ taskkv_status make_plan(const taskkv_params* p, HostPlan& hp) {
   hp.o_step = take(U * 4);
   hp.o_pacc = take((size_t)ditems * G * d * 4);
   hp.o_pml = take((size_t)ditems * G * 2 * 4);
-  hp.o_kpool = take((size_t)pool * d * es);
-  hp.o_vpool = take((size_t)pool * d * es);
+  hp.o_ptab = take(page_rows > 0 ? (size_t)U * hp.page_stride * 4 : 0);
+  hp.o_kpool = take(page_rows > 0 ? 0 : (size_t)pool * d * es);      // a paged cache keeps its rows in the pool's pages
+  hp.o_vpool = take(page_rows > 0 ? 0 : (size_t)pool * d * es);
   const size_t cache_bytes = o;
   o = 0;
   hp.w_C = take((size_t)c_total * 4);
@@ -259,7 +277,22 @@ void note_launch_end(int32_t id, cudaStream_t s) {
 }
 }  // namespace taskkv
 
+struct taskkv_pool {
+  int32_t page_rows = 0, n_pages = 0, head_dim = 0, dtype = 0;
+  void* mem = nullptr;
+  bool own = false;
+  unsigned char* k_pages = nullptr;   // [n_pages][page_rows][d]
+  unsigned char* v_pages = nullptr;
+  int32_t* free_ids = nullptr;        // device stack of free page ids
+  int32_t* top = nullptr;             // device: number of free pages
+  int64_t free_host = 0;              // the host's count (exact: what a call takes follows from the schedules)
+  int32_t caches = 0;                 // caches alive
+};
+
 struct taskkv_cache {
+  taskkv_pool* pool = nullptr;             // paged caches
+  std::vector<int32_t> appended;           // [R] tokens appended to layer r so far (paged caches: page accounting)
+  int64_t pages_held = 0;                  // pages this cache has taken off its pool
   taskkv_params prm;
   HostPlan hp;
   DeviceProblem dp;
@@ -493,6 +526,15 @@ void fill_device_problem(taskkv_cache* c) {
   d.part_ml = reinterpret_cast<float*>(cm + hp.o_pml);
   d.k_pool = cm + hp.o_kpool;
   d.v_pool = cm + hp.o_vpool;
+  d.page_rows = hp.page_rows;
+  d.page_stride = hp.page_stride;
+  d.page_tab = reinterpret_cast<int32_t*>(cm + hp.o_ptab);
+  if (c->pool) {
+    d.k_pool = c->pool->k_pages;
+    d.v_pool = c->pool->v_pages;
+    d.pool_free = c->pool->free_ids;
+    d.pool_top = c->pool->top;
+  }
   if (wm) {
     d.C = reinterpret_cast<float*>(wm + hp.w_C);
     d.pooled = reinterpret_cast<float*>(wm + hp.w_pool);
@@ -608,7 +650,7 @@ namespace {
 taskkv_status compress_impl(const taskkv_params* p, const void* const* q_win, const void* const* k,
                             const void* const* v, const void* const* window_lse, void* cache_mem,
                             size_t cache_bytes, void* workspace_mem, size_t workspace_bytes, taskkv_stream stream,
-                            taskkv_cache** out_cache);
+                            taskkv_cache** out_cache, taskkv_pool* pool = nullptr);
 }  // namespace
 
 taskkv_status taskkv_compress_ex(const taskkv_params* p, const void* const* q_win, const void* const* k,
@@ -632,13 +674,20 @@ namespace {
 // Plans the problem, takes or allocates the memory, and puts the tables and a clean state on the device (enqueued
 // on `s`); no layer is compressed yet.
 taskkv_status cache_create_impl(const taskkv_params* p, void* cache_mem, size_t cache_bytes, void* workspace_mem,
-                                size_t workspace_bytes, cudaStream_t s, taskkv_cache** out_cache) {
+                                size_t workspace_bytes, cudaStream_t s, taskkv_cache** out_cache,
+                                taskkv_pool* pool = nullptr) {
   if (!p || !out_cache) return TASKKV_EINVAL;
   *out_cache = nullptr;
   taskkv_cache* c = new (std::nothrow) taskkv_cache();
   if (!c) return TASKKV_EALLOC;
-  taskkv_status st = make_plan(p, c->hp);
+  taskkv_status st = make_plan(p, c->hp, pool ? pool->page_rows : 0);
   if (st != TASKKV_OK) { delete c; return st; }
+  if (pool) {
+    if (pool->head_dim != p->head_dim || pool->dtype != p->dtype) { delete c; return TASKKV_EINVAL; }
+    if (c->hp.pages_compress > pool->free_host) { delete c; return TASKKV_EALLOC; }     // would not fit: nothing launched
+    c->pool = pool;
+  }
+  c->appended.assign((size_t)p->n_layers, 0);
   c->prm = *p;
   c->prm.seq_lens = c->hp.seq_lens.data();
   c->prm.mid_budget_per_layer = nullptr;          // the per-(sequence, layer) budgets live in the plan
@@ -710,15 +759,20 @@ bool pointers_ok(const taskkv_params* p, const void* const* q_win, const void* c
 taskkv_status compress_impl(const taskkv_params* p, const void* const* q_win, const void* const* k,
                             const void* const* v, const void* const* window_lse, void* cache_mem,
                             size_t cache_bytes, void* workspace_mem, size_t workspace_bytes, taskkv_stream stream,
-                            taskkv_cache** out_cache) {
+                            taskkv_cache** out_cache, taskkv_pool* pool) {
   if (!p || !q_win || !k || !v || !out_cache) return TASKKV_EINVAL;
   *out_cache = nullptr;
   if (p->batch < 1 || !pointers_ok(p, q_win, k, v, window_lse)) return TASKKV_EINVAL;
   if (p->shard_kv_heads > 0) return TASKKV_EINVAL;      // a shard needs the other shards' vectors: begin / finish
   cudaStream_t s = static_cast<cudaStream_t>(stream);
   taskkv_cache* c = nullptr;
-  const taskkv_status st = cache_create_impl(p, cache_mem, cache_bytes, workspace_mem, workspace_bytes, s, &c);
+  const taskkv_status st = cache_create_impl(p, cache_mem, cache_bytes, workspace_mem, workspace_bytes, s, &c, pool);
   if (st != TASKKV_OK) return st;
+  if (pool) {
+    pool->free_host -= c->hp.pages_compress;
+    c->pages_held = c->hp.pages_compress;
+    ++pool->caches;
+  }
   set_layer_pointers(c, 0, p->n_layers, q_win, k, v);
   cudaError_t e = upload_pointers(c, s);
   WindowHostInfo wh;
@@ -740,6 +794,90 @@ taskkv_status compress_impl(const taskkv_params* p, const void* const* q_win, co
   return TASKKV_OK;
 }
 }  // namespace
+
+size_t taskkv_pool_bytes(int32_t page_rows, int32_t n_pages, int32_t head_dim, int32_t dtype) {
+  if (page_rows < kGatherRows || page_rows % kGatherRows != 0 || n_pages < 1) return 0;
+  if ((head_dim != 64 && head_dim != 128) || (dtype != TASKKV_F32 && dtype != TASKKV_BF16)) return 0;
+  const size_t page = (size_t)page_rows * head_dim * (dtype == TASKKV_F32 ? 4 : 2);
+  return 2 * align_up((size_t)n_pages * page) + align_up((size_t)n_pages * 4) + kAlign;
+}
+
+taskkv_status taskkv_pool_create(int32_t page_rows, int32_t n_pages, int32_t head_dim, int32_t dtype, void* mem,
+                                 size_t bytes, taskkv_stream stream, taskkv_pool** out_pool) {
+  if (!out_pool) return TASKKV_EINVAL;
+  *out_pool = nullptr;
+  const size_t need = taskkv_pool_bytes(page_rows, n_pages, head_dim, dtype);
+  if (need == 0) return TASKKV_EINVAL;
+  if (mem && (((uintptr_t)mem & (kAlign - 1)) != 0)) return TASKKV_EINVAL;
+  if (mem && bytes < need) return TASKKV_EALLOC;
+  taskkv_pool* pool = new (std::nothrow) taskkv_pool();
+  if (!pool) return TASKKV_EALLOC;
+  pool->page_rows = page_rows;
+  pool->n_pages = n_pages;
+  pool->head_dim = head_dim;
+  pool->dtype = dtype;
+  if (mem) {
+    pool->mem = mem;
+  } else {
+    if (cudaMalloc(&pool->mem, need) != cudaSuccess) {
+      cudaGetLastError();
+      delete pool;
+      return TASKKV_EALLOC;
+    }
+    pool->own = true;
+  }
+  const size_t page = (size_t)page_rows * head_dim * (dtype == TASKKV_F32 ? 4 : 2);
+  unsigned char* m = static_cast<unsigned char*>(pool->mem);
+  pool->k_pages = m;
+  pool->v_pages = m + align_up((size_t)n_pages * page);
+  pool->free_ids = reinterpret_cast<int32_t*>(m + 2 * align_up((size_t)n_pages * page));
+  pool->top = reinterpret_cast<int32_t*>(m + 2 * align_up((size_t)n_pages * page) + align_up((size_t)n_pages * 4));
+  // every page is free: the stack holds n_pages - 1 ... 0, so that page 0 is taken first
+  std::vector<int32_t> ids((size_t)n_pages);
+  for (int32_t i = 0; i < n_pages; ++i) ids[(size_t)i] = n_pages - 1 - i;
+  cudaStream_t s = static_cast<cudaStream_t>(stream);
+  cudaError_t e = cudaMemcpyAsync(pool->free_ids, ids.data(), ids.size() * 4, cudaMemcpyHostToDevice, s);
+  if (e == cudaSuccess) e = cudaMemcpyAsync(pool->top, &n_pages, 4, cudaMemcpyHostToDevice, s);
+  if (e == cudaSuccess) e = cudaStreamSynchronize(s);       // the host buffers above go out of scope
+  if (e != cudaSuccess) {
+    cudaGetLastError();
+    taskkv_pool_destroy(pool);
+    return TASKKV_ECUDA;
+  }
+  pool->free_host = n_pages;
+  *out_pool = pool;
+  return TASKKV_OK;
+}
+
+int32_t taskkv_pool_free_pages(const taskkv_pool* pool) { return pool ? (int32_t)pool->free_host : -1; }
+
+void taskkv_pool_destroy(taskkv_pool* pool) {
+  if (!pool) return;
+  if (pool->own) {
+    cudaDeviceSynchronize();
+    cudaFree(pool->mem);
+  }
+  delete pool;
+}
+
+taskkv_status taskkv_plan_paged(const taskkv_params* p, int32_t page_rows, taskkv_plan_info* out, int64_t* pages_needed) {
+  if (!out || page_rows < kGatherRows) return TASKKV_EINVAL;
+  HostPlan hp;
+  const taskkv_status st = make_plan(p, hp, page_rows);
+  if (st != TASKKV_OK) return st;
+  *out = hp.info;
+  if (pages_needed) *pages_needed = hp.pages_compress;
+  return TASKKV_OK;
+}
+
+taskkv_status taskkv_compress_paged(const taskkv_params* p, const void* const* q_win, const void* const* k,
+                                    const void* const* v, taskkv_pool* pool, void* cache_mem, size_t cache_bytes,
+                                    void* workspace_mem, size_t workspace_bytes, taskkv_stream stream,
+                                    taskkv_cache** out_cache) {
+  if (!pool) return TASKKV_EINVAL;
+  return compress_impl(p, q_win, k, v, nullptr, cache_mem, cache_bytes, workspace_mem, workspace_bytes, stream,
+                       out_cache, pool);
+}
 
 taskkv_status taskkv_cache_create(const taskkv_params* p, void* cache_mem, size_t cache_bytes, void* workspace_mem,
                                   size_t workspace_bytes, taskkv_stream stream, taskkv_cache** out_cache) {
@@ -921,11 +1059,45 @@ bool layer_view(const taskkv_cache* c, int32_t layer_begin, int32_t layer_count,
 }
 }  // namespace
 
+namespace {
+// Paged caches: the pages that appending one token to layers [l0, l0 + nl) takes off the pool -- a unit needs one when
+// its last page is full -- and the bookkeeping once the call is accepted.  Which units are the long ones is known only
+// on the device, how many of each kind a (sequence, layer) has is fixed by Eq. 16, so the count is exact.
+int64_t append_pages(const taskkv_cache* c, int32_t l0, int32_t nl) {
+  if (!c->pool) return 0;
+  const int P = c->hp.page_rows, B = c->prm.batch, R = c->prm.n_layers, nkv = c->prm.n_kv_heads;
+  int64_t need = 0;
+  for (int r = l0; r < l0 + nl; ++r) {
+    const int a = c->appended[(size_t)r];
+    if (a >= c->prm.max_new_tokens) continue;                 // at capacity: nothing is appended
+    for (int b = 0; b < B; ++b) {
+      const size_t br = (size_t)b * R + r;
+      const int64_t h = c->hp.full[br];
+      if ((c->hp.seq_lens[b] + a) % P == 0) need += h;
+      if ((c->hp.kept_len[br] + a) % P == 0) need += nkv - h;
+    }
+  }
+  return need;
+}
+taskkv_status take_append_pages(taskkv_cache* c, int32_t l0, int32_t nl) {
+  if (!c->pool) return TASKKV_OK;
+  const int64_t need = append_pages(c, l0, nl);
+  if (need > c->pool->free_host) return TASKKV_EALLOC;
+  c->pool->free_host -= need;
+  c->pages_held += need;
+  for (int r = l0; r < l0 + nl; ++r)
+    if (c->appended[(size_t)r] < c->prm.max_new_tokens) ++c->appended[(size_t)r];
+  return TASKKV_OK;
+}
+}  // namespace
+
 taskkv_status taskkv_append_ex(taskkv_cache* c, const void* k_new, const void* v_new, int32_t layer_begin,
                                int32_t layer_count, taskkv_stream stream) {
   if (!c || !k_new || !v_new || (((uintptr_t)k_new | (uintptr_t)v_new) & 15)) return TASKKV_EINVAL;
   taskkv::DeviceProblem view;
   if (!layer_view(c, layer_begin, layer_count, &view)) return TASKKV_EINVAL;
+  const taskkv_status st = take_append_pages(c, layer_begin, layer_count);
+  if (st != TASKKV_OK) return st;
   return cuda_status(launch_append(view, c->prm.dtype, k_new, v_new, static_cast<cudaStream_t>(stream)));
 }
 
@@ -949,6 +1121,8 @@ taskkv_status taskkv_decode_step_ex(const void* q, const void* k_new, const void
   if (((uintptr_t)q | (uintptr_t)out | (uintptr_t)k_new | (uintptr_t)v_new) & 15) return TASKKV_EINVAL;
   taskkv::DeviceProblem view;
   if (!layer_view(c, layer_begin, layer_count, &view)) return TASKKV_EINVAL;
+  const taskkv_status st = take_append_pages(c, layer_begin, layer_count);
+  if (st != TASKKV_OK) return st;
   return cuda_status(launch_decode(view, c->prm.dtype, q, nullptr, k_new, v_new, out,
                                    static_cast<cudaStream_t>(stream)));
 }
@@ -992,6 +1166,7 @@ taskkv_status taskkv_decode_host(const void* q, const void* k_new, const void* v
     e = cudaMemcpyAsync(dkn, k_new, k_bytes, cudaMemcpyHostToDevice, s);
     if (e == cudaSuccess) e = cudaMemcpyAsync(dvn, v_new, k_bytes, cudaMemcpyHostToDevice, s);
   }
+  if (e == cudaSuccess && k_new && take_append_pages(c, 0, c->dp.R) != TASKKV_OK) return TASKKV_EALLOC;
   if (e == cudaSuccess)
     e = launch_decode(c->dp, c->prm.dtype, dq, nullptr, k_new ? dkn : nullptr, k_new ? dvn : nullptr, dout, s);
   if (e == cudaSuccess) e = cudaMemcpyAsync(out, dout, q_bytes, cudaMemcpyDeviceToHost, s);
@@ -1011,7 +1186,9 @@ int64_t taskkv_cache_query_bytes(const taskkv_cache* c, int32_t what) {
     case TASKKV_Q_SCORES: return c->work_mem ? c->hp.c_total * 4 : -1;
     case TASKKV_Q_TOPT: return c->work_mem ? U * c->dp.top_t * 4 : -1;
     case TASKKV_Q_STATUS: return 4;
-    case TASKKV_Q_KPOOL: case TASKKV_Q_VPOOL: return c->dp.pool_rows * c->dp.d * es;
+    case TASKKV_Q_KPOOL: case TASKKV_Q_VPOOL:
+      return (c->pool ? (int64_t)c->pool->n_pages * c->pool->page_rows : c->dp.pool_rows) * c->dp.d * es;
+    case TASKKV_Q_PAGETAB: return c->pool ? U * c->dp.page_stride * 4 : -1;
     default: return -1;
   }
 }
@@ -1034,6 +1211,7 @@ taskkv_status taskkv_cache_query(const taskkv_cache* c, int32_t what, void* host
     case TASKKV_Q_STATUS: src = c->dp.status; break;
     case TASKKV_Q_KPOOL: src = c->dp.k_pool; break;
     case TASKKV_Q_VPOOL: src = c->dp.v_pool; break;
+    case TASKKV_Q_PAGETAB: src = c->dp.page_tab; break;
     default: return TASKKV_EINVAL;
   }
   if (cudaDeviceSynchronize() != cudaSuccess) return TASKKV_ECUDA;
@@ -1049,6 +1227,13 @@ taskkv_status taskkv_cache_plan(const taskkv_cache* c, taskkv_plan_info* out) {
 
 void taskkv_cache_destroy(taskkv_cache* c) {
   if (!c) return;
+  if (c->pool) {
+    // the pages go back onto the pool's stack once everything that uses them has finished
+    cudaDeviceSynchronize();
+    if (c->cache_mem && launch_release_pages(c->dp, nullptr) == cudaSuccess) cudaDeviceSynchronize();
+    c->pool->free_host += c->pages_held;
+    --c->pool->caches;
+  }
   if (c->own_cache || c->own_work || c->stage) cudaDeviceSynchronize();
   if (c->own_cache) cudaFree(c->cache_mem);
   if (c->own_work) cudaFree(c->work_mem);

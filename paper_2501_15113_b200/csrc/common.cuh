@@ -93,6 +93,13 @@ struct DeviceProblem {
   int32_t* step_cnt;          // [U] combine blocks of a unit that finished the current fused step (0 between calls)
   void* k_pool;
   void* v_pool;
+  // Paged cache: the pools are arrays of pages of page_rows rows (a multiple of 64) owned by a page pool that several
+  // caches share; unit u's row r lives in page page_tab[u * page_stride + r / page_rows] at slot r % page_rows.
+  // page_rows == 0: one contiguous segment per unit, starting at seg_off[u].
+  int32_t page_rows, page_stride;
+  int32_t* page_tab;          // [U][page_stride]
+  int32_t* pool_free;         // the pool's stack of free page ids; the top `*pool_top` entries are free
+  int32_t* pool_top;
   // decode scratch
   float* part_acc;            // [items][G][d]
   float* part_ml;             // [items][G][2]
@@ -163,6 +170,8 @@ cudaError_t launch_separator_plan(const DeviceProblem& p, int batch, int layer0,
 // (q_win[b]: [n][L][d], k[b], v[b]: [n_kv][N_b][d]); host arrays of `batch` device pointers.
 cudaError_t launch_set_layer_pointers(const DeviceProblem& p, int batch, int layer, int elem_size, const void* const* q_win,
                                       const void* const* k, const void* const* v, cudaStream_t s);
+// paged caches: every page of the cache's units back onto the pool's stack
+cudaError_t launch_release_pages(const DeviceProblem& p, cudaStream_t s);
 // Eq. 17 on the device for the units of a range of layers (nothing to do unless budget_frac > 0)
 cudaError_t launch_budget(const DeviceProblem& p, int batch, int layer0, int n_layers, cudaStream_t s);
 // gather work items [item0, item0 + n_items) = those of layers [layer0, layer0 + n_layers) (layer-major numbering)
@@ -284,6 +293,25 @@ __device__ __forceinline__ int upper_unit(const int32_t* off, int n, int x) {
 }
 
 __device__ __forceinline__ void set_status(int32_t* status, int32_t code) { atomicCAS(status, 0, code); }
+
+// Pool row of row r of unit u (seg = seg_off[u]).  Rows r .. r + n - 1 are consecutive pool rows as long as they do
+// not cross a multiple of page_rows.
+__device__ __forceinline__ size_t pool_row(const DeviceProblem& p, int u, int64_t seg, int r) {
+  if (p.page_rows == 0) return (size_t)seg + (size_t)r;
+  const int pg = p.page_tab[(size_t)u * p.page_stride + r / p.page_rows];
+  return (size_t)pg * p.page_rows + (size_t)(r % p.page_rows);
+}
+// Takes n pages off the pool's stack; returns the index of the first of them in pool_free, or -1 (and ESTATE) if the
+// pool has fewer -- the host keeps count and refuses such calls before they are launched.
+__device__ __forceinline__ int pool_pop(const DeviceProblem& p, int n) {
+  const int base = atomicSub(p.pool_top, n) - n;
+  if (base < 0) {
+    atomicAdd(p.pool_top, n);
+    set_status(p.status, TASKKV_ESTATE);
+    return -1;
+  }
+  return base;
+}
 
 #endif  // __CUDACC__
 

@@ -20,7 +20,9 @@ constexpr int kAttnThreads = 128;
 constexpr int kAttnWarps = kAttnThreads / 32;
 constexpr int kUnroll = 4;
 
-template <typename T, int D, int G>
+// PAGED (both attention kernels): the rows of a unit live in pages of the shared pool; the rows one loop iteration
+// touches never cross a page (a page holds a multiple of 64 rows), so an iteration looks its page up once.
+template <typename T, int D, int G, bool PAGED>
 __global__ void __launch_bounds__(kAttnThreads) decode_attn_kernel(DeviceProblem p, const T* __restrict__ q,
                                                                    const int32_t* __restrict__ lengths,
                                                                    const unsigned char* __restrict__ k_new,
@@ -66,14 +68,28 @@ __global__ void __launch_bounds__(kAttnThreads) decode_attn_kernel(DeviceProblem
     const int64_t seg = p.seg_off[u];
     const unsigned char* kn_row = k_new + (size_t)vu * ROW_BYTES;
     const unsigned char* vn_row = v_new + (size_t)vu * ROW_BYTES;
-    if (new_r >= rbeg && new_r < rend && tid < ROW_BYTES / 16) {
-      unsigned char* kd = static_cast<unsigned char*>(p.k_pool) + ((size_t)seg + new_r) * ROW_BYTES + tid * 16;
-      unsigned char* vd = static_cast<unsigned char*>(p.v_pool) + ((size_t)seg + new_r) * ROW_BYTES + tid * 16;
-      *reinterpret_cast<uint4*>(kd) = *reinterpret_cast<const uint4*>(kn_row + tid * 16);
-      *reinterpret_cast<uint4*>(vd) = *reinterpret_cast<const uint4*>(vn_row + tid * 16);
+    if (new_r >= rbeg && new_r < rend) {
+      bool have_page = true;
+      if (PAGED && new_r % p.page_rows == 0) {
+        // the appended row opens a new page: one comes off the pool (only this block touches the unit's new row)
+        if (tid == 0) {
+          const int at = pool_pop(p, 1);
+          if (at >= 0) p.page_tab[(size_t)u * p.page_stride + new_r / p.page_rows] = p.pool_free[at];
+          s_unit = at;                              // (the unit index has been read by everybody)
+        }
+        __syncthreads();
+        have_page = s_unit >= 0;                    // an empty pool: status ESTATE, the row is not stored
+      }
+      if (have_page && tid < ROW_BYTES / 16) {
+        const size_t drow = pool_row(p, u, seg, new_r);
+        unsigned char* kd = static_cast<unsigned char*>(p.k_pool) + drow * ROW_BYTES + tid * 16;
+        unsigned char* vd = static_cast<unsigned char*>(p.v_pool) + drow * ROW_BYTES + tid * 16;
+        *reinterpret_cast<uint4*>(kd) = *reinterpret_cast<const uint4*>(kn_row + tid * 16);
+        *reinterpret_cast<uint4*>(vd) = *reinterpret_cast<const uint4*>(vn_row + tid * 16);
+      }
     }
-    const unsigned char* kp = static_cast<const unsigned char*>(p.k_pool) + (size_t)seg * ROW_BYTES + sl * 16;
-    const unsigned char* vp = static_cast<const unsigned char*>(p.v_pool) + (size_t)seg * ROW_BYTES + sl * 16;
+    const unsigned char* kp = static_cast<const unsigned char*>(p.k_pool) + (PAGED ? 0 : (size_t)seg * ROW_BYTES) + sl * 16;
+    const unsigned char* vp = static_cast<const unsigned char*>(p.v_pool) + (PAGED ? 0 : (size_t)seg * ROW_BYTES) + sl * 16;
 
     float qf[G][EPL];
 #pragma unroll
@@ -96,15 +112,17 @@ __global__ void __launch_bounds__(kAttnThreads) decode_attn_kernel(DeviceProblem
     auto rows_loop = [&](auto has_new) {
     for (int base = rbeg; base < rend; base += NSG * kUnroll) {   // warp-uniform trip count
       const int r0 = base + gsg;
+      // pool row of row `base` minus base: adding a row index of this iteration gives its pool row
+      const size_t rowoff = PAGED ? pool_row(p, u, seg, base) - (size_t)base : 0;
       uint4 kraw[kUnroll], vraw[kUnroll];
 #pragma unroll
       for (int i = 0; i < kUnroll; ++i) {
         const int r = r0 + i * NSG;
         if (r < rend) {
           kraw[i] = *reinterpret_cast<const uint4*>((decltype(has_new)::value && r == new_r) ? kn_row + sl * 16
-                                                                                             : kp + (size_t)r * ROW_BYTES);
+                                                                                             : kp + (rowoff + (size_t)r) * ROW_BYTES);
           vraw[i] = *reinterpret_cast<const uint4*>((decltype(has_new)::value && r == new_r) ? vn_row + sl * 16
-                                                                                             : vp + (size_t)r * ROW_BYTES);
+                                                                                             : vp + (rowoff + (size_t)r) * ROW_BYTES);
         } else {
           kraw[i] = make_uint4(0, 0, 0, 0);
           vraw[i] = make_uint4(0, 0, 0, 0);
@@ -228,7 +246,7 @@ __device__ __forceinline__ uint32_t word_of(const uint4& v, int i) {
   return i == 0 ? v.x : i == 1 ? v.y : i == 2 ? v.z : v.w;
 }
 
-template <int D, int G>
+template <int D, int G, bool PAGED>
 __global__ void __launch_bounds__(kAttnThreads) decode_attn_mma_kernel(DeviceProblem p,
                                                                        const __nv_bfloat16* __restrict__ q,
                                                                        const int32_t* __restrict__ lengths,
@@ -277,14 +295,28 @@ __global__ void __launch_bounds__(kAttnThreads) decode_attn_mma_kernel(DevicePro
     const int64_t seg = p.seg_off[u];
     const unsigned char* kn_row = k_new + (size_t)vu * ROW_BYTES;
     const unsigned char* vn_row = v_new + (size_t)vu * ROW_BYTES;
-    if (new_r >= rbeg && new_r < rend && tid < ROW_BYTES / 16) {
-      unsigned char* kd = static_cast<unsigned char*>(p.k_pool) + ((size_t)seg + new_r) * ROW_BYTES + tid * 16;
-      unsigned char* vd = static_cast<unsigned char*>(p.v_pool) + ((size_t)seg + new_r) * ROW_BYTES + tid * 16;
-      *reinterpret_cast<uint4*>(kd) = *reinterpret_cast<const uint4*>(kn_row + tid * 16);
-      *reinterpret_cast<uint4*>(vd) = *reinterpret_cast<const uint4*>(vn_row + tid * 16);
+    if (new_r >= rbeg && new_r < rend) {
+      bool have_page = true;
+      if (PAGED && new_r % p.page_rows == 0) {
+        // the appended row opens a new page: one comes off the pool (only this block touches the unit's new row)
+        if (tid == 0) {
+          const int at = pool_pop(p, 1);
+          if (at >= 0) p.page_tab[(size_t)u * p.page_stride + new_r / p.page_rows] = p.pool_free[at];
+          s_unit = at;                              // (the unit index has been read by everybody)
+        }
+        __syncthreads();
+        have_page = s_unit >= 0;                    // an empty pool: status ESTATE, the row is not stored
+      }
+      if (have_page && tid < ROW_BYTES / 16) {
+        const size_t drow = pool_row(p, u, seg, new_r);
+        unsigned char* kd = static_cast<unsigned char*>(p.k_pool) + drow * ROW_BYTES + tid * 16;
+        unsigned char* vd = static_cast<unsigned char*>(p.v_pool) + drow * ROW_BYTES + tid * 16;
+        *reinterpret_cast<uint4*>(kd) = *reinterpret_cast<const uint4*>(kn_row + tid * 16);
+        *reinterpret_cast<uint4*>(vd) = *reinterpret_cast<const uint4*>(vn_row + tid * 16);
+      }
     }
-    const unsigned char* kp = static_cast<const unsigned char*>(p.k_pool) + (size_t)seg * ROW_BYTES;
-    const unsigned char* vp = static_cast<const unsigned char*>(p.v_pool) + (size_t)seg * ROW_BYTES;
+    const unsigned char* kp = static_cast<const unsigned char*>(p.k_pool) + (PAGED ? 0 : (size_t)seg * ROW_BYTES);
+    const unsigned char* vp = static_cast<const unsigned char*>(p.v_pool) + (PAGED ? 0 : (size_t)seg * ROW_BYTES);
 
     // Q fragments: head g on M row g
     uint32_t qa[KC][2];
@@ -305,6 +337,8 @@ __global__ void __launch_bounds__(kAttnThreads) decode_attn_mma_kernel(DevicePro
     // two copies of the row loop: only the item that holds the new token's row pays for telling it apart
     auto rows_loop = [&](auto has_new) {
     for (int blk = rbeg + warp * kBlk; blk < rend; blk += kAttnWarps * kBlk) {   // warp-uniform
+      // pool row of row `blk` minus blk: adding a row index of this 16-row block gives its pool row
+      const size_t rowoff = PAGED ? pool_row(p, u, seg, blk) - (size_t)blk : 0;
       uint4 kraw[2][KP], vraw[4][VP];
 #pragma unroll
       for (int j = 0; j < 2; ++j) {
@@ -312,7 +346,7 @@ __global__ void __launch_bounds__(kAttnThreads) decode_attn_mma_kernel(DevicePro
 #pragma unroll
         for (int i = 0; i < KP; ++i)
           kraw[j][i] = r < rend ? *reinterpret_cast<const uint4*>(((decltype(has_new)::value && r == new_r)
-                                                                       ? kn_row : kp + (size_t)r * ROW_BYTES) +
+                                                                       ? kn_row : kp + (rowoff + (size_t)r) * ROW_BYTES) +
                                                                   (i * 4 + t) * 16)
                                 : make_uint4(0, 0, 0, 0);
       }
@@ -322,7 +356,7 @@ __global__ void __launch_bounds__(kAttnThreads) decode_attn_mma_kernel(DevicePro
 #pragma unroll
         for (int i = 0; i < VP; ++i)
           vraw[x][i] = r < rend ? *reinterpret_cast<const uint4*>(((decltype(has_new)::value && r == new_r)
-                                                                       ? vn_row : vp + (size_t)r * ROW_BYTES) +
+                                                                       ? vn_row : vp + (rowoff + (size_t)r) * ROW_BYTES) +
                                                                   i * 128 + g * 16)
                                 : make_uint4(0, 0, 0, 0);
       }
@@ -491,10 +525,17 @@ cudaError_t launch_typed(const DeviceProblem& p, const void* q, const int32_t* l
   cudaError_t e;
   {
     LaunchScope ls(K_DECODE_ATTN, s);
-    if constexpr (sizeof(T) == 2)
-      e = launch_dependent(decode_attn_mma_kernel<D, G>, (unsigned)grid, kAttnThreads, s, p, static_cast<const T*>(q), lengths, kn, vn);
-    else
-      e = launch_dependent(decode_attn_kernel<T, D, G>, (unsigned)grid, kAttnThreads, s, p, static_cast<const T*>(q), lengths, kn, vn);
+    if (p.page_rows > 0) {
+      if constexpr (sizeof(T) == 2)
+        e = launch_dependent(decode_attn_mma_kernel<D, G, true>, (unsigned)grid, kAttnThreads, s, p, static_cast<const T*>(q), lengths, kn, vn);
+      else
+        e = launch_dependent(decode_attn_kernel<T, D, G, true>, (unsigned)grid, kAttnThreads, s, p, static_cast<const T*>(q), lengths, kn, vn);
+    } else {
+      if constexpr (sizeof(T) == 2)
+        e = launch_dependent(decode_attn_mma_kernel<D, G, false>, (unsigned)grid, kAttnThreads, s, p, static_cast<const T*>(q), lengths, kn, vn);
+      else
+        e = launch_dependent(decode_attn_kernel<T, D, G, false>, (unsigned)grid, kAttnThreads, s, p, static_cast<const T*>(q), lengths, kn, vn);
+    }
   }
   if (e != cudaSuccess) return e;
   {

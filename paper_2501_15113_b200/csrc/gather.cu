@@ -37,13 +37,16 @@ __global__ void __launch_bounds__(kGatherThreads, 10) gather_kernel(DeviceProble
   const int N = p.unit_N[u];
   const int r0 = (item - p.gather_off[w]) * kGatherRows;
   const int64_t seg = p.seg_off[u];
-  if (seg + len > p.pool_rows) return;                // planning overflow, already flagged
+  if (p.page_rows == 0 && seg + len > p.pool_rows) return;   // planning overflow, already flagged
+  if (r0 >= len) return;                                     // an item between a shard's block end and the next block
   const bool identity = (len == N);
   const int32_t* idx = p.idx + (size_t)u * p.idx_stride;
   const unsigned char* ksrc = static_cast<const unsigned char*>(p.k_ptr[u]);
   const unsigned char* vsrc = static_cast<const unsigned char*>(p.v_ptr[u]);
-  unsigned char* kdst = static_cast<unsigned char*>(p.k_pool) + (size_t)seg * ROW_BYTES;
-  unsigned char* vdst = static_cast<unsigned char*>(p.v_pool) + (size_t)seg * ROW_BYTES;
+  // the block's 64 rows are consecutive pool rows (a page holds a multiple of 64 rows), starting at dst0
+  const size_t dst0 = pool_row(p, u, seg, r0);
+  unsigned char* kdst = static_cast<unsigned char*>(p.k_pool) + dst0 * ROW_BYTES;
+  unsigned char* vdst = static_cast<unsigned char*>(p.v_pool) + dst0 * ROW_BYTES;
   const int rr = threadIdx.x / VPR, vc = threadIdx.x % VPR;
 
   for (int base = 0; base < PASSES; base += ROUND) {
@@ -62,8 +65,8 @@ __global__ void __launch_bounds__(kGatherThreads, 10) gather_kernel(DeviceProble
     for (int ps = 0; ps < ROUND; ++ps) {
       const int r = r0 + (base + ps) * RPP + rr;
       if (r < len) {
-        *reinterpret_cast<uint4*>(kdst + (size_t)r * ROW_BYTES + vc * 16) = kreg[ps];
-        *reinterpret_cast<uint4*>(vdst + (size_t)r * ROW_BYTES + vc * 16) = vreg[ps];
+        *reinterpret_cast<uint4*>(kdst + (size_t)(r - r0) * ROW_BYTES + vc * 16) = kreg[ps];
+        *reinterpret_cast<uint4*>(vdst + (size_t)(r - r0) * ROW_BYTES + vc * 16) = vreg[ps];
       }
     }
   }
@@ -80,10 +83,23 @@ __global__ void __launch_bounds__(256) append_kernel(DeviceProblem p, const unsi
   const int u = view_unit(p, vu);
   const int len = p.len[u];
   const int64_t seg = p.seg_off[u];
-  const bool ok = len < p.cap[u] && seg + len < p.pool_rows;
+  bool ok = len < p.cap[u] && (p.page_rows > 0 || seg + len < p.pool_rows);
+  if (ok && p.page_rows > 0 && len % p.page_rows == 0) {
+    // the row opens a new page: one comes off the pool
+    int pg = -1;
+    if (lane == 0) {
+      const int at = pool_pop(p, 1);
+      if (at >= 0) {
+        pg = p.pool_free[at];
+        p.page_tab[(size_t)u * p.page_stride + len / p.page_rows] = pg;
+      }
+    }
+    pg = __shfl_sync(0xffffffffu, pg, 0);
+    ok = pg >= 0;
+  }
   __syncwarp();
   if (ok && lane < VPR) {
-    const size_t dst = ((size_t)seg + len) * ROW_BYTES + lane * 16;
+    const size_t dst = pool_row(p, u, seg, len) * ROW_BYTES + lane * 16;
     const size_t src = (size_t)vu * ROW_BYTES + lane * 16;
     *reinterpret_cast<uint4*>(static_cast<unsigned char*>(p.k_pool) + dst) =
         *reinterpret_cast<const uint4*>(k_new + src);
@@ -116,7 +132,7 @@ __global__ void __launch_bounds__(kGatherThreads) compensate_kernel(DeviceProble
   if (g >= c) return;
   const int vc = threadIdx.x % VPR;
   const int64_t seg = p.seg_off[u];
-  if (seg + len > p.pool_rows) return;                // planning overflow, already flagged
+  if (p.page_rows == 0 && seg + len > p.pool_rows) return;   // planning overflow, already flagged
   const int32_t* idx = p.idx + (size_t)u * p.idx_stride;
   int j0 = idx[s1 + g];
   int j1 = (g + 1 < c) ? idx[s1 + g + 1] : N - s2;
@@ -135,8 +151,9 @@ __global__ void __launch_bounds__(kGatherThreads) compensate_kernel(DeviceProble
     for (int e = 0; e < EPV; ++e) { ka[e] += kf[e]; va[e] += vf[e]; }
   }
   const float cnt = (float)max(j1 - j0, 1);
-  T* kdst = reinterpret_cast<T*>(static_cast<unsigned char*>(p.k_pool) + ((size_t)seg + s1 + g) * ROW_BYTES) + vc * EPV;
-  T* vdst = reinterpret_cast<T*>(static_cast<unsigned char*>(p.v_pool) + ((size_t)seg + s1 + g) * ROW_BYTES) + vc * EPV;
+  const size_t drow = pool_row(p, u, seg, s1 + g);
+  T* kdst = reinterpret_cast<T*>(static_cast<unsigned char*>(p.k_pool) + drow * ROW_BYTES) + vc * EPV;
+  T* vdst = reinterpret_cast<T*>(static_cast<unsigned char*>(p.v_pool) + drow * ROW_BYTES) + vc * EPV;
 #pragma unroll
   for (int e = 0; e < EPV; ++e) {
     store_out(kdst + e, ka[e] / cnt);

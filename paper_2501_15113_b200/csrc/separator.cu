@@ -124,6 +124,38 @@ __global__ void __launch_bounds__(128) separator_plan_kernel(DeviceProblem p, in
       }
     }
   }
+  // ---- paged cache: the block takes the pages of its units' retained rows off the pool in one step (growth takes
+  // pages later, one at a time) and deals them out in unit order
+  if (p.page_rows > 0) {
+    __shared__ int s_pages[TASKKV_MAX_KV_HEADS];
+    __shared__ int s_base;
+    if (tid < nl) s_pages[tid] = (len + p.page_rows - 1) / p.page_rows;
+    __syncthreads();
+    if (tid == 0) {
+      int total = 0;
+      for (int h = 0; h < nl; ++h) total += s_pages[h];
+      s_base = total > 0 ? pool_pop(p, total) : 0;
+    }
+    __syncthreads();
+    if (tid < nl && s_base >= 0) {
+      int before = 0;
+      for (int h = 0; h < tid; ++h) before += s_pages[h];
+      int32_t* tab = p.page_tab + (size_t)(br * nl + tid) * p.page_stride;
+      for (int i = 0; i < s_pages[tid]; ++i) tab[i] = p.pool_free[s_base + before + i];
+    }
+  }
+}
+
+// Gives every page of the cache's units back to the pool (a paged cache is being destroyed).
+__global__ void __launch_bounds__(128) release_pages_kernel(DeviceProblem p) {
+  const int u = blockIdx.x * blockDim.x + threadIdx.x;
+  if (u >= p.U) return;
+  const int pages = (p.len[u] + p.page_rows - 1) / p.page_rows;
+  if (pages <= 0) return;
+  const int pos = atomicAdd(p.pool_top, pages);
+  const int32_t* tab = p.page_tab + (size_t)u * p.page_stride;
+  for (int i = 0; i < pages; ++i) p.pool_free[pos + i] = tab[i];
+  p.len[u] = 0;
 }
 
 // Eq. 17 with the budget given as a fraction of the full cache: k = floor((B - N h) / (n - h)) - s1 - s2 with
@@ -188,6 +220,13 @@ cudaError_t launch_set_layer_pointers(const DeviceProblem& p, int batch, int lay
     if (e != cudaSuccess) return e;
   }
   return cudaSuccess;
+}
+
+cudaError_t launch_release_pages(const DeviceProblem& p, cudaStream_t s) {
+  if (p.page_rows <= 0 || p.U <= 0) return cudaSuccess;
+  LaunchScope ls(K_PLAN, s);
+  release_pages_kernel<<<(p.U + 127) / 128, 128, 0, s>>>(p);
+  return cudaGetLastError();
 }
 
 cudaError_t launch_budget(const DeviceProblem& p, int batch, int layer0, int n_layers, cudaStream_t s) {

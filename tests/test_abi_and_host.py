@@ -127,6 +127,13 @@ def test_invalid_arguments_are_rejected_before_any_launch(tk):
     assert tk.lib.taskkv_compress_shard_begin(None, None, None, None, None, None, 0, None, 0, None, C.byref(h)) == tk.EINVAL
     assert tk.lib.taskkv_compress_shard_finish(None, None, None) == tk.EINVAL
     assert tk.lib.taskkv_cache_semantic(None, None, None) == tk.EINVAL
+    assert tk.lib.taskkv_compress_paged(None, None, None, None, None, None, 0, None, 0, None, C.byref(h)) == tk.EINVAL
+    assert tk.lib.taskkv_pool_create(32, 8, 128, tk.BF16, None, 0, None, C.byref(h)) == tk.EINVAL
+    assert tk.lib.taskkv_pool_create(64, 8, 128, tk.BF16, None, 0, None, None) == tk.EINVAL
+    assert tk.lib.taskkv_pool_create(64, 8, 128, tk.BF16, 256, 16, None, C.byref(h)) == tk.EALLOC   # buffer too small
+    assert tk.lib.taskkv_plan_paged(None, 64, None, None) == tk.EINVAL
+    assert tk.lib.taskkv_pool_free_pages(None) == -1
+    tk.lib.taskkv_pool_destroy(None)
     assert tk.lib.taskkv_exact_semantic(None, None, None, 1, 8, 8, 128, 512, None, None, None, 0, None) == tk.EINVAL
     # argument checks come before any device work: a head dimension or a head grouping the kernels do not take
     assert tk.lib.taskkv_exact_semantic(16, 16, 16, 1, 8, 8, 96, 512, 16, None, None, 0, None) == tk.EINVAL
@@ -171,3 +178,34 @@ def test_plan_of_a_head_shard_is_the_upper_bound(tk):
                    window=32, dtype="bf16", n_hetero=[[0]], promote_center=False, budget_frac=0.5, shard_kv_heads=8,
                    shard_first=2)
     assert tk.taskkv_plan(p0).pool_rows == 2 * (s1 + s2 + O.mid_budget(0.5 * 8 * 4000, 4000, 0, 8, s1, s2)) and kmid > 0
+
+
+def test_plan_of_a_paged_cache_counts_pages_per_unit(tk):
+    """Pages a compression takes = sum over units of ceil(retained rows / page rows), the full heads per (sequence,
+    layer) from Eq. 16; the pool holds K and V pages plus the free-page stack; page sizes that are not a multiple of
+    the gather's 64-row items, and paged caches of a head shard, are refused."""
+    R, n, lens, s1, s2, k, mn = 3, 8, [3000, 1700, 260], 4, 64, 100, 7
+    nh = [[tk.taskkv_hetero_count(n, 0.25, 4, R, r) for r in range(R)] for _ in lens]
+    kw = dict(n_layers=R, n_heads=n, n_kv_heads=n, head_dim=128, seq_lens=lens, sink=s1, recent=s2, mid_budget=k,
+              window=32, dtype="bf16", max_new_tokens=mn)
+    p = tk.Params(**kw)
+    flat = tk.taskkv_plan(p)
+    for P in (64, 128, 1024):
+        info, pages = tk.taskkv_plan_paged(p, P)
+        want = 0
+        for b, N in enumerate(lens):
+            for r in range(R):
+                full = min(n, nh[b][r] + 1)
+                kept = min(N, s1 + s2 + k)
+                want += full * -(-N // P) + (n - full) * -(-kept // P)
+        assert pages == want and info.n_units == flat.n_units and info.retained_rows == flat.retained_rows
+        assert info.cache_bytes < flat.cache_bytes
+        assert tk.lib.taskkv_pool_bytes(P, pages, 128, tk.BF16) >= 2 * pages * P * 128 * 2 + 4 * pages
+    for bad in (0, 32, 96, -64):
+        with pytest.raises(tk.TaskKVError):
+            tk.taskkv_plan_paged(p, bad)
+        assert tk.lib.taskkv_pool_bytes(bad, 16, 128, tk.BF16) == 0
+    assert tk.lib.taskkv_pool_bytes(64, 0, 128, tk.BF16) == 0 and tk.lib.taskkv_pool_bytes(64, 16, 96, tk.BF16) == 0
+    shard = tk.Params(**dict(kw, n_heads=4, n_kv_heads=4, shard_kv_heads=8, shard_first=0))
+    with pytest.raises(tk.TaskKVError):
+        tk.taskkv_plan_paged(shard, 64)

@@ -1165,3 +1165,146 @@ def test_head_sharded_compression_equals_the_unsharded_call(case):
     whole.close()
     for (_, _, c, _) in shards:
         c.close()
+
+
+# ---------------------------------------------------------------------------
+# Paged cache: rows in pages of a pool shared by several caches, block tables per unit
+# ---------------------------------------------------------------------------
+@pytest.mark.parametrize("case", [
+    dict(n=16, n_kv=4, d=128, N=0, L=32, s1=4, s2=64, k=120, dtype="bf16", R=3, seq_lens=[2100, 1300], nh=1, P=64),
+    dict(n=8, n_kv=8, d=128, N=0, L=32, s1=4, s2=64, k=150, dtype="bf16", R=2, seq_lens=[5000], nh=2, P=256),
+    dict(n=4, n_kv=4, d=64, N=0, L=16, s1=4, s2=32, k=60, dtype="f32", R=2, seq_lens=[900, 700], nh=1, P=128),
+], ids=["bf16_gqa_p64", "bf16_mha_p256", "f32_p128"])
+def test_paged_cache_equals_the_contiguous_cache(case):
+    """The same compression with the rows in pages: classes, lengths and retained positions are the contiguous
+    cache's, every unit's rows read back through its page table are the same bytes, and so are the decode outputs of
+    many steps (fused and append + decode), during which units run off the end of their last page and take new pages
+    from the pool; the host's count of free pages follows exactly, and destroying the cache returns every page."""
+    tk, Pm = _tk(), _parity()
+    P = case.pop("P")
+    steps = 70 if P == 64 else 40
+    wl = small("paged", **case, steps=steps)
+    wl.mid_budget = [case["k"] + 17 * r for r in range(wl.n_layers)]
+    qs, ks, vs = W.materialize(wl, DEV)
+    params = tk.params_from_workload(wl, max_new_tokens=steps)
+    flat = tk.taskkv_compress_ex(params, qs, ks, vs)
+    info, pages = tk.taskkv_plan_paged(params, P)
+    assert int(info.cache_bytes) < int(flat.info.cache_bytes) // 4          # tables only
+    pool = tk.Pool(P, pages + 2 * int(info.n_units) + 3, wl.head_dim, wl.dtype, DEV)
+    total = pool.free_pages()
+    paged = tk.taskkv_compress_paged(params, qs, ks, vs, pool)
+    assert paged.status() == 0 and pool.free_pages() == total - pages
+    lens = flat.lengths()
+    assert np.array_equal(paged.lengths(), lens) and np.array_equal(paged.classes(), flat.classes())
+    assert np.array_equal(paged.query(tk.Q_INDICES), flat.query(tk.Q_INDICES))
+    tab = paged.query(tk.Q_PAGETAB)
+    used = np.concatenate([tab[u, :(lens[u] + P - 1) // P] for u in range(len(lens))])
+    assert len(set(used.tolist())) == len(used) == pages and used.min() >= 0 and used.max() < pool.n_pages
+    for u in range(len(lens)):
+        for which in ("k", "v"):
+            assert torch.equal(paged.pool_rows(which, u).view(torch.uint8), flat.pool_rows(which, u).view(torch.uint8))
+    # one layer against the oracle, straight from the paged cache
+    rep = Pm.Report()
+    ref = Pm.oracle_layer(wl, 0, 1, qs[0][1], ks[0][1], vs[0][1])
+    Pm.compare_layer(paged, wl, 0, 1, ref, rep, v=vs[0][1])
+    rep.check_bounds(wl.name)
+    # decode: units cross page ends at different steps (lengths differ by unit)
+    R = wl.n_layers
+    for s_ in range(steps):
+        q, kn, vn = W.gen_decode_step(wl, s_, DEV)
+        if s_ % 3 == 0:
+            flat.taskkv_append(kn, vn)
+            paged.taskkv_append(kn, vn)
+            a, b = flat.taskkv_decode(q), paged.taskkv_decode(q)
+        elif s_ % 3 == 1:
+            a, b = flat.taskkv_decode_step(q, kn, vn), paged.taskkv_decode_step(q, kn, vn)
+        else:
+            a, b = flat.taskkv_decode_step(q, kn, vn), torch.empty_like(q)
+            for r in range(R):
+                b[:, r:r + 1] = paged.taskkv_decode_step_ex(q[:, r:r + 1].contiguous(), kn[:, r:r + 1].contiguous(),
+                                                            vn[:, r:r + 1].contiguous(), r, 1)
+        assert torch.equal(a.view(torch.uint8), b.view(torch.uint8)), f"step {s_}"
+    assert paged.status() == 0 and flat.status() == 0
+    lens2 = paged.lengths()
+    assert np.array_equal(lens2, lens + steps)
+    held = int(sum((int(x) + P - 1) // P for x in lens2))
+    assert held > pages and pool.free_pages() == total - held          # the host's count, page for page
+    for u in (0, len(lens) - 1):
+        assert torch.equal(paged.pool_rows("k", u).view(torch.uint8), flat.pool_rows("k", u).view(torch.uint8))
+    # the decode attention of the paged cache against the oracle on its own rows
+    q, _, _ = W.gen_decode_step(wl, 999, DEV)
+    out = paged.taskkv_decode(q)
+    G = wl.group
+    for u in (1, len(lens) - 2):
+        b_, r_, h_ = u // (R * wl.n_kv_heads), (u // wl.n_kv_heads) % R, u % wl.n_kv_heads
+        kc, vc = Pm.to64(paged.pool_rows("k", u)), Pm.to64(paged.pool_rows("v", u))
+        for g in range(G):
+            want = O.decode_attention(Pm.to64(q[b_, r_, h_ * G + g]), kc, vc)
+            assert np.abs(Pm.to64(out[b_, r_, h_ * G + g]) - want).max() < Pm.TOL_OUT[wl.dtype]
+    paged.close()
+    assert pool.free_pages() == total
+    flat.close()
+    pool.close()
+
+
+def test_paged_caches_share_a_pool_and_reuse_freed_pages():
+    """Two caches in one pool; the pool is sized so that a third fits only after the first is destroyed.  A
+    compression that would not fit is refused (EALLOC) before anything is launched and leaves the count untouched;
+    after the destruction the third cache gets the freed pages and is as correct as the others; an append that
+    needs more pages than are left is refused as well."""
+    tk = _tk()
+    P = 64
+    wls = [small(f"pool{i}", n=8, n_kv=4, d=128, N=0, L=32, s1=4, s2=64, k=100, dtype="bf16", R=2,
+                 seq_lens=[(1500, 1800, 1500)[i]], nh=1, steps=4, seed=50 + i) for i in range(3)]
+    need = [tk.taskkv_plan_paged(tk.params_from_workload(w, max_new_tokens=200), P)[1] for w in wls]
+    assert need[2] == need[0]                   # Eq. 16 fixes the number of full heads: pages depend on the lengths only
+    pool = tk.Pool(P, need[0] + need[1] + 9, 128, "bf16", DEV)
+    data = [W.materialize(w, DEV) for w in wls]
+    params = [tk.params_from_workload(w, max_new_tokens=200) for w in wls]
+    caches = [tk.taskkv_compress_paged(params[i], *data[i], pool) for i in range(2)]
+    assert pool.free_pages() == 9
+    with pytest.raises(tk.TaskKVError) as ei:
+        tk.taskkv_compress_paged(params[2], *data[2], pool)
+    assert ei.value.status == tk.EALLOC and pool.free_pages() == 9
+    flats = [tk.taskkv_compress_ex(params[i], *data[i]) for i in range(3)]
+
+    def step(i, s_):
+        q, kn, vn = W.gen_decode_step(wls[i], s_, DEV)
+        a = flats[i].taskkv_decode_step(q, kn, vn)
+        b = caches[i].taskkv_decode_step(q, kn, vn)
+        assert torch.equal(a.view(torch.uint8), b.view(torch.uint8))
+
+    step(0, 0)
+    step(1, 0)
+    caches[0].close()
+    assert pool.free_pages() >= need[0] + 9 - 8                      # cache 1 may have opened up to 8 pages
+    caches[0] = None
+    third = tk.taskkv_compress_paged(params[2], *data[2], pool)         # takes the pages cache 0 gave back
+    caches.append(third)
+    assert third.status() == 0
+    assert np.array_equal(third.lengths(), flats[2].lengths())
+    for u in range(8):
+        assert torch.equal(third.pool_rows("v", u).view(torch.uint8), flats[2].pool_rows("v", u).view(torch.uint8))
+    step(1, 1)
+    step(2, 0)
+    # run the pool dry: appends are refused once a step needs more pages than are left, and nothing is corrupted
+    refused = False
+    for s_ in range(1, 200):
+        q, kn, vn = W.gen_decode_step(wls[2], s_, DEV)
+        try:
+            b = third.taskkv_decode_step(q, kn, vn)
+        except tk.TaskKVError as exc:
+            assert exc.status == tk.EALLOC
+            refused = True
+            break
+        a = flats[2].taskkv_decode_step(q, kn, vn)
+        assert torch.equal(a.view(torch.uint8), b.view(torch.uint8))
+    assert refused and third.status() == 0 and caches[1].status() == 0
+    step(1, 2) if pool.free_pages() >= 8 else None
+    for c in caches:
+        if c is not None:
+            c.close()
+    assert pool.free_pages() == pool.n_pages
+    for f in flats:
+        f.close()
+    pool.close()
