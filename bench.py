@@ -401,10 +401,12 @@ def run_paged(tk, wl, qs, ks, vs, steps_in, args, comp_bytes, decode_bytes, peak
     as the contiguous cache."""
     import torch
     n_dec = len(steps_in)
-    params = tk.params_from_workload(wl, max_new_tokens=4 * n_dec + 4, mid_policy=POLICIES[args.policy])
+    params = tk.params_from_workload(wl, max_new_tokens=n_dec, mid_policy=POLICIES[args.policy])
     P = args.page_rows
     info, pages = tk.taskkv_plan_paged(params, P)
-    pool = tk.Pool(P, pages + 2 * int(info.n_units), wl.head_dim, wl.dtype, qs[0].device)
+    pool = tk.Pool(P, pages + (n_dec // P + 2) * int(info.n_units), wl.head_dim, wl.dtype, qs[0].device)
+    cmem = torch.empty(int(info.cache_bytes), dtype=torch.uint8, device=qs[0].device)
+    wmem = torch.empty(int(info.workspace_bytes), dtype=torch.uint8, device=qs[0].device)
     stream = torch.cuda.current_stream()
 
     def timed(fn):
@@ -419,7 +421,7 @@ def run_paged(tk, wl, qs, ks, vs, steps_in, args, comp_bytes, decode_bytes, peak
     comp, dec = [], []
     status = 0
     for it in range(4):
-        ms, cache = timed(lambda: tk.taskkv_compress_paged(params, qs, ks, vs, pool))
+        ms, cache = timed(lambda: tk.taskkv_compress_paged(params, qs, ks, vs, pool, cache_mem=cmem, workspace_mem=wmem))
         out = torch.empty_like(steps_in[0][0])
 
         def steps():
@@ -432,6 +434,20 @@ def run_paged(tk, wl, qs, ks, vs, steps_in, args, comp_bytes, decode_bytes, peak
             dec.append(msd / n_dec)
         status = max(status, cache.status())
         cache.close()
+    # per-kernel durations of one more pass, every launch bracketed by events
+    tk.taskkv_timing_enable(True)
+    cache = tk.taskkv_compress_paged(params, qs, ks, vs, pool, cache_mem=cmem, workspace_mem=wmem)
+    for (q, kn, vn) in steps_in:
+        cache.taskkv_decode_step(q, kn, vn, out=out)
+    torch.cuda.synchronize()
+    recs = tk.taskkv_timing_collect()
+    tk.taskkv_timing_enable(False)
+    cache.close()
+    per = {}
+    for name, ms in recs:
+        a = per.setdefault(name, [0, 0.0])
+        a[0] += 1
+        a[1] += ms
     free_after = pool.free_pages()
     n_pages = pool.n_pages
     pool.close()
@@ -439,7 +455,7 @@ def run_paged(tk, wl, qs, ks, vs, steps_in, args, comp_bytes, decode_bytes, peak
     return {"page_rows": P, "pages": pages, "pool_pages": n_pages, "all_pages_returned": free_after == n_pages,
             "compress_ms": cms, "compress_frac_of_peak": comp_bytes / (cms * 1e-3) / 1e9 / peak,
             "decode_ms_per_step": dms, "decode_frac_of_peak": decode_bytes / (dms * 1e-3) / 1e9 / peak,
-            "device_status": status}
+            "kernel_avg_ms": {k: v[1] / v[0] for k, v in per.items()}, "device_status": status}
 
 
 def run_layer_streamed(tk, wl, qs, ks, vs, args, steps_in):

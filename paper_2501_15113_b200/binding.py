@@ -553,12 +553,17 @@ def taskkv_plan_paged(params: Params, page_rows: int):
 
 
 def taskkv_compress_paged(params: Params, q_win: Sequence[torch.Tensor], k: Sequence[torch.Tensor],
-                          v: Sequence[torch.Tensor], pool: Pool, stream=None) -> Cache:
+                          v: Sequence[torch.Tensor], pool: Pool, stream=None,
+                          cache_mem: Optional[torch.Tensor] = None,
+                          workspace_mem: Optional[torch.Tensor] = None) -> Cache:
     """As taskkv_compress_ex, the compacted rows going to pages of `pool`."""
-    info, _ = taskkv_plan_paged(params, pool.page_rows)
     dev = k[0].device
-    cache_mem = torch.empty(int(info.cache_bytes), dtype=torch.uint8, device=dev)
-    workspace_mem = torch.empty(int(info.workspace_bytes), dtype=torch.uint8, device=dev)
+    if cache_mem is None or workspace_mem is None:
+        info, _ = taskkv_plan_paged(params, pool.page_rows)
+        if cache_mem is None:
+            cache_mem = torch.empty(int(info.cache_bytes), dtype=torch.uint8, device=dev)
+        if workspace_mem is None:
+            workspace_mem = torch.empty(int(info.workspace_bytes), dtype=torch.uint8, device=dev)
     for t in list(q_win) + list(k) + list(v):
         if not t.is_contiguous() or not t.is_cuda:
             raise ValueError("inputs must be contiguous CUDA tensors")

@@ -292,6 +292,21 @@ __device__ __forceinline__ int upper_unit(const int32_t* off, int n, int x) {
   return lo;
 }
 
+// The same by all 32 lanes of a converged warp: 32 probes per round, so 1024 entries take two dependent loads instead
+// of ten.  Every lane returns the index.
+__device__ __forceinline__ int upper_unit_warp(const int32_t* off, int n, int x, int lane) {
+  int lo = 0, hi = n;                                   // off[lo] <= x < off[hi]
+  while (hi - lo > 1) {
+    const int step = (hi - lo + 31) >> 5;
+    const int at = lo + (lane + 1) * step;
+    const bool le = at < hi && off[at] <= x;            // true for the lanes below some point: off is non-decreasing
+    const int c = __popc(__ballot_sync(0xffffffffu, le));
+    hi = min(hi, lo + (c + 1) * step);
+    lo += c * step;
+  }
+  return lo;
+}
+
 __device__ __forceinline__ void set_status(int32_t* status, int32_t code) { atomicCAS(status, 0, code); }
 
 // Pool row of row r of unit u (seg = seg_off[u]).  Rows r .. r + n - 1 are consecutive pool rows as long as they do

@@ -21,7 +21,41 @@ constexpr int kAttnWarps = kAttnThreads / 32;
 constexpr int kUnroll = 4;
 
 // PAGED (both attention kernels): the rows of a unit live in pages of the shared pool; the rows one loop iteration
-// touches never cross a page (a page holds a multiple of 64 rows), so an iteration looks its page up once.
+// touches never cross a page (a page holds a multiple of 64 rows).  A work item's 512 rows lie in at most 8 pages:
+// every lane reads one of their table entries when the item starts (lane i and i + 8, ... hold the i-th), and an
+// iteration gets its page by a shuffle, so no table load sits between an iteration and its row loads.
+struct ItemPages {
+  int first;   // table index of the item's first page
+  int mine;    // page held by this lane
+};
+__device__ __forceinline__ ItemPages item_pages(const DeviceProblem& p, int u, int rbeg, int lane) {
+  ItemPages ip;
+  ip.first = rbeg / p.page_rows;
+  const int pi = ip.first + (lane & 7);
+  ip.mine = pi < p.page_stride ? p.page_tab[(size_t)u * p.page_stride + pi] : 0;
+  return ip;
+}
+// Walks the item's rows in steps of at most one page: where() gives the pool row of the current row minus that row's
+// index (for all lanes of a converged warp), advance() moves on.  One division per item instead of one per step.
+struct PageWalk {
+  int pi;    // page of the current row, counted from the item's first
+  int rem;   // its row within that page
+  __device__ __forceinline__ void start(const DeviceProblem& p, const ItemPages& ip, int r) {
+    pi = r / p.page_rows - ip.first;
+    rem = r % p.page_rows;
+  }
+  __device__ __forceinline__ size_t where(const DeviceProblem& p, const ItemPages& ip, int r) const {
+    const int pg = __shfl_sync(0xffffffffu, ip.mine, pi);
+    return (size_t)((int64_t)pg * p.page_rows + rem - r);
+  }
+  __device__ __forceinline__ void advance(const DeviceProblem& p, int step) {
+    rem += step;
+    if (rem >= p.page_rows) {
+      rem -= p.page_rows;
+      ++pi;
+    }
+  }
+};
 template <typename T, int D, int G, bool PAGED>
 __global__ void __launch_bounds__(kAttnThreads) decode_attn_kernel(DeviceProblem p, const T* __restrict__ q,
                                                                    const int32_t* __restrict__ lengths,
@@ -36,7 +70,7 @@ __global__ void __launch_bounds__(kAttnThreads) decode_attn_kernel(DeviceProblem
   __shared__ float sm_m[NSG][G];
   __shared__ float sm_l[NSG][G];
   __shared__ __align__(16) float sm_acc[NSG][G][D];
-  __shared__ int s_unit;
+  __shared__ int s_unit, s_rbeg;
 
   grid_dependency_wait();
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
@@ -50,7 +84,13 @@ __global__ void __launch_bounds__(kAttnThreads) decode_attn_kernel(DeviceProblem
 
   for (int item = item0 + blockIdx.x; item < item1; item += gridDim.x) {
     __syncthreads();                                // previous item's shared state consumed
-    if (tid == 0) s_unit = w0 + upper_unit(p.dec_off + w0, p.view_U, item);
+    if (warp == 0) {
+      const int wi = w0 + upper_unit_warp(p.dec_off + w0, p.view_U, item, lane);
+      if (lane == 0) {
+        s_unit = wi;
+        s_rbeg = (item - p.dec_off[wi]) * kDecodeChunk;
+      }
+    }
     __syncthreads();
     const int w = s_unit;
     const LmUnit lu = lm_unit(p, w);
@@ -62,7 +102,7 @@ __global__ void __launch_bounds__(kAttnThreads) decode_attn_kernel(DeviceProblem
     const int new_r = (k_new != nullptr && len < p.cap[u]) ? len : -1;
     if (new_r >= 0) ++len;
     if (lengths) len = min(max(lengths[vu], 0), len);
-    const int rbeg = (item - p.dec_off[w]) * kDecodeChunk;
+    const int rbeg = s_rbeg;
     if (rbeg >= len) continue;                      // an item of the reserve beyond the segment's length
     const int rend = min(len, rbeg + kDecodeChunk);
     const int64_t seg = p.seg_off[u];
@@ -88,6 +128,8 @@ __global__ void __launch_bounds__(kAttnThreads) decode_attn_kernel(DeviceProblem
         *reinterpret_cast<uint4*>(vd) = *reinterpret_cast<const uint4*>(vn_row + tid * 16);
       }
     }
+    ItemPages ip{0, 0};
+    if (PAGED) ip = item_pages(p, u, rbeg, lane);
     const unsigned char* kp = static_cast<const unsigned char*>(p.k_pool) + (PAGED ? 0 : (size_t)seg * ROW_BYTES) + sl * 16;
     const unsigned char* vp = static_cast<const unsigned char*>(p.v_pool) + (PAGED ? 0 : (size_t)seg * ROW_BYTES) + sl * 16;
 
@@ -110,19 +152,28 @@ __global__ void __launch_bounds__(kAttnThreads) decode_attn_kernel(DeviceProblem
 
     // two copies of the row loop: only the item that holds the new token's row pays for telling it apart
     auto rows_loop = [&](auto has_new) {
+    PageWalk pw{0, 0};
+    if (PAGED) pw.start(p, ip, rbeg);
     for (int base = rbeg; base < rend; base += NSG * kUnroll) {   // warp-uniform trip count
       const int r0 = base + gsg;
       // pool row of row `base` minus base: adding a row index of this iteration gives its pool row
-      const size_t rowoff = PAGED ? pool_row(p, u, seg, base) - (size_t)base : 0;
+      size_t rowoff = 0;
+      if (PAGED) {
+        rowoff = pw.where(p, ip, base);
+        pw.advance(p, NSG * kUnroll);
+      }
       uint4 kraw[kUnroll], vraw[kUnroll];
+      // one 64-bit address per array and iteration; the unrolled loads differ by compile-time offsets
+      const unsigned char* kb = kp + (rowoff + (size_t)r0) * ROW_BYTES;
+      const unsigned char* vb = vp + (rowoff + (size_t)r0) * ROW_BYTES;
 #pragma unroll
       for (int i = 0; i < kUnroll; ++i) {
         const int r = r0 + i * NSG;
         if (r < rend) {
           kraw[i] = *reinterpret_cast<const uint4*>((decltype(has_new)::value && r == new_r) ? kn_row + sl * 16
-                                                                                             : kp + (rowoff + (size_t)r) * ROW_BYTES);
+                                                                                             : kb + i * NSG * ROW_BYTES);
           vraw[i] = *reinterpret_cast<const uint4*>((decltype(has_new)::value && r == new_r) ? vn_row + sl * 16
-                                                                                             : vp + (rowoff + (size_t)r) * ROW_BYTES);
+                                                                                             : vb + i * NSG * ROW_BYTES);
         } else {
           kraw[i] = make_uint4(0, 0, 0, 0);
           vraw[i] = make_uint4(0, 0, 0, 0);
@@ -247,7 +298,7 @@ __device__ __forceinline__ uint32_t word_of(const uint4& v, int i) {
 }
 
 template <int D, int G, bool PAGED>
-__global__ void __launch_bounds__(kAttnThreads) decode_attn_mma_kernel(DeviceProblem p,
+__global__ void __launch_bounds__(kAttnThreads, 4) decode_attn_mma_kernel(DeviceProblem p,
                                                                        const __nv_bfloat16* __restrict__ q,
                                                                        const int32_t* __restrict__ lengths,
                                                                        const unsigned char* __restrict__ k_new,
@@ -262,7 +313,7 @@ __global__ void __launch_bounds__(kAttnThreads) decode_attn_mma_kernel(DevicePro
   __shared__ float sm_m[kAttnWarps][G];
   __shared__ float sm_l[kAttnWarps][G];
   __shared__ __align__(16) float sm_acc[kAttnWarps][G][D];
-  __shared__ int s_unit;
+  __shared__ int s_unit, s_rbeg;
 
   grid_dependency_wait();
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
@@ -277,7 +328,13 @@ __global__ void __launch_bounds__(kAttnThreads) decode_attn_mma_kernel(DevicePro
 
   for (int item = item0 + blockIdx.x; item < item1; item += gridDim.x) {
     __syncthreads();
-    if (tid == 0) s_unit = w0 + upper_unit(p.dec_off + w0, p.view_U, item);
+    if (warp == 0) {
+      const int wi = w0 + upper_unit_warp(p.dec_off + w0, p.view_U, item, lane);
+      if (lane == 0) {
+        s_unit = wi;
+        s_rbeg = (item - p.dec_off[wi]) * kDecodeChunk;
+      }
+    }
     __syncthreads();
     const int w = s_unit;
     const LmUnit lu = lm_unit(p, w);
@@ -289,7 +346,7 @@ __global__ void __launch_bounds__(kAttnThreads) decode_attn_mma_kernel(DevicePro
     const int new_r = (k_new != nullptr && len < p.cap[u]) ? len : -1;
     if (new_r >= 0) ++len;
     if (lengths) len = min(max(lengths[vu], 0), len);
-    const int rbeg = (item - p.dec_off[w]) * kDecodeChunk;
+    const int rbeg = s_rbeg;
     if (rbeg >= len) continue;                      // an item of the reserve beyond the segment's length
     const int rend = min(len, rbeg + kDecodeChunk);
     const int64_t seg = p.seg_off[u];
@@ -315,8 +372,10 @@ __global__ void __launch_bounds__(kAttnThreads) decode_attn_mma_kernel(DevicePro
         *reinterpret_cast<uint4*>(vd) = *reinterpret_cast<const uint4*>(vn_row + tid * 16);
       }
     }
-    const unsigned char* kp = static_cast<const unsigned char*>(p.k_pool) + (PAGED ? 0 : (size_t)seg * ROW_BYTES);
-    const unsigned char* vp = static_cast<const unsigned char*>(p.v_pool) + (PAGED ? 0 : (size_t)seg * ROW_BYTES);
+    ItemPages ip{0, 0};
+    if (PAGED) ip = item_pages(p, u, rbeg, lane);
+    const unsigned char* kp = static_cast<const unsigned char*>(p.k_pool);
+    const unsigned char* vp = static_cast<const unsigned char*>(p.v_pool);
 
     // Q fragments: head g on M row g
     uint32_t qa[KC][2];
@@ -334,20 +393,34 @@ __global__ void __launch_bounds__(kAttnThreads) decode_attn_mma_kernel(DevicePro
 #pragma unroll
       for (int e = 0; e < 4; ++e) o[mb][e] = 0.f;
 
+    // byte offset of this lane's first K vector (row g, piece t) and V vector (row 2t, piece g) within a block
+    const int klane = g * ROW_BYTES + t * 16, vlane = 2 * t * ROW_BYTES + g * 16;
     // two copies of the row loop: only the item that holds the new token's row pays for telling it apart
     auto rows_loop = [&](auto has_new) {
+    PageWalk pw{0, 0};
+    if (PAGED) pw.start(p, ip, rbeg + warp * kBlk);
+    // kb, vb: this lane's first K and V vector of the current 16-row block; the unrolled loads differ from them by
+    // compile-time offsets.  Contiguous layout: row r of the unit is pool row seg + r, the pointers step from block
+    // to block; paged: they are set from the block's page.
+    const unsigned char* kb = kp + ((size_t)seg + (size_t)(rbeg + warp * kBlk)) * ROW_BYTES + klane;
+    const unsigned char* vb = vp + ((size_t)seg + (size_t)(rbeg + warp * kBlk)) * ROW_BYTES + vlane;
     for (int blk = rbeg + warp * kBlk; blk < rend; blk += kAttnWarps * kBlk) {   // warp-uniform
-      // pool row of row `blk` minus blk: adding a row index of this 16-row block gives its pool row
-      const size_t rowoff = PAGED ? pool_row(p, u, seg, blk) - (size_t)blk : 0;
+      if (PAGED) {
+        // pool row of row `blk` minus blk: adding a row index of this 16-row block gives its pool row
+        const size_t rowoff = pw.where(p, ip, blk);
+        pw.advance(p, kAttnWarps * kBlk);
+        kb = kp + (rowoff + (size_t)blk) * ROW_BYTES + klane;
+        vb = vp + (rowoff + (size_t)blk) * ROW_BYTES + vlane;
+      }
       uint4 kraw[2][KP], vraw[4][VP];
 #pragma unroll
       for (int j = 0; j < 2; ++j) {
         const int r = blk + 8 * j + g;
 #pragma unroll
         for (int i = 0; i < KP; ++i)
-          kraw[j][i] = r < rend ? *reinterpret_cast<const uint4*>(((decltype(has_new)::value && r == new_r)
-                                                                       ? kn_row : kp + (rowoff + (size_t)r) * ROW_BYTES) +
-                                                                  (i * 4 + t) * 16)
+          kraw[j][i] = r < rend ? *reinterpret_cast<const uint4*>((decltype(has_new)::value && r == new_r)
+                                                                      ? kn_row + (i * 4 + t) * 16
+                                                                      : kb + j * 8 * ROW_BYTES + i * 64)
                                 : make_uint4(0, 0, 0, 0);
       }
 #pragma unroll
@@ -355,9 +428,9 @@ __global__ void __launch_bounds__(kAttnThreads) decode_attn_mma_kernel(DevicePro
         const int r = blk + 2 * t + (x & 1) + 8 * (x >> 1);
 #pragma unroll
         for (int i = 0; i < VP; ++i)
-          vraw[x][i] = r < rend ? *reinterpret_cast<const uint4*>(((decltype(has_new)::value && r == new_r)
-                                                                       ? vn_row : vp + (rowoff + (size_t)r) * ROW_BYTES) +
-                                                                  i * 128 + g * 16)
+          vraw[x][i] = r < rend ? *reinterpret_cast<const uint4*>((decltype(has_new)::value && r == new_r)
+                                                                      ? vn_row + i * 128 + g * 16
+                                                                      : vb + ((x & 1) + 8 * (x >> 1)) * ROW_BYTES + i * 128)
                                 : make_uint4(0, 0, 0, 0);
       }
       // S^T for the two 8-row halves of the block
@@ -414,6 +487,10 @@ __global__ void __launch_bounds__(kAttnThreads) decode_attn_mma_kernel(DevicePro
           a[2 + hf] = __byte_perm(word_of(vraw[2][pc], wi), word_of(vraw[3][pc], wi), sel);   // rows 2t+8, 2t+9
         }
         mma_bf16_16816(o[mb], a[0], a[1], a[2], a[3], pb0, pb1);
+      }
+      if (!PAGED) {
+        kb += kAttnWarps * kBlk * ROW_BYTES;
+        vb += kAttnWarps * kBlk * ROW_BYTES;
       }
     }
 

@@ -29,7 +29,10 @@ __global__ void __launch_bounds__(kGatherThreads, 10) gather_kernel(DeviceProble
   __shared__ int s_w;
   grid_dependency_wait();
   const int item = item0 + (int)blockIdx.x;
-  if (threadIdx.x == 0) s_w = w0 + upper_unit(p.gather_off + w0, wn, item);
+  if (threadIdx.x < 32) {
+    const int wi = w0 + upper_unit_warp(p.gather_off + w0, wn, item, (int)threadIdx.x);
+    if (threadIdx.x == 0) s_w = wi;
+  }
   __syncthreads();
   const int w = s_w;
   const int u = lm_unit(p, w).u;
