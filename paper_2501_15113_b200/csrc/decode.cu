@@ -534,13 +534,22 @@ __global__ void __launch_bounds__(kAttnThreads, 4) decode_attn_mma_kernel(Device
 // One block per (view unit, query head of the group): merge the unit's partials.  First the block finds
 // the largest running maximum, then each warp accumulates every fourth partial against it (independent
 // loads, fixed order), and the four warps are summed in shared memory.
+constexpr int kCombineThreads = 256;
+constexpr int kCombineWarps = kCombineThreads / 32;
+constexpr int kCombineStage = 1024;     // partial results weighted per round (one round up to 524288 rows)
+
+// One block per (view unit, query head of the group).  The weights exp2(m_i - M) of the unit's partial results
+// are computed once, by all threads, into shared memory; the accumulation loop then has nothing but independent
+// 16-byte loads in it (a long unit has over a hundred partials and one block: its latency is the kernel's).
 template <typename T, int D, int G>
-__global__ void __launch_bounds__(kAttnThreads) decode_combine_kernel(DeviceProblem p, const int32_t* __restrict__ lengths,
-                                                                      int fused_step, T* __restrict__ out) {
+__global__ void __launch_bounds__(kCombineThreads) decode_combine_kernel(DeviceProblem p,
+                                                                         const int32_t* __restrict__ lengths,
+                                                                         int fused_step, T* __restrict__ out) {
   constexpr int EPL = D / 32;
-  __shared__ float s_max[kAttnWarps];
-  __shared__ float s_l[kAttnWarps];
-  __shared__ float s_acc[kAttnWarps][D];
+  __shared__ float s_red[kCombineWarps];
+  __shared__ float s_l[kCombineWarps];
+  __shared__ float s_w[kCombineStage];
+  __shared__ __align__(16) float s_acc[kCombineWarps][D];
   grid_dependency_wait();
   const int u = blockIdx.x / G, g = blockIdx.x % G;     // u: view unit
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
@@ -552,33 +561,57 @@ __global__ void __launch_bounds__(kAttnThreads) decode_combine_kernel(DeviceProb
   if (lengths) len = min(max(lengths[u], 0), len);
   // the unit's items that hold rows (the table also numbers the reserve for appended tokens)
   const int i0 = p.dec_off[lm_index(p, unit)], i1 = i0 + (len + kDecodeChunk - 1) / kDecodeChunk;
+  const float2* ml = reinterpret_cast<const float2*>(p.part_ml);
   float M = -INFINITY;
-  for (int i = i0 + tid; i < i1; i += kAttnThreads) M = fmaxf(M, p.part_ml[((size_t)i * G + g) * 2]);
+  for (int i = i0 + tid; i < i1; i += kCombineThreads) M = fmaxf(M, ml[(size_t)i * G + g].x);
   M = warp_max(M);
-  if (lane == 0) s_max[warp] = M;
+  if (lane == 0) s_red[warp] = M;
   __syncthreads();
-  M = fmaxf(fmaxf(s_max[0], s_max[1]), fmaxf(s_max[2], s_max[3]));
+  M = s_red[0];
+#pragma unroll
+  for (int w = 1; w < kCombineWarps; ++w) M = fmaxf(M, s_red[w]);
   float acc[EPL];
 #pragma unroll
   for (int e = 0; e < EPL; ++e) acc[e] = 0.f;
   float L = 0.f;
-#pragma unroll 4
-  for (int i = i0 + warp; i < i1; i += kAttnWarps) {
-    const float mi = p.part_ml[((size_t)i * G + g) * 2];
-    const float li = p.part_ml[((size_t)i * G + g) * 2 + 1];
-    const float wgt = (mi == -INFINITY) ? 0.f : exp2f(mi - M);
-    L = fmaf(wgt, li, L);
-    const float* pa = p.part_acc + ((size_t)i * G + g) * D + lane * EPL;
+  for (int c0 = i0; c0 < i1; c0 += kCombineStage) {
+    const int cn = min(kCombineStage, i1 - c0);
+    __syncthreads();                                    // the previous round's weights have been used
+    for (int j = tid; j < cn; j += kCombineThreads) {
+      const float2 v = ml[(size_t)(c0 + j) * G + g];
+      const float wgt = (v.x == -INFINITY) ? 0.f : exp2f(v.x - M);
+      s_w[j] = wgt;
+      L = fmaf(wgt, v.y, L);
+    }
+    __syncthreads();
+#pragma unroll 8
+    for (int j = warp; j < cn; j += kCombineWarps) {
+      const float wgt = s_w[j];
+      const float* pa = p.part_acc + ((size_t)(c0 + j) * G + g) * D + lane * EPL;
+      float v[EPL];
+      if constexpr (EPL == 4) {
+        const float4 t = *reinterpret_cast<const float4*>(pa);
+        v[0] = t.x; v[1] = t.y; v[2] = t.z; v[3] = t.w;
+      } else {
+        const float2 t = *reinterpret_cast<const float2*>(pa);
+        v[0] = t.x; v[1] = t.y;
+      }
 #pragma unroll
-    for (int e = 0; e < EPL; ++e) acc[e] = fmaf(wgt, pa[e], acc[e]);
+      for (int e = 0; e < EPL; ++e) acc[e] = fmaf(wgt, v[e], acc[e]);
+    }
   }
+  L = warp_sum(L);
 #pragma unroll
   for (int e = 0; e < EPL; ++e) s_acc[warp][lane * EPL + e] = acc[e];
   if (lane == 0) s_l[warp] = L;
   __syncthreads();
   if (tid < D) {
-    const float Lt = (s_l[0] + s_l[1]) + (s_l[2] + s_l[3]);
-    const float a = (s_acc[0][tid] + s_acc[1][tid]) + (s_acc[2][tid] + s_acc[3][tid]);
+    float Lt = 0.f, a = 0.f;
+#pragma unroll
+    for (int w = 0; w < kCombineWarps; ++w) {
+      Lt += s_l[w];
+      a += s_acc[w][tid];
+    }
     store_out(out + ((size_t)u * G + g) * D + tid, Lt > 0.f ? a / Lt : 0.f);
   }
   // fused step: the last of the unit's G blocks (each has read the old length by now) raises the length
@@ -617,7 +650,7 @@ cudaError_t launch_typed(const DeviceProblem& p, const void* q, const int32_t* l
   if (e != cudaSuccess) return e;
   {
     LaunchScope ls(K_DECODE_COMBINE, s);
-    e = launch_dependent(decode_combine_kernel<T, D, G>, (unsigned)(p.view_U * G), kAttnThreads, s, p, lengths,
+    e = launch_dependent(decode_combine_kernel<T, D, G>, (unsigned)(p.view_U * G), kCombineThreads, s, p, lengths,
                          k_new != nullptr ? 1 : 0, static_cast<T*>(out));
   }
   return e;
