@@ -254,7 +254,9 @@ taskkv_status taskkv_compress_shard_finish(taskkv_cache* c, const float* sem_all
  *   taskkv_pool_create    a pool of n_pages pages of page_rows rows (a multiple of 64) of head_dim elements of
  *                         `dtype`, for K and for V, in `mem` (device, 256-byte aligned, at least
  *                         taskkv_pool_bytes(...) bytes, owned by the caller) or, with mem == NULL, in memory the
- *                         library allocates.
+ *                         library allocates.  Layout of that memory: the K pages [n_pages][page_rows][head_dim],
+ *                         the V pages likewise from the next multiple of 256 bytes, then the library's list of
+ *                         free pages.
  *   taskkv_compress_paged as taskkv_compress_ex, with the compacted rows going to pages of `pool`; cache_mem then
  *                         holds only tables (taskkv_plan_paged gives the sizes and the pages the compression takes).
  *                         max_new_tokens still bounds how far a unit may grow (it sizes the page tables and the

@@ -426,19 +426,16 @@ class Cache:
         ln = int(self.query(Q_LENGTHS)[u])
         d = self.params.c.head_dim
         es = 2 if self.params.c.dtype == BF16 else 4
-        raw = self.query(Q_KPOOL if which == "k" else Q_VPOOL)
         if self._keep is not None and "pool" in self._keep:
-            P = self._keep["pool"].page_rows
-            tab = self.query(Q_PAGETAB)[u]
-            parts = []
-            for i in range((ln + P - 1) // P):
-                rows = min(P, ln - i * P)
-                start = int(tab[i]) * P * d * es
-                parts.append(raw[start:start + rows * d * es])
-            seg = np.concatenate(parts) if parts else raw[:0]
-        else:
-            off = self.query(Q_OFFSETS)
-            seg = raw[int(off[u]) * d * es:(int(off[u]) + ln) * d * es]
+            pool = self._keep["pool"]
+            P = pool.page_rows
+            n = (ln + P - 1) // P
+            tab = torch.from_numpy(self.query(Q_PAGETAB)[u, :n].astype(np.int64)).to(pool.mem.device)
+            pages = (pool.k_pages if which == "k" else pool.v_pages)[tab]          # [n, P, d]
+            return pages.reshape(n * P, d)[:ln].cpu().contiguous()
+        raw = self.query(Q_KPOOL if which == "k" else Q_VPOOL)
+        off = self.query(Q_OFFSETS)
+        seg = raw[int(off[u]) * d * es:(int(off[u]) + ln) * d * es]
         t = torch.from_numpy(seg.copy())
         return t.view(self.params.torch_dtype).reshape(ln, d)
 
@@ -528,6 +525,12 @@ class Pool:
             raise TaskKVError(EINVAL, "taskkv_pool_bytes")
         self.mem = torch.empty(nbytes, dtype=torch.uint8, device=device)
         self.page_rows, self.n_pages = page_rows, n_pages
+        # layout of the pool memory (taskkv.h): K pages, then V pages from the next multiple of 256 bytes
+        tdt = torch.bfloat16 if dt == BF16 else torch.float32
+        page_bytes = page_rows * head_dim * (2 if dt == BF16 else 4)
+        v_off = (n_pages * page_bytes + 255) // 256 * 256
+        self.k_pages = self.mem[:n_pages * page_bytes].view(tdt).view(n_pages, page_rows, head_dim)
+        self.v_pages = self.mem[v_off:v_off + n_pages * page_bytes].view(tdt).view(n_pages, page_rows, head_dim)
         h = C.c_void_p()
         with torch.cuda.device(self.mem.device):
             _check(lib.taskkv_pool_create(page_rows, n_pages, head_dim, dt, self.mem.data_ptr(), nbytes,

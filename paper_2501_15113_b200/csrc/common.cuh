@@ -190,6 +190,11 @@ cudaError_t launch_decode(const DeviceProblem& p, int dtype, const void* q, cons
 // kernels: attention -> combine -> attention of a layer-by-layer decode loop, separator -> plan -> gather.
 #ifdef __CUDACC__
 __device__ __forceinline__ void grid_dependency_wait() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
+// Lets the next kernel in the stream (if launched with launch_dependent()) become resident once every block of this
+// grid has got here or exited: its blocks then run whatever they do before their own grid_dependency_wait() -- reads
+// of tables this grid does not write -- under this grid's tail.  Called after this kernel's own wait, so that by the
+// time a dependent block runs, everything before this grid in the stream is complete.
+__device__ __forceinline__ void grid_launch_dependents() { asm volatile("griddepcontrol.launch_dependents;" ::: "memory"); }
 
 template <class... KArgs, class... Args>
 cudaError_t launch_dependent(void (*kernel)(KArgs...), unsigned grid, unsigned block, cudaStream_t s, Args... args) {

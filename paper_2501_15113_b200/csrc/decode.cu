@@ -72,7 +72,6 @@ __global__ void __launch_bounds__(kAttnThreads) decode_attn_kernel(DeviceProblem
   __shared__ __align__(16) float sm_acc[NSG][G][D];
   __shared__ int s_unit, s_rbeg;
 
-  grid_dependency_wait();
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
   const int sg = lane / LPR, sl = lane % LPR;
   const int gsg = warp * RPW + sg;
@@ -82,10 +81,18 @@ __global__ void __launch_bounds__(kAttnThreads) decode_attn_kernel(DeviceProblem
   const int item0 = p.dec_base[p.view_l0 * lm_batch(p)], item1 = p.dec_base[(p.view_l0 + p.view_nl) * lm_batch(p)];
   const float scale2 = kLog2e * rsqrtf((float)D);
 
+  // The table of work items is written when the cache is planned, not by the kernel before this one in the
+  // stream: the block's first item is looked up before the wait, under that kernel's tail.
+  int wi_first = 0;
+  if (warp == 0 && item0 + (int)blockIdx.x < item1)
+    wi_first = w0 + upper_unit_warp(p.dec_off + w0, p.view_U, item0 + (int)blockIdx.x, lane);
+  grid_dependency_wait();
+  grid_launch_dependents();
   for (int item = item0 + blockIdx.x; item < item1; item += gridDim.x) {
     __syncthreads();                                // previous item's shared state consumed
     if (warp == 0) {
-      const int wi = w0 + upper_unit_warp(p.dec_off + w0, p.view_U, item, lane);
+      const int wi = item == item0 + (int)blockIdx.x ? wi_first
+                                                     : w0 + upper_unit_warp(p.dec_off + w0, p.view_U, item, lane);
       if (lane == 0) {
         s_unit = wi;
         s_rbeg = (item - p.dec_off[wi]) * kDecodeChunk;
@@ -315,7 +322,6 @@ __global__ void __launch_bounds__(kAttnThreads, 4) decode_attn_mma_kernel(Device
   __shared__ __align__(16) float sm_acc[kAttnWarps][G][D];
   __shared__ int s_unit, s_rbeg;
 
-  grid_dependency_wait();
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
   const int g = lane >> 2, t = lane & 3;
   // the view's layers are a contiguous range of layer-major indices, hence of work items
@@ -326,10 +332,18 @@ __global__ void __launch_bounds__(kAttnThreads, 4) decode_attn_mma_kernel(Device
   // d of accumulator row (mb, hf) of this lane's two output rows: e = hf * MB + mb, piece e / 8, element e % 8
   auto pd = [&](int mb, int hf, int gg) { const int e = hf * MB + mb; return (e >> 3) * 64 + gg * 8 + (e & 7); };
 
+  // The table of work items is written when the cache is planned, not by the kernel before this one in the
+  // stream: the block's first item is looked up before the wait, under that kernel's tail.
+  int wi_first = 0;
+  if (warp == 0 && item0 + (int)blockIdx.x < item1)
+    wi_first = w0 + upper_unit_warp(p.dec_off + w0, p.view_U, item0 + (int)blockIdx.x, lane);
+  grid_dependency_wait();
+  grid_launch_dependents();
   for (int item = item0 + blockIdx.x; item < item1; item += gridDim.x) {
     __syncthreads();
     if (warp == 0) {
-      const int wi = w0 + upper_unit_warp(p.dec_off + w0, p.view_U, item, lane);
+      const int wi = item == item0 + (int)blockIdx.x ? wi_first
+                                                     : w0 + upper_unit_warp(p.dec_off + w0, p.view_U, item, lane);
       if (lane == 0) {
         s_unit = wi;
         s_rbeg = (item - p.dec_off[wi]) * kDecodeChunk;
@@ -550,17 +564,21 @@ __global__ void __launch_bounds__(kCombineThreads) decode_combine_kernel(DeviceP
   __shared__ float s_l[kCombineWarps];
   __shared__ float s_w[kCombineStage];
   __shared__ __align__(16) float s_acc[kCombineWarps][D];
-  grid_dependency_wait();
+  // Lengths, capacities and the item table are not written by the attention kernel before this one: they are read
+  // before the wait, under that kernel's tail (the lengths were last written by this kernel's previous launch or by
+  // an append, both complete before the attention kernel let this one start).
   const int u = blockIdx.x / G, g = blockIdx.x % G;     // u: view unit
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
   const int unit = view_unit(p, u);
   int len = p.len[unit];
-  const bool grown = fused_step && len < p.cap[unit];   // the attention pass has appended the new token's row
+  const bool grown = fused_step && len < p.cap[unit];   // the attention pass appends the new token's row
   const int len_next = len + (grown ? 1 : 0);
   len = len_next;
   if (lengths) len = min(max(lengths[u], 0), len);
   // the unit's items that hold rows (the table also numbers the reserve for appended tokens)
   const int i0 = p.dec_off[lm_index(p, unit)], i1 = i0 + (len + kDecodeChunk - 1) / kDecodeChunk;
+  grid_dependency_wait();
+  grid_launch_dependents();
   const float2* ml = reinterpret_cast<const float2*>(p.part_ml);
   float M = -INFINITY;
   for (int i = i0 + tid; i < i1; i += kCombineThreads) M = fmaxf(M, ml[(size_t)i * G + g].x);

@@ -23,16 +23,32 @@ def _parity():
 
 
 def run_workload(wl: W.Workload, layers=None, decode_steps=None, check_pool=True, force_class=-1,
-                 check_scores=True, decode_layers=None, expect_class_ties=()):
+                 check_scores=True, decode_layers=None, expect_class_ties=(), page_rows=0):
     """Compress + decode on the GPU, oracle on the chosen (b, r) pairs, compare everything.  Decode outputs are
     compared on `decode_layers` (default: every chosen pair).  Ends with the bounds every test must keep: no class
-    near-tie except at the (b, r) named in `expect_class_ties`, boundary ties within one per 10,000 selections."""
+    near-tie except at the (b, r) named in `expect_class_ties`, boundary ties within one per 10,000 selections.
+    With page_rows > 0 the cache is a paged one in a pool with room for exactly the pages the run takes."""
     import os
     tk, P = _tk(), _parity()
     qs, ks, vs = W.materialize(wl, DEV)
     steps = wl.decode_steps if decode_steps is None else decode_steps
     params = tk.params_from_workload(wl, max_new_tokens=steps, force_class=force_class)
-    cache = tk.taskkv_compress_ex(params, qs, ks, vs)
+    pool = None
+    if page_rows:
+        # exactly the pages of the compression plus those the decode steps open
+        info, pages = tk.taskkv_plan_paged(params, page_rows)
+        lens0 = []
+        for b in range(wl.batch):
+            for r in range(wl.n_layers):
+                full = min(wl.n_kv_heads, wl.n_hetero[b][r] + (1 if wl.promote_center else 0))
+                lens0 += [wl.seq_lens[b]] * full + [wl.kept_len(b, r)] * (wl.n_kv_heads - full)
+        grow = sum(-(-(x + steps) // page_rows) - -(-x // page_rows) for x in lens0)
+        assert pages == sum(-(-x // page_rows) for x in lens0)
+        pool = tk.Pool(page_rows, pages + grow, wl.head_dim, wl.dtype, DEV)
+        cache = tk.taskkv_compress_paged(params, qs, ks, vs, pool)
+        assert pool.free_pages() == grow
+    else:
+        cache = tk.taskkv_compress_ex(params, qs, ks, vs)
     assert cache.status() == 0
     rep = P.Report()
     scores = cache.query(tk.Q_SCORES) if check_scores else None
@@ -50,7 +66,7 @@ def run_workload(wl: W.Workload, layers=None, decode_steps=None, check_pool=True
     # totals the host planned must match what the device produced
     off = cache.query(tk.Q_OFFSETS)
     cap = cache.query(tk.Q_CAPACITY)
-    assert off[-1] == cache.info.pool_rows == int(cap.sum())
+    assert pool is not None or off[-1] == cache.info.pool_rows == int(cap.sum())
     assert int(cache.lengths().sum()) == cache.info.retained_rows == wl.retained_rows() or force_class != -1
 
     # decode: append + attend, every step compared on the chosen layers
@@ -73,7 +89,12 @@ def run_workload(wl: W.Workload, layers=None, decode_steps=None, check_pool=True
     lens = cache.lengths()
     assert int(lens.sum()) == int(cache.info.retained_rows) + steps * int(cache.info.n_units) or force_class != -1
     print(f"\n[{wl.name}] {rep.summary()}")
+    if pool is not None:
+        assert pool.free_pages() == 0            # the run took every page, by the host's count and on the device
     cache.close()
+    if pool is not None:
+        assert pool.free_pages() == pool.n_pages
+        pool.close()
     P.write_report(os.environ.get("PYTEST_CURRENT_TEST", wl.name).split(" ")[0], rep)
     rep.check_bounds(wl.name, expect_class_ties)
     return rep
@@ -275,6 +296,28 @@ def test_mistral_config_full_size_every_sequence():
     rep = run_workload(wl, layers=pairs, decode_steps=2, check_pool=False,
                        decode_layers=[(0, 0), (3, 17), (7, 5), (15, 31)])
     assert rep.units == 19 * 8
+
+
+def test_mistral_config_full_size_paged_cache():
+    """Config 4 at full size in a paged cache (256-row pages, the pool holding exactly the pages the run takes):
+    the oracle checks six (sequence, layer) pairs, rows read back through the page tables included, then three
+    decode steps (append + attention, units opening new pages) on three of them."""
+    from paper_2501_15113_b200 import configs
+    wl = configs.config4_mistral(decode_steps=3)
+    pairs = [(0, 0), (3, 17), (7, 5), (9, 30), (12, 1), (15, 31)]
+    rep = run_workload(wl, layers=pairs, decode_steps=3, check_pool=True, decode_layers=[(3, 17), (9, 30), (15, 31)],
+                       page_rows=256)
+    assert rep.units == 6 * 8
+
+
+def test_llama2_config_full_size_paged_cache_small_pages():
+    """Config 2 at full size in a paged cache of 64-row pages (the smallest), four layers checked by the oracle with
+    the rows read back through the page tables, 70 decode steps so that every unit opens at least one page."""
+    from paper_2501_15113_b200 import configs
+    wl = configs.config2_llama2()
+    rep = run_workload(wl, layers=[(0, r) for r in (0, 11, 20, 31)], decode_steps=70, check_pool=True,
+                       decode_layers=[(0, 11), (0, 31)], page_rows=64)
+    assert rep.units == 4 * 32
 
 
 def test_llama3_shaped_gqa_with_budget_schedule():
