@@ -388,6 +388,9 @@ taskkv_status taskkv_decode_noalloc(const void* q, const void* k_pool, const voi
 int64_t       taskkv_cache_query_bytes(const taskkv_cache* c, int32_t what);
 taskkv_status taskkv_cache_query(const taskkv_cache* c, int32_t what, void* host_dst, size_t bytes);
 taskkv_status taskkv_cache_plan(const taskkv_cache* c, taskkv_plan_info* out);
+/* Frees what the library owns of the cache (synchronising the device first if that is device memory).  A paged
+ * cache gives its pages back to the pool: the call waits for the device, pushes them onto the pool's free list and
+ * waits again, so that the next call on the pool may take them.  NULL is accepted. */
 void          taskkv_cache_destroy(taskkv_cache* c);
 
 const char*   taskkv_status_str(taskkv_status s);
