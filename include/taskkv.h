@@ -267,7 +267,10 @@ taskkv_status taskkv_compress_shard_finish(taskkv_cache* c, const float* sem_all
  * append that would not fit with EALLOC before anything is launched.  Calls that use one pool -- compressions,
  * appends and decode steps of its caches, and their destruction -- must be ordered with respect to one another by the
  * caller (one stream, or events); the pool must outlive its caches.
- * A paged cache cannot be head-sharded or filled layer by layer (EINVAL). */
+ * A paged cache cannot be head-sharded or filled layer by layer (EINVAL).
+ * Should the device find the pool empty all the same (calls on one pool that the caller did not order), the
+ * row is not stored and the cache's status word gets ESTATE; such a cache is to be destroyed, which returns the pages
+ * it verifiably holds and never writes outside the pool's list. */
 typedef struct taskkv_pool taskkv_pool;
 size_t        taskkv_pool_bytes(int32_t page_rows, int32_t n_pages, int32_t head_dim, int32_t dtype);
 taskkv_status taskkv_pool_create(int32_t page_rows, int32_t n_pages, int32_t head_dim, int32_t dtype, void* mem,

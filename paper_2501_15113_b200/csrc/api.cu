@@ -533,6 +533,7 @@ void fill_device_problem(taskkv_cache* c) {
     d.k_pool = c->pool->k_pages;
     d.v_pool = c->pool->v_pages;
     d.pool_free = c->pool->free_ids;
+    d.pool_pages = c->pool->n_pages;
     d.pool_top = c->pool->top;
   }
   if (wm) {

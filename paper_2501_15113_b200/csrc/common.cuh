@@ -97,6 +97,7 @@ struct DeviceProblem {
   // caches share; unit u's row r lives in page page_tab[u * page_stride + r / page_rows] at slot r % page_rows.
   // page_rows == 0: one contiguous segment per unit, starting at seg_off[u].
   int32_t page_rows, page_stride;
+  int32_t pool_pages;         // pages of the pool (length of pool_free)
   int32_t* page_tab;          // [U][page_stride]
   int32_t* pool_free;         // the pool's stack of free page ids; the top `*pool_top` entries are free
   int32_t* pool_top;

@@ -150,11 +150,20 @@ __global__ void __launch_bounds__(128) separator_plan_kernel(DeviceProblem p, in
 __global__ void __launch_bounds__(128) release_pages_kernel(DeviceProblem p) {
   const int u = blockIdx.x * blockDim.x + threadIdx.x;
   if (u >= p.U) return;
-  const int pages = (p.len[u] + p.page_rows - 1) / p.page_rows;
+  const int pages = min((p.len[u] + p.page_rows - 1) / p.page_rows, p.page_stride);
   if (pages <= 0) return;
   const int pos = atomicAdd(p.pool_top, pages);
   const int32_t* tab = p.page_tab + (size_t)u * p.page_stride;
-  for (int i = 0; i < pages; ++i) p.pool_free[pos + i] = tab[i];
+  // (a cache left inconsistent by an earlier ESTATE -- a pop from an empty pool -- must not write outside the stack
+  // or put a number on it that is no page)
+  bool ok = pos >= 0 && pos + pages <= p.pool_pages;
+  for (int i = 0; ok && i < pages; ++i) ok = tab[i] >= 0 && tab[i] < p.pool_pages;
+  if (ok) {
+    for (int i = 0; i < pages; ++i) p.pool_free[pos + i] = tab[i];
+  } else {
+    atomicSub(p.pool_top, pages);
+    set_status(p.status, TASKKV_ESTATE);
+  }
   p.len[u] = 0;
 }
 
