@@ -60,7 +60,8 @@ template <typename T, int D, int G, bool PAGED>
 __global__ void __launch_bounds__(kAttnThreads) decode_attn_kernel(DeviceProblem p, const T* __restrict__ q,
                                                                    const int32_t* __restrict__ lengths,
                                                                    const unsigned char* __restrict__ k_new,
-                                                                   const unsigned char* __restrict__ v_new) {
+                                                                   const unsigned char* __restrict__ v_new,
+                                                                   T* __restrict__ out) {
   constexpr int EPL = 16 / (int)sizeof(T);          // elements per lane (one 16-byte vector)
   constexpr int LPR = D / EPL;                      // lanes per row
   constexpr int RPW = 32 / LPR;                     // rows per warp instruction
@@ -71,6 +72,7 @@ __global__ void __launch_bounds__(kAttnThreads) decode_attn_kernel(DeviceProblem
   __shared__ float sm_l[NSG][G];
   __shared__ __align__(16) float sm_acc[NSG][G][D];
   __shared__ int s_unit, s_rbeg;
+  __shared__ int s_direct;     // >= 0: the item is its unit's only one, the output goes to view unit s_direct
 
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
   const int sg = lane / LPR, sl = lane % LPR;
@@ -112,6 +114,7 @@ __global__ void __launch_bounds__(kAttnThreads) decode_attn_kernel(DeviceProblem
     const int rbeg = s_rbeg;
     if (rbeg >= len) continue;                      // an item of the reserve beyond the segment's length
     const int rend = min(len, rbeg + kDecodeChunk);
+    if (tid == 0) s_direct = len <= kDecodeChunk ? vu : -1;     // read back after the row loop (no register held)
     const int64_t seg = p.seg_off[u];
     const unsigned char* kn_row = k_new + (size_t)vu * ROW_BYTES;
     const unsigned char* vn_row = v_new + (size_t)vu * ROW_BYTES;
@@ -262,6 +265,12 @@ __global__ void __launch_bounds__(kAttnThreads) decode_attn_kernel(DeviceProblem
         a = fmaf(w, sm_acc[x][g][dd], a);
         ll = fmaf(w, sm_l[x][g], ll);
       }
+      if (s_direct >= 0) {
+        // the unit's only item: this is Eq. 1 over the whole segment (what the combine pass would make of one
+        // partial, bit for bit); the combine pass skips such units
+        store_out(out + ((size_t)s_direct * G + g) * D + dd, ll > 0.f ? a / ll : 0.f);
+        continue;
+      }
       p.part_acc[((size_t)item * G + g) * D + dd] = a;
       if (dd == 0) {
         p.part_ml[((size_t)item * G + g) * 2 + 0] = M;
@@ -309,7 +318,8 @@ __global__ void __launch_bounds__(kAttnThreads, 4) decode_attn_mma_kernel(Device
                                                                        const __nv_bfloat16* __restrict__ q,
                                                                        const int32_t* __restrict__ lengths,
                                                                        const unsigned char* __restrict__ k_new,
-                                                                       const unsigned char* __restrict__ v_new) {
+                                                                       const unsigned char* __restrict__ v_new,
+                                                                       __nv_bfloat16* __restrict__ out) {
   constexpr int ROW_BYTES = D * 2;
   constexpr int KC = D / 16;            // k-chunks of the first product
   constexpr int KP = D / 32;            // 16-byte pieces of a K row per lane
@@ -321,6 +331,7 @@ __global__ void __launch_bounds__(kAttnThreads, 4) decode_attn_mma_kernel(Device
   __shared__ float sm_l[kAttnWarps][G];
   __shared__ __align__(16) float sm_acc[kAttnWarps][G][D];
   __shared__ int s_unit, s_rbeg;
+  __shared__ int s_direct;     // >= 0: the item is its unit's only one, the output goes to view unit s_direct
 
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
   const int g = lane >> 2, t = lane & 3;
@@ -363,6 +374,7 @@ __global__ void __launch_bounds__(kAttnThreads, 4) decode_attn_mma_kernel(Device
     const int rbeg = s_rbeg;
     if (rbeg >= len) continue;                      // an item of the reserve beyond the segment's length
     const int rend = min(len, rbeg + kDecodeChunk);
+    if (tid == 0) s_direct = len <= kDecodeChunk ? vu : -1;     // read back after the row loop (no register held)
     const int64_t seg = p.seg_off[u];
     const unsigned char* kn_row = k_new + (size_t)vu * ROW_BYTES;
     const unsigned char* vn_row = v_new + (size_t)vu * ROW_BYTES;
@@ -536,6 +548,11 @@ __global__ void __launch_bounds__(kAttnThreads, 4) decode_attn_mma_kernel(Device
         a = fmaf(w, sm_acc[x][hh][dd], a);
         ll = fmaf(w, sm_l[x][hh], ll);
       }
+      if (s_direct >= 0) {
+        // the unit's only item: Eq. 1 over the whole segment, as in the scalar kernel
+        store_out(out + ((size_t)s_direct * G + hh) * D + dd, ll > 0.f ? a / ll : 0.f);
+        continue;
+      }
       p.part_acc[((size_t)item * G + hh) * D + dd] = a;
       if (dd == 0) {
         p.part_ml[((size_t)item * G + hh) * 2 + 0] = M;
@@ -579,6 +596,7 @@ __global__ void __launch_bounds__(kCombineThreads) decode_combine_kernel(DeviceP
   const int i0 = p.dec_off[lm_index(p, unit)], i1 = i0 + (len + kDecodeChunk - 1) / kDecodeChunk;
   grid_dependency_wait();
   grid_launch_dependents();
+  if (i1 - i0 != 1) {                                   // a unit of one item has its output from the attention kernel
   const float2* ml = reinterpret_cast<const float2*>(p.part_ml);
   float M = -INFINITY;
   for (int i = i0 + tid; i < i1; i += kCombineThreads) M = fmaxf(M, ml[(size_t)i * G + g].x);
@@ -632,6 +650,7 @@ __global__ void __launch_bounds__(kCombineThreads) decode_combine_kernel(DeviceP
     }
     store_out(out + ((size_t)u * G + g) * D + tid, Lt > 0.f ? a / Lt : 0.f);
   }
+  }
   // fused step: the last of the unit's G blocks (each has read the old length by now) raises the length
   if (fused_step && tid == 0) {
     if (atomicAdd(&p.step_cnt[unit], 1) == G - 1) {
@@ -655,14 +674,14 @@ cudaError_t launch_typed(const DeviceProblem& p, const void* q, const int32_t* l
     LaunchScope ls(K_DECODE_ATTN, s);
     if (p.page_rows > 0) {
       if constexpr (sizeof(T) == 2)
-        e = launch_dependent(decode_attn_mma_kernel<D, G, true>, (unsigned)grid, kAttnThreads, s, p, static_cast<const T*>(q), lengths, kn, vn);
+        e = launch_dependent(decode_attn_mma_kernel<D, G, true>, (unsigned)grid, kAttnThreads, s, p, static_cast<const T*>(q), lengths, kn, vn, static_cast<T*>(out));
       else
-        e = launch_dependent(decode_attn_kernel<T, D, G, true>, (unsigned)grid, kAttnThreads, s, p, static_cast<const T*>(q), lengths, kn, vn);
+        e = launch_dependent(decode_attn_kernel<T, D, G, true>, (unsigned)grid, kAttnThreads, s, p, static_cast<const T*>(q), lengths, kn, vn, static_cast<T*>(out));
     } else {
       if constexpr (sizeof(T) == 2)
-        e = launch_dependent(decode_attn_mma_kernel<D, G, false>, (unsigned)grid, kAttnThreads, s, p, static_cast<const T*>(q), lengths, kn, vn);
+        e = launch_dependent(decode_attn_mma_kernel<D, G, false>, (unsigned)grid, kAttnThreads, s, p, static_cast<const T*>(q), lengths, kn, vn, static_cast<T*>(out));
       else
-        e = launch_dependent(decode_attn_kernel<T, D, G, false>, (unsigned)grid, kAttnThreads, s, p, static_cast<const T*>(q), lengths, kn, vn);
+        e = launch_dependent(decode_attn_kernel<T, D, G, false>, (unsigned)grid, kAttnThreads, s, p, static_cast<const T*>(q), lengths, kn, vn, static_cast<T*>(out));
     }
   }
   if (e != cudaSuccess) return e;
