@@ -518,13 +518,23 @@ def taskkv_compress_shard_begin(params: Params, q_win: Sequence[torch.Tensor], k
 class Pool:
     """A page pool for paged caches (taskkv_pool*) plus the torch buffer backing it."""
 
-    def __init__(self, page_rows: int, n_pages: int, head_dim: int, dtype, device, stream=None):
+    def __init__(self, page_rows: int, n_pages: int, head_dim: int, dtype, device, stream=None,
+                 library_memory: bool = False):
         dt = BF16 if dtype in (BF16, "bf16", torch.bfloat16) else F32
         nbytes = int(lib.taskkv_pool_bytes(page_rows, n_pages, head_dim, dt))
         if nbytes == 0:
             raise TaskKVError(EINVAL, "taskkv_pool_bytes")
-        self.mem = torch.empty(nbytes, dtype=torch.uint8, device=device)
         self.page_rows, self.n_pages = page_rows, n_pages
+        if library_memory:
+            # the library allocates (and frees) the pool; its pages cannot be viewed from here
+            self.mem = self.k_pages = self.v_pages = None
+            h = C.c_void_p()
+            with torch.cuda.device(torch.device(device)):
+                _check(lib.taskkv_pool_create(page_rows, n_pages, head_dim, dt, None, 0, _stream_handle(stream),
+                                              C.byref(h)), "taskkv_pool_create")
+            self._h = h
+            return
+        self.mem = torch.empty(nbytes, dtype=torch.uint8, device=device)
         # layout of the pool memory (taskkv.h): K pages, then V pages from the next multiple of 256 bytes
         tdt = torch.bfloat16 if dt == BF16 else torch.float32
         page_bytes = page_rows * head_dim * (2 if dt == BF16 else 4)

@@ -1351,3 +1351,28 @@ def test_paged_caches_share_a_pool_and_reuse_freed_pages():
     for f in flats:
         f.close()
     pool.close()
+
+
+def test_paged_cache_in_a_pool_the_library_allocates():
+    """taskkv_pool_create with no caller memory: the library allocates the pool; compression and decode steps equal
+    the contiguous cache's, the count of free pages follows, the pool is freed by taskkv_pool_destroy."""
+    tk = _tk()
+    wl = small("ownpool", n=8, n_kv=4, d=128, N=0, L=32, s1=4, s2=64, k=90, dtype="bf16", R=2, seq_lens=[1700, 900],
+               nh=1, steps=5)
+    qs, ks, vs = W.materialize(wl, DEV)
+    params = tk.params_from_workload(wl, max_new_tokens=5)
+    _, pages = tk.taskkv_plan_paged(params, 128)
+    pool = tk.Pool(128, pages + 16, 128, "bf16", DEV, library_memory=True)
+    paged = tk.taskkv_compress_paged(params, qs, ks, vs, pool)
+    flat = tk.taskkv_compress_ex(params, qs, ks, vs)
+    assert pool.free_pages() == 16 and np.array_equal(paged.lengths(), flat.lengths())
+    assert np.array_equal(paged.query(tk.Q_INDICES), flat.query(tk.Q_INDICES))
+    for s_ in range(5):
+        q, kn, vn = W.gen_decode_step(wl, s_, DEV)
+        assert torch.equal(paged.taskkv_decode_step(q, kn, vn).view(torch.uint8),
+                           flat.taskkv_decode_step(q, kn, vn).view(torch.uint8))
+    assert paged.status() == 0
+    paged.close()
+    assert pool.free_pages() == pool.n_pages
+    flat.close()
+    pool.close()
