@@ -732,6 +732,10 @@ taskkv_status cache_create_impl(const taskkv_params* p, void* cache_mem, size_t 
   cudaError_t e = cudaMemcpyAsync(c->cache_mem, c->meta.data(), c->hp.meta_bytes, cudaMemcpyHostToDevice, s);
   if (e == cudaSuccess)
     e = cudaMemsetAsync(static_cast<unsigned char*>(c->cache_mem) + c->hp.o_status, 0, c->hp.o_pacc - c->hp.o_status, s);
+  // page tables: entries of pages a unit does not hold are 0, so that no table entry ever names memory outside the pool
+  if (e == cudaSuccess && c->hp.page_rows > 0)
+    e = cudaMemsetAsync(static_cast<unsigned char*>(c->cache_mem) + c->hp.o_ptab, 0,
+                        (size_t)c->hp.info.n_units * c->hp.page_stride * 4, s);
   if (e != cudaSuccess) {
     cudaGetLastError();
     taskkv_cache_destroy(c);

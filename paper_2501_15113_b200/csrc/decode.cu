@@ -655,7 +655,9 @@ __global__ void __launch_bounds__(kCombineThreads) decode_combine_kernel(DeviceP
   if (fused_step && tid == 0) {
     if (atomicAdd(&p.step_cnt[unit], 1) == G - 1) {
       p.step_cnt[unit] = 0;
-      if (grown) p.len[unit] = len_next;
+      // (a recorded device error -- a paged cache whose pool ran dry under this very step -- freezes the lengths:
+      // no row is counted whose page may not exist)
+      if (grown) { if (p.page_rows == 0 || *p.status == 0) p.len[unit] = len_next; }
       else set_status(p.status, TASKKV_ESTATE);
     }
   }

@@ -143,6 +143,8 @@ __global__ void __launch_bounds__(128) separator_plan_kernel(DeviceProblem p, in
       int32_t* tab = p.page_tab + (size_t)(br * nl + tid) * p.page_stride;
       for (int i = 0; i < s_pages[tid]; ++i) tab[i] = p.pool_free[s_base + before + i];
     }
+    // an empty pool (ESTATE is set): the block's units hold nothing, so that gather and decode pass them by
+    if (tid < nl && s_base < 0) p.len[br * nl + tid] = 0;
   }
 }
 
