@@ -540,40 +540,38 @@ window_tc_kernel(const __grid_constant__ TcMaps maps, DeviceProblem p, const __g
 }
 
 // Folds the partial statistics of one unit: slots (item, warp) of pass 1 -> one offset per row.
-// One warp per (unit, row): lanes take every 32nd slot, then a shuffle tree; the order is fixed.
+// One block per unit, one thread per row: the thread walks the unit's slots in order (a fixed order whatever the
+// launch), its neighbours reading the neighbouring rows of the same slot (coalesced); four slots are loaded ahead of
+// the dependent max / sum updates.
 __global__ void __launch_bounds__(128) window_tc_reduce_kernel(DeviceProblem p, UnitRange ur, int chunk_keys,
                                                                int parts, int n_real) {
   const int u = ur.unit(blockIdx.x);
   const int slots = (p.unit_N[u] + chunk_keys - 1) / chunk_keys * parts;
-  const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
   const float2* part = reinterpret_cast<const float2*>(p.stat_part) + (size_t)u * p.chunks_max * p.rows_pad;
-  const int row = blockIdx.y * 4 + warp;
-  if (row < p.rows) {
-    float M = -INFINITY, z = 0.f;
-    for (int c = lane; c < slots; c += 32) {
-      const float2 o = part[(size_t)c * p.rows_pad + row];
-      if (o.x > -INFINITY) {
-        const float Mn = fmaxf(M, o.x);
-        z = z * exp2f(M - Mn) + o.y * exp2f(o.x - Mn);
-        M = Mn;
-      }
-    }
-#pragma unroll
-    for (int o = 16; o > 0; o >>= 1) {
-      const float M2 = __shfl_xor_sync(0xffffffffu, M, o);
-      const float z2 = __shfl_xor_sync(0xffffffffu, z, o);
-      const float Mn = fmaxf(M, M2);
-      if (Mn > -INFINITY) z = z * exp2f(M - Mn) + z2 * exp2f(M2 - Mn);
+  const int row = threadIdx.x;
+  if (row >= p.rows) return;
+  float M = -INFINITY, z = 0.f;
+  auto fold = [&](const float2 o) {
+    if (o.x > -INFINITY) {
+      const float Mn = fmaxf(M, o.x);
+      z = z * exp2f(M - Mn) + o.y * exp2f(o.x - Mn);
       M = Mn;
     }
-    // one offset per row: score * scale - (max + log2(sum) + log2(rows)) is log2 of the row's share of C
-    // prefix mode (n_real > 0): a query row at or beyond the end of the sequence does not exist; an infinite
-    // offset takes it out of every column sum
-    const bool absent = n_real > 0 && p.unit_N[u] - p.rows + row >= n_real;
-    if (lane == 0)
-      p.stat[(size_t)u * (2 * p.rows_pad) + row] =
-          (z > 0.f && !absent) ? M + log2f(z) + log2f((float)p.rows) : INFINITY;
+  };
+  int c = 0;
+  for (; c + 4 <= slots; c += 4) {
+    float2 o[4];
+#pragma unroll
+    for (int i = 0; i < 4; ++i) o[i] = part[(size_t)(c + i) * p.rows_pad + row];
+#pragma unroll
+    for (int i = 0; i < 4; ++i) fold(o[i]);
   }
+  for (; c < slots; ++c) fold(part[(size_t)c * p.rows_pad + row]);
+  // one offset per row: score * scale - (max + log2(sum) + log2(rows)) is log2 of the row's share of C
+  // prefix mode (n_real > 0): a query row at or beyond the end of the sequence does not exist; an infinite
+  // offset takes it out of every column sum
+  const bool absent = n_real > 0 && p.unit_N[u] - p.rows + row >= n_real;
+  p.stat[(size_t)u * (2 * p.rows_pad) + row] = (z > 0.f && !absent) ? M + log2f(z) + log2f((float)p.rows) : INFINITY;
 }
 
 // Keys per work item.  Every item costs a Q load and, in pass 2, a statistics load, so long items are
@@ -654,7 +652,7 @@ cudaError_t launch_tc_d(const DeviceProblem& p, const WindowHostInfo& h, cudaStr
       {
         LaunchScope ls(K_WINDOW_REDUCE, s);
         const UnitRange ur{b0 * per_seq_all + first, per_seq, per_seq_all, nb * per_seq};
-        window_tc_reduce_kernel<<<dim3(nb * per_seq, (p.rows + 3) / 4), 128, 0, s>>>(p, ur, a.chunk_keys, parts, 0);
+        window_tc_reduce_kernel<<<nb * per_seq, 128, 0, s>>>(p, ur, a.chunk_keys, parts, 0);
       }
     }
     a.pass = 2;
@@ -714,7 +712,7 @@ cudaError_t launch_prefix_d(const DeviceProblem& p, const void* q, const void* k
   {
     LaunchScope ls(K_WINDOW_REDUCE, s);
     const UnitRange ur{0, a.n_local, a.n_local, a.n_local};
-    window_tc_reduce_kernel<<<dim3(a.n_local, (p.rows + 3) / 4), 128, 0, s>>>(p, ur, a.chunk_keys, 2, N);
+    window_tc_reduce_kernel<<<a.n_local, 128, 0, s>>>(p, ur, a.chunk_keys, 2, N);
   }
   a.pass = 2;
   {
