@@ -493,11 +493,16 @@ window_tc_kernel(const __grid_constant__ TcMaps maps, DeviceProblem p, const __g
                 cs[3] += ex2(fmaf(__uint_as_float(r[c + 3]), scale2, -off.w));
               }
             } else {
+              // window row c0 + c sees keys up to N - L + (c0 + c) % L.  The residue is counted along (one
+              // division per 32 rows): a division per element made this tile cost fourteen ordinary ones
+              int res = c0 % L;
+              const int need = j - (N - L);         // the row's residue must reach this for key j to be visible
 #pragma unroll
               for (int c = 0; c < 32; ++c) {
                 const float off = myStat[c0 + c];
-                const bool vis = (j < N) && (j <= N - L + ((c0 + c) % L));
+                const bool vis = (j < N) && (need <= res);
                 if (vis) cs[c & 3] += ex2(fmaf(__uint_as_float(r[c]), scale2, -off));
+                res = (res + 1 == L) ? 0 : res + 1;
               }
             }
           }
