@@ -356,6 +356,14 @@ def test_cluster_select(case):
     run_workload(wl, check_pool=False)
 
 
+def test_sequence_longer_than_a_cluster_holds_streams_its_keys():
+    """N > 262144: more keys than the largest cluster keeps in registers; the selection streams them from L2 once per
+    bisection step (select_kernel), the window scores take their two-pass path with 129 work items per unit, and the
+    decode splits the full head into 517 work items."""
+    wl = small("very_long", n=2, n_kv=2, d=64, N=264500, L=16, s1=4, s2=200, k=3000, dtype="bf16", nh=0, steps=2)
+    run_workload(wl, check_pool=False)
+
+
 def test_cluster_select_equal_scores_keep_the_lower_positions():
     """All keys of a head equal: every score before the window is the same number (on the GPU and in the oracle
     alike), so both selections are decided by position alone, and the run of equal keys that is kept crosses from one
