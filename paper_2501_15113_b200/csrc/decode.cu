@@ -572,8 +572,11 @@ constexpr int kCombineStage = 1024;     // partial results weighted per round (o
 // One block per (view unit, query head of the group).  The weights exp2(m_i - M) of the unit's partial results
 // are computed once, by all threads, into shared memory; the accumulation loop then has nothing but independent
 // 16-byte loads in it (a long unit has over a hundred partials and one block: its latency is the kernel's).
-template <typename T, int D, int G>
-__global__ void __launch_bounds__(kCombineThreads) decode_combine_kernel(DeviceProblem p,
+// PRE: partial outputs a warp loads ahead of the weights (8: 64 registers, four blocks per SM (the lean one: six), for grids that are
+// resident at once anyway -- it takes two round trips to L2 off the merge; 0: the lean variant for many thousands of
+// blocks, most of them with nothing to merge).
+template <typename T, int D, int G, int PRE>
+__global__ void __launch_bounds__(kCombineThreads, PRE > 0 ? 4 : 6) decode_combine_kernel(DeviceProblem p,
                                                                          const int32_t* __restrict__ lengths,
                                                                          int fused_step, T* __restrict__ out) {
   constexpr int EPL = D / 32;
@@ -598,8 +601,20 @@ __global__ void __launch_bounds__(kCombineThreads) decode_combine_kernel(DeviceP
   grid_launch_dependents();
   if (i1 - i0 != 1) {                                   // a unit of one item has its output from the attention kernel
   const float2* ml = reinterpret_cast<const float2*>(p.part_ml);
-  float M = -INFINITY;
-  for (int i = i0 + tid; i < i1; i += kCombineThreads) M = fmaxf(M, ml[(size_t)i * G + g].x);
+  const int n = i1 - i0;
+  // Issued together, right after the wait: this thread's (max, sum) pair and this warp's first kPre partial outputs
+  // (they do not depend on the weights), so that the merge costs two round trips to L2 instead of four.
+  constexpr int kPre = PRE;
+  using Vec = typename std::conditional<EPL == 4, float4, float2>::type;
+  Vec pre[kPre > 0 ? kPre : 1];
+#pragma unroll
+  for (int q = 0; q < kPre; ++q) {
+    const int j = warp + q * kCombineWarps;
+    if (j < n) pre[q] = *reinterpret_cast<const Vec*>(p.part_acc + ((size_t)(i0 + j) * G + g) * D + lane * EPL);
+  }
+  const float2 v0 = tid < n ? ml[(size_t)(i0 + tid) * G + g] : make_float2(-INFINITY, 0.f);
+  float M = v0.x;
+  for (int i = i0 + tid + kCombineThreads; i < i1; i += kCombineThreads) M = fmaxf(M, ml[(size_t)i * G + g].x);
   M = warp_max(M);
   if (lane == 0) s_red[warp] = M;
   __syncthreads();
@@ -610,31 +625,33 @@ __global__ void __launch_bounds__(kCombineThreads) decode_combine_kernel(DeviceP
 #pragma unroll
   for (int e = 0; e < EPL; ++e) acc[e] = 0.f;
   float L = 0.f;
+  auto add = [&](float wgt, const Vec& t) {
+    if constexpr (EPL == 4) {
+      acc[0] = fmaf(wgt, t.x, acc[0]); acc[1] = fmaf(wgt, t.y, acc[1]);
+      acc[2] = fmaf(wgt, t.z, acc[2]); acc[3] = fmaf(wgt, t.w, acc[3]);
+    } else {
+      acc[0] = fmaf(wgt, t.x, acc[0]); acc[1] = fmaf(wgt, t.y, acc[1]);
+    }
+  };
   for (int c0 = i0; c0 < i1; c0 += kCombineStage) {
     const int cn = min(kCombineStage, i1 - c0);
     __syncthreads();                                    // the previous round's weights have been used
     for (int j = tid; j < cn; j += kCombineThreads) {
-      const float2 v = ml[(size_t)(c0 + j) * G + g];
+      const float2 v = (c0 == i0 && j == tid) ? v0 : ml[(size_t)(c0 + j) * G + g];
       const float wgt = (v.x == -INFINITY) ? 0.f : exp2f(v.x - M);
       s_w[j] = wgt;
       L = fmaf(wgt, v.y, L);
     }
     __syncthreads();
-#pragma unroll 8
-    for (int j = warp; j < cn; j += kCombineWarps) {
-      const float wgt = s_w[j];
-      const float* pa = p.part_acc + ((size_t)(c0 + j) * G + g) * D + lane * EPL;
-      float v[EPL];
-      if constexpr (EPL == 4) {
-        const float4 t = *reinterpret_cast<const float4*>(pa);
-        v[0] = t.x; v[1] = t.y; v[2] = t.z; v[3] = t.w;
-      } else {
-        const float2 t = *reinterpret_cast<const float2*>(pa);
-        v[0] = t.x; v[1] = t.y;
-      }
+    int j = warp;                                       // every warp adds its partials in ascending order
+    if (c0 == i0) {
 #pragma unroll
-      for (int e = 0; e < EPL; ++e) acc[e] = fmaf(wgt, v[e], acc[e]);
+      for (int q = 0; q < kPre; ++q, j += kCombineWarps)
+        if (j < cn) add(s_w[j], pre[q]);
     }
+#pragma unroll 8
+    for (; j < cn; j += kCombineWarps)
+      add(s_w[j], *reinterpret_cast<const Vec*>(p.part_acc + ((size_t)(c0 + j) * G + g) * D + lane * EPL));
   }
   L = warp_sum(L);
 #pragma unroll
@@ -689,8 +706,13 @@ cudaError_t launch_typed(const DeviceProblem& p, const void* q, const int32_t* l
   if (e != cudaSuccess) return e;
   {
     LaunchScope ls(K_DECODE_COMBINE, s);
-    e = launch_dependent(decode_combine_kernel<T, D, G>, (unsigned)(p.view_U * G), kCombineThreads, s, p, lengths,
-                         k_new != nullptr ? 1 : 0, static_cast<T*>(out));
+    // up to 16 blocks per SM: the variant that loads ahead (its blocks are resident within a few waves)
+    if ((int64_t)p.view_U * G <= 148 * 16)
+      e = launch_dependent(decode_combine_kernel<T, D, G, 8>, (unsigned)(p.view_U * G), kCombineThreads, s, p, lengths,
+                           k_new != nullptr ? 1 : 0, static_cast<T*>(out));
+    else
+      e = launch_dependent(decode_combine_kernel<T, D, G, 0>, (unsigned)(p.view_U * G), kCombineThreads, s, p, lengths,
+                           k_new != nullptr ? 1 : 0, static_cast<T*>(out));
   }
   return e;
 }
