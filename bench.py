@@ -647,11 +647,11 @@ def ncu_traffic(wl, retained_rows):
     if wl.dtype != "bf16" or wl.head_dim != 128:
         return None, None
     if wl.n_heads == wl.n_kv_heads:
-        # 378.44 MB read + 4.66 MB written for 739,056 retained rows of 256 bytes, K and V
-        return 383.10e6 / 739056 * retained_rows, "profiles/decode_attn_llama2_4layers.md (one query head per KV head)"
+        # 378.42 MB read + 4.25 MB written for 739,056 retained rows of 256 bytes, K and V
+        return 382.67e6 / 739056 * retained_rows, "profiles/decode_attn_llama2_4layers.md (one query head per KV head)"
     if wl.group == 4:
-        # 859.10 MB read + 10.08 MB written for a launch whose K and V rows are 859.03 MB
-        return 869.18e6 / (859.03e6 / 512.0) * retained_rows, "profiles/decode_attn_llama2_4layers.md (four query heads per KV head)"
+        # 859.09 MB read + 9.02 MB written for a launch whose K and V rows are 859.03 MB
+        return 868.11e6 / (859.03e6 / 512.0) * retained_rows, "profiles/decode_attn_llama2_4layers.md (four query heads per KV head)"
     return None, None
 
 
