@@ -266,7 +266,8 @@ taskkv_status taskkv_compress_shard_finish(taskkv_cache* c, const float* sem_all
  * the host (how many pages a call takes follows from the schedules, not from the data) and refuses a compression or an
  * append that would not fit with EALLOC before anything is launched.  Calls that use one pool -- compressions,
  * appends and decode steps of its caches, and their destruction -- must be ordered with respect to one another by the
- * caller (one stream, or events); the pool must outlive its caches.
+ * caller (one stream, or events).  taskkv_pool_destroy on a pool that still has caches only marks it: the last of
+ * its caches to be destroyed releases it (caller-supplied pool memory must stay valid until then).
  * A paged cache cannot be head-sharded or filled layer by layer (EINVAL).
  * Should the device find the pool empty all the same (calls on one pool that the caller did not order), the
  * row is not stored and the cache's status word gets ESTATE; such a cache is to be destroyed, which returns the pages

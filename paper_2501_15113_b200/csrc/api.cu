@@ -287,6 +287,7 @@ struct taskkv_pool {
   int32_t* top = nullptr;             // device: number of free pages
   int64_t free_host = 0;              // the host's count (exact: what a call takes follows from the schedules)
   int32_t caches = 0;                 // caches alive
+  bool orphan = false;                // taskkv_pool_destroy came while caches were alive: the last one frees the pool
 };
 
 struct taskkv_cache {
@@ -856,13 +857,23 @@ taskkv_status taskkv_pool_create(int32_t page_rows, int32_t n_pages, int32_t hea
 
 int32_t taskkv_pool_free_pages(const taskkv_pool* pool) { return pool ? (int32_t)pool->free_host : -1; }
 
-void taskkv_pool_destroy(taskkv_pool* pool) {
-  if (!pool) return;
+namespace {
+void free_pool(taskkv_pool* pool) {
   if (pool->own) {
     cudaDeviceSynchronize();
     cudaFree(pool->mem);
   }
   delete pool;
+}
+}  // namespace
+
+void taskkv_pool_destroy(taskkv_pool* pool) {
+  if (!pool) return;
+  if (pool->caches > 0) {      // caches still point at it: the last of them to be destroyed frees the pool
+    pool->orphan = true;
+    return;
+  }
+  free_pool(pool);
 }
 
 taskkv_status taskkv_plan_paged(const taskkv_params* p, int32_t page_rows, taskkv_plan_info* out, int64_t* pages_needed) {
@@ -1237,7 +1248,7 @@ void taskkv_cache_destroy(taskkv_cache* c) {
     cudaDeviceSynchronize();
     if (c->cache_mem && launch_release_pages(c->dp, nullptr) == cudaSuccess) cudaDeviceSynchronize();
     c->pool->free_host += c->pages_held;
-    --c->pool->caches;
+    if (--c->pool->caches == 0 && c->pool->orphan) free_pool(c->pool);
   }
   if (c->own_cache || c->own_work || c->stage) cudaDeviceSynchronize();
   if (c->own_cache) cudaFree(c->cache_mem);

@@ -1384,3 +1384,24 @@ def test_paged_cache_in_a_pool_the_library_allocates():
     assert pool.free_pages() == pool.n_pages
     flat.close()
     pool.close()
+
+
+def test_pool_destroyed_before_its_cache_is_released_by_the_cache():
+    """taskkv_pool_destroy while a cache still lives in the pool only marks the pool; the cache keeps working and
+    its destruction releases the pool."""
+    tk = _tk()
+    wl = small("orphan", n=4, n_kv=4, d=128, N=1200, L=32, s1=4, s2=64, k=80, dtype="bf16", R=1, nh=1, steps=3)
+    qs, ks, vs = W.materialize(wl, DEV)
+    params = tk.params_from_workload(wl, max_new_tokens=3)
+    _, pages = tk.taskkv_plan_paged(params, 64)
+    pool = tk.Pool(64, pages + 8, 128, "bf16", DEV, library_memory=True)
+    paged = tk.taskkv_compress_paged(params, qs, ks, vs, pool)
+    flat = tk.taskkv_compress_ex(params, qs, ks, vs)
+    pool.close()                                        # the pool's handle is gone; its memory is not
+    for s_ in range(3):
+        q, kn, vn = W.gen_decode_step(wl, s_, DEV)
+        assert torch.equal(paged.taskkv_decode_step(q, kn, vn).view(torch.uint8),
+                           flat.taskkv_decode_step(q, kn, vn).view(torch.uint8))
+    assert paged.status() == 0
+    paged.close()                                       # releases the pool
+    flat.close()
