@@ -430,8 +430,14 @@ class Cache:
             pool = self._keep["pool"]
             P = pool.page_rows
             n = (ln + P - 1) // P
-            tab = torch.from_numpy(self.query(Q_PAGETAB)[u, :n].astype(np.int64)).to(pool.mem.device)
-            pages = (pool.k_pages if which == "k" else pool.v_pages)[tab]          # [n, P, d]
+            tab = self.query(Q_PAGETAB)[u, :n].astype(np.int64)
+            if pool.k_pages is None:
+                # a pool the library allocated: its pages come back through the query (the whole pool: tests only)
+                raw = self.query(Q_KPOOL if which == "k" else Q_VPOOL)
+                pb = P * d * es
+                seg = np.concatenate([raw[int(t) * pb:(int(t) + 1) * pb] for t in tab]) if n else raw[:0]
+                return torch.from_numpy(seg[:ln * d * es].copy()).view(self.params.torch_dtype).reshape(ln, d)
+            pages = (pool.k_pages if which == "k" else pool.v_pages)[torch.from_numpy(tab).to(pool.mem.device)]   # [n, P, d]
             return pages.reshape(n * P, d)[:ln].cpu().contiguous()
         raw = self.query(Q_KPOOL if which == "k" else Q_VPOOL)
         off = self.query(Q_OFFSETS)

@@ -1375,6 +1375,9 @@ def test_paged_cache_in_a_pool_the_library_allocates():
     flat = tk.taskkv_compress_ex(params, qs, ks, vs)
     assert pool.free_pages() == 16 and np.array_equal(paged.lengths(), flat.lengths())
     assert np.array_equal(paged.query(tk.Q_INDICES), flat.query(tk.Q_INDICES))
+    for u in (0, 5, 15):
+        assert torch.equal(paged.pool_rows("k", u).view(torch.uint8), flat.pool_rows("k", u).view(torch.uint8))
+        assert torch.equal(paged.pool_rows("v", u).view(torch.uint8), flat.pool_rows("v", u).view(torch.uint8))
     for s_ in range(5):
         q, kn, vn = W.gen_decode_step(wl, s_, DEV)
         assert torch.equal(paged.taskkv_decode_step(q, kn, vn).view(torch.uint8),
