@@ -268,6 +268,9 @@ taskkv_status taskkv_compress_shard_finish(taskkv_cache* c, const float* sem_all
  * appends and decode steps of its caches, and their destruction -- must be ordered with respect to one another by the
  * caller (one stream, or events).  taskkv_pool_destroy on a pool that still has caches only marks it: the last of
  * its caches to be destroyed releases it (caller-supplied pool memory must stay valid until then).
+ * The count follows the calls the library sees: an append or a fused step replayed from a captured CUDA graph takes
+ * its pages on the device without the count knowing, so replay only calls that append nothing (taskkv_decode_ex) on
+ * a paged cache, or none.
  * A paged cache cannot be head-sharded or filled layer by layer (EINVAL).
  * Should the device find the pool empty all the same (calls on one pool that the caller did not order), the
  * row is not stored and the cache's status word gets ESTATE; such a cache is to be destroyed, which returns the pages
