@@ -306,7 +306,44 @@ struct taskkv_cache {
   size_t stage_bytes = 0;
   std::vector<unsigned char> layer_done;   // [R] layers compressed so far (layer-streamed caches)
   int shard_stage = 0;                     // head-sharded caches: 1 after begin (vectors ready), 2 after finish
+  // The last call that wrote lengths or page tables (compression, append, fused step): its stream and layers.  A
+  // decode on the same stream over other layers may read its unit data before its dependency wait (launch_decode).
+  bool lw_valid = false;
+  cudaStream_t lw_stream = nullptr;
+  int32_t lw_l0 = 0, lw_nl = 0;
+  unsigned long long lw_capture = 0;       // id of the stream capture that call was recorded in (0: launched directly)
 };
+
+namespace {
+// Id of the capture `s` is recording into, 0 if it is not capturing.
+unsigned long long capture_id(cudaStream_t s) {
+  cudaStreamCaptureStatus st = cudaStreamCaptureStatusNone;
+  unsigned long long id = 0;
+  if (cudaStreamGetCaptureInfo(s, &st, &id) != cudaSuccess) {
+    cudaGetLastError();
+    return ~0ull;                          // unknown: matches nothing
+  }
+  return st == cudaStreamCaptureStatusActive ? id : 0;
+}
+void note_length_writer(taskkv_cache* c, int32_t l0, int32_t nl, cudaStream_t s) {
+  c->lw_valid = true;
+  c->lw_stream = s;
+  c->lw_l0 = l0;
+  c->lw_nl = nl;
+  c->lw_capture = capture_id(s);
+}
+// Whether the kernel before the next launch on `s` cannot be one of this cache's that writes the lengths or page
+// tables of layers [l0, l0 + nl): the last such call went to the same stream (so anything launched on `s` since is
+// not one), in the same way -- both launched directly, or both recorded into the same graph, whose replays keep
+// their order; a graph's first call never qualifies, whatever ran before a replay -- and covered other layers.
+// Conservative otherwise.
+bool unit_data_settled(const taskkv_cache* c, int32_t l0, int32_t nl, cudaStream_t s) {
+  if (!c->lw_valid || c->lw_stream != s) return false;
+  const unsigned long long id = capture_id(s);
+  if (id == ~0ull || id != c->lw_capture) return false;
+  return l0 + nl <= c->lw_l0 || c->lw_l0 + c->lw_nl <= l0;
+}
+}  // namespace
 
 namespace {
 // Two ways of overlapping the steps of different layers, both over chunks of layers and with streams the library
@@ -951,6 +988,7 @@ taskkv_status taskkv_compress_shard_finish(taskkv_cache* c, const float* sem_all
   cudaStream_t s = static_cast<cudaStream_t>(stream);
   const int B = c->prm.batch, R = c->prm.n_layers;
   c->dp.sem_all = sem_all;         // only the separator reads it; the cache keeps no reference afterwards
+  c->lw_valid = false;
   cudaError_t e = launch_separator_plan(c->dp, B, 0, R, s);
   c->dp.sem_all = nullptr;
   if (e == cudaSuccess) e = launch_gather(c->dp, c->prm.dtype, B, 0, R, 0, c->hp.info.gather_items, s);
@@ -983,6 +1021,7 @@ taskkv_status taskkv_compress_layer(taskkv_cache* c, int32_t layer, const void* 
   wh.k = k;
   wh.lse = window_lse;
   wh.base_layer = layer;
+  c->lw_valid = false;      // the plan kernel writes this layer's lengths: the next decode reads nothing early
   if (e == cudaSuccess) e = compress_layers(c, wh, layer, 1, s);
   if (e != cudaSuccess) {
     std::fprintf(stderr, "taskkv_compress_layer: CUDA error: %s\n", cudaGetErrorString(e));
@@ -1114,6 +1153,7 @@ taskkv_status taskkv_append_ex(taskkv_cache* c, const void* k_new, const void* v
   if (!layer_view(c, layer_begin, layer_count, &view)) return TASKKV_EINVAL;
   const taskkv_status st = take_append_pages(c, layer_begin, layer_count);
   if (st != TASKKV_OK) return st;
+  note_length_writer(c, layer_begin, layer_count, static_cast<cudaStream_t>(stream));
   return cuda_status(launch_append(view, c->prm.dtype, k_new, v_new, static_cast<cudaStream_t>(stream)));
 }
 
@@ -1128,7 +1168,8 @@ taskkv_status taskkv_decode_ex(const void* q, taskkv_cache* c, const int32_t* le
   taskkv::DeviceProblem view;
   if (!layer_view(c, layer_begin, layer_count, &view)) return TASKKV_EINVAL;
   return cuda_status(launch_decode(view, c->prm.dtype, q, lengths, nullptr, nullptr, out,
-                                   static_cast<cudaStream_t>(stream)));
+                                   static_cast<cudaStream_t>(stream),
+                                   unit_data_settled(c, layer_begin, layer_count, static_cast<cudaStream_t>(stream))));
 }
 
 taskkv_status taskkv_decode_step_ex(const void* q, const void* k_new, const void* v_new, taskkv_cache* c, void* out,
@@ -1139,8 +1180,10 @@ taskkv_status taskkv_decode_step_ex(const void* q, const void* k_new, const void
   if (!layer_view(c, layer_begin, layer_count, &view)) return TASKKV_EINVAL;
   const taskkv_status st = take_append_pages(c, layer_begin, layer_count);
   if (st != TASKKV_OK) return st;
+  const bool early = unit_data_settled(c, layer_begin, layer_count, static_cast<cudaStream_t>(stream));
+  note_length_writer(c, layer_begin, layer_count, static_cast<cudaStream_t>(stream));
   return cuda_status(launch_decode(view, c->prm.dtype, q, nullptr, k_new, v_new, out,
-                                   static_cast<cudaStream_t>(stream)));
+                                   static_cast<cudaStream_t>(stream), early));
 }
 
 taskkv_status taskkv_decode_step(const void* q, const void* k_new, const void* v_new, taskkv_cache* c, void* out,
@@ -1184,6 +1227,7 @@ taskkv_status taskkv_decode_host(const void* q, const void* k_new, const void* v
   }
   if (e == cudaSuccess && k_new && take_append_pages(c, 0, c->dp.R) != TASKKV_OK) return TASKKV_EALLOC;
   if (e == cudaSuccess)
+    if (k_new) note_length_writer(c, 0, c->dp.R, s);
     e = launch_decode(c->dp, c->prm.dtype, dq, nullptr, k_new ? dkn : nullptr, k_new ? dvn : nullptr, dout, s);
   if (e == cudaSuccess) e = cudaMemcpyAsync(out, dout, q_bytes, cudaMemcpyDeviceToHost, s);
   if (e != cudaSuccess) return TASKKV_ECUDA;

@@ -182,7 +182,8 @@ cudaError_t launch_compensate(const DeviceProblem& p, int dtype, const UnitRange
 cudaError_t launch_append(const DeviceProblem& p, int dtype, const void* k_new, const void* v_new,
                           cudaStream_t s);
 cudaError_t launch_decode(const DeviceProblem& p, int dtype, const void* q, const int32_t* lengths,
-                          const void* k_new, const void* v_new, void* out, cudaStream_t s);
+                          const void* k_new, const void* v_new, void* out, cudaStream_t s,
+                          bool early_unit_data = false);
 
 // Programmatic dependent launch: a kernel launched with launch_dependent() may be set up, and its blocks may become
 // resident, while the kernel before it in the stream is still draining; grid_dependency_wait() at its start returns

@@ -61,7 +61,7 @@ __global__ void __launch_bounds__(kAttnThreads) decode_attn_kernel(DeviceProblem
                                                                    const int32_t* __restrict__ lengths,
                                                                    const unsigned char* __restrict__ k_new,
                                                                    const unsigned char* __restrict__ v_new,
-                                                                   T* __restrict__ out) {
+                                                                   T* __restrict__ out, int early) {
   constexpr int EPL = 16 / (int)sizeof(T);          // elements per lane (one 16-byte vector)
   constexpr int LPR = D / EPL;                      // lanes per row
   constexpr int RPW = 32 / LPR;                     // rows per warp instruction
@@ -88,8 +88,19 @@ __global__ void __launch_bounds__(kAttnThreads) decode_attn_kernel(DeviceProblem
   int wi_first = 0;
   if (warp == 0 && item0 + (int)blockIdx.x < item1)
     wi_first = w0 + upper_unit_warp(p.dec_off + w0, p.view_U, item0 + (int)blockIdx.x, lane);
-  grid_dependency_wait();
-  grid_launch_dependents();
+  // `early` (set by the host when the kernel before this one in the stream cannot be one that writes these units'
+  // lengths or page tables: see launch_decode): the first item's unit data is read before the wait as well, and the
+  // wait comes just before the block first touches what the caller's kernels produce (q, the new token's rows) or
+  // writes anything.  (A block all of whose items are beyond their segments' lengths leaves without waiting.)
+  bool waited = false;
+  auto wait_once = [&]() {
+    if (!waited) {
+      grid_dependency_wait();
+      grid_launch_dependents();
+      waited = true;
+    }
+  };
+  if (!early) wait_once();
   for (int item = item0 + blockIdx.x; item < item1; item += gridDim.x) {
     __syncthreads();                                // previous item's shared state consumed
     if (warp == 0) {
@@ -118,6 +129,7 @@ __global__ void __launch_bounds__(kAttnThreads) decode_attn_kernel(DeviceProblem
     const int64_t seg = p.seg_off[u];
     const unsigned char* kn_row = k_new + (size_t)vu * ROW_BYTES;
     const unsigned char* vn_row = v_new + (size_t)vu * ROW_BYTES;
+    wait_once();
     if (new_r >= rbeg && new_r < rend) {
       bool have_page = true;
       if (PAGED && new_r % p.page_rows == 0) {
@@ -319,7 +331,7 @@ __global__ void __launch_bounds__(kAttnThreads, 4) decode_attn_mma_kernel(Device
                                                                        const int32_t* __restrict__ lengths,
                                                                        const unsigned char* __restrict__ k_new,
                                                                        const unsigned char* __restrict__ v_new,
-                                                                       __nv_bfloat16* __restrict__ out) {
+                                                                       __nv_bfloat16* __restrict__ out, int early) {
   constexpr int ROW_BYTES = D * 2;
   constexpr int KC = D / 16;            // k-chunks of the first product
   constexpr int KP = D / 32;            // 16-byte pieces of a K row per lane
@@ -348,8 +360,19 @@ __global__ void __launch_bounds__(kAttnThreads, 4) decode_attn_mma_kernel(Device
   int wi_first = 0;
   if (warp == 0 && item0 + (int)blockIdx.x < item1)
     wi_first = w0 + upper_unit_warp(p.dec_off + w0, p.view_U, item0 + (int)blockIdx.x, lane);
-  grid_dependency_wait();
-  grid_launch_dependents();
+  // `early` (set by the host when the kernel before this one in the stream cannot be one that writes these units'
+  // lengths or page tables: see launch_decode): the first item's unit data is read before the wait as well, and the
+  // wait comes just before the block first touches what the caller's kernels produce (q, the new token's rows) or
+  // writes anything.  (A block all of whose items are beyond their segments' lengths leaves without waiting.)
+  bool waited = false;
+  auto wait_once = [&]() {
+    if (!waited) {
+      grid_dependency_wait();
+      grid_launch_dependents();
+      waited = true;
+    }
+  };
+  if (!early) wait_once();
   for (int item = item0 + blockIdx.x; item < item1; item += gridDim.x) {
     __syncthreads();
     if (warp == 0) {
@@ -378,6 +401,7 @@ __global__ void __launch_bounds__(kAttnThreads, 4) decode_attn_mma_kernel(Device
     const int64_t seg = p.seg_off[u];
     const unsigned char* kn_row = k_new + (size_t)vu * ROW_BYTES;
     const unsigned char* vn_row = v_new + (size_t)vu * ROW_BYTES;
+    wait_once();
     if (new_r >= rbeg && new_r < rend) {
       bool have_page = true;
       if (PAGED && new_r % p.page_rows == 0) {
@@ -682,7 +706,7 @@ __global__ void __launch_bounds__(kCombineThreads, PRE > 0 ? 4 : 6) decode_combi
 
 template <typename T, int D, int G>
 cudaError_t launch_typed(const DeviceProblem& p, const void* q, const int32_t* lengths, const void* k_new,
-                         const void* v_new, void* out, cudaStream_t s) {
+                         const void* v_new, void* out, cudaStream_t s, int early) {
   const unsigned char* kn = static_cast<const unsigned char*>(k_new);
   const unsigned char* vn = static_cast<const unsigned char*>(v_new);
   // persistent blocks: 16 per SM (measured best on B200 with 512-row items)
@@ -693,14 +717,14 @@ cudaError_t launch_typed(const DeviceProblem& p, const void* q, const int32_t* l
     LaunchScope ls(K_DECODE_ATTN, s);
     if (p.page_rows > 0) {
       if constexpr (sizeof(T) == 2)
-        e = launch_dependent(decode_attn_mma_kernel<D, G, true>, (unsigned)grid, kAttnThreads, s, p, static_cast<const T*>(q), lengths, kn, vn, static_cast<T*>(out));
+        e = launch_dependent(decode_attn_mma_kernel<D, G, true>, (unsigned)grid, kAttnThreads, s, p, static_cast<const T*>(q), lengths, kn, vn, static_cast<T*>(out), early);
       else
-        e = launch_dependent(decode_attn_kernel<T, D, G, true>, (unsigned)grid, kAttnThreads, s, p, static_cast<const T*>(q), lengths, kn, vn, static_cast<T*>(out));
+        e = launch_dependent(decode_attn_kernel<T, D, G, true>, (unsigned)grid, kAttnThreads, s, p, static_cast<const T*>(q), lengths, kn, vn, static_cast<T*>(out), early);
     } else {
       if constexpr (sizeof(T) == 2)
-        e = launch_dependent(decode_attn_mma_kernel<D, G, false>, (unsigned)grid, kAttnThreads, s, p, static_cast<const T*>(q), lengths, kn, vn, static_cast<T*>(out));
+        e = launch_dependent(decode_attn_mma_kernel<D, G, false>, (unsigned)grid, kAttnThreads, s, p, static_cast<const T*>(q), lengths, kn, vn, static_cast<T*>(out), early);
       else
-        e = launch_dependent(decode_attn_kernel<T, D, G, false>, (unsigned)grid, kAttnThreads, s, p, static_cast<const T*>(q), lengths, kn, vn, static_cast<T*>(out));
+        e = launch_dependent(decode_attn_kernel<T, D, G, false>, (unsigned)grid, kAttnThreads, s, p, static_cast<const T*>(q), lengths, kn, vn, static_cast<T*>(out), early);
     }
   }
   if (e != cudaSuccess) return e;
@@ -719,12 +743,12 @@ cudaError_t launch_typed(const DeviceProblem& p, const void* q, const int32_t* l
 
 template <typename T, int D>
 cudaError_t launch_group(const DeviceProblem& p, const void* q, const int32_t* lengths, const void* k_new,
-                         const void* v_new, void* out, cudaStream_t s) {
+                         const void* v_new, void* out, cudaStream_t s, int early) {
   switch (p.G) {
-    case 1: return launch_typed<T, D, 1>(p, q, lengths, k_new, v_new, out, s);
-    case 2: return launch_typed<T, D, 2>(p, q, lengths, k_new, v_new, out, s);
-    case 4: return launch_typed<T, D, 4>(p, q, lengths, k_new, v_new, out, s);
-    case 8: return launch_typed<T, D, 8>(p, q, lengths, k_new, v_new, out, s);
+    case 1: return launch_typed<T, D, 1>(p, q, lengths, k_new, v_new, out, s, early);
+    case 2: return launch_typed<T, D, 2>(p, q, lengths, k_new, v_new, out, s, early);
+    case 4: return launch_typed<T, D, 4>(p, q, lengths, k_new, v_new, out, s, early);
+    case 8: return launch_typed<T, D, 8>(p, q, lengths, k_new, v_new, out, s, early);
     default: return cudaErrorInvalidValue;
   }
 }
@@ -732,11 +756,15 @@ cudaError_t launch_group(const DeviceProblem& p, const void* q, const int32_t* l
 }  // namespace
 
 cudaError_t launch_decode(const DeviceProblem& p, int dtype, const void* q, const int32_t* lengths,
-                          const void* k_new, const void* v_new, void* out, cudaStream_t s) {
+                          const void* k_new, const void* v_new, void* out, cudaStream_t s, bool early_unit_data) {
+  // Reading lengths and page tables before the dependency wait is sound only if the kernel before this one in the
+  // stream does not write them for these units; a caller's array of lengths is never read early.
+  const int early = (early_unit_data && lengths == nullptr) ? 1 : 0;
   if (dtype == TASKKV_F32)
-    return p.d == 64 ? launch_group<float, 64>(p, q, lengths, k_new, v_new, out, s) : launch_group<float, 128>(p, q, lengths, k_new, v_new, out, s);
-  return p.d == 64 ? launch_group<__nv_bfloat16, 64>(p, q, lengths, k_new, v_new, out, s)
-                   : launch_group<__nv_bfloat16, 128>(p, q, lengths, k_new, v_new, out, s);
+    return p.d == 64 ? launch_group<float, 64>(p, q, lengths, k_new, v_new, out, s, early)
+                     : launch_group<float, 128>(p, q, lengths, k_new, v_new, out, s, early);
+  return p.d == 64 ? launch_group<__nv_bfloat16, 64>(p, q, lengths, k_new, v_new, out, s, early)
+                   : launch_group<__nv_bfloat16, 128>(p, q, lengths, k_new, v_new, out, s, early);
 }
 
 }  // namespace taskkv
