@@ -1408,3 +1408,72 @@ def test_pool_destroyed_before_its_cache_is_released_by_the_cache():
     assert paged.status() == 0
     paged.close()                                       # releases the pool
     flat.close()
+
+
+def test_unit_data_read_early_never_changes_a_result():
+    """A per-layer decode call whose predecessor in the stream cannot write its lengths reads them before its
+    dependency wait.  One cache takes a sequence of per-layer fused steps on one stream (the case that qualifies), with
+    the same layer twice in a row, a CUDA graph of two layers replayed three times and direct calls right after it; a
+    second cache takes the same steps with every call on a stream other than the one before (never qualifies) and a
+    synchronisation in between.  Outputs, lengths and rows must agree bit for bit."""
+    tk = _tk()
+    wl = small("early", n=8, n_kv=4, d=128, N=0, L=32, s1=4, s2=64, k=100, dtype="bf16", R=3, seq_lens=[1500, 900],
+               nh=1, steps=1)
+    qs, ks, vs = W.materialize(wl, DEV)
+    params = tk.params_from_workload(wl, max_new_tokens=64)
+    a = tk.taskkv_compress_ex(params, qs, ks, vs)
+    b = tk.taskkv_compress_ex(params, qs, ks, vs)
+    torch.cuda.synchronize()
+    seq = [0, 1, 2, 2, 0, 0, 1, 2, 1, 1, 0, 2]                     # layers, in call order
+    inputs = {}
+
+    def layer_inputs(i, r):
+        if (i, r) not in inputs:
+            q, kn, vn = W.gen_decode_step(wl, 100 + i, DEV)
+            inputs[(i, r)] = tuple(x[:, r:r + 1].contiguous() for x in (q, kn, vn))
+        return inputs[(i, r)]
+
+    other = [torch.cuda.Stream(), torch.cuda.Stream()]
+
+    calls = [0]
+
+    def ref_call(r, q, kn, vn):                                    # never two calls in a row on one stream
+        st = other[calls[0] % 2]
+        calls[0] += 1
+        with torch.cuda.stream(st):
+            out = b.taskkv_decode_step_ex(q, kn, vn, r, 1, stream=st)
+        torch.cuda.synchronize()
+        return out
+
+    outs_a, outs_b = [], []
+    for i, r in enumerate(seq):
+        q, kn, vn = layer_inputs(i, r)
+        outs_a.append(a.taskkv_decode_step_ex(q, kn, vn, r, 1))
+        outs_b.append(ref_call(r, q, kn, vn))
+    # a graph of two per-layer steps, replayed, then direct calls on the layers it touched
+    gi = len(seq)
+    g_in = [layer_inputs(gi, 0), layer_inputs(gi, 1)]
+    g_out = [torch.empty_like(g_in[0][0]), torch.empty_like(g_in[1][0])]
+    torch.cuda.synchronize()
+    graph = torch.cuda.CUDAGraph()
+    with torch.cuda.graph(graph):                                  # (capture launches nothing)
+        a.taskkv_decode_step_ex(*g_in[0], 0, 1, out=g_out[0])
+        a.taskkv_decode_step_ex(*g_in[1], 1, 1, out=g_out[1])
+    for rep in range(3):
+        graph.replay()
+        torch.cuda.synchronize()
+        outs_a += [x.clone() for x in g_out]
+        outs_b += [ref_call(0, *g_in[0]), ref_call(1, *g_in[1])]
+    for i, r in enumerate([1, 0, 1, 2], start=gi + 1):
+        q, kn, vn = layer_inputs(i, r)
+        outs_a.append(a.taskkv_decode_step_ex(q, kn, vn, r, 1))
+        outs_b.append(ref_call(r, q, kn, vn))
+    torch.cuda.synchronize()
+    assert a.status() == 0 and b.status() == 0
+    assert np.array_equal(a.lengths(), b.lengths())
+    for i, (x, y) in enumerate(zip(outs_a, outs_b)):
+        assert torch.equal(x.view(torch.uint8), y.view(torch.uint8)), f"call {i}"
+    for u in range(len(a.lengths())):
+        assert torch.equal(a.pool_rows("k", u).view(torch.uint8), b.pool_rows("k", u).view(torch.uint8))
+    a.close()
+    b.close()
