@@ -1477,3 +1477,49 @@ def test_unit_data_read_early_never_changes_a_result():
         assert torch.equal(a.pool_rows("k", u).view(torch.uint8), b.pool_rows("k", u).view(torch.uint8))
     a.close()
     b.close()
+
+
+def test_direct_call_after_a_graph_replay_sees_the_replayed_lengths():
+    """The rule for reading unit data early takes a graph launch to be a unit in stream order: a kernel launched
+    directly after a replay starts once the whole graph has finished, whatever its last kernel triggered.  Here the
+    host's record points at another layer (a direct step on layer 1), a graph holding a fused step on layer 0 is
+    replayed, and a direct fused step on layer 0 follows at once and reads its lengths early: 150 rounds against a
+    cache that takes the same steps with nothing read early."""
+    tk = _tk()
+    rounds = 150
+    wl = small("replay", n=8, n_kv=4, d=128, N=0, L=32, s1=4, s2=64, k=100, dtype="bf16", R=2, seq_lens=[1400, 800],
+               nh=1, steps=1)
+    qs, ks, vs = W.materialize(wl, DEV)
+    params = tk.params_from_workload(wl, max_new_tokens=2 * rounds + 4)
+    a = tk.taskkv_compress_ex(params, qs, ks, vs)
+    b = tk.taskkv_compress_ex(params, qs, ks, vs)
+    q, kn, vn = W.gen_decode_step(wl, 7, DEV)
+    l0 = tuple(x[:, 0:1].contiguous() for x in (q, kn, vn))
+    l1 = tuple(x[:, 1:2].contiguous() for x in (q, kn, vn))
+    g_out = torch.empty_like(l0[0])
+    torch.cuda.synchronize()
+    graph = torch.cuda.CUDAGraph()
+    with torch.cuda.graph(graph):
+        a.taskkv_decode_step_ex(*l0, 0, 1, out=g_out)
+    other = [torch.cuda.Stream(), torch.cuda.Stream()]
+    n_ref = [0]
+
+    def ref(r, x):
+        st = other[n_ref[0] % 2]
+        n_ref[0] += 1
+        out = b.taskkv_decode_step_ex(*x, r, 1, stream=st)
+        torch.cuda.synchronize()
+        return out
+
+    for i in range(rounds):
+        a.taskkv_decode_step_ex(*l1, 1, 1)              # the host's record now names layer 1
+        graph.replay()                                  # raises the lengths of layer 0 ...
+        got = a.taskkv_decode_step_ex(*l0, 0, 1)        # ... which this call reads before its dependency wait
+        torch.cuda.synchronize()
+        ref(1, l1)
+        ref(0, l0)
+        want = ref(0, l0)
+        assert torch.equal(got.view(torch.uint8), want.view(torch.uint8)), f"round {i}"
+    assert np.array_equal(a.lengths(), b.lengths()) and a.status() == 0 and b.status() == 0
+    a.close()
+    b.close()
